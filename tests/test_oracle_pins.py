@@ -1,0 +1,375 @@
+"""Pins for the CPU oracle: each test ties it to something other than itself (hand-computed
+values, exact integer arithmetic, closed forms, invariants, a library routine, the restated
+Algorithm 2), chosen so that a dropped term, a wrong index or a transposed operand fails one."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import nm_inputs as gen
+import oracle
+from oracle import BF16, COL_MAJOR, F32, F64, ROW_MAJOR, alg2
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_golden(name):
+    out = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, *v = line.split()
+            out[k] = [float(x) for x in v]
+    return out
+
+
+def _bits(x):
+    """float array of bf16-representable values -> bf16 bit patterns (checked exact)."""
+    x = np.asarray(x, dtype=np.float32)
+    b = (x.view(np.uint32) >> 16).astype(np.uint16)
+    assert np.all((x.view(np.uint32) & 0xFFFF) == 0), "value not representable in bf16"
+    return b
+
+
+# ---- P1: hand-computed case, both layouts ------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_hand_computed_case_both_layouts(dtype):
+    g = _read_golden("matmul_1x3_3x2.txt")
+    M, N, K = int(g["M"][0]), int(g["N"][0]), int(g["K"][0])
+    conv = (lambda v: np.asarray(v, np.float32)) if dtype == F32 else _bits
+    A = conv(g["A"])
+    for key, layout in (("B_row_major", ROW_MAJOR), ("B_col_major", COL_MAJOR)):
+        Cq, C64, bound = oracle.matmul(A, conv(g[key]), M, N, K, dtype, F32, layout)
+        assert C64.ravel().tolist() == g["C"]
+        assert Cq.ravel().tolist() == g["C"]
+        assert bound.ravel().tolist() == g["C"]          # all terms positive: bound equals the sum
+
+
+# ---- P2: brute force against exact integer arithmetic on every tiny shape --------------------------
+
+def test_brute_force_tiny_shapes_int64():
+    rng = np.random.default_rng(7)
+    vals = np.array([-1, 0, 1, 2])
+    for M, N, K in itertools.product(range(1, 5), repeat=3):
+        Ai = rng.choice(vals, size=(M, K))
+        Bi = rng.choice(vals, size=(K, N))
+        Ci = np.zeros((M, N), dtype=np.int64)
+        Si = np.zeros((M, N), dtype=np.int64)
+        for m in range(M):
+            for n in range(N):
+                for k in range(K):
+                    Ci[m, n] += int(Ai[m, k]) * int(Bi[k, n])
+                    Si[m, n] += abs(int(Ai[m, k]) * int(Bi[k, n]))
+        for layout in (ROW_MAJOR, COL_MAJOR):
+            Bst = Bi if layout == ROW_MAJOR else Bi.T
+            for dt, conv in ((F32, lambda v: np.ascontiguousarray(v, np.float32)),
+                             (BF16, lambda v: _bits(np.ascontiguousarray(v, np.float32)))):
+                Cq, C64, bound = oracle.matmul(conv(Ai), conv(Bst), M, N, K, dt, F32, layout)
+                assert np.array_equal(C64, Ci.astype(np.float64)), (M, N, K, layout, dt)
+                assert np.array_equal(Cq, Ci.astype(np.float32))
+                assert np.array_equal(bound, Si.astype(np.float64))
+
+
+# ---- P3: small integers at the real K: fp64, int64 agree exactly ---------------------------------
+
+@pytest.mark.parametrize("layout", [ROW_MAJOR, COL_MAJOR])
+def test_small_integer_exactness_full_k(layout):
+    M, K, N = 3, 7168, 40
+    A = gen.small_int_bf16((M, K), -8, 8, seed=11)
+    B = gen.small_int_bf16((K, N), -8, 8, seed=12)
+    Ai = gen.bits_to_f32(A).astype(np.int64)
+    Bi = gen.bits_to_f32(B).astype(np.int64)
+    Ci = Ai @ Bi                                           # exact integer product
+    assert np.abs(Ci).max() < 2 ** 24
+    Bst = B if layout == ROW_MAJOR else gen.to_col_major(B)
+    Cq, C64, _ = oracle.matmul(A, Bst, M, N, K, BF16, F32, layout)
+    assert np.array_equal(C64, Ci.astype(np.float64))
+    assert np.array_equal(Cq, Ci.astype(np.float32))
+
+
+# ---- P4: rounding ties of the final cast to bf16 -------------------------------------------------
+
+def test_rounding_ties_to_even():
+    with open(os.path.join(GOLDEN, "rounding_ties.txt")) as f:
+        rows = [tuple(float(x) for x in l.split()) for l in f if l.strip() and not l.startswith("#")]
+    for total, expect in rows:
+        # a column of ones and one remainder, summing to exactly `total`
+        K = 64
+        A = _bits(np.ones((1, K), np.float32))
+        col = np.full(K, np.sign(total) * 4.0, np.float32)
+        col[0] = total - np.sign(total) * 4.0 * (K - 1)
+        Cq, C64, _ = oracle.matmul(A, _bits(col.reshape(K, 1)), 1, 1, K, BF16, BF16)
+        assert C64[0, 0] == total
+        assert gen.bits_to_f32(Cq)[0, 0] == expect, (total, expect)
+    # direct conversions, including a value that double rounding through fp32 would get wrong:
+    # 1 + 2^-8 + 2^-40 lies just above the tie between 1 and 1+2^-7, so the bf16 result is 1+2^-7;
+    # rounding to fp32 first gives exactly the tie, which ties-to-even would send down to 1.
+    x = 1.0 + 2.0 ** -8 + 2.0 ** -40
+    assert gen.bits_to_f32(oracle.f64_to_bf16(np.array([x])))[0] == np.float32(1.0 + 2.0 ** -7)
+    assert gen.bits_to_f32(oracle.f64_to_bf16(np.array([1.0 + 2.0 ** -8])))[0] == np.float32(1.0)
+    assert gen.bits_to_f32(oracle.f64_to_bf16(np.array([1.0 + 3 * 2.0 ** -8])))[0] == np.float32(1.0 + 2.0 ** -6)
+
+
+def test_bf16_widening_is_the_upper_half_of_fp32():
+    rng = np.random.default_rng(3)
+    bits = rng.integers(0, 0x7F80, size=4096, dtype=np.uint16)       # finite positive patterns
+    bits[::2] |= 0x8000
+    assert np.array_equal(oracle.bf16_to_f64(bits), gen.bits_to_f32(bits).astype(np.float64))
+    assert np.array_equal(oracle.f64_to_bf16(oracle.bf16_to_f64(bits)), bits)  # grid points are fixed
+
+
+# ---- P5: identity / one-hot -------------------------------------------------------------------
+
+@pytest.mark.parametrize("layout", [ROW_MAJOR, COL_MAJOR])
+def test_identity_and_one_hot(layout):
+    M, K, N = 4, 37, 23
+    A = gen.normal_bf16((M, K), 1.0, seed=21)
+    B = gen.normal_bf16((K, N), 0.02, seed=22)
+    st = (lambda X: X) if layout == ROW_MAJOR else gen.to_col_major
+    eye = _bits(np.eye(K, dtype=np.float32))
+    Cq, _, _ = oracle.matmul(A, st(eye), M, K, K, BF16, BF16, layout)
+    assert np.array_equal(Cq, A)                                       # B = I  ->  C = A
+    for k in (0, 5, K - 1):
+        e = np.zeros((1, K), np.float32); e[0, k] = 1.0
+        Cq, _, _ = oracle.matmul(_bits(e), st(B), 1, N, K, BF16, BF16, layout)
+        assert np.array_equal(Cq[0], B[k])                             # A = e_k -> row k of B
+    Bsel = np.zeros((K, N), np.float32)
+    ks = [(3 * n + 1) % K for n in range(N)]
+    for n, k in enumerate(ks):
+        Bsel[k, n] = 1.0
+    Cq, _, _ = oracle.matmul(A, st(_bits(Bsel)), M, N, K, BF16, BF16, layout)
+    assert np.array_equal(Cq, A[:, ks])                                # column n = e_k -> A[:, k]
+
+
+# ---- P6: closed forms ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("layout", [ROW_MAJOR, COL_MAJOR])
+def test_closed_forms(layout):
+    K, N = 301, 19
+    A = np.ones((1, K), np.float32)
+    Bn = np.tile(np.arange(1, N + 1, dtype=np.float32), (K, 1))       # B[k,n] = n+1
+    Bk = np.tile(np.arange(K, dtype=np.float32).reshape(K, 1), (1, N))  # B[k,n] = k
+    st = (lambda X: X) if layout == ROW_MAJOR else (lambda X: np.ascontiguousarray(X.T))
+    _, C64, _ = oracle.matmul(A, st(Bn), 1, N, K, F32, F32, layout)
+    assert np.array_equal(C64[0], K * np.arange(1, N + 1, dtype=np.float64))
+    _, C64, _ = oracle.matmul(A, st(Bk), 1, N, K, F32, F32, layout)
+    assert np.array_equal(C64[0], np.full(N, K * (K - 1) / 2))
+
+
+# ---- P7: Algorithm 2 restated: constants, coverage, agreement with the definition ----------------
+
+def test_alg2_constants_match_hand_derivation():
+    g = _read_golden("alg2_constants.txt")
+    c = alg2.executor_pool(int(g["K"][0]), int(g["N"][0]), int(g["P"][0]))
+    for k in ("kParts", "fractalNum", "S", "V", "nPartW", "groupSize"):
+        assert c[k] == int(g[k][0]), k
+
+
+def test_alg2_covers_every_block_once_and_equals_definition():
+    K, N = 7168, 576
+    T = gen.normal_bf16((1, K), 1.0, seed=1000)
+    W = gen.normal_bf16((K, N), 0.02, seed=1001)
+    Cb, tmpBuf, produced = alg2.matmul2(T, W, K, N)
+    assert sorted(produced) == list(range(252))                        # bijection onto 0..S-1
+    assert not np.isnan(tmpBuf).any()                                  # every partial written
+    Cq, C64, bound = oracle.matmul(T, W, 1, N, K, BF16, BF16)
+    err = np.abs(gen.bits_to_f32(Cb).astype(np.float64) - C64[0])
+    assert np.all(err <= 1e-5 * bound[0] + 1e-6 + oracle.ulp_bf16(C64[0]))
+    # small integers: every summation order is exact, so the two must agree bit for bit
+    Ti = gen.small_int_bf16((1, K), -8, 8, seed=31)
+    Wi = gen.small_int_bf16((K, N), -8, 8, seed=32)
+    Cb, _, _ = alg2.matmul2(Ti, Wi, K, N)
+    Cq, _, _ = oracle.matmul(Ti, Wi, 1, N, K, BF16, BF16)
+    assert np.array_equal(Cb, Cq[0])
+
+
+# ---- P8: linearity and the concatenation property of the fused product ------------------------------
+
+def test_linearity_and_concatenation():
+    M, K, N1, N2 = 2, 257, 33, 9
+    rng = np.random.default_rng(5)
+    A1, A2 = rng.standard_normal((M, K)), rng.standard_normal((M, K))
+    B1, B2 = rng.standard_normal((K, N1)), rng.standard_normal((K, N2))
+    f = lambda A, B: oracle.matmul(A, B, M, B.shape[1], K, F64, F64)
+    _, C1, b1 = f(A1, B1)
+    _, C2, _ = f(A2, B1)
+    _, C12, _ = f(2 * A1 + A2, B1)
+    assert np.all(np.abs(C12 - (2 * C1 + C2)) <= 1e-12 * (1 + 3 * b1))
+    # (B1 | B2): one product over the concatenation equals the two separate ones (Eq. 3)
+    _, Ccat, _ = f(A1, np.concatenate([B1, B2], axis=1))
+    _, C1b, _ = f(A1, B2)
+    assert np.array_equal(Ccat[:, :N1], C1) and np.array_equal(Ccat[:, N1:], C1b)
+
+
+# ---- P9: library cross-check ----------------------------------------------------------------------
+
+@pytest.mark.parametrize("layout", [ROW_MAJOR, COL_MAJOR])
+def test_numpy_float64_cross_check(layout):
+    M, K, N = 5, 1031, 67
+    A = gen.normal_bf16((M, K), 1.0, seed=41)
+    B = gen.normal_bf16((K, N), 0.02, seed=42)
+    ref = gen.bits_to_f32(A).astype(np.float64) @ gen.bits_to_f32(B).astype(np.float64)
+    refb = np.abs(gen.bits_to_f32(A).astype(np.float64)) @ np.abs(gen.bits_to_f32(B).astype(np.float64))
+    Bst = B if layout == ROW_MAJOR else gen.to_col_major(B)
+    _, C64, bound = oracle.matmul(A, Bst, M, N, K, BF16, F32, layout, threads=2)
+    assert np.all(np.abs(C64 - ref) <= 1e-12 * refb)
+    assert np.allclose(bound, refb, rtol=1e-12)
+    # sampled-column evaluation is the same function
+    cols = [0, 13, N - 1]
+    _, Cs, bs = oracle.matmul_columns(A, Bst, M, N, K, cols, BF16, F32, layout)
+    assert np.array_equal(Cs, C64[:, cols]) and np.array_equal(bs, bound[:, cols])
+
+
+def test_batched_strided_addressing():
+    T, H, K, N = 3, 4, 16, 24
+    q = gen.normal_bf16((T, H, K + 8), 1.0, seed=51)         # q_nope read in place from [T,H,K+8]
+    W = gen.normal_bf16((H, K, N), 0.02, seed=52)
+    Cq, C64, _ = oracle.matmul_batched(q, W, T, N, K, H, H * (K + 8), K + 8, K * N, H * N, N,
+                                       T * H * N, BF16, BF16)
+    qf, Wf = gen.bits_to_f32(q).astype(np.float64), gen.bits_to_f32(W).astype(np.float64)
+    ref = np.einsum("thk,hkn->thn", qf[:, :, :K], Wf)
+    assert np.allclose(C64.reshape(T, H, N), ref, rtol=0, atol=1e-12)
+
+
+# ---- P10: invariants of the vector-side stages and of attention -----------------------------------
+
+def test_rmsnorm_invariants():
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal(512)
+    y = oracle.rmsnorm(x, np.ones(512), 0.0)
+    assert abs(np.sqrt(np.mean(y * y)) - 1.0) < 1e-12                   # unit RMS for gamma = 1
+    assert np.allclose(oracle.rmsnorm(7.5 * x, np.ones(512), 0.0), y, atol=1e-12)  # scale invariance
+    g = rng.standard_normal(512)
+    assert np.allclose(oracle.rmsnorm(x, g, 0.0), y * g, atol=1e-12)
+    # eps enters under the root, added to the mean square
+    assert np.allclose(oracle.rmsnorm(x, np.ones(512), 0.25), x / np.sqrt(np.mean(x * x) + 0.25), atol=1e-12)
+
+
+def test_rope_invariants():
+    rng = np.random.default_rng(10)
+    q, k = rng.standard_normal(64), rng.standard_normal(64)
+    assert np.array_equal(oracle.rope(q, 0), q)                         # pos 0 is the identity
+    y = oracle.rope(q, 1234)
+    assert np.allclose(y[0::2] ** 2 + y[1::2] ** 2, q[0::2] ** 2 + q[1::2] ** 2, atol=1e-12)
+    d1 = oracle.rope(q, 17) @ oracle.rope(k, 5)
+    d2 = oracle.rope(q, 1017) @ oracle.rope(k, 1005)
+    assert abs(d1 - d2) < 1e-9                                          # depends on m - n only
+    # first pair turns by pos radians (frequency base^0 = 1), last pair by pos * base^(-62/64)
+    e = np.zeros(64); e[0] = 1.0
+    y = oracle.rope(e, 2)
+    assert np.allclose(y[:2], [np.cos(2.0), np.sin(2.0)], atol=1e-15)
+    e = np.zeros(64); e[62] = 1.0
+    ang = 3 * 10000.0 ** (-62 / 64)
+    assert np.allclose(oracle.rope(e, 3)[62:], [np.cos(ang), np.sin(ang)], atol=1e-15)
+
+
+def test_attention_invariants():
+    rng = np.random.default_rng(12)
+    H, S, dqk, dv = 3, 11, 12, 8
+    Q = rng.standard_normal((H, dqk))
+    cache = rng.standard_normal((S, dqk))
+    O, P = oracle.mla_attention(Q, cache, dv, 0.3, want_p=True)
+    assert np.allclose(P.sum(axis=1), 1.0, atol=1e-14)                  # rows sum to one
+    # against the textbook formula in numpy
+    s = 0.3 * Q @ cache.T
+    p = np.exp(s - s.max(axis=1, keepdims=True)); p /= p.sum(axis=1, keepdims=True)
+    assert np.allclose(P, p, atol=1e-14) and np.allclose(O, p @ cache[:, :dv], atol=1e-13)
+    # one row -> that row; equal rows -> that row; q = 0 -> column mean
+    assert np.allclose(oracle.mla_attention(Q, cache[:1], dv, 0.3), np.tile(cache[0, :dv], (H, 1)))
+    same = np.tile(cache[2], (S, 1))
+    assert np.allclose(oracle.mla_attention(Q, same, dv, 0.3), np.tile(cache[2, :dv], (H, 1)), atol=1e-14)
+    assert np.allclose(oracle.mla_attention(np.zeros((H, dqk)), cache, dv, 0.3),
+                       np.tile(cache[:, :dv].mean(axis=0), (H, 1)), atol=1e-14)
+    # P12: permuting the cache rows leaves the output unchanged
+    perm = rng.permutation(S)
+    assert np.allclose(oracle.mla_attention(Q, cache[perm], dv, 0.3), O, atol=1e-13)
+    # shift invariance of softmax: large scores do not overflow
+    assert np.all(np.isfinite(oracle.mla_attention(100 * Q, 100 * cache, dv, 1.0)))
+
+
+# ---- P11: the absorbed form equals textbook MLA on a tiny instance ----------------------------------
+
+def test_absorbed_equals_textbook_mla():
+    rng = np.random.default_rng(13)
+    H, S, dc, dn, dr, dv = 2, 5, 8, 4, 4, 4
+    c = rng.standard_normal((S, dc))              # latent rows
+    kr = rng.standard_normal((S, dr))             # shared rope keys
+    q_nope = rng.standard_normal((H, dn))
+    q_rope = rng.standard_normal((H, dr))
+    W_UK = rng.standard_normal((H, dn, dc))       # q_lat[h] = q_nope[h] * W_UK[h]
+    W_UV = rng.standard_normal((H, dc, dv))       # o[h] = o_lat[h] * W_UV[h]
+    scale = 1.0 / np.sqrt(dn + dr)
+    # textbook: materialise per-head keys and values
+    o_ref = np.zeros((H, dv))
+    for h in range(H):
+        k_nope = c @ W_UK[h].T                    # k_nope[j] = W_UK[h] * c_j
+        v = c @ W_UV[h]
+        s = scale * (k_nope @ q_nope[h] + kr @ q_rope[h])
+        p = np.exp(s - s.max()); p /= p.sum()
+        o_ref[h] = p @ v
+    # absorbed, through the oracle's own functions
+    _, q_lat, _ = oracle.matmul_batched(q_nope, W_UK, 1, dc, dn, H, H * dn, dn, dn * dc, H * dc, dc,
+                                        H * dc, F64, F64)
+    Q = np.concatenate([q_lat.reshape(H, dc), q_rope], axis=1)
+    cache = np.concatenate([c, kr], axis=1)
+    o_lat = oracle.mla_attention(Q, cache, dc, scale)
+    _, o, _ = oracle.matmul_batched(o_lat, W_UV, 1, dv, dc, H, H * dc, dc, dc * dv, H * dv, dv,
+                                    H * dv, F64, F64)
+    assert np.allclose(o.reshape(H, dv), o_ref, rtol=0, atol=1e-12)
+
+
+# ---- the composed step: stages are wired as the definition says -----------------------------------
+
+SMALL_DIMS = dict(d=96, q_lora=48, kv_lora=32, rope=8, nope=16, v=16, H=4)
+
+
+def test_decode_step_matches_stagewise_recomputation():
+    dims, S = SMALL_DIMS, 9
+    w = gen.mla_weights(dims, seed=61)
+    h = gen.mla_token(dims, seed=62)
+    cache = gen.mla_cache(S, dims, seed=63)
+    cache0 = cache.copy()
+    r = oracle.mla_decode_step(dims, w, h, cache, S)
+    d, ql, dc, dr, dn, dv, H = (dims[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
+    f = lambda b: gen.bits_to_f32(b).astype(np.float64)
+    rb = lambda x: f(oracle.f64_to_bf16(x))
+    c_q = rb(f(h) @ f(w["W_DQ"]))
+    assert np.array_equal(c_q, f(r["c_q"]))
+    c_qn = rb(c_q / np.sqrt(np.mean(c_q ** 2) + 1e-6) * f(w["gamma_q"]))
+    assert np.array_equal(c_qn, f(r["c_qn"]))
+    q = rb(c_qn @ f(w["W_UQR"])).reshape(H, dn + dr)
+    assert np.allclose(q, f(r["q"]), atol=1e-2)
+    q = f(r["q"])                                             # continue from the oracle's rounded values
+    ckr = rb(f(h) @ f(w["W_DKVKR"]))
+    assert np.array_equal(ckr, f(r["ckr"]))
+    # row S-1 was written, rows before it untouched
+    assert np.array_equal(cache[:S - 1], cache0[:S - 1])
+    row = f(cache[S - 1])
+    assert np.allclose(row[:dc], rb(ckr[:dc] / np.sqrt(np.mean(ckr[:dc] ** 2) + 1e-6) * f(w["gamma_kv"])), atol=1e-2)
+    assert np.allclose(row[dc:], oracle.rope(ckr[dc:], S - 1), atol=2e-2)
+    q_rope = np.stack([oracle.rope(q[hh, dn:], S - 1) for hh in range(H)])
+    assert np.allclose(f(r["q_rope"]), q_rope, atol=2e-2)
+    q_lat = np.einsum("hk,hkn->hn", q[:, :dn], f(w["W_UK"]))
+    assert np.allclose(f(r["q_lat"]), q_lat, atol=1e-2)
+    Q = np.concatenate([f(r["q_lat"]), f(r["q_rope"])], axis=1)
+    o_lat = oracle.mla_attention(Q, f(cache[:S]), dc, 1 / np.sqrt(dn + dr))
+    assert np.allclose(r["o_lat_f64"], o_lat, atol=1e-14)
+    o = np.einsum("hk,hkn->hn", f(r["o_lat"]), f(w["W_UV"]))
+    assert np.allclose(f(r["o"]), o, atol=1e-2)
+    out = f(r["o"]).reshape(-1) @ f(w["W_O"])
+    assert np.allclose(f(r["out"]), out, atol=1e-2, rtol=1e-2)
+
+
+def test_decode_step_seq_len_one_attends_only_the_new_row():
+    dims = SMALL_DIMS
+    w = gen.mla_weights(dims, seed=71, with_wo=False)
+    h = gen.mla_token(dims, seed=72)
+    cache = gen.mla_cache(1, dims, seed=73)
+    r = oracle.mla_decode_step(dims, w, h, cache, 1)
+    f = lambda b: gen.bits_to_f32(b).astype(np.float64)
+    assert np.array_equal(f(r["o_lat"]), np.tile(f(cache[0, :dims["kv_lora"]]), (dims["H"], 1)))
+    assert "out" not in r

@@ -1,0 +1,144 @@
+/*
+ * nm - narrow matrix multiplication and single-token MLA decode for NVIDIA B200 (sm_100a).
+ *
+ * C-ABI boundary.  Every pointer is a DEVICE pointer unless a parameter is documented as
+ * "host".  The caller owns every buffer and every stream; calls enqueue work on the given
+ * stream and return without synchronising.  The library never allocates device memory: kernels
+ * that need scratch (split-K partial sums, split-KV partial outputs) take it from a workspace
+ * the caller provides.  On any error nothing is enqueued and a negative code is returned.
+ *
+ * Conventions
+ *   A  row-major M x K, element (m,k) at m*K + k           (the token rows, 1 <= M <= 16)
+ *   B  K x N weights; NM_ROW_MAJOR: element (k,n) at k*N + n
+ *                     NM_COL_MAJOR: element (k,n) at n*K + k  (an [out,in] weight such as
+ *                     W^{DKV} in R^{d_c x d}, MLA Operator Optimization section)
+ *   C  row-major M x N, element (m,n) at m*N + n
+ *   The other narrow case of the Narrow Dimension condition, N = 1, is served by transposition:
+ *   C^T[1 x M] = B^T[1 x K] * A^T[K x M], i.e. pass the row-major A as a column-major B.
+ *   Arithmetic: inputs are widened exactly to fp32, products accumulate in fp32, partial sums
+ *   stay fp32, and the result is rounded once (round-to-nearest-even) to the output type
+ *   (Data Type Issue section; Algorithm 2, gather stage and output cast).
+ */
+#ifndef NM_H
+#define NM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void *nm_stream;          /* a cudaStream_t */
+
+typedef enum {
+    NM_F32 = 0,                   /* fp32 in, fp32 out */
+    NM_BF16 = 1,                  /* bf16 in, fp32 accumulate, bf16 out */
+    NM_BF16_F32OUT = 2            /* bf16 in, fp32 accumulate, fp32 out (unrounded sums) */
+} nm_dtype;
+
+typedef enum { NM_ROW_MAJOR = 0, NM_COL_MAJOR = 1 } nm_layout;
+
+enum {
+    NM_OK = 0,
+    NM_ERR_INVALID_ARG = -1,      /* null pointer, M outside 1..16, N or K < 1, bad stride */
+    NM_ERR_UNSUPPORTED = -2,      /* dtype / layout / dimension combination not built */
+    NM_ERR_ALIGNMENT = -3,        /* a pointer is not aligned to its element size */
+    NM_ERR_WORKSPACE = -4,        /* workspace missing or too small */
+    NM_ERR_CUDA = -5,             /* a CUDA call failed; see nm_last_cuda_error() */
+    NM_ERR_TIMEOUT = -6           /* a bounded device-side wait expired (nm_check_status) */
+};
+
+#define NM_MAX_M 16
+
+/* ---- misc ------------------------------------------------------------------------------- */
+
+int nm_version(void);
+const char *nm_status_string(int status);
+/* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
+const char *nm_last_cuda_error(void);
+
+/* ---- workspace --------------------------------------------------------------------------- */
+
+/*
+ * Bytes of scratch nm_matmul / nm_matmul_batched may need for this problem: split-K partial
+ * sums (fp32) plus arrival counters (Algorithm 1, "Partial Sum Buffer" tmpBuf and gather
+ * stage).  H = 1 for the unbatched call.  The size does not depend on tuning overrides.
+ */
+size_t nm_matmul_workspace_bytes(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B);
+
+/*
+ * Clear the arrival counters at the start of a workspace (enqueues one memset on `stream`).
+ * Must be done once before first use; the kernels leave the counters at zero afterwards, so
+ * no clearing is needed between calls.  `bytes` must be at least NM_WS_COUNTER_BYTES.
+ */
+#define NM_WS_COUNTER_BYTES 65536
+int nm_workspace_init(void *workspace, size_t bytes, nm_stream stream);
+
+/*
+ * Register a process-wide default workspace for nm_matmul and nm_matmul_batched (the calls
+ * that follow the paper's problem statement and therefore carry no workspace argument).  The
+ * memory stays owned by the caller and must outlive its use.  The call clears the counters with
+ * a synchronous memset.  Two calls that use the default workspace must not overlap on the GPU
+ * (use the _ws variants with distinct workspaces on concurrent streams).
+ */
+int nm_set_workspace(void *workspace, size_t bytes);
+
+/* ---- narrow matrix product ------------------------------------------------------------------ */
+
+/*
+ * C[M x N] = A[M x K] * B[K x N], 1 <= M <= 16  (Narrow Dimension condition; Eq. 4 for
+ * M = 1, K = 7168, N = 576; Algorithm 1 for the split-K / gather structure).
+ * Any N, K >= 1 is accepted; the vectorised path needs 16-byte aligned A, B and N (row-major)
+ * or K (column-major) a multiple of 16 bytes' worth of elements, otherwise a scalar kernel runs.
+ * Uses the default workspace when the chosen tiling splits K; returns NM_ERR_WORKSPACE if none
+ * is registered or it is too small.
+ */
+int nm_matmul(const void *A, const void *B, void *C, int M, int N, int K,
+              nm_dtype dtype, nm_layout layout_B, nm_stream stream);
+
+/* Same product with an explicit workspace (counters cleared once by nm_workspace_init). */
+int nm_matmul_ws(const void *A, const void *B, void *C, int M, int N, int K,
+                 nm_dtype dtype, nm_layout layout_B, void *workspace, size_t workspace_bytes,
+                 nm_stream stream);
+
+/*
+ * H independent narrow products (per-head absorbed-MLA projections):
+ *   C(m,h,:) = A(m,h,:) * B_h,   A(m,h,k) at m*lda + h*strideA + k,
+ *   B_h dense K x N in layout_B at B + h*strideB,   C(m,h,n) at m*ldc + h*strideC + n
+ * (all strides in elements).  q_nope can thus be read in place from q[T][H][nope+rope]
+ * with lda = H*(nope+rope), strideA = nope+rope.
+ */
+int nm_matmul_batched(const void *A, const void *B, void *C, int M, int N, int K, int H,
+                      long lda, long strideA, long strideB, long ldc, long strideC,
+                      nm_dtype dtype, nm_layout layout_B, nm_stream stream);
+
+int nm_matmul_batched_ws(const void *A, const void *B, void *C, int M, int N, int K, int H,
+                         long lda, long strideA, long strideB, long ldc, long strideC,
+                         nm_dtype dtype, nm_layout layout_B, void *workspace,
+                         size_t workspace_bytes, nm_stream stream);
+
+/*
+ * End-to-end form with HOST operands: A_host (M x K) and C_host (M x N) are host buffers
+ * (pinned for asynchronous copies), B stays on the device (the resident weight).  A is copied
+ * through `A_staging` and C through `C_staging` (device buffers of M*K and M*N elements).
+ * Enqueues copy-in, the product (explicit workspace) and copy-out on `stream`.
+ */
+int nm_matmul_host(const void *A_host, const void *B, void *C_host, void *A_staging,
+                   void *C_staging, int M, int N, int K, nm_dtype dtype, nm_layout layout_B,
+                   void *workspace, size_t workspace_bytes, nm_stream stream);
+
+/* ---- tuning aids (sweeps and tests; not needed for normal use) --------------------------------- */
+
+/* Override the tiling heuristic: columns per CTA tile of the row-major kernel and number of
+ * k-splits; 0 restores the heuristic.  Values are clamped to what the workspace bound covers. */
+int nm_debug_set_plan(int tile_n, int nsplit);
+/* Report the plan for a problem: out[0..5] = kernel kind (0 row-major vector, 1 column-major
+ * vector, 2 scalar), columns per tile, k-splits, k-rows per split, column tiles, CTAs. */
+int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B, int vec_ok,
+                      int *out /* host, 6 ints */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NM_H */

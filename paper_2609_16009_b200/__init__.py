@@ -1,0 +1,157 @@
+"""Thin Python binding over the C-ABI library ``libnm.so`` (argument marshalling only).
+
+Every function has the name of the C entry point it calls.  Tensors are ``torch`` CUDA tensors
+used purely as device memory: bf16 data may be passed as ``torch.bfloat16`` or as its raw
+``int16``/``uint16`` bits.  There is no CPU path: importing this package without the built
+library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libnm.so")
+
+F32, BF16, BF16_F32OUT = 0, 1, 2
+ROW_MAJOR, COL_MAJOR = 0, 1
+MAX_M = 16
+WS_COUNTER_BYTES = 65536
+
+if not os.path.exists(LIB_PATH):
+    # No CPU fallback exists: either the library gets built here (nvcc present) or the import fails.
+    try:
+        import importlib.util as _ilu
+        _spec = _ilu.spec_from_file_location("_nm_build", os.path.join(_PKG, "build.py"))
+        _build = _ilu.module_from_spec(_spec)
+        _spec.loader.exec_module(_build)
+        _build.build()
+    except Exception as exc:  # noqa: BLE001
+        raise ImportError(f"{LIB_PATH} is missing and could not be built with nvcc ({exc}); "
+                          "there is no CPU fallback") from exc
+_lib = C.CDLL(LIB_PATH)
+
+
+class NmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib.nm_status_string(status).decode()
+        cuda = _lib.nm_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({status})" + (f" [{cuda}]" if status == -5 and cuda else ""))
+
+
+_vp, _i, _l, _sz = C.c_void_p, C.c_int, C.c_long, C.c_size_t
+_lib.nm_version.restype = _i
+_lib.nm_status_string.restype = C.c_char_p
+_lib.nm_status_string.argtypes = [_i]
+_lib.nm_last_cuda_error.restype = C.c_char_p
+_lib.nm_matmul_workspace_bytes.restype = _sz
+_lib.nm_matmul_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
+_lib.nm_workspace_init.argtypes = [_vp, _sz, _vp]
+_lib.nm_set_workspace.argtypes = [_vp, _sz]
+_lib.nm_matmul.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]
+_lib.nm_matmul_ws.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]
+_lib.nm_matmul_batched.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _l, _l, _l, _l, _l, _i, _i, _vp]
+_lib.nm_matmul_batched_ws.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _l, _l, _l, _l, _l, _i, _i, _vp, _sz, _vp]
+_lib.nm_matmul_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]
+_lib.nm_debug_set_plan.argtypes = [_i, _i]
+_lib.nm_debug_get_plan.argtypes = [_i, _i, _i, _i, _i, _i, _i, C.POINTER(_i)]
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise NmError(status, where)
+
+
+def _ptr(t) -> int | None:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def nm_version() -> int:
+    return _lib.nm_version()
+
+
+def nm_status_string(status: int) -> str:
+    return _lib.nm_status_string(status).decode()
+
+
+def nm_matmul_workspace_bytes(M, N, K, H=1, dtype=BF16, layout_B=ROW_MAJOR) -> int:
+    return int(_lib.nm_matmul_workspace_bytes(M, N, K, H, dtype, layout_B))
+
+
+def nm_workspace_init(workspace, stream=None) -> None:
+    _check(_lib.nm_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream(stream)), "nm_workspace_init")
+
+
+def nm_set_workspace(workspace) -> None:
+    if workspace is None:
+        _check(_lib.nm_set_workspace(None, 0), "nm_set_workspace")
+    else:
+        _check(_lib.nm_set_workspace(_ptr(workspace), workspace.numel() * workspace.element_size()),
+               "nm_set_workspace")
+
+
+def nm_matmul(A, B, C_out, M, N, K, dtype, layout_B, stream=None) -> None:
+    _check(_lib.nm_matmul(_ptr(A), _ptr(B), _ptr(C_out), M, N, K, dtype, layout_B, _stream(stream)),
+           "nm_matmul")
+
+
+def nm_matmul_ws(A, B, C_out, M, N, K, dtype, layout_B, workspace, stream=None) -> None:
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.nm_matmul_ws(_ptr(A), _ptr(B), _ptr(C_out), M, N, K, dtype, layout_B,
+                             _ptr(workspace), nbytes, _stream(stream)), "nm_matmul_ws")
+
+
+def nm_matmul_batched(A, B, C_out, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout_B,
+                      stream=None) -> None:
+    _check(_lib.nm_matmul_batched(_ptr(A), _ptr(B), _ptr(C_out), M, N, K, H, lda, strideA, strideB,
+                                  ldc, strideC, dtype, layout_B, _stream(stream)), "nm_matmul_batched")
+
+
+def nm_matmul_batched_ws(A, B, C_out, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout_B,
+                         workspace, stream=None) -> None:
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.nm_matmul_batched_ws(_ptr(A), _ptr(B), _ptr(C_out), M, N, K, H, lda, strideA, strideB,
+                                     ldc, strideC, dtype, layout_B, _ptr(workspace), nbytes,
+                                     _stream(stream)), "nm_matmul_batched_ws")
+
+
+def nm_matmul_host(A_host, B, C_host, A_staging, C_staging, M, N, K, dtype, layout_B, workspace,
+                   stream=None) -> None:
+    """A_host / C_host are pinned CPU tensors; the rest are CUDA tensors."""
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.nm_matmul_host(_ptr(A_host), _ptr(B), _ptr(C_host), _ptr(A_staging), _ptr(C_staging),
+                               M, N, K, dtype, layout_B, _ptr(workspace), nbytes, _stream(stream)),
+           "nm_matmul_host")
+
+
+def nm_debug_set_plan(tile_n: int = 0, nsplit: int = 0) -> None:
+    _check(_lib.nm_debug_set_plan(tile_n, nsplit), "nm_debug_set_plan")
+
+
+def nm_debug_get_plan(M, N, K, H=1, dtype=BF16, layout_B=ROW_MAJOR, vec_ok=True) -> dict:
+    out = (_i * 6)()
+    _check(_lib.nm_debug_get_plan(M, N, K, H, dtype, layout_B, int(vec_ok), out), "nm_debug_get_plan")
+    return dict(kind=out[0], tile_n=out[1], nsplit=out[2], k_rows=out[3], tiles=out[4], ctas=out[5])
+
+
+def new_workspace(nbytes: int, device="cuda", stream=None) -> torch.Tensor:
+    """Allocate (with torch) and initialise a workspace of at least ``nbytes`` bytes."""
+    ws = torch.empty(max(int(nbytes), WS_COUNTER_BYTES), dtype=torch.uint8, device=device)
+    nm_workspace_init(ws, stream)
+    return ws

@@ -1,0 +1,77 @@
+// Shared device/host helpers for the nm kernels (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/nm.h"
+
+#if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ < 1000)
+#error "nm kernels are written for sm_100a"
+#endif
+
+namespace nm {
+
+constexpr int kSMs = 148;                 // B200: 2 dies x 74 SMs
+constexpr int kMaxSplit = 64;             // upper bound on k-splits (sizes the workspace)
+constexpr int kMaxTileN = 2048;           // upper bound on columns per CTA tile
+constexpr size_t kCounterBytes = NM_WS_COUNTER_BYTES;
+constexpr int kNumCounters = int(kCounterBytes / sizeof(unsigned));
+
+// Records a CUDA failure for nm_last_cuda_error() and maps it to NM_ERR_CUDA.
+int record_cuda_error(cudaError_t e, const char *where);
+
+#define NM_CUDA_TRY(expr)                                                        \
+    do {                                                                         \
+        cudaError_t _e = (expr);                                                 \
+        if (_e != cudaSuccess) return ::nm::record_cuda_error(_e, #expr);        \
+    } while (0)
+
+// ---- element traits -------------------------------------------------------------------------
+
+struct bf16_t { uint16_t bits; };
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kVec = 4;        // elements per 16-byte load
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&f)[4]) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ float widen(float x) { return x; }
+};
+template <> struct Elem<bf16_t> {
+    static constexpr int kVec = 8;
+    // bf16 is the upper half of an fp32: widening is a shift (exact).
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&f)[8]) {
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+    __device__ static __forceinline__ float widen(bf16_t x) { return __uint_as_float(uint32_t(x.bits) << 16); }
+};
+
+// Output rounding: one round-to-nearest-even step from the fp32 sum.
+template <typename T> __device__ __forceinline__ T round_out(float x);
+template <> __device__ __forceinline__ float round_out<float>(float x) { return x; }
+template <> __device__ __forceinline__ bf16_t round_out<bf16_t>(float x) {
+    bf16_t r; r.bits = __bfloat16_as_ushort(__float2bfloat16_rn(x)); return r;
+}
+
+// 16-byte streaming load: read-only path, no L1 allocation (each weight byte is used once).
+__device__ __forceinline__ uint4 ld_stream16(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Load that bypasses L1 (data written by other SMs in the same launch).
+__device__ __forceinline__ float ld_cg(const float *p) { return __ldcg(p); }
+
+__host__ __device__ constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+}  // namespace nm

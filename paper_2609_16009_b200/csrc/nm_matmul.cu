@@ -1,0 +1,282 @@
+// Host side of the narrow matrix product: argument checks, tiling plan, launches, C-ABI entry points.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+
+#include "nm_matmul_kernels.cuh"
+
+namespace nm {
+
+NM_EXTERN(row, bf16_t, bf16_t)
+NM_EXTERN(row, bf16_t, float)
+NM_EXTERN(row, float, float)
+NM_EXTERN(col, bf16_t, bf16_t)
+NM_EXTERN(col, bf16_t, float)
+NM_EXTERN(col, float, float)
+
+// ---- error bookkeeping ---------------------------------------------------------------------------
+static thread_local char g_cuda_error[256] = "";
+
+int record_cuda_error(cudaError_t e, const char *where)
+{
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", where, cudaGetErrorString(e));
+    return NM_ERR_CUDA;
+}
+
+// ---- default workspace and tuning overrides ----------------------------------------------------------
+static void *g_ws = nullptr;
+static size_t g_ws_bytes = 0;
+static int g_force_tn = 0, g_force_split = 0;
+
+enum PlanKind { kRowVec = 0, kColVec = 1, kGeneric = 2 };
+
+struct Plan {
+    PlanKind kind;
+    int tn, tpr, rg, nsplit, kr, ntiles;
+};
+
+static inline int elem_size(nm_dtype d) { return d == NM_F32 ? 4 : 2; }
+static inline int vec_elems(nm_dtype d) { return 16 / elem_size(d); }
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Pick the column tile and the number of k-splits.  The stream is HBM-bound, so the plan wants
+// (a) enough CTAs to cover all 148 SMs a few times over, (b) per-CTA segments of B as long and as
+// contiguous as the shape allows, (c) few enough splits that the partial-sum traffic stays a few
+// per cent of |B|.
+static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout, bool vec_ok)
+{
+    Plan p{};
+    const int V = vec_elems(dtype);
+    if (!vec_ok) {
+        p.kind = kGeneric; p.tn = kThreads; p.ntiles = ceil_div(N, kThreads); p.nsplit = 1; p.kr = K;
+        p.tpr = p.rg = 0;
+        return p;
+    }
+    const int target = (M <= 4 ? 4 : 2) * kSMs;       // CTAs wanted in flight
+    if (layout == NM_ROW_MAJOR) {
+        p.kind = kRowVec;
+        // threads per row: 8 -> 32 (128-byte to 512-byte row segments); wider when N is large
+        int tpr = 8;
+        const int chunks = N / V;
+        if (chunks >= 32 * 64) tpr = 32;
+        else if (chunks >= 16 * 24) tpr = 16;
+        if (g_force_tn > 0) tpr = g_force_tn / V;
+        if (tpr < 1) tpr = 1;
+        if (tpr > kThreads) tpr = kThreads;
+        p.tpr = tpr;
+        p.tn = tpr * V;
+        p.rg = kThreads / tpr;
+    } else {
+        p.kind = kColVec;
+        p.tn = (M <= 4 ? 4 : 2) * (kThreads / 32);
+        p.tpr = p.rg = 0;
+    }
+    p.ntiles = ceil_div(N, p.tn);
+    int nsplit = 1;
+    const long ctas = (long)p.ntiles * H;
+    if (ctas < target) nsplit = (int)((target + ctas - 1) / ctas);
+    // keep at least ~64 k-rows (row kernel) / 512 k (column kernel) per split
+    const int min_kr = (p.kind == kRowVec) ? 2 * p.rg : 512;
+    if (nsplit > K / min_kr) nsplit = K / min_kr;
+    if (g_force_split > 0) nsplit = g_force_split;
+    if (nsplit > kMaxSplit) nsplit = kMaxSplit;
+    if (nsplit < 1) nsplit = 1;
+    if ((long)p.ntiles * H > kNumCounters) nsplit = 1;
+    int kr = ceil_div(K, nsplit);
+    kr = ceil_div(kr, V) * V;
+    nsplit = ceil_div(K, kr);
+    p.nsplit = nsplit;
+    p.kr = kr;
+    return p;
+}
+
+static size_t partial_floats(const Plan &p, int M, int H)
+{
+    return p.nsplit > 1 ? (size_t)H * p.ntiles * p.nsplit * M * p.tn : 0;
+}
+
+static int check_common(const void *A, const void *B, const void *C, int M, int N, int K, int H,
+                        nm_dtype dtype, nm_layout layout)
+{
+    if (!A || !B || !C) return NM_ERR_INVALID_ARG;
+    if (M < 1 || M > NM_MAX_M || N < 1 || K < 1 || H < 1) return NM_ERR_INVALID_ARG;
+    if (dtype != NM_F32 && dtype != NM_BF16 && dtype != NM_BF16_F32OUT) return NM_ERR_UNSUPPORTED;
+    if (layout != NM_ROW_MAJOR && layout != NM_COL_MAJOR) return NM_ERR_UNSUPPORTED;
+    if (H > 65535) return NM_ERR_UNSUPPORTED;
+    const uintptr_t es = (uintptr_t)elem_size(dtype);
+    const uintptr_t os = (dtype == NM_BF16) ? 2 : 4;
+    if (((uintptr_t)A % es) || ((uintptr_t)B % es) || ((uintptr_t)C % os)) return NM_ERR_ALIGNMENT;
+    return NM_OK;
+}
+
+static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int K, int H,
+                       long lda, long strideA, long strideB, long ldc, long strideC,
+                       nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream)
+{
+    int rc = check_common(A, B, C, M, N, K, H, dtype, layout);
+    if (rc != NM_OK) return rc;
+    if (lda < K || ldc < N || strideA < 0 || strideB < 0 || strideC < 0) return NM_ERR_INVALID_ARG;
+
+    const int V = vec_elems(dtype);
+    // The 16-byte paths need B aligned with rows (columns) that stay aligned, and an aligned A for
+    // the column kernel (it copies A into shared memory with 16-byte loads).
+    const bool b_ok = aligned16(B) && (strideB % V == 0) &&
+                      (layout == NM_ROW_MAJOR ? (N % V == 0) : (K % V == 0));
+    const bool a_ok = aligned16(A) && (lda % V == 0) && (strideA % V == 0);
+    const bool vec_ok = b_ok && (layout == NM_ROW_MAJOR || a_ok);
+    Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok);
+
+    MatmulArgs a{};
+    a.A = A; a.B = B; a.C = C;
+    a.M = M; a.N = N; a.K = K; a.H = H;
+    a.lda = lda; a.strideA = strideA; a.strideB = strideB; a.ldc = ldc; a.strideC = strideC;
+    a.tn = p.tn; a.tpr = p.tpr; a.rg = p.rg; a.nsplit = p.nsplit; a.kr = p.kr; a.ntiles = p.ntiles;
+    a.a_vec = a_ok ? 1 : 0;
+    if (p.nsplit > 1) {
+        const size_t need = kCounterBytes + partial_floats(p, M, H) * sizeof(float);
+        if (!ws || ws_bytes < need) return NM_ERR_WORKSPACE;
+        if (!aligned16(ws)) return NM_ERR_ALIGNMENT;
+        a.counters = reinterpret_cast<unsigned *>(ws);
+        a.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + kCounterBytes);
+    }
+
+    cudaError_t e = cudaErrorInvalidValue;
+    if (p.kind == kGeneric) {
+        if (dtype == NM_F32)            e = launch_generic<float, float>(a, layout, stream);
+        else if (dtype == NM_BF16)      e = launch_generic<bf16_t, bf16_t>(a, layout, stream);
+        else                            e = launch_generic<bf16_t, float>(a, layout, stream);
+    } else if (p.kind == kRowVec) {
+        if (dtype == NM_F32)            e = launch_row<float, float>(a, stream);
+        else if (dtype == NM_BF16)      e = launch_row<bf16_t, bf16_t>(a, stream);
+        else                            e = launch_row<bf16_t, float>(a, stream);
+    } else {
+        if (dtype == NM_F32)            e = launch_col<float, float>(a, stream);
+        else if (dtype == NM_BF16)      e = launch_col<bf16_t, bf16_t>(a, stream);
+        else                            e = launch_col<bf16_t, float>(a, stream);
+    }
+    if (e != cudaSuccess) return record_cuda_error(e, "narrow matmul launch");
+    return NM_OK;
+}
+
+// internal entry used by the decode step
+int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, int H,
+                   long lda, long strideA, long strideB, long ldc, long strideC,
+                   nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream)
+{
+    return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout, ws, ws_bytes, stream);
+}
+
+}  // namespace nm
+
+using namespace nm;
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+int nm_version(void) { return 100; }
+
+const char *nm_status_string(int status)
+{
+    switch (status) {
+    case NM_OK: return "ok";
+    case NM_ERR_INVALID_ARG: return "invalid argument";
+    case NM_ERR_UNSUPPORTED: return "unsupported dtype, layout or dimension";
+    case NM_ERR_ALIGNMENT: return "pointer not aligned";
+    case NM_ERR_WORKSPACE: return "workspace missing or too small";
+    case NM_ERR_CUDA: return "CUDA error";
+    case NM_ERR_TIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown status";
+    }
+}
+
+const char *nm_last_cuda_error(void) { return g_cuda_error; }
+
+size_t nm_matmul_workspace_bytes(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B)
+{
+    (void)K; (void)dtype; (void)layout_B;
+    if (M < 1 || N < 1 || H < 1) return 0;
+    // Upper bound over every plan the library may choose: at most kMaxSplit partial tiles of at
+    // most (N rounded up to a tile) x M floats per head, plus the counters.
+    const size_t npad = (size_t)N + kMaxTileN;
+    return kCounterBytes + (size_t)kMaxSplit * (size_t)M * npad * (size_t)H * sizeof(float);
+}
+
+int nm_workspace_init(void *workspace, size_t bytes, nm_stream stream)
+{
+    if (!workspace || bytes < kCounterBytes) return NM_ERR_WORKSPACE;
+    NM_CUDA_TRY(cudaMemsetAsync(workspace, 0, kCounterBytes, (cudaStream_t)stream));
+    return NM_OK;
+}
+
+int nm_set_workspace(void *workspace, size_t bytes)
+{
+    if (!workspace) { g_ws = nullptr; g_ws_bytes = 0; return NM_OK; }
+    if (bytes < kCounterBytes) return NM_ERR_WORKSPACE;
+    NM_CUDA_TRY(cudaMemset(workspace, 0, kCounterBytes));
+    g_ws = workspace; g_ws_bytes = bytes;
+    return NM_OK;
+}
+
+int nm_matmul(const void *A, const void *B, void *C, int M, int N, int K,
+              nm_dtype dtype, nm_layout layout_B, nm_stream stream)
+{
+    return matmul_impl(A, B, C, M, N, K, 1, K, 0, 0, N, 0, dtype, layout_B, g_ws, g_ws_bytes, (cudaStream_t)stream);
+}
+
+int nm_matmul_ws(const void *A, const void *B, void *C, int M, int N, int K,
+                 nm_dtype dtype, nm_layout layout_B, void *workspace, size_t workspace_bytes, nm_stream stream)
+{
+    return matmul_impl(A, B, C, M, N, K, 1, K, 0, 0, N, 0, dtype, layout_B, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+int nm_matmul_batched(const void *A, const void *B, void *C, int M, int N, int K, int H,
+                      long lda, long strideA, long strideB, long ldc, long strideC,
+                      nm_dtype dtype, nm_layout layout_B, nm_stream stream)
+{
+    return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout_B, g_ws, g_ws_bytes, (cudaStream_t)stream);
+}
+
+int nm_matmul_batched_ws(const void *A, const void *B, void *C, int M, int N, int K, int H,
+                         long lda, long strideA, long strideB, long ldc, long strideC,
+                         nm_dtype dtype, nm_layout layout_B, void *workspace, size_t workspace_bytes, nm_stream stream)
+{
+    return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout_B, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+int nm_matmul_host(const void *A_host, const void *B, void *C_host, void *A_staging, void *C_staging,
+                   int M, int N, int K, nm_dtype dtype, nm_layout layout_B,
+                   void *workspace, size_t workspace_bytes, nm_stream stream)
+{
+    if (!A_host || !C_host || !A_staging || !C_staging) return NM_ERR_INVALID_ARG;
+    int rc = check_common(A_staging, B, C_staging, M, N, K, 1, dtype, layout_B);
+    if (rc != NM_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t a_bytes = (size_t)M * K * elem_size(dtype);
+    const size_t c_bytes = (size_t)M * N * (dtype == NM_BF16 ? 2 : 4);
+    NM_CUDA_TRY(cudaMemcpyAsync(A_staging, A_host, a_bytes, cudaMemcpyHostToDevice, s));
+    rc = matmul_impl(A_staging, B, C_staging, M, N, K, 1, K, 0, 0, N, 0, dtype, layout_B, workspace, workspace_bytes, s);
+    if (rc != NM_OK) return rc;
+    NM_CUDA_TRY(cudaMemcpyAsync(C_host, C_staging, c_bytes, cudaMemcpyDeviceToHost, s));
+    return NM_OK;
+}
+
+/* Tuning override for sweeps: columns per tile (row-major kernel) and k-splits; 0 = heuristic. */
+int nm_debug_set_plan(int tile_n, int nsplit)
+{
+    if (tile_n < 0 || nsplit < 0 || tile_n > kMaxTileN || nsplit > kMaxSplit) return NM_ERR_INVALID_ARG;
+    g_force_tn = tile_n; g_force_split = nsplit;
+    return NM_OK;
+}
+
+/* Reports the plan the library would use: out[0..5] = kind, tile_n, nsplit, k-rows per split, tiles, CTAs. */
+int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B, int vec_ok, int *out)
+{
+    if (!out) return NM_ERR_INVALID_ARG;
+    Plan p = make_plan(M, N, K, H, dtype, layout_B, vec_ok != 0);
+    out[0] = p.kind; out[1] = p.tn; out[2] = p.nsplit; out[3] = p.kr; out[4] = p.ntiles;
+    out[5] = p.ntiles * p.nsplit * H;
+    return NM_OK;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

@@ -1,0 +1,377 @@
+// Narrow matrix product kernels: C[MxN] = A[MxK] * B[KxN], 1 <= M <= 16, on CUDA cores.
+//
+// B is streamed from HBM exactly once with 16-byte read-only loads; A is staged in shared memory;
+// products accumulate in fp32 registers; K may be split over CTAs, in which case every CTA stores
+// an fp32 partial tile and the last CTA to arrive at a tile sums the partials in split order
+// (deterministic) and rounds once to the output type.  This is the split-K / partial-sum-buffer /
+// gather structure of Algorithm 1, with the device-wide barrier replaced by an arrival counter so
+// that no CTA ever waits on another.
+#pragma once
+
+#include "nm_common.cuh"
+
+namespace nm {
+
+constexpr int kThreads = 256;
+constexpr int kSmemFloats = 8192;         // 32 KB: A chunk during the stream, reduction buffer after
+
+struct MatmulArgs {
+    const void *A, *B;
+    void *C;
+    int M, N, K, H;
+    long lda, strideA, strideB, ldc, strideC;
+    int tn;        // columns per CTA tile
+    int tpr;       // row kernel: threads per B row (tn / kVec)
+    int rg;        // row kernel: row groups per CTA (kThreads / tpr)
+    int nsplit;    // k-splits (gridDim.y)
+    int kr;        // k-rows per split (multiple of kVec)
+    int ntiles;    // column tiles (gridDim.x)
+    int a_vec;     // A rows can be staged with 16-byte loads
+    float *partial;
+    unsigned *counters;
+};
+
+template <int M> struct RowCfg {
+    static constexpr int kUnroll = (M <= 4) ? 8 : (M <= 8 ? 6 : 4);
+    static constexpr int kMinBlocks = (M <= 2) ? 3 : (M <= 8 ? 2 : 1);
+    static constexpr int kChunk = ((kSmemFloats / M) / 8) * 8;     // k-rows of A held in smem
+    static constexpr int kPass = (M < 4) ? M : 4;                  // m-rows reduced per pass
+};
+
+// ---- split-K completion shared by both kernels -----------------------------------------------------
+//
+// Called by all threads of the CTA after its partial tile has been written to `partial`.  The
+// last CTA to arrive at (h, tile) reads all nsplit partial tiles in order and writes C; it then
+// puts the counter back to zero, so the workspace needs no clearing between launches.
+template <int M, typename TO>
+__device__ __forceinline__ void splitk_complete(const MatmulArgs &a, int tile, int h, int *s_last)
+{
+    const int tid = threadIdx.x;
+    __threadfence();
+    __syncthreads();
+    unsigned *cnt = a.counters + (size_t)h * a.ntiles + tile;
+    if (tid == 0) {
+        unsigned t = atomicAdd(cnt, 1u);
+        *s_last = (t == (unsigned)(a.nsplit - 1));
+    }
+    __syncthreads();
+    if (!*s_last) return;
+    __threadfence();
+    const float *P = a.partial + ((size_t)h * a.ntiles + tile) * a.nsplit * (size_t)(M * a.tn);
+    TO *C = (TO *)a.C + (long)h * a.strideC;
+    for (int i = tid; i < M * a.tn; i += kThreads) {
+        const int m = i / a.tn, c = i - m * a.tn, n = tile * a.tn + c;
+        if (n < a.N) {
+            float s = 0.f;
+            for (int sp = 0; sp < a.nsplit; ++sp) s += ld_cg(P + ((size_t)sp * M + m) * a.tn + c);
+            C[(long)m * a.ldc + n] = round_out<TO>(s);
+        }
+    }
+    if (tid == 0) *cnt = 0u;
+}
+
+// ---- row-major B (n contiguous): each thread owns kVec consecutive columns ---------------------------
+template <int M, typename TI>
+__device__ __forceinline__ void fma_row(float (&acc)[M][Elem<TI>::kVec], const uint4 &v,
+                                        const float *As /* &As[0][row] */)
+{
+    constexpr int V = Elem<TI>::kVec;
+    float b[V];
+    Elem<TI>::unpack(v, b);
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        const float am = As[m * RowCfg<M>::kChunk];
+#pragma unroll
+        for (int j = 0; j < V; ++j) acc[m][j] = fmaf(am, b[j], acc[m][j]);
+    }
+}
+
+template <int M, typename TI, typename TO>
+__global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel(const MatmulArgs a)
+{
+    using E = Elem<TI>;
+    constexpr int V = E::kVec;
+    constexpr int U = RowCfg<M>::kUnroll;
+    constexpr int KC = RowCfg<M>::kChunk;
+    constexpr int MP = RowCfg<M>::kPass;
+    __shared__ __align__(16) float smem[kSmemFloats];
+    __shared__ int s_last;
+
+    const int tid = threadIdx.x;
+    const int tx = tid % a.tpr, ty = tid / a.tpr;
+    const int tile = blockIdx.x, split = blockIdx.y, h = blockIdx.z;
+    const int n0 = tile * a.tn + tx * V;
+    const bool active = (ty < a.rg) && (n0 < a.N);
+    const int kb = split * a.kr;
+    const int ke = min(a.K, kb + a.kr);
+    const int rg = a.rg;
+    const long ldb = a.N;
+    const TI *__restrict__ A = (const TI *)a.A + (long)h * a.strideA;
+    const TI *__restrict__ B = (const TI *)a.B + (long)h * a.strideB;
+
+    float acc[M][V];
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int j = 0; j < V; ++j) acc[m][j] = 0.f;
+
+    for (int kc = kb; kc < ke; kc += KC) {
+        const int klen = min(KC, ke - kc);
+        const TI *bp = B + (long)kc * ldb + n0;
+        // First batch of weight loads goes out before A is staged, so the two latencies overlap.
+        uint4 v[U];
+        int r = ty;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int rr = r + u * rg;
+            v[u] = (active && rr < klen) ? ld_stream16(bp + (long)rr * ldb) : make_uint4(0, 0, 0, 0);
+        }
+        __syncthreads();                                  // readers of the previous chunk are done
+        if (a.a_vec) {
+            const int nv = klen / V;                      // klen is a multiple of kVec on this path
+            for (int m = 0; m < M; ++m) {
+                const uint4 *src = (const uint4 *)(A + (long)m * a.lda + kc);
+                for (int i = tid; i < nv; i += kThreads) {
+                    float f[V];
+                    E::unpack(__ldg(src + i), f);
+#pragma unroll
+                    for (int j = 0; j < V; ++j) smem[m * KC + i * V + j] = f[j];
+                }
+                for (int i = nv * V + tid; i < klen; i += kThreads) smem[m * KC + i] = E::widen(A[(long)m * a.lda + kc + i]);
+            }
+        } else {
+            for (int m = 0; m < M; ++m)
+                for (int i = tid; i < klen; i += kThreads) smem[m * KC + i] = E::widen(A[(long)m * a.lda + kc + i]);
+        }
+        __syncthreads();
+        if (active) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int rr = r + u * rg;
+                if (rr < klen) fma_row<M, TI>(acc, v[u], smem + rr);
+            }
+            r += U * rg;
+            for (; r + (U - 1) * rg < klen; r += U * rg) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) v[u] = ld_stream16(bp + (long)(r + u * rg) * ldb);
+#pragma unroll
+                for (int u = 0; u < U; ++u) fma_row<M, TI>(acc, v[u], smem + r + u * rg);
+            }
+            for (; r < klen; r += rg) {
+                const uint4 w = ld_stream16(bp + (long)r * ldb);
+                fma_row<M, TI>(acc, w, smem + r);
+            }
+        }
+    }
+
+    // Reduce the rg row groups of the CTA through shared memory, MP rows of C per pass.
+    float *red = smem;
+    TO *C = (TO *)a.C + (long)h * a.strideC;
+    float *P = a.partial ? a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * a.tn) : nullptr;
+#pragma unroll
+    for (int m0 = 0; m0 < M; m0 += MP) {
+        __syncthreads();
+        if (ty < rg) {
+#pragma unroll
+            for (int mm = 0; mm < MP; ++mm) {
+                if (m0 + mm < M) {
+                    float4 *dst = (float4 *)(red + (size_t)(ty * MP + mm) * a.tn + tx * V);
+#pragma unroll
+                    for (int j = 0; j < V; j += 4)
+                        dst[j / 4] = make_float4(acc[m0 + mm][j], acc[m0 + mm][j + 1], acc[m0 + mm][j + 2], acc[m0 + mm][j + 3]);
+                }
+            }
+        }
+        __syncthreads();
+        for (int i = tid; i < MP * a.tn; i += kThreads) {
+            const int mm = i / a.tn, c = i - mm * a.tn, m = m0 + mm, n = tile * a.tn + c;
+            if (m < M && n < a.N) {
+                float s = 0.f;
+                for (int g = 0; g < rg; ++g) s += red[(size_t)(g * MP + mm) * a.tn + c];
+                if (a.nsplit == 1) C[(long)m * a.ldc + n] = round_out<TO>(s);
+                else               P[(size_t)m * a.tn + c] = s;
+            }
+        }
+    }
+    if (a.nsplit > 1) splitk_complete<M, TO>(a, tile, h, &s_last);
+}
+
+// ---- column-major B (k contiguous): each warp owns kCols columns, lanes stride along k ------------------
+template <int M> struct ColCfg {
+    static constexpr int kCols = (M <= 4) ? 4 : 2;                 // columns per warp
+    static constexpr int kWarps = kThreads / 32;
+    static constexpr int kTile = kCols * kWarps;                   // columns per CTA
+};
+
+template <int M, typename TI, typename TO>
+__global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
+{
+    using E = Elem<TI>;
+    constexpr int V = E::kVec;
+    constexpr int CW = ColCfg<M>::kCols;
+    constexpr int STEP = 32 * V;                                   // k covered by a warp per load
+    // A chunk kept in its storage type: M x KC elements in 32 KB
+    constexpr int KC = (((kSmemFloats * 4 / (int)sizeof(TI)) / M) / STEP) * STEP;
+    __shared__ __align__(16) float smem[kSmemFloats];
+    __shared__ int s_last;
+    uint4 *As = (uint4 *)smem;                                     // [M][KC / V] 16-byte vectors
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tile = blockIdx.x, split = blockIdx.y, h = blockIdx.z;
+    const int col0 = tile * a.tn + warp * CW;
+    const int kb = split * a.kr;
+    const int ke = min(a.K, kb + a.kr);
+    const TI *__restrict__ A = (const TI *)a.A + (long)h * a.strideA;
+    const TI *__restrict__ B = (const TI *)a.B + (long)h * a.strideB;
+    const long ldb = a.K;
+
+    float acc[M][CW];
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int c = 0; c < CW; ++c) acc[m][c] = 0.f;
+
+    for (int kc = kb; kc < ke; kc += KC) {
+        const int klen = min(KC, ke - kc);                         // multiple of V
+        uint4 b0[CW], b1[CW];
+        int kk = lane * V;
+        // first two batches of weight loads go out before A is staged
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+            const bool okc = col0 + c < a.N;
+            const TI *bp = B + (long)(col0 + c) * ldb + kc;
+            b0[c] = (okc && kk < klen) ? ld_stream16(bp + kk) : make_uint4(0, 0, 0, 0);
+            b1[c] = (okc && kk + STEP < klen) ? ld_stream16(bp + kk + STEP) : make_uint4(0, 0, 0, 0);
+        }
+        __syncthreads();
+        const int nv = klen / V;
+        for (int m = 0; m < M; ++m) {
+            const uint4 *src = (const uint4 *)(A + (long)m * a.lda + kc);
+            for (int i = tid; i < nv; i += kThreads) As[m * (KC / V) + i] = __ldg(src + i);
+        }
+        __syncthreads();
+        for (; kk < klen; kk += 2 * STEP) {
+            const bool second = kk + STEP < klen;
+            float bf0[CW][V], bf1[CW][V];
+#pragma unroll
+            for (int c = 0; c < CW; ++c) { E::unpack(b0[c], bf0[c]); E::unpack(b1[c], bf1[c]); }
+            // next two batches
+            const int kn = kk + 2 * STEP;
+#pragma unroll
+            for (int c = 0; c < CW; ++c) {
+                const bool okc = col0 + c < a.N;
+                const TI *bp = B + (long)(col0 + c) * ldb + kc;
+                b0[c] = (okc && kn < klen) ? ld_stream16(bp + kn) : make_uint4(0, 0, 0, 0);
+                b1[c] = (okc && kn + STEP < klen) ? ld_stream16(bp + kn + STEP) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                float af[V];
+                E::unpack(As[m * (KC / V) + kk / V], af);
+#pragma unroll
+                for (int c = 0; c < CW; ++c)
+#pragma unroll
+                    for (int j = 0; j < V; ++j) acc[m][c] = fmaf(af[j], bf0[c][j], acc[m][c]);
+                if (second) {
+                    E::unpack(As[m * (KC / V) + (kk + STEP) / V], af);
+#pragma unroll
+                    for (int c = 0; c < CW; ++c)
+#pragma unroll
+                        for (int j = 0; j < V; ++j) acc[m][c] = fmaf(af[j], bf1[c][j], acc[m][c]);
+                }
+            }
+        }
+    }
+
+    // butterfly over the 32 lanes; lane (m*CW + c) keeps element (m, c)
+    float mine = 0.f;
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+            float s = acc[m][c];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (lane == m * CW + c) mine = s;
+        }
+    if (lane < M * CW) {
+        const int m = lane / CW, c = lane - m * CW, n = col0 + c;
+        if (n < a.N) {
+            if (a.nsplit == 1) {
+                ((TO *)a.C + (long)h * a.strideC)[(long)m * a.ldc + n] = round_out<TO>(mine);
+            } else {
+                float *P = a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * a.tn);
+                P[(size_t)m * a.tn + warp * CW + c] = mine;
+            }
+        }
+    }
+    if (a.nsplit > 1) splitk_complete<M, TO>(a, tile, h, &s_last);
+}
+
+// ---- scalar kernel for shapes the vector paths cannot take (odd N / K, unaligned pointers) ------------------
+template <typename TI, typename TO>
+__global__ void __launch_bounds__(kThreads) nm_generic_kernel(const MatmulArgs a, int layout)
+{
+    const int n = blockIdx.x * kThreads + threadIdx.x, h = blockIdx.z;
+    if (n >= a.N) return;
+    const TI *__restrict__ A = (const TI *)a.A + (long)h * a.strideA;
+    const TI *__restrict__ B = (const TI *)a.B + (long)h * a.strideB;
+    float acc[NM_MAX_M];
+#pragma unroll
+    for (int m = 0; m < NM_MAX_M; ++m) acc[m] = 0.f;
+    for (int k = 0; k < a.K; ++k) {
+        const long ib = (layout == NM_ROW_MAJOR) ? (long)k * a.N + n : (long)n * a.K + k;
+        const float b = Elem<TI>::widen(B[ib]);
+#pragma unroll
+        for (int m = 0; m < NM_MAX_M; ++m)
+            if (m < a.M) acc[m] = fmaf(Elem<TI>::widen(A[(long)m * a.lda + k]), b, acc[m]);
+    }
+    TO *C = (TO *)a.C + (long)h * a.strideC;
+#pragma unroll
+    for (int m = 0; m < NM_MAX_M; ++m)
+        if (m < a.M) C[(long)m * a.ldc + n] = round_out<TO>(acc[m]);
+}
+
+// ---- launch helpers (explicitly instantiated per element type in their own translation units) ------------
+#define NM_FOR_EACH_M(X) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16)
+
+template <typename TI, typename TO>
+cudaError_t launch_row(const MatmulArgs &a, cudaStream_t s)
+{
+    dim3 grid(a.ntiles, a.nsplit, a.H);
+    switch (a.M) {
+#define NM_X(m) case m: nm_row_kernel<m, TI, TO><<<grid, kThreads, 0, s>>>(a); break;
+        NM_FOR_EACH_M(NM_X)
+#undef NM_X
+    default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+template <typename TI, typename TO>
+cudaError_t launch_col(const MatmulArgs &a, cudaStream_t s)
+{
+    dim3 grid(a.ntiles, a.nsplit, a.H);
+    switch (a.M) {
+#define NM_X(m) case m: nm_col_kernel<m, TI, TO><<<grid, kThreads, 0, s>>>(a); break;
+        NM_FOR_EACH_M(NM_X)
+#undef NM_X
+    default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+template <typename TI, typename TO>
+cudaError_t launch_generic(const MatmulArgs &a, int layout, cudaStream_t s)
+{
+    dim3 grid(ceil_div(a.N, kThreads), 1, a.H);
+    nm_generic_kernel<TI, TO><<<grid, kThreads, 0, s>>>(a, layout);
+    return cudaGetLastError();
+}
+
+#define NM_INSTANTIATE(KIND, TI, TO) \
+    template cudaError_t launch_##KIND<TI, TO>(const MatmulArgs &, cudaStream_t);
+#define NM_EXTERN(KIND, TI, TO) \
+    extern template cudaError_t launch_##KIND<TI, TO>(const MatmulArgs &, cudaStream_t);
+
+}  // namespace nm

@@ -1,0 +1,82 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the public headers
+declare, and its host-only logic (status strings, workspace sizing, tiling plans, argument
+validation that needs no device) behaves.  No kernel is launched here."""
+import ctypes
+import glob
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2609_16009_b200 import build
+    path = build.build()
+    return ctypes.CDLL(path)
+
+
+def declared_functions():
+    names = []
+    for h in glob.glob(os.path.join(ROOT, "include", "*.h")):
+        text = open(h).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names += re.findall(r"\b(nm_[a-z0-9_]+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert "nm_matmul" in names and "nm_matmul_batched" in names
+    missing = [n for n in names if not hasattr(lib, n)]
+    assert not missing, f"declared in include/ but not exported: {missing}"
+
+
+def test_status_strings_and_version(lib):
+    lib.nm_status_string.restype = ctypes.c_char_p
+    assert lib.nm_version() >= 100
+    assert lib.nm_status_string(0) == b"ok"
+    seen = {lib.nm_status_string(-i) for i in range(1, 7)}
+    assert len(seen) == 6 and b"unknown status" not in seen
+    assert lib.nm_status_string(-99) == b"unknown status"
+
+
+def test_workspace_bound_covers_every_plan(lib):
+    lib.nm_matmul_workspace_bytes.restype = ctypes.c_size_t
+    out = (ctypes.c_int * 6)()
+    for M in (1, 3, 16):
+        for (N, K, H) in ((576, 7168, 1), (1536, 7168, 1), (24576, 1536, 1), (512, 128, 128), (8, 100000, 1), (7168, 16384, 1)):
+            for layout in (0, 1):
+                for tile_n, nsplit in ((0, 0), (64, 64), (2048, 64), (8, 64), (136, 7)):
+                    assert lib.nm_debug_set_plan(tile_n, nsplit) == 0
+                    assert lib.nm_debug_get_plan(M, N, K, H, 1, layout, 1, out) == 0
+                    kind, tn, ns, kr, tiles, ctas = list(out)
+                    assert 1 <= ns <= 64 and kr % 8 == 0 and (ns - 1) * kr < K <= ns * kr
+                    assert tiles * tn >= N > (tiles - 1) * tn
+                    need = 65536 + (H * tiles * ns * M * tn * 4 if ns > 1 else 0)
+                    assert need <= lib.nm_matmul_workspace_bytes(M, N, K, H, 1, layout)
+    lib.nm_debug_set_plan(0, 0)
+
+
+def test_heuristic_fills_the_gpu_for_the_paper_shape(lib):
+    out = (ctypes.c_int * 6)()
+    lib.nm_debug_set_plan(0, 0)
+    for layout in (0, 1):
+        assert lib.nm_debug_get_plan(1, 576, 7168, 1, 1, layout, 1, out) == 0
+        assert out[5] >= 148, "MatMul 2 shape must cover every SM"
+    # a shape that cannot use 16-byte loads falls back to the scalar kernel, unsplit
+    assert lib.nm_debug_get_plan(1, 577, 7168, 1, 1, 0, 0, out) == 0
+    assert out[0] == 2 and out[2] == 1
+
+
+def test_argument_validation_needs_no_device(lib):
+    vp = ctypes.c_void_p
+    lib.nm_matmul.argtypes = [vp, vp, vp] + [ctypes.c_int] * 5 + [vp]
+    assert lib.nm_matmul(None, None, None, 1, 8, 8, 1, 0, None) == -1
+    assert lib.nm_matmul(vp(256), vp(512), vp(1024), 0, 8, 8, 1, 0, None) == -1
+    assert lib.nm_matmul(vp(256), vp(512), vp(1024), 17, 8, 8, 1, 0, None) == -1
+    assert lib.nm_matmul(vp(256), vp(512), vp(1024), 1, 8, 8, 7, 0, None) == -2
+    assert lib.nm_matmul(vp(257), vp(512), vp(1024), 1, 8, 8, 1, 0, None) == -3
+    assert lib.nm_set_workspace(vp(4096), ctypes.c_size_t(16)) == -4

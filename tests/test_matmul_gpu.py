@@ -1,0 +1,237 @@
+"""Parity of the CUDA narrow matrix product with the CPU oracle, through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+import nm_inputs as gen
+import oracle
+from gpu_util import (NP_IN, ORACLE_IN, ORACLE_OUT, assert_matmul_close, guards_intact, out_buffer,
+                      out_to_f64, to_dev)
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16, BF16_F32OUT = 0, 1, 2
+ROW, COL = 0, 1
+
+
+@pytest.fixture(scope="module")
+def nm():
+    import paper_2609_16009_b200 as nm
+    ws = nm.new_workspace(64 << 20)
+    nm.nm_set_workspace(ws)
+    yield nm
+    nm.nm_debug_set_plan(0, 0)
+    nm.nm_set_workspace(None)
+
+
+def run_case(nm, A, B_row, M, N, K, dtype, layout, what, full_oracle=True, cols=None, twice=True):
+    B = B_row if layout == ROW else gen.to_col_major(B_row)
+    dA, dB = to_dev(A), to_dev(B)
+    whole, dC = out_buffer(M * N, dtype)
+    nm.nm_matmul(dA, dB, dC, M, N, K, dtype, layout)
+    torch.cuda.synchronize()
+    got = out_to_f64(dC, dtype).reshape(M, N)
+    assert guards_intact(whole, M * N, dtype), f"{what}: wrote outside C"
+    if twice:   # determinism: no float atomics, fixed-order reductions
+        first = dC.clone()
+        nm.nm_matmul(dA, dB, dC, M, N, K, dtype, layout)
+        torch.cuda.synchronize()
+        assert torch.equal(first, dC), f"{what}: two runs differ"
+    if cols is None:
+        Cq, C64, bound = oracle.matmul(A, B, M, N, K, ORACLE_IN[dtype], ORACLE_OUT[dtype], layout, threads=8)
+        assert_matmul_close(got, Cq, C64, bound, dtype, what)
+    else:
+        Cq, C64, bound = oracle.matmul_columns(A, B, M, N, K, cols, ORACLE_IN[dtype], ORACLE_OUT[dtype], layout)
+        assert_matmul_close(got[:, cols], Cq, C64, bound, dtype, what)
+    return got
+
+
+def make_inputs(M, K, N, dtype, seed):
+    if dtype == F32:
+        return gen.uniform_f32((M, K), -1, 1, seed), gen.uniform_f32((K, N), -1, 1, seed + 1)
+    return gen.narrow_bf16(M, K, N, seed)
+
+
+# ---- the named configurations ------------------------------------------------------------------------
+
+def test_gemv_fp32_512(nm):
+    A, B = gen.gemv_fp32(seed=0)
+    run_case(nm, A, B, 1, 512, 512, F32, ROW, "fp32 GEMV 512x512")
+    run_case(nm, A, B, 1, 512, 512, F32, COL, "fp32 GEMV 512x512 col-major")
+
+
+@pytest.mark.parametrize("N", [1536, 576])
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("dtype", [BF16, BF16_F32OUT])
+def test_down_projection_shapes(nm, N, layout, dtype):
+    A, B = gen.narrow_bf16(1, 7168, N, seed=1000 + N)
+    run_case(nm, A, B, 1, N, 7168, dtype, layout, f"M=1 K=7168 N={N} layout={layout}")
+
+
+@pytest.mark.parametrize("K,N", [(1536, 24576), (7168, 18432)])
+@pytest.mark.parametrize("M", [1, 2, 4, 8, 16])
+def test_m_sweep_full_size_sampled_columns(nm, K, N, M):
+    A, B = gen.narrow_bf16(M, K, N, seed=2000 + M)
+    rng = np.random.default_rng(M)
+    cols = sorted(set([0, 7, 8, 255, 256, N - 1, N - 8] + rng.integers(0, N, 56).tolist()))
+    run_case(nm, A, B, M, N, K, BF16, ROW, f"M={M} K={K} N={N}", cols=cols)
+
+
+# ---- every M, ragged shapes, both layouts, all dtypes ------------------------------------------------------
+
+@pytest.mark.parametrize("M", list(range(1, 17)))
+@pytest.mark.parametrize("layout", [ROW, COL])
+def test_every_m_vector_path(nm, M, layout):
+    # several tiles in N with a ragged last tile; several k-chunks with a ragged tail
+    K, N = 1000, 840
+    A, B = gen.narrow_bf16(M, K, N, seed=300 + M)
+    run_case(nm, A, B, M, N, K, BF16, layout, f"M={M} K={K} N={N} layout={layout}")
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16, BF16_F32OUT])
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("M,K,N", [(1, 1, 1), (3, 5, 7), (2, 129, 33), (16, 77, 1), (5, 1023, 259),
+                                    (1, 8, 8), (4, 4096, 8), (7, 8, 2048), (16, 2600, 72)])
+def test_ragged_and_degenerate_shapes(nm, dtype, layout, M, K, N):
+    A, B = make_inputs(M, K, N, dtype, seed=400 + M + K + N)
+    run_case(nm, A, B, M, N, K, dtype, layout, f"dtype={dtype} layout={layout} {M}x{K}x{N}")
+
+
+@pytest.mark.parametrize("layout", [ROW, COL])
+def test_long_k_spans_several_shared_memory_chunks(nm, layout):
+    M, K, N = 16, 9000, 64
+    A, B = gen.narrow_bf16(M, K, N, seed=500)
+    nm.nm_debug_set_plan(0, 1)           # no split: one CTA walks all of K in chunks
+    try:
+        run_case(nm, A, B, M, N, K, BF16, layout, f"long K layout={layout}")
+    finally:
+        nm.nm_debug_set_plan(0, 0)
+
+
+# ---- split-K: forced plans, determinism -----------------------------------------------------------------
+
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("nsplit", [1, 2, 7, 16, 64])
+@pytest.mark.parametrize("tile_n", [0, 64, 136, 512])
+def test_forced_plans_agree(nm, layout, nsplit, tile_n):
+    M, K, N = 3, 7168, 576
+    A, B = gen.narrow_bf16(M, K, N, seed=600)
+    nm.nm_debug_set_plan(tile_n, nsplit)
+    try:
+        run_case(nm, A, B, M, N, K, BF16, layout, f"forced tile_n={tile_n} nsplit={nsplit} layout={layout}")
+    finally:
+        nm.nm_debug_set_plan(0, 0)
+
+
+@pytest.mark.parametrize("layout", [ROW, COL])
+def test_small_integers_bit_exact_full_k(nm, layout):
+    # every product and every partial sum is an integer below 2^24: any summation order is exact,
+    # so the fp32 result must match the oracle bit for bit
+    M, K, N = 4, 7168, 576
+    A = gen.small_int_bf16((M, K), -8, 8, seed=701)
+    B = gen.small_int_bf16((K, N), -8, 8, seed=702)
+    got = run_case(nm, A, B, M, N, K, BF16_F32OUT, layout, "small ints")
+    _, C64, _ = oracle.matmul(A, B if layout == ROW else gen.to_col_major(B), M, N, K, oracle.BF16, oracle.F32, layout, threads=8)
+    assert np.array_equal(got, C64)
+
+
+def test_rounding_ties_to_even_on_device(nm):
+    K = 64
+    A = gen.bf16_bits(torch.ones(1, K))
+    cols = []
+    for total in (257.0, 259.0, 255.0, -257.0):
+        col = np.full(K, np.sign(total) * 4.0, np.float32)
+        col[0] = total - np.sign(total) * 4.0 * (K - 1)
+        cols.append(col)
+    B = gen.bf16_bits(torch.from_numpy(np.stack(cols, axis=1)))        # K x 4
+    Bp = np.zeros((K, 8), np.uint16); Bp[:, :4] = B
+    got = run_case(nm, A, Bp, 1, 8, K, BF16, ROW, "ties")
+    assert got[0, :4].tolist() == [256.0, 260.0, 255.0, -256.0]
+
+
+# ---- batched per-head products ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("T", [1, 4, 16])
+def test_per_head_absorbed_products(nm, T):
+    H, nope, dc, dv, rope = 128, 128, 512, 128, 64
+    d = gen.per_head(T, seed=3000 + T)
+    # q_nope read in place from q[T][H][nope+rope]
+    q = gen.normal_bf16((T, H, nope + rope), 1.0, seed=3100 + T)
+    dq, dW = to_dev(q), to_dev(d["W_UK"])
+    whole, dC = out_buffer(T * H * dc, BF16)
+    nm.nm_matmul_batched(dq, dW, dC, T, dc, nope, H, H * (nope + rope), nope + rope, nope * dc, H * dc, dc, BF16, ROW)
+    torch.cuda.synchronize()
+    assert guards_intact(whole, T * H * dc, BF16)
+    Cq, C64, bound = oracle.matmul_batched(q, d["W_UK"], T, dc, nope, H, H * (nope + rope), nope + rope,
+                                           nope * dc, H * dc, dc, T * H * dc, oracle.BF16, oracle.BF16, threads=8)
+    assert_matmul_close(out_to_f64(dC, BF16), Cq, C64, bound, BF16, f"W_UK T={T}")
+    # o_lat [T,H,dc] * W_UV [H,dc,dv]
+    dO, dW = to_dev(d["o_lat"]), to_dev(d["W_UV"])
+    whole, dC = out_buffer(T * H * dv, BF16)
+    nm.nm_matmul_batched(dO, dW, dC, T, dv, dc, H, H * dc, dc, dc * dv, H * dv, dv, BF16, ROW)
+    torch.cuda.synchronize()
+    assert guards_intact(whole, T * H * dv, BF16)
+    Cq, C64, bound = oracle.matmul_batched(d["o_lat"], d["W_UV"], T, dv, dc, H, H * dc, dc, dc * dv, H * dv, dv,
+                                           T * H * dv, oracle.BF16, oracle.BF16, threads=8)
+    assert_matmul_close(out_to_f64(dC, BF16), Cq, C64, bound, BF16, f"W_UV T={T}")
+
+
+@pytest.mark.parametrize("layout", [ROW, COL])
+def test_batched_small_ragged(nm, layout):
+    T, H, K, N = 3, 5, 40, 24
+    A = gen.normal_bf16((T, H, K), 1.0, seed=3200)
+    W = gen.normal_bf16((H, K, N), 0.02, seed=3201)
+    Wst = W if layout == ROW else np.ascontiguousarray(W.transpose(0, 2, 1))
+    dA, dW = to_dev(A), to_dev(Wst)
+    whole, dC = out_buffer(T * H * N, BF16_F32OUT)
+    nm.nm_matmul_batched(dA, dW, dC, T, N, K, H, H * K, K, K * N, H * N, N, BF16_F32OUT, layout)
+    torch.cuda.synchronize()
+    assert guards_intact(whole, T * H * N, BF16_F32OUT)
+    Cq, C64, bound = oracle.matmul_batched(A, Wst, T, N, K, H, H * K, K, K * N, H * N, N, T * H * N,
+                                           oracle.BF16, oracle.F32, layout)
+    assert_matmul_close(out_to_f64(dC, BF16_F32OUT), Cq, C64, bound, BF16_F32OUT, "batched ragged")
+
+
+# ---- host-operand entry point ------------------------------------------------------------------------------
+
+def test_matmul_host_operands(nm):
+    M, K, N = 2, 7168, 576
+    A, B = gen.narrow_bf16(M, K, N, seed=800)
+    A_host = torch.from_numpy(A.view(np.int16).copy()).pin_memory()
+    C_host = torch.zeros(M * N, dtype=torch.int16).pin_memory()
+    dB = to_dev(B)
+    dA = torch.empty(M * K, dtype=torch.int16, device="cuda")
+    dC = torch.empty(M * N, dtype=torch.int16, device="cuda")
+    ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(M, N, K))
+    nm.nm_matmul_host(A_host, dB, C_host, dA, dC, M, N, K, BF16, ROW, ws)
+    torch.cuda.synchronize()
+    Cq, C64, bound = oracle.matmul(A, B, M, N, K, oracle.BF16, oracle.BF16, ROW, threads=8)
+    assert_matmul_close(oracle.bf16_to_f64(C_host.numpy().view(np.uint16)), Cq, C64, bound, BF16, "host operands")
+
+
+# ---- error behaviour (host-side only; nothing is enqueued) --------------------------------------------------
+
+def test_error_codes(nm):
+    A = torch.zeros(16 * 64, dtype=torch.int16, device="cuda")
+    B = torch.zeros(64 * 64, dtype=torch.int16, device="cuda")
+    Cb = torch.zeros(16 * 64, dtype=torch.int16, device="cuda")
+    def status(fn, *a):
+        try:
+            fn(*a)
+            return 0
+        except nm.NmError as e:
+            return e.status
+    assert status(nm.nm_matmul, A, B, Cb, 0, 64, 64, BF16, ROW) == -1
+    assert status(nm.nm_matmul, A, B, Cb, 17, 64, 64, BF16, ROW) == -1
+    assert status(nm.nm_matmul, A, B, Cb, 1, 0, 64, BF16, ROW) == -1
+    assert status(nm.nm_matmul, None, B, Cb, 1, 64, 64, BF16, ROW) == -1
+    assert status(nm.nm_matmul, A, B, Cb, 1, 64, 64, 9, ROW) == -2
+    assert status(nm.nm_matmul, A, B, Cb, 1, 64, 64, BF16, 5) == -2
+    assert status(nm.nm_matmul, A.data_ptr() + 1, B, Cb, 1, 64, 64, BF16, ROW) == -3
+    # split-K without a workspace
+    nm.nm_debug_set_plan(0, 4)
+    try:
+        assert status(nm.nm_matmul_ws, A, B, Cb, 1, 64, 64, BF16, ROW, None) == -4
+    finally:
+        nm.nm_debug_set_plan(0, 0)
+    torch.cuda.synchronize()

@@ -58,6 +58,14 @@ const char *nm_status_string(int status);
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char *nm_last_cuda_error(void);
 
+/*
+ * Synchronises `stream`, then reads and clears the device status word.  Returns NM_ERR_TIMEOUT
+ * if a kernel gave up on a bounded wait (its output is then invalid), NM_OK otherwise.  Every
+ * device-side wait in this library (on an mbarrier fed by a TMA copy or a tensor-core commit) is
+ * limited to about a second, after which the kernel flags the error and runs to its end.
+ */
+int nm_check_status(nm_stream stream);
+
 /* ---- workspace --------------------------------------------------------------------------- */
 
 /*
@@ -128,11 +136,22 @@ int nm_matmul_host(const void *A_host, const void *B, void *C_host, void *A_stag
                    void *C_staging, int M, int N, int K, nm_dtype dtype, nm_layout layout_B,
                    void *workspace, size_t workspace_bytes, nm_stream stream);
 
+/*
+ * Programmatic dependent launch for nm_matmul / nm_matmul_batched (off by default).  When on,
+ * a product may start streaming its weights while the previous kernel in the stream is still
+ * running, and waits for that kernel only before it reads A or writes anything.  Turn it on only
+ * when B is not written by the work that precedes the call in the stream (resident weights).
+ */
+int nm_set_programmatic_launch(int enable);
+
 /* ---- tuning aids (sweeps and tests; not needed for normal use) --------------------------------- */
 
 /* Override the tiling heuristic: columns per CTA tile of the row-major kernel and number of
  * k-splits; 0 restores the heuristic.  Values are clamped to what the workspace bound covers. */
 int nm_debug_set_plan(int tile_n, int nsplit);
+/* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel instead
+ * of the TMA ring) and the ring depth in stages (0 heuristic). */
+int nm_debug_set_kernel(int kind, int stages);
 /* Report the plan for a problem: out[0..5] = kernel kind (0 row-major vector, 1 column-major
  * vector, 2 scalar), columns per tile, k-splits, k-rows per split, column tiles, CTAs. */
 int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B, int vec_ok,

@@ -57,6 +57,9 @@ _lib.nm_matmul_batched.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _l, _l, _l, _l
 _lib.nm_matmul_batched_ws.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _l, _l, _l, _l, _l, _i, _i, _vp, _sz, _vp]
 _lib.nm_matmul_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]
 _lib.nm_debug_set_plan.argtypes = [_i, _i]
+_lib.nm_debug_set_kernel.argtypes = [_i, _i]
+_lib.nm_set_programmatic_launch.argtypes = [_i]
+_lib.nm_check_status.argtypes = [_vp]
 _lib.nm_debug_get_plan.argtypes = [_i, _i, _i, _i, _i, _i, _i, C.POINTER(_i)]
 
 
@@ -142,6 +145,19 @@ def nm_matmul_host(A_host, B, C_host, A_staging, C_staging, M, N, K, dtype, layo
 
 def nm_debug_set_plan(tile_n: int = 0, nsplit: int = 0) -> None:
     _check(_lib.nm_debug_set_plan(tile_n, nsplit), "nm_debug_set_plan")
+
+
+def nm_debug_set_kernel(kind: int = -1, stages: int = 0) -> None:
+    _check(_lib.nm_debug_set_kernel(kind, stages), "nm_debug_set_kernel")
+
+
+def nm_set_programmatic_launch(enable: bool) -> None:
+    _check(_lib.nm_set_programmatic_launch(int(enable)), "nm_set_programmatic_launch")
+
+
+def nm_check_status(stream=None) -> None:
+    """Synchronise the stream and raise if a kernel gave up on a bounded wait."""
+    _check(_lib.nm_check_status(_stream(stream)), "nm_check_status")
 
 
 def nm_debug_get_plan(M, N, K, H=1, dtype=BF16, layout_B=ROW_MAJOR, vec_ok=True) -> dict:

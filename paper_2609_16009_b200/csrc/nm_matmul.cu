@@ -4,6 +4,7 @@
 #include <cstring>
 
 #include "nm_matmul_kernels.cuh"
+#include "nm_row_tma.cuh"
 
 namespace nm {
 
@@ -13,6 +14,12 @@ NM_EXTERN(row, float, float)
 NM_EXTERN(col, bf16_t, bf16_t)
 NM_EXTERN(col, bf16_t, float)
 NM_EXTERN(col, float, float)
+NM_EXTERN_TMA(8, bf16_t)
+NM_EXTERN_TMA(8, float)
+NM_EXTERN_TMA(16, bf16_t)
+NM_EXTERN_TMA(16, float)
+NM_EXTERN_TMA(32, bf16_t)
+NM_EXTERN_TMA(32, float)
 
 // ---- error bookkeeping ---------------------------------------------------------------------------
 static thread_local char g_cuda_error[256] = "";
@@ -26,13 +33,14 @@ int record_cuda_error(cudaError_t e, const char *where)
 // ---- default workspace and tuning overrides ----------------------------------------------------------
 static void *g_ws = nullptr;
 static size_t g_ws_bytes = 0;
-static int g_force_tn = 0, g_force_split = 0;
+static int g_force_tn = 0, g_force_split = 0, g_force_kind = -1, g_force_stages = 0;
+static int g_use_pdl = 0;
 
-enum PlanKind { kRowVec = 0, kColVec = 1, kGeneric = 2 };
+enum PlanKind { kRowVec = 0, kColVec = 1, kGeneric = 2, kRowTma = 3 };
 
 struct Plan {
     PlanKind kind;
-    int tn, tpr, rg, nsplit, kr, ntiles;
+    int tn, tpr, rg, nsplit, kr, ntiles, nstage;
 };
 
 static inline int elem_size(nm_dtype d) { return d == NM_F32 ? 4 : 2; }
@@ -43,7 +51,51 @@ static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t
 // (a) enough CTAs to cover all 148 SMs a few times over, (b) per-CTA segments of B as long and as
 // contiguous as the shape allows, (c) few enough splits that the partial-sum traffic stays a few
 // per cent of |B|.
-static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout, bool vec_ok)
+// Plan for the TMA-ring kernel.  Cost model, in units of one streamed weight element per CTA:
+// waves over the resident-CTA slots x (elements per CTA + a fixed per-CTA cost + the partial-sum
+// traffic a split adds).  The search is tiny (3 tile widths x 64 split counts).
+static Plan make_tma_plan(int M, int N, int K, int H)
+{
+    const int occ = (M <= 8) ? 2 : 1;       // resident CTAs per SM the plan aims for (measured best)
+    const long slots = (long)kSMs * occ;
+    Plan best{};
+    double best_cost = 1e300;
+    for (int tpr = 8; tpr <= 32; tpr *= 2) {
+        const int tn = tpr * 8;
+        if (g_force_tn > 0 && tn != g_force_tn) continue;
+        const int ntiles = ceil_div(N, tn);
+        if ((long)ntiles * H > kNumCounters && g_force_split > 1) continue;
+        for (int ns = 1; ns <= kMaxSplit; ++ns) {
+            if (g_force_split > 0 && ns != g_force_split) continue;
+            if (ns > 1 && (long)ntiles * H > kNumCounters) break;
+            int kr = ceil_div(ceil_div(K, ns), 8) * 8;
+            const int ns_eff = ceil_div(K, kr);
+            if (ns_eff != ns && g_force_split == 0) continue;       // duplicate of a smaller split count
+            const long ctas = (long)ntiles * ns_eff * H;
+            const long waves = (ctas + slots - 1) / slots;
+            const double per_cta = (double)kr * tn + 8192.0 + (ns_eff > 1 ? 4.0 * M * tn + 64.0 * ns_eff : 0.0);
+            const double cost = (double)waves * per_cta * (tn == 64 ? 1.0 : 1.001);
+            if (cost < best_cost) {
+                best_cost = cost;
+                best.kind = kRowTma; best.tn = tn; best.tpr = tpr; best.rg = kTmaConsumers / tpr;
+                best.nsplit = ns_eff; best.kr = kr; best.ntiles = ntiles;
+                // 16 KB stages; the ring takes what is left of ~200 KB per SM after the A chunk
+                int nstage = (M <= 2) ? 3 : (occ == 2) ? 5 : 10;
+                if (g_force_stages > 0) nstage = g_force_stages;
+                if (nstage < 2) nstage = 2;
+                if (nstage > 11) nstage = 11;
+                best.nstage = nstage;
+            }
+        }
+    }
+    if (best_cost == 1e300) {       // forced values matched nothing: fall back to one wide tile, no split
+        best.kind = kRowTma; best.tn = 64; best.tpr = 8; best.rg = 32; best.nsplit = 1; best.kr = ceil_div(K, 8) * 8;
+        best.ntiles = ceil_div(N, 64); best.nstage = 8;
+    }
+    return best;
+}
+
+static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout, bool vec_ok, bool tma_ok)
 {
     Plan p{};
     const int V = vec_elems(dtype);
@@ -52,6 +104,7 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
         p.tpr = p.rg = 0;
         return p;
     }
+    if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H);
     const int target = (M <= 4 ? 4 : 2) * kSMs;       // CTAs wanted in flight
     if (layout == NM_ROW_MAJOR) {
         p.kind = kRowVec;
@@ -90,6 +143,35 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     return p;
 }
 
+// Tensor maps of recently used weight matrices (encoding one costs about a microsecond of host time).
+struct MapKey { const void *B; int N, K, H; long strideB; int tn, kt; };
+struct MapEntry { MapKey key; CUtensorMap map; bool valid; };
+static thread_local MapEntry g_maps[16];
+static thread_local int g_map_next = 0;
+
+static const CUtensorMap *get_weight_map(const void *B, int N, int K, int H, long strideB, int tn, int kt)
+{
+    for (auto &e : g_maps) {
+        const MapKey &k = e.key;
+        if (e.valid && k.B == B && k.N == N && k.K == K && k.H == H && k.strideB == strideB && k.tn == tn && k.kt == kt)
+            return &e.map;
+    }
+    EncodeTiledFn enc = tensor_map_encoder();
+    if (!enc) return nullptr;
+    MapEntry &e = g_maps[g_map_next];
+    g_map_next = (g_map_next + 1) % 16;
+    e.key = MapKey{B, N, K, H, strideB, tn, kt};
+    const cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)K, (cuuint64_t)H};
+    const cuuint64_t strides[2] = {(cuuint64_t)N * 2, (cuuint64_t)(H > 1 ? strideB : (long)K * N) * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)tn, (cuuint32_t)kt, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(B), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    e.valid = (r == CUDA_SUCCESS);
+    return e.valid ? &e.map : nullptr;
+}
+
 static size_t partial_floats(const Plan &p, int M, int H)
 {
     return p.nsplit > 1 ? (size_t)H * p.ntiles * p.nsplit * M * p.tn : 0;
@@ -124,7 +206,10 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
                       (layout == NM_ROW_MAJOR ? (N % V == 0) : (K % V == 0));
     const bool a_ok = aligned16(A) && (lda % V == 0) && (strideA % V == 0);
     const bool vec_ok = b_ok && (layout == NM_ROW_MAJOR || a_ok);
-    Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok);
+    bool tma_ok = b_ok && a_ok && layout == NM_ROW_MAJOR && dtype != NM_F32 && tensor_map_encoder() != nullptr &&
+                  (long)N * 2 < (1L << 40) && strideB >= 0;
+    if (g_force_kind == kRowVec) tma_ok = false;
+    Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok);
 
     MatmulArgs a{};
     a.A = A; a.B = B; a.C = C;
@@ -141,7 +226,18 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     }
 
     cudaError_t e = cudaErrorInvalidValue;
-    if (p.kind == kGeneric) {
+    if (p.kind == kRowTma) {
+        const int kt = (kTmaConsumers / p.tpr) * 4;
+        const CUtensorMap *map = get_weight_map(B, N, K, H, strideB, p.tn, kt);
+        if (!map) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+        TmaArgs ta{};
+        ta.base = a; ta.nstage = p.nstage; ta.use_pdl = g_use_pdl; ta.status = device_status_ptr();
+        const size_t smem = (size_t)p.nstage * kt * p.tn * 2 + kAChunkFloats * sizeof(float) + 2 * p.nstage * sizeof(uint64_t);
+        const bool f32out = (dtype == NM_BF16_F32OUT);
+        if (p.tpr == 8)       e = f32out ? launch_row_tma<8, float>(*map, ta, smem, stream)  : launch_row_tma<8, bf16_t>(*map, ta, smem, stream);
+        else if (p.tpr == 16) e = f32out ? launch_row_tma<16, float>(*map, ta, smem, stream) : launch_row_tma<16, bf16_t>(*map, ta, smem, stream);
+        else                  e = f32out ? launch_row_tma<32, float>(*map, ta, smem, stream) : launch_row_tma<32, bf16_t>(*map, ta, smem, stream);
+    } else if (p.kind == kGeneric) {
         if (dtype == NM_F32)            e = launch_generic<float, float>(a, layout, stream);
         else if (dtype == NM_BF16)      e = launch_generic<bf16_t, bf16_t>(a, layout, stream);
         else                            e = launch_generic<bf16_t, float>(a, layout, stream);
@@ -268,11 +364,25 @@ int nm_debug_set_plan(int tile_n, int nsplit)
     return NM_OK;
 }
 
+/* Force the kernel family (-1 heuristic, 0 plain row-major kernel instead of the TMA ring) and the ring depth. */
+int nm_debug_set_kernel(int kind, int stages)
+{
+    g_force_kind = kind; g_force_stages = stages;
+    return NM_OK;
+}
+
+int nm_set_programmatic_launch(int enable)
+{
+    g_use_pdl = enable ? 1 : 0;
+    return NM_OK;
+}
+
 /* Reports the plan the library would use: out[0..5] = kind, tile_n, nsplit, k-rows per split, tiles, CTAs. */
 int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B, int vec_ok, int *out)
 {
     if (!out) return NM_ERR_INVALID_ARG;
-    Plan p = make_plan(M, N, K, H, dtype, layout_B, vec_ok != 0);
+    Plan p = make_plan(M, N, K, H, dtype, layout_B, vec_ok != 0,
+                       vec_ok != 0 && layout_B == NM_ROW_MAJOR && dtype != NM_F32 && g_force_kind != kRowVec);
     out[0] = p.kind; out[1] = p.tn; out[2] = p.nsplit; out[3] = p.kr; out[4] = p.ntiles;
     out[5] = p.ntiles * p.nsplit * H;
     return NM_OK;

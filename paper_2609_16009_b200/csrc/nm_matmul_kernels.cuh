@@ -59,10 +59,11 @@ __device__ __forceinline__ void splitk_complete(const MatmulArgs &a, int tile, i
     __threadfence();
     const float *P = a.partial + ((size_t)h * a.ntiles + tile) * a.nsplit * (size_t)(M * a.tn);
     TO *C = (TO *)a.C + (long)h * a.strideC;
-    for (int i = tid; i < M * a.tn; i += kThreads) {
+    for (int i = tid; i < M * a.tn; i += blockDim.x) {
         const int m = i / a.tn, c = i - m * a.tn, n = tile * a.tn + c;
         if (n < a.N) {
             float s = 0.f;
+#pragma unroll 4
             for (int sp = 0; sp < a.nsplit; ++sp) s += ld_cg(P + ((size_t)sp * M + m) * a.tn + c);
             C[(long)m * a.ldc + n] = round_out<TO>(s);
         }

@@ -21,6 +21,8 @@ def nm():
     nm.nm_set_workspace(ws)
     yield nm
     nm.nm_debug_set_plan(0, 0)
+    nm.nm_debug_set_kernel(-1, 0)
+    nm.nm_check_status()
     nm.nm_set_workspace(None)
 
 
@@ -110,17 +112,50 @@ def test_long_k_spans_several_shared_memory_chunks(nm, layout):
 
 # ---- split-K: forced plans, determinism -----------------------------------------------------------------
 
-@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("layout,kernel", [(ROW, -1), (ROW, 0), (COL, -1)])
 @pytest.mark.parametrize("nsplit", [1, 2, 7, 16, 64])
-@pytest.mark.parametrize("tile_n", [0, 64, 136, 512])
-def test_forced_plans_agree(nm, layout, nsplit, tile_n):
+@pytest.mark.parametrize("tile_n", [0, 64, 128, 136, 256, 512])
+def test_forced_plans_agree(nm, layout, kernel, nsplit, tile_n):
+    # kernel -1: the library's choice (TMA ring for row-major bf16); 0: the plain-load kernel
     M, K, N = 3, 7168, 576
     A, B = gen.narrow_bf16(M, K, N, seed=600)
     nm.nm_debug_set_plan(tile_n, nsplit)
+    nm.nm_debug_set_kernel(kernel, 0)
     try:
-        run_case(nm, A, B, M, N, K, BF16, layout, f"forced tile_n={tile_n} nsplit={nsplit} layout={layout}")
+        run_case(nm, A, B, M, N, K, BF16, layout, f"forced tile_n={tile_n} nsplit={nsplit} layout={layout} kernel={kernel}")
     finally:
         nm.nm_debug_set_plan(0, 0)
+        nm.nm_debug_set_kernel(-1, 0)
+
+
+@pytest.mark.parametrize("M", list(range(1, 17)))
+@pytest.mark.parametrize("tile_n", [64, 128, 256])
+def test_tma_ring_every_m_and_tile(nm, M, tile_n):
+    # K spans several A chunks (256 rows at M=16) and ends mid-stage; N ends mid-tile
+    K, N = 1000, 840
+    A, B = gen.narrow_bf16(M, K, N, seed=900 + M)
+    for stages in (2, 0):
+        nm.nm_debug_set_plan(tile_n, 2)
+        nm.nm_debug_set_kernel(-1, stages)
+        try:
+            assert nm.nm_debug_get_plan(M, N, K)["kind"] == 3
+            run_case(nm, A, B, M, N, K, BF16, ROW, f"tma M={M} tile_n={tile_n} stages={stages}")
+        finally:
+            nm.nm_debug_set_plan(0, 0)
+            nm.nm_debug_set_kernel(-1, 0)
+    nm.nm_check_status()
+
+
+def test_plain_row_kernel_every_m(nm):
+    K, N = 1000, 840
+    nm.nm_debug_set_kernel(0, 0)
+    try:
+        for M in range(1, 17):
+            A, B = gen.narrow_bf16(M, K, N, seed=950 + M)
+            assert nm.nm_debug_get_plan(M, N, K)["kind"] == 0
+            run_case(nm, A, B, M, N, K, BF16, ROW, f"plain row kernel M={M}")
+    finally:
+        nm.nm_debug_set_kernel(-1, 0)
 
 
 @pytest.mark.parametrize("layout", [ROW, COL])

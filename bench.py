@@ -1,0 +1,330 @@
+#!/usr/bin/env python
+"""Benchmark of the narrow-MatMul / MLA-decode hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mla|projections] [--seq-len S]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores (reported baseline)
+
+One step is one pass of the whole hot path over one token.  Prints ONE JSON line (rank 0).
+`value` is the algorithmic HBM traffic of a step (weights + activations + KV rows, each once)
+divided by the device time of the step, summed over ranks: GB/s.  `ms_per_step` is the decode
+latency.  Every rank runs an independent replica (the path has no exchange step): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+import nm_inputs as gen  # noqa: E402
+
+DIMS = gen.DSV3_DIMS
+L2_BYTES = 126 * 1024 * 1024
+
+
+# --------------------------------------------------------------------------------------------------
+# workloads
+# --------------------------------------------------------------------------------------------------
+def projection_specs(dims=DIMS):
+    """The narrow products of one decode step at M = 1: (name, K, N, heads)."""
+    d, ql, dc, dr, dn, dv, H = (dims[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
+    return [("W_DQ", d, ql, 1), ("W_DKVKR", d, dc + dr, 1), ("W_UQR", ql, H * (dn + dr), 1),
+            ("W_UK", dn, dc, H), ("W_UV", dc, dv, H), ("W_O", H * dv, d, 1)]
+
+
+def algorithmic_bytes(specs, M=1):
+    return sum((K * N + M * K + M * N) * 2 * H for _, K, N, H in specs)
+
+
+class ProjectionChain:
+    """All narrow products of the decode step, M = 1, each fed a resident activation vector."""
+
+    name = "projections"
+
+    def __init__(self, nm, device, seed=4000):
+        self.nm = nm
+        self.specs = projection_specs()
+        w = gen.mla_weights(DIMS, seed=seed, with_wo=True)
+        self.W = {k: torch.from_numpy(w[k].view(np.int16)).to(device) for k in ("W_DQ", "W_DKVKR", "W_UQR", "W_UK", "W_UV", "W_O")}
+        self.h_host = torch.from_numpy(gen.mla_token(DIMS, seed=seed + 100).view(np.int16).copy()).pin_memory()
+        self.x = {}
+        self.y = {}
+        for name, K, N, H in self.specs:
+            self.x[name] = torch.from_numpy(gen.normal_bf16((H * K,), 1.0, seed + 200 + len(self.x)).view(np.int16)).to(device)
+            self.y[name] = torch.empty(H * N, dtype=torch.int16, device=device)
+        self.out_host = torch.empty(DIMS["d"], dtype=torch.int16).pin_memory()
+        need = max(nm.nm_matmul_workspace_bytes(1, N, K, H) for _, K, N, H in self.specs)
+        self.ws = nm.new_workspace(need, device=device)
+        self.bytes_per_step = algorithmic_bytes(self.specs)
+        self.dominant = "W_O"
+        self.dominant_bytes = algorithmic_bytes([s for s in self.specs if s[0] == "W_O"])
+        self.launches_per_step = len(self.specs)
+        self.h2d = self.h_host.numel() * 2
+        self.d2h = self.out_host.numel() * 2
+
+    def describe(self):
+        return {"workload": "narrow products of one DeepSeek-V3 MLA decode step, M=1 (W_DQ 7168x1536, W_DKV|KR 7168x576, "
+                            "W_UQR 1536x24576, W_UK/W_UV per head x128, W_O 16384x7168), bf16 row-major",
+                "l2": "weights 374 MB per step > 126 MB L2, so every step streams from HBM; no flush"}
+
+    def launch(self, name, stream):
+        nm = self.nm
+        _, K, N, H = next(s for s in self.specs if s[0] == name)
+        if H == 1:
+            nm.nm_matmul_ws(self.x[name], self.W[name], self.y[name], 1, N, K, nm.BF16, nm.ROW_MAJOR, self.ws, stream)
+        else:
+            nm.nm_matmul_batched_ws(self.x[name], self.W[name], self.y[name], 1, N, K, H, H * K, K, K * N, H * N, N,
+                                    nm.BF16, nm.ROW_MAJOR, self.ws, stream)
+
+    def step(self, stream, dom_events=None):
+        for name, _, _, _ in self.specs:
+            if dom_events is not None and name == self.dominant:
+                dom_events[0].record(stream)
+                self.launch(name, stream)
+                dom_events[1].record(stream)
+            else:
+                self.launch(name, stream)
+
+    def step_e2e(self, stream):
+        # token in from pinned host memory, result out to pinned host memory, inside the timed region
+        self.x["W_DQ"].copy_(self.h_host, non_blocking=True)
+        self.step(stream)
+        self.out_host.copy_(self.y["W_O"], non_blocking=True)
+
+
+def make_workload(kind, nm, device, seq_len):
+    if kind == "projections":
+        return ProjectionChain(nm, device)
+    raise SystemExit(f"unknown workload {kind}")
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7), ("sw_power_cap", 8)):
+                if r[col].lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU oracle arm
+# --------------------------------------------------------------------------------------------------
+_ORACLE_INPUTS = None
+
+
+def oracle_sample(threads):
+    """One pass of the oracle, as it stands, over the narrow products of the step (all six weight
+    matrices, M = 1) on the host cores.  Returns (seconds, algorithmic bytes, description)."""
+    import oracle
+    global _ORACLE_INPUTS
+    specs = projection_specs()
+    if _ORACLE_INPUTS is None:
+        w = gen.mla_weights(DIMS, seed=4000, with_wo=True)
+        x = {name: gen.normal_bf16((H * K,), 1.0, 4200 + i) for i, (name, K, N, H) in enumerate(specs)}
+        oracle.lib()
+        _ORACLE_INPUTS = (w, x)
+    w, x = _ORACLE_INPUTS
+    t0 = time.perf_counter()
+    for name, K, N, H in specs:
+        if H == 1:
+            oracle.matmul(x[name], w[name], 1, N, K, oracle.BF16, oracle.BF16, oracle.ROW_MAJOR, threads=threads)
+        else:
+            oracle.matmul_batched(x[name], w[name], 1, N, K, H, H * K, K, K * N, H * N, N, H * N,
+                                  oracle.BF16, oracle.BF16, oracle.ROW_MAJOR, threads=threads)
+    dt = time.perf_counter() - t0
+    return dt, algorithmic_bytes(specs), "all six narrow products of one decode step at M=1 (374 MB of bf16 weights), one pass"
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    import oracle
+    threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+    for _ in range(args.warmup):
+        oracle_sample(threads)
+    times, nbytes, what = [], 0, ""
+    for _ in range(args.steps):
+        dt, nbytes, what = oracle_sample(threads)
+        times.append(dt)
+    total = sum(times)
+    value = nbytes * len(times) / total / 1e9
+    line = {"impl": "reference", "metric": "narrow MatMul HBM GB/s", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / len(times) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "CPU oracle (fp64 triple loop) on a bounded sample: " + what},
+            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": what},
+            "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------------
+# main arm
+# --------------------------------------------------------------------------------------------------
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="projections")
+    ap.add_argument("--seq-len", type=int, default=4096)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    import paper_2609_16009_b200 as nm
+    wl = make_workload(args.workload, nm, device, args.seq_len)
+    stream = torch.cuda.Stream(device)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            wl.step(stream)
+        barrier()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        # ---- device-timed region: exactly `steps` steps, inputs resident in HBM ------------------------
+        dom = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(args.steps):
+            wl.step(stream, dom[i])
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        dom_ms = statistics.mean(a.elapsed_time(b) for a, b in dom)
+        # ---- end-to-end region: host token in, host result out, every step -----------------------------
+        for _ in range(3):
+            wl.step_e2e(stream)
+        barrier()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(args.steps):
+            wl.step_e2e(stream)
+            stream.synchronize()              # the host reads the result of every step
+        t1.record(stream)
+        barrier()
+        e2e_ms = t0.elapsed_time(t1)
+        clocks = sampler.stop()
+    nm.nm_check_status(stream)
+
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms, dom_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms, dom_ms = t.tolist()
+
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        total_bytes = wl.bytes_per_step * args.steps * world
+        value = total_bytes / (ms * 1e-3) / 1e9
+        e2e_value = total_bytes / (e2e_ms * 1e-3) / 1e9
+        achieved = wl.dominant_bytes / (dom_ms * 1e-3) / 1e9
+        line = {"metric": "narrow MatMul HBM GB/s", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": wl.describe(),
+                "pct_of_8TBs": value / world / 8000.0,
+                "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h,
+                        "ms_per_step": e2e_ms / args.steps},
+                "gpu_launches": wl.launches_per_step * args.steps,
+                "clocks": clocks,
+                "roofline": {"bound": "hbm", "kernel": wl.dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                             "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                             "us_per_launch": dom_ms * 1e3}}
+        if not args.no_cpu_baseline:
+            import oracle
+            threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+            oracle_sample(threads)
+            dt, nbytes, what = oracle_sample(threads)
+            line["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+                                    "sample": what, "seconds": dt}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

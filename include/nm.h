@@ -46,7 +46,8 @@ enum {
     NM_ERR_ALIGNMENT = -3,        /* a pointer is not aligned to its element size */
     NM_ERR_WORKSPACE = -4,        /* workspace missing or too small */
     NM_ERR_CUDA = -5,             /* a CUDA call failed; see nm_last_cuda_error() */
-    NM_ERR_TIMEOUT = -6           /* a bounded device-side wait expired (nm_check_status) */
+    NM_ERR_TIMEOUT = -6,          /* a bounded device-side wait expired (nm_check_status) */
+    NM_ERR_TOO_LARGE = -7         /* problem needs more scratch than nm_matmul_static has built in */
 };
 
 #define NM_MAX_M 16
@@ -135,6 +136,32 @@ int nm_matmul_batched_ws(const void *A, const void *B, void *C, int M, int N, in
 int nm_matmul_host(const void *A_host, const void *B, void *C_host, void *A_staging,
                    void *C_staging, int M, int N, int K, nm_dtype dtype, nm_layout layout_B,
                    void *workspace, size_t workspace_bytes, nm_stream stream);
+
+/*
+ * The same product for callers that must not allocate.  (The paper has no counterpart: this is
+ * an addition for embedding the library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits or cannot succeed - a plugin inside
+ * a serving runtime whose memory pool was sized up front and has claimed the whole GPU, a latency
+ * critical loop that may not take the device-wide synchronisation an allocation implies, or a
+ * host that simply has no allocator to lend (a thin C program that only maps its inputs and
+ * outputs).  Such a caller passes A, B and C as usual and nothing else: the split-K partial sums
+ * and arrival counters go into a fixed NM_STATIC_SCRATCH_BYTES array that is part of the library's
+ * device image (every GPU that loads the library holds it until the process exits).  The call
+ * itself uses no cudaMalloc, cudaFree or any other allocating routine.
+ *
+ * Limits and rules:
+ *  - a problem whose tiling needs more scratch than the array holds is refused with
+ *    NM_ERR_TOO_LARGE and nothing is enqueued (the products of the MLA decode step at M <= 16 fit);
+ *  - the first call on each device looks up the array's device address and enqueues one 64 KB
+ *    memset of the counters on `stream`; make that first call before starting any stream capture;
+ *  - all calls on a GPU share the one array, which keeps whatever the last call left in it; the
+ *    kernels restore the counters themselves, but two calls that overlap on the GPU (different
+ *    streams, or programmatic launch) race on the partial sums - issue them on one stream.
+ */
+#define NM_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+int nm_matmul_static(const void *A, const void *B, void *C, int M, int N, int K,
+                     nm_dtype dtype, nm_layout layout_B, nm_stream stream);
 
 /*
  * Programmatic dependent launch for nm_matmul / nm_matmul_batched (off by default).  When on,

@@ -56,6 +56,7 @@ _lib.nm_matmul_ws.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]
 _lib.nm_matmul_batched.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _l, _l, _l, _l, _l, _i, _i, _vp]
 _lib.nm_matmul_batched_ws.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _l, _l, _l, _l, _l, _i, _i, _vp, _sz, _vp]
 _lib.nm_matmul_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _sz, _vp]
+_lib.nm_matmul_static.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]
 _lib.nm_debug_set_plan.argtypes = [_i, _i]
 _lib.nm_debug_set_kernel.argtypes = [_i, _i]
 _lib.nm_set_programmatic_launch.argtypes = [_i]
@@ -141,6 +142,17 @@ def nm_matmul_host(A_host, B, C_host, A_staging, C_staging, M, N, K, dtype, layo
     _check(_lib.nm_matmul_host(_ptr(A_host), _ptr(B), _ptr(C_host), _ptr(A_staging), _ptr(C_staging),
                                M, N, K, dtype, layout_B, _ptr(workspace), nbytes, _stream(stream)),
            "nm_matmul_host")
+
+
+STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
+
+
+def nm_matmul_static(A, B, C_out, M, N, K, dtype, layout_B, stream=None) -> None:
+    """nm_matmul without any workspace: the scratch is a fixed array inside the library, for
+    callers that cannot allocate.  Calls on one GPU must not overlap; the first call on a device
+    should come before any stream capture."""
+    _check(_lib.nm_matmul_static(_ptr(A), _ptr(B), _ptr(C_out), M, N, K, dtype, layout_B, _stream(stream)),
+           "nm_matmul_static")
 
 
 def nm_debug_set_plan(tile_n: int = 0, nsplit: int = 0) -> None:

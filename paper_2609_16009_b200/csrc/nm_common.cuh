@@ -72,6 +72,12 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p) {
 // Load that bypasses L1 (data written by other SMs in the same launch).
 __device__ __forceinline__ float ld_cg(const float *p) { return __ldcg(p); }
 
+// Validates, plans and enqueues one (batched) narrow product; `ws` may be null when the plan does
+// not split K.  Defined in nm_matmul.cu.
+int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, int H,
+                   long lda, long strideA, long strideB, long ldc, long strideC,
+                   nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream);
+
 __host__ __device__ constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 }  // namespace nm

@@ -281,6 +281,7 @@ const char *nm_status_string(int status)
     case NM_ERR_WORKSPACE: return "workspace missing or too small";
     case NM_ERR_CUDA: return "CUDA error";
     case NM_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case NM_ERR_TOO_LARGE: return "problem too large for the built-in scratch of nm_matmul_static";
     default: return "unknown status";
     }
 }

@@ -77,9 +77,10 @@ int nm_check_status(nm_stream stream);
 size_t nm_matmul_workspace_bytes(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B);
 
 /*
- * Clear the arrival counters at the start of a workspace (enqueues one memset on `stream`).
- * Must be done once before first use; the kernels leave the counters at zero afterwards, so
- * no clearing is needed between calls.  `bytes` must be at least NM_WS_COUNTER_BYTES.
+ * Clear a workspace (enqueues one memset of `bytes` on `stream`); what matters are the arrival
+ * counters in it.  Must be done once before first use; the kernels leave the counters at zero
+ * afterwards, so no clearing is needed between calls.  `bytes` must be at least
+ * NM_WS_COUNTER_BYTES.
  */
 #define NM_WS_COUNTER_BYTES 65536
 int nm_workspace_init(void *workspace, size_t bytes, nm_stream stream);
@@ -163,6 +164,85 @@ int nm_matmul_host(const void *A_host, const void *B, void *C_host, void *A_stag
 int nm_matmul_static(const void *A, const void *B, void *C, int M, int N, int K,
                      nm_dtype dtype, nm_layout layout_B, nm_stream stream);
 
+/* ---- single-token MLA decode step ------------------------------------------------------------------ */
+
+/*
+ * Vector-side stages that consume the narrow products (MLA Operator Optimization section: "RMS,
+ * RoPE and caching normalization" start right after MatMul 2).  All tensors bf16.
+ *   nm_rmsnorm:  y[i] = x[i] * rsqrt(mean(x^2) + eps) * gamma[i],  i < n  (n <= 16384), rounded to bf16
+ *   nm_rope:     n_vec vectors of `dim` elements (vector v at x + v*x_stride, written to
+ *                y + v*y_stride, strides in elements); interleaved pairs (x[2i], x[2i+1]) turn by the
+ *                angle whose (cos, sin) is cos_sin[2i], cos_sin[2i+1] (fp32, one table row)
+ *   nm_rope_table: fills table[(p - pos_begin)*dim + 2i + {0,1}] = (cos, sin)(p * base^(-2i/dim))
+ *                for pos_begin <= p < pos_begin + n_pos, computed in fp64 on the device
+ */
+int nm_rmsnorm(const void *x, const void *gamma, void *y, int n, float eps, nm_stream stream);
+int nm_rope(const void *x, void *y, int n_vec, int dim, long x_stride, long y_stride,
+            const float *cos_sin, nm_stream stream);
+int nm_rope_table(float *table, long pos_begin, int n_pos, int dim, double base, nm_stream stream);
+
+/*
+ * Absorbed latent attention for all heads of one token over cache rows [0, n_rows):
+ *   s[h,j] = scale * <Q[h,:], cache[j,:]>,  p = softmax_j(s),  o[h,:] = sum_j p[h,j] * cache[j,:kv_lora]
+ * Q is [H][kv_lora+rope] bf16 (per head q_lat | q_rope), cache is [>= n_rows][kv_lora+rope] bf16.
+ * If `extra_row` >= 0 that cache row is attended as well (the row the step has just written; it is
+ * merged in the combine so that the pass over the old rows need not wait for it).  Outputs:
+ * o_bf16 [H][kv_lora] (may be NULL) and o_f32 [H][kv_lora] unrounded (may be NULL).
+ * Supported: H = 128, kv_lora = 512, rope = 64 on the tensor-core path.  Workspace: see
+ * nm_mla_attention_workspace_bytes.  The pass over the rows is a tcgen05 kernel split over the
+ * sequence; a second kernel merges the splits with their log-sum-exp weights.
+ */
+size_t nm_mla_attention_workspace_bytes(int H, int n_rows, int kv_lora);
+int nm_mla_attention(const void *Q, const void *kv_cache, void *o_bf16, float *o_f32, int H,
+                     int n_rows, long extra_row, int kv_lora, int rope, float scale,
+                     void *workspace, size_t workspace_bytes, nm_stream stream);
+/* Two-phase form used by the decode step: the split pass, then the merge. */
+int nm_mla_attention_partial(const void *Q, const void *kv_cache, int H, int n_rows, int kv_lora,
+                             int rope, float scale, void *workspace, size_t workspace_bytes,
+                             nm_stream stream);
+int nm_mla_attention_combine(const void *Q, const void *kv_cache, void *o_bf16, float *o_f32, int H,
+                             int n_rows, long extra_row, int kv_lora, int rope, float scale,
+                             void *workspace, size_t workspace_bytes, nm_stream stream);
+
+/*
+ * One decode step for one token (DeepSeek-V3-style MLA, absorbed form).  Stages, each rounded to
+ * bf16 as the paper rounds MatMul 2's output before RoPE / RMSNorm (Algorithm 2, output cast):
+ *   c_q = h*W_DQ; c_qn = RMSNorm(c_q; gamma_q); q = c_qn*W_UQR ([H][nope+rope]);
+ *   q_rope = RoPE(q[:, nope:], pos); q_lat[h] = q[h,:nope]*W_UK[h];
+ *   ckr = h*(W_DKV|W_KR) (Eq. 3); cache[pos] = [RMSNorm(ckr[:kv_lora]; gamma_kv) | RoPE(ckr[kv_lora:], pos)];
+ *   o_lat = attention([q_lat|q_rope], cache[0..seq_len)); o[h] = o_lat[h]*W_UV[h]; out = flatten(o)*W_O.
+ * pos = seq_len - 1: seq_len counts the rows attended including the one this step writes.
+ * Dense weights are K x N in `layout_dense`; W_UK is [H][nope][kv_lora], W_UV is [H][kv_lora][v],
+ * row-major.  W_O may be NULL (the step then ends at o).  rope_cos_sin points at the table row for
+ * pos (`rope` floats).  The narrow products of the KV chain run on `side` concurrently with the
+ * tensor-core attention pass over the old rows on `main` (Data Independence condition); pass
+ * side == main for a serial schedule.  Optional outputs (device, may be NULL) receive every
+ * intermediate for stage-wise checking.  Workspace: nm_mla_workspace_bytes, counters cleared once
+ * with nm_workspace_init.
+ */
+typedef struct {
+    int d, q_lora, kv_lora, rope, nope, v, H;
+    int seq_len;
+    int layout_dense;              /* nm_layout of W_DQ, W_UQR, W_DKVKR, W_O */
+    float rms_eps, softmax_scale;
+    const void *h, *W_DQ, *gamma_q, *W_UQR, *W_DKVKR, *gamma_kv, *W_UK, *W_UV, *W_O;
+    const float *rope_cos_sin;
+    void *kv_cache;                /* [>= seq_len][kv_lora+rope] bf16; row seq_len-1 is written */
+    void *out;                     /* [d] bf16 (ignored when W_O is NULL) */
+    void *workspace;
+    size_t workspace_bytes;
+    /* optional intermediates, bf16 unless noted */
+    void *c_q, *c_qn, *q, *q_full /* [H][kv_lora+rope] = q_lat | q_rope */, *ckr, *o_lat, *o;
+    float *o_lat_f32;
+} nm_mla_params;
+
+size_t nm_mla_workspace_bytes(const nm_mla_params *p);
+int nm_mla_decode_step(const nm_mla_params *p, nm_stream main_stream, nm_stream side_stream);
+/* The same step with the token and the result in HOST memory (pinned): copies h in and out back
+ * on main_stream around the step.  h_staging / out_staging are device buffers of d bf16 each. */
+int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *out_host,
+                            void *h_staging, void *out_staging, nm_stream main_stream, nm_stream side_stream);
+
 /*
  * Programmatic dependent launch for nm_matmul / nm_matmul_batched (off by default).  When on,
  * a product may start streaming its weights while the previous kernel in the stream is still
@@ -179,6 +259,8 @@ int nm_debug_set_plan(int tile_n, int nsplit);
 /* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel instead
  * of the TMA ring) and the ring depth in stages (0 heuristic). */
 int nm_debug_set_kernel(int kind, int stages);
+/* Attention pass: 0 tensor-core kernel when the shape allows (default), 1 CUDA-core kernel. */
+int nm_debug_set_attention(int impl);
 /* Report the plan for a problem: out[0..5] = kernel kind (0 row-major vector, 1 column-major
  * vector, 2 scalar), columns per tile, k-splits, k-rows per split, column tiles, CTAs. */
 int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B, int vec_ok,

@@ -64,6 +64,31 @@ _lib.nm_check_status.argtypes = [_vp]
 _lib.nm_debug_get_plan.argtypes = [_i, _i, _i, _i, _i, _i, _i, C.POINTER(_i)]
 
 
+class MlaParams(C.Structure):
+    """Mirror of nm_mla_params (include/nm.h)."""
+    _fields_ = ([(n, _i) for n in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H", "seq_len", "layout_dense")]
+                + [("rms_eps", C.c_float), ("softmax_scale", C.c_float)]
+                + [(n, _vp) for n in ("h", "W_DQ", "gamma_q", "W_UQR", "W_DKVKR", "gamma_kv", "W_UK", "W_UV", "W_O",
+                                      "rope_cos_sin", "kv_cache", "out", "workspace")]
+                + [("workspace_bytes", _sz)]
+                + [(n, _vp) for n in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o", "o_lat_f32")])
+
+
+_lib.nm_rmsnorm.argtypes = [_vp, _vp, _vp, _i, C.c_float, _vp]
+_lib.nm_rope.argtypes = [_vp, _vp, _i, _i, _l, _l, _vp, _vp]
+_lib.nm_rope_table.argtypes = [_vp, _l, _i, _i, C.c_double, _vp]
+_lib.nm_mla_attention_workspace_bytes.restype = _sz
+_lib.nm_mla_attention_workspace_bytes.argtypes = [_i, _i, _i]
+_lib.nm_mla_attention.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _l, _i, _i, C.c_float, _vp, _sz, _vp]
+_lib.nm_mla_attention_partial.argtypes = [_vp, _vp, _i, _i, _i, _i, C.c_float, _vp, _sz, _vp]
+_lib.nm_mla_attention_combine.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _l, _i, _i, C.c_float, _vp, _sz, _vp]
+_lib.nm_mla_workspace_bytes.restype = _sz
+_lib.nm_mla_workspace_bytes.argtypes = [C.POINTER(MlaParams)]
+_lib.nm_mla_decode_step.argtypes = [C.POINTER(MlaParams), _vp, _vp]
+_lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.nm_debug_set_attention.argtypes = [_i]
+
+
 def _check(status: int, where: str) -> None:
     if status != 0:
         raise NmError(status, where)
@@ -183,3 +208,81 @@ def new_workspace(nbytes: int, device="cuda", stream=None) -> torch.Tensor:
     ws = torch.empty(max(int(nbytes), WS_COUNTER_BYTES), dtype=torch.uint8, device=device)
     nm_workspace_init(ws, stream)
     return ws
+
+
+# ---- MLA decode step -----------------------------------------------------------------------------------
+
+def nm_rmsnorm(x, gamma, y, n, eps, stream=None) -> None:
+    _check(_lib.nm_rmsnorm(_ptr(x), _ptr(gamma), _ptr(y), n, eps, _stream(stream)), "nm_rmsnorm")
+
+
+def nm_rope(x, y, n_vec, dim, x_stride, y_stride, cos_sin, stream=None) -> None:
+    _check(_lib.nm_rope(_ptr(x), _ptr(y), n_vec, dim, x_stride, y_stride, _ptr(cos_sin), _stream(stream)), "nm_rope")
+
+
+def nm_rope_table(table, pos_begin, n_pos, dim, base=10000.0, stream=None) -> None:
+    _check(_lib.nm_rope_table(_ptr(table), pos_begin, n_pos, dim, base, _stream(stream)), "nm_rope_table")
+
+
+def nm_mla_attention_workspace_bytes(H, n_rows, kv_lora) -> int:
+    return int(_lib.nm_mla_attention_workspace_bytes(H, n_rows, kv_lora))
+
+
+def nm_mla_attention(Q, kv_cache, o_bf16, o_f32, H, n_rows, extra_row, kv_lora, rope, scale, workspace, stream=None) -> None:
+    _check(_lib.nm_mla_attention(_ptr(Q), _ptr(kv_cache), _ptr(o_bf16), _ptr(o_f32), H, n_rows, extra_row, kv_lora, rope,
+                                 scale, _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "nm_mla_attention")
+
+
+def nm_mla_attention_partial(Q, kv_cache, H, n_rows, kv_lora, rope, scale, workspace, stream=None) -> None:
+    _check(_lib.nm_mla_attention_partial(_ptr(Q), _ptr(kv_cache), H, n_rows, kv_lora, rope, scale, _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)),
+           "nm_mla_attention_partial")
+
+
+def nm_mla_attention_combine(Q, kv_cache, o_bf16, o_f32, H, n_rows, extra_row, kv_lora, rope, scale, workspace,
+                             stream=None) -> None:
+    _check(_lib.nm_mla_attention_combine(_ptr(Q), _ptr(kv_cache), _ptr(o_bf16), _ptr(o_f32), H, n_rows, extra_row, kv_lora,
+                                         rope, scale, _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                         _stream(stream)), "nm_mla_attention_combine")
+
+
+def mla_params(dims: dict, seq_len: int, tensors: dict, rms_eps=1e-6, softmax_scale=None, layout_dense=ROW_MAJOR,
+               workspace=None) -> MlaParams:
+    """Fill an nm_mla_params from a dict of device tensors (keys as the struct's pointer fields;
+    missing optional ones stay NULL)."""
+    p = MlaParams()
+    for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"):
+        setattr(p, k, int(dims[k]))
+    p.seq_len, p.layout_dense = int(seq_len), int(layout_dense)
+    p.rms_eps = float(rms_eps)
+    p.softmax_scale = float(softmax_scale if softmax_scale is not None else (dims["nope"] + dims["rope"]) ** -0.5)
+    for name, _t in MlaParams._fields_:
+        if _t is _vp and name in tensors and tensors[name] is not None:
+            setattr(p, name, _ptr(tensors[name]))
+    if workspace is not None:
+        p.workspace = _ptr(workspace)
+        p.workspace_bytes = workspace.numel() * workspace.element_size()
+    return p
+
+
+def nm_mla_workspace_bytes(p: MlaParams) -> int:
+    return int(_lib.nm_mla_workspace_bytes(C.byref(p)))
+
+
+def nm_mla_decode_step(p: MlaParams, main_stream=None, side_stream=None) -> None:
+    ms = _stream(main_stream)
+    ss = ms if side_stream is None else _stream(side_stream)
+    _check(_lib.nm_mla_decode_step(C.byref(p), ms, ss), "nm_mla_decode_step")
+
+
+def nm_mla_decode_step_host(p: MlaParams, h_host, out_host, h_staging, out_staging, main_stream=None,
+                            side_stream=None) -> None:
+    ms = _stream(main_stream)
+    ss = ms if side_stream is None else _stream(side_stream)
+    _check(_lib.nm_mla_decode_step_host(C.byref(p), _ptr(h_host), _ptr(out_host), _ptr(h_staging), _ptr(out_staging),
+                                        ms, ss), "nm_mla_decode_step_host")
+
+
+def nm_debug_set_attention(impl: int) -> None:
+    _check(_lib.nm_debug_set_attention(impl), "nm_debug_set_attention")

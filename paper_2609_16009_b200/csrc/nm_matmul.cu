@@ -301,7 +301,7 @@ size_t nm_matmul_workspace_bytes(int M, int N, int K, int H, nm_dtype dtype, nm_
 int nm_workspace_init(void *workspace, size_t bytes, nm_stream stream)
 {
     if (!workspace || bytes < kCounterBytes) return NM_ERR_WORKSPACE;
-    NM_CUDA_TRY(cudaMemsetAsync(workspace, 0, kCounterBytes, (cudaStream_t)stream));
+    NM_CUDA_TRY(cudaMemsetAsync(workspace, 0, bytes, (cudaStream_t)stream));
     return NM_OK;
 }
 

@@ -1,0 +1,305 @@
+"""Parity of the MLA decode step with the CPU oracle: every stage in isolation (fed the oracle's
+bf16 stage inputs) and the whole step end to end."""
+import numpy as np
+import pytest
+import torch
+
+import nm_inputs as gen
+import oracle
+from gpu_util import assert_matmul_close, out_to_f64, to_dev
+
+pytestmark = pytest.mark.gpu
+
+DIMS = gen.DSV3_DIMS
+BF16, ROW = 1, 0
+
+
+def f64(bits):
+    return oracle.bf16_to_f64(np.asarray(bits, dtype=np.uint16))
+
+
+def dev_bits_to_f64(t):
+    return oracle.bf16_to_f64(t.cpu().numpy().view(np.uint16))
+
+
+def rel_max(got, ref):
+    return float(np.abs(got - ref).max() / np.abs(ref).max())
+
+
+@pytest.fixture(scope="module")
+def nm():
+    import paper_2609_16009_b200 as nm
+    yield nm
+    nm.nm_debug_set_attention(0)
+    nm.nm_check_status()
+
+
+@pytest.fixture(scope="module")
+def weights():
+    w = gen.mla_weights(DIMS, seed=4000, with_wo=True)
+    dw = {k: to_dev(v) for k, v in w.items()}
+    return w, dw
+
+
+def oracle_step(w, S, seed=4200, with_wo=True):
+    h = gen.mla_token(DIMS, seed=4100)
+    cache = gen.mla_cache(S, DIMS, seed=seed)
+    ww = dict(w)
+    if not with_wo:
+        ww.pop("W_O", None)
+    r = oracle.mla_decode_step(DIMS, ww, h, cache, S, threads=8)
+    return h, cache, r
+
+
+@pytest.fixture(scope="module")
+def ref1024(weights):
+    w, _ = weights
+    return oracle_step(w, 1024)
+
+
+def rope_row(nm, pos):
+    table = torch.empty(DIMS["rope"], dtype=torch.float32, device="cuda")
+    nm.nm_rope_table(table, pos, 1, DIMS["rope"])
+    return table
+
+
+# ---- vector-side stages ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("pos", [0, 1, 1023, 16383, 1000003])
+def test_rope_table_matches_oracle_angles(nm, pos):
+    dim = DIMS["rope"]
+    table = rope_row(nm, pos).cpu().numpy().astype(np.float64)
+    # the oracle's rotation of unit vectors (1,0) gives (cos, sin) of every pair
+    e = np.zeros(dim); e[0::2] = 1.0
+    cs = oracle.rope(e, pos)
+    assert np.abs(table - cs).max() <= 2.0 ** -23         # fp32 rounding of values in [-1, 1]
+
+
+def test_rmsnorm_stage(nm, ref1024, weights):
+    w, dw = weights
+    _, _, r = ref1024
+    y = torch.zeros(DIMS["q_lora"], dtype=torch.int16, device="cuda")
+    nm.nm_rmsnorm(to_dev(r["c_q"]), dw["gamma_q"], y, DIMS["q_lora"], 1e-6)
+    torch.cuda.synchronize()
+    got, ref = dev_bits_to_f64(y), f64(r["c_qn"])
+    assert np.all(np.abs(got - ref) <= 1e-5 * np.abs(ref) + oracle.ulp_bf16(ref))
+    assert np.mean(got == ref) > 0.99                      # a rounding flip is rare
+
+
+@pytest.mark.parametrize("n", [1, 7, 512, 1536, 16384])
+def test_rmsnorm_sizes(nm, n):
+    x = gen.normal_bf16((n,), 3.0, seed=50 + n)
+    g = gen.normal_bf16((n,), 0.02, seed=51 + n, mean=1.0)
+    y = torch.zeros(n, dtype=torch.int16, device="cuda")
+    nm.nm_rmsnorm(to_dev(x), to_dev(g), y, n, 1e-6)
+    torch.cuda.synchronize()
+    ref = f64(oracle.f64_to_bf16(oracle.rmsnorm(f64(x), f64(g), 1e-6)))
+    assert np.all(np.abs(dev_bits_to_f64(y) - ref) <= 1e-5 * np.abs(ref) + oracle.ulp_bf16(ref))
+
+
+def test_rope_stage(nm, ref1024):
+    _, _, r = ref1024
+    H, dn, dr = DIMS["H"], DIMS["nope"], DIMS["rope"]
+    pos = 1023
+    q = to_dev(r["q"])                                      # [H][nope+rope]
+    y = torch.zeros(H * dr, dtype=torch.int16, device="cuda")
+    nm.nm_rope(q.view(-1)[dn:], y, H, dr, dn + dr, dr, rope_row(nm, pos))
+    torch.cuda.synchronize()
+    got, ref = dev_bits_to_f64(y).reshape(H, dr), f64(r["q_rope"])
+    qf = f64(r["q"])[:, dn:]
+    mag = np.abs(qf[:, 0::2]) + np.abs(qf[:, 1::2])         # size of the terms of each output
+    mag = np.repeat(mag, 2, axis=1)
+    assert np.all(np.abs(got - ref) <= 1e-5 * mag + oracle.ulp_bf16(ref))
+
+
+# ---- narrow products of the step, each fed the oracle's inputs ---------------------------------------------
+
+def test_matmul_stages_of_the_step(nm, ref1024, weights):
+    w, dw = weights
+    h, cache, r = ref1024
+    d, ql, dc, dr, dn, dv, H = (DIMS[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
+    dq, dkv = dn + dr, dc + dr
+    ws = nm.new_workspace(max(nm.nm_matmul_workspace_bytes(1, H * dq, ql), nm.nm_matmul_workspace_bytes(1, dc, dn, H)))
+
+    def run(A, Wd, M, N, K, ref_bits, bound, what):
+        C = torch.zeros(M * N, dtype=torch.int16, device="cuda")
+        nm.nm_matmul_ws(to_dev(A), Wd, C, M, N, K, BF16, ROW, ws)
+        torch.cuda.synchronize()
+        ref = f64(ref_bits).reshape(M, N)
+        tol = 1e-5 * bound.reshape(M, N) + 1e-6 + 2 * oracle.ulp_bf16(ref)   # oracle value already rounded: one ulp each side
+        err = np.abs(dev_bits_to_f64(C).reshape(M, N) - ref)
+        assert np.all(err <= tol), f"{what}: {np.sum(err > tol)} outside tolerance, worst {err.max()}"
+
+    run(h, dw["W_DQ"], 1, ql, d, r["c_q"], r["bound_c_q"], "c_q = h*W_DQ")
+    run(r["c_qn"], dw["W_UQR"], 1, H * dq, ql, r["q"], r["bound_q"], "q = c_qn*W_UQR")
+    run(h, dw["W_DKVKR"], 1, dkv, d, r["ckr"], r["bound_ckr"], "ckr = h*(W_DKV|W_KR)")
+    run(r["o"].reshape(-1), dw["W_O"], 1, d, H * dv, r["out"], r["bound_out"], "out = o*W_O")
+    # per-head: q_lat written with the attention operand's stride, o from o_lat
+    qfull = torch.zeros(H * dkv, dtype=torch.int16, device="cuda")
+    nm.nm_matmul_batched_ws(to_dev(r["q"]), dw["W_UK"], qfull, 1, dc, dn, H, H * dq, dq, dn * dc, H * dkv, dkv, BF16, ROW, ws)
+    o = torch.zeros(H * dv, dtype=torch.int16, device="cuda")
+    nm.nm_matmul_batched_ws(to_dev(r["o_lat"]), dw["W_UV"], o, 1, dv, dc, H, H * dc, dc, dc * dv, H * dv, dv, BF16, ROW, ws)
+    torch.cuda.synchronize()
+    got = dev_bits_to_f64(qfull).reshape(H, dkv)[:, :dc]
+    ref = f64(r["q_lat"])
+    assert np.all(np.abs(got - ref) <= 1e-5 * r["bound_q_lat"] + 1e-6 + 2 * oracle.ulp_bf16(ref))
+    got, ref = dev_bits_to_f64(o).reshape(H, dv), f64(r["o"])
+    assert np.all(np.abs(got - ref) <= 1e-5 * r["bound_o"] + 1e-6 + 2 * oracle.ulp_bf16(ref))
+
+
+# ---- attention stage -----------------------------------------------------------------------------------
+
+def attention_case(nm, S, impl, extra, seed=7000):
+    """Q ~ what the step produces in scale; cache rows ~ N(0,1).  extra: attend the last row through
+    the merge (as the step does) or through the row pass."""
+    H, dc, dr = DIMS["H"], DIMS["kv_lora"], DIMS["rope"]
+    dkv = dc + dr
+    Q = np.concatenate([gen.normal_bf16((H, dc), 0.18, seed), gen.normal_bf16((H, dr), 0.78, seed + 1)], axis=1)
+    cache = gen.normal_bf16((S, dkv), 1.0, seed + 2)
+    scale = (DIMS["nope"] + dr) ** -0.5
+    ref = oracle.mla_attention(f64(Q), f64(cache), dc, scale, threads=8)
+    ws = torch.empty(nm.nm_mla_attention_workspace_bytes(H, S, dc), dtype=torch.uint8, device="cuda")
+    o16 = torch.zeros(H * dc, dtype=torch.int16, device="cuda")
+    o32 = torch.zeros(H * dc, dtype=torch.float32, device="cuda")
+    nm.nm_debug_set_attention(impl)
+    try:
+        n_rows, extra_row = (S - 1, S - 1) if extra else (S, -1)
+        nm.nm_mla_attention(to_dev(Q), to_dev(cache), o16, o32, H, n_rows, extra_row, dc, dr, scale, ws)
+        torch.cuda.synchronize()
+    finally:
+        nm.nm_debug_set_attention(0)
+    got32 = o32.cpu().numpy().astype(np.float64).reshape(H, dc)
+    assert rel_max(got32, ref) <= 2e-3, f"S={S} impl={impl}: unrounded output off by {rel_max(got32, ref):.2e}"
+    got16 = dev_bits_to_f64(o16).reshape(H, dc)
+    assert np.all(np.abs(got16 - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
+    return rel_max(got32, ref)
+
+
+@pytest.mark.parametrize("S", [1, 2, 63, 64, 65, 200, 1000, 1024, 4096])
+@pytest.mark.parametrize("extra", [True, False])
+def test_attention_stage_cuda_cores(nm, S, extra):
+    if S == 1 and not extra:
+        attention_case(nm, S, 1, False)
+        return
+    err = attention_case(nm, S, 1, extra)
+    assert err <= 1e-5                                       # fp32 throughout: far inside the bound
+
+
+@pytest.mark.parametrize("S", [1, 2, 63, 64, 65, 129, 200, 1000, 1024, 4096, 16384])
+@pytest.mark.parametrize("extra", [True, False])
+def test_attention_stage_default_path(nm, S, extra):
+    attention_case(nm, S, 0, extra)
+
+
+# ---- the whole step ---------------------------------------------------------------------------------------
+
+def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None):
+    H, dc, dr, dn, dv, d, ql = (DIMS[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d", "q_lora"))
+    dkv, dq = dc + dr, dn + dr
+    t = dict(dw)
+    if not with_wo:
+        t.pop("W_O")
+    t["h"] = to_dev(h)
+    t["kv_cache"] = to_dev(cache_in)
+    t["rope_cos_sin"] = rope_row(nm, S - 1)
+    outs = {"c_q": ql, "c_qn": ql, "q": H * dq, "q_full": H * dkv, "ckr": dkv, "o_lat": H * dc, "o": H * dv, "out": d}
+    for k, n in outs.items():
+        t[k] = torch.zeros(n, dtype=torch.int16, device="cuda")
+    t["o_lat_f32"] = torch.zeros(H * dc, dtype=torch.float32, device="cuda")
+    p = nm.mla_params(DIMS, S, t)
+    ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p))
+    p = nm.mla_params(DIMS, S, t, workspace=ws)
+    main = torch.cuda.Stream()
+    side = torch.cuda.Stream() if overlap else None
+    torch.cuda.synchronize()
+    nm.nm_mla_decode_step(p, main, side)
+    torch.cuda.synchronize()
+    nm.nm_check_status()
+    return t
+
+
+def check_step(t, r, cache_ref, S, with_wo=True):
+    H, dc, dr, dn = DIMS["H"], DIMS["kv_lora"], DIMS["rope"], DIMS["nope"]
+    dkv = dc + dr
+    # first-stage products see exactly the oracle's inputs: tight bound
+    for name, bound in (("c_q", "bound_c_q"), ("ckr", "bound_ckr")):
+        got, ref = dev_bits_to_f64(t[name]), f64(r[name])
+        assert np.all(np.abs(got - ref) <= 1e-5 * r[bound] + 1e-6 + 2 * oracle.ulp_bf16(ref)), name
+    # later stages inherit at most a rounding flip from their inputs: compare against the scale of the tensor
+    for name, ref in (("c_qn", f64(r["c_qn"])), ("q", f64(r["q"]).reshape(-1))):
+        assert rel_max(dev_bits_to_f64(t[name]), ref) <= 1e-2, name
+    qf = dev_bits_to_f64(t["q_full"]).reshape(H, dkv)
+    assert rel_max(qf[:, :dc], f64(r["q_lat"])) <= 1e-2 and rel_max(qf[:, dc:], f64(r["q_rope"])) <= 1e-2
+    # the cache: old rows untouched, the new row equals the oracle's up to a rounding flip
+    cache = t["kv_cache"].cpu().numpy().view(np.uint16).reshape(-1, dkv)
+    assert np.array_equal(cache[:S - 1], cache_ref[:S - 1])
+    assert np.all(np.abs(f64(cache[S - 1]) - f64(cache_ref[S - 1])) <= 2 * oracle.ulp_bf16(f64(cache_ref[S - 1])) + 1e-6)
+    # softmax-containing outputs: max relative error <= 2e-3 (unrounded), plus one ulp once rounded
+    o32 = t["o_lat_f32"].cpu().numpy().astype(np.float64).reshape(H, dc)
+    assert rel_max(o32, r["o_lat_f64"]) <= 2e-3, f"o_lat: {rel_max(o32, r['o_lat_f64']):.2e}"
+    names = [("o_lat", r["o_lat"]), ("o", r["o"])] + ([("out", r["out"])] if with_wo else [])
+    for name, ref_bits in names:
+        got, ref = dev_bits_to_f64(t[name]), f64(ref_bits).reshape(-1)
+        assert np.all(np.abs(got - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref)), name
+
+
+@pytest.mark.parametrize("overlap", [True, False])
+def test_decode_step_s1024(nm, weights, ref1024, overlap):
+    w, dw = weights
+    h, cache_ref, r = ref1024
+    cache_in = gen.mla_cache(1024, DIMS, seed=4200)
+    t = run_step(nm, dw, h, cache_in, 1024, overlap=overlap)
+    check_step(t, r, cache_ref, 1024)
+
+
+@pytest.mark.parametrize("S", [1, 2, 65, 4096])
+def test_decode_step_other_lengths(nm, weights, S):
+    w, dw = weights
+    h, cache_ref, r = oracle_step(w, S, seed=4300 + S)
+    cache_in = gen.mla_cache(S, DIMS, seed=4300 + S)
+    t = run_step(nm, dw, h, cache_in, S)
+    check_step(t, r, cache_ref, S)
+
+
+def test_decode_step_without_wo_and_repeatable(nm, weights):
+    w, dw = weights
+    S = 300
+    h, cache_ref, r = oracle_step(w, S, seed=4400, with_wo=False)
+    cache_in = gen.mla_cache(S, DIMS, seed=4400)
+    t1 = run_step(nm, dw, h, cache_in, S, with_wo=False)
+    check_step(t1, r, cache_ref, S, with_wo=False)
+    t2 = run_step(nm, dw, h, cache_in, S, with_wo=False)
+    for k in ("c_q", "q_full", "o_lat", "o"):
+        assert torch.equal(t1[k], t2[k]), f"{k}: two runs differ"
+
+
+def test_decode_step_host_operands(nm, weights, ref1024):
+    w, dw = weights
+    h, cache_ref, r = ref1024
+    d = DIMS["d"]
+    t = dict(dw)
+    t["kv_cache"] = to_dev(gen.mla_cache(1024, DIMS, seed=4200))
+    t["rope_cos_sin"] = rope_row(nm, 1023)
+    t["h"] = torch.zeros(d, dtype=torch.int16, device="cuda")
+    t["out"] = torch.zeros(d, dtype=torch.int16, device="cuda")
+    p = nm.mla_params(DIMS, 1024, t)
+    ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p))
+    p = nm.mla_params(DIMS, 1024, t, workspace=ws)
+    h_host = torch.from_numpy(h.view(np.int16).copy()).pin_memory()
+    out_host = torch.zeros(d, dtype=torch.int16).pin_memory()
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    nm.nm_mla_decode_step_host(p, h_host, out_host, t["h"], t["out"], main, side)
+    torch.cuda.synchronize()
+    ref = f64(r["out"])
+    got = oracle.bf16_to_f64(out_host.numpy().view(np.uint16))
+    assert np.all(np.abs(got - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
+
+
+def test_step_error_codes(nm, weights):
+    _, dw = weights
+    t = dict(dw)
+    p = nm.mla_params(DIMS, 16, t)                          # h, cache, table, workspace missing
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_mla_decode_step(p)
+    assert e.value.status == -1

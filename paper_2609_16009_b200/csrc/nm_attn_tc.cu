@@ -1,6 +1,321 @@
-// Tensor-core latent attention (placeholder until the tcgen05 kernel lands).
+// Latent attention pass on the tensor cores (tcgen05 + TMEM), one sequence split per CTA pair.
+//
+// For all 128 heads at once and a run of cache rows, tile by tile (64 rows):
+//   S[128 x 64]   = Q[128 x 576] * tile^T      tcgen05.mma, both operands K-major in shared memory
+//   P             = exp2(S*c - m)              fp32 in registers (one thread per head); written to TMEM as
+//                                              two bf16 terms, P_hi = bf16(P) and P_lo = bf16(P - P_hi), so
+//                                              that P*V keeps about 16 bits of P instead of 8
+//   O[128 x 256] += P[128 x 64] * tile[:, half]  tcgen05.mma, A from TMEM, B = the same shared-memory
+//                                                bytes read MN-major
+// Q and the cache tile arrive by TMA (128-byte swizzle, no multicast) and are consumed in place by
+// the MMA unit; the accumulators never leave TMEM until the split is finished.  The 512 output
+// columns do not fit TMEM next to S, so two CTAs share a split, each owning 256 columns.  The running
+// maximum is updated lazily: O is rescaled only when a row maximum grows by more than 2^8, so the
+// usual tile costs no pass over the accumulator.  Splits are merged by attn_combine_kernel.
+//
+// Roles: warp 0 lane 0 issues TMA, warp 1 owns TMEM and its lane 0 issues the MMAs, warps 2-5 hold
+// one head per thread.  Every wait is bounded (mbar_wait); on expiry the CTA raises the status word,
+// skips the remaining waits, frees its TMEM and returns.
+#include "nm_async.cuh"
 #include "nm_mla.cuh"
 
 namespace nm {
-int attention_partial_tc(const void *, const void *, AttnPartials, AttnPlan, int, float, cudaStream_t) { return NM_ERR_UNSUPPORTED; }
+
+namespace {
+
+constexpr int kHeads = 128;
+constexpr int kDqk = 576;                 // 512 latent + 64 rope
+constexpr int kDv = 512;
+constexpr int kDvHalf = 256;
+constexpr int kT = kAttnTileRows;         // cache rows per tile (64)
+constexpr int kKBlocks = kDqk / 64;       // 9 blocks of 64 elements (one 128-byte swizzle span)
+constexpr int kQBlockBytes = kHeads * 128;   // 16 KB
+constexpr int kKVBlockBytes = kT * 128;      // 8 KB
+constexpr int kQBytes = kKBlocks * kQBlockBytes;     // 147456
+constexpr int kKVBytes = kKBlocks * kKVBlockBytes;   // 73728
+constexpr int kSmemBytes = kQBytes + kKVBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColO = 0, kColS = 256, kColP = 320, kColPlo = 352;
+constexpr float kLazyThreshold = 8.0f;    // log2 units
+
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));     // first source -> upper half
+    return r;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, AttnPartials part,
+               int n_rows, int rows_per_split, float scale_log2, unsigned *status)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;            // swizzle atoms want 1024-byte alignment
+    unsigned char *smem = smem_raw + (base - raw_addr);
+    const uint32_t q_addr = base, kv_addr = base + kQBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kQBytes + kKVBytes);
+    const uint32_t bar_q = smem_u32(bars + 0), bar_kv_full = smem_u32(bars + 1), bar_kv_empty = smem_u32(bars + 2),
+                   bar_s = smem_u32(bars + 3), bar_p = smem_u32(bars + 4), bar_o = smem_u32(bars + 5);
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sp = blockIdx.x, half = blockIdx.y;
+    const int r0 = sp * rows_per_split, r1 = min(n_rows, r0 + rows_per_split);
+    const int ntiles = ceil_div(r1 - r0, kT);
+
+    if (tid == 0) {
+        s_abort = 0;
+        mbar_init(bar_q, 1); mbar_init(bar_kv_full, 1); mbar_init(bar_kv_empty, 1);
+        mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+        mbar_init_fence();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+    pdl_launch_dependents();
+
+    if (warp == 0) {
+        // ---------------- TMA producer --------------------------------------------------------------
+        if (lane == 0) {
+            pdl_wait_prior_grids();                               // Q comes from the kernels before this one
+            tma_prefetch_descriptor(&map_q);
+            tma_prefetch_descriptor(&map_kv);
+            const uint64_t keep = l2_policy_evict_last(), stream = l2_policy_evict_first();
+            mbar_arrive_expect_tx(bar_q, kQBytes);
+            for (int c = 0; c < kKBlocks; ++c) tma_load_2d(q_addr + c * kQBlockBytes, &map_q, c * 64, 0, bar_q, keep);
+            for (int t = 0; t < ntiles; ++t) {
+                if (t > 0 && !mbar_try_wait(bar_kv_empty, (t - 1) & 1) && !mbar_wait(bar_kv_empty, (t - 1) & 1, &s_abort, status)) break;
+                mbar_arrive_expect_tx(bar_kv_full, kKVBytes);
+                for (int c = 0; c < kKBlocks; ++c)
+                    tma_load_2d(kv_addr + c * kKVBlockBytes, &map_kv, c * 64, r0 + t * kT, bar_kv_full, stream);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ---------------------------------------------------------------
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc(kT, false), idesc_o = instr_desc(kDvHalf, true);
+            mbar_wait(bar_q, 0, &s_abort, status);
+            for (int t = 0; t < ntiles; ++t) {
+                mbar_wait(bar_kv_full, t & 1, &s_abort, status);
+                tc_fence_after();
+                for (int c = 0; c < kKBlocks; ++c)
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ss(tmem + kColS, smem_desc(q_addr + c * kQBlockBytes + kk * 32, 16, 1024),
+                               smem_desc(kv_addr + c * kKVBlockBytes + kk * 32, 16, 1024), idesc_s, (c | kk) != 0);
+                mma_commit(bar_s);
+                mbar_wait(bar_p, t & 1, &s_abort, status);
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < kT / 16; ++kk) {
+                    const uint64_t vdesc = smem_desc(kv_addr + (4 * half) * kKVBlockBytes + kk * 2048, kKVBlockBytes, 1024);
+                    mma_ts(tmem + kColO, tmem + kColP + kk * 8, vdesc, idesc_o, (t | kk) != 0);
+                    mma_ts(tmem + kColO, tmem + kColPlo + kk * 8, vdesc, idesc_o, true);
+                }
+                mma_commit(bar_o);
+                mma_commit(bar_kv_empty);
+            }
+        }
+    } else {
+        // ---------------- one head per thread: softmax, lazy rescale, epilogue ----------------------------
+        const int quad = warp & 3;                                 // TMEM lanes this warp may touch
+        const int head = quad * 32 + lane;
+        const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
+        float m_used = -INFINITY, l = 0.f;
+        for (int t = 0; t < ntiles; ++t) {
+            mbar_wait(bar_s, t & 1, &s_abort, status);
+            tc_fence_after();
+            uint32_t sr[2][32];
+            tmem_ld32(lane_base + kColS, sr[0]);
+            tmem_ld32(lane_base + kColS + 32, sr[1]);
+            tmem_wait_ld();
+            const int valid = min(kT, r1 - (r0 + t * kT));
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < kT; ++j)
+                if (j < valid) mx = fmaxf(mx, __uint_as_float(sr[j >> 5][j & 31]));
+            const float mx2 = mx * scale_log2;
+            const bool grow = (t == 0) || (mx2 > m_used + kLazyThreshold);
+            if (t > 0) {                                           // previous P*V must be done before P or O change
+                mbar_wait(bar_o, (t - 1) & 1, &s_abort, status);
+                tc_fence_after();
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float f = grow ? fast_exp2(m_used - mx2) : 1.0f;
+                    for (int c = 0; c < kDvHalf / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(lane_base + kColO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st32(lane_base + kColO + c * 32, o);
+                    }
+                    tmem_wait_st();
+                    if (grow) l *= f;
+                }
+            }
+            if (grow) m_used = mx2;
+            uint32_t pr[32], plo[32];
+            float lsum = 0.f;
+#pragma unroll
+            for (int j = 0; j < kT; j += 2) {
+                const float p0 = (j < valid) ? fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), scale_log2, -m_used)) : 0.f;
+                const float p1 = (j + 1 < valid) ? fast_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), scale_log2, -m_used)) : 0.f;
+                lsum += p0 + p1;
+                const uint32_t hi = pack_bf16x2(p0, p1);
+                pr[j >> 1] = hi;
+                plo[j >> 1] = pack_bf16x2(p0 - __uint_as_float(hi << 16), p1 - __uint_as_float(hi & 0xffff0000u));
+            }
+            l += lsum;
+            tmem_st32(lane_base + kColP, pr);
+            tmem_st32(lane_base + kColPlo, plo);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p);
+        }
+        // epilogue: unnormalised O (this CTA's 256 columns) and (m, l) to the partial buffers
+        if (ntiles > 0) {
+            mbar_wait(bar_o, (ntiles - 1) & 1, &s_abort, status);
+            tc_fence_after();
+            float *dst = part.O + ((size_t)sp * kHeads + head) * kDv + half * kDvHalf;
+            for (int c = 0; c < kDvHalf / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(lane_base + kColO + c * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; i += 4)
+                    *reinterpret_cast<uint4 *>(dst + c * 32 + i) = make_uint4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+            }
+            if (half == 0) {
+                part.ml[((size_t)sp * kHeads + head) * 2] = m_used * 0.6931471805599453f;   // back to natural-log units
+                part.ml[((size_t)sp * kHeads + head) * 2 + 1] = l;
+            }
+        }
+    }
+
+    // ---- teardown: everyone meets, TMEM goes back ---------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (s_abort && tid == 0) {
+        // a wait expired: give copies already issued a bounded chance to land before the CTA exits
+        for (int i = 0; i < (1 << 16) && !mbar_try_wait(bar_q, 0); ++i) {}
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// Tensor maps: bf16 [rows][576], boxes of 64 columns (128 bytes, the swizzle span) x box_rows rows.
+bool encode_rows_map(CUtensorMap *map, const void *ptr, int rows, int box_rows)
+{
+    EncodeTiledFn enc = tensor_map_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kDqk, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kDqk * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows, float scale,
+                         cudaStream_t stream)
+{
+    if (n_rows < 1 || plan.nsplit < 1) return NM_ERR_UNSUPPORTED;
+    if (((uintptr_t)Q & 15u) || ((uintptr_t)cache & 15u)) return NM_ERR_UNSUPPORTED;
+    CUtensorMap map_q, map_kv;
+    // The cache map covers exactly the rows attended: rows past n_rows read as zeros (and are masked),
+    // whatever the rest of the buffer holds.
+    if (!encode_rows_map(&map_q, Q, kHeads, kHeads) || !encode_rows_map(&map_kv, cache, n_rows, kT)) return NM_ERR_UNSUPPORTED;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return record_cuda_error(e, "attention kernel attribute");
+        configured = true;
+    }
+    const float scale_log2 = scale * 1.4426950408889634f;
+    attn_tc_kernel<<<dim3(plan.nsplit, 2), kThreads, kSmemBytes, stream>>>(map_q, map_kv, part, n_rows, plan.rows_per_split,
+                                                                          scale_log2, device_status_ptr());
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (tensor cores) launch");
+}
+
 }  // namespace nm

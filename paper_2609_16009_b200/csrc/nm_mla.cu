@@ -218,7 +218,10 @@ AttnPlan plan_attention(int H, int n_rows, int kv_lora)
     AttnPlan p{};
     (void)H; (void)kv_lora;
     const int tiles = ceil_div(n_rows > 0 ? n_rows : 0, kAttnTileRows);
-    int nsplit = tiles < kMaxAttnSplits ? tiles : kMaxAttnSplits;
+    // 64 splits x 2 column halves = 128 CTAs: one wave of the 148 SMs, leaving a few for the narrow
+    // products that run beside the attention pass
+    constexpr int kSplitTarget = 64;
+    int nsplit = tiles < kSplitTarget ? tiles : kSplitTarget;
     if (nsplit < 1) nsplit = (n_rows > 0) ? 1 : 0;
     p.nsplit = nsplit;
     p.rows_per_split = nsplit ? ceil_div(tiles, nsplit) * kAttnTileRows : 0;

@@ -102,10 +102,102 @@ class ProjectionChain:
         self.out_host.copy_(self.y["W_O"], non_blocking=True)
 
 
+class MlaStep:
+    """The whole single-token decode step (nm_mla_decode_step): Q chain, KV chain on a side stream,
+    tensor-core latent attention over the cache, output side including W_O."""
+
+    name = "mla"
+
+    def __init__(self, nm, device, seq_len, seed=4000):
+        self.nm = nm
+        self.S = seq_len
+        d, ql, dc, dr, dn, dv, H = (DIMS[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
+        w = gen.mla_weights(DIMS, seed=seed, with_wo=True)
+        t = {k: torch.from_numpy(v.view(np.int16)).to(device) for k, v in w.items()}
+        self.h_host = torch.from_numpy(gen.mla_token(DIMS, seed=seed + 100).view(np.int16).copy()).pin_memory()
+        self.out_host = torch.empty(d, dtype=torch.int16).pin_memory()
+        t["h"] = self.h_host.to(device)
+        t["out"] = torch.zeros(d, dtype=torch.int16, device=device)
+        t["kv_cache"] = torch.from_numpy(gen.mla_cache(seq_len, DIMS, seed=seed + 200).view(np.int16)).to(device)
+        t["rope_cos_sin"] = torch.empty(dr, dtype=torch.float32, device=device)
+        nm.nm_rope_table(t["rope_cos_sin"], seq_len - 1, 1, dr)
+        self.t = t
+        p = nm.mla_params(DIMS, seq_len, t)
+        self.ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p), device=device)
+        self.p = nm.mla_params(DIMS, seq_len, t, workspace=self.ws)
+        self.side = torch.cuda.Stream(device)
+        self.specs = projection_specs()
+        self.kv_bytes = seq_len * (dc + dr) * 2 + (dc + dr) * 2        # rows read once + the row written
+        self.bytes_per_step = algorithmic_bytes(self.specs) + self.kv_bytes
+        self.dominant = "W_O product (nm_row_tma_kernel, K=16384, N=7168, M=1)"
+        self.dominant_bytes = algorithmic_bytes([s for s in self.specs if s[0] == "W_O"])
+        self.launches_per_step = 11
+        self.h2d = d * 2
+        self.d2h = d * 2
+
+    def describe(self):
+        return {"workload": f"full single-token MLA decode step, DeepSeek-V3 dims (hidden 7168, q_lora 1536, kv_lora 512, rope 64, "
+                            f"nope 128, v 128, 128 heads), seq_len {self.S}, bf16 weights row-major, W_O included",
+                "seq_len": self.S,
+                "l2": "weights 374 MB per step > 126 MB L2, so every step streams from HBM; no flush",
+                "overlap": "KV chain (W_DKV|KR product, RMSNorm, RoPE, cache write) on a side stream beside the tcgen05 attention pass"}
+
+    def step(self, stream, dom_events=None):
+        if dom_events is not None:
+            self.p.event_before_wo, self.p.event_after_wo = dom_events[0].cuda_event, dom_events[1].cuda_event
+        else:
+            self.p.event_before_wo, self.p.event_after_wo = None, None
+        self.nm.nm_mla_decode_step(self.p, stream, self.side)
+
+    def step_e2e(self, stream):
+        self.p.event_before_wo, self.p.event_after_wo = None, None
+        self.nm.nm_mla_decode_step_host(self.p, self.h_host, self.out_host, self.t["h"], self.t["out"], stream, self.side)
+
+
 def make_workload(kind, nm, device, seq_len):
     if kind == "projections":
         return ProjectionChain(nm, device)
+    if kind == "mla":
+        return MlaStep(nm, device, seq_len)
     raise SystemExit(f"unknown workload {kind}")
+
+
+def matmul_sweep(nm, device):
+    """GB/s of single narrow products (cold L2: the launches of a CUDA graph rotate through copies of
+    B that together exceed 512 MB).  Reported beside the step; not part of the timed region."""
+    out = []
+    cases = [(1, 7168, 1536, 0), (1, 7168, 576, 0), (1, 7168, 1536, 1), (1, 7168, 576, 1)]
+    for M in (1, 2, 4, 8, 16):
+        cases += [(M, 1536, 24576, 0), (M, 7168, 18432, 0)]
+    g0 = torch.Generator(device="cpu"); g0.manual_seed(7)
+    for M, K, N, layout in cases:
+        nbytes = K * N * 2
+        R = max(2, min(64, (1 << 29) // nbytes + 1))
+        Bs = (torch.randn(R, K * N, device=device) * 0.02).to(torch.bfloat16)
+        A = torch.randn(M * K, device=device).to(torch.bfloat16)
+        C = torch.empty(R, M * N, device=device, dtype=torch.bfloat16)
+        ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(M, N, K), device=device)
+        s = torch.cuda.Stream(device)
+        with torch.cuda.stream(s):
+            for i in range(R):
+                nm.nm_matmul_ws(A, Bs[i], C[i], M, N, K, nm.BF16, layout, ws, s)
+            s.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for i in range(R):
+                    nm.nm_matmul_ws(A, Bs[i], C[i], M, N, K, nm.BF16, layout, ws, s)
+            g.replay(); s.synchronize()
+            ts = []
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(s); g.replay(); b.record(s); s.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3 / R)
+        us = statistics.median(ts)
+        algo = (K * N + M * K + M * N) * 2
+        out.append({"M": M, "K": K, "N": N, "layout_B": "col" if layout else "row", "us": round(us, 2),
+                    "GBps": round(algo / us / 1e3, 1), "pct_of_8TBs": round(algo / us / 1e3 / 80.0, 1)})
+        del Bs, C, g
+    return out
 
 
 # --------------------------------------------------------------------------------------------------
@@ -159,22 +251,30 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # CPU oracle arm
 # --------------------------------------------------------------------------------------------------
-_ORACLE_INPUTS = None
+_ORACLE_INPUTS = {}
 
 
-def oracle_sample(threads):
-    """One pass of the oracle, as it stands, over the narrow products of the step (all six weight
-    matrices, M = 1) on the host cores.  Returns (seconds, algorithmic bytes, description)."""
+def oracle_sample(threads, kind="mla", seq_len=4096):
+    """One pass of the oracle, as it stands, on the host cores over the same workload: the naive
+    decode step at `seq_len` (kind "mla") or the six narrow products alone (kind "projections").
+    Returns (seconds, algorithmic bytes, description)."""
     import oracle
-    global _ORACLE_INPUTS
     specs = projection_specs()
-    if _ORACLE_INPUTS is None:
+    key = (kind, seq_len)
+    if key not in _ORACLE_INPUTS:
         w = gen.mla_weights(DIMS, seed=4000, with_wo=True)
-        x = {name: gen.normal_bf16((H * K,), 1.0, 4200 + i) for i, (name, K, N, H) in enumerate(specs)}
         oracle.lib()
-        _ORACLE_INPUTS = (w, x)
-    w, x = _ORACLE_INPUTS
+        if kind == "mla":
+            _ORACLE_INPUTS[key] = (w, gen.mla_token(DIMS, seed=4100), gen.mla_cache(seq_len, DIMS, seed=4200))
+        else:
+            _ORACLE_INPUTS[key] = (w, {name: gen.normal_bf16((H * K,), 1.0, 4200 + i) for i, (name, K, N, H) in enumerate(specs)}, None)
+    w, x, cache = _ORACLE_INPUTS[key]
     t0 = time.perf_counter()
+    if kind == "mla":
+        oracle.mla_decode_step(DIMS, w, x, cache, seq_len, threads=threads)
+        dt = time.perf_counter() - t0
+        nbytes = algorithmic_bytes(specs) + (seq_len + 1) * (DIMS["kv_lora"] + DIMS["rope"]) * 2
+        return dt, nbytes, f"the whole naive decode step at seq_len {seq_len} (374 MB of bf16 weights + cache), one pass"
     for name, K, N, H in specs:
         if H == 1:
             oracle.matmul(x[name], w[name], 1, N, K, oracle.BF16, oracle.BF16, oracle.ROW_MAJOR, threads=threads)
@@ -190,16 +290,17 @@ def run_reference(args, rank):
         return
     import oracle
     threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
-    for _ in range(args.warmup):
-        oracle_sample(threads)
+    steps = min(args.steps, 20)              # bounded: the oracle is slow by design
+    for _ in range(min(args.warmup, 2)):
+        oracle_sample(threads, args.workload, args.seq_len)
     times, nbytes, what = [], 0, ""
-    for _ in range(args.steps):
-        dt, nbytes, what = oracle_sample(threads)
+    for _ in range(steps):
+        dt, nbytes, what = oracle_sample(threads, args.workload, args.seq_len)
         times.append(dt)
     total = sum(times)
     value = nbytes * len(times) / total / 1e9
-    line = {"impl": "reference", "metric": "narrow MatMul HBM GB/s", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / len(times) * 1e3,
+    line = {"impl": "reference", "metric": "narrow MatMul HBM GB/s (MLA single-token decode step)", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": steps, "warmup": min(args.warmup, 2), "ms_per_step": total / len(times) * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": "CPU oracle (fp64 triple loop) on a bounded sample: " + what},
             "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": what},
@@ -225,7 +326,8 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="projections")
+    ap.add_argument("--workload", default="mla", choices=["mla", "projections"])
+    ap.add_argument("--sweep", action="store_true", help="also report GB/s of single narrow products vs M")
     ap.add_argument("--seq-len", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -267,6 +369,8 @@ def main():
         sampler.start()
         # ---- device-timed region: exactly `steps` steps, inputs resident in HBM ------------------------
         dom = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in dom:                      # events get their handles on first record
+            a.record(stream); b.record(stream)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record(stream)
@@ -302,8 +406,9 @@ def main():
         value = total_bytes / (ms * 1e-3) / 1e9
         e2e_value = total_bytes / (e2e_ms * 1e-3) / 1e9
         achieved = wl.dominant_bytes / (dom_ms * 1e-3) / 1e9
-        line = {"metric": "narrow MatMul HBM GB/s", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        line = {"metric": "narrow MatMul HBM GB/s (MLA single-token decode step)", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms / args.steps, "decode_us": ms / args.steps * 1e3,
+                "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": wl.describe(),
                 "pct_of_8TBs": value / world / 8000.0,
@@ -314,11 +419,13 @@ def main():
                 "roofline": {"bound": "hbm", "kernel": wl.dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                              "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
                              "us_per_launch": dom_ms * 1e3}}
+        if args.sweep:
+            line["narrow_matmul_vs_M"] = matmul_sweep(nm, device)
         if not args.no_cpu_baseline:
             import oracle
             threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
-            oracle_sample(threads)
-            dt, nbytes, what = oracle_sample(threads)
+            oracle_sample(threads, args.workload, args.seq_len)
+            dt, nbytes, what = oracle_sample(threads, args.workload, args.seq_len)
             line["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
                                     "sample": what, "seconds": dt}
         print(json.dumps(line), flush=True)

@@ -234,6 +234,8 @@ typedef struct {
     /* optional intermediates, bf16 unless noted */
     void *c_q, *c_qn, *q, *q_full /* [H][kv_lora+rope] = q_lat | q_rope */, *ckr, *o_lat, *o;
     float *o_lat_f32;
+    /* optional cudaEvent_t pair recorded on main_stream around the W_O product (for profiling) */
+    void *event_before_wo, *event_after_wo;
 } nm_mla_params;
 
 size_t nm_mla_workspace_bytes(const nm_mla_params *p);

@@ -71,7 +71,8 @@ class MlaParams(C.Structure):
                 + [(n, _vp) for n in ("h", "W_DQ", "gamma_q", "W_UQR", "W_DKVKR", "gamma_kv", "W_UK", "W_UV", "W_O",
                                       "rope_cos_sin", "kv_cache", "out", "workspace")]
                 + [("workspace_bytes", _sz)]
-                + [(n, _vp) for n in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o", "o_lat_f32")])
+                + [(n, _vp) for n in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o", "o_lat_f32",
+                                      "event_before_wo", "event_after_wo")])
 
 
 _lib.nm_rmsnorm.argtypes = [_vp, _vp, _vp, _i, C.c_float, _vp]

@@ -392,8 +392,11 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     // ---- output side -----------------------------------------------------------------------------------
     NM_TRY(matmul_enqueue(o_lat, p->W_UV, o, 1, dv, dc, H, (long)H * dc, dc, (long)dc * dv, (long)H * dv, dv,
                           NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms));
-    if (p->W_O)
+    if (p->W_O) {
+        if (p->event_before_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_before_wo, ms));
         NM_TRY(matmul_enqueue(o, p->W_O, p->out, 1, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms));
+        if (p->event_after_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_after_wo, ms));
+    }
     return NM_OK;
 }
 

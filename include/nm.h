@@ -261,6 +261,10 @@ int nm_debug_set_plan(int tile_n, int nsplit);
 /* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel instead
  * of the TMA ring) and the ring depth in stages (0 heuristic). */
 int nm_debug_set_kernel(int kind, int stages);
+/* Decode step: MB of W_O prefetched into L2 beside the attention pass (default 40, 0 = off). */
+int nm_debug_set_step_prefetch(int megabytes);
+/* Decode step: chain its kernels with programmatic dependent launch (default 1) or not (0). */
+int nm_debug_set_step_pdl(int enable);
 /* Attention pass: 0 tensor-core kernel when the shape allows (default), 1 CUDA-core kernel. */
 int nm_debug_set_attention(int impl);
 /* Report the plan for a problem: out[0..5] = kernel kind (0 row-major vector, 1 column-major

@@ -88,6 +88,8 @@ _lib.nm_mla_workspace_bytes.argtypes = [C.POINTER(MlaParams)]
 _lib.nm_mla_decode_step.argtypes = [C.POINTER(MlaParams), _vp, _vp]
 _lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_debug_set_attention.argtypes = [_i]
+_lib.nm_debug_set_step_pdl.argtypes = [_i]
+_lib.nm_debug_set_step_prefetch.argtypes = [_i]
 
 
 def _check(status: int, where: str) -> None:
@@ -283,6 +285,14 @@ def nm_mla_decode_step_host(p: MlaParams, h_host, out_host, h_staging, out_stagi
     ss = ms if side_stream is None else _stream(side_stream)
     _check(_lib.nm_mla_decode_step_host(C.byref(p), _ptr(h_host), _ptr(out_host), _ptr(h_staging), _ptr(out_staging),
                                         ms, ss), "nm_mla_decode_step_host")
+
+
+def nm_debug_set_step_prefetch(megabytes: int) -> None:
+    _check(_lib.nm_debug_set_step_prefetch(int(megabytes)), "nm_debug_set_step_prefetch")
+
+
+def nm_debug_set_step_pdl(enable: bool) -> None:
+    _check(_lib.nm_debug_set_step_pdl(int(enable)), "nm_debug_set_step_pdl")
 
 
 def nm_debug_set_attention(impl: int) -> None:

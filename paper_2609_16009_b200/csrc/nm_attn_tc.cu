@@ -152,14 +152,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (warp == 0) {
         // ---------------- TMA producer --------------------------------------------------------------
         if (lane == 0) {
-            pdl_wait_prior_grids();                               // Q comes from the kernels before this one
             tma_prefetch_descriptor(&map_q);
             tma_prefetch_descriptor(&map_kv);
             const uint64_t keep = l2_policy_evict_last(), stream = l2_policy_evict_first();
+            // The rows of the first tile were written by earlier steps, not by the kernels just before
+            // this one: fetch them before waiting for those kernels, then fetch Q, which they produce.
+            if (ntiles > 0) {
+                mbar_arrive_expect_tx(bar_kv_full, kKVBytes);
+                for (int c = 0; c < kKBlocks; ++c) tma_load_2d(kv_addr + c * kKVBlockBytes, &map_kv, c * 64, r0, bar_kv_full, stream);
+            }
+            pdl_wait_prior_grids();
             mbar_arrive_expect_tx(bar_q, kQBytes);
             for (int c = 0; c < kKBlocks; ++c) tma_load_2d(q_addr + c * kQBlockBytes, &map_q, c * 64, 0, bar_q, keep);
-            for (int t = 0; t < ntiles; ++t) {
-                if (t > 0 && !mbar_try_wait(bar_kv_empty, (t - 1) & 1) && !mbar_wait(bar_kv_empty, (t - 1) & 1, &s_abort, status)) break;
+            for (int t = 1; t < ntiles; ++t) {
+                if (!mbar_try_wait(bar_kv_empty, (t - 1) & 1) && !mbar_wait(bar_kv_empty, (t - 1) & 1, &s_abort, status)) break;
                 mbar_arrive_expect_tx(bar_kv_full, kKVBytes);
                 for (int c = 0; c < kKBlocks; ++c)
                     tma_load_2d(kv_addr + c * kKVBlockBytes, &map_kv, c * 64, r0 + t * kT, bar_kv_full, stream);
@@ -297,7 +303,7 @@ bool encode_rows_map(CUtensorMap *map, const void *ptr, int rows, int box_rows)
 }  // namespace
 
 int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows, float scale,
-                         cudaStream_t stream)
+                         cudaStream_t stream, bool programmatic_launch)
 {
     if (n_rows < 1 || plan.nsplit < 1) return NM_ERR_UNSUPPORTED;
     if (((uintptr_t)Q & 15u) || ((uintptr_t)cache & 15u)) return NM_ERR_UNSUPPORTED;
@@ -312,9 +318,18 @@ int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, At
         configured = true;
     }
     const float scale_log2 = scale * 1.4426950408889634f;
-    attn_tc_kernel<<<dim3(plan.nsplit, 2), kThreads, kSmemBytes, stream>>>(map_q, map_kv, part, n_rows, plan.rows_per_split,
-                                                                          scale_log2, device_status_ptr());
-    cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan.nsplit, 2);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = programmatic_launch ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, map_q, map_kv, part, n_rows, plan.rows_per_split, scale_log2,
+                                       device_status_ptr());
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (tensor cores) launch");
 }
 

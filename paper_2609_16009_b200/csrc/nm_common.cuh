@@ -73,10 +73,16 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p) {
 __device__ __forceinline__ float ld_cg(const float *p) { return __ldcg(p); }
 
 // Validates, plans and enqueues one (batched) narrow product; `ws` may be null when the plan does
-// not split K.  Defined in nm_matmul.cu.
+// not split K.  With programmatic_launch the kernel may begin (and prefetch B) before the previous
+// kernel in the stream has finished; it still waits for it before reading A or writing anything.
+// Defined in nm_matmul.cu.
 int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, int H,
                    long lda, long strideA, long strideB, long ldc, long strideC,
-                   nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream);
+                   nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream,
+                   bool programmatic_launch = false);
+
+// How the row-major bf16 product K x N (H heads) at this M will be split: k-rows per split and splits.
+void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit);
 
 __host__ __device__ constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
 

@@ -51,48 +51,45 @@ static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t
 // (a) enough CTAs to cover all 148 SMs a few times over, (b) per-CTA segments of B as long and as
 // contiguous as the shape allows, (c) few enough splits that the partial-sum traffic stays a few
 // per cent of |B|.
-// Plan for the TMA-ring kernel.  Cost model, in units of one streamed weight element per CTA:
-// waves over the resident-CTA slots x (elements per CTA + a fixed per-CTA cost + the partial-sum
-// traffic a split adds).  The search is tiny (3 tile widths x 64 split counts).
+// Plan for the TMA-ring kernel, from measurements on B200 (sweeps over tile width, k-splits and ring
+// depth for the decode step's shapes and the M-sweep shapes):
+//  * 64-column tiles unless that makes more than ~384 CTAs (then 128, then 256 columns);
+//  * about one to two CTAs per SM in total: 256 for products of 32 MB and more, 160 below that
+//    (each extra split costs a partial tile and lengthens the gather), 148 when M > 8 (one resident
+//    CTA per SM);
+//  * k-rows per split a multiple of the stage height, so that no TMA box straddles two splits;
+//  * five 16 KB stages (two resident CTAs per SM), three when there are more CTAs than that, ten
+//    when M > 8.
 static Plan make_tma_plan(int M, int N, int K, int H)
 {
-    const int occ = (M <= 8) ? 2 : 1;       // resident CTAs per SM the plan aims for (measured best)
-    const long slots = (long)kSMs * occ;
-    Plan best{};
-    double best_cost = 1e300;
-    for (int tpr = 8; tpr <= 32; tpr *= 2) {
-        const int tn = tpr * 8;
-        if (g_force_tn > 0 && tn != g_force_tn) continue;
-        const int ntiles = ceil_div(N, tn);
-        if ((long)ntiles * H > kNumCounters && g_force_split > 1) continue;
-        for (int ns = 1; ns <= kMaxSplit; ++ns) {
-            if (g_force_split > 0 && ns != g_force_split) continue;
-            if (ns > 1 && (long)ntiles * H > kNumCounters) break;
-            int kr = ceil_div(ceil_div(K, ns), 8) * 8;
-            const int ns_eff = ceil_div(K, kr);
-            if (ns_eff != ns && g_force_split == 0) continue;       // duplicate of a smaller split count
-            const long ctas = (long)ntiles * ns_eff * H;
-            const long waves = (ctas + slots - 1) / slots;
-            const double per_cta = (double)kr * tn + 8192.0 + (ns_eff > 1 ? 4.0 * M * tn + 64.0 * ns_eff : 0.0);
-            const double cost = (double)waves * per_cta * (tn == 64 ? 1.0 : 1.001);
-            if (cost < best_cost) {
-                best_cost = cost;
-                best.kind = kRowTma; best.tn = tn; best.tpr = tpr; best.rg = kTmaConsumers / tpr;
-                best.nsplit = ns_eff; best.kr = kr; best.ntiles = ntiles;
-                // 16 KB stages; the ring takes what is left of ~200 KB per SM after the A chunk
-                int nstage = (M <= 2) ? 3 : (occ == 2) ? 5 : 10;
-                if (g_force_stages > 0) nstage = g_force_stages;
-                if (nstage < 2) nstage = 2;
-                if (nstage > 11) nstage = 11;
-                best.nstage = nstage;
-            }
-        }
-    }
-    if (best_cost == 1e300) {       // forced values matched nothing: fall back to one wide tile, no split
-        best.kind = kRowTma; best.tn = 64; best.tpr = 8; best.rg = 32; best.nsplit = 1; best.kr = ceil_div(K, 8) * 8;
-        best.ntiles = ceil_div(N, 64); best.nstage = 8;
-    }
-    return best;
+    Plan p{};
+    p.kind = kRowTma;
+    int tn = 64;
+    while ((long)ceil_div(N, tn) * H > 384 && tn < 256) tn *= 2;
+    if (g_force_tn == 64 || g_force_tn == 128 || g_force_tn == 256) tn = g_force_tn;
+    const int tpr = tn / 8;
+    const int kt = (kTmaConsumers / tpr) * 4;
+    const int ntiles = ceil_div(N, tn);
+    const long base = (long)ntiles * H;
+    const double total_bytes = 2.0 * K * N * H;
+    const int target = (M > 8) ? kSMs : (total_bytes < 32e6 ? 160 : 256);
+    int ns = (int)((target + base / 2) / base);
+    if (ns > K / 128) ns = K / 128;
+    if (g_force_split > 0) ns = g_force_split;
+    if (ns > kMaxSplit) ns = kMaxSplit;
+    if (ns < 1) ns = 1;
+    if (base > kNumCounters) ns = 1;
+    int kr = ceil_div(ceil_div(K, ns), kt) * kt;
+    if (g_force_split > 0) kr = ceil_div(ceil_div(K, ns), 8) * 8;      // forced plans keep the requested split count
+    ns = ceil_div(K, kr);
+    p.tn = tn; p.tpr = tpr; p.rg = kTmaConsumers / tpr; p.nsplit = ns; p.kr = kr; p.ntiles = ntiles;
+    const long ctas = base * ns;
+    int nstage = (M > 8) ? 10 : (ctas > 2 * kSMs ? 3 : 5);
+    if (g_force_stages > 0) nstage = g_force_stages;
+    if (nstage < 2) nstage = 2;
+    if (nstage > 11) nstage = 11;
+    p.nstage = nstage;
+    return p;
 }
 
 static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout, bool vec_ok, bool tma_ok)
@@ -193,7 +190,7 @@ static int check_common(const void *A, const void *B, const void *C, int M, int 
 
 static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int K, int H,
                        long lda, long strideA, long strideB, long ldc, long strideC,
-                       nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream)
+                       nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream, bool pdl = false)
 {
     int rc = check_common(A, B, C, M, N, K, H, dtype, layout);
     if (rc != NM_OK) return rc;
@@ -231,7 +228,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         const CUtensorMap *map = get_weight_map(B, N, K, H, strideB, p.tn, kt);
         if (!map) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
         TmaArgs ta{};
-        ta.base = a; ta.nstage = p.nstage; ta.use_pdl = g_use_pdl; ta.status = device_status_ptr();
+        ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
         const size_t smem = (size_t)p.nstage * kt * p.tn * 2 + kAChunkFloats * sizeof(float) + 2 * p.nstage * sizeof(uint64_t);
         const bool f32out = (dtype == NM_BF16_F32OUT);
         if (p.tpr == 8)       e = f32out ? launch_row_tma<8, float>(*map, ta, smem, stream)  : launch_row_tma<8, bf16_t>(*map, ta, smem, stream);
@@ -254,12 +251,20 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     return NM_OK;
 }
 
+void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit)
+{
+    const Plan p = make_tma_plan(M, N, K, H);
+    *k_rows_per_split = p.kr;
+    *nsplit = p.nsplit;
+}
+
 // internal entry used by the decode step
 int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, int H,
                    long lda, long strideA, long strideB, long ldc, long strideC,
-                   nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream)
+                   nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream, bool programmatic_launch)
 {
-    return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout, ws, ws_bytes, stream);
+    return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout, ws, ws_bytes, stream,
+                       programmatic_launch);
 }
 
 }  // namespace nm

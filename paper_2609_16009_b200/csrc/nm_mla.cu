@@ -27,11 +27,49 @@ __device__ __forceinline__ float block_sum(float v, float *scratch /* >= 32 floa
 }
 
 // y = x * rsqrt(mean(x^2) + eps) * gamma, one CTA, everything in fp32, one rounding to bf16.
+// x and gamma are fetched with 16-byte loads where alignment allows, all issued before the sum.
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ gamma,
                                                       uint16_t *__restrict__ y, int n, float eps)
 {
     __shared__ float scratch[32];
     pdl_wait_prior_grids();
+    const bool vec = (n % 8 == 0) && n <= 8 * 256 * 4 && ((((uintptr_t)x | (uintptr_t)gamma | (uintptr_t)y) & 15u) == 0);
+    if (vec) {
+        constexpr int kMaxPerThread = 4;
+        uint4 xv[kMaxPerThread], gv[kMaxPerThread];
+        const int nv = n / 8;
+#pragma unroll
+        for (int j = 0; j < kMaxPerThread; ++j) {
+            const int i = threadIdx.x + j * 256;
+            if (i < nv) { xv[j] = reinterpret_cast<const uint4 *>(x)[i]; gv[j] = __ldg(reinterpret_cast<const uint4 *>(gamma) + i); }
+        }
+        float ss = 0.f;
+#pragma unroll
+        for (int j = 0; j < kMaxPerThread; ++j)
+            if (threadIdx.x + j * 256 < nv) {
+                float f[8];
+                Elem<bf16_t>::unpack(xv[j], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+            }
+        ss = block_sum(ss, scratch);
+        const float r = 1.0f / sqrtf(ss / (float)n + eps);
+#pragma unroll
+        for (int j = 0; j < kMaxPerThread; ++j) {
+            const int i = threadIdx.x + j * 256;
+            if (i < nv) {
+                float f[8], g[8];
+                Elem<bf16_t>::unpack(xv[j], f);
+                Elem<bf16_t>::unpack(gv[j], g);
+                uint32_t o[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    o[e] = (uint32_t)f32_to_bf16_bits(f[2 * e] * r * g[2 * e]) | ((uint32_t)f32_to_bf16_bits(f[2 * e + 1] * r * g[2 * e + 1]) << 16);
+                reinterpret_cast<uint4 *>(y)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        return;
+    }
     float ss = 0.f;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
         const float v = bf16_bits_to_f32(x[i]);
@@ -74,27 +112,59 @@ __global__ void rope_table_kernel(float *table, long pos_begin, int n_pos, int d
 }
 
 // The consumers of MatMul 2 in one kernel: RMSNorm of the latent part, RoPE of the key part,
-// both rounded to bf16 and written into the cache row.
+// both rounded to bf16 and written into the cache row.  dc <= 512 elements per 256 threads x 2.
 __global__ void __launch_bounds__(256) kv_finish_kernel(const uint16_t *__restrict__ ckr, const uint16_t *__restrict__ gamma,
                                                         const float *__restrict__ cs, uint16_t *__restrict__ cache_row,
                                                         int dc, int dr, float eps)
 {
     __shared__ float scratch[32];
     pdl_wait_prior_grids();
-    float ss = 0.f;
-    for (int i = threadIdx.x; i < dc; i += blockDim.x) {
-        const float v = bf16_bits_to_f32(ckr[i]);
-        ss = fmaf(v, v, ss);
+    const int i0 = 2 * threadIdx.x;                                // two latent elements per thread
+    float x0 = 0.f, x1 = 0.f, g0 = 0.f, g1 = 0.f;
+    if (i0 < dc) {
+        const uint32_t xv = *reinterpret_cast<const uint32_t *>(ckr + i0), gv = *reinterpret_cast<const uint32_t *>(gamma + i0);
+        x0 = __uint_as_float(xv << 16); x1 = __uint_as_float(xv & 0xffff0000u);
+        g0 = __uint_as_float(gv << 16); g1 = __uint_as_float(gv & 0xffff0000u);
     }
-    ss = block_sum(ss, scratch);
+    float r0v = 0.f, r1v = 0.f, c = 0.f, sn = 0.f;
+    if (threadIdx.x < dr / 2) {
+        const uint32_t rv = *reinterpret_cast<const uint32_t *>(ckr + dc + i0);
+        r0v = __uint_as_float(rv << 16); r1v = __uint_as_float(rv & 0xffff0000u);
+        c = cs[i0]; sn = cs[i0 + 1];
+    }
+    const float ss = block_sum(fmaf(x0, x0, x1 * x1), scratch);
     const float r = 1.0f / sqrtf(ss / (float)dc + eps);
-    for (int i = threadIdx.x; i < dc; i += blockDim.x)
-        cache_row[i] = f32_to_bf16_bits(bf16_bits_to_f32(ckr[i]) * r * bf16_bits_to_f32(gamma[i]));
-    for (int i = threadIdx.x; i < dr / 2; i += blockDim.x) {
-        const float c = cs[2 * i], s = cs[2 * i + 1];
-        const float x0 = bf16_bits_to_f32(ckr[dc + 2 * i]), x1 = bf16_bits_to_f32(ckr[dc + 2 * i + 1]);
-        cache_row[dc + 2 * i] = f32_to_bf16_bits(x0 * c - x1 * s);
-        cache_row[dc + 2 * i + 1] = f32_to_bf16_bits(x0 * s + x1 * c);
+    if (i0 < dc)
+        *reinterpret_cast<uint32_t *>(cache_row + i0) = (uint32_t)f32_to_bf16_bits(x0 * r * g0) | ((uint32_t)f32_to_bf16_bits(x1 * r * g1) << 16);
+    if (threadIdx.x < dr / 2)
+        *reinterpret_cast<uint32_t *>(cache_row + dc + i0) =
+            (uint32_t)f32_to_bf16_bits(r0v * c - r1v * sn) | ((uint32_t)f32_to_bf16_bits(r0v * sn + r1v * c) << 16);
+}
+
+// Pull weight bytes into L2 ahead of the products that will stream them: one contiguous block (W_UV)
+// and `nranges` ranges of `range_bytes`, `range_stride` apart (the head of every k-split of W_O), in
+// 4 KB bulk prefetches.  Issued on the side stream while the tensor-core attention pass (which needs
+// little HBM bandwidth) runs on the main stream; the CTAs need no shared memory, so they fit beside it.
+__global__ void __launch_bounds__(128) l2_prefetch_kernel(const char *__restrict__ block, long block_bytes,
+                                                          const char *__restrict__ base, long range_stride, int nranges, long range_bytes)
+{
+    constexpr long kChunk = 4096;
+    const long block_chunks = (block_bytes + kChunk - 1) / kChunk;
+    const long chunks_per_range = (range_bytes + kChunk - 1) / kChunk;
+    const long total = block_chunks + chunks_per_range * nranges;
+    for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
+        const char *p;
+        long n;
+        if (i < block_chunks) {
+            p = block + i * kChunk;
+            n = min(kChunk, block_bytes - i * kChunk);
+        } else {
+            const long j = i - block_chunks, r = j / chunks_per_range, off = (j - r * chunks_per_range) * kChunk;
+            p = base + r * range_stride + off;
+            n = min(kChunk, range_bytes - off);
+        }
+        n &= ~15L;
+        if (n > 0) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"((uint32_t)n) : "memory");
     }
 }
 
@@ -172,44 +242,97 @@ __global__ void __launch_bounds__(128) attn_partial_simt_kernel(const uint16_t *
 // One CTA per head.  Partial (m, l, O) of split s means: o = O / l with scores shifted by m.  The
 // extra row contributes a single score.  Result: sum_s e^{m_s - M} O_s + e^{s_x - M} c_x over
 // sum_s e^{m_s - M} l_s + e^{s_x - M}.
-__global__ void __launch_bounds__(128) attn_combine_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
-                                                           AttnPartials part, int nsplit, long extra_row, int dc, int dr,
-                                                           float scale, uint16_t *__restrict__ o_bf16, float *__restrict__ o_f32)
+constexpr int kCombineThreads = 512;      // 4 groups of 128 threads; each group takes every 4th split
+
+__global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
+                                                                       AttnPartials part, int nsplit, long extra_row, int dc, int dr,
+                                                                       float scale, uint16_t *__restrict__ o_bf16, float *__restrict__ o_f32)
 {
     const int h = blockIdx.x, H = gridDim.x, dkv = dc + dr;
+    const int grp = threadIdx.x >> 7, t = threadIdx.x & 127;
     __shared__ float scratch[32];
-    __shared__ float sw[kMaxAttnSplits];
+    __shared__ float sm[kMaxAttnSplits], sl[kMaxAttnSplits], sw[kMaxAttnSplits];
+    __shared__ float4 red[3][128];
     pdl_wait_prior_grids();
+    // every split's (m, l) in one round of loads
+    for (int s = threadIdx.x; s < nsplit; s += blockDim.x) {
+        const float2 v = __ldcg(reinterpret_cast<const float2 *>(part.ml + ((size_t)s * H + h) * 2));
+        sm[s] = v.x; sl[s] = v.y;
+    }
+    // first batch of partial rows goes out before anything that needs the weights
+    const int c = 4 * t;                                           // dc == 512: four columns per thread
+    const float *src = part.O + (size_t)h * dc + c;
+    constexpr int kBatch = 8;
+    float4 v[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+        const int s = grp + 4 * u;
+        v[u] = (s < nsplit) ? __ldcg(reinterpret_cast<const float4 *>(src + (size_t)s * H * dc)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     float sx = -INFINITY;
     if (extra_row >= 0) {
         const uint16_t *qh = Q + (size_t)h * dkv, *row = cache + (size_t)extra_row * dkv;
         float acc = 0.f;
         for (int i = threadIdx.x; i < dkv; i += blockDim.x) acc = fmaf(bf16_bits_to_f32(qh[i]), bf16_bits_to_f32(row[i]), acc);
         sx = block_sum(acc, scratch) * scale;
+    } else {
+        __syncthreads();
     }
     float Mx = sx;
-    for (int s = 0; s < nsplit; ++s) Mx = fmaxf(Mx, part.ml[((size_t)s * H + h) * 2]);
-    for (int s = threadIdx.x; s < nsplit; s += blockDim.x) {
-        const float ms = part.ml[((size_t)s * H + h) * 2];
-        sw[s] = (ms == -INFINITY) ? 0.f : __expf(ms - Mx);
-    }
-    __syncthreads();
+    for (int s = 0; s < nsplit; ++s) Mx = fmaxf(Mx, sm[s]);
     const float wx = (extra_row >= 0) ? __expf(sx - Mx) : 0.f;
     float L = wx;
-    for (int s = 0; s < nsplit; ++s) L += sw[s] * part.ml[((size_t)s * H + h) * 2 + 1];
-    const float inv = 1.0f / L;
-    for (int c = threadIdx.x; c < dc; c += blockDim.x) {
-        float acc = (extra_row >= 0) ? wx * bf16_bits_to_f32(cache[(size_t)extra_row * dkv + c]) : 0.f;
-        for (int s = 0; s < nsplit; ++s) acc = fmaf(sw[s], part.O[((size_t)s * H + h) * dc + c], acc);
-        const float o = acc * inv;
-        if (o_f32) o_f32[(size_t)h * dc + c] = o;
-        if (o_bf16) o_bf16[(size_t)h * dc + c] = f32_to_bf16_bits(o);
+    for (int s = 0; s < nsplit; ++s) {                             // same order in every thread
+        const float w = (sm[s] == -INFINITY) ? 0.f : __expf(sm[s] - Mx);
+        if (threadIdx.x == 0) sw[s] = w;
+        L = fmaf(w, sl[s], L);
+    }
+    __syncthreads();
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (grp == 0 && extra_row >= 0) {
+        const uint2 rv = *reinterpret_cast<const uint2 *>(cache + (size_t)extra_row * dkv + c);
+        acc = make_float4(wx * __uint_as_float(rv.x << 16), wx * __uint_as_float(rv.x & 0xffff0000u),
+                          wx * __uint_as_float(rv.y << 16), wx * __uint_as_float(rv.y & 0xffff0000u));
+    }
+    for (int s0 = 0; s0 < nsplit; s0 += 4 * kBatch) {
+        if (s0 > 0) {
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int s = s0 + grp + 4 * u;
+                v[u] = (s < nsplit) ? __ldcg(reinterpret_cast<const float4 *>(src + (size_t)s * H * dc)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int s = s0 + grp + 4 * u;
+            const float w = (s < nsplit) ? sw[s] : 0.f;
+            acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
+            acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
+        }
+    }
+    if (grp > 0) red[grp - 1][t] = acc;
+    __syncthreads();
+    if (grp == 0) {
+#pragma unroll
+        for (int g = 0; g < 3; ++g) {                              // fixed order: deterministic
+            const float4 r = red[g][t];
+            acc.x += r.x; acc.y += r.y; acc.z += r.z; acc.w += r.w;
+        }
+        const float inv = 1.0f / L;
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        if (o_f32) *reinterpret_cast<float4 *>(o_f32 + (size_t)h * dc + c) = acc;
+        if (o_bf16)
+            *reinterpret_cast<uint2 *>(o_bf16 + (size_t)h * dc + c) =
+                make_uint2((uint32_t)f32_to_bf16_bits(acc.x) | ((uint32_t)f32_to_bf16_bits(acc.y) << 16),
+                           (uint32_t)f32_to_bf16_bits(acc.z) | ((uint32_t)f32_to_bf16_bits(acc.w) << 16));
     }
 }
 
 // ---- host -------------------------------------------------------------------------------------------
 
 static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel
+static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
+static int g_prefetch_mb = 40;       // MB of W_O pulled into L2 beside the attention pass (plus all of W_UV); 0 = off
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -256,7 +379,7 @@ static cudaError_t launch_pdl(void (*kern)(Args...), dim3 grid, dim3 block, cuda
 }
 
 static int attention_partial(const void *Q, const void *cache, int H, int n_rows, int dc, int dr, float scale,
-                             void *ws, size_t ws_bytes, cudaStream_t s)
+                             void *ws, size_t ws_bytes, cudaStream_t s, bool pdl = false)
 {
     if (!Q || !cache || !ws) return NM_ERR_INVALID_ARG;
     if (H < 1 || n_rows < 0 || dc != 512 || dr != 64) return NM_ERR_UNSUPPORTED;
@@ -265,26 +388,25 @@ static int attention_partial(const void *Q, const void *cache, int H, int n_rows
     const AttnPlan p = plan_attention(H, n_rows, dc);
     AttnPartials part = carve_partials(ws, H);
     if (g_attn_impl == 0 && H == 128) {
-        int rc = attention_partial_tc(Q, cache, part, p, n_rows, scale, s);
+        int rc = attention_partial_tc(Q, cache, part, p, n_rows, scale, s, pdl);
         if (rc != NM_ERR_UNSUPPORTED) return rc;
     }
-    attn_partial_simt_kernel<<<dim3(p.nsplit, H), 128, 0, s>>>(static_cast<const uint16_t *>(Q), static_cast<const uint16_t *>(cache),
-                                                             part, n_rows, p.rows_per_split, dc, dr, scale);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(attn_partial_simt_kernel, dim3(p.nsplit, H), dim3(128), s, pdl, static_cast<const uint16_t *>(Q),
+                               static_cast<const uint16_t *>(cache), part, n_rows, p.rows_per_split, dc, dr, scale);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (CUDA cores) launch");
 }
 
 static int attention_combine(const void *Q, const void *cache, void *o_bf16, float *o_f32, int H, int n_rows, long extra_row,
-                             int dc, int dr, float scale, void *ws, size_t ws_bytes, cudaStream_t s)
+                             int dc, int dr, float scale, void *ws, size_t ws_bytes, cudaStream_t s, bool pdl = false)
 {
     if (!Q || !cache || !ws || (!o_bf16 && !o_f32)) return NM_ERR_INVALID_ARG;
     if (H < 1 || n_rows < 0 || dc != 512 || dr != 64) return NM_ERR_UNSUPPORTED;
     if (n_rows == 0 && extra_row < 0) return NM_ERR_INVALID_ARG;
     if (ws_bytes < attention_ws_bytes(H, dc)) return NM_ERR_WORKSPACE;
     const AttnPlan p = plan_attention(H, n_rows, dc);
-    attn_combine_kernel<<<H, 128, 0, s>>>(static_cast<const uint16_t *>(Q), static_cast<const uint16_t *>(cache), carve_partials(ws, H),
-                                          p.nsplit, extra_row, dc, dr, scale, static_cast<uint16_t *>(o_bf16), o_f32);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(attn_combine_kernel, dim3(H), dim3(kCombineThreads), s, pdl, static_cast<const uint16_t *>(Q),
+                               static_cast<const uint16_t *>(cache), carve_partials(ws, H), p.nsplit, extra_row, dc, dr, scale,
+                               static_cast<uint16_t *>(o_bf16), o_f32);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention combine launch");
 }
 
@@ -336,7 +458,7 @@ static int check_params(const nm_mla_params *p)
 #define NM_LAUNCH_CHECK(what) do { cudaError_t _e = cudaGetLastError(); if (_e != cudaSuccess) return record_cuda_error(_e, what); } while (0)
 
 // Events used to fork the KV chain onto the side stream and join it again (created once per thread).
-struct StepEvents { cudaEvent_t fork = nullptr, join = nullptr; };
+struct StepEvents { cudaEvent_t fork = nullptr, join = nullptr, q_ready = nullptr; };
 static thread_local StepEvents g_events;
 
 static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
@@ -360,43 +482,77 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     if (forked && !g_events.fork) {
         NM_CUDA_TRY(cudaEventCreateWithFlags(&g_events.fork, cudaEventDisableTiming));
         NM_CUDA_TRY(cudaEventCreateWithFlags(&g_events.join, cudaEventDisableTiming));
+        NM_CUDA_TRY(cudaEventCreateWithFlags(&g_events.q_ready, cudaEventDisableTiming));
     }
 
-    // ---- Q chain, main stream ------------------------------------------------------------------------
-    NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms));
-    rmsnorm_kernel<<<1, 256, 0, ms>>>(c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
-    NM_LAUNCH_CHECK("rmsnorm launch");
-    NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms));
-    rope_kernel<<<ceil_div(H * dr / 2, 256), 256, 0, ms>>>(q + dn, q_full + dc, H, dr, dq, dkv, p->rope_cos_sin);
-    NM_LAUNCH_CHECK("rope launch");
-    // q_lat[h] = q[h, :nope] * W_UK[h], written straight into the attention operand [H][dc+dr]
-    NM_TRY(matmul_enqueue(q, p->W_UK, q_full, 1, dc, dn, H, (long)H * dq, dq, (long)dn * dc, (long)H * dkv, dkv,
-                          NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms));
+    // Programmatic dependent launch inside the step: every kernel after the first on its stream may
+    // start (and, for the products, prefetch its weights) while its predecessor drains; each waits
+    // for the predecessor before it reads activations or writes.  The first kernel on each stream
+    // keeps the ordinary dependency on whatever the caller enqueued before the step.
+    const bool pdl = g_step_pdl != 0;
+#define NM_LAUNCH(kern, grid, block, stream, ...)                                             \
+    do {                                                                                      \
+        cudaError_t _e = launch_pdl(kern, dim3(grid), dim3(block), stream, pdl, __VA_ARGS__); \
+        if (_e != cudaSuccess) return record_cuda_error(_e, #kern);                           \
+    } while (0)
 
-    // ---- KV chain (the paper's MatMul 2 and its consumers): side stream, concurrent with the attention
-    //      pass over the old rows ---------------------------------------------------------------------------
+    // ---- KV chain (the paper's MatMul 2 and its consumers) on the side stream, forked at the start so that
+    //      it shares the machine with the first products of the Q chain and is long done when the merge
+    //      needs the new cache row ---------------------------------------------------------------------------
     if (forked) {
         NM_CUDA_TRY(cudaEventRecord(g_events.fork, ms));
         NM_CUDA_TRY(cudaStreamWaitEvent(ss, g_events.fork, 0));
     }
-    NM_TRY(matmul_enqueue(p->h, p->W_DKVKR, ckr, 1, dkv, d, 1, d, 0, 0, dkv, 0, NM_BF16, lay, sws, L.side_ws_bytes, ss));
-    kv_finish_kernel<<<1, 256, 0, ss>>>(ckr, (const uint16_t *)p->gamma_kv, p->rope_cos_sin, cache + (size_t)pos * dkv, dc, dr, p->rms_eps);
-    NM_LAUNCH_CHECK("kv finish launch");
+    NM_TRY(matmul_enqueue(p->h, p->W_DKVKR, ckr, 1, dkv, d, 1, d, 0, 0, dkv, 0, NM_BF16, lay, sws, L.side_ws_bytes, ss, false));
+    NM_LAUNCH(kv_finish_kernel, 1, 256, ss, (const uint16_t *)ckr, (const uint16_t *)p->gamma_kv, p->rope_cos_sin,
+              cache + (size_t)pos * dkv, dc, dr, p->rms_eps);
     if (forked) NM_CUDA_TRY(cudaEventRecord(g_events.join, ss));
 
+    // ---- Q chain, main stream ------------------------------------------------------------------------
+    NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, !forked && pdl));
+    NM_LAUNCH(rmsnorm_kernel, 1, 256, ms, (const uint16_t *)c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
+    NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl));
+    NM_LAUNCH(rope_kernel, ceil_div(H * dr / 2, 256), 256, ms, (const uint16_t *)(q + dn), q_full + dc, H, dr, (long)dq, (long)dkv,
+              p->rope_cos_sin);
+    // q_lat[h] = q[h, :nope] * W_UK[h], written straight into the attention operand [H][dc+dr]
+    NM_TRY(matmul_enqueue(q, p->W_UK, q_full, 1, dc, dn, H, (long)H * dq, dq, (long)dn * dc, (long)H * dkv, dkv,
+                          NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms, pdl));
+
+    // ---- beside the attention pass: the side stream pulls W_UV and the head of every k-split of W_O into
+    //      L2, so that the output-side products start from L2 instead of HBM (Data Independence: the
+    //      weights do not depend on the attention result) ------------------------------------------------------
+    if (forked && g_prefetch_mb > 0 && pos > 0) {
+        NM_CUDA_TRY(cudaEventRecord(g_events.q_ready, ms));
+        NM_CUDA_TRY(cudaStreamWaitEvent(ss, g_events.q_ready, 0));
+        int kr = 0, ns = 0;
+        long rows = 0;
+        const long row_bytes = (long)d * 2;
+        if (p->W_O && lay == NM_ROW_MAJOR) {
+            matmul_row_major_split(1, d, H * dv, 1, &kr, &ns);
+            rows = ((long)g_prefetch_mb << 20) / ns / row_bytes;
+            if (rows > kr) rows = kr;
+        }
+        l2_prefetch_kernel<<<2 * kSMs, 128, 0, ss>>>((const char *)p->W_UV, (long)H * dc * dv * 2, (const char *)p->W_O,
+                                                     (long)kr * row_bytes, rows > 0 ? ns : 0, rows * row_bytes);
+        NM_LAUNCH_CHECK("L2 prefetch launch");
+    }
+
     // ---- attention over the old rows (tensor cores), main stream; the new row joins in the merge -----------
-    NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms));
+    NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms, pdl));
     if (forked) NM_CUDA_TRY(cudaStreamWaitEvent(ms, g_events.join, 0));
-    NM_TRY(attention_combine(q_full, cache, o_lat, p->o_lat_f32, H, (int)pos, pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms));
+    NM_TRY(attention_combine(q_full, cache, o_lat, p->o_lat_f32, H, (int)pos, pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms,
+                             pdl && !forked));
 
     // ---- output side -----------------------------------------------------------------------------------
     NM_TRY(matmul_enqueue(o_lat, p->W_UV, o, 1, dv, dc, H, (long)H * dc, dc, (long)dc * dv, (long)H * dv, dv,
-                          NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms));
+                          NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms, pdl));
     if (p->W_O) {
         if (p->event_before_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_before_wo, ms));
-        NM_TRY(matmul_enqueue(o, p->W_O, p->out, 1, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms));
+        NM_TRY(matmul_enqueue(o, p->W_O, p->out, 1, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms,
+                              pdl && !p->event_before_wo));
         if (p->event_after_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_after_wo, ms));
     }
+#undef NM_LAUNCH
     return NM_OK;
 }
 
@@ -485,6 +641,21 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     NM_CUDA_TRY(cudaMemcpyAsync(h_staging, h_host, (size_t)p->d * 2, cudaMemcpyHostToDevice, ms));
     NM_TRY(step_impl(&q, ms, (cudaStream_t)side_stream));
     NM_CUDA_TRY(cudaMemcpyAsync(out_host, out_staging, (size_t)p->d * 2, cudaMemcpyDeviceToHost, ms));
+    return NM_OK;
+}
+
+/* MB of W_O the decode step prefetches into L2 beside the attention pass (0 turns the prefetch off). */
+int nm_debug_set_step_prefetch(int megabytes)
+{
+    if (megabytes < 0 || megabytes > 100) return NM_ERR_INVALID_ARG;
+    g_prefetch_mb = megabytes;
+    return NM_OK;
+}
+
+/* Chain the kernels of the decode step with programmatic dependent launch (default on). */
+int nm_debug_set_step_pdl(int enable)
+{
+    g_step_pdl = enable ? 1 : 0;
     return NM_OK;
 }
 

@@ -25,6 +25,6 @@ AttnPlan plan_attention(int H, int n_rows, int kv_lora);
 // Tensor-core (tcgen05 / TMEM) pass over the rows of each split.  Returns NM_ERR_UNSUPPORTED when
 // the shape is not one it takes (the caller then uses the CUDA-core kernel).
 int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows,
-                         float scale, cudaStream_t stream);
+                         float scale, cudaStream_t stream, bool programmatic_launch);
 
 }  // namespace nm

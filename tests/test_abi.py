@@ -60,12 +60,14 @@ def test_workspace_bound_covers_every_plan(lib):
     lib.nm_debug_set_plan(0, 0)
 
 
-def test_heuristic_fills_the_gpu_for_the_paper_shape(lib):
+def test_heuristic_spreads_the_paper_shape_over_the_gpu(lib):
     out = (ctypes.c_int * 6)()
     lib.nm_debug_set_plan(0, 0)
     for layout in (0, 1):
         assert lib.nm_debug_get_plan(1, 576, 7168, 1, 1, layout, 1, out) == 0
-        assert out[5] >= 148, "MatMul 2 shape must cover every SM"
+        # measured optimum on B200 is 108-144 CTAs: enough splits to use most SMs, few enough that
+        # the gather of the partial sums stays short
+        assert 100 <= out[5] <= 320, "MatMul 2 shape must be split over most of the 148 SMs"
     # a shape that cannot use 16-byte loads falls back to the scalar kernel, unsplit
     assert lib.nm_debug_get_plan(1, 577, 7168, 1, 1, 0, 0, out) == 0
     assert out[0] == 2 and out[2] == 1

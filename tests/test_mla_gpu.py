@@ -273,6 +273,50 @@ def test_decode_step_without_wo_and_repeatable(nm, weights):
         assert torch.equal(t1[k], t2[k]), f"{k}: two runs differ"
 
 
+def test_decode_step_same_bits_with_and_without_programmatic_launch(nm, weights, ref1024):
+    w, dw = weights
+    h, cache_ref, r = ref1024
+    cache_in = gen.mla_cache(1024, DIMS, seed=4200)
+    t1 = run_step(nm, dw, h, cache_in, 1024)
+    nm.nm_debug_set_step_pdl(False)
+    try:
+        t2 = run_step(nm, dw, h, cache_in, 1024)
+    finally:
+        nm.nm_debug_set_step_pdl(True)
+    for k in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o", "out", "kv_cache"):
+        assert torch.equal(t1[k], t2[k]), k
+    check_step(t2, r, cache_ref, 1024)
+
+
+def test_decode_step_back_to_back_steps_do_not_interfere(nm, weights, ref1024):
+    # several steps enqueued without host synchronisation in between: programmatic launch lets a
+    # step's first kernels overlap the previous step's tail; results must not change
+    w, dw = weights
+    h, cache_ref, r = ref1024
+    H, dc, dr, dn, dv, d, ql = (DIMS[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d", "q_lora"))
+    t = dict(dw)
+    t["h"] = to_dev(h)
+    t["kv_cache"] = to_dev(gen.mla_cache(1024, DIMS, seed=4200))
+    t["rope_cos_sin"] = rope_row(nm, 1023)
+    t["out"] = torch.zeros(d, dtype=torch.int16, device="cuda")
+    p = nm.mla_params(DIMS, 1024, t)
+    ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p))
+    p = nm.mla_params(DIMS, 1024, t, workspace=ws)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = []
+    with torch.cuda.stream(main):
+        for _ in range(6):
+            nm.nm_mla_decode_step(p, main, side)
+            outs.append(t["out"].clone())
+    torch.cuda.synchronize()
+    nm.nm_check_status()
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0])
+    ref = f64(r["out"])
+    assert np.all(np.abs(dev_bits_to_f64(outs[0]) - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
+
+
 def test_decode_step_host_operands(nm, weights, ref1024):
     w, dw = weights
     h, cache_ref, r = ref1024

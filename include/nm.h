@@ -261,6 +261,10 @@ int nm_debug_set_plan(int tile_n, int nsplit);
 /* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel instead
  * of the TMA ring) and the ring depth in stages (0 heuristic). */
 int nm_debug_set_kernel(int kind, int stages);
+/* Attention kernel: device buffer of 12 uint64 that receives phase timestamps (ns) of CTA (0,0):
+ * start, set-up done, Q landed, first tile landed, scores ready, P written, last P*V done, after
+ * cluster barrier 1, O parked in shared memory, after barrier 2, cluster sum written, end.  NULL = off. */
+int nm_debug_set_attention_trace(void *device_buffer);
 /* Decode step: MB of W_O prefetched into L2 beside the attention pass (default 40, 0 = off). */
 int nm_debug_set_step_prefetch(int megabytes);
 /* Decode step: chain its kernels with programmatic dependent launch (default 1) or not (0). */

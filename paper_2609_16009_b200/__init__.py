@@ -90,6 +90,7 @@ _lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _v
 _lib.nm_debug_set_attention.argtypes = [_i]
 _lib.nm_debug_set_step_pdl.argtypes = [_i]
 _lib.nm_debug_set_step_prefetch.argtypes = [_i]
+_lib.nm_debug_set_attention_trace.argtypes = [_vp]
 
 
 def _check(status: int, where: str) -> None:
@@ -285,6 +286,10 @@ def nm_mla_decode_step_host(p: MlaParams, h_host, out_host, h_staging, out_stagi
     ss = ms if side_stream is None else _stream(side_stream)
     _check(_lib.nm_mla_decode_step_host(C.byref(p), _ptr(h_host), _ptr(out_host), _ptr(h_staging), _ptr(out_staging),
                                         ms, ss), "nm_mla_decode_step_host")
+
+
+def nm_debug_set_attention_trace(buf) -> None:
+    _check(_lib.nm_debug_set_attention_trace(_ptr(buf)), "nm_debug_set_attention_trace")
 
 
 def nm_debug_set_step_prefetch(megabytes: int) -> None:

@@ -11,7 +11,14 @@
 // the MMA unit; the accumulators never leave TMEM until the split is finished.  The 512 output
 // columns do not fit TMEM next to S, so two CTAs share a split, each owning 256 columns.  The running
 // maximum is updated lazily: O is rescaled only when a row maximum grows by more than 2^8, so the
-// usual tile costs no pass over the accumulator.  Splits are merged by attn_combine_kernel.
+// usual tile costs no pass over the accumulator.
+//
+// The CTAs of kAttnCluster consecutive splits form a thread-block cluster and merge their results
+// through distributed shared memory before anything goes to global memory: each CTA rescales its
+// O rows to the cluster-wide maximum and parks them in its own shared memory (the Q buffer is free
+// by then), then each CTA sums one quarter of the heads over all peers and writes that quarter.
+// Global partial traffic and the work of the final merge (attn_combine_kernel) shrink by the
+// cluster size.
 //
 // Roles: warp 0 lane 0 issues TMA, warp 1 owns TMEM and its lane 0 issues the MMAs, warps 2-5 hold
 // one head per thread.  Every wait is bounded (mbar_wait); on expiry the CTA raises the status word,
@@ -38,6 +45,8 @@ constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 0, kColS = 256, kColP = 320, kColPlo = 352;
 constexpr float kLazyThreshold = 8.0f;    // log2 units
+constexpr int kCl = kAttnCluster;          // CTAs (splits) per cluster
+constexpr int kHeadsPerRank = kHeads / kCl;
 
 // Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
@@ -106,6 +115,38 @@ __device__ __forceinline__ float fast_exp2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    __syncwarp();                                                  // the aligned forms want the warp converged
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in the peer CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t peer_smem(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local_addr), "r"(rank));
+    return a;
+}
+__device__ __forceinline__ float4 ld_peer_f4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 ld_peer_f2(uint32_t addr)
+{
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     uint32_t r;
@@ -115,8 +156,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, AttnPartials part,
-               int n_rows, int rows_per_split, float scale_log2, unsigned *status)
+               int n_rows, int rows_per_split, float scale_log2, unsigned *status, unsigned long long *trace)
 {
+    // Optional phase timestamps (ns) of CTA (0,0), for tuning: trace[i] is written when non-null.
+#define NM_TRACE(i) do { if (trace && blockIdx.x == 0 && blockIdx.y == 0) trace[i] = global_timer_ns(); } while (0)
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;            // swizzle atoms want 1024-byte alignment
@@ -127,13 +170,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                    bar_s = smem_u32(bars + 3), bar_p = smem_u32(bars + 4), bar_o = smem_u32(bars + 5);
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ __align__(8) float s_ml[kHeads][2];                // this split's (m in log2 units, l) per head
+    __shared__ float s_w[kCl][kHeadsPerRank];                     // weights of the slots in the final sum
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sp = blockIdx.x, half = blockIdx.y;
     const int r0 = sp * rows_per_split, r1 = min(n_rows, r0 + rows_per_split);
-    const int ntiles = ceil_div(r1 - r0, kT);
+    const int ntiles = (r1 > r0) ? ceil_div(r1 - r0, kT) : 0;      // 0 for the padding CTAs of the last cluster
 
     if (tid == 0) {
+        NM_TRACE(0);
         s_abort = 0;
         mbar_init(bar_q, 1); mbar_init(bar_kv_full, 1); mbar_init(bar_kv_empty, 1);
         mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
@@ -148,6 +194,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
     pdl_launch_dependents();
+    const uint32_t rank = cluster_rank();
+    const int cluster_id = sp / kCl;
+    float m_own = -INFINITY, l_own = 0.f;                         // softmax threads: this split's (m, l)
 
     if (warp == 0) {
         // ---------------- TMA producer --------------------------------------------------------------
@@ -162,8 +211,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 for (int c = 0; c < kKBlocks; ++c) tma_load_2d(kv_addr + c * kKVBlockBytes, &map_kv, c * 64, r0, bar_kv_full, stream);
             }
             pdl_wait_prior_grids();
-            mbar_arrive_expect_tx(bar_q, kQBytes);
-            for (int c = 0; c < kKBlocks; ++c) tma_load_2d(q_addr + c * kQBlockBytes, &map_q, c * 64, 0, bar_q, keep);
+            if (ntiles > 0) {                                      // a padding CTA of the last cluster loads nothing
+                mbar_arrive_expect_tx(bar_q, kQBytes);
+                for (int c = 0; c < kKBlocks; ++c) tma_load_2d(q_addr + c * kQBlockBytes, &map_q, c * 64, 0, bar_q, keep);
+            }
             for (int t = 1; t < ntiles; ++t) {
                 if (!mbar_try_wait(bar_kv_empty, (t - 1) & 1) && !mbar_wait(bar_kv_empty, (t - 1) & 1, &s_abort, status)) break;
                 mbar_arrive_expect_tx(bar_kv_full, kKVBytes);
@@ -175,10 +226,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // ---------------- MMA issuer ---------------------------------------------------------------
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(kT, false), idesc_o = instr_desc(kDvHalf, true);
-            mbar_wait(bar_q, 0, &s_abort, status);
+            NM_TRACE(1);
+            if (ntiles > 0) mbar_wait(bar_q, 0, &s_abort, status);
+            NM_TRACE(2);
             for (int t = 0; t < ntiles; ++t) {
                 mbar_wait(bar_kv_full, t & 1, &s_abort, status);
                 tc_fence_after();
+                if (t == 0) NM_TRACE(3);
                 for (int c = 0; c < kKBlocks; ++c)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
@@ -206,6 +260,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int t = 0; t < ntiles; ++t) {
             mbar_wait(bar_s, t & 1, &s_abort, status);
             tc_fence_after();
+            if (t == 0 && tid == 64) NM_TRACE(4);
             uint32_t sr[2][32];
             tmem_ld32(lane_base + kColS, sr[0]);
             tmem_ld32(lane_base + kColS + 32, sr[1]);
@@ -252,38 +307,111 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p);
+            if (t == 0 && tid == 64) NM_TRACE(5);
         }
-        // epilogue: unnormalised O (this CTA's 256 columns) and (m, l) to the partial buffers
+        // the last P*V must have landed before O is read; then publish this split's (m, l)
         if (ntiles > 0) {
             mbar_wait(bar_o, (ntiles - 1) & 1, &s_abort, status);
             tc_fence_after();
-            float *dst = part.O + ((size_t)sp * kHeads + head) * kDv + half * kDvHalf;
+        }
+        if (tid == 64) NM_TRACE(6);
+        m_own = m_used; l_own = l;
+    }
+
+    // ---- merge of the cluster's splits through distributed shared memory -----------------------------------
+    // Each CTA parks its (unscaled) O rows and its (m, l) in its own shared memory as soon as its last
+    // P*V is done (the Q tile is free by then; layout [head][64 float4], the float4 index XOR-ed with
+    // (head & 7) so that neither the row-per-thread writes nor the row-contiguous reads conflict).
+    // After one cluster barrier, rank r combines heads [32r, 32r+32) over all peers - weights
+    // 2^(m_peer - max m) - reading the peers' rows with many loads in flight, and writes one partial
+    // per cluster.  A last barrier keeps every CTA's shared memory alive until its peers have read it.
+    if (warp >= 2) {
+        const int quad = warp & 3, head = quad * 32 + lane;
+        const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
+        s_ml[head][0] = (ntiles > 0) ? m_own : -INFINITY;
+        s_ml[head][1] = l_own;
+        if (ntiles > 0) {
             for (int c = 0; c < kDvHalf / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(lane_base + kColO + c * 32, o);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; i += 4)
-                    *reinterpret_cast<uint4 *>(dst + c * 32 + i) = make_uint4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+                for (int i = 0; i < 32; i += 4) {
+                    const uint32_t q4 = (uint32_t)(c * 8 + i / 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(q_addr + (uint32_t)(head * 64 + (q4 ^ (head & 7u))) * 16u),
+                                 "r"(o[i]), "r"(o[i + 1]), "r"(o[i + 2]), "r"(o[i + 3]) : "memory");
+                }
             }
-            if (half == 0) {
-                part.ml[((size_t)sp * kHeads + head) * 2] = m_used * 0.6931471805599453f;   // back to natural-log units
-                part.ml[((size_t)sp * kHeads + head) * 2 + 1] = l;
+        }
+        if (tid == 64) NM_TRACE(7);
+    }
+    cluster_sync_all();                                            // every peer's rows and (m, l) are parked
+    if (tid == 64) NM_TRACE(8);
+    if (warp >= 2) {
+        const int t = tid - 64;                                    // 0..127
+        if (t < kCl * kHeadsPerRank) {                             // weight of peer r for owned head hl
+            const int hl = t % kHeadsPerRank, r = t / kHeadsPerRank, head = (int)rank * kHeadsPerRank + hl;
+            float pm[kCl], pl[kCl], M = -INFINITY;
+#pragma unroll
+            for (int rr = 0; rr < kCl; ++rr) {
+                const float2 v = ld_peer_f2(peer_smem(smem_u32(&s_ml[head][0]), rr));
+                pm[rr] = v.x; pl[rr] = v.y;
+                M = fmaxf(M, v.x);
+            }
+            s_w[r][hl] = (pm[r] == -INFINITY) ? 0.f : fast_exp2(pm[r] - M);
+            if (r == 0 && half == 0) {
+                float Ltot = 0.f;
+#pragma unroll
+                for (int rr = 0; rr < kCl; ++rr) Ltot = fmaf(pm[rr] == -INFINITY ? 0.f : fast_exp2(pm[rr] - M), pl[rr], Ltot);
+                part.ml[((size_t)cluster_id * kHeads + head) * 2] = M * 0.6931471805599453f;     // natural-log units
+                part.ml[((size_t)cluster_id * kHeads + head) * 2 + 1] = Ltot;
+            }
+        }
+        named_barrier_sync(1, 128);
+        if (tid == 64) NM_TRACE(9);
+        constexpr int kIters = kHeadsPerRank * 64 / 128, kBatch = 8;
+        for (int i0 = 0; i0 < kIters; i0 += kBatch) {
+            float4 v[kBatch][kCl];
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {                     // kBatch * kCl remote loads in flight
+                const int idx = t + 128 * (i0 + b);
+                const int hl = idx / 64, q4 = idx % 64, head = (int)rank * kHeadsPerRank + hl;
+                const uint32_t local = q_addr + (uint32_t)(head * 64 + (q4 ^ (head & 7))) * 16u;
+#pragma unroll
+                for (int r = 0; r < kCl; ++r)
+                    v[b][r] = (s_w[r][hl] != 0.f) ? ld_peer_f4(peer_smem(local, r)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const int idx = t + 128 * (i0 + b);
+                const int hl = idx / 64, q4 = idx % 64, head = (int)rank * kHeadsPerRank + hl;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int r = 0; r < kCl; ++r) {                    // rank order: deterministic
+                    const float w = s_w[r][hl];
+                    acc.x = fmaf(w, v[b][r].x, acc.x); acc.y = fmaf(w, v[b][r].y, acc.y);
+                    acc.z = fmaf(w, v[b][r].z, acc.z); acc.w = fmaf(w, v[b][r].w, acc.w);
+                }
+                *reinterpret_cast<float4 *>(part.O + ((size_t)cluster_id * kHeads + head) * kDv + half * kDvHalf + q4 * 4) = acc;
             }
         }
     }
+    if (tid == 64) NM_TRACE(10);
+    cluster_sync_all();                                            // peers are done reading this CTA's shared memory
 
-    // ---- teardown: everyone meets, TMEM goes back ---------------------------------------------------------
+    // ---- teardown: TMEM goes back ---------------------------------------------------------------------------
     tc_fence_before();
     __syncthreads();
     if (s_abort && tid == 0) {
         // a wait expired: give copies already issued a bounded chance to land before the CTA exits
-        for (int i = 0; i < (1 << 16) && !mbar_try_wait(bar_q, 0); ++i) {}
+        for (int i = 0; i < (1 << 16) && ntiles > 0 && !mbar_try_wait(bar_q, 0); ++i) {}
     }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+    if (tid == 0) NM_TRACE(11);
+#undef NM_TRACE
 }
 
 // Tensor maps: bf16 [rows][576], boxes of 64 columns (128 bytes, the swizzle span) x box_rows rows.
@@ -302,6 +430,9 @@ bool encode_rows_map(CUtensorMap *map, const void *ptr, int rows, int box_rows)
 
 }  // namespace
 
+static unsigned long long *g_attn_trace = nullptr;
+void set_attention_trace(unsigned long long *p) { g_attn_trace = p; }
+
 int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows, float scale,
                          cudaStream_t stream, bool programmatic_launch)
 {
@@ -319,17 +450,19 @@ int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, At
     }
     const float scale_log2 = scale * 1.4426950408889634f;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan.nsplit, 2);
+    cfg.gridDim = dim3(ceil_div(plan.nsplit, kCl) * kCl, 2);      // padded to whole clusters; padding CTAs have no rows
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kCl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = programmatic_launch ? 1 : 0;
+    cfg.numAttrs = programmatic_launch ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, map_q, map_kv, part, n_rows, plan.rows_per_split, scale_log2,
-                                       device_status_ptr());
+                                       device_status_ptr(), g_attn_trace);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (tensor cores) launch");
 }
 

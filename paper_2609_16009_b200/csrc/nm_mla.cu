@@ -8,6 +8,8 @@
 
 namespace nm {
 
+static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel
+
 // ---- small vector kernels ---------------------------------------------------------------------------
 
 __device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
@@ -330,25 +332,27 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 
 // ---- host -------------------------------------------------------------------------------------------
 
-static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel
 static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
 static int g_prefetch_mb = 40;       // MB of W_O pulled into L2 beside the attention pass (plus all of W_UV); 0 = off
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-AttnPlan plan_attention(int H, int n_rows, int kv_lora)
+AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int kv_lora)
 {
     AttnPlan p{};
-    (void)H; (void)kv_lora;
+    (void)kv_lora;
     const int tiles = ceil_div(n_rows > 0 ? n_rows : 0, kAttnTileRows);
-    // 64 splits x 2 column halves = 128 CTAs: one wave of the 148 SMs, leaving a few for the narrow
-    // products that run beside the attention pass
+    // 64 splits x 2 column halves = 128 CTAs: one wave of the 148 SMs
     constexpr int kSplitTarget = 64;
     int nsplit = tiles < kSplitTarget ? tiles : kSplitTarget;
     if (nsplit < 1) nsplit = (n_rows > 0) ? 1 : 0;
-    p.nsplit = nsplit;
     p.rows_per_split = nsplit ? ceil_div(tiles, nsplit) * kAttnTileRows : 0;
     p.nsplit = p.rows_per_split ? ceil_div(n_rows, p.rows_per_split) : 0;
+    // The tensor-core kernel takes 128 heads and 16-byte aligned operands (TMA); both passes of an
+    // attention call derive the same answer from the same arguments.
+    p.tensor_core = (g_attn_impl == 0 && H == 128 && n_rows > 0 && (((uintptr_t)Q | (uintptr_t)cache) & 15u) == 0 &&
+                     tensor_map_encoder() != nullptr) ? 1 : 0;
+    p.npartial = p.tensor_core ? ceil_div(p.nsplit, kAttnCluster) : p.nsplit;
     return p;
 }
 
@@ -385,12 +389,9 @@ static int attention_partial(const void *Q, const void *cache, int H, int n_rows
     if (H < 1 || n_rows < 0 || dc != 512 || dr != 64) return NM_ERR_UNSUPPORTED;
     if (ws_bytes < attention_ws_bytes(H, dc)) return NM_ERR_WORKSPACE;
     if (n_rows == 0) return NM_OK;
-    const AttnPlan p = plan_attention(H, n_rows, dc);
+    const AttnPlan p = plan_attention(Q, cache, H, n_rows, dc);
     AttnPartials part = carve_partials(ws, H);
-    if (g_attn_impl == 0 && H == 128) {
-        int rc = attention_partial_tc(Q, cache, part, p, n_rows, scale, s, pdl);
-        if (rc != NM_ERR_UNSUPPORTED) return rc;
-    }
+    if (p.tensor_core) return attention_partial_tc(Q, cache, part, p, n_rows, scale, s, pdl);
     cudaError_t e = launch_pdl(attn_partial_simt_kernel, dim3(p.nsplit, H), dim3(128), s, pdl, static_cast<const uint16_t *>(Q),
                                static_cast<const uint16_t *>(cache), part, n_rows, p.rows_per_split, dc, dr, scale);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (CUDA cores) launch");
@@ -403,9 +404,9 @@ static int attention_combine(const void *Q, const void *cache, void *o_bf16, flo
     if (H < 1 || n_rows < 0 || dc != 512 || dr != 64) return NM_ERR_UNSUPPORTED;
     if (n_rows == 0 && extra_row < 0) return NM_ERR_INVALID_ARG;
     if (ws_bytes < attention_ws_bytes(H, dc)) return NM_ERR_WORKSPACE;
-    const AttnPlan p = plan_attention(H, n_rows, dc);
+    const AttnPlan p = plan_attention(Q, cache, H, n_rows, dc);
     cudaError_t e = launch_pdl(attn_combine_kernel, dim3(H), dim3(kCombineThreads), s, pdl, static_cast<const uint16_t *>(Q),
-                               static_cast<const uint16_t *>(cache), carve_partials(ws, H), p.nsplit, extra_row, dc, dr, scale,
+                               static_cast<const uint16_t *>(cache), carve_partials(ws, H), p.npartial, extra_row, dc, dr, scale,
                                static_cast<uint16_t *>(o_bf16), o_f32);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention combine launch");
 }
@@ -539,6 +540,9 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
 
     // ---- attention over the old rows (tensor cores), main stream; the new row joins in the merge -----------
     NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms, pdl));
+    // The merge needs the cache row the KV chain wrote.  Joining here also keeps the merge from being
+    // launched early: its CTAs could not share an SM with the attention CTAs (registers) and would
+    // only hold up the prefetch kernel in the block scheduler.
     if (forked) NM_CUDA_TRY(cudaStreamWaitEvent(ms, g_events.join, 0));
     NM_TRY(attention_combine(q_full, cache, o_lat, p->o_lat_f32, H, (int)pos, pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms,
                              pdl && !forked));
@@ -641,6 +645,13 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     NM_CUDA_TRY(cudaMemcpyAsync(h_staging, h_host, (size_t)p->d * 2, cudaMemcpyHostToDevice, ms));
     NM_TRY(step_impl(&q, ms, (cudaStream_t)side_stream));
     NM_CUDA_TRY(cudaMemcpyAsync(out_host, out_staging, (size_t)p->d * 2, cudaMemcpyDeviceToHost, ms));
+    return NM_OK;
+}
+
+/* Device buffer of 12 uint64 that receives phase timestamps of the attention kernel (NULL = off). */
+int nm_debug_set_attention_trace(void *device_buffer)
+{
+    set_attention_trace(static_cast<unsigned long long *>(device_buffer));
     return NM_OK;
 }
 

@@ -131,6 +131,9 @@ class MlaStep:
         self.bytes_per_step = algorithmic_bytes(self.specs) + self.kv_bytes
         self.dominant = "W_O product (nm_row_tma_kernel, K=16384, N=7168, M=1)"
         self.dominant_bytes = algorithmic_bytes([s for s in self.specs if s[0] == "W_O"])
+        # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this shape, from
+        # the ncu capture summarised in profiles/ncu_nm_row_tma_WO_M1_K16384_N7168.txt
+        self.dominant_traffic = 234_948_352 + 3_600_128
         self.launches_per_step = 11
         self.h2d = d * 2
         self.d2h = d * 2
@@ -154,12 +157,111 @@ class MlaStep:
         self.nm.nm_mla_decode_step_host(self.p, self.h_host, self.out_host, self.t["h"], self.t["out"], stream, self.side)
 
 
-def make_workload(kind, nm, device, seq_len):
-    if kind == "projections":
+class SingleProduct:
+    """One narrow product C[MxN] = A[MxK] * B[KxN] (bf16), B rotated through copies that together
+    exceed 512 MB so that every launch streams from HBM.  For kernel-level captures."""
+
+    name = "matmul"
+
+    def __init__(self, nm, device, M, K, N, layout):
+        self.nm, self.M, self.K, self.N, self.layout = nm, M, K, N, layout
+        nbytes = K * N * 2
+        self.R = max(2, min(64, (1 << 29) // nbytes + 1))
+        self.B = (torch.randn(self.R, K * N, device=device) * 0.02).to(torch.bfloat16)
+        self.A = torch.randn(M * K, device=device).to(torch.bfloat16)
+        self.C = torch.empty(M * N, device=device, dtype=torch.bfloat16)
+        self.A_host = self.A.cpu().pin_memory()
+        self.C_host = torch.empty(M * N, dtype=torch.bfloat16).pin_memory()
+        self.ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(M, N, K), device=device)
+        self.i = 0
+        self.bytes_per_step = (K * N + M * K + M * N) * 2
+        self.dominant = f"narrow product M={M} K={K} N={N}"
+        self.dominant_bytes = self.bytes_per_step
+        self.launches_per_step = 1
+        self.h2d, self.d2h = M * K * 2, M * N * 2
+
+    def describe(self):
+        return {"workload": f"single narrow product M={self.M} K={self.K} N={self.N} bf16, B {'column' if self.layout else 'row'}-major",
+                "l2": f"B rotates through {self.R} copies (> 512 MB in total): every launch reads HBM"}
+
+    def step(self, stream, dom_events=None):
+        self.i = (self.i + 1) % self.R
+        if dom_events is not None:
+            dom_events[0].record(stream)
+        self.nm.nm_matmul_ws(self.A, self.B[self.i], self.C, self.M, self.N, self.K, self.nm.BF16, self.layout, self.ws, stream)
+        if dom_events is not None:
+            dom_events[1].record(stream)
+
+    def step_e2e(self, stream):
+        self.i = (self.i + 1) % self.R
+        self.nm.nm_matmul_host(self.A_host, self.B[self.i], self.C_host, self.A, self.C, self.M, self.N, self.K, self.nm.BF16,
+                               self.layout, self.ws, stream)
+
+
+class AttentionOnly:
+    """The latent-attention pass alone (tcgen05 kernel + merge) over seq_len cache rows."""
+
+    name = "attention"
+
+    def __init__(self, nm, device, seq_len):
+        self.nm, self.S = nm, seq_len
+        H, dc, dr = DIMS["H"], DIMS["kv_lora"], DIMS["rope"]
+        self.Q = (torch.randn(H, dc + dr, device=device) * 0.3).to(torch.bfloat16)
+        self.cache = torch.randn(seq_len, dc + dr, device=device).to(torch.bfloat16)
+        self.o = torch.empty(H * dc, dtype=torch.bfloat16, device=device)
+        self.ws = torch.empty(nm.nm_mla_attention_workspace_bytes(H, seq_len, dc), dtype=torch.uint8, device=device)
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        self.bytes_per_step = (seq_len + H) * (dc + dr) * 2 + H * dc * 2
+        self.flops_per_step = 2 * H * seq_len * (dc + dr + dc)
+        self.dominant = "attn_tc_kernel"
+        self.dominant_bytes = self.bytes_per_step
+        self.launches_per_step = 2
+        self.h2d = self.d2h = 0
+
+    def describe(self):
+        return {"workload": f"latent attention pass alone, 128 heads, seq_len {self.S}", "l2": "256 MB written between launches"}
+
+    def step(self, stream, dom_events=None):
+        H, dc, dr = DIMS["H"], DIMS["kv_lora"], DIMS["rope"]
+        self.flush.fill_(1)
+        if dom_events is not None:
+            dom_events[0].record(stream)
+        self.nm.nm_mla_attention(self.Q, self.cache, self.o, None, H, self.S, -1, dc, dr, (DIMS["nope"] + dr) ** -0.5, self.ws, stream)
+        if dom_events is not None:
+            dom_events[1].record(stream)
+
+    step_e2e = step
+
+
+def make_workload(args, nm, device):
+    if args.workload == "projections":
         return ProjectionChain(nm, device)
-    if kind == "mla":
-        return MlaStep(nm, device, seq_len)
-    raise SystemExit(f"unknown workload {kind}")
+    if args.workload == "mla":
+        return MlaStep(nm, device, args.seq_len)
+    if args.workload == "matmul":
+        M, K, N = (int(x) for x in args.mkn.split(","))
+        return SingleProduct(nm, device, M, K, N, 1 if args.layout == "col" else 0)
+    if args.workload == "attention":
+        return AttentionOnly(nm, device, args.seq_len)
+    raise SystemExit(f"unknown workload {args.workload}")
+
+
+def print_timeline(wl, stream, steps=6):
+    """Kernel timeline of one step (start offset, duration, name) from CUPTI through torch.profiler:
+    shows which kernels overlap (side-stream work beside the main stream, programmatic launches)."""
+    from torch.profiler import ProfilerActivity, profile
+    with profile(activities=[ProfilerActivity.CUDA]) as prof:
+        for _ in range(steps):
+            wl.step(stream)
+        torch.cuda.synchronize()
+    evs = sorted((e for e in prof.events() if e.device_type == torch.autograd.DeviceType.CUDA), key=lambda e: e.time_range.start)
+    per = len(evs) // steps
+    k0 = (steps - 2) * per
+    t0 = evs[k0].time_range.start
+    print(f"# kernel timeline of one step ({per} kernels), microseconds from the step's first kernel")
+    for e in evs[k0:k0 + per]:
+        print(f"{e.time_range.start - t0:9.1f}  +{e.time_range.end - e.time_range.start:7.1f}  {e.name[:90]}")
+    print(f"# next step starts at {evs[k0 + per].time_range.start - t0:.1f}")
 
 
 def matmul_sweep(nm, device):
@@ -326,7 +428,10 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="mla", choices=["mla", "projections"])
+    ap.add_argument("--workload", default="mla", choices=["mla", "projections", "matmul", "attention"])
+    ap.add_argument("--mkn", default="1,16384,7168", help="M,K,N of --workload matmul")
+    ap.add_argument("--layout", default="row", choices=["row", "col"])
+    ap.add_argument("--timeline", action="store_true", help="print the kernel timeline of one step and exit")
     ap.add_argument("--sweep", action="store_true", help="also report GB/s of single narrow products vs M")
     ap.add_argument("--seq-len", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -352,8 +457,15 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     import paper_2609_16009_b200 as nm
-    wl = make_workload(args.workload, nm, device, args.seq_len)
+    wl = make_workload(args, nm, device)
     stream = torch.cuda.Stream(device)
+    if args.timeline:
+        with torch.cuda.stream(stream):
+            for _ in range(max(args.warmup, 10)):
+                wl.step(stream)
+            torch.cuda.synchronize()
+            print_timeline(wl, stream)
+        return
 
     def barrier():
         torch.cuda.synchronize()
@@ -417,7 +529,8 @@ def main():
                 "gpu_launches": wl.launches_per_step * args.steps,
                 "clocks": clocks,
                 "roofline": {"bound": "hbm", "kernel": wl.dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                             "frac": achieved / peak, "peak_kind": peak_kind, "algorithmic_bytes": wl.dominant_bytes,
+                             "traffic": getattr(wl, "dominant_traffic", None),
                              "us_per_launch": dom_ms * 1e3}}
         if args.sweep:
             line["narrow_matmul_vs_M"] = matmul_sweep(nm, device)

@@ -253,13 +253,22 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
  */
 int nm_set_programmatic_launch(int enable);
 
+/*
+ * Row-major bf16 products with M >= m and at least 32 MB of weights run on the tensor cores with the
+ * operands swapped (weights as the MMA's M dimension, token rows as its N dimension): from M = 3 on
+ * the CUDA-core path is bound by fp32 FMA issue rather than by HBM.  Products are exact and
+ * accumulation is fp32 on both paths.  Default 3; pass 17 to keep every M on the CUDA cores (the
+ * paper's placement), 1 to use the tensor cores from M = 1.
+ */
+int nm_set_tensor_core_min_m(int m);
+
 /* ---- tuning aids (sweeps and tests; not needed for normal use) --------------------------------- */
 
 /* Override the tiling heuristic: columns per CTA tile of the row-major kernel and number of
  * k-splits; 0 restores the heuristic.  Values are clamped to what the workspace bound covers. */
 int nm_debug_set_plan(int tile_n, int nsplit);
-/* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel instead
- * of the TMA ring) and the ring depth in stages (0 heuristic). */
+/* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel; 3 TMA-ring
+ * CUDA-core kernel; 4 swap-AB tensor-core kernel) and the ring depth in stages (0 heuristic). */
 int nm_debug_set_kernel(int kind, int stages);
 /* Attention kernel: device buffer of 12 uint64 that receives phase timestamps (ns) of CTA (0,0):
  * start, set-up done, Q landed, first tile landed, scores ready, P written, last P*V done, after

@@ -59,6 +59,7 @@ _lib.nm_matmul_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp
 _lib.nm_matmul_static.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]
 _lib.nm_debug_set_plan.argtypes = [_i, _i]
 _lib.nm_debug_set_kernel.argtypes = [_i, _i]
+_lib.nm_set_tensor_core_min_m.argtypes = [_i]
 _lib.nm_set_programmatic_launch.argtypes = [_i]
 _lib.nm_check_status.argtypes = [_vp]
 _lib.nm_debug_get_plan.argtypes = [_i, _i, _i, _i, _i, _i, _i, C.POINTER(_i)]
@@ -186,6 +187,10 @@ def nm_matmul_static(A, B, C_out, M, N, K, dtype, layout_B, stream=None) -> None
 
 def nm_debug_set_plan(tile_n: int = 0, nsplit: int = 0) -> None:
     _check(_lib.nm_debug_set_plan(tile_n, nsplit), "nm_debug_set_plan")
+
+
+def nm_set_tensor_core_min_m(m: int) -> None:
+    _check(_lib.nm_set_tensor_core_min_m(int(m)), "nm_set_tensor_core_min_m")
 
 
 def nm_debug_set_kernel(kind: int = -1, stages: int = 0) -> None:

@@ -5,6 +5,7 @@
 
 #include "nm_matmul_kernels.cuh"
 #include "nm_row_tma.cuh"
+#include "nm_row_tc.cuh"
 
 namespace nm {
 
@@ -35,8 +36,9 @@ static void *g_ws = nullptr;
 static size_t g_ws_bytes = 0;
 static int g_force_tn = 0, g_force_split = 0, g_force_kind = -1, g_force_stages = 0;
 static int g_use_pdl = 0;
+static int g_tc_min_m = 3;        // row-major bf16 products with M >= this (and >= 32 MB of weights) go to the swap-AB tensor-core kernel
 
-enum PlanKind { kRowVec = 0, kColVec = 1, kGeneric = 2, kRowTma = 3 };
+enum PlanKind { kRowVec = 0, kColVec = 1, kGeneric = 2, kRowTma = 3, kRowTc = 4 };
 
 struct Plan {
     PlanKind kind;
@@ -53,7 +55,7 @@ static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t
 // per cent of |B|.
 // Plan for the TMA-ring kernel, from measurements on B200 (sweeps over tile width, k-splits and ring
 // depth for the decode step's shapes and the M-sweep shapes):
-//  * 64-column tiles unless that makes more than ~384 CTAs (then 128, then 256 columns);
+//  * 64-column tiles unless that makes more CTAs than are resident at once (then 128, then 256 columns);
 //  * about one to two CTAs per SM in total: 256 for products of 32 MB and more, 160 below that
 //    (each extra split costs a partial tile and lengthens the gather), 148 when M > 8 (one resident
 //    CTA per SM);
@@ -65,7 +67,8 @@ static Plan make_tma_plan(int M, int N, int K, int H)
     Plan p{};
     p.kind = kRowTma;
     int tn = 64;
-    while ((long)ceil_div(N, tn) * H > 384 && tn < 256) tn *= 2;
+    const long tile_cap = (M > 8) ? kSMs : 2 * kSMs;   // a single wave of resident CTAs (two per SM, one when M > 8)
+    while ((long)ceil_div(N, tn) * H > tile_cap && tn < 256) tn *= 2;
     if (g_force_tn == 64 || g_force_tn == 128 || g_force_tn == 256) tn = g_force_tn;
     const int tpr = tn / 8;
     const int kt = (kTmaConsumers / tpr) * 4;
@@ -75,6 +78,7 @@ static Plan make_tma_plan(int M, int N, int K, int H)
     const int target = (M > 8) ? kSMs : (total_bytes < 32e6 ? 160 : 256);
     int ns = (int)((target + base / 2) / base);
     if (ns > K / 128) ns = K / 128;
+    if (ns > K / (40 * M)) ns = K / (40 * M);          // partial sums stay below ~10 % of the weight bytes
     if (g_force_split > 0) ns = g_force_split;
     if (ns > kMaxSplit) ns = kMaxSplit;
     if (ns < 1) ns = 1;
@@ -92,6 +96,34 @@ static Plan make_tma_plan(int M, int N, int K, int H)
     return p;
 }
 
+// Plan for the swap-AB tensor-core kernel: 128-column tiles, k-rows per split a multiple of the 64-row
+// stage, about two CTAs per SM in total, five 18 KB stages.
+static Plan make_tc_plan(int M, int N, int K, int H)
+{
+    Plan p{};
+    p.kind = kRowTc;
+    p.tn = kTcTN; p.tpr = 0; p.rg = 0;
+    p.ntiles = ceil_div(N, kTcTN);
+    const long base = (long)p.ntiles * H;
+    // one CTA per SM measured best for this kernel (its ring alone keeps 90 KB in flight per SM)
+    int ns = (int)((kSMs + base / 2) / base);
+    if (ns > K / 128) ns = K / 128;
+    if (ns > K / (40 * M)) ns = K / (40 * M);          // partial sums stay below ~10 % of the weight bytes
+    if (g_force_split > 0) ns = g_force_split;
+    if (ns > kMaxSplit) ns = kMaxSplit;
+    if (ns < 1) ns = 1;
+    if (base > kNumCounters) ns = 1;
+    const int kr = ceil_div(ceil_div(K, ns), kTcKT) * kTcKT;
+    p.kr = kr;
+    p.nsplit = ceil_div(K, kr);
+    int nstage = 5;
+    if (g_force_stages > 0) nstage = g_force_stages;
+    if (nstage < 2) nstage = 2;
+    if (nstage > 10) nstage = 10;
+    p.nstage = nstage;
+    return p;
+}
+
 static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout, bool vec_ok, bool tma_ok)
 {
     Plan p{};
@@ -101,6 +133,12 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
         p.tpr = p.rg = 0;
         return p;
     }
+    // Measured on B200: from M = 3 on, the CUDA-core kernel falls off the HBM roofline on large weight
+    // matrices (fp32 FMA issue) while the tensor-core kernel stays on it; small matrices are
+    // latency-bound either way and the CUDA-core kernel has the shorter fixed cost.
+    const bool tc_pays = M >= g_tc_min_m && 2.0 * K * N * H >= 32e6;
+    if (layout == NM_ROW_MAJOR && tma_ok && g_force_kind != kRowTma && (tc_pays || g_force_kind == kRowTc))
+        return make_tc_plan(M, N, K, H);
     if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H);
     const int target = (M <= 4 ? 4 : 2) * kSMs;       // CTAs wanted in flight
     if (layout == NM_ROW_MAJOR) {
@@ -141,29 +179,34 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
 }
 
 // Tensor maps of recently used weight matrices (encoding one costs about a microsecond of host time).
-struct MapKey { const void *B; int N, K, H; long strideB; int tn, kt; };
-struct MapEntry { MapKey key; CUtensorMap map; bool valid; };
+struct MapKey { const void *B; int N, K, H; long strideB; int tn, kt; };      // tn = box columns, kt = box rows (16 marks a token map)
+struct MapEntry { MapKey key; CUtensorMap map; bool valid; long row_stride; };
 static thread_local MapEntry g_maps[16];
 static thread_local int g_map_next = 0;
 
-static const CUtensorMap *get_weight_map(const void *B, int N, int K, int H, long strideB, int tn, int kt)
+static const CUtensorMap *get_weight_map(const void *B, int N, int K, int H, long strideB, int tn, int kt, bool swizzle128 = false,
+                                         long row_stride = 0)
 {
+    if (row_stride == 0) row_stride = N;
     for (auto &e : g_maps) {
         const MapKey &k = e.key;
-        if (e.valid && k.B == B && k.N == N && k.K == K && k.H == H && k.strideB == strideB && k.tn == tn && k.kt == kt)
+        if (e.valid && k.B == B && k.N == N && k.K == K && k.H == H && k.strideB == strideB && k.tn == tn &&
+            k.kt == (swizzle128 ? -kt : kt) && e.row_stride == row_stride)
             return &e.map;
     }
     EncodeTiledFn enc = tensor_map_encoder();
     if (!enc) return nullptr;
     MapEntry &e = g_maps[g_map_next];
     g_map_next = (g_map_next + 1) % 16;
-    e.key = MapKey{B, N, K, H, strideB, tn, kt};
+    e.key = MapKey{B, N, K, H, strideB, tn, swizzle128 ? -kt : kt};
+    e.row_stride = row_stride;
     const cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)K, (cuuint64_t)H};
-    const cuuint64_t strides[2] = {(cuuint64_t)N * 2, (cuuint64_t)(H > 1 ? strideB : (long)K * N) * 2};
+    const cuuint64_t strides[2] = {(cuuint64_t)row_stride * 2, (cuuint64_t)(H > 1 ? strideB : (long)K * row_stride) * 2};
     const cuuint32_t box[3] = {(cuuint32_t)tn, (cuuint32_t)kt, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(B), dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     e.valid = (r == CUDA_SUCCESS);
     return e.valid ? &e.map : nullptr;
@@ -207,6 +250,13 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
                   (long)N * 2 < (1L << 40) && strideB >= 0;
     if (g_force_kind == kRowVec) tma_ok = false;
     Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok);
+    const CUtensorMap *tc_map_b = nullptr, *tc_map_a = nullptr;
+    if (p.kind == kRowTc) {
+        // weights [H][K][N] in 64x64 swizzled boxes; tokens [H][M][K] (row stride lda) in 64 x 16 swizzled boxes
+        tc_map_b = get_weight_map(B, N, K, H, strideB, 64, kTcKT, true);
+        tc_map_a = get_weight_map(A, K, M, H, strideA, 64, 16, true, lda);
+        if (!tc_map_b || !tc_map_a) p = make_tma_plan(M, N, K, H);      // strides the encoder refuses: CUDA-core kernel
+    }
 
     MatmulArgs a{};
     a.A = A; a.B = B; a.C = C;
@@ -223,7 +273,12 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     }
 
     cudaError_t e = cudaErrorInvalidValue;
-    if (p.kind == kRowTma) {
+    if (p.kind == kRowTc) {
+        const CUtensorMap *mb = tc_map_b, *ma = tc_map_a;
+        TmaArgs ta{};
+        ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
+        e = (dtype == NM_BF16_F32OUT) ? launch_row_tc<float>(*mb, *ma, ta, stream) : launch_row_tc<bf16_t>(*mb, *ma, ta, stream);
+    } else if (p.kind == kRowTma) {
         const int kt = (kTmaConsumers / p.tpr) * 4;
         const CUtensorMap *map = get_weight_map(B, N, K, H, strideB, p.tn, kt);
         if (!map) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
@@ -367,6 +422,14 @@ int nm_debug_set_plan(int tile_n, int nsplit)
 {
     if (tile_n < 0 || nsplit < 0 || tile_n > kMaxTileN || nsplit > kMaxSplit) return NM_ERR_INVALID_ARG;
     g_force_tn = tile_n; g_force_split = nsplit;
+    return NM_OK;
+}
+
+/* Smallest M that goes to the swap-AB tensor-core kernel (row-major bf16 B); 17 keeps every M on CUDA cores. */
+int nm_set_tensor_core_min_m(int m)
+{
+    if (m < 1 || m > NM_MAX_M + 1) return NM_ERR_INVALID_ARG;
+    g_tc_min_m = m;
     return NM_OK;
 }
 

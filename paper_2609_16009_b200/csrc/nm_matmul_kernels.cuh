@@ -31,6 +31,14 @@ struct MatmulArgs {
     unsigned *counters;
 };
 
+// Extra launch state of the TMA-fed kernels.
+struct TmaArgs {
+    MatmulArgs base;
+    int nstage;            // ring depth
+    int use_pdl;           // kernel was launched with programmatic stream serialization
+    unsigned *status;      // device status word
+};
+
 template <int M> struct RowCfg {
     static constexpr int kUnroll = (M <= 4) ? 8 : (M <= 8 ? 6 : 4);
     static constexpr int kMinBlocks = (M <= 2) ? 3 : (M <= 8 ? 2 : 1);
@@ -43,8 +51,8 @@ template <int M> struct RowCfg {
 // Called by all threads of the CTA after its partial tile has been written to `partial`.  The
 // last CTA to arrive at (h, tile) reads all nsplit partial tiles in order and writes C; it then
 // puts the counter back to zero, so the workspace needs no clearing between launches.
-template <int M, typename TO>
-__device__ __forceinline__ void splitk_complete(const MatmulArgs &a, int tile, int h, int *s_last)
+template <typename TO>
+__device__ __forceinline__ void splitk_complete_rt(const MatmulArgs &a, int M, int tile, int h, int *s_last)
 {
     const int tid = threadIdx.x;
     __threadfence();
@@ -69,6 +77,12 @@ __device__ __forceinline__ void splitk_complete(const MatmulArgs &a, int tile, i
         }
     }
     if (tid == 0) *cnt = 0u;
+}
+
+template <int M, typename TO>
+__device__ __forceinline__ void splitk_complete(const MatmulArgs &a, int tile, int h, int *s_last)
+{
+    splitk_complete_rt<TO>(a, M, tile, h, s_last);
 }
 
 // ---- row-major B (n contiguous): each thread owns kVec consecutive columns ---------------------------

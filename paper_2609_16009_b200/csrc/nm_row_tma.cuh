@@ -37,13 +37,6 @@ template <int M> struct TmaCfg {
     static constexpr int kPass = (kMP < 4) ? kMP : 4;
 };
 
-struct TmaArgs {
-    MatmulArgs base;
-    int nstage;            // ring depth
-    int use_pdl;           // kernel was launched with programmatic stream serialization
-    unsigned *status;      // device status word
-};
-
 template <int M, int TPR, typename TO>
 __global__ void __launch_bounds__(kTmaThreads, TmaCfg<M>::kMinBlocks)
 nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)

@@ -136,7 +136,7 @@ def test_tma_ring_every_m_and_tile(nm, M, tile_n):
     A, B = gen.narrow_bf16(M, K, N, seed=900 + M)
     for stages in (2, 0):
         nm.nm_debug_set_plan(tile_n, 2)
-        nm.nm_debug_set_kernel(-1, stages)
+        nm.nm_debug_set_kernel(3, stages)
         try:
             assert nm.nm_debug_get_plan(M, N, K)["kind"] == 3
             run_case(nm, A, B, M, N, K, BF16, ROW, f"tma M={M} tile_n={tile_n} stages={stages}")
@@ -144,6 +144,51 @@ def test_tma_ring_every_m_and_tile(nm, M, tile_n):
             nm.nm_debug_set_plan(0, 0)
             nm.nm_debug_set_kernel(-1, 0)
     nm.nm_check_status()
+
+
+@pytest.mark.parametrize("M", [1, 2, 5, 8, 9, 13, 16])
+@pytest.mark.parametrize("nsplit", [0, 1, 3])
+def test_tensor_core_swap_ab_kernel(nm, M, nsplit):
+    # weights as the MMA's M dimension, tokens as its N: same tolerance as the CUDA-core kernels.
+    # K ends mid-stage (1000 = 15*64 + 40) and N ends mid-tile (840 = 6*128 + 72).
+    K, N = 1000, 840
+    A, B = gen.narrow_bf16(M, K, N, seed=1200 + M)
+    nm.nm_debug_set_plan(0, nsplit)
+    nm.nm_debug_set_kernel(4, 0)
+    try:
+        assert nm.nm_debug_get_plan(M, N, K)["kind"] == 4
+        run_case(nm, A, B, M, N, K, BF16, ROW, f"tensor-core M={M} nsplit={nsplit}")
+        run_case(nm, A, B, M, N, K, BF16_F32OUT, ROW, f"tensor-core fp32 out M={M} nsplit={nsplit}")
+    finally:
+        nm.nm_debug_set_plan(0, 0)
+        nm.nm_debug_set_kernel(-1, 0)
+    nm.nm_check_status()
+
+
+def test_tensor_core_kernel_small_integers_bit_exact(nm):
+    M, K, N = 16, 7168, 576
+    A = gen.small_int_bf16((M, K), -8, 8, seed=1301)
+    B = gen.small_int_bf16((K, N), -8, 8, seed=1302)
+    nm.nm_debug_set_kernel(4, 0)
+    try:
+        got = run_case(nm, A, B, M, N, K, BF16_F32OUT, ROW, "tensor-core small ints")
+    finally:
+        nm.nm_debug_set_kernel(-1, 0)
+    _, C64, _ = oracle.matmul(A, B, M, N, K, oracle.BF16, oracle.F32, ROW, threads=8)
+    assert np.array_equal(got, C64)
+
+
+def test_default_kernel_choice_by_m(nm):
+    # CUDA cores (TMA ring) for one or two token rows and for small weight matrices, tensor cores from
+    # three rows on for large ones; the threshold is adjustable
+    assert nm.nm_debug_get_plan(2, 18432, 7168)["kind"] == 3
+    assert nm.nm_debug_get_plan(3, 18432, 7168)["kind"] == 4
+    assert nm.nm_debug_get_plan(16, 576, 7168)["kind"] == 3
+    nm.nm_set_tensor_core_min_m(17)
+    try:
+        assert nm.nm_debug_get_plan(16, 18432, 7168)["kind"] == 3
+    finally:
+        nm.nm_set_tensor_core_min_m(3)
 
 
 def test_plain_row_kernel_every_m(nm):

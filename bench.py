@@ -414,6 +414,21 @@ def run_reference(args, rank):
 # --------------------------------------------------------------------------------------------------
 # main arm
 # --------------------------------------------------------------------------------------------------
+def reduce_over_ranks(values, dist, device):
+    """Max over ranks of per-rank timings (every rank runs an independent replica; the job's step
+    time is that of the slowest rank).  `dist` is torch.distributed or None for a single process."""
+    if dist is None:
+        return list(values)
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput_gbs(bytes_per_step, steps, world, ms):
+    """Whole-job GB/s: every rank moves bytes_per_step per step; time is the slowest rank's."""
+    return bytes_per_step * steps * world / (ms * 1e-3) / 1e9
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -507,16 +522,12 @@ def main():
         clocks = sampler.stop()
     nm.nm_check_status(stream)
 
-    if dist is not None:
-        t = torch.tensor([ms, e2e_ms, dom_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms, dom_ms = t.tolist()
+    ms, e2e_ms, dom_ms = reduce_over_ranks([ms, e2e_ms, dom_ms], dist, device)
 
     if rank == 0:
         peak, peak_kind = load_peaks()
-        total_bytes = wl.bytes_per_step * args.steps * world
-        value = total_bytes / (ms * 1e-3) / 1e9
-        e2e_value = total_bytes / (e2e_ms * 1e-3) / 1e9
+        value = job_throughput_gbs(wl.bytes_per_step, args.steps, world, ms)
+        e2e_value = job_throughput_gbs(wl.bytes_per_step, args.steps, world, e2e_ms)
         achieved = wl.dominant_bytes / (dom_ms * 1e-3) / 1e9
         line = {"metric": "narrow MatMul HBM GB/s (MLA single-token decode step)", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms / args.steps, "decode_us": ms / args.steps * 1e3,

@@ -125,6 +125,7 @@ class MlaStep:
         p = nm.mla_params(DIMS, seq_len, t)
         self.ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p), device=device)
         self.p = nm.mla_params(DIMS, seq_len, t, workspace=self.ws)
+        self.p.programmatic_entry = 1        # steps follow each other like the layers of a model: weights are static
         self.side = torch.cuda.Stream(device)
         self.specs = projection_specs()
         self.kv_bytes = seq_len * (dc + dr) * 2 + (dc + dr) * 2        # rows read once + the row written
@@ -143,7 +144,8 @@ class MlaStep:
                             f"nope 128, v 128, 128 heads), seq_len {self.S}, bf16 weights row-major, W_O included",
                 "seq_len": self.S,
                 "l2": "weights 374 MB per step > 126 MB L2, so every step streams from HBM; no flush",
-                "overlap": "KV chain (W_DKV|KR product, RMSNorm, RoPE, cache write) on a side stream beside the tcgen05 attention pass"}
+                "overlap": "side stream: KV chain beside the W_DQ product, L2 prefetch of W_UV/W_O beside the tcgen05 attention pass; "
+                           "programmatic dependent launch along the main stream, also across steps"}
 
     def step(self, stream, dom_events=None):
         if dom_events is not None:
@@ -501,12 +503,14 @@ def main():
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record(stream)
+        # the dominant kernel is bracketed by events on every 8th step only: the events break the
+        # programmatic launch of that kernel, and the step time should not carry that on every step
         for i in range(args.steps):
-            wl.step(stream, dom[i])
+            wl.step(stream, dom[i] if i % 8 == 0 else None)
         e1.record(stream)
         barrier()
         ms = e0.elapsed_time(e1)
-        dom_ms = statistics.mean(a.elapsed_time(b) for a, b in dom)
+        dom_ms = statistics.mean(a.elapsed_time(b) for a, b in dom[::8])
         # ---- end-to-end region: host token in, host result out, every step -----------------------------
         for _ in range(3):
             wl.step_e2e(stream)

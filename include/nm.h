@@ -236,6 +236,10 @@ typedef struct {
     float *o_lat_f32;
     /* optional cudaEvent_t pair recorded on main_stream around the W_O product (for profiling) */
     void *event_before_wo, *event_after_wo;
+    /* non-zero: the step's first product may start (and prefetch its weights) while the work enqueued
+     * before the step on main_stream is still running - back-to-back layers or steps.  Only valid if
+     * that earlier work writes none of this step's weights.  0 keeps the ordinary stream order. */
+    int programmatic_entry;
 } nm_mla_params;
 
 size_t nm_mla_workspace_bytes(const nm_mla_params *p);

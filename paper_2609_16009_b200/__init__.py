@@ -73,7 +73,8 @@ class MlaParams(C.Structure):
                                       "rope_cos_sin", "kv_cache", "out", "workspace")]
                 + [("workspace_bytes", _sz)]
                 + [(n, _vp) for n in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o", "o_lat_f32",
-                                      "event_before_wo", "event_after_wo")])
+                                      "event_before_wo", "event_after_wo")]
+                + [("programmatic_entry", _i)])
 
 
 _lib.nm_rmsnorm.argtypes = [_vp, _vp, _vp, _i, C.c_float, _vp]

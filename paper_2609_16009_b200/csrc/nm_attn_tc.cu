@@ -1,17 +1,19 @@
 // Latent attention pass on the tensor cores (tcgen05 + TMEM), one sequence split per CTA pair.
 //
-// For all 128 heads at once and a run of cache rows, tile by tile (64 rows):
-//   S[128 x 64]   = Q[128 x 576] * tile^T      tcgen05.mma, both operands K-major in shared memory
+// For all 128 heads at once and a run of cache rows, tile by tile (32 rows; two tiles in flight):
+//   S[128 x 32]   = Q[128 x 576] * tile^T      tcgen05.mma, both operands K-major in shared memory
 //   P             = exp2(S*c - m)              fp32 in registers (one thread per head); written to TMEM as
 //                                              two bf16 terms, P_hi = bf16(P) and P_lo = bf16(P - P_hi), so
 //                                              that P*V keeps about 16 bits of P instead of 8
-//   O[128 x 256] += P[128 x 64] * tile[:, half]  tcgen05.mma, A from TMEM, B = the same shared-memory
+//   O[128 x 256] += P[128 x 32] * tile[:, half]  tcgen05.mma, A from TMEM, B = the same shared-memory
 //                                                bytes read MN-major
 // Q and the cache tile arrive by TMA (128-byte swizzle, no multicast) and are consumed in place by
 // the MMA unit; the accumulators never leave TMEM until the split is finished.  The 512 output
 // columns do not fit TMEM next to S, so two CTAs share a split, each owning 256 columns.  The running
 // maximum is updated lazily: O is rescaled only when a row maximum grows by more than 2^8, so the
-// usual tile costs no pass over the accumulator.
+// usual tile costs no pass over the accumulator.  The cache tiles, S and P are double-buffered: while the
+// softmax threads work on tile t, the tensor pipe computes the scores of tile t+1 and the P*V of tile
+// t-1, and TMA fetches the next tile.
 //
 // The CTAs of kAttnCluster consecutive splits form a thread-block cluster and merge their results
 // through distributed shared memory before anything goes to global memory: each CTA rescales its
@@ -35,16 +37,18 @@ constexpr int kHeads = 128;
 constexpr int kDqk = 576;                 // 512 latent + 64 rope
 constexpr int kDv = 512;
 constexpr int kDvHalf = 256;
-constexpr int kT = kAttnTileRows;         // cache rows per tile (64)
+constexpr int kT = 32;                    // cache rows per pipeline stage (two stages in shared memory)
+constexpr int kKVStages = 2;
 constexpr int kKBlocks = kDqk / 64;       // 9 blocks of 64 elements (one 128-byte swizzle span)
 constexpr int kQBlockBytes = kHeads * 128;   // 16 KB
 constexpr int kKVBlockBytes = kT * 128;      // 8 KB
 constexpr int kQBytes = kKBlocks * kQBlockBytes;     // 147456
-constexpr int kKVBytes = kKBlocks * kKVBlockBytes;   // 73728
-constexpr int kSmemBytes = kQBytes + kKVBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int kKVBytes = kKBlocks * kKVBlockBytes;   // 36864 per stage
+constexpr int kSmemBytes = kQBytes + kKVStages * kKVBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColO = 0, kColS = 256, kColP = 320, kColPlo = 352;
+// TMEM columns: O (fp32, 256), then per pipeline stage S (fp32, 32), P_hi and P_lo (bf16 pairs, 16 each)
+constexpr uint32_t kColO = 0, kColS = 256, kColP = 320, kColPlo = 352;      // stage b adds 32*b to S, 16*b to P_hi / P_lo
 constexpr float kLazyThreshold = 8.0f;    // log2 units
 constexpr int kCl = kAttnCluster;          // CTAs (splits) per cluster
 constexpr int kHeadsPerRank = kHeads / kCl;
@@ -104,10 +108,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;            // swizzle atoms want 1024-byte alignment
     unsigned char *smem = smem_raw + (base - raw_addr);
-    const uint32_t q_addr = base, kv_addr = base + kQBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kQBytes + kKVBytes);
-    const uint32_t bar_q = smem_u32(bars + 0), bar_kv_full = smem_u32(bars + 1), bar_kv_empty = smem_u32(bars + 2),
-                   bar_s = smem_u32(bars + 3), bar_p = smem_u32(bars + 4), bar_o = smem_u32(bars + 5);
+    const uint32_t q_addr = base, kv_addr = base + kQBytes;        // kv stage b at kv_addr + b * kKVBytes
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kQBytes + kKVStages * kKVBytes);
+    // q: Q landed.  Per stage b: kv_full (tile landed), s_full (scores in TMEM), p_full (P written, 128
+    // arrivals), pv_done (P*V of the tile finished: frees the cache stage and the P buffers).
+    const uint32_t bar_q = smem_u32(bars + 0), bar_kv_full = smem_u32(bars + 1), bar_s_full = smem_u32(bars + 3),
+                   bar_p_full = smem_u32(bars + 5), bar_pv_done = smem_u32(bars + 7);
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ __align__(8) float s_ml[kHeads][2];                // this split's (m in log2 units, l) per head
@@ -121,14 +127,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (tid == 0) {
         NM_TRACE(0);
         s_abort = 0;
-        mbar_init(bar_q, 1); mbar_init(bar_kv_full, 1); mbar_init(bar_kv_empty, 1);
-        mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+        mbar_init(bar_q, 1);
+        for (int b = 0; b < kKVStages; ++b) {
+            mbar_init(bar_kv_full + 8 * b, 1); mbar_init(bar_s_full + 8 * b, 1);
+            mbar_init(bar_p_full + 8 * b, 128); mbar_init(bar_pv_done + 8 * b, 1);
+        }
         mbar_init_fence();
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 1) tmem_alloc(&s_tmem_base, kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -144,114 +150,156 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             tma_prefetch_descriptor(&map_q);
             tma_prefetch_descriptor(&map_kv);
             const uint64_t keep = l2_policy_evict_last(), stream = l2_policy_evict_first();
-            // The rows of the first tile were written by earlier steps, not by the kernels just before
-            // this one: fetch them before waiting for those kernels, then fetch Q, which they produce.
-            if (ntiles > 0) {
-                mbar_arrive_expect_tx(bar_kv_full, kKVBytes);
-                for (int c = 0; c < kKBlocks; ++c) tma_load_2d(kv_addr + c * kKVBlockBytes, &map_kv, c * 64, r0, bar_kv_full, stream);
-            }
+            auto load_tile = [&](int t) {
+                const int b = t & 1;
+                mbar_arrive_expect_tx(bar_kv_full + 8 * b, kKVBytes);
+                for (int c = 0; c < kKBlocks; ++c)
+                    tma_load_2d(kv_addr + b * kKVBytes + c * kKVBlockBytes, &map_kv, c * 64, r0 + t * kT, bar_kv_full + 8 * b, stream);
+            };
+            // The cache rows were written by earlier steps, not by the kernels just before this one:
+            // fetch the first two tiles before waiting for those kernels, then fetch Q, which they produce.
+            for (int t = 0; t < min(ntiles, kKVStages); ++t) load_tile(t);
+            // Only two tiles fit in shared memory, far too few to cover the HBM latency of a tile that
+            // takes under a microsecond to consume: the rest of this split's rows are pulled into L2 now
+            // (a few hundred KB), so that every later tile load is an L2 hit.
+            if (half == 0)
+                for (int t = kKVStages; t < ntiles; ++t)
+                    for (int c = 0; c < kKBlocks; ++c) tma_prefetch_l2_2d(&map_kv, c * 64, r0 + t * kT);
             pdl_wait_prior_grids();
             if (ntiles > 0) {                                      // a padding CTA of the last cluster loads nothing
                 mbar_arrive_expect_tx(bar_q, kQBytes);
                 for (int c = 0; c < kKBlocks; ++c) tma_load_2d(q_addr + c * kQBlockBytes, &map_q, c * 64, 0, bar_q, keep);
             }
-            for (int t = 1; t < ntiles; ++t) {
-                if (!mbar_try_wait(bar_kv_empty, (t - 1) & 1) && !mbar_wait(bar_kv_empty, (t - 1) & 1, &s_abort, status)) break;
-                mbar_arrive_expect_tx(bar_kv_full, kKVBytes);
-                for (int c = 0; c < kKBlocks; ++c)
-                    tma_load_2d(kv_addr + c * kKVBlockBytes, &map_kv, c * 64, r0 + t * kT, bar_kv_full, stream);
+            for (int t = kKVStages; t < ntiles; ++t) {             // stage b is free once the P*V of tile t-2 is done
+                const uint32_t bar = bar_pv_done + 8 * (t & 1), par = ((t - kKVStages) >> 1) & 1;
+                if (!mbar_try_wait(bar, par) && !mbar_wait(bar, par, &s_abort, status)) break;
+                load_tile(t);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ---------------------------------------------------------------
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(128, kT, false, false), idesc_o = instr_desc(128, kDvHalf, false, true);
-            NM_TRACE(1);
-            if (ntiles > 0) mbar_wait(bar_q, 0, &s_abort, status);
-            NM_TRACE(2);
-            for (int t = 0; t < ntiles; ++t) {
-                mbar_wait(bar_kv_full, t & 1, &s_abort, status);
+            auto scores = [&](int t) {                             // S[t&1] = Q * tile(t)^T  (tile t has landed)
+                const int b = t & 1;
                 tc_fence_after();
-                if (t == 0) NM_TRACE(3);
                 for (int c = 0; c < kKBlocks; ++c)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        mma_ss(tmem + kColS, smem_desc(q_addr + c * kQBlockBytes + kk * 32, 16, 1024),
-                               smem_desc(kv_addr + c * kKVBlockBytes + kk * 32, 16, 1024), idesc_s, (c | kk) != 0);
-                mma_commit(bar_s);
-                mbar_wait(bar_p, t & 1, &s_abort, status);
+                        mma_ss(tmem + kColS + 32 * b, smem_desc(q_addr + c * kQBlockBytes + kk * 32, 16, 1024),
+                               smem_desc(kv_addr + b * kKVBytes + c * kKVBlockBytes + kk * 32, 16, 1024), idesc_s, (c | kk) != 0);
+                mma_commit(bar_s_full + 8 * b);
+            };
+            auto pv = [&](int t) {                                 // O += P[t&1] * tile(t)[:, half]  (P of tile t is written)
+                const int b = t & 1;
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < kT / 16; ++kk) {
-                    const uint64_t vdesc = smem_desc(kv_addr + (4 * half) * kKVBlockBytes + kk * 2048, kKVBlockBytes, 1024);
-                    mma_ts(tmem + kColO, tmem + kColP + kk * 8, vdesc, idesc_o, (t | kk) != 0);
-                    mma_ts(tmem + kColO, tmem + kColPlo + kk * 8, vdesc, idesc_o, true);
+                    const uint64_t vdesc = smem_desc(kv_addr + b * kKVBytes + (4 * half) * kKVBlockBytes + kk * 2048, kKVBlockBytes, 1024);
+                    mma_ts(tmem + kColO, tmem + kColP + 16 * b + kk * 8, vdesc, idesc_o, (t | kk) != 0);
+                    mma_ts(tmem + kColO, tmem + kColPlo + 16 * b + kk * 8, vdesc, idesc_o, true);
                 }
-                mma_commit(bar_o);
-                mma_commit(bar_kv_empty);
+                mma_commit(bar_pv_done + 8 * b);
+            };
+            NM_TRACE(1);
+            if (ntiles > 0) mbar_wait(bar_q, 0, &s_abort, status);
+            NM_TRACE(2);
+            // Two independent streams of work share this thread: scores of tile ts (needs the tile in
+            // shared memory and S[ts&1] free, i.e. the P*V of tile ts-2 issued) and P*V of tile tp (needs
+            // the softmax of tile tp).  Whichever is ready is issued; neither blocks the other.
+            int ts = 0, tp = 0;
+            uint64_t idle_since = 0;
+            while (tp < ntiles) {
+                bool progress = false;
+                if (ts < ntiles && ts <= tp + 1 && mbar_try_wait(bar_kv_full + 8 * (ts & 1), (ts >> 1) & 1)) {
+                    scores(ts);
+                    if (ts == 0) NM_TRACE(3);
+                    ++ts;
+                    progress = true;
+                }
+                if (mbar_try_wait(bar_p_full + 8 * (tp & 1), (tp >> 1) & 1)) {
+                    pv(tp);
+                    ++tp;
+                    progress = true;
+                }
+                if (progress) {
+                    idle_since = 0;
+                } else {                                           // bounded: give up after about a second without progress
+                    if (s_abort) break;
+                    const uint64_t now = global_timer_ns();
+                    if (idle_since == 0) idle_since = now;
+                    else if (now - idle_since > kWaitLimitNs) {
+                        s_abort = 1;
+                        if (status) atomicOr(status, kStatusWaitExpired);
+                        break;
+                    }
+                }
             }
         }
     } else {
-        // ---------------- one head per thread: softmax, lazy rescale, epilogue ----------------------------
+        // ---------------- one head per thread: softmax, lazy rescale ------------------------------------------
         const int quad = warp & 3;                                 // TMEM lanes this warp may touch
-        const int head = quad * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
         float m_used = -INFINITY, l = 0.f;
         for (int t = 0; t < ntiles; ++t) {
-            mbar_wait(bar_s, t & 1, &s_abort, status);
+            const int b = t & 1;
+            mbar_wait(bar_s_full + 8 * b, (t >> 1) & 1, &s_abort, status);
             tc_fence_after();
             if (t == 0 && tid == 64) NM_TRACE(4);
-            uint32_t sr[2][32];
-            tmem_ld32(lane_base + kColS, sr[0]);
-            tmem_ld32(lane_base + kColS + 32, sr[1]);
+            uint32_t sr[32];
+            tmem_ld32(lane_base + kColS + 32 * b, sr);
             tmem_wait_ld();
             const int valid = min(kT, r1 - (r0 + t * kT));
             float mx = -INFINITY;
 #pragma unroll
             for (int j = 0; j < kT; ++j)
-                if (j < valid) mx = fmaxf(mx, __uint_as_float(sr[j >> 5][j & 31]));
+                if (j < valid) mx = fmaxf(mx, __uint_as_float(sr[j]));
             const float mx2 = mx * scale_log2;
             const bool grow = (t == 0) || (mx2 > m_used + kLazyThreshold);
-            if (t > 0) {                                           // previous P*V must be done before P or O change
-                mbar_wait(bar_o, (t - 1) & 1, &s_abort, status);
+            // P[b] was last read by the P*V of tile t-2
+            if (t >= kKVStages) {
+                mbar_wait(bar_pv_done + 8 * b, ((t - kKVStages) >> 1) & 1, &s_abort, status);
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, grow)) {
-                    const float f = grow ? fast_exp2(m_used - mx2) : 1.0f;
-                    for (int c = 0; c < kDvHalf / 32; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(lane_base + kColO + c * 32, o);
-                        tmem_wait_ld();
+            }
+            if (t > 0 && __any_sync(0xffffffffu, grow)) {
+                // rare: the maximum grew by more than 2^8.  O may only be touched between two P*V passes.
+                mbar_wait(bar_pv_done + 8 * ((t - 1) & 1), ((t - 1) >> 1) & 1, &s_abort, status);
+                tc_fence_after();
+                const float f = grow ? fast_exp2(m_used - mx2) : 1.0f;
+                for (int c = 0; c < kDvHalf / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(lane_base + kColO + c * 32, o);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                        tmem_st32(lane_base + kColO + c * 32, o);
-                    }
-                    tmem_wait_st();
-                    if (grow) l *= f;
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                    tmem_st32(lane_base + kColO + c * 32, o);
                 }
+                tmem_wait_st();
+                if (grow) l *= f;
             }
             if (grow) m_used = mx2;
-            uint32_t pr[32], plo[32];
+            uint32_t pr[16], plo[16];
             float lsum = 0.f;
 #pragma unroll
             for (int j = 0; j < kT; j += 2) {
-                const float p0 = (j < valid) ? fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), scale_log2, -m_used)) : 0.f;
-                const float p1 = (j + 1 < valid) ? fast_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), scale_log2, -m_used)) : 0.f;
+                const float p0 = (j < valid) ? fast_exp2(fmaf(__uint_as_float(sr[j]), scale_log2, -m_used)) : 0.f;
+                const float p1 = (j + 1 < valid) ? fast_exp2(fmaf(__uint_as_float(sr[j + 1]), scale_log2, -m_used)) : 0.f;
                 lsum += p0 + p1;
                 const uint32_t hi = pack_bf16x2(p0, p1);
                 pr[j >> 1] = hi;
                 plo[j >> 1] = pack_bf16x2(p0 - __uint_as_float(hi << 16), p1 - __uint_as_float(hi & 0xffff0000u));
             }
             l += lsum;
-            tmem_st32(lane_base + kColP, pr);
-            tmem_st32(lane_base + kColPlo, plo);
+            tmem_st16(lane_base + kColP + 16 * b, pr);
+            tmem_st16(lane_base + kColPlo + 16 * b, plo);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar_p);
+            mbar_arrive(bar_p_full + 8 * b);
             if (t == 0 && tid == 64) NM_TRACE(5);
         }
-        // the last P*V must have landed before O is read; then publish this split's (m, l)
+        // the last P*V must have landed before O is read
         if (ntiles > 0) {
-            mbar_wait(bar_o, (ntiles - 1) & 1, &s_abort, status);
+            mbar_wait(bar_pv_done + 8 * ((ntiles - 1) & 1), ((ntiles - 1) >> 1) & 1, &s_abort, status);
             tc_fence_after();
         }
         if (tid == 64) NM_TRACE(6);

@@ -140,7 +140,7 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     if (layout == NM_ROW_MAJOR && tma_ok && g_force_kind != kRowTma && (tc_pays || g_force_kind == kRowTc))
         return make_tc_plan(M, N, K, H);
     if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H);
-    const int target = (M <= 4 ? 4 : 2) * kSMs;       // CTAs wanted in flight
+    const int target = 192;                           // CTAs wanted in total (measured: 144-240 is the flat optimum)
     if (layout == NM_ROW_MAJOR) {
         p.kind = kRowVec;
         // threads per row: 8 -> 32 (128-byte to 512-byte row segments); wider when N is large
@@ -162,10 +162,12 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     p.ntiles = ceil_div(N, p.tn);
     int nsplit = 1;
     const long ctas = (long)p.ntiles * H;
-    if (ctas < target) nsplit = (int)((target + ctas - 1) / ctas);
-    // keep at least ~64 k-rows (row kernel) / 512 k (column kernel) per split
+    if (ctas < kSMs) nsplit = (int)((target + ctas / 2) / ctas);
+    // keep at least ~64 k-rows (row kernel) / 512 k (column kernel) per split, and the partial sums
+    // below ~10 % of the weight bytes
     const int min_kr = (p.kind == kRowVec) ? 2 * p.rg : 512;
     if (nsplit > K / min_kr) nsplit = K / min_kr;
+    if (nsplit > K / (40 * M)) nsplit = K / (40 * M);
     if (g_force_split > 0) nsplit = g_force_split;
     if (nsplit > kMaxSplit) nsplit = kMaxSplit;
     if (nsplit < 1) nsplit = 1;

@@ -510,7 +510,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     if (forked) NM_CUDA_TRY(cudaEventRecord(g_events.join, ss));
 
     // ---- Q chain, main stream ------------------------------------------------------------------------
-    NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, !forked && pdl));
+    NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl && (!forked || p->programmatic_entry)));
     NM_LAUNCH(rmsnorm_kernel, 1, 256, ms, (const uint16_t *)c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
     NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl));
     NM_LAUNCH(rope_kernel, ceil_div(H * dr / 2, 256), 256, ms, (const uint16_t *)(q + dn), q_full + dc, H, dr, (long)dq, (long)dkv,

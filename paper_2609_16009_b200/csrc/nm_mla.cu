@@ -556,6 +556,18 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
                               pdl && !p->event_before_wo));
         if (p->event_after_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_after_wo, ms));
     }
+    // Under stream capture every stream that was forked must be joined again before the capture ends:
+    // the prefetch kernel on the side stream is otherwise left dangling.  Outside a capture the join is
+    // left out (the next step's fork orders the streams anyway, and a wait here would keep the next
+    // step's first product from starting early).
+    if (forked) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        NM_CUDA_TRY(cudaStreamIsCapturing(ms, &cap));
+        if (cap == cudaStreamCaptureStatusActive) {
+            NM_CUDA_TRY(cudaEventRecord(g_events.q_ready, ss));
+            NM_CUDA_TRY(cudaStreamWaitEvent(ms, g_events.q_ready, 0));
+        }
+    }
 #undef NM_LAUNCH
     return NM_OK;
 }

@@ -317,6 +317,39 @@ def test_decode_step_back_to_back_steps_do_not_interfere(nm, weights, ref1024):
     assert np.all(np.abs(dev_bits_to_f64(outs[0]) - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
 
 
+def test_decode_step_replayed_from_a_cuda_graph(nm, weights, ref1024):
+    # both streams, the events between them and the programmatic launches are captured once; replays must
+    # reproduce the directly launched result bit for bit
+    w, dw = weights
+    h, cache_ref, r = ref1024
+    d = DIMS["d"]
+    t = dict(dw)
+    t["h"] = to_dev(h)
+    t["kv_cache"] = to_dev(gen.mla_cache(1024, DIMS, seed=4200))
+    t["rope_cos_sin"] = rope_row(nm, 1023)
+    t["out"] = torch.zeros(d, dtype=torch.int16, device="cuda")
+    p = nm.mla_params(DIMS, 1024, t)
+    ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p))
+    p = nm.mla_params(DIMS, 1024, t, workspace=ws)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(main):
+        nm.nm_mla_decode_step(p, main, side)          # direct launch (also does every one-time set-up)
+        torch.cuda.synchronize()
+        direct = t["out"].clone()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=main):
+            nm.nm_mla_decode_step(p, main, side)
+        for _ in range(3):
+            t["out"].zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(t["out"], direct)
+    nm.nm_check_status()
+    ref = f64(r["out"])
+    assert np.all(np.abs(dev_bits_to_f64(direct) - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
+
+
 def test_decode_step_host_operands(nm, weights, ref1024):
     w, dw = weights
     h, cache_ref, r = ref1024

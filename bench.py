@@ -286,39 +286,53 @@ def print_timeline(wl, stream, steps=6):
 
 def matmul_sweep(nm, device):
     """GB/s of single narrow products (cold L2: the launches of a CUDA graph rotate through copies of
-    B that together exceed 512 MB).  Reported beside the step; not part of the timed region."""
+    B that together exceed 512 MB).  Two figures per case: launches in plain stream order (each kernel
+    starts when the one before has finished: latency of an isolated call plus the launch gap), and
+    launched programmatically (a kernel may fetch its weights while its predecessor drains, as inside
+    the decode step).  Reported beside the step; not part of the timed region."""
     out = []
-    cases = [(1, 7168, 1536, 0), (1, 7168, 576, 0), (1, 7168, 1536, 1), (1, 7168, 576, 1)]
+    cases = [(1, 512, 512, 0, "f32"), (1, 7168, 1536, 0, "bf16"), (1, 7168, 576, 0, "bf16"), (1, 7168, 1536, 1, "bf16"),
+             (1, 7168, 576, 1, "bf16")]
     for M in (1, 2, 4, 8, 16):
-        cases += [(M, 1536, 24576, 0), (M, 7168, 18432, 0)]
-    g0 = torch.Generator(device="cpu"); g0.manual_seed(7)
-    for M, K, N, layout in cases:
-        nbytes = K * N * 2
+        cases += [(M, 1536, 24576, 0, "bf16"), (M, 7168, 18432, 0, "bf16")]
+    for M, K, N, layout, dt in cases:
+        es = 4 if dt == "f32" else 2
+        tdt = torch.float32 if dt == "f32" else torch.bfloat16
+        code = nm.F32 if dt == "f32" else nm.BF16
+        nbytes = K * N * es
         R = max(2, min(64, (1 << 29) // nbytes + 1))
-        Bs = (torch.randn(R, K * N, device=device) * 0.02).to(torch.bfloat16)
-        A = torch.randn(M * K, device=device).to(torch.bfloat16)
-        C = torch.empty(R, M * N, device=device, dtype=torch.bfloat16)
+        Bs = (torch.randn(R, K * N, device=device) * 0.02).to(tdt)
+        A = torch.randn(M * K, device=device).to(tdt)
+        C = torch.empty(R, M * N, device=device, dtype=tdt)
         ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(M, N, K), device=device)
         s = torch.cuda.Stream(device)
-        with torch.cuda.stream(s):
-            for i in range(R):
-                nm.nm_matmul_ws(A, Bs[i], C[i], M, N, K, nm.BF16, layout, ws, s)
-            s.synchronize()
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=s):
+        row = {"M": M, "K": K, "N": N, "dtype": dt, "layout_B": "col" if layout else "row"}
+        algo = (K * N + M * K + M * N) * es
+        for mode in ("serial", "programmatic"):
+            nm.nm_set_programmatic_launch(mode == "programmatic")
+            with torch.cuda.stream(s):
                 for i in range(R):
-                    nm.nm_matmul_ws(A, Bs[i], C[i], M, N, K, nm.BF16, layout, ws, s)
-            g.replay(); s.synchronize()
-            ts = []
-            for _ in range(5):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(s); g.replay(); b.record(s); s.synchronize()
-                ts.append(a.elapsed_time(b) * 1e3 / R)
-        us = statistics.median(ts)
-        algo = (K * N + M * K + M * N) * 2
-        out.append({"M": M, "K": K, "N": N, "layout_B": "col" if layout else "row", "us": round(us, 2),
-                    "GBps": round(algo / us / 1e3, 1), "pct_of_8TBs": round(algo / us / 1e3 / 80.0, 1)})
-        del Bs, C, g
+                    nm.nm_matmul_ws(A, Bs[i], C[i], M, N, K, code, layout, ws, s)
+                s.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=s):
+                    for i in range(R):
+                        nm.nm_matmul_ws(A, Bs[i], C[i], M, N, K, code, layout, ws, s)
+                g.replay(); s.synchronize()
+                ts = []
+                for _ in range(5):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(s); g.replay(); b.record(s); s.synchronize()
+                    ts.append(a.elapsed_time(b) * 1e3 / R)
+            us = statistics.median(ts)
+            key = "" if mode == "serial" else "_programmatic"
+            row["us" + key] = round(us, 2)
+            row["GBps" + key] = round(algo / us / 1e3, 1)
+            del g
+        nm.nm_set_programmatic_launch(False)
+        row["pct_of_8TBs"] = round(max(row["GBps"], row["GBps_programmatic"]) / 80.0, 1)
+        out.append(row)
+        del Bs, C
     return out
 
 

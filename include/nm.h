@@ -278,6 +278,9 @@ int nm_debug_set_kernel(int kind, int stages);
  * start, set-up done, Q landed, first tile landed, scores ready, P written, last P*V done, after
  * cluster barrier 1, O parked in shared memory, after barrier 2, cluster sum written, end.  NULL = off. */
 int nm_debug_set_attention_trace(void *device_buffer);
+/* Decode step: 1 (default) runs RoPE + W_UK and attention-merge + W_UV as fused per-head kernels, 0 as
+ * separate kernels (rope, batched product, merge, batched product). */
+int nm_debug_set_step_fusion(int enable);
 /* Decode step: MB of W_O prefetched into L2 beside the attention pass (default 40, 0 = off). */
 int nm_debug_set_step_prefetch(int megabytes);
 /* Decode step: chain its kernels with programmatic dependent launch (default 1) or not (0). */

@@ -92,6 +92,7 @@ _lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _v
 _lib.nm_debug_set_attention.argtypes = [_i]
 _lib.nm_debug_set_step_pdl.argtypes = [_i]
 _lib.nm_debug_set_step_prefetch.argtypes = [_i]
+_lib.nm_debug_set_step_fusion.argtypes = [_i]
 _lib.nm_debug_set_attention_trace.argtypes = [_vp]
 
 
@@ -296,6 +297,10 @@ def nm_mla_decode_step_host(p: MlaParams, h_host, out_host, h_staging, out_stagi
 
 def nm_debug_set_attention_trace(buf) -> None:
     _check(_lib.nm_debug_set_attention_trace(_ptr(buf)), "nm_debug_set_attention_trace")
+
+
+def nm_debug_set_step_fusion(enable: bool) -> None:
+    _check(_lib.nm_debug_set_step_fusion(int(enable)), "nm_debug_set_step_fusion")
 
 
 def nm_debug_set_step_prefetch(megabytes: int) -> None:

@@ -1,0 +1,242 @@
+// Per-head stages of the single-token decode step, one CTA per head, each fused with the small vector
+// stage that feeds it (the paper's point that RMSNorm / RoPE-like consumers should start right where
+// the narrow product ends, MLA Operator Optimization section):
+//
+//   q_finish_kernel   q_rope[h] = RoPE(q[h, nope:]),  q_lat[h] = q[h, :nope] * W_UK[h]      (128 -> 512)
+//   uv_merge_kernel   o_lat[h]  = merge of the attention partials (+ the new cache row),
+//                     o[h]      = bf16(o_lat[h]) * W_UV[h]                                   (512 -> 128)
+//
+// Both stream the head's 128 KB of weights with 32 independent 16-byte read-only loads per thread,
+// the first batches issued before the programmatic-launch wait (weights do not depend on earlier
+// kernels), accumulate in fp32, reduce the row groups through shared memory and round once to bf16.
+#include "nm_async.cuh"
+#include "nm_mla.cuh"
+
+namespace nm {
+
+namespace {
+
+constexpr int kHeadThreads = 256;
+
+__device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+__device__ __forceinline__ uint16_t f32_to_bf16(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+
+__device__ __forceinline__ float block_sum_256(float v, float *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kHeadThreads / 32; ++w) t += scratch[w];
+    return t;
+}
+
+// y[0..N) = x[0..K) * W[K][N] (row-major bf16), x in shared memory as fp32.  256 threads: N/8 column
+// groups x (2048/N) row groups, 32 rows per thread.  `w` holds this thread's 32 weight vectors, loaded
+// by the caller (so that the loads can be issued before the inputs exist).
+template <int K, int N>
+struct HeadMatvec {
+    static constexpr int kColGroups = N / 8;
+    static constexpr int kRowGroups = kHeadThreads / kColGroups;
+    static constexpr int kRowsPerThread = K / kRowGroups;
+    static_assert(kRowsPerThread == 32, "shapes of the absorbed MLA products: 128x512 and 512x128");
+
+    __device__ static __forceinline__ void load(const uint16_t *__restrict__ W, uint4 (&w)[32], int first, int count)
+    {
+        const int tx = threadIdx.x % kColGroups, ty = threadIdx.x / kColGroups;
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i >= first && i < first + count) w[i] = ld_stream16(W + (size_t)(ty + i * kRowGroups) * N + tx * 8);
+    }
+
+    // returns in `out8` the 8 column sums of this thread's column group when ty == 0 (others: unspecified)
+    __device__ static __forceinline__ void run(const uint4 (&w)[32], const float *x_s, float *red /* kRowGroups*N floats */, float (&out8)[8])
+    {
+        const int tx = threadIdx.x % kColGroups, ty = threadIdx.x / kColGroups;
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            float b[8];
+            Elem<bf16_t>::unpack(w[i], b);
+            const float a = x_s[ty + i * kRowGroups];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = fmaf(a, b[j], acc[j]);
+        }
+        float4 *dst = reinterpret_cast<float4 *>(red + (size_t)ty * N + tx * 8);
+        dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+        __syncthreads();
+        if (ty == 0) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) out8[j] = 0.f;
+            for (int g = 0; g < kRowGroups; ++g) {                 // fixed order: deterministic
+                const float4 *src = reinterpret_cast<const float4 *>(red + (size_t)g * N + tx * 8);
+                const float4 v0 = src[0], v1 = src[1];
+                out8[0] += v0.x; out8[1] += v0.y; out8[2] += v0.z; out8[3] += v0.w;
+                out8[4] += v1.x; out8[5] += v1.y; out8[6] += v1.z; out8[7] += v1.w;
+            }
+        }
+    }
+};
+
+__device__ __forceinline__ uint4 pack8_bf16(const float (&v)[8])
+{
+    return make_uint4((uint32_t)f32_to_bf16(v[0]) | ((uint32_t)f32_to_bf16(v[1]) << 16),
+                      (uint32_t)f32_to_bf16(v[2]) | ((uint32_t)f32_to_bf16(v[3]) << 16),
+                      (uint32_t)f32_to_bf16(v[4]) | ((uint32_t)f32_to_bf16(v[5]) << 16),
+                      (uint32_t)f32_to_bf16(v[6]) | ((uint32_t)f32_to_bf16(v[7]) << 16));
+}
+
+// q: [H][nope+rope] bf16; W_UK: [H][nope][dc]; q_full: [H][dc+rope] (q_lat | q_rope).  nope = 128, dc = 512.
+__global__ void __launch_bounds__(kHeadThreads) q_finish_kernel(const uint16_t *__restrict__ q, const uint16_t *__restrict__ W_UK,
+                                                                const float *__restrict__ cs, uint16_t *__restrict__ q_full, int rope)
+{
+    constexpr int K = 128, N = 512;
+    using MV = HeadMatvec<K, N>;
+    __shared__ __align__(16) float x_s[K];
+    __shared__ __align__(16) float red[MV::kRowGroups * N];
+    const int h = blockIdx.x;
+    const uint16_t *W = W_UK + (size_t)h * K * N;
+    uint4 w[32];
+    MV::load(W, w, 0, 32);                                        // weights first: they depend on nothing
+    pdl_launch_dependents();
+    pdl_wait_prior_grids();                                       // q comes from the W_UQR product
+    const uint16_t *qh = q + (size_t)h * (K + rope);
+    if (threadIdx.x < K) x_s[threadIdx.x] = bf16_to_f32(qh[threadIdx.x]);
+    if (threadIdx.x < rope / 2) {                                 // interleaved pairs, rounded to bf16
+        const int i = threadIdx.x;
+        const float c = cs[2 * i], s = cs[2 * i + 1];
+        const float x0 = bf16_to_f32(qh[K + 2 * i]), x1 = bf16_to_f32(qh[K + 2 * i + 1]);
+        uint16_t *dst = q_full + (size_t)h * (N + rope) + N + 2 * i;
+        *reinterpret_cast<uint32_t *>(dst) = (uint32_t)f32_to_bf16(x0 * c - x1 * s) | ((uint32_t)f32_to_bf16(x0 * s + x1 * c) << 16);
+    }
+    __syncthreads();
+    float out8[8];
+    MV::run(w, x_s, red, out8);
+    if (threadIdx.x / MV::kColGroups == 0)
+        *reinterpret_cast<uint4 *>(q_full + (size_t)h * (N + rope) + (threadIdx.x % MV::kColGroups) * 8) = pack8_bf16(out8);
+}
+
+// Merge of the attention partials (see attn_combine_kernel for the algebra) followed by W_UV.
+// dc = 512, dv = 128.
+__global__ void __launch_bounds__(kHeadThreads) uv_merge_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
+                                                                AttnPartials part, int npart, long extra_row, int rope, float scale,
+                                                                const uint16_t *__restrict__ W_UV, uint16_t *__restrict__ o_lat_bf16,
+                                                                float *__restrict__ o_lat_f32, uint16_t *__restrict__ o)
+{
+    constexpr int K = 512, N = 128;
+    using MV = HeadMatvec<K, N>;
+    __shared__ __align__(16) float x_s[K];
+    __shared__ __align__(16) float red[MV::kRowGroups * N];
+    __shared__ float scratch[32];
+    __shared__ float sm[kMaxAttnSplits], sl[kMaxAttnSplits], sw[kMaxAttnSplits];
+    const int h = blockIdx.x, H = gridDim.x, dkv = K + rope, tid = threadIdx.x;
+    const uint16_t *W = W_UV + (size_t)h * K * N;
+    uint4 w[32];
+    MV::load(W, w, 0, 16);                                        // half of the weights before the inputs exist
+    pdl_launch_dependents();
+    pdl_wait_prior_grids();                                       // partials come from the attention kernel
+    for (int s = tid; s < npart; s += kHeadThreads) {
+        const float2 v = __ldcg(reinterpret_cast<const float2 *>(part.ml + ((size_t)s * H + h) * 2));
+        sm[s] = v.x; sl[s] = v.y;
+    }
+    // two columns per thread; the partial rows of up to 8 parts in flight
+    const int c = 2 * tid;
+    const float *src = part.O + (size_t)h * K + c;
+    constexpr int kBatch = 8;
+    float2 v[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u)
+        v[u] = (u < npart) ? __ldcg(reinterpret_cast<const float2 *>(src + (size_t)u * H * K)) : make_float2(0.f, 0.f);
+    float sx = -INFINITY;
+    if (extra_row >= 0) {
+        const uint16_t *qh = Q + (size_t)h * dkv, *row = cache + (size_t)extra_row * dkv;
+        float acc = 0.f;
+        for (int i = tid; i < dkv; i += kHeadThreads) acc = fmaf(bf16_to_f32(qh[i]), bf16_to_f32(row[i]), acc);
+        sx = block_sum_256(acc, scratch) * scale;
+    } else {
+        __syncthreads();
+    }
+    float Mx = sx;
+    for (int s = 0; s < npart; ++s) Mx = fmaxf(Mx, sm[s]);
+    const float wx = (extra_row >= 0) ? __expf(sx - Mx) : 0.f;
+    float L = wx;
+    for (int s = 0; s < npart; ++s) {                              // same order in every thread
+        const float wgt = (sm[s] == -INFINITY) ? 0.f : __expf(sm[s] - Mx);
+        if (tid == 0) sw[s] = wgt;
+        L = fmaf(wgt, sl[s], L);
+    }
+    __syncthreads();
+    float2 acc = make_float2(0.f, 0.f);
+    if (extra_row >= 0) {
+        const uint32_t rv = *reinterpret_cast<const uint32_t *>(cache + (size_t)extra_row * dkv + c);
+        acc = make_float2(wx * __uint_as_float(rv << 16), wx * __uint_as_float(rv & 0xffff0000u));
+    }
+    for (int s0 = 0; s0 < npart; s0 += kBatch) {
+        if (s0 > 0) {
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+                v[u] = (s0 + u < npart) ? __ldcg(reinterpret_cast<const float2 *>(src + (size_t)(s0 + u) * H * K)) : make_float2(0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const float wgt = (s0 + u < npart) ? sw[s0 + u] : 0.f;
+            acc.x = fmaf(wgt, v[u].x, acc.x);
+            acc.y = fmaf(wgt, v[u].y, acc.y);
+        }
+    }
+    MV::load(W, w, 16, 16);                                       // the other half of the weights
+    const float inv = 1.0f / L;
+    const float o0 = acc.x * inv, o1 = acc.y * inv;
+    const uint16_t b0 = f32_to_bf16(o0), b1 = f32_to_bf16(o1);
+    if (o_lat_f32) *reinterpret_cast<float2 *>(o_lat_f32 + (size_t)h * K + c) = make_float2(o0, o1);
+    if (o_lat_bf16) *reinterpret_cast<uint32_t *>(o_lat_bf16 + (size_t)h * K + c) = (uint32_t)b0 | ((uint32_t)b1 << 16);
+    x_s[c] = bf16_to_f32(b0);                                      // W_UV sees the rounded o_lat, as the stage-wise definition says
+    x_s[c + 1] = bf16_to_f32(b1);
+    __syncthreads();
+    float out8[8];
+    MV::run(w, x_s, red, out8);
+    if (tid / MV::kColGroups == 0) *reinterpret_cast<uint4 *>(o + (size_t)h * N + (tid % MV::kColGroups) * 8) = pack8_bf16(out8);
+}
+
+template <typename... Args>
+cudaError_t launch_with_pdl(void (*kern)(Args...), int grid, cudaStream_t s, bool pdl, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kHeadThreads); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
+}  // namespace
+
+bool head_kernels_apply(int H, int nope, int rope, int dc, int dv)
+{
+    return H >= 1 && nope == 128 && dc == 512 && dv == 128 && rope >= 2 && rope <= 2 * kHeadThreads && (rope & 1) == 0;
+}
+
+int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl)
+{
+    cudaError_t e = launch_with_pdl(q_finish_kernel, H, s, pdl, (const uint16_t *)q, (const uint16_t *)W_UK, cos_sin, (uint16_t *)q_full, rope);
+    return e == cudaSuccess ? NM_OK : record_cuda_error(e, "q_finish launch");
+}
+
+int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
+                    const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl)
+{
+    cudaError_t e = launch_with_pdl(uv_merge_kernel, H, s, pdl, (const uint16_t *)Q, (const uint16_t *)cache, part, npart, extra_row, rope,
+                                    scale, (const uint16_t *)W_UV, (uint16_t *)o_lat_bf16, o_lat_f32, (uint16_t *)o);
+    return e == cudaSuccess ? NM_OK : record_cuda_error(e, "uv_merge launch");
+}
+
+}  // namespace nm

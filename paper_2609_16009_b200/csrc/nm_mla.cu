@@ -333,6 +333,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 // ---- host -------------------------------------------------------------------------------------------
 
 static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
+static int g_fused_heads = 1;        // per-head stages fused with their vector stage (q_finish, uv_merge) when the dims allow
 static int g_prefetch_mb = 40;       // MB of W_O pulled into L2 beside the attention pass (plus all of W_UV); 0 = off
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -513,11 +514,17 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl && (!forked || p->programmatic_entry)));
     NM_LAUNCH(rmsnorm_kernel, 1, 256, ms, (const uint16_t *)c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
     NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl));
-    NM_LAUNCH(rope_kernel, ceil_div(H * dr / 2, 256), 256, ms, (const uint16_t *)(q + dn), q_full + dc, H, dr, (long)dq, (long)dkv,
-              p->rope_cos_sin);
-    // q_lat[h] = q[h, :nope] * W_UK[h], written straight into the attention operand [H][dc+dr]
-    NM_TRY(matmul_enqueue(q, p->W_UK, q_full, 1, dc, dn, H, (long)H * dq, dq, (long)dn * dc, (long)H * dkv, dkv,
-                          NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms, pdl));
+    const bool fused = g_fused_heads && head_kernels_apply(H, dn, dr, dc, dv);
+    if (fused) {
+        // RoPE of the rope part and q_lat[h] = q[h, :nope] * W_UK[h] in one kernel, one CTA per head
+        NM_TRY(launch_q_finish(q, p->W_UK, p->rope_cos_sin, q_full, H, dr, ms, pdl));
+    } else {
+        NM_LAUNCH(rope_kernel, ceil_div(H * dr / 2, 256), 256, ms, (const uint16_t *)(q + dn), q_full + dc, H, dr, (long)dq, (long)dkv,
+                  p->rope_cos_sin);
+        // q_lat[h] = q[h, :nope] * W_UK[h], written straight into the attention operand [H][dc+dr]
+        NM_TRY(matmul_enqueue(q, p->W_UK, q_full, 1, dc, dn, H, (long)H * dq, dq, (long)dn * dc, (long)H * dkv, dkv,
+                              NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms, pdl));
+    }
 
     // ---- beside the attention pass: the side stream pulls W_UV and the head of every k-split of W_O into
     //      L2, so that the output-side products start from L2 instead of HBM (Data Independence: the
@@ -544,12 +551,17 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     // launched early: its CTAs could not share an SM with the attention CTAs (registers) and would
     // only hold up the prefetch kernel in the block scheduler.
     if (forked) NM_CUDA_TRY(cudaStreamWaitEvent(ms, g_events.join, 0));
-    NM_TRY(attention_combine(q_full, cache, o_lat, p->o_lat_f32, H, (int)pos, pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms,
-                             pdl && !forked));
-
-    // ---- output side -----------------------------------------------------------------------------------
-    NM_TRY(matmul_enqueue(o_lat, p->W_UV, o, 1, dv, dc, H, (long)H * dc, dc, (long)dc * dv, (long)H * dv, dv,
-                          NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms, pdl));
+    if (fused) {
+        // merge of the attention partials (+ the new row) and o[h] = o_lat[h] * W_UV[h] in one kernel
+        const AttnPlan ap = plan_attention(q_full, cache, H, (int)pos, dc);
+        NM_TRY(launch_uv_merge(q_full, cache, carve_partials(aws, H), ap.npartial, pos, dr, p->softmax_scale, p->W_UV, o_lat,
+                               p->o_lat_f32, o, H, ms, pdl && !forked));
+    } else {
+        NM_TRY(attention_combine(q_full, cache, o_lat, p->o_lat_f32, H, (int)pos, pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms,
+                                 pdl && !forked));
+        NM_TRY(matmul_enqueue(o_lat, p->W_UV, o, 1, dv, dc, H, (long)H * dc, dc, (long)dc * dv, (long)H * dv, dv,
+                              NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms, pdl));
+    }
     if (p->W_O) {
         if (p->event_before_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_before_wo, ms));
         NM_TRY(matmul_enqueue(o, p->W_O, p->out, 1, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms,
@@ -657,6 +669,13 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     NM_CUDA_TRY(cudaMemcpyAsync(h_staging, h_host, (size_t)p->d * 2, cudaMemcpyHostToDevice, ms));
     NM_TRY(step_impl(&q, ms, (cudaStream_t)side_stream));
     NM_CUDA_TRY(cudaMemcpyAsync(out_host, out_staging, (size_t)p->d * 2, cudaMemcpyDeviceToHost, ms));
+    return NM_OK;
+}
+
+/* 1 (default): RoPE + W_UK and merge + W_UV run as fused per-head kernels; 0: separate kernels. */
+int nm_debug_set_step_fusion(int enable)
+{
+    g_fused_heads = enable ? 1 : 0;
     return NM_OK;
 }
 

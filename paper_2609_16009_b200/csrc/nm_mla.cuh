@@ -30,6 +30,12 @@ AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int
 int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows,
                          float scale, cudaStream_t stream, bool programmatic_launch);
 
+// Fused per-head stages of the decode step (nm_head_kernels.cu); they take nope = 128, kv_lora = 512, v = 128.
+bool head_kernels_apply(int H, int nope, int rope, int dc, int dv);
+int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl);
+int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
+                    const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl);
+
 // Tuning aid: 12 phase timestamps (ns) of CTA (0,0) of the tensor-core kernel go to `p` when non-null.
 void set_attention_trace(unsigned long long *p);
 

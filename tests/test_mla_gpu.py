@@ -261,6 +261,27 @@ def test_decode_step_other_lengths(nm, weights, S):
     check_step(t, r, cache_ref, S)
 
 
+def test_decode_step_fused_and_unfused_per_head_stages_agree(nm, weights, ref1024):
+    w, dw = weights
+    h, cache_ref, r = ref1024
+    cache_in = gen.mla_cache(1024, DIMS, seed=4200)
+    t1 = run_step(nm, dw, h, cache_in, 1024)
+    nm.nm_debug_set_step_fusion(False)
+    try:
+        t2 = run_step(nm, dw, h, cache_in, 1024)
+        check_step(t2, r, cache_ref, 1024)
+    finally:
+        nm.nm_debug_set_step_fusion(True)
+    # the two routes sum in different orders: q_full is the same bf16 value up to a rounding flip on a few
+    # elements; what follows the softmax inherits those flips and is compared on the scale of the tensor
+    a, b = dev_bits_to_f64(t1["q_full"]), dev_bits_to_f64(t2["q_full"])
+    assert np.all(np.abs(a - b) <= 2 * oracle.ulp_bf16(b) + 1e-6)
+    assert np.mean(a == b) > 0.97
+    for k in ("o_lat", "o", "out"):
+        a, b = dev_bits_to_f64(t1[k]), dev_bits_to_f64(t2[k])
+        assert np.all(np.abs(a - b) <= 2e-3 * np.abs(b).max() + oracle.ulp_bf16(b)), k      # rounded outputs: one ulp on top
+
+
 def test_decode_step_without_wo_and_repeatable(nm, weights):
     w, dw = weights
     S = 300

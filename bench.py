@@ -108,12 +108,18 @@ class MlaStep:
 
     name = "mla"
 
-    def __init__(self, nm, device, seq_len, seed=4000):
+    def __init__(self, nm, device, seq_len, seed=4000, schedule="two-stream"):
         self.nm = nm
         self.S = seq_len
+        self.schedule = schedule
         d, ql, dc, dr, dn, dv, H = (DIMS[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
         w = gen.mla_weights(DIMS, seed=seed, with_wo=True)
         t = {k: torch.from_numpy(v.view(np.int16)).to(device) for k, v in w.items()}
+        if schedule == "fused":
+            # the three down-projections stored as one matrix (W_DQ | W_DKV | W_KR): a storage choice made
+            # when the weights are loaded, like the paper's concatenation of W_DKV and W_KR
+            t["W_DQKV"] = torch.from_numpy(np.concatenate([w["W_DQ"], w["W_DKVKR"]], axis=1).view(np.int16)).to(device)
+            del t["W_DQ"], t["W_DKVKR"]
         self.h_host = torch.from_numpy(gen.mla_token(DIMS, seed=seed + 100).view(np.int16).copy()).pin_memory()
         self.out_host = torch.empty(d, dtype=torch.int16).pin_memory()
         t["h"] = self.h_host.to(device)
@@ -137,7 +143,7 @@ class MlaStep:
         # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this shape, from
         # the ncu capture summarised in profiles/ncu_nm_row_tma_WO_M1_K16384_N7168.txt
         self.dominant_traffic = 234_948_352 + 3_600_128
-        self.launches_per_step = 11
+        self.launches_per_step = 7 if schedule == "fused" else 9
         self.h2d = d * 2
         self.d2h = d * 2
 
@@ -146,8 +152,11 @@ class MlaStep:
                             f"nope 128, v 128, 128 heads), seq_len {self.S}, bf16 weights row-major, W_O included",
                 "seq_len": self.S,
                 "l2": "weights 374 MB per step > 126 MB L2, so every step streams from HBM; no flush",
-                "overlap": "side stream: KV chain beside the W_DQ product, L2 prefetch of W_UV/W_O beside the tcgen05 attention pass; "
-                           "programmatic dependent launch along the main stream, also across steps"}
+                "schedule": self.schedule,
+                "overlap": ("one stream: h*(W_DQ|W_DKV|W_KR) as one product; " if self.schedule == "fused" else
+                            "two streams: KV chain (W_DKV|KR product, RMSNorm, RoPE, cache write) beside the W_DQ product; ")
+                           + "L2 prefetch of W_UV/W_O by idle lanes of the tcgen05 attention kernel; programmatic dependent "
+                             "launch along the chain, also across steps"}
 
     def step(self, stream, dom_events=None):
         if dom_events is not None:
@@ -257,7 +266,7 @@ def make_workload(args, nm, device):
     if args.workload == "projections":
         return ProjectionChain(nm, device)
     if args.workload == "mla":
-        return MlaStep(nm, device, args.seq_len)
+        return MlaStep(nm, device, args.seq_len, schedule=args.schedule)
     if args.workload == "matmul":
         M, K, N = (int(x) for x in args.mkn.split(","))
         return SingleProduct(nm, device, M, K, N, 1 if args.layout == "col" else 0)
@@ -480,6 +489,8 @@ def main():
     ap.add_argument("--workload", default="mla", choices=["mla", "projections", "matmul", "attention"])
     ap.add_argument("--mkn", default="1,16384,7168", help="M,K,N of --workload matmul")
     ap.add_argument("--layout", default="row", choices=["row", "col"])
+    ap.add_argument("--schedule", default="two-stream", choices=["fused", "two-stream"],
+                    help="decode step: down-projections as one concatenated product on one stream, or W_DKV|KR on a side stream")
     ap.add_argument("--timeline", action="store_true", help="print the kernel timeline of one step and exit")
     ap.add_argument("--sweep", action="store_true", help="also report GB/s of single narrow products vs M")
     ap.add_argument("--seq-len", type=int, default=4096)

@@ -240,6 +240,11 @@ typedef struct {
      * before the step on main_stream is still running - back-to-back layers or steps.  Only valid if
      * that earlier work writes none of this step's weights.  0 keeps the ordinary stream order. */
     int programmatic_entry;
+    /* optional: the three down-projections stored as ONE row-major matrix [d][q_lora + kv_lora + rope] =
+     * (W_DQ | W_DKV | W_KR), the paper's concatenation of Eq. 3 extended by W_DQ (all three multiply the
+     * same h).  When given (and layout_dense is row-major) the step computes them as one product on
+     * main_stream and needs no side stream; W_DQ and W_DKVKR are then ignored and may be NULL. */
+    const void *W_DQKV;
 } nm_mla_params;
 
 size_t nm_mla_workspace_bytes(const nm_mla_params *p);
@@ -278,10 +283,13 @@ int nm_debug_set_kernel(int kind, int stages);
  * start, set-up done, Q landed, first tile landed, scores ready, P written, last P*V done, after
  * cluster barrier 1, O parked in shared memory, after barrier 2, cluster sum written, end.  NULL = off. */
 int nm_debug_set_attention_trace(void *device_buffer);
+/* Decode step tuning: launch the merge + W_UV kernel programmatically (default 1); include W_UV in the L2
+ * prefetch (default 1). */
+int nm_debug_set_step_knobs(int uv_programmatic, int prefetch_w_uv);
 /* Decode step: 1 (default) runs RoPE + W_UK and attention-merge + W_UV as fused per-head kernels, 0 as
  * separate kernels (rope, batched product, merge, batched product). */
 int nm_debug_set_step_fusion(int enable);
-/* Decode step: MB of W_O prefetched into L2 beside the attention pass (default 40, 0 = off). */
+/* Decode step: MB of W_O that the attention kernel's softmax threads prefetch into L2 (default 40, 0 = off). */
 int nm_debug_set_step_prefetch(int megabytes);
 /* Decode step: chain its kernels with programmatic dependent launch (default 1) or not (0). */
 int nm_debug_set_step_pdl(int enable);

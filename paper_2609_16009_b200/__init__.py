@@ -74,7 +74,7 @@ class MlaParams(C.Structure):
                 + [("workspace_bytes", _sz)]
                 + [(n, _vp) for n in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o", "o_lat_f32",
                                       "event_before_wo", "event_after_wo")]
-                + [("programmatic_entry", _i)])
+                + [("programmatic_entry", _i), ("W_DQKV", _vp)])
 
 
 _lib.nm_rmsnorm.argtypes = [_vp, _vp, _vp, _i, C.c_float, _vp]

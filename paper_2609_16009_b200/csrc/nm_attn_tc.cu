@@ -100,7 +100,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, AttnPartials part,
-               int n_rows, int rows_per_split, float scale_log2, unsigned *status, unsigned long long *trace)
+               int n_rows, int rows_per_split, float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
 {
     // Optional phase timestamps (ns) of CTA (0,0), for tuning: trace[i] is written when non-null.
 #define NM_TRACE(i) do { if (trace && blockIdx.x == 0 && blockIdx.y == 0) trace[i] = global_timer_ns(); } while (0)
@@ -143,6 +143,33 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const uint32_t rank = cluster_rank();
     const int cluster_id = sp / kCl;
     float m_own = -INFINITY, l_own = 0.f;                         // softmax threads: this split's (m, l)
+
+    // The softmax threads, once the scores of their first tile are in (so that the tile loads, which the
+    // whole pass waits for, do not queue behind it), pull the weights of the products that follow the
+    // attention - W_UV and the head of every k-split of W_O - into L2 in 4 KB bulk prefetches: the pass
+    // needs little HBM bandwidth, and those weights do not depend on its result.
+    auto prefetch_weights = [&]() {
+        constexpr long kChunk = 4096;
+        const long block_chunks = (pf.block_bytes + kChunk - 1) / kChunk;
+        const long chunks_per_range = (pf.range_bytes + kChunk - 1) / kChunk;
+        const long total = block_chunks + chunks_per_range * pf.nranges;
+        const long nthreads = (long)gridDim.x * gridDim.y * 128;
+        const long me = ((long)blockIdx.y * gridDim.x + blockIdx.x) * 128 + (tid - 64);
+        for (long i = me; i < total; i += nthreads) {
+            const char *ptr;
+            long n;
+            if (i < block_chunks) {
+                ptr = pf.block + i * kChunk;
+                n = min(kChunk, pf.block_bytes - i * kChunk);
+            } else {
+                const long j = i - block_chunks, r = j / chunks_per_range, off = (j - r * chunks_per_range) * kChunk;
+                ptr = pf.base + r * pf.range_stride + off;
+                n = min(kChunk, pf.range_bytes - off);
+            }
+            n &= ~15L;
+            if (n > 0) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr), "r"((uint32_t)n) : "memory");
+        }
+    };
 
     if (warp == 0) {
         // ---------------- TMA producer --------------------------------------------------------------
@@ -241,11 +268,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const int quad = warp & 3;                                 // TMEM lanes this warp may touch
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
         float m_used = -INFINITY, l = 0.f;
+        if (ntiles == 0) prefetch_weights();
         for (int t = 0; t < ntiles; ++t) {
             const int b = t & 1;
             mbar_wait(bar_s_full + 8 * b, (t >> 1) & 1, &s_abort, status);
             tc_fence_after();
             if (t == 0 && tid == 64) NM_TRACE(4);
+            if (t == 0) prefetch_weights();
             uint32_t sr[32];
             tmem_ld32(lane_base + kColS + 32 * b, sr);
             tmem_wait_ld();
@@ -422,7 +451,7 @@ static unsigned long long *g_attn_trace = nullptr;
 void set_attention_trace(unsigned long long *p) { g_attn_trace = p; }
 
 int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows, float scale,
-                         cudaStream_t stream, bool programmatic_launch)
+                         cudaStream_t stream, bool programmatic_launch, L2Prefetch prefetch)
 {
     if (n_rows < 1 || plan.nsplit < 1) return NM_ERR_UNSUPPORTED;
     if (((uintptr_t)Q & 15u) || ((uintptr_t)cache & 15u)) return NM_ERR_UNSUPPORTED;
@@ -450,7 +479,7 @@ int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, At
     cfg.attrs = attr;
     cfg.numAttrs = programmatic_launch ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, map_q, map_kv, part, n_rows, plan.rows_per_split, scale_log2,
-                                       device_status_ptr(), g_attn_trace);
+                                       device_status_ptr(), g_attn_trace, prefetch);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (tensor cores) launch");
 }
 

@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(kHeadThreads) uv_merge_kernel(const uint16_t *
     const int h = blockIdx.x, H = gridDim.x, dkv = K + rope, tid = threadIdx.x;
     const uint16_t *W = W_UV + (size_t)h * K * N;
     uint4 w[32];
-    MV::load(W, w, 0, 16);                                        // half of the weights before the inputs exist
+    MV::load(W, w, 0, 32);                                        // all of the head's weights before the inputs exist
     pdl_launch_dependents();
     pdl_wait_prior_grids();                                       // partials come from the attention kernel
     for (int s = tid; s < npart; s += kHeadThreads) {
@@ -191,7 +191,6 @@ __global__ void __launch_bounds__(kHeadThreads) uv_merge_kernel(const uint16_t *
             acc.y = fmaf(wgt, v[u].y, acc.y);
         }
     }
-    MV::load(W, w, 16, 16);                                       // the other half of the weights
     const float inv = 1.0f / L;
     const float o0 = acc.x * inv, o1 = acc.y * inv;
     const uint16_t b0 = f32_to_bf16(o0), b1 = f32_to_bf16(o1);
@@ -203,6 +202,64 @@ __global__ void __launch_bounds__(kHeadThreads) uv_merge_kernel(const uint16_t *
     float out8[8];
     MV::run(w, x_s, red, out8);
     if (tid / MV::kColGroups == 0) *reinterpret_cast<uint4 *>(o + (size_t)h * N + (tid % MV::kColGroups) * 8) = pack8_bf16(out8);
+}
+
+// The vector stages behind the fused down-projection h * (W_DQ | W_DKV | W_KR): CTA 0 normalises the
+// query latent (c_qn = RMSNorm(c_q; gamma_q)), CTA 1 finishes the cache row (RMSNorm of the KV latent,
+// RoPE of the key part).  x: [q_lora + dc + rope] bf16 as the product wrote it.
+__global__ void __launch_bounds__(kHeadThreads) down_finish_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ gamma_q,
+                                                                   const uint16_t *__restrict__ gamma_kv, const float *__restrict__ cs,
+                                                                   uint16_t *__restrict__ c_qn, uint16_t *__restrict__ cache_row,
+                                                                   int q_lora, int dc, int rope, float eps)
+{
+    __shared__ float scratch[32];
+    const int tid = threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait_prior_grids();
+    if (blockIdx.x == 0) {
+        // up to 8 elements per thread (q_lora <= 2048, multiple of 8 checked by the host)
+        const int i0 = 8 * tid;
+        float f[8], g[8];
+        const bool on = i0 < q_lora;
+        if (on) {
+            Elem<bf16_t>::unpack(*reinterpret_cast<const uint4 *>(x + i0), f);
+            Elem<bf16_t>::unpack(__ldg(reinterpret_cast<const uint4 *>(gamma_q + i0)), g);
+        }
+        float ss = 0.f;
+        if (on)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+        ss = block_sum_256(ss, scratch);
+        const float r = 1.0f / sqrtf(ss / (float)q_lora + eps);
+        if (on) {
+            float y[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) y[e] = f[e] * r * g[e];
+            *reinterpret_cast<uint4 *>(c_qn + i0) = pack8_bf16(y);
+        }
+    } else {
+        const uint16_t *ckr = x + q_lora;
+        const int i0 = 2 * tid;                                    // dc <= 512
+        float x0 = 0.f, x1 = 0.f, g0 = 0.f, g1 = 0.f;
+        if (i0 < dc) {
+            const uint32_t xv = *reinterpret_cast<const uint32_t *>(ckr + i0), gv = *reinterpret_cast<const uint32_t *>(gamma_kv + i0);
+            x0 = __uint_as_float(xv << 16); x1 = __uint_as_float(xv & 0xffff0000u);
+            g0 = __uint_as_float(gv << 16); g1 = __uint_as_float(gv & 0xffff0000u);
+        }
+        float r0v = 0.f, r1v = 0.f, c = 0.f, sn = 0.f;
+        if (tid < rope / 2) {
+            const uint32_t rv = *reinterpret_cast<const uint32_t *>(ckr + dc + i0);
+            r0v = __uint_as_float(rv << 16); r1v = __uint_as_float(rv & 0xffff0000u);
+            c = cs[i0]; sn = cs[i0 + 1];
+        }
+        const float ss = block_sum_256(fmaf(x0, x0, x1 * x1), scratch);
+        const float r = 1.0f / sqrtf(ss / (float)dc + eps);
+        if (i0 < dc)
+            *reinterpret_cast<uint32_t *>(cache_row + i0) = (uint32_t)f32_to_bf16(x0 * r * g0) | ((uint32_t)f32_to_bf16(x1 * r * g1) << 16);
+        if (tid < rope / 2)
+            *reinterpret_cast<uint32_t *>(cache_row + dc + i0) =
+                (uint32_t)f32_to_bf16(r0v * c - r1v * sn) | ((uint32_t)f32_to_bf16(r0v * sn + r1v * c) << 16);
+    }
 }
 
 template <typename... Args>
@@ -223,6 +280,19 @@ cudaError_t launch_with_pdl(void (*kern)(Args...), int grid, cudaStream_t s, boo
 bool head_kernels_apply(int H, int nope, int rope, int dc, int dv)
 {
     return H >= 1 && nope == 128 && dc == 512 && dv == 128 && rope >= 2 && rope <= 2 * kHeadThreads && (rope & 1) == 0;
+}
+
+bool down_finish_applies(int q_lora, int dc, int rope)
+{
+    return q_lora % 8 == 0 && q_lora <= 8 * kHeadThreads && dc % 2 == 0 && dc <= 2 * kHeadThreads && rope % 2 == 0 && rope <= dc;
+}
+
+int launch_down_finish(const void *x, const void *gamma_q, const void *gamma_kv, const float *cos_sin, void *c_qn, void *cache_row,
+                       int q_lora, int dc, int rope, float eps, cudaStream_t s, bool pdl)
+{
+    cudaError_t e = launch_with_pdl(down_finish_kernel, 2, s, pdl, (const uint16_t *)x, (const uint16_t *)gamma_q, (const uint16_t *)gamma_kv,
+                                    cos_sin, (uint16_t *)c_qn, (uint16_t *)cache_row, q_lora, dc, rope, eps);
+    return e == cudaSuccess ? NM_OK : record_cuda_error(e, "down_finish launch");
 }
 
 int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl)

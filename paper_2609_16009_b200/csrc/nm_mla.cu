@@ -143,33 +143,6 @@ __global__ void __launch_bounds__(256) kv_finish_kernel(const uint16_t *__restri
             (uint32_t)f32_to_bf16_bits(r0v * c - r1v * sn) | ((uint32_t)f32_to_bf16_bits(r0v * sn + r1v * c) << 16);
 }
 
-// Pull weight bytes into L2 ahead of the products that will stream them: one contiguous block (W_UV)
-// and `nranges` ranges of `range_bytes`, `range_stride` apart (the head of every k-split of W_O), in
-// 4 KB bulk prefetches.  Issued on the side stream while the tensor-core attention pass (which needs
-// little HBM bandwidth) runs on the main stream; the CTAs need no shared memory, so they fit beside it.
-__global__ void __launch_bounds__(128) l2_prefetch_kernel(const char *__restrict__ block, long block_bytes,
-                                                          const char *__restrict__ base, long range_stride, int nranges, long range_bytes)
-{
-    constexpr long kChunk = 4096;
-    const long block_chunks = (block_bytes + kChunk - 1) / kChunk;
-    const long chunks_per_range = (range_bytes + kChunk - 1) / kChunk;
-    const long total = block_chunks + chunks_per_range * nranges;
-    for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
-        const char *p;
-        long n;
-        if (i < block_chunks) {
-            p = block + i * kChunk;
-            n = min(kChunk, block_bytes - i * kChunk);
-        } else {
-            const long j = i - block_chunks, r = j / chunks_per_range, off = (j - r * chunks_per_range) * kChunk;
-            p = base + r * range_stride + off;
-            n = min(kChunk, range_bytes - off);
-        }
-        n &= ~15L;
-        if (n > 0) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"((uint32_t)n) : "memory");
-    }
-}
-
 // ---- attention over a split of the rows on CUDA cores (kept for sequence splits the tensor-core
 //      kernel does not take: fewer rows than one MMA tile) -------------------------------------------------
 //
@@ -334,6 +307,8 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 
 static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
 static int g_fused_heads = 1;        // per-head stages fused with their vector stage (q_finish, uv_merge) when the dims allow
+static int g_uv_pdl = 1;             // tuning: launch uv_merge programmatically
+static int g_prefetch_uv = 1;        // tuning: include W_UV in the L2 prefetch
 static int g_prefetch_mb = 40;       // MB of W_O pulled into L2 beside the attention pass (plus all of W_UV); 0 = off
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -384,7 +359,7 @@ static cudaError_t launch_pdl(void (*kern)(Args...), dim3 grid, dim3 block, cuda
 }
 
 static int attention_partial(const void *Q, const void *cache, int H, int n_rows, int dc, int dr, float scale,
-                             void *ws, size_t ws_bytes, cudaStream_t s, bool pdl = false)
+                             void *ws, size_t ws_bytes, cudaStream_t s, bool pdl = false, L2Prefetch prefetch = L2Prefetch{})
 {
     if (!Q || !cache || !ws) return NM_ERR_INVALID_ARG;
     if (H < 1 || n_rows < 0 || dc != 512 || dr != 64) return NM_ERR_UNSUPPORTED;
@@ -392,7 +367,7 @@ static int attention_partial(const void *Q, const void *cache, int H, int n_rows
     if (n_rows == 0) return NM_OK;
     const AttnPlan p = plan_attention(Q, cache, H, n_rows, dc);
     AttnPartials part = carve_partials(ws, H);
-    if (p.tensor_core) return attention_partial_tc(Q, cache, part, p, n_rows, scale, s, pdl);
+    if (p.tensor_core) return attention_partial_tc(Q, cache, part, p, n_rows, scale, s, pdl, prefetch);
     cudaError_t e = launch_pdl(attn_partial_simt_kernel, dim3(p.nsplit, H), dim3(128), s, pdl, static_cast<const uint16_t *>(Q),
                                static_cast<const uint16_t *>(cache), part, n_rows, p.rows_per_split, dc, dr, scale);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (CUDA cores) launch");
@@ -416,7 +391,7 @@ static int attention_combine(const void *Q, const void *cache, void *o_bf16, flo
 // [attention partials][intermediates].  Each matmul workspace is [64 KB counters][partials].
 struct StepLayout {
     size_t main_ws, main_ws_bytes, side_ws, side_ws_bytes, attn, attn_bytes;
-    size_t c_q, c_qn, q, q_full, ckr, o_lat, o, total;
+    size_t c_q, c_qn, q, q_full, ckr, o_lat, o, x_down, total;
 };
 
 static StepLayout step_layout(const nm_mla_params *p)
@@ -428,7 +403,7 @@ static StepLayout step_layout(const nm_mla_params *p)
         const size_t b = nm_matmul_workspace_bytes(1, N, K, H, NM_BF16, NM_ROW_MAJOR);
         if (b > main_need) main_need = b;
     };
-    upd(p->q_lora, p->d, 1); upd(p->H * dq, p->q_lora, 1); upd(p->kv_lora, p->nope, p->H); upd(p->v, p->kv_lora, p->H);
+    upd(p->q_lora, p->d, 1); upd(p->q_lora + dkv, p->d, 1); upd(p->H * dq, p->q_lora, 1); upd(p->kv_lora, p->nope, p->H); upd(p->v, p->kv_lora, p->H);
     upd(p->d, p->H * p->v, 1);
     size_t off = 0;
     L.main_ws = off; L.main_ws_bytes = main_need; off += align_up(main_need, 256);
@@ -438,6 +413,7 @@ static StepLayout step_layout(const nm_mla_params *p)
     auto take = [&](size_t elems) { size_t o = off; off += align_up(elems * 2, 256); return o; };
     L.c_q = take(p->q_lora); L.c_qn = take(p->q_lora); L.q = take((size_t)p->H * dq); L.q_full = take((size_t)p->H * dkv);
     L.ckr = take(dkv); L.o_lat = take((size_t)p->H * p->kv_lora); L.o = take((size_t)p->H * p->v);
+    L.x_down = take((size_t)p->q_lora + dkv);
     L.total = off;
     return L;
 }
@@ -445,9 +421,9 @@ static StepLayout step_layout(const nm_mla_params *p)
 static int check_params(const nm_mla_params *p)
 {
     if (!p) return NM_ERR_INVALID_ARG;
-    if (!p->h || !p->W_DQ || !p->gamma_q || !p->W_UQR || !p->W_DKVKR || !p->gamma_kv || !p->W_UK || !p->W_UV ||
-        !p->rope_cos_sin || !p->kv_cache || !p->workspace)
+    if (!p->h || !p->gamma_q || !p->W_UQR || !p->gamma_kv || !p->W_UK || !p->W_UV || !p->rope_cos_sin || !p->kv_cache || !p->workspace)
         return NM_ERR_INVALID_ARG;
+    if (!p->W_DQKV && (!p->W_DQ || !p->W_DKVKR)) return NM_ERR_INVALID_ARG;
     if (p->W_O && !p->out) return NM_ERR_INVALID_ARG;
     if (p->d < 1 || p->q_lora < 1 || p->H < 1 || p->nope < 1 || p->v < 1 || p->seq_len < 1) return NM_ERR_INVALID_ARG;
     if (p->kv_lora != 512 || p->rope != 64) return NM_ERR_UNSUPPORTED;
@@ -460,7 +436,7 @@ static int check_params(const nm_mla_params *p)
 #define NM_LAUNCH_CHECK(what) do { cudaError_t _e = cudaGetLastError(); if (_e != cudaSuccess) return record_cuda_error(_e, what); } while (0)
 
 // Events used to fork the KV chain onto the side stream and join it again (created once per thread).
-struct StepEvents { cudaEvent_t fork = nullptr, join = nullptr, q_ready = nullptr; };
+struct StepEvents { cudaEvent_t fork = nullptr, join = nullptr; };
 static thread_local StepEvents g_events;
 
 static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
@@ -480,11 +456,10 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     uint16_t *o_lat = (uint16_t *)buf(p->o_lat, L.o_lat), *o = (uint16_t *)buf(p->o, L.o);
     uint16_t *cache = static_cast<uint16_t *>(p->kv_cache);
     void *mws = ws + L.main_ws, *sws = ws + L.side_ws, *aws = ws + L.attn;
-    const bool forked = (ss != ms);
+    const bool forked = (ss != ms) && !(p->W_DQKV && p->layout_dense == NM_ROW_MAJOR && down_finish_applies(p->q_lora, p->kv_lora, p->rope));
     if (forked && !g_events.fork) {
         NM_CUDA_TRY(cudaEventCreateWithFlags(&g_events.fork, cudaEventDisableTiming));
         NM_CUDA_TRY(cudaEventCreateWithFlags(&g_events.join, cudaEventDisableTiming));
-        NM_CUDA_TRY(cudaEventCreateWithFlags(&g_events.q_ready, cudaEventDisableTiming));
     }
 
     // Programmatic dependent launch inside the step: every kernel after the first on its stream may
@@ -498,21 +473,35 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         if (_e != cudaSuccess) return record_cuda_error(_e, #kern);                           \
     } while (0)
 
-    // ---- KV chain (the paper's MatMul 2 and its consumers) on the side stream, forked at the start so that
-    //      it shares the machine with the first products of the Q chain and is long done when the merge
-    //      needs the new cache row ---------------------------------------------------------------------------
-    if (forked) {
-        NM_CUDA_TRY(cudaEventRecord(g_events.fork, ms));
-        NM_CUDA_TRY(cudaStreamWaitEvent(ss, g_events.fork, 0));
-    }
-    NM_TRY(matmul_enqueue(p->h, p->W_DKVKR, ckr, 1, dkv, d, 1, d, 0, 0, dkv, 0, NM_BF16, lay, sws, L.side_ws_bytes, ss, false));
-    NM_LAUNCH(kv_finish_kernel, 1, 256, ss, (const uint16_t *)ckr, (const uint16_t *)p->gamma_kv, p->rope_cos_sin,
-              cache + (size_t)pos * dkv, dc, dr, p->rms_eps);
-    if (forked) NM_CUDA_TRY(cudaEventRecord(g_events.join, ss));
+    const bool fused_down = p->W_DQKV && lay == NM_ROW_MAJOR && down_finish_applies(ql, dc, dr);
+    if (fused_down) {
+        // ---- one product for all three down-projections, h * (W_DQ | W_DKV | W_KR) (Eq. 3 extended by W_DQ),
+        //      then both vector stages in one two-CTA kernel: no side stream, an unbroken programmatic chain
+        uint16_t *x_down = reinterpret_cast<uint16_t *>(ws + L.x_down);
+        NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws,
+                              L.main_ws_bytes, ms, pdl && p->programmatic_entry));
+        NM_TRY(launch_down_finish(x_down, p->gamma_q, p->gamma_kv, p->rope_cos_sin, c_qn, cache + (size_t)pos * dkv, ql, dc, dr,
+                                  p->rms_eps, ms, pdl));
+        if (p->c_q) NM_CUDA_TRY(cudaMemcpyAsync(p->c_q, x_down, (size_t)ql * 2, cudaMemcpyDeviceToDevice, ms));
+        if (p->ckr) NM_CUDA_TRY(cudaMemcpyAsync(p->ckr, x_down + ql, (size_t)dkv * 2, cudaMemcpyDeviceToDevice, ms));
+    } else {
+        // ---- KV chain (the paper's MatMul 2 and its consumers) on the side stream, forked at the start so that
+        //      it shares the machine with the first product of the Q chain and is long done when the merge
+        //      needs the new cache row -------------------------------------------------------------------------
+        if (forked) {
+            NM_CUDA_TRY(cudaEventRecord(g_events.fork, ms));
+            NM_CUDA_TRY(cudaStreamWaitEvent(ss, g_events.fork, 0));
+        }
+        NM_TRY(matmul_enqueue(p->h, p->W_DKVKR, ckr, 1, dkv, d, 1, d, 0, 0, dkv, 0, NM_BF16, lay, sws, L.side_ws_bytes, ss, false));
+        NM_LAUNCH(kv_finish_kernel, 1, 256, ss, (const uint16_t *)ckr, (const uint16_t *)p->gamma_kv, p->rope_cos_sin,
+                  cache + (size_t)pos * dkv, dc, dr, p->rms_eps);
+        if (forked) NM_CUDA_TRY(cudaEventRecord(g_events.join, ss));
 
-    // ---- Q chain, main stream ------------------------------------------------------------------------
-    NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl && (!forked || p->programmatic_entry)));
-    NM_LAUNCH(rmsnorm_kernel, 1, 256, ms, (const uint16_t *)c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
+        // ---- Q chain, main stream ----------------------------------------------------------------------------
+        NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms,
+                              pdl && (!forked || p->programmatic_entry)));
+        NM_LAUNCH(rmsnorm_kernel, 1, 256, ms, (const uint16_t *)c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
+    }
     NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl));
     const bool fused = g_fused_heads && head_kernels_apply(H, dn, dr, dc, dv);
     if (fused) {
@@ -526,27 +515,26 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
                               NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms, pdl));
     }
 
-    // ---- beside the attention pass: the side stream pulls W_UV and the head of every k-split of W_O into
-    //      L2, so that the output-side products start from L2 instead of HBM (Data Independence: the
-    //      weights do not depend on the attention result) ------------------------------------------------------
-    if (forked && g_prefetch_mb > 0 && pos > 0) {
-        NM_CUDA_TRY(cudaEventRecord(g_events.q_ready, ms));
-        NM_CUDA_TRY(cudaStreamWaitEvent(ss, g_events.q_ready, 0));
-        int kr = 0, ns = 0;
-        long rows = 0;
-        const long row_bytes = (long)d * 2;
+    // ---- beside the attention pass: idle lanes of the attention kernel pull W_UV and the head of every
+    //      k-split of W_O into L2, so that the output-side products start from L2 instead of HBM (Data
+    //      Independence: the weights do not depend on the attention result) -----------------------------------
+    L2Prefetch pf{};
+    if (g_prefetch_mb > 0 && pos > 0) {
+        pf.block = (const char *)p->W_UV;
+        pf.block_bytes = g_prefetch_uv ? (long)H * dc * dv * 2 : 0;
         if (p->W_O && lay == NM_ROW_MAJOR) {
+            int kr = 0, ns = 1;
             matmul_row_major_split(1, d, H * dv, 1, &kr, &ns);
-            rows = ((long)g_prefetch_mb << 20) / ns / row_bytes;
+            const long row_bytes = (long)d * 2;
+            long rows = ((long)g_prefetch_mb << 20) / ns / row_bytes;
             if (rows > kr) rows = kr;
+            pf.base = (const char *)p->W_O; pf.range_stride = (long)kr * row_bytes; pf.nranges = rows > 0 ? ns : 0;
+            pf.range_bytes = rows * row_bytes;
         }
-        l2_prefetch_kernel<<<2 * kSMs, 128, 0, ss>>>((const char *)p->W_UV, (long)H * dc * dv * 2, (const char *)p->W_O,
-                                                     (long)kr * row_bytes, rows > 0 ? ns : 0, rows * row_bytes);
-        NM_LAUNCH_CHECK("L2 prefetch launch");
     }
 
     // ---- attention over the old rows (tensor cores), main stream; the new row joins in the merge -----------
-    NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms, pdl));
+    NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms, pdl, pf));
     // The merge needs the cache row the KV chain wrote.  Joining here also keeps the merge from being
     // launched early: its CTAs could not share an SM with the attention CTAs (registers) and would
     // only hold up the prefetch kernel in the block scheduler.
@@ -555,7 +543,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         // merge of the attention partials (+ the new row) and o[h] = o_lat[h] * W_UV[h] in one kernel
         const AttnPlan ap = plan_attention(q_full, cache, H, (int)pos, dc);
         NM_TRY(launch_uv_merge(q_full, cache, carve_partials(aws, H), ap.npartial, pos, dr, p->softmax_scale, p->W_UV, o_lat,
-                               p->o_lat_f32, o, H, ms, pdl && !forked));
+                               p->o_lat_f32, o, H, ms, pdl && !forked && g_uv_pdl));
     } else {
         NM_TRY(attention_combine(q_full, cache, o_lat, p->o_lat_f32, H, (int)pos, pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms,
                                  pdl && !forked));
@@ -567,18 +555,6 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         NM_TRY(matmul_enqueue(o, p->W_O, p->out, 1, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms,
                               pdl && !p->event_before_wo));
         if (p->event_after_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_after_wo, ms));
-    }
-    // Under stream capture every stream that was forked must be joined again before the capture ends:
-    // the prefetch kernel on the side stream is otherwise left dangling.  Outside a capture the join is
-    // left out (the next step's fork orders the streams anyway, and a wait here would keep the next
-    // step's first product from starting early).
-    if (forked) {
-        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-        NM_CUDA_TRY(cudaStreamIsCapturing(ms, &cap));
-        if (cap == cudaStreamCaptureStatusActive) {
-            NM_CUDA_TRY(cudaEventRecord(g_events.q_ready, ss));
-            NM_CUDA_TRY(cudaStreamWaitEvent(ms, g_events.q_ready, 0));
-        }
     }
 #undef NM_LAUNCH
     return NM_OK;
@@ -669,6 +645,12 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     NM_CUDA_TRY(cudaMemcpyAsync(h_staging, h_host, (size_t)p->d * 2, cudaMemcpyHostToDevice, ms));
     NM_TRY(step_impl(&q, ms, (cudaStream_t)side_stream));
     NM_CUDA_TRY(cudaMemcpyAsync(out_host, out_staging, (size_t)p->d * 2, cudaMemcpyDeviceToHost, ms));
+    return NM_OK;
+}
+
+int nm_debug_set_step_knobs(int uv_pdl, int prefetch_uv)
+{
+    g_uv_pdl = uv_pdl; g_prefetch_uv = prefetch_uv;
     return NM_OK;
 }
 

@@ -27,11 +27,25 @@ AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int
 
 // Tensor-core (tcgen05 / TMEM) pass over the rows of each split.  Returns NM_ERR_UNSUPPORTED when
 // the shape is not one it takes (the caller then uses the CUDA-core kernel).
+// Weight bytes the attention kernel's idle lanes pull into L2 while the tensor cores work: one
+// contiguous block plus `nranges` ranges of `range_bytes`, `range_stride` apart (all may be empty).
+struct L2Prefetch {
+    const char *block;
+    long block_bytes;
+    const char *base;
+    long range_stride;
+    int nranges;
+    long range_bytes;
+};
+
 int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows,
-                         float scale, cudaStream_t stream, bool programmatic_launch);
+                         float scale, cudaStream_t stream, bool programmatic_launch, L2Prefetch prefetch);
 
 // Fused per-head stages of the decode step (nm_head_kernels.cu); they take nope = 128, kv_lora = 512, v = 128.
 bool head_kernels_apply(int H, int nope, int rope, int dc, int dv);
+bool down_finish_applies(int q_lora, int dc, int rope);
+int launch_down_finish(const void *x, const void *gamma_q, const void *gamma_kv, const float *cos_sin, void *c_qn, void *cache_row,
+                       int q_lora, int dc, int rope, float eps, cudaStream_t s, bool pdl);
 int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl);
 int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
                     const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl);

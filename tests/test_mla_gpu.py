@@ -193,12 +193,14 @@ def test_attention_stage_default_path(nm, S, extra):
 
 # ---- the whole step ---------------------------------------------------------------------------------------
 
-def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None):
+def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None, concat_down=False):
     H, dc, dr, dn, dv, d, ql = (DIMS[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d", "q_lora"))
     dkv, dq = dc + dr, dn + dr
     t = dict(dw)
     if not with_wo:
         t.pop("W_O")
+    if concat_down:      # (W_DQ | W_DKV | W_KR) stored as one matrix; the separate ones are not passed
+        t["W_DQKV"] = torch.cat([t.pop("W_DQ").view(d, ql), t.pop("W_DKVKR").view(d, dkv)], dim=1).contiguous().view(-1)
     t["h"] = to_dev(h)
     t["kv_cache"] = to_dev(cache_in)
     t["rope_cos_sin"] = rope_row(nm, S - 1)
@@ -250,6 +252,16 @@ def test_decode_step_s1024(nm, weights, ref1024, overlap):
     cache_in = gen.mla_cache(1024, DIMS, seed=4200)
     t = run_step(nm, dw, h, cache_in, 1024, overlap=overlap)
     check_step(t, r, cache_ref, 1024)
+
+
+@pytest.mark.parametrize("S", [1, 70, 1024])
+def test_decode_step_with_concatenated_down_projections(nm, weights, S):
+    # h * (W_DQ | W_DKV | W_KR) as one product on one stream (Eq. 3's concatenation extended by W_DQ)
+    w, dw = weights
+    h, cache_ref, r = oracle_step(w, S, seed=4500 + S)
+    cache_in = gen.mla_cache(S, DIMS, seed=4500 + S)
+    t = run_step(nm, dw, h, cache_in, S, concat_down=True)
+    check_step(t, r, cache_ref, S)
 
 
 @pytest.mark.parametrize("S", [1, 2, 65, 4096])

@@ -23,7 +23,7 @@
 // cluster size.
 //
 // Roles: warp 0 lane 0 issues TMA, warp 1 owns TMEM and its lane 0 issues the MMAs, warps 2-5 hold
-// one head per thread.  Every wait is bounded (mbar_wait); on expiry the CTA raises the status word,
+// one head per thread, warp 6 prefetches the weights of the products that follow into L2.  Every wait is bounded (mbar_wait); on expiry the CTA raises the status word,
 // skips the remaining waits, frees its TMEM and returns.
 #include "nm_async.cuh"
 #include "nm_mla.cuh"
@@ -45,10 +45,14 @@ constexpr int kKVBlockBytes = kT * 128;      // 8 KB
 constexpr int kQBytes = kKBlocks * kQBlockBytes;     // 147456
 constexpr int kKVBytes = kKBlocks * kKVBlockBytes;   // 36864 per stage
 constexpr int kSmemBytes = kQBytes + kKVStages * kKVBytes + 1024 /* alignment slack */ + 256 /* barriers */;
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;               // TMA, MMA, 4 softmax warps, weight prefetch
 constexpr uint32_t kTmemCols = 512;
-// TMEM columns: O (fp32, 256), then per pipeline stage S (fp32, 32), P_hi and P_lo (bf16 pairs, 16 each)
-constexpr uint32_t kColO = 0, kColS = 256, kColP = 320, kColPlo = 352;      // stage b adds 32*b to S, 16*b to P_hi / P_lo
+// TMEM columns: O (fp32, 256), then per pipeline stage kSAcc score accumulators (fp32, 32 columns each; the 36
+// k-steps of a tile's scores are dealt round-robin to them, because back-to-back MMAs into one narrow
+// accumulator wait for each other, and the softmax threads add them up), then P_hi and P_lo (bf16 pairs, 16 each)
+constexpr int kSAcc = 3;
+constexpr uint32_t kColO = 0, kColS = 256, kColP = kColS + 2 * 32 * kSAcc, kColPlo = kColP + 32;   // stage b adds 32*kSAcc*b to S, 16*b to P_hi / P_lo
+static_assert(kColPlo + 32 <= 512, "TMEM columns");
 constexpr float kLazyThreshold = 8.0f;    // log2 units
 constexpr int kCl = kAttnCluster;          // CTAs (splits) per cluster
 constexpr int kHeadsPerRank = kHeads / kCl;
@@ -98,7 +102,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return r;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)    // register cap 144: leaves room for a CTA of the merge kernel that follows
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, AttnPartials part,
                int n_rows, int rows_per_split, float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
 {
@@ -144,17 +148,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int cluster_id = sp / kCl;
     float m_own = -INFINITY, l_own = 0.f;                         // softmax threads: this split's (m, l)
 
-    // The softmax threads, once the scores of their first tile are in (so that the tile loads, which the
-    // whole pass waits for, do not queue behind it), pull the weights of the products that follow the
-    // attention - W_UV and the head of every k-split of W_O - into L2 in 4 KB bulk prefetches: the pass
-    // needs little HBM bandwidth, and those weights do not depend on its result.
+    // A warp of its own, once the first cache tile has landed (so that the loads the whole pass waits for
+    // do not queue behind it), pulls the weights of the products that follow the attention - W_UV and the
+    // head of every k-split of W_O - into L2 in 8 KB bulk prefetches: the pass needs little HBM bandwidth,
+    // and those weights do not depend on its result.  The prefetch instruction stalls its thread while the
+    // request queue is full (microseconds here), which is why no thread of the pipeline issues it.
     auto prefetch_weights = [&]() {
-        constexpr long kChunk = 4096;
+        constexpr long kChunk = 8192;
         const long block_chunks = (pf.block_bytes + kChunk - 1) / kChunk;
         const long chunks_per_range = (pf.range_bytes + kChunk - 1) / kChunk;
         const long total = block_chunks + chunks_per_range * pf.nranges;
-        const long nthreads = (long)gridDim.x * gridDim.y * 128;
-        const long me = ((long)blockIdx.y * gridDim.x + blockIdx.x) * 128 + (tid - 64);
+        const long nthreads = (long)gridDim.x * gridDim.y * 32;
+        const long me = ((long)blockIdx.y * gridDim.x + blockIdx.x) * 32 + lane;
         for (long i = me; i < total; i += nthreads) {
             const char *ptr;
             long n;
@@ -207,14 +212,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // ---------------- MMA issuer ---------------------------------------------------------------
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(128, kT, false, false), idesc_o = instr_desc(128, kDvHalf, false, true);
+            // The descriptors of a tile's 36 k-steps differ only in the start-address field (16-byte units, no
+            // carry out of it for addresses below 256 KB): one base each, compile-time offsets added per step.
+            const uint64_t q_desc0 = smem_desc(q_addr, 16, 1024), kv_desc0 = smem_desc(kv_addr, 16, 1024);
             auto scores = [&](int t) {                             // S[t&1] = Q * tile(t)^T  (tile t has landed)
                 const int b = t & 1;
+                const uint64_t kv_desc = kv_desc0 + (uint64_t)((b * kKVBytes) >> 4);
+                const uint32_t s_col = tmem + kColS + 32 * kSAcc * b;
                 tc_fence_after();
-                for (int c = 0; c < kKBlocks; ++c)
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        mma_ss(tmem + kColS + 32 * b, smem_desc(q_addr + c * kQBlockBytes + kk * 32, 16, 1024),
-                               smem_desc(kv_addr + b * kKVBytes + c * kKVBlockBytes + kk * 32, 16, 1024), idesc_s, (c | kk) != 0);
+                for (int step = 0; step < kKBlocks * 4; ++step) {
+                    const int c = step >> 2, kk = step & 3;
+                    mma_ss(s_col + 32 * (step % kSAcc), q_desc0 + (uint64_t)((c * kQBlockBytes + kk * 32) >> 4),
+                           kv_desc + (uint64_t)((c * kKVBlockBytes + kk * 32) >> 4), idesc_s, step >= kSAcc);
+                }
                 mma_commit(bar_s_full + 8 * b);
             };
             auto pv = [&](int t) {                                 // O += P[t&1] * tile(t)[:, half]  (P of tile t is written)
@@ -239,8 +250,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             while (tp < ntiles) {
                 bool progress = false;
                 if (ts < ntiles && ts <= tp + 1 && mbar_try_wait(bar_kv_full + 8 * (ts & 1), (ts >> 1) & 1)) {
+                    if (ts == 0) NM_TRACE(12);
                     scores(ts);
                     if (ts == 0) NM_TRACE(3);
+                    if (ts == 1) NM_TRACE(13);
                     ++ts;
                     progress = true;
                 }
@@ -263,21 +276,43 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
             }
         }
+    } else if (warp == 6) {
+        // ---------------- weight prefetch ----------------------------------------------------------------
+        if (ntiles > 0) {                                          // sleep-poll: this warp must not take issue slots from the pipeline
+            const uint64_t t0 = global_timer_ns();
+            while (!mbar_try_wait(bar_kv_full, 0)) {
+                __nanosleep(128);
+                if (s_abort || global_timer_ns() - t0 > kWaitLimitNs) break;
+            }
+        }
+        prefetch_weights();
     } else {
         // ---------------- one head per thread: softmax, lazy rescale ------------------------------------------
         const int quad = warp & 3;                                 // TMEM lanes this warp may touch
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
         float m_used = -INFINITY, l = 0.f;
-        if (ntiles == 0) prefetch_weights();
         for (int t = 0; t < ntiles; ++t) {
             const int b = t & 1;
             mbar_wait(bar_s_full + 8 * b, (t >> 1) & 1, &s_abort, status);
             tc_fence_after();
             if (t == 0 && tid == 64) NM_TRACE(4);
-            if (t == 0) prefetch_weights();
+            if (t == 1 && tid == 64) NM_TRACE(14);
             uint32_t sr[32];
-            tmem_ld32(lane_base + kColS + 32 * b, sr);
-            tmem_wait_ld();
+            tmem_ld32(lane_base + kColS + 32 * kSAcc * b, sr);
+            if (kSAcc > 1) {
+                uint32_t s1[32], s2[32];
+                tmem_ld32(lane_base + kColS + 32 * kSAcc * b + 32, s1);
+                if (kSAcc > 2) tmem_ld32(lane_base + kColS + 32 * kSAcc * b + 64, s2);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < kT; ++j) {
+                    float v = __uint_as_float(sr[j]) + __uint_as_float(s1[j]);
+                    if (kSAcc > 2) v += __uint_as_float(s2[j]);
+                    sr[j] = __float_as_uint(v);
+                }
+            } else {
+                tmem_wait_ld();
+            }
             const int valid = min(kT, r1 - (r0 + t * kT));
             float mx = -INFINITY;
 #pragma unroll
@@ -325,6 +360,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             tc_fence_before();
             mbar_arrive(bar_p_full + 8 * b);
             if (t == 0 && tid == 64) NM_TRACE(5);
+            if (t == 1 && tid == 64) NM_TRACE(15);
         }
         // the last P*V must have landed before O is read
         if (ntiles > 0) {
@@ -342,7 +378,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // After one cluster barrier, rank r combines heads [32r, 32r+32) over all peers - weights
     // 2^(m_peer - max m) - reading the peers' rows with many loads in flight, and writes one partial
     // per cluster.  A last barrier keeps every CTA's shared memory alive until its peers have read it.
-    if (warp >= 2) {
+    if (warp >= 2 && warp < 6) {
         const int quad = warp & 3, head = quad * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
         s_ml[head][0] = (ntiles > 0) ? m_own : -INFINITY;
@@ -364,7 +400,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     cluster_sync_all();                                            // every peer's rows and (m, l) are parked
     if (tid == 64) NM_TRACE(8);
-    if (warp >= 2) {
+    if (warp >= 2 && warp < 6) {
         const int t = tid - 64;                                    // 0..127
         if (t < kCl * kHeadsPerRank) {                             // weight of peer r for owned head hl
             const int hl = t % kHeadsPerRank, r = t / kHeadsPerRank, head = (int)rank * kHeadsPerRank + hl;
@@ -386,7 +422,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         named_barrier_sync(1, 128);
         if (tid == 64) NM_TRACE(9);
-        constexpr int kIters = kHeadsPerRank * 64 / 128, kBatch = 8;
+        constexpr int kIters = kHeadsPerRank * 64 / 128, kBatch = 4;
         for (int i0 = 0; i0 < kIters; i0 += kBatch) {
             float4 v[kBatch][kCl];
 #pragma unroll

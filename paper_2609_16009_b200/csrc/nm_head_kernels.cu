@@ -125,21 +125,31 @@ __global__ void __launch_bounds__(kHeadThreads) q_finish_kernel(const uint16_t *
 
 // Merge of the attention partials (see attn_combine_kernel for the algebra) followed by W_UV.
 // dc = 512, dv = 128.
-__global__ void __launch_bounds__(kHeadThreads) uv_merge_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
-                                                                AttnPartials part, int npart, long extra_row, int rope, float scale,
-                                                                const uint16_t *__restrict__ W_UV, uint16_t *__restrict__ o_lat_bf16,
-                                                                float *__restrict__ o_lat_f32, uint16_t *__restrict__ o)
+//
+// Sized to share an SM with a CTA of the attention kernel that precedes it (which holds nearly all of the
+// shared memory and about half of the registers): under 8 KB of shared memory, at most 128 registers per
+// thread.  Launched programmatically, it is therefore resident - with the first half of the head's 128 KB
+// of weights already in registers - when the attention result arrives; the second half (an L2 hit after the
+// prefetch issued by the attention kernel) is fetched while the partials are merged.
+constexpr int kUvPre = 16;                                         // weight vectors per thread loaded before the inputs exist
+constexpr int kUvMaxParts = 64;                                    // partials per head the merge takes (the planner never makes more)
+__global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
+                                                                   AttnPartials part, int npart, long extra_row, int rope, float scale,
+                                                                   const uint16_t *__restrict__ W_UV, uint16_t *__restrict__ o_lat_bf16,
+                                                                   float *__restrict__ o_lat_f32, uint16_t *__restrict__ o)
 {
     constexpr int K = 512, N = 128;
-    using MV = HeadMatvec<K, N>;
+    constexpr int kColGroups = N / 8, kRowGroups = kHeadThreads / kColGroups;        // 16 x 16; 32 rows per thread
     __shared__ __align__(16) float x_s[K];
-    __shared__ __align__(16) float red[MV::kRowGroups * N];
+    __shared__ __align__(16) float red[(kRowGroups / 2) * N];      // row groups 2j and 2j+1 sit in one warp: added by shuffle
     __shared__ float scratch[32];
-    __shared__ float sm[kMaxAttnSplits], sl[kMaxAttnSplits], sw[kMaxAttnSplits];
+    __shared__ float sm[kUvMaxParts], sl[kUvMaxParts], sw[kUvMaxParts];
     const int h = blockIdx.x, H = gridDim.x, dkv = K + rope, tid = threadIdx.x;
-    const uint16_t *W = W_UV + (size_t)h * K * N;
-    uint4 w[32];
-    MV::load(W, w, 0, 32);                                        // all of the head's weights before the inputs exist
+    const int tx = tid % kColGroups, ty = tid / kColGroups;
+    const uint16_t *W = W_UV + (size_t)h * K * N + (size_t)ty * N + tx * 8;          // row ty + i*kRowGroups for i = 0..31
+    uint4 w[kUvPre];
+#pragma unroll
+    for (int i = 0; i < kUvPre; ++i) w[i] = ld_stream16(W + (size_t)i * kRowGroups * N);
     pdl_launch_dependents();
     pdl_wait_prior_grids();                                       // partials come from the attention kernel
     for (int s = tid; s < npart; s += kHeadThreads) {
@@ -199,9 +209,52 @@ __global__ void __launch_bounds__(kHeadThreads) uv_merge_kernel(const uint16_t *
     x_s[c] = bf16_to_f32(b0);                                      // W_UV sees the rounded o_lat, as the stage-wise definition says
     x_s[c + 1] = bf16_to_f32(b1);
     __syncthreads();
-    float out8[8];
-    MV::run(w, x_s, red, out8);
-    if (tid / MV::kColGroups == 0) *reinterpret_cast<uint4 *>(o + (size_t)h * N + (tid % MV::kColGroups) * 8) = pack8_bf16(out8);
+
+    // ---- o[h] = o_lat[h] * W_UV[h]: rows ty + i*16; the second half of the weights replaces the first in
+    //      the same registers, eight vectors at a time, while the first half is being used
+    float a8[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) a8[j] = 0.f;
+    auto use = [&](const uint4 &wv, int i) {
+        float b[8];
+        Elem<bf16_t>::unpack(wv, b);
+        const float a = x_s[ty + i * kRowGroups];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) a8[j] = fmaf(a, b[j], a8[j]);
+    };
+    uint4 w2[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w2[i] = ld_stream16(W + (size_t)(kUvPre + i) * kRowGroups * N);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) use(w[i], i);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = ld_stream16(W + (size_t)(kUvPre + 8 + i) * kRowGroups * N);
+#pragma unroll
+    for (int i = 8; i < 16; ++i) use(w[i], i);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) use(w2[i], kUvPre + i);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) use(w[i], kUvPre + 8 + i);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) a8[j] += __shfl_xor_sync(0xffffffffu, a8[j], 16);     // row groups 2j + 2j+1
+    if ((tid & 16) == 0) {
+        float4 *dst = reinterpret_cast<float4 *>(red + (size_t)(ty >> 1) * N + tx * 8);
+        dst[0] = make_float4(a8[0], a8[1], a8[2], a8[3]);
+        dst[1] = make_float4(a8[4], a8[5], a8[6], a8[7]);
+    }
+    __syncthreads();
+    if (ty == 0) {
+        float out8[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) out8[j] = 0.f;
+        for (int g = 0; g < kRowGroups / 2; ++g) {                 // fixed order: deterministic
+            const float4 *src4 = reinterpret_cast<const float4 *>(red + (size_t)g * N + tx * 8);
+            const float4 v0 = src4[0], v1 = src4[1];
+            out8[0] += v0.x; out8[1] += v0.y; out8[2] += v0.z; out8[3] += v0.w;
+            out8[4] += v1.x; out8[5] += v1.y; out8[6] += v1.z; out8[7] += v1.w;
+        }
+        *reinterpret_cast<uint4 *>(o + (size_t)h * N + tx * 8) = pack8_bf16(out8);
+    }
 }
 
 // The vector stages behind the fused down-projection h * (W_DQ | W_DKV | W_KR): CTA 0 normalises the
@@ -304,6 +357,7 @@ int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void 
 int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
                     const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl)
 {
+    if (npart < 0 || npart > kUvMaxParts) return NM_ERR_UNSUPPORTED;
     cudaError_t e = launch_with_pdl(uv_merge_kernel, H, s, pdl, (const uint16_t *)Q, (const uint16_t *)cache, part, npart, extra_row, rope,
                                     scale, (const uint16_t *)W_UV, (uint16_t *)o_lat_bf16, o_lat_f32, (uint16_t *)o);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "uv_merge launch");

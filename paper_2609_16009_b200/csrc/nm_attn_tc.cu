@@ -102,12 +102,15 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return r;
 }
 
-__global__ void __launch_bounds__(kThreads, 2)    // register cap 144: leaves room for a CTA of the merge kernel that follows
+// at most 120 registers per thread: leaves room on the SM for a CTA of the merge kernel that follows
+__global__ void __maxnreg__(120)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, AttnPartials part,
                int n_rows, int rows_per_split, float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
 {
     // Optional phase timestamps (ns) of CTA (0,0), for tuning: trace[i] is written when non-null.
 #define NM_TRACE(i) do { if (trace && blockIdx.x == 0 && blockIdx.y == 0) trace[i] = global_timer_ns(); } while (0)
+    // ... and four stamps of every CTA (start, Q landed, last P*V done, end) from trace[32] on
+#define NM_TRACE_CTA(i) do { if (trace) trace[32 + 4 * (blockIdx.y * gridDim.x + blockIdx.x) + (i)] = global_timer_ns(); } while (0)
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;            // swizzle atoms want 1024-byte alignment
@@ -130,6 +133,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     if (tid == 0) {
         NM_TRACE(0);
+        NM_TRACE_CTA(0);
         s_abort = 0;
         mbar_init(bar_q, 1);
         for (int b = 0; b < kKVStages; ++b) {
@@ -242,6 +246,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             NM_TRACE(1);
             if (ntiles > 0) mbar_wait(bar_q, 0, &s_abort, status);
             NM_TRACE(2);
+            NM_TRACE_CTA(1);
             // Two independent streams of work share this thread: scores of tile ts (needs the tile in
             // shared memory and S[ts&1] free, i.e. the P*V of tile ts-2 issued) and P*V of tile tp (needs
             // the softmax of tile tp).  Whichever is ready is issued; neither blocks the other.
@@ -368,6 +373,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             tc_fence_after();
         }
         if (tid == 64) NM_TRACE(6);
+        if (tid == 64) NM_TRACE_CTA(2);
         m_own = m_used; l_own = l;
     }
 
@@ -464,7 +470,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
     if (tid == 0) NM_TRACE(11);
+    if (tid == 0) NM_TRACE_CTA(3);
 #undef NM_TRACE
+#undef NM_TRACE_CTA
 }
 
 // Tensor maps: bf16 [rows][576], boxes of 64 columns (128 bytes, the swizzle span) x box_rows rows.
@@ -485,6 +493,7 @@ bool encode_rows_map(CUtensorMap *map, const void *ptr, int rows, int box_rows)
 
 static unsigned long long *g_attn_trace = nullptr;
 void set_attention_trace(unsigned long long *p) { g_attn_trace = p; }
+unsigned long long *attention_trace() { return g_attn_trace; }
 
 int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows, float scale,
                          cudaStream_t stream, bool programmatic_launch, L2Prefetch prefetch)
@@ -504,7 +513,9 @@ int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, At
     const float scale_log2 = scale * 1.4426950408889634f;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ceil_div(plan.nsplit, kCl) * kCl, 2);      // padded to whole clusters; padding CTAs have no rows
-    cfg.blockDim = dim3(kThreads);
+    // the prefetch warp is launched only when there is something to prefetch (fewer registers held on the SM)
+    const bool has_prefetch = prefetch.block_bytes > 0 || (prefetch.nranges > 0 && prefetch.range_bytes > 0);
+    cfg.blockDim = dim3(has_prefetch ? kThreads : kThreads - 32);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];

@@ -127,17 +127,20 @@ __global__ void __launch_bounds__(kHeadThreads) q_finish_kernel(const uint16_t *
 // dc = 512, dv = 128.
 //
 // Sized to share an SM with a CTA of the attention kernel that precedes it (which holds nearly all of the
-// shared memory and about half of the registers): under 8 KB of shared memory, at most 128 registers per
-// thread.  Launched programmatically, it is therefore resident - with the first half of the head's 128 KB
-// of weights already in registers - when the attention result arrives; the second half (an L2 hit after the
-// prefetch issued by the attention kernel) is fetched while the partials are merged.
+// shared memory and under half of the registers; the register file is split over the four schedulers, two
+// warps of each kernel per scheduler, so the two kernels' registers per thread must add up to 256 or less): under 8 KB of shared memory, at most 128 registers per
+// thread.  Launched programmatically, it is therefore resident - with half of the head's 128 KB
+// of weights already in registers - when the attention result arrives; the rest (an L2 hit after its own
+// prefetch) is fetched once the partial rows have left their registers.
 constexpr int kUvPre = 16;                                         // weight vectors per thread loaded before the inputs exist
 constexpr int kUvMaxParts = 64;                                    // partials per head the merge takes (the planner never makes more)
 __global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
                                                                    AttnPartials part, int npart, long extra_row, int rope, float scale,
                                                                    const uint16_t *__restrict__ W_UV, uint16_t *__restrict__ o_lat_bf16,
-                                                                   float *__restrict__ o_lat_f32, uint16_t *__restrict__ o)
+                                                                   float *__restrict__ o_lat_f32, uint16_t *__restrict__ o, const L2Prefetch pf,
+                                                                   unsigned long long *trace)
 {
+#define UV_TRACE(i) do { if (trace && tid == 0 && (blockIdx.x == 0 || blockIdx.x == 77)) trace[1100 + (blockIdx.x ? 16 : 0) + (i)] = global_timer_ns(); } while (0)
     constexpr int K = 512, N = 128;
     constexpr int kColGroups = N / 8, kRowGroups = kHeadThreads / kColGroups;        // 16 x 16; 32 rows per thread
     __shared__ __align__(16) float x_s[K];
@@ -147,42 +150,88 @@ __global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_
     const int h = blockIdx.x, H = gridDim.x, dkv = K + rope, tid = threadIdx.x;
     const int tx = tid % kColGroups, ty = tid / kColGroups;
     const uint16_t *W = W_UV + (size_t)h * K * N + (size_t)ty * N + tx * 8;          // row ty + i*kRowGroups for i = 0..31
+    UV_TRACE(0);
     uint4 w[kUvPre];
 #pragma unroll
     for (int i = 0; i < kUvPre; ++i) w[i] = ld_stream16(W + (size_t)i * kRowGroups * N);
     pdl_launch_dependents();
-    pdl_wait_prior_grids();                                       // partials come from the attention kernel
-    for (int s = tid; s < npart; s += kHeadThreads) {
-        const float2 v = __ldcg(reinterpret_cast<const float2 *>(part.ml + ((size_t)s * H + h) * 2));
-        sm[s] = v.x; sl[s] = v.y;
+    // While the attention kernel (which needs little HBM bandwidth) runs, this grid is resident and idle:
+    // it pulls into L2 the rest of its own weights and the ranges of the next product's weights it was
+    // given (the head of every k-split of W_O) - they do not depend on the attention result.  The request
+    // stalls its thread while the queue is full; nothing here is waiting for these threads yet.
+    if (pf.nranges >= 0) {
+        constexpr long kChunk = 4096;
+        if (tid < (K - kUvPre * kRowGroups) * N * 2 / kChunk)       // rows kUvPre*16.. of this head: contiguous
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"((const char *)(W_UV + (size_t)h * K * N + (size_t)kUvPre * kRowGroups * N) + tid * kChunk),
+                         "r"((uint32_t)kChunk) : "memory");
+        const long chunks_per_range = (pf.range_bytes + kChunk - 1) / kChunk, total = chunks_per_range * pf.nranges;
+        for (long i = (long)h * kHeadThreads + tid; i < total; i += (long)H * kHeadThreads) {
+            const long r = i / chunks_per_range, off = (i - r * chunks_per_range) * kChunk;
+            const long n = min(kChunk, pf.range_bytes - off) & ~15L;
+            if (n > 0) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(pf.base + r * pf.range_stride + off), "r"((uint32_t)n) : "memory");
+        }
     }
-    // two columns per thread; the partial rows of up to 8 parts in flight
+    UV_TRACE(1);
+    pdl_wait_prior_grids();                                       // partials come from the attention kernel
+    UV_TRACE(2);
+    // Everything the merge needs is asked for at once, so that one L2 round trip covers it: the partial rows
+    // of up to 16 parts (two columns per thread), the (m, l) pairs, and the operands of the new row's score.
     const int c = 2 * tid;
     const float *src = part.O + (size_t)h * K + c;
-    constexpr int kBatch = 8;
+    constexpr int kBatch = 16;
     float2 v[kBatch];
 #pragma unroll
     for (int u = 0; u < kBatch; ++u)
         v[u] = (u < npart) ? __ldcg(reinterpret_cast<const float2 *>(src + (size_t)u * H * K)) : make_float2(0.f, 0.f);
+    for (int s = tid; s < npart; s += kHeadThreads) {
+        const float2 ml = __ldcg(reinterpret_cast<const float2 *>(part.ml + ((size_t)s * H + h) * 2));
+        sm[s] = ml.x; sl[s] = ml.y;
+    }
     float sx = -INFINITY;
     if (extra_row >= 0) {
-        const uint16_t *qh = Q + (size_t)h * dkv, *row = cache + (size_t)extra_row * dkv;
-        float acc = 0.f;
-        for (int i = tid; i < dkv; i += kHeadThreads) acc = fmaf(bf16_to_f32(qh[i]), bf16_to_f32(row[i]), acc);
-        sx = block_sum_256(acc, scratch) * scale;
+        float dot = 0.f;
+        if (tid < dkv / 8) {                                       // dkv = 576: 72 threads, eight elements each
+            float qf[8], rf[8];
+            Elem<bf16_t>::unpack(__ldcg(reinterpret_cast<const uint4 *>(Q + (size_t)h * dkv) + tid), qf);
+            Elem<bf16_t>::unpack(__ldcg(reinterpret_cast<const uint4 *>(cache + (size_t)extra_row * dkv) + tid), rf);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) dot = fmaf(qf[e], rf[e], dot);
+        }
+        sx = block_sum_256(dot, scratch) * scale;
     } else {
         __syncthreads();
     }
-    float Mx = sx;
-    for (int s = 0; s < npart; ++s) Mx = fmaxf(Mx, sm[s]);
-    const float wx = (extra_row >= 0) ? __expf(sx - Mx) : 0.f;
-    float L = wx;
-    for (int s = 0; s < npart; ++s) {                              // same order in every thread
-        const float wgt = (sm[s] == -INFINITY) ? 0.f : __expf(sm[s] - Mx);
-        if (tid == 0) sw[s] = wgt;
-        L = fmaf(wgt, sl[s], L);
+    UV_TRACE(3);
+    // weights of the parts: exp(m_s - max), the new row's exp(sx - max), and the normaliser L.  Up to 32 parts
+    // (the tensor-core pass makes at most 16) are handled by one warp with shuffles in a fixed order.
+    if (npart <= 32) {
+        if (tid < 32) {
+            const float m = (tid < npart) ? sm[tid] : -INFINITY, l = (tid < npart) ? sl[tid] : 0.f;
+            float Mx = fmaxf(m, sx);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) Mx = fmaxf(Mx, __shfl_xor_sync(0xffffffffu, Mx, o));
+            const float wgt = (m == -INFINITY) ? 0.f : __expf(m - Mx);
+            float L = wgt * l;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+            const float wx = (extra_row >= 0) ? __expf(sx - Mx) : 0.f;
+            sw[tid] = wgt;
+            if (tid == 0) { scratch[16] = wx; scratch[17] = L + wx; }
+        }
+    } else if (tid == 0) {
+        float Mx = sx;
+        for (int s = 0; s < npart; ++s) Mx = fmaxf(Mx, sm[s]);
+        const float wx = (extra_row >= 0) ? __expf(sx - Mx) : 0.f;
+        float L = wx;
+        for (int s = 0; s < npart; ++s) {
+            const float wgt = (sm[s] == -INFINITY) ? 0.f : __expf(sm[s] - Mx);
+            sw[s] = wgt;
+            L = fmaf(wgt, sl[s], L);
+        }
+        scratch[16] = wx; scratch[17] = L;
     }
     __syncthreads();
+    const float wx = scratch[16], L = scratch[17];
     float2 acc = make_float2(0.f, 0.f);
     if (extra_row >= 0) {
         const uint32_t rv = *reinterpret_cast<const uint32_t *>(cache + (size_t)extra_row * dkv + c);
@@ -201,6 +250,11 @@ __global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_
             acc.y = fmaf(wgt, v[u].y, acc.y);
         }
     }
+    UV_TRACE(4);
+    // the second half of the weights (L2 hits) takes the registers the partial rows have left
+    uint4 w2[K / kRowGroups - kUvPre];
+#pragma unroll
+    for (int i = 0; i < K / kRowGroups - kUvPre; ++i) w2[i] = ld_stream16(W + (size_t)(kUvPre + i) * kRowGroups * N);
     const float inv = 1.0f / L;
     const float o0 = acc.x * inv, o1 = acc.y * inv;
     const uint16_t b0 = f32_to_bf16(o0), b1 = f32_to_bf16(o1);
@@ -210,8 +264,8 @@ __global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_
     x_s[c + 1] = bf16_to_f32(b1);
     __syncthreads();
 
-    // ---- o[h] = o_lat[h] * W_UV[h]: rows ty + i*16; the second half of the weights replaces the first in
-    //      the same registers, eight vectors at a time, while the first half is being used
+    UV_TRACE(5);
+    // ---- o[h] = o_lat[h] * W_UV[h]: rows ty + i*16 ------------------------------------------------------------
     float a8[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) a8[j] = 0.f;
@@ -222,19 +276,11 @@ __global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_
 #pragma unroll
         for (int j = 0; j < 8; ++j) a8[j] = fmaf(a, b[j], a8[j]);
     };
-    uint4 w2[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) w2[i] = ld_stream16(W + (size_t)(kUvPre + i) * kRowGroups * N);
+    for (int i = 0; i < kUvPre; ++i) use(w[i], i);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) use(w[i], i);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) w[i] = ld_stream16(W + (size_t)(kUvPre + 8 + i) * kRowGroups * N);
-#pragma unroll
-    for (int i = 8; i < 16; ++i) use(w[i], i);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) use(w2[i], kUvPre + i);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) use(w[i], kUvPre + 8 + i);
+    for (int i = 0; i < K / kRowGroups - kUvPre; ++i) use(w2[i], kUvPre + i);
+    UV_TRACE(6);
 #pragma unroll
     for (int j = 0; j < 8; ++j) a8[j] += __shfl_xor_sync(0xffffffffu, a8[j], 16);     // row groups 2j + 2j+1
     if ((tid & 16) == 0) {
@@ -255,6 +301,8 @@ __global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_
         }
         *reinterpret_cast<uint4 *>(o + (size_t)h * N + tx * 8) = pack8_bf16(out8);
     }
+    UV_TRACE(7);
+#undef UV_TRACE
 }
 
 // The vector stages behind the fused down-projection h * (W_DQ | W_DKV | W_KR): CTA 0 normalises the
@@ -355,11 +403,12 @@ int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void 
 }
 
 int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
-                    const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl)
+                    const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl, L2Prefetch prefetch)
 {
     if (npart < 0 || npart > kUvMaxParts) return NM_ERR_UNSUPPORTED;
+    if (!prefetch.base && !prefetch.block) prefetch.nranges = -1;  // no prefetch at all
     cudaError_t e = launch_with_pdl(uv_merge_kernel, H, s, pdl, (const uint16_t *)Q, (const uint16_t *)cache, part, npart, extra_row, rope,
-                                    scale, (const uint16_t *)W_UV, (uint16_t *)o_lat_bf16, o_lat_f32, (uint16_t *)o);
+                                    scale, (const uint16_t *)W_UV, (uint16_t *)o_lat_bf16, o_lat_f32, (uint16_t *)o, prefetch, attention_trace());
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "uv_merge launch");
 }
 

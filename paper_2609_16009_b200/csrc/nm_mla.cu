@@ -534,7 +534,11 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     }
 
     // ---- attention over the old rows (tensor cores), main stream; the new row joins in the merge -----------
-    NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms, pdl, pf));
+    // When the merge kernel is launched programmatically it sits beside the attention CTAs from their start and
+    // issues the prefetch itself (its threads are idle until the attention result exists); otherwise a warp of
+    // the attention kernel does.
+    const bool uv_early = fused && pdl && !forked && g_uv_pdl;
+    NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms, pdl, uv_early ? L2Prefetch{} : pf));
     // The merge needs the cache row the KV chain wrote.  Joining here also keeps the merge from being
     // launched early: its CTAs could not share an SM with the attention CTAs (registers) and would
     // only hold up the prefetch kernel in the block scheduler.
@@ -543,7 +547,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         // merge of the attention partials (+ the new row) and o[h] = o_lat[h] * W_UV[h] in one kernel
         const AttnPlan ap = plan_attention(q_full, cache, H, (int)pos, dc);
         NM_TRY(launch_uv_merge(q_full, cache, carve_partials(aws, H), ap.npartial, pos, dr, p->softmax_scale, p->W_UV, o_lat,
-                               p->o_lat_f32, o, H, ms, pdl && !forked && g_uv_pdl));
+                               p->o_lat_f32, o, H, ms, uv_early, uv_early ? pf : L2Prefetch{}));
     } else {
         NM_TRY(attention_combine(q_full, cache, o_lat, p->o_lat_f32, H, (int)pos, pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms,
                                  pdl && !forked));

@@ -48,9 +48,12 @@ int launch_down_finish(const void *x, const void *gamma_q, const void *gamma_kv,
                        int q_lora, int dc, int rope, float eps, cudaStream_t s, bool pdl);
 int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl);
 int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
-                    const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl);
+                    const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl,
+                    L2Prefetch prefetch = L2Prefetch{});
 
-// Tuning aid: 12 phase timestamps (ns) of CTA (0,0) of the tensor-core kernel go to `p` when non-null.
+// Tuning aid: phase timestamps (ns) of the tensor-core kernel go to `p` when non-null: 32 slots for CTA (0,0),
+// then four per CTA (start, Q landed, last P*V done, end); 32 + 4 * 256 values at most.
 void set_attention_trace(unsigned long long *p);
+unsigned long long *attention_trace();
 
 }  // namespace nm

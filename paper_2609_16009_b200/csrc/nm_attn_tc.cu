@@ -88,13 +88,6 @@ __device__ __forceinline__ float4 ld_peer_f4(uint32_t addr)
     asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
     return v;
 }
-__device__ __forceinline__ float2 ld_peer_f2(uint32_t addr)
-{
-    float2 v;
-    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
-    return v;
-}
-
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     uint32_t r;
@@ -123,7 +116,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                    bar_p_full = smem_u32(bars + 5), bar_pv_done = smem_u32(bars + 7);
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ __align__(8) float s_ml[kHeads][2];                // this split's (m in log2 units, l) per head
+    __shared__ __align__(8) float s_mlp[kCl][kHeadsPerRank][2];   // (m in log2 units, l) of the owned heads, written by each peer
     __shared__ float s_w[kCl][kHeadsPerRank];                     // weights of the slots in the final sum
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -147,6 +140,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
+    // First half of a cluster barrier: by the time its second half is waited for (before the merge) every
+    // peer has started, which is what writing into a peer's shared memory requires.
+    __syncwarp();
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     pdl_launch_dependents();
     const uint32_t rank = cluster_rank();
     const int cluster_id = sp / kCl;
@@ -232,6 +229,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
                 mma_commit(bar_s_full + 8 * b);
             };
+            // Scores of tiles 0 and 1 together (both landed, both S buffers free): each k-step's slice of Q is
+            // read from shared memory once and used for both tiles - the Q operand is what these MMAs cost.
+            auto scores_pair = [&]() {
+                tc_fence_after();
+#pragma unroll
+                for (int step = 0; step < kKBlocks * 4; ++step) {
+                    const int c = step >> 2, kk = step & 3;
+                    const uint64_t qd = q_desc0 + (uint64_t)((c * kQBlockBytes + kk * 32) >> 4);
+                    const uint64_t kd = kv_desc0 + (uint64_t)((c * kKVBlockBytes + kk * 32) >> 4);
+                    mma_ss_a_fill(tmem + kColS + 32 * (step % kSAcc), qd, kd, idesc_s, step >= kSAcc);
+                    mma_ss_a_lastuse(tmem + kColS + 32 * kSAcc + 32 * (step % kSAcc), qd, kd + (uint64_t)(kKVBytes >> 4), idesc_s, step >= kSAcc);
+                }
+                mma_commit(bar_s_full);
+                mma_commit(bar_s_full + 8);
+            };
             auto pv = [&](int t) {                                 // O += P[t&1] * tile(t)[:, half]  (P of tile t is written)
                 const int b = t & 1;
                 tc_fence_after();
@@ -254,7 +266,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             uint64_t idle_since = 0;
             while (tp < ntiles) {
                 bool progress = false;
-                if (ts < ntiles && ts <= tp + 1 && mbar_try_wait(bar_kv_full + 8 * (ts & 1), (ts >> 1) & 1)) {
+                if (ts == 0 && ntiles >= 2 && mbar_try_wait(bar_kv_full, 0) && mbar_try_wait(bar_kv_full + 8, 0)) {
+                    NM_TRACE(12);
+                    scores_pair();
+                    NM_TRACE(3);
+                    NM_TRACE(13);
+                    ts = 2;
+                    progress = true;
+                } else if (ts < ntiles && ts <= tp + 1 && mbar_try_wait(bar_kv_full + 8 * (ts & 1), (ts >> 1) & 1)) {
                     if (ts == 0) NM_TRACE(12);
                     scores(ts);
                     if (ts == 0) NM_TRACE(3);
@@ -381,14 +400,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // Each CTA parks its (unscaled) O rows and its (m, l) in its own shared memory as soon as its last
     // P*V is done (the Q tile is free by then; layout [head][64 float4], the float4 index XOR-ed with
     // (head & 7) so that neither the row-per-thread writes nor the row-contiguous reads conflict).
+    // Its (m, l) pairs it pushes to the peers that own the heads.
     // After one cluster barrier, rank r combines heads [32r, 32r+32) over all peers - weights
     // 2^(m_peer - max m) - reading the peers' rows with many loads in flight, and writes one partial
     // per cluster.  A last barrier keeps every CTA's shared memory alive until its peers have read it.
+    __syncwarp();
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");       // all peers are running (they arrived at kernel start)
     if (warp >= 2 && warp < 6) {
         const int quad = warp & 3, head = quad * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
-        s_ml[head][0] = (ntiles > 0) ? m_own : -INFINITY;
-        s_ml[head][1] = l_own;
+        // (m, l) goes straight into the shared memory of the peer that owns the head: after the barrier the
+        // owner finds all four pairs locally
+        const uint32_t slot = peer_smem(smem_u32(&s_mlp[rank][head % kHeadsPerRank][0]), (uint32_t)head / kHeadsPerRank);
+        asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(slot), "f"((ntiles > 0) ? m_own : -INFINITY), "f"(l_own) : "memory");
         if (ntiles > 0) {
             for (int c = 0; c < kDvHalf / 32; ++c) {
                 uint32_t o[32];
@@ -413,9 +437,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             float pm[kCl], pl[kCl], M = -INFINITY;
 #pragma unroll
             for (int rr = 0; rr < kCl; ++rr) {
-                const float2 v = ld_peer_f2(peer_smem(smem_u32(&s_ml[head][0]), rr));
-                pm[rr] = v.x; pl[rr] = v.y;
-                M = fmaxf(M, v.x);
+                pm[rr] = s_mlp[rr][hl][0]; pl[rr] = s_mlp[rr][hl][1];
+                M = fmaxf(M, pm[rr]);
             }
             s_w[r][hl] = (pm[r] == -INFINITY) ? 0.f : fast_exp2(pm[r] - M);
             if (r == 0 && half == 0) {

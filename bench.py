@@ -108,7 +108,7 @@ class MlaStep:
 
     name = "mla"
 
-    def __init__(self, nm, device, seq_len, seed=4000, schedule="two-stream"):
+    def __init__(self, nm, device, seq_len, seed=4000, schedule="fused"):
         self.nm = nm
         self.S = seq_len
         self.schedule = schedule
@@ -143,7 +143,7 @@ class MlaStep:
         # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this shape, from
         # the ncu capture summarised in profiles/ncu_nm_row_tma_WO_M1_K16384_N7168.txt
         self.dominant_traffic = 234_948_352 + 3_600_128
-        self.launches_per_step = 7 if schedule == "fused" else 9
+        self.launches_per_step = 6 if schedule == "fused" else 7
         self.h2d = d * 2
         self.d2h = d * 2
 
@@ -155,8 +155,9 @@ class MlaStep:
                 "schedule": self.schedule,
                 "overlap": ("one stream: h*(W_DQ|W_DKV|W_KR) as one product; " if self.schedule == "fused" else
                             "two streams: KV chain (W_DKV|KR product, RMSNorm, RoPE, cache write) beside the W_DQ product; ")
-                           + "L2 prefetch of W_UV/W_O by idle lanes of the tcgen05 attention kernel; programmatic dependent "
-                             "launch along the chain, also across steps"}
+                           + "RMSNorm / RoPE / cache write inside the completion of the products that feed them; L2 prefetch of "
+                             "W_UV and 40 MB of W_O while the tcgen05 attention kernel runs; programmatic dependent launch along "
+                             "the chain, also across steps"}
 
     def step(self, stream, dom_events=None):
         if dom_events is not None:
@@ -489,7 +490,7 @@ def main():
     ap.add_argument("--workload", default="mla", choices=["mla", "projections", "matmul", "attention"])
     ap.add_argument("--mkn", default="1,16384,7168", help="M,K,N of --workload matmul")
     ap.add_argument("--layout", default="row", choices=["row", "col"])
-    ap.add_argument("--schedule", default="two-stream", choices=["fused", "two-stream"],
+    ap.add_argument("--schedule", default="fused", choices=["fused", "two-stream"],
                     help="decode step: down-projections as one concatenated product on one stream, or W_DKV|KR on a side stream")
     ap.add_argument("--timeline", action="store_true", help="print the kernel timeline of one step and exit")
     ap.add_argument("--sweep", action="store_true", help="also report GB/s of single narrow products vs M")

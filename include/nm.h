@@ -279,13 +279,19 @@ int nm_debug_set_plan(int tile_n, int nsplit);
 /* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel; 3 TMA-ring
  * CUDA-core kernel; 4 swap-AB tensor-core kernel) and the ring depth in stages (0 heuristic). */
 int nm_debug_set_kernel(int kind, int stages);
-/* Attention kernel: device buffer of 12 uint64 that receives phase timestamps (ns) of CTA (0,0):
- * start, set-up done, Q landed, first tile landed, scores ready, P written, last P*V done, after
- * cluster barrier 1, O parked in shared memory, after barrier 2, cluster sum written, end.  NULL = off. */
+/* Tuning aid: phase timestamps (ns, %globaltimer) of the decode step's kernels go to `device_buffer` (8192
+ * unsigned 64-bit values) when non-null: [0,32) phases of CTA (0,0) of the attention kernel; from 32 four per
+ * attention CTA (start, Q landed, last P*V done, end); from 1100 eight phases of two CTAs of the merge + W_UV
+ * kernel; from 2048 / 4096 / 6144 four per CTA (start, inputs ready, loop done, end) of the down-projection, W_UQR
+ * and W_O products.  NULL = off. */
 int nm_debug_set_attention_trace(void *device_buffer);
-/* Decode step tuning: launch the merge + W_UV kernel programmatically (default 1); include W_UV in the L2
- * prefetch (default 1). */
+/* Decode step tuning: uv_programmatic bit 0 - launch the merge + W_UV kernel programmatically (default 1), bit 1 -
+ * run RMSNorm / RoPE / cache write as kernels of their own instead of inside the products' completion;
+ * prefetch_w_uv - include W_UV in the L2 prefetch (default 1). */
 int nm_debug_set_step_knobs(int uv_programmatic, int prefetch_w_uv);
+/* Decode step tuning: force (tile_n, nsplit, ring stages) of one of its products - which = 0 the down-projection,
+ * 1 W_UQR, 2 W_O; zeros give the plan back to the planner. */
+int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages);
 /* Decode step: 1 (default) runs RoPE + W_UK and attention-merge + W_UV as fused per-head kernels, 0 as
  * separate kernels (rope, batched product, merge, batched product). */
 int nm_debug_set_step_fusion(int enable);

@@ -14,6 +14,8 @@
 
 namespace nm {
 
+struct VecTail;
+
 constexpr int kSMs = 148;                 // B200: 2 dies x 74 SMs
 constexpr int kMaxSplit = 64;             // upper bound on k-splits (sizes the workspace)
 constexpr int kMaxTileN = 2048;           // upper bound on columns per CTA tile
@@ -75,14 +77,18 @@ __device__ __forceinline__ float ld_cg(const float *p) { return __ldcg(p); }
 // Validates, plans and enqueues one (batched) narrow product; `ws` may be null when the plan does
 // not split K.  With programmatic_launch the kernel may begin (and prefetch B) before the previous
 // kernel in the stream has finished; it still waits for it before reading A or writing anything.
-// Defined in nm_matmul.cu.
+// `tail`: vector stages to run when the product's last tile completes (see VecTail); only the TMA ring kernel
+// takes it (M = 1, bf16 output) - *tail_taken says whether it did, the caller launches them itself otherwise.
+// `chained`: the launch is one link of a programmatic chain of kernels (the decode step); the planner then
+// prefers one CTA per SM with a deep ring and fewer k-splits.  Defined in nm_matmul.cu.
 int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, int H,
                    long lda, long strideA, long strideB, long ldc, long strideC,
                    nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream,
-                   bool programmatic_launch = false);
+                   bool programmatic_launch = false, unsigned long long *trace = nullptr, const struct VecTail *tail = nullptr,
+                   bool *tail_taken = nullptr, bool chained = false);
 
 // How the row-major bf16 product K x N (H heads) at this M will be split: k-rows per split and splits.
-void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit);
+void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit, bool chained = false);
 
 __host__ __device__ constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
 

@@ -62,7 +62,7 @@ static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t
 //  * k-rows per split a multiple of the stage height, so that no TMA box straddles two splits;
 //  * five 16 KB stages (two resident CTAs per SM), three when there are more CTAs than that, ten
 //    when M > 8.
-static Plan make_tma_plan(int M, int N, int K, int H)
+static Plan make_tma_plan(int M, int N, int K, int H, bool chained = false)
 {
     Plan p{};
     p.kind = kRowTma;
@@ -89,6 +89,21 @@ static Plan make_tma_plan(int M, int N, int K, int H)
     p.tn = tn; p.tpr = tpr; p.rg = kTmaConsumers / tpr; p.nsplit = ns; p.kr = kr; p.ntiles = ntiles;
     const long ctas = base * ns;
     int nstage = (M > 8) ? 10 : (ctas > 2 * kSMs ? 3 : 5);
+    if (chained && M <= 2 && g_force_split == 0 && g_force_tn == 0) {
+        // Launched programmatically inside a chain of kernels (the decode step): the CTAs are resident, and fill
+        // their rings, while the previous kernel drains, so a deep ring is prefetch for free; and every split-K
+        // gather at the end is a dependent round trip through L2 on the chain's critical path.  Measured in the
+        // step: at most one CTA per SM with an 8-stage ring, no split once there are about 100 tiles.
+        const int ns_c = base >= 96 ? 1 : (int)((kSMs * 9 / 10 + base / 2) / base);
+        int ns2 = ns_c < 1 ? 1 : ns_c;
+        if (ns2 > K / 128) ns2 = K / 128 > 0 ? K / 128 : 1;
+        if (ns2 > kMaxSplit) ns2 = kMaxSplit;
+        if (base * ns2 <= kSMs && base <= kNumCounters) {
+            kr = ceil_div(ceil_div(K, ns2), kt) * kt;
+            p.kr = kr; p.nsplit = ceil_div(K, kr);
+            nstage = 8;
+        }
+    }
     if (g_force_stages > 0) nstage = g_force_stages;
     if (nstage < 2) nstage = 2;
     if (nstage > 11) nstage = 11;
@@ -124,7 +139,7 @@ static Plan make_tc_plan(int M, int N, int K, int H)
     return p;
 }
 
-static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout, bool vec_ok, bool tma_ok)
+static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout, bool vec_ok, bool tma_ok, bool chained = false)
 {
     Plan p{};
     const int V = vec_elems(dtype);
@@ -139,7 +154,7 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     const bool tc_pays = M >= g_tc_min_m && 2.0 * K * N * H >= 32e6;
     if (layout == NM_ROW_MAJOR && tma_ok && g_force_kind != kRowTma && (tc_pays || g_force_kind == kRowTc))
         return make_tc_plan(M, N, K, H);
-    if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H);
+    if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H, chained);
     const int target = 192;                           // CTAs wanted in total (measured: 144-240 is the flat optimum)
     if (layout == NM_ROW_MAJOR) {
         p.kind = kRowVec;
@@ -235,8 +250,10 @@ static int check_common(const void *A, const void *B, const void *C, int M, int 
 
 static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int K, int H,
                        long lda, long strideA, long strideB, long ldc, long strideC,
-                       nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream, bool pdl = false)
+                       nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream, bool pdl = false,
+                       unsigned long long *trace = nullptr, const VecTail *tail = nullptr, bool *tail_taken = nullptr, bool chained = false)
 {
+    if (tail_taken) *tail_taken = false;
     int rc = check_common(A, B, C, M, N, K, H, dtype, layout);
     if (rc != NM_OK) return rc;
     if (lda < K || ldc < N || strideA < 0 || strideB < 0 || strideC < 0) return NM_ERR_INVALID_ARG;
@@ -251,13 +268,13 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     bool tma_ok = b_ok && a_ok && layout == NM_ROW_MAJOR && dtype != NM_F32 && tensor_map_encoder() != nullptr &&
                   (long)N * 2 < (1L << 40) && strideB >= 0;
     if (g_force_kind == kRowVec) tma_ok = false;
-    Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok);
+    Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok, chained);
     const CUtensorMap *tc_map_b = nullptr, *tc_map_a = nullptr;
     if (p.kind == kRowTc) {
         // weights [H][K][N] in 64x64 swizzled boxes; tokens [H][M][K] (row stride lda) in 64 x 16 swizzled boxes
         tc_map_b = get_weight_map(B, N, K, H, strideB, 64, kTcKT, true);
         tc_map_a = get_weight_map(A, K, M, H, strideA, 64, 16, true, lda);
-        if (!tc_map_b || !tc_map_a) p = make_tma_plan(M, N, K, H);      // strides the encoder refuses: CUDA-core kernel
+        if (!tc_map_b || !tc_map_a) p = make_tma_plan(M, N, K, H, chained);      // strides the encoder refuses: CUDA-core kernel
     }
 
     MatmulArgs a{};
@@ -286,6 +303,13 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         if (!map) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
         TmaArgs ta{};
         ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
+        ta.trace = trace;
+        if (tail && tail->enabled && M == 1 && dtype == NM_BF16 && H == 1 && ws && ws_bytes >= kCounterBytes && aligned16(ws) &&
+            p.ntiles < kNumCounters - 1) {
+            ta.tail = *tail;
+            ta.tail.counter = reinterpret_cast<unsigned *>(ws) + (kNumCounters - 1);     // the last counter is never a tile's
+            if (tail_taken) *tail_taken = true;
+        }
         const size_t smem = (size_t)p.nstage * kt * p.tn * 2 + kAChunkFloats * sizeof(float) + 2 * p.nstage * sizeof(uint64_t);
         const bool f32out = (dtype == NM_BF16_F32OUT);
         if (p.tpr == 8)       e = f32out ? launch_row_tma<8, float>(*map, ta, smem, stream)  : launch_row_tma<8, bf16_t>(*map, ta, smem, stream);
@@ -308,9 +332,9 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     return NM_OK;
 }
 
-void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit)
+void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit, bool chained)
 {
-    const Plan p = make_tma_plan(M, N, K, H);
+    const Plan p = make_tma_plan(M, N, K, H, chained);
     *k_rows_per_split = p.kr;
     *nsplit = p.nsplit;
 }
@@ -318,10 +342,11 @@ void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, i
 // internal entry used by the decode step
 int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, int H,
                    long lda, long strideA, long strideB, long ldc, long strideC,
-                   nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream, bool programmatic_launch)
+                   nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream, bool programmatic_launch,
+                   unsigned long long *trace, const VecTail *tail, bool *tail_taken, bool chained)
 {
     return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout, ws, ws_bytes, stream,
-                       programmatic_launch);
+                       programmatic_launch, trace, tail, tail_taken, chained);
 }
 
 }  // namespace nm

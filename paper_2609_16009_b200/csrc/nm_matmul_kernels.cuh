@@ -32,12 +32,95 @@ struct MatmulArgs {
 };
 
 // Extra launch state of the TMA-fed kernels.
+// The vector stages that consume a down-projection of the decode step, run by whichever CTA completes the
+// product's last tile (a grid-wide arrival counter: nobody waits): RMSNorm of x[0, q_lora) -> c_qn, and / or
+// RMSNorm of x[kv_off, kv_off + dc) and RoPE of the next `rope` elements -> cache_row.  x is the product's C.
+// This is the paper's remark that the normalisation, RoPE and caching start right where MatMul 2 ends
+// (MLA Operator Optimization), taken literally: no kernel boundary in between.
+struct VecTail {
+    int enabled;
+    int q_lora, kv_off, dc, rope;          // q_lora == 0: no query part; dc == 0: no KV part
+    float eps;
+    const uint16_t *gamma_q, *gamma_kv;
+    const float *cos_sin;                  // [rope/2][2] for the row's position
+    uint16_t *c_qn, *cache_row;
+    unsigned *counter;                     // zero on entry, left at zero
+};
+
 struct TmaArgs {
     MatmulArgs base;
     int nstage;            // ring depth
     int use_pdl;           // kernel was launched with programmatic stream serialization
     unsigned *status;      // device status word
+    unsigned long long *trace;   // tuning aid: when non-null every CTA stores four timestamps (start, inputs ready, loop done, end)
+    VecTail tail;
 };
+
+// Sum over the CTA (any size up to 1024 threads, a multiple of 32), same value in every thread.
+__device__ __forceinline__ float cta_sum(float v, float *scratch /* 32 floats */)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int w = 0; w < nw; ++w) t += scratch[w];
+    return t;
+}
+
+__device__ __forceinline__ uint32_t pack2_bf16_rn(float lo, float hi)
+{
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+}
+
+// All threads of one CTA; x was written by other CTAs of this grid (read past L1).
+__device__ __forceinline__ void vec_tail_run(const VecTail &t, const uint16_t *x, float *scratch)
+{
+    const int tid = threadIdx.x;
+    if (t.q_lora > 0) {                                            // up to 8 elements per thread (q_lora <= 2048, multiple of 8)
+        const int i0 = 8 * tid;
+        const bool on = i0 < t.q_lora;
+        float f[8], g[8];
+        if (on) {
+            Elem<bf16_t>::unpack(__ldcg(reinterpret_cast<const uint4 *>(x + i0)), f);
+            Elem<bf16_t>::unpack(__ldg(reinterpret_cast<const uint4 *>(t.gamma_q + i0)), g);
+        }
+        float ss = 0.f;
+        if (on)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+        ss = cta_sum(ss, scratch);
+        const float r = 1.0f / sqrtf(ss / (float)t.q_lora + t.eps);
+        if (on) {
+            uint4 o;
+            o.x = pack2_bf16_rn(f[0] * r * g[0], f[1] * r * g[1]); o.y = pack2_bf16_rn(f[2] * r * g[2], f[3] * r * g[3]);
+            o.z = pack2_bf16_rn(f[4] * r * g[4], f[5] * r * g[5]); o.w = pack2_bf16_rn(f[6] * r * g[6], f[7] * r * g[7]);
+            *reinterpret_cast<uint4 *>(t.c_qn + i0) = o;
+        }
+    }
+    if (t.dc > 0) {                                                // two elements per thread (dc <= 512, rope <= dc)
+        const uint16_t *ckr = x + t.kv_off;
+        const int i0 = 2 * tid;
+        float x0 = 0.f, x1 = 0.f, g0 = 0.f, g1 = 0.f;
+        if (i0 < t.dc) {
+            const uint32_t xv = __ldcg(reinterpret_cast<const uint32_t *>(ckr + i0)), gv = __ldg(reinterpret_cast<const uint32_t *>(t.gamma_kv + i0));
+            x0 = __uint_as_float(xv << 16); x1 = __uint_as_float(xv & 0xffff0000u);
+            g0 = __uint_as_float(gv << 16); g1 = __uint_as_float(gv & 0xffff0000u);
+        }
+        float r0 = 0.f, r1 = 0.f, c = 0.f, sn = 0.f;
+        if (i0 < t.rope) {
+            const uint32_t rv = __ldcg(reinterpret_cast<const uint32_t *>(ckr + t.dc + i0));
+            r0 = __uint_as_float(rv << 16); r1 = __uint_as_float(rv & 0xffff0000u);
+            c = t.cos_sin[i0]; sn = t.cos_sin[i0 + 1];
+        }
+        const float ss = cta_sum(fmaf(x0, x0, x1 * x1), scratch);
+        const float r = 1.0f / sqrtf(ss / (float)t.dc + t.eps);
+        if (i0 < t.dc) *reinterpret_cast<uint32_t *>(t.cache_row + i0) = pack2_bf16_rn(x0 * r * g0, x1 * r * g1);
+        if (i0 < t.rope) *reinterpret_cast<uint32_t *>(t.cache_row + t.dc + i0) = pack2_bf16_rn(r0 * c - r1 * sn, r0 * sn + r1 * c);
+    }
+}
 
 template <int M> struct RowCfg {
     static constexpr int kUnroll = (M <= 4) ? 8 : (M <= 8 ? 6 : 4);

@@ -5,6 +5,7 @@
 
 #include "nm_async.cuh"
 #include "nm_mla.cuh"
+#include "nm_matmul_kernels.cuh"
 
 namespace nm {
 
@@ -305,6 +306,8 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 
 // ---- host -------------------------------------------------------------------------------------------
 
+static int g_step_plan[3][3] = {};   // tuning: forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
+static int g_fused_tails = 1;        // run RMSNorm / RoPE / cache write inside the completion of the product that feeds them
 static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
 static int g_fused_heads = 1;        // per-head stages fused with their vector stage (q_finish, uv_merge) when the dims allow
 static int g_uv_pdl = 1;             // tuning: launch uv_merge programmatically
@@ -432,6 +435,16 @@ static int check_params(const nm_mla_params *p)
     return NM_OK;
 }
 
+// Tuning aid: slice of the trace buffer (see set_attention_trace) for one product of the step.
+static unsigned long long *trace_at(size_t offset) { return attention_trace() ? attention_trace() + offset : nullptr; }
+
+// Tuning aid: a forced plan around one product of the step.
+struct ScopedPlan {
+    bool on;
+    explicit ScopedPlan(const int (&f)[3]) : on(f[0] || f[1] || f[2]) { if (on) { nm_debug_set_plan(f[0], f[1]); nm_debug_set_kernel(-1, f[2]); } }
+    ~ScopedPlan() { if (on) { nm_debug_set_plan(0, 0); nm_debug_set_kernel(-1, 0); } }
+};
+
 #define NM_TRY(expr) do { int _rc = (expr); if (_rc != NM_OK) return _rc; } while (0)
 #define NM_LAUNCH_CHECK(what) do { cudaError_t _e = cudaGetLastError(); if (_e != cudaSuccess) return record_cuda_error(_e, what); } while (0)
 
@@ -473,15 +486,28 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         if (_e != cudaSuccess) return record_cuda_error(_e, #kern);                           \
     } while (0)
 
+    // The vector stages behind the down-projections (RMSNorm of the query latent; RMSNorm, RoPE and the cache-row
+    // write of the KV part) run inside the product that feeds them, in the CTA that completes its last tile,
+    // when that product is the TMA ring kernel; otherwise as kernels of their own.
+    const bool tails_ok = g_fused_tails && down_finish_applies(ql, dc, dr);
+    VecTail tq{}, tkv{};
+    tq.enabled = 1; tq.q_lora = ql; tq.eps = p->rms_eps; tq.gamma_q = (const uint16_t *)p->gamma_q; tq.c_qn = c_qn;
+    tkv.enabled = 1; tkv.kv_off = 0; tkv.dc = dc; tkv.rope = dr; tkv.eps = p->rms_eps; tkv.gamma_kv = (const uint16_t *)p->gamma_kv;
+    tkv.cos_sin = p->rope_cos_sin; tkv.cache_row = cache + (size_t)pos * dkv;
+    bool taken = false;
     const bool fused_down = p->W_DQKV && lay == NM_ROW_MAJOR && down_finish_applies(ql, dc, dr);
     if (fused_down) {
         // ---- one product for all three down-projections, h * (W_DQ | W_DKV | W_KR) (Eq. 3 extended by W_DQ),
-        //      then both vector stages in one two-CTA kernel: no side stream, an unbroken programmatic chain
+        //      with both vector stages in its completion: no side stream, an unbroken programmatic chain
         uint16_t *x_down = reinterpret_cast<uint16_t *>(ws + L.x_down);
+        VecTail both = tq;
+        both.kv_off = ql; both.dc = dc; both.rope = dr; both.gamma_kv = tkv.gamma_kv; both.cos_sin = tkv.cos_sin; both.cache_row = tkv.cache_row;
+        ScopedPlan sp(g_step_plan[0]);
         NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws,
-                              L.main_ws_bytes, ms, pdl && p->programmatic_entry));
-        NM_TRY(launch_down_finish(x_down, p->gamma_q, p->gamma_kv, p->rope_cos_sin, c_qn, cache + (size_t)pos * dkv, ql, dc, dr,
-                                  p->rms_eps, ms, pdl));
+                              L.main_ws_bytes, ms, pdl && p->programmatic_entry, trace_at(2048), tails_ok ? &both : nullptr, &taken, true));
+        if (!taken)
+            NM_TRY(launch_down_finish(x_down, p->gamma_q, p->gamma_kv, p->rope_cos_sin, c_qn, cache + (size_t)pos * dkv, ql, dc, dr,
+                                      p->rms_eps, ms, pdl));
         if (p->c_q) NM_CUDA_TRY(cudaMemcpyAsync(p->c_q, x_down, (size_t)ql * 2, cudaMemcpyDeviceToDevice, ms));
         if (p->ckr) NM_CUDA_TRY(cudaMemcpyAsync(p->ckr, x_down + ql, (size_t)dkv * 2, cudaMemcpyDeviceToDevice, ms));
     } else {
@@ -492,17 +518,22 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
             NM_CUDA_TRY(cudaEventRecord(g_events.fork, ms));
             NM_CUDA_TRY(cudaStreamWaitEvent(ss, g_events.fork, 0));
         }
-        NM_TRY(matmul_enqueue(p->h, p->W_DKVKR, ckr, 1, dkv, d, 1, d, 0, 0, dkv, 0, NM_BF16, lay, sws, L.side_ws_bytes, ss, false));
-        NM_LAUNCH(kv_finish_kernel, 1, 256, ss, (const uint16_t *)ckr, (const uint16_t *)p->gamma_kv, p->rope_cos_sin,
-                  cache + (size_t)pos * dkv, dc, dr, p->rms_eps);
+        NM_TRY(matmul_enqueue(p->h, p->W_DKVKR, ckr, 1, dkv, d, 1, d, 0, 0, dkv, 0, NM_BF16, lay, sws, L.side_ws_bytes, ss, false, nullptr,
+                              tails_ok ? &tkv : nullptr, &taken, false));
+        if (!taken)
+            NM_LAUNCH(kv_finish_kernel, 1, 256, ss, (const uint16_t *)ckr, (const uint16_t *)p->gamma_kv, p->rope_cos_sin,
+                      cache + (size_t)pos * dkv, dc, dr, p->rms_eps);
         if (forked) NM_CUDA_TRY(cudaEventRecord(g_events.join, ss));
 
         // ---- Q chain, main stream ----------------------------------------------------------------------------
         NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms,
-                              pdl && (!forked || p->programmatic_entry)));
-        NM_LAUNCH(rmsnorm_kernel, 1, 256, ms, (const uint16_t *)c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
+                              pdl && (!forked || p->programmatic_entry), nullptr, tails_ok ? &tq : nullptr, &taken, !forked));
+        if (!taken) NM_LAUNCH(rmsnorm_kernel, 1, 256, ms, (const uint16_t *)c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
     }
-    NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl));
+    {
+        ScopedPlan sp(g_step_plan[1]);
+        NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl, trace_at(4096), nullptr, nullptr, true));
+    }
     const bool fused = g_fused_heads && head_kernels_apply(H, dn, dr, dc, dv);
     if (fused) {
         // RoPE of the rope part and q_lat[h] = q[h, :nope] * W_UK[h] in one kernel, one CTA per head
@@ -524,7 +555,10 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         pf.block_bytes = g_prefetch_uv ? (long)H * dc * dv * 2 : 0;
         if (p->W_O && lay == NM_ROW_MAJOR) {
             int kr = 0, ns = 1;
-            matmul_row_major_split(1, d, H * dv, 1, &kr, &ns);
+            {
+                ScopedPlan sp(g_step_plan[2]);
+                matmul_row_major_split(1, d, H * dv, 1, &kr, &ns, true);
+            }
             const long row_bytes = (long)d * 2;
             long rows = ((long)g_prefetch_mb << 20) / ns / row_bytes;
             if (rows > kr) rows = kr;
@@ -556,8 +590,9 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     }
     if (p->W_O) {
         if (p->event_before_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_before_wo, ms));
+        ScopedPlan sp(g_step_plan[2]);
         NM_TRY(matmul_enqueue(o, p->W_O, p->out, 1, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms,
-                              pdl && !p->event_before_wo));
+                              pdl && !p->event_before_wo, trace_at(6144), nullptr, nullptr, true));
         if (p->event_after_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_after_wo, ms));
     }
 #undef NM_LAUNCH
@@ -652,9 +687,16 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     return NM_OK;
 }
 
+int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages)
+{
+    if (which < 0 || which > 2) return NM_ERR_INVALID_ARG;
+    g_step_plan[which][0] = tile_n; g_step_plan[which][1] = nsplit; g_step_plan[which][2] = stages;
+    return NM_OK;
+}
+
 int nm_debug_set_step_knobs(int uv_pdl, int prefetch_uv)
 {
-    g_uv_pdl = uv_pdl; g_prefetch_uv = prefetch_uv;
+    g_uv_pdl = uv_pdl & 1; g_prefetch_uv = prefetch_uv & 1; g_fused_tails = (uv_pdl & 2) ? 0 : 1;
     return NM_OK;
 }
 

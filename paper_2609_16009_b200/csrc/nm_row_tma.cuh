@@ -66,8 +66,10 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
     const int ke = min(a.K, kb + a.kr);
     const int n_it = ceil_div(ke - kb, KT);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + NS);
+    unsigned long long *trace = ta.trace ? ta.trace + 4 * (((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) : nullptr;
 
     if (tid == 0) {
+        if (trace) trace[0] = global_timer_ns();
         s_abort = 0;
         s_issued = 0;
         for (int s = 0; s < NS; ++s) {
@@ -152,6 +154,7 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
         fetch_chunk(kb);
         store_chunk();
         named_barrier_sync(1, kTmaConsumers);
+        if (trace && tid == 0) trace[1] = global_timer_ns();
         if (n_it > ITS_PER_CHUNK) fetch_chunk(kb + KCH);
 
         const int rows_last = (ke - kb) - (n_it - 1) * KT;            // rows in the last stage (1..KT)
@@ -218,6 +221,7 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
 
     // ---- all 288 threads: reduce the row groups through shared memory (the ring is free now) ------
     __syncthreads();
+    if (trace && tid == 0) trace[2] = global_timer_ns();
     if (s_abort) {
         // A wait expired.  Give copies that were issued a bounded chance to land before the CTA exits.
         if (tid == 0) {
@@ -264,6 +268,20 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
         }
     }
     if (a.nsplit > 1) splitk_complete<M, TO>(a, tile, h, &s_last);
+    if constexpr (M == 1 && sizeof(TO) == 2) {
+        if (ta.tail.enabled && (a.nsplit == 1 || s_last)) {        // this CTA has just completed its tile (uniform over the CTA)
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) s_last = (atomicAdd(ta.tail.counter, 1u) == (unsigned)(a.ntiles * a.H - 1));
+            __syncthreads();
+            if (s_last) {                                          // ... and it was the last tile of the product
+                __threadfence();
+                if (tid == 0) *ta.tail.counter = 0u;
+                vec_tail_run(ta.tail, reinterpret_cast<const uint16_t *>(a.C), reinterpret_cast<float *>(ring));
+            }
+        }
+    }
+    if (trace && tid == 0) trace[3] = global_timer_ns();
 }
 
 template <int TPR, typename TO>

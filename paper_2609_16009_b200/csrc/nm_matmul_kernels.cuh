@@ -75,8 +75,8 @@ __device__ __forceinline__ uint32_t pack2_bf16_rn(float lo, float hi)
     return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
 }
 
-// All threads of one CTA; x was written by other CTAs of this grid (read past L1).
-__device__ __forceinline__ void vec_tail_run(const VecTail &t, const uint16_t *x, float *scratch)
+// All threads of one CTA.  xs: the product's output row as fp32 values already rounded to bf16, in shared memory.
+__device__ __forceinline__ void vec_tail_run(const VecTail &t, const float *xs, float *scratch)
 {
     const int tid = threadIdx.x;
     if (t.q_lora > 0) {                                            // up to 8 elements per thread (q_lora <= 2048, multiple of 8)
@@ -84,7 +84,8 @@ __device__ __forceinline__ void vec_tail_run(const VecTail &t, const uint16_t *x
         const bool on = i0 < t.q_lora;
         float f[8], g[8];
         if (on) {
-            Elem<bf16_t>::unpack(__ldcg(reinterpret_cast<const uint4 *>(x + i0)), f);
+            const float4 a = *reinterpret_cast<const float4 *>(xs + i0), b = *reinterpret_cast<const float4 *>(xs + i0 + 4);
+            f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
             Elem<bf16_t>::unpack(__ldg(reinterpret_cast<const uint4 *>(t.gamma_q + i0)), g);
         }
         float ss = 0.f;
@@ -101,18 +102,17 @@ __device__ __forceinline__ void vec_tail_run(const VecTail &t, const uint16_t *x
         }
     }
     if (t.dc > 0) {                                                // two elements per thread (dc <= 512, rope <= dc)
-        const uint16_t *ckr = x + t.kv_off;
+        const float *ckr = xs + t.kv_off;
         const int i0 = 2 * tid;
         float x0 = 0.f, x1 = 0.f, g0 = 0.f, g1 = 0.f;
         if (i0 < t.dc) {
-            const uint32_t xv = __ldcg(reinterpret_cast<const uint32_t *>(ckr + i0)), gv = __ldg(reinterpret_cast<const uint32_t *>(t.gamma_kv + i0));
-            x0 = __uint_as_float(xv << 16); x1 = __uint_as_float(xv & 0xffff0000u);
+            const uint32_t gv = __ldg(reinterpret_cast<const uint32_t *>(t.gamma_kv + i0));
+            x0 = ckr[i0]; x1 = ckr[i0 + 1];
             g0 = __uint_as_float(gv << 16); g1 = __uint_as_float(gv & 0xffff0000u);
         }
         float r0 = 0.f, r1 = 0.f, c = 0.f, sn = 0.f;
         if (i0 < t.rope) {
-            const uint32_t rv = __ldcg(reinterpret_cast<const uint32_t *>(ckr + t.dc + i0));
-            r0 = __uint_as_float(rv << 16); r1 = __uint_as_float(rv & 0xffff0000u);
+            r0 = ckr[t.dc + i0]; r1 = ckr[t.dc + i0 + 1];
             c = t.cos_sin[i0]; sn = t.cos_sin[i0 + 1];
         }
         const float ss = cta_sum(fmaf(x0, x0, x1 * x1), scratch);
@@ -120,6 +120,59 @@ __device__ __forceinline__ void vec_tail_run(const VecTail &t, const uint16_t *x
         if (i0 < t.dc) *reinterpret_cast<uint32_t *>(t.cache_row + i0) = pack2_bf16_rn(x0 * r * g0, x1 * r * g1);
         if (i0 < t.rope) *reinterpret_cast<uint32_t *>(t.cache_row + t.dc + i0) = pack2_bf16_rn(r0 * c - r1 * sn, r0 * sn + r1 * c);
     }
+}
+
+// Completion of a product that carries a VecTail (M = 1, bf16 output, one head).  One arrival counter for the
+// whole grid instead of one per tile: every CTA publishes its tile (split-K: its fp32 partial tile; otherwise
+// the finished bf16 columns) and arrives; the last CTA of the grid gathers every column - partials summed in
+// split order, rounded once - writes C, keeps the rounded row in shared memory and runs the vector stages on
+// it.  One fence / atomic / load round trip through L2 in all, where a per-tile gather followed by a grid-wide
+// counter would take two.  `xs` needs N floats (+32 of scratch behind them).
+__device__ __forceinline__ void tail_complete(const MatmulArgs &a, const VecTail &t, int *s_last, float *xs)
+{
+    const int tid = threadIdx.x;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) *s_last = (atomicAdd(t.counter, 1u) == (unsigned)(a.ntiles * a.nsplit - 1));
+    __syncthreads();
+    if (!*s_last) return;
+    __threadfence();
+    if (tid == 0) *t.counter = 0u;
+    uint16_t *C = reinterpret_cast<uint16_t *>(a.C);
+    // eight columns per thread and pass, all their partials requested before the first is used
+    constexpr int kCols = 8;
+    for (int n0 = 0; n0 < a.N; n0 += kCols * blockDim.x) {
+        float s[kCols];
+        const float *P[kCols];
+#pragma unroll
+        for (int j = 0; j < kCols; ++j) {
+            const int n = min(n0 + j * (int)blockDim.x + tid, a.N - 1);
+            const int tile = n / a.tn, c = n - tile * a.tn;
+            P[j] = a.partial + (size_t)tile * a.nsplit * a.tn + c;
+            s[j] = 0.f;
+        }
+        if (a.nsplit > 1) {
+#pragma unroll 4
+            for (int sp = 0; sp < a.nsplit; ++sp)
+#pragma unroll
+                for (int j = 0; j < kCols; ++j) s[j] += ld_cg(P[j] + (size_t)sp * a.tn);
+        }
+#pragma unroll
+        for (int j = 0; j < kCols; ++j) {
+            const int n = n0 + j * (int)blockDim.x + tid;
+            if (n < a.N) {
+                if (a.nsplit > 1) {
+                    const __nv_bfloat16 b = __float2bfloat16_rn(s[j]);
+                    C[n] = __bfloat16_as_ushort(b);
+                    xs[n] = __bfloat162float(b);
+                } else {
+                    xs[n] = __uint_as_float((uint32_t)__ldcg(C + n) << 16);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    vec_tail_run(t, xs, xs + ((a.N + 31) & ~31));
 }
 
 template <int M> struct RowCfg {

@@ -110,6 +110,14 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
         // ---------------- consumers ---------------------------------------------------------------
         const int tx = tid % TPR, ty = tid / TPR;
         const bf16_t *__restrict__ A = (const bf16_t *)a.A + (long)h * a.strideA;
+        if constexpr (M == 1 && sizeof(TO) == 2) {
+            // whichever CTA ends up running the vector stages wants their constants in L2 by then
+            if (ta.tail.enabled) {
+                if (ta.tail.q_lora > 0 && tid * 64 < ta.tail.q_lora) asm volatile("prefetch.global.L2 [%0];" ::"l"(ta.tail.gamma_q + tid * 64));
+                if (ta.tail.dc > 0 && tid * 64 < ta.tail.dc) asm volatile("prefetch.global.L2 [%0];" ::"l"(ta.tail.gamma_kv + tid * 64));
+                if (ta.tail.dc > 0 && tid * 32 < ta.tail.rope) asm volatile("prefetch.global.L2 [%0];" ::"l"(ta.tail.cos_sin + tid * 32));
+            }
+        }
         if (MP != M)
             for (int i = tid; i < kAChunkFloats; i += kTmaConsumers) As[i] = 0.f;
         pdl_wait_prior_grids();                       // A (and the workspace) come from earlier kernels
@@ -267,20 +275,14 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
             }
         }
     }
-    if (a.nsplit > 1) splitk_complete<M, TO>(a, tile, h, &s_last);
     if constexpr (M == 1 && sizeof(TO) == 2) {
-        if (ta.tail.enabled && (a.nsplit == 1 || s_last)) {        // this CTA has just completed its tile (uniform over the CTA)
-            __threadfence();
-            __syncthreads();
-            if (tid == 0) s_last = (atomicAdd(ta.tail.counter, 1u) == (unsigned)(a.ntiles * a.H - 1));
-            __syncthreads();
-            if (s_last) {                                          // ... and it was the last tile of the product
-                __threadfence();
-                if (tid == 0) *ta.tail.counter = 0u;
-                vec_tail_run(ta.tail, reinterpret_cast<const uint16_t *>(a.C), reinterpret_cast<float *>(ring));
-            }
+        if (ta.tail.enabled) {
+            tail_complete(a, ta.tail, &s_last, reinterpret_cast<float *>(ring));
+            if (trace && tid == 0) trace[3] = global_timer_ns();
+            return;
         }
     }
+    if (a.nsplit > 1) splitk_complete<M, TO>(a, tile, h, &s_last);
     if (trace && tid == 0) trace[3] = global_timer_ns();
 }
 

@@ -166,6 +166,42 @@ class MlaStep:
             self.p.event_before_wo, self.p.event_after_wo = None, None
         self.nm.nm_mla_decode_step(self.p, stream, self.side)
 
+    def extra_measurements(self, stream):
+        """Outside the timed region, reported beside it: the same step replayed from a CUDA graph of ten steps
+        (device time without per-launch work of the host-side queue), and the step without its last product
+        (W_O = NULL; it is 63 % of the step's bytes)."""
+        out = {}
+        def timed(fn, n):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(n):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b)
+        self.p.event_before_wo, self.p.event_after_wo = None, None
+        try:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for _ in range(10):
+                    self.nm.nm_mla_decode_step(self.p, stream, self.side)
+            g.replay(); torch.cuda.synchronize()
+            out["graph_replay"] = {"decode_us": min(timed(g.replay, 20) for _ in range(3)) / 200 * 1e3, "steps_per_graph": 10}
+            del g
+        except Exception as exc:          # capture is an extra; the main number does not depend on it
+            out["graph_replay"] = {"error": repr(exc)}
+        wo = self.p.W_O
+        self.p.W_O = None
+        try:
+            fn = lambda: self.nm.nm_mla_decode_step(self.p, stream, self.side)
+            timed(fn, 50)
+            us = min(timed(fn, 200) for _ in range(3)) / 200 * 1e3
+            nb = self.bytes_per_step - self.dominant_bytes
+            out["without_W_O"] = {"decode_us": us, "GBps": nb / us / 1e3, "algorithmic_bytes": nb}
+        finally:
+            self.p.W_O = wo
+        return out
+
     def step_e2e(self, stream):
         """Token in from pinned host memory, step, result out to pinned host memory.  The whole
         sequence (two copies, the kernels of both streams) is captured once into a CUDA graph and
@@ -294,6 +330,48 @@ def print_timeline(wl, stream, steps=6):
     print(f"# next step starts at {evs[k0 + per].time_range.start - t0:.1f}")
 
 
+def batched_case(nm, device, T, K, N, H):
+    """One batched per-head product (bf16, row-major weights [H][K][N], activations [T][H][K]) timed like the
+    other sweep cases: CUDA-graph replay over rotating copies of the weights, serial and programmatic."""
+    nbytes = H * K * N * 2
+    R = max(2, min(64, (1 << 29) // nbytes + 1))
+    Bs = (torch.randn(R, H * K * N, device=device) * 0.02).to(torch.bfloat16)
+    A = torch.randn(T * H * K, device=device).to(torch.bfloat16)
+    C = torch.empty(R, T * H * N, device=device, dtype=torch.bfloat16)
+    ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(T, N, K, H), device=device)
+    s = torch.cuda.Stream(device)
+    row = {"M": T, "K": K, "N": N, "H": H, "dtype": "bf16", "layout_B": "row", "batched": True}
+    algo = (H * K * N + T * H * K + T * H * N) * 2
+    def launch(i):
+        nm.nm_matmul_batched_ws(A, Bs[i], C[i], T, N, K, H, H * K, K, K * N, H * N, N, nm.BF16, nm.ROW_MAJOR, ws, s)
+    for mode in ("serial", "programmatic"):
+        nm.nm_set_programmatic_launch(mode == "programmatic")
+        with torch.cuda.stream(s):
+            for i in range(R):
+                launch(i)
+            s.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for i in range(R):
+                    launch(i)
+            g.replay(); s.synchronize()
+            ts = []
+            for _ in range(21):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(s); g.replay(); b.record(s); s.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3 / R)
+        ts.sort()
+        us = statistics.median(ts)
+        key = "" if mode == "serial" else "_programmatic"
+        row["us" + key] = round(us, 2)
+        row["us_mean_p5_p95" + key] = [round(statistics.mean(ts), 2), round(ts[1], 2), round(ts[-2], 2)]
+        row["GBps" + key] = round(algo / us / 1e3, 1)
+        del g
+    nm.nm_set_programmatic_launch(False)
+    row["pct_of_8TBs"] = round(max(row["GBps"], row["GBps_programmatic"]) / 80.0, 1)
+    return row
+
+
 def matmul_sweep(nm, device):
     """GB/s of single narrow products (cold L2: the launches of a CUDA graph rotate through copies of
     B that together exceed 512 MB).  Two figures per case: launches in plain stream order (each kernel
@@ -305,7 +383,16 @@ def matmul_sweep(nm, device):
              (1, 7168, 576, 1, "bf16")]
     for M in (1, 2, 4, 8, 16):
         cases += [(M, 1536, 24576, 0, "bf16"), (M, 7168, 18432, 0, "bf16")]
-    for M, K, N, layout, dt in cases:
+    # the per-head products of the absorbed MLA form, T tokens at once: q_nope * W_UK (128 -> 512) and
+    # o_lat * W_UV (512 -> 128), 128 heads, activations laid out [T][128][K]
+    for T in (1, 4, 16):
+        cases += [(T, 128, 512, 0, "bf16", 128), (T, 512, 128, 0, "bf16", 128)]
+    for case in cases:
+        M, K, N, layout, dt = case[:5]
+        H = case[5] if len(case) > 5 else 1
+        if H > 1:
+            out.append(batched_case(nm, device, M, K, N, H))
+            continue
         es = 4 if dt == "f32" else 2
         tdt = torch.float32 if dt == "f32" else torch.bfloat16
         code = nm.F32 if dt == "f32" else nm.BF16
@@ -330,13 +417,15 @@ def matmul_sweep(nm, device):
                         nm.nm_matmul_ws(A, Bs[i], C[i], M, N, K, code, layout, ws, s)
                 g.replay(); s.synchronize()
                 ts = []
-                for _ in range(5):
+                for _ in range(21):
                     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     a.record(s); g.replay(); b.record(s); s.synchronize()
                     ts.append(a.elapsed_time(b) * 1e3 / R)
+            ts.sort()
             us = statistics.median(ts)
             key = "" if mode == "serial" else "_programmatic"
             row["us" + key] = round(us, 2)
+            row["us_mean_p5_p95" + key] = [round(statistics.mean(ts), 2), round(ts[1], 2), round(ts[-2], 2)]
             row["GBps" + key] = round(algo / us / 1e3, 1)
             del g
         nm.nm_set_programmatic_launch(False)
@@ -568,6 +657,7 @@ def main():
         barrier()
         e2e_ms = t0.elapsed_time(t1)
         clocks = sampler.stop()
+        extras = wl.extra_measurements(stream) if hasattr(wl, "extra_measurements") else {}
     nm.nm_check_status(stream)
 
     ms, e2e_ms, dom_ms = reduce_over_ranks([ms, e2e_ms, dom_ms], dist, device)
@@ -593,15 +683,21 @@ def main():
                              "frac": achieved / peak, "peak_kind": peak_kind, "algorithmic_bytes": wl.dominant_bytes,
                              "traffic": getattr(wl, "dominant_traffic", None),
                              "us_per_launch": dom_ms * 1e3}}
+        line.update(extras)
         if args.sweep:
             line["narrow_matmul_vs_M"] = matmul_sweep(nm, device)
         if not args.no_cpu_baseline:
             import oracle
             threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
-            oracle_sample(threads, args.workload, args.seq_len)
-            dt, nbytes, what = oracle_sample(threads, args.workload, args.seq_len)
-            line["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
-                                    "sample": what, "seconds": dt}
+            oracle_sample(threads, args.workload, args.seq_len)                    # warm-up pass (page faults, thread pool)
+            total, passes, nbytes, what = 0.0, 0, 0, ""
+            while total < 10.0 and passes < 200:                                   # about ten seconds of CPU work
+                dt, nbytes, what = oracle_sample(threads, args.workload, args.seq_len)
+                total += dt
+                passes += 1
+            line["cpu_baseline"] = {"value": nbytes * passes / total / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+                                    "sample": f"{passes} passes of " + what.replace(", one pass", ""), "seconds": total,
+                                    "ms_per_step": total / passes * 1e3}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

@@ -91,6 +91,8 @@ _lib.nm_mla_decode_step.argtypes = [C.POINTER(MlaParams), _vp, _vp]
 _lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_debug_set_attention.argtypes = [_i]
 _lib.nm_debug_set_step_pdl.argtypes = [_i]
+_lib.nm_debug_set_step_knobs.argtypes = [_i, _i]
+_lib.nm_debug_set_step_plan.argtypes = [_i, _i, _i, _i]
 _lib.nm_debug_set_step_prefetch.argtypes = [_i]
 _lib.nm_debug_set_step_fusion.argtypes = [_i]
 _lib.nm_debug_set_attention_trace.argtypes = [_vp]
@@ -305,6 +307,14 @@ def nm_debug_set_step_fusion(enable: bool) -> None:
 
 def nm_debug_set_step_prefetch(megabytes: int) -> None:
     _check(_lib.nm_debug_set_step_prefetch(int(megabytes)), "nm_debug_set_step_prefetch")
+
+
+def nm_debug_set_step_knobs(uv_programmatic: int = 1, prefetch_w_uv: int = 1) -> None:
+    _check(_lib.nm_debug_set_step_knobs(int(uv_programmatic), int(prefetch_w_uv)), "nm_debug_set_step_knobs")
+
+
+def nm_debug_set_step_plan(which: int, tile_n: int = 0, nsplit: int = 0, stages: int = 0) -> None:
+    _check(_lib.nm_debug_set_step_plan(which, tile_n, nsplit, stages), "nm_debug_set_step_plan")
 
 
 def nm_debug_set_step_pdl(enable: bool) -> None:

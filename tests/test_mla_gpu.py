@@ -294,6 +294,48 @@ def test_decode_step_fused_and_unfused_per_head_stages_agree(nm, weights, ref102
         assert np.all(np.abs(a - b) <= 2e-3 * np.abs(b).max() + oracle.ulp_bf16(b)), k      # rounded outputs: one ulp on top
 
 
+@pytest.mark.parametrize("concat_down", [False, True])
+def test_decode_step_vector_stages_inside_and_outside_the_products_agree(nm, weights, ref1024, concat_down):
+    # RMSNorm / RoPE / cache-row write in the completion of the down-projection products (default) against the
+    # same stages as kernels of their own: both routes against the oracle, and against each other
+    w, dw = weights
+    h, cache_ref, r = ref1024
+    cache_in = gen.mla_cache(1024, DIMS, seed=4200)
+    t1 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
+    check_step(t1, r, cache_ref, 1024)
+    nm.nm_debug_set_step_knobs(1 | 2, 1)
+    try:
+        t2 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
+        check_step(t2, r, cache_ref, 1024)
+    finally:
+        nm.nm_debug_set_step_knobs(1, 1)
+    # the products are bit-identical (same plan, same summation order); the norms sum their squares in a
+    # different order, so c_qn and the cache row may differ by a rounding flip
+    for k in ("c_q", "ckr"):
+        assert torch.equal(t1[k], t2[k]), k
+    for k in ("c_qn", "kv_cache"):
+        a, b = dev_bits_to_f64(t1[k]), dev_bits_to_f64(t2[k])
+        assert np.all(np.abs(a - b) <= oracle.ulp_bf16(b) + 1e-6), k
+        assert np.mean(a == b) > 0.99, k
+
+
+def test_decode_step_forced_product_plans_inside_the_step(nm, weights, ref1024):
+    # the step's products under other tilings / k-splits / ring depths than the planner's: same result within
+    # the bound (parity against the oracle), the plan goes back to the planner afterwards
+    w, dw = weights
+    h, cache_ref, r = ref1024
+    cache_in = gen.mla_cache(1024, DIMS, seed=4200)
+    try:
+        for which, plan in ((0, (64, 7, 3)), (1, (256, 2, 4)), (2, (128, 3, 5)), (2, (64, 2, 5))):
+            nm.nm_debug_set_step_plan(which, *plan)
+            t = run_step(nm, dw, h, cache_in, 1024, concat_down=True)
+            check_step(t, r, cache_ref, 1024)
+            nm.nm_debug_set_step_plan(which, 0, 0, 0)
+    finally:
+        for which in range(3):
+            nm.nm_debug_set_step_plan(which, 0, 0, 0)
+
+
 def test_decode_step_without_wo_and_repeatable(nm, weights):
     w, dw = weights
     S = 300

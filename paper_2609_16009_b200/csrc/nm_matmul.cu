@@ -132,6 +132,8 @@ static Plan make_tc_plan(int M, int N, int K, int H)
     p.kr = kr;
     p.nsplit = ceil_div(K, kr);
     int nstage = 5;
+    const int its = ceil_div(kr, kTcKT);                // a ring deeper than the CTA's k-range only costs shared memory
+    if (nstage > its) nstage = its;
     if (g_force_stages > 0) nstage = g_force_stages;
     if (nstage < 2) nstage = 2;
     if (nstage > 10) nstage = 10;
@@ -151,7 +153,10 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     // Measured on B200: from M = 3 on, the CUDA-core kernel falls off the HBM roofline on large weight
     // matrices (fp32 FMA issue) while the tensor-core kernel stays on it; small matrices are
     // latency-bound either way and the CUDA-core kernel has the shorter fixed cost.
-    const bool tc_pays = M >= g_tc_min_m && 2.0 * K * N * H >= 32e6;
+    // Thresholds from sweeps of both kernels over 8-34 MB matrices and the batched per-head shapes: from 16 MB
+    // (8 MB when batched over heads) the tensor-core kernel wins from M = 3 on; at 8 MB in one matrix the two tie.
+    const double wbytes = 2.0 * K * N * H;
+    const bool tc_pays = M >= g_tc_min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6));
     if (layout == NM_ROW_MAJOR && tma_ok && g_force_kind != kRowTma && (tc_pays || g_force_kind == kRowTc))
         return make_tc_plan(M, N, K, H);
     if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H, chained);

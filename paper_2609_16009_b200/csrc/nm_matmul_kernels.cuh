@@ -182,12 +182,63 @@ template <int M> struct RowCfg {
     static constexpr int kPass = (M < 4) ? M : 4;                  // m-rows reduced per pass
 };
 
+// Sum of the nsplit partial tiles of one (head, tile), in split order, rounded once and written to C.
+template <typename TO>
+__device__ __forceinline__ void splitk_gather(const float *P, TO *C, int M, int tn, int nsplit, int N, int tile, long ldc)
+{
+    // Four outputs per thread and pass, and the partials of all four requested four splits at a time before any
+    // is used: a chain of L2 round trips otherwise (M * tile_n outputs x nsplit partials, one CTA).  The inner
+    // loops are free of branches - a slot past the thread's last output repeats that output's address and its
+    // sum is dropped - so that the loads really are issued back to back.
+    constexpr int kOut = 4;
+    const int tid = threadIdx.x, total = M * tn, stride = (int)blockDim.x;
+    const size_t split_stride = (size_t)M * tn;
+    for (int i0 = 0; i0 < total; i0 += kOut * stride) {
+        const int live = min(kOut, (total - i0 - tid + stride - 1) / stride);     // outputs this thread has in this pass
+        if (live <= 0) continue;
+        float s[kOut];
+        const float *src[kOut];
+#pragma unroll
+        for (int j = 0; j < kOut; ++j) {
+            src[j] = P + (i0 + min(j, live - 1) * stride + tid);
+            s[j] = 0.f;
+        }
+        int sp = 0;
+        for (; sp + 4 <= nsplit; sp += 4) {
+            float v[4][kOut];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int j = 0; j < kOut; ++j) v[u][j] = ld_cg(src[j] + (sp + u) * split_stride);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)                            // split order: deterministic
+#pragma unroll
+                for (int j = 0; j < kOut; ++j) s[j] += v[u][j];
+        }
+        for (; sp < nsplit; ++sp) {
+            float v[kOut];
+#pragma unroll
+            for (int j = 0; j < kOut; ++j) v[j] = ld_cg(src[j] + sp * split_stride);
+#pragma unroll
+            for (int j = 0; j < kOut; ++j) s[j] += v[j];
+        }
+#pragma unroll
+        for (int j = 0; j < kOut; ++j) {
+            if (j < live) {
+                const int i = i0 + j * stride + tid;
+                const int m = i / tn, c = i - m * tn, n = tile * tn + c;
+                if (n < N) C[(long)m * ldc + n] = round_out<TO>(s[j]);
+            }
+        }
+    }
+}
+
 // ---- split-K completion shared by both kernels -----------------------------------------------------
 //
 // Called by all threads of the CTA after its partial tile has been written to `partial`.  The
 // last CTA to arrive at (h, tile) reads all nsplit partial tiles in order and writes C; it then
 // puts the counter back to zero, so the workspace needs no clearing between launches.
-template <typename TO>
+template <typename TO, bool kBatched = true>
 __device__ __forceinline__ void splitk_complete_rt(const MatmulArgs &a, int M, int tile, int h, int *s_last)
 {
     const int tid = threadIdx.x;
@@ -203,14 +254,18 @@ __device__ __forceinline__ void splitk_complete_rt(const MatmulArgs &a, int M, i
     __threadfence();
     const float *P = a.partial + ((size_t)h * a.ntiles + tile) * a.nsplit * (size_t)(M * a.tn);
     TO *C = (TO *)a.C + (long)h * a.strideC;
-    for (int i = tid; i < M * a.tn; i += blockDim.x) {
-        const int m = i / a.tn, c = i - m * a.tn, n = tile * a.tn + c;
-        if (n < a.N) {
-            float s = 0.f;
+    if constexpr (!kBatched) {                                     // few outputs per thread (M <= 2): the plain loop, and
+        for (int i = tid; i < M * a.tn; i += blockDim.x) {         // nothing that would change the main loop's registers
+            const int m = i / a.tn, c = i - m * a.tn, n = tile * a.tn + c;
+            if (n < a.N) {
+                float s = 0.f;
 #pragma unroll 4
-            for (int sp = 0; sp < a.nsplit; ++sp) s += ld_cg(P + ((size_t)sp * M + m) * a.tn + c);
-            C[(long)m * a.ldc + n] = round_out<TO>(s);
+                for (int sp = 0; sp < a.nsplit; ++sp) s += ld_cg(P + ((size_t)sp * M + m) * a.tn + c);
+                C[(long)m * a.ldc + n] = round_out<TO>(s);
+            }
         }
+    } else {
+        splitk_gather<TO>(P, C, M, a.tn, a.nsplit, a.N, tile, a.ldc);
     }
     if (tid == 0) *cnt = 0u;
 }
@@ -218,7 +273,7 @@ __device__ __forceinline__ void splitk_complete_rt(const MatmulArgs &a, int M, i
 template <int M, typename TO>
 __device__ __forceinline__ void splitk_complete(const MatmulArgs &a, int tile, int h, int *s_last)
 {
-    splitk_complete_rt<TO>(a, M, tile, h, s_last);
+    splitk_complete_rt<TO, (M > 2)>(a, M, tile, h, s_last);
 }
 
 // ---- row-major B (n contiguous): each thread owns kVec consecutive columns ---------------------------

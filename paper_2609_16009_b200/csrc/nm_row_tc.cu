@@ -29,7 +29,7 @@ constexpr int kStage = kBStage + kAStage;
 constexpr uint32_t kTmemColsTc = 32;
 
 template <typename TO>
-__global__ void __launch_bounds__(kTcThreads, 2)
+__global__ void __launch_bounds__(kTcThreads, 4)
 nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_a, const TmaArgs ta)
 {
     const MatmulArgs &a = ta.base;

@@ -183,7 +183,10 @@ def test_default_kernel_choice_by_m(nm):
     # three rows on for large ones; the threshold is adjustable
     assert nm.nm_debug_get_plan(2, 18432, 7168)["kind"] == 3
     assert nm.nm_debug_get_plan(3, 18432, 7168)["kind"] == 4
-    assert nm.nm_debug_get_plan(16, 576, 7168)["kind"] == 3
+    assert nm.nm_debug_get_plan(16, 576, 7168)["kind"] == 3          # 8 MB in one matrix: CUDA cores at every M
+    assert nm.nm_debug_get_plan(4, 1536, 7168)["kind"] == 4          # 22 MB: from M = 3 on
+    assert nm.nm_debug_get_plan(4, 512, 128, H=128)["kind"] == 4     # batched per-head products, 16.8 MB in all
+    assert nm.nm_debug_get_plan(2, 512, 128, H=128)["kind"] == 3
     nm.nm_set_tensor_core_min_m(17)
     try:
         assert nm.nm_debug_get_plan(16, 18432, 7168)["kind"] == 3

@@ -190,6 +190,26 @@ class MlaStep:
             del g
         except Exception as exc:          # capture is an extra; the main number does not depend on it
             out["graph_replay"] = {"error": repr(exc)}
+        # the small-batch step (nm_mla_decode_batch): T sequences of this length, one new token each
+        out["small_batch"] = []
+        dkv = DIMS["kv_lora"] + DIMS["rope"]
+        for T in (4, 16):
+            stride = (self.S + 8) * dkv
+            cache = self.t["kv_cache"].view(-1)[:self.S * dkv].repeat(T, 1)
+            cache = torch.nn.functional.pad(cache, (0, stride - self.S * dkv)).contiguous().view(-1)
+            h = self.t["h"].repeat(T)
+            cs = self.t["rope_cos_sin"].repeat(T)
+            res = torch.zeros(T * DIMS["d"], dtype=torch.int16, device=cache.device)
+            ws = self.nm.new_workspace(self.nm.nm_mla_batch_workspace_bytes(self.p, T), device=cache.device)
+            pb = self.nm.mla_params(DIMS, 1, self.t, workspace=ws)
+            b = self.nm.mla_batch([self.S] * T, h, cs, cache, stride, out=res)
+            fn = lambda: self.nm.nm_mla_decode_batch(pb, b, stream)
+            timed(fn, 20)
+            us = min(timed(fn, 100) for _ in range(3)) / 100 * 1e3
+            nb = self.bytes_per_step - self.kv_bytes + T * self.kv_bytes       # weights once, every sequence's cache rows
+            out["small_batch"].append({"T": T, "step_us": us, "us_per_token": us / T, "tokens_per_s": T / us * 1e6,
+                                       "GBps": nb / us / 1e3})
+            del cache, ws
         wo = self.p.W_O
         self.p.W_O = None
         try:

@@ -248,6 +248,38 @@ typedef struct {
 } nm_mla_params;
 
 size_t nm_mla_workspace_bytes(const nm_mla_params *p);
+
+/* Small-batch decode: the same step for T independent sequences at once, one new token each (the paper's "larger
+ * token" direction, Condition 5 of its last section, carried through the whole operator).  Every narrow product
+ * takes the T tokens as its M rows, so the weights are streamed once for all of them; the vector stages and the
+ * attention pass run per sequence inside shared launches.  Results are those of T single-token steps.
+ *   T            1..16
+ *   seq_lens     HOST array [T]: rows attended by sequence t including its new token (>= 1)
+ *   h            device [T][d] bf16
+ *   rope_cos_sin device [T][rope] fp32, row t for position seq_lens[t] - 1 (nm_rope_table)
+ *   kv_cache     device bf16; sequence t owns rows [0, seq_lens[t]) at kv_cache + t * cache_stride elements,
+ *                row width kv_lora + rope; row seq_lens[t] - 1 is written
+ *   cache_stride elements between the caches of consecutive sequences (multiple of 8, >= seq_lens[t] * row width)
+ *   out          device [T][d] bf16 (ignored when the params' W_O is NULL)
+ *   q_full, o_lat, o   optional device outputs [T][H][kv_lora+rope], [T][H][kv_lora], [T][H][v] bf16
+ * From nm_mla_params it takes the dimensions, weights, rms_eps, softmax_scale, layout_dense, workspace and
+ * workspace_bytes (>= nm_mla_batch_workspace_bytes(p, T)); its h, kv_cache, seq_len, rope_cos_sin, out and
+ * intermediates are ignored.  Dimensions: kv_lora 512, rope 64, nope 128, v 128, H 128.  One stream; the kernels
+ * are chained with programmatic dependent launch.  Errors as nm_mla_decode_step; nothing is enqueued on error
+ * except as noted there. */
+typedef struct nm_mla_batch {
+    int T;
+    const int *seq_lens;
+    const void *h;
+    const float *rope_cos_sin;
+    void *kv_cache;
+    long cache_stride;
+    void *out;
+    void *q_full, *o_lat, *o;
+} nm_mla_batch;
+
+size_t nm_mla_batch_workspace_bytes(const nm_mla_params *p, int T);
+int nm_mla_decode_batch(const nm_mla_params *p, const nm_mla_batch *b, nm_stream main_stream);
 int nm_mla_decode_step(const nm_mla_params *p, nm_stream main_stream, nm_stream side_stream);
 /* The same step with the token and the result in HOST memory (pinned): copies h in and out back
  * on main_stream around the step.  h_staging / out_staging are device buffers of d bf16 each. */

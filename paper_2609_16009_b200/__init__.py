@@ -77,6 +77,15 @@ class MlaParams(C.Structure):
                 + [("programmatic_entry", _i), ("W_DQKV", _vp)])
 
 
+class MlaBatch(C.Structure):
+    """Mirror of nm_mla_batch (include/nm.h)."""
+    _fields_ = [("T", _i), ("seq_lens", C.POINTER(_i)), ("h", _vp), ("rope_cos_sin", _vp), ("kv_cache", _vp),
+                ("cache_stride", C.c_long), ("out", _vp), ("q_full", _vp), ("o_lat", _vp), ("o", _vp)]
+
+
+_lib.nm_mla_batch_workspace_bytes.restype = _sz
+_lib.nm_mla_batch_workspace_bytes.argtypes = [C.POINTER(MlaParams), _i]
+_lib.nm_mla_decode_batch.argtypes = [C.POINTER(MlaParams), C.POINTER(MlaBatch), _vp]
 _lib.nm_rmsnorm.argtypes = [_vp, _vp, _vp, _i, C.c_float, _vp]
 _lib.nm_rope.argtypes = [_vp, _vp, _i, _i, _l, _l, _vp, _vp]
 _lib.nm_rope_table.argtypes = [_vp, _l, _i, _i, C.c_double, _vp]
@@ -287,6 +296,26 @@ def nm_mla_decode_step(p: MlaParams, main_stream=None, side_stream=None) -> None
     ms = _stream(main_stream)
     ss = ms if side_stream is None else _stream(side_stream)
     _check(_lib.nm_mla_decode_step(C.byref(p), ms, ss), "nm_mla_decode_step")
+
+
+def nm_mla_batch_workspace_bytes(p: MlaParams, T: int) -> int:
+    return int(_lib.nm_mla_batch_workspace_bytes(C.byref(p), int(T)))
+
+
+def mla_batch(seq_lens, h, rope_cos_sin, kv_cache, cache_stride, out=None, q_full=None, o_lat=None, o=None) -> MlaBatch:
+    """Fill an nm_mla_batch; seq_lens is a host sequence of ints (kept alive by the returned object)."""
+    b = MlaBatch()
+    b.T = len(seq_lens)
+    b._seq_lens = (_i * b.T)(*[int(x) for x in seq_lens])
+    b.seq_lens = C.cast(b._seq_lens, C.POINTER(_i))
+    b.h, b.rope_cos_sin, b.kv_cache = _ptr(h), _ptr(rope_cos_sin), _ptr(kv_cache)
+    b.cache_stride = int(cache_stride)
+    b.out, b.q_full, b.o_lat, b.o = _ptr(out), _ptr(q_full), _ptr(o_lat), _ptr(o)
+    return b
+
+
+def nm_mla_decode_batch(p: MlaParams, b: MlaBatch, main_stream=None) -> None:
+    _check(_lib.nm_mla_decode_batch(C.byref(p), C.byref(b), _stream(main_stream)), "nm_mla_decode_batch")
 
 
 def nm_mla_decode_step_host(p: MlaParams, h_host, out_host, h_staging, out_staging, main_stream=None,

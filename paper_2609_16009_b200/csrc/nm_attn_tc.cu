@@ -57,6 +57,14 @@ constexpr float kLazyThreshold = 8.0f;    // log2 units
 constexpr int kCl = kAttnCluster;          // CTAs (splits) per cluster
 constexpr int kHeadsPerRank = kHeads / kCl;
 
+// Per-sequence arguments of one launch (blockIdx.z selects the sequence; a single-sequence call fills entry 0).
+struct AttnSeqs {
+    CUtensorMap kv[kMaxBatch];
+    int n_rows[kMaxBatch];
+    int rows_per_split[kMaxBatch];
+    long ml_stride, o_stride;             // floats between the partials of consecutive sequences
+};
+
 __device__ __forceinline__ float fast_exp2(float x)
 {
     float y;
@@ -97,13 +105,18 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 
 // at most 120 registers per thread: leaves room on the SM for a CTA of the merge kernel that follows
 __global__ void __maxnreg__(120)
-attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, AttnPartials part,
-               int n_rows, int rows_per_split, float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
+attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ AttnSeqs seqs, AttnPartials part,
+               float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
 {
+    const int seq = blockIdx.z;
+    const CUtensorMap *map_kv_p = &seqs.kv[seq];
+    const int n_rows = seqs.n_rows[seq], rows_per_split = seqs.rows_per_split[seq];
+    part.ml += (size_t)seq * seqs.ml_stride;
+    part.O += (size_t)seq * seqs.o_stride;
     // Optional phase timestamps (ns) of CTA (0,0), for tuning: trace[i] is written when non-null.
-#define NM_TRACE(i) do { if (trace && blockIdx.x == 0 && blockIdx.y == 0) trace[i] = global_timer_ns(); } while (0)
+#define NM_TRACE(i) do { if (trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) trace[i] = global_timer_ns(); } while (0)
     // ... and four stamps of every CTA (start, Q landed, last P*V done, end) from trace[32] on
-#define NM_TRACE_CTA(i) do { if (trace) trace[32 + 4 * (blockIdx.y * gridDim.x + blockIdx.x) + (i)] = global_timer_ns(); } while (0)
+#define NM_TRACE_CTA(i) do { if (trace && blockIdx.z == 0) trace[32 + 4 * (blockIdx.y * gridDim.x + blockIdx.x) + (i)] = global_timer_ns(); } while (0)
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;            // swizzle atoms want 1024-byte alignment
@@ -159,8 +172,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const long block_chunks = (pf.block_bytes + kChunk - 1) / kChunk;
         const long chunks_per_range = (pf.range_bytes + kChunk - 1) / kChunk;
         const long total = block_chunks + chunks_per_range * pf.nranges;
-        const long nthreads = (long)gridDim.x * gridDim.y * 32;
-        const long me = ((long)blockIdx.y * gridDim.x + blockIdx.x) * 32 + lane;
+        const long nthreads = (long)gridDim.x * gridDim.y * gridDim.z * 32;
+        const long me = (((long)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 32 + lane;
         for (long i = me; i < total; i += nthreads) {
             const char *ptr;
             long n;
@@ -181,13 +194,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // ---------------- TMA producer --------------------------------------------------------------
         if (lane == 0) {
             tma_prefetch_descriptor(&map_q);
-            tma_prefetch_descriptor(&map_kv);
+            tma_prefetch_descriptor(map_kv_p);
             const uint64_t keep = l2_policy_evict_last(), stream = l2_policy_evict_first();
             auto load_tile = [&](int t) {
                 const int b = t & 1;
                 mbar_arrive_expect_tx(bar_kv_full + 8 * b, kKVBytes);
                 for (int c = 0; c < kKBlocks; ++c)
-                    tma_load_2d(kv_addr + b * kKVBytes + c * kKVBlockBytes, &map_kv, c * 64, r0 + t * kT, bar_kv_full + 8 * b, stream);
+                    tma_load_2d(kv_addr + b * kKVBytes + c * kKVBlockBytes, map_kv_p, c * 64, r0 + t * kT, bar_kv_full + 8 * b, stream);
             };
             // The cache rows were written by earlier steps, not by the kernels just before this one:
             // fetch the first two tiles before waiting for those kernels, then fetch Q, which they produce.
@@ -197,11 +210,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             // (a few hundred KB), so that every later tile load is an L2 hit.
             if (half == 0)
                 for (int t = kKVStages; t < ntiles; ++t)
-                    for (int c = 0; c < kKBlocks; ++c) tma_prefetch_l2_2d(&map_kv, c * 64, r0 + t * kT);
+                    for (int c = 0; c < kKBlocks; ++c) tma_prefetch_l2_2d(map_kv_p, c * 64, r0 + t * kT);
             pdl_wait_prior_grids();
             if (ntiles > 0) {                                      // a padding CTA of the last cluster loads nothing
                 mbar_arrive_expect_tx(bar_q, kQBytes);
-                for (int c = 0; c < kKBlocks; ++c) tma_load_2d(q_addr + c * kQBlockBytes, &map_q, c * 64, 0, bar_q, keep);
+                for (int c = 0; c < kKBlocks; ++c) tma_load_2d(q_addr + c * kQBlockBytes, &map_q, c * 64, seq * kHeads, bar_q, keep);
             }
             for (int t = kKVStages; t < ntiles; ++t) {             // stage b is free once the P*V of tile t-2 is done
                 const uint32_t bar = bar_pv_done + 8 * (t & 1), par = ((t - kKVStages) >> 1) & 1;
@@ -518,15 +531,29 @@ static unsigned long long *g_attn_trace = nullptr;
 void set_attention_trace(unsigned long long *p) { g_attn_trace = p; }
 unsigned long long *attention_trace() { return g_attn_trace; }
 
-int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows, float scale,
-                         cudaStream_t stream, bool programmatic_launch, L2Prefetch prefetch)
+static int launch_attn_tc(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split, int nsplit,
+                          AttnPartials part, long ml_stride, long o_stride, float scale, cudaStream_t stream, bool programmatic_launch,
+                          L2Prefetch prefetch)
 {
-    if (n_rows < 1 || plan.nsplit < 1) return NM_ERR_UNSUPPORTED;
-    if (((uintptr_t)Q & 15u) || ((uintptr_t)cache & 15u)) return NM_ERR_UNSUPPORTED;
-    CUtensorMap map_q, map_kv;
-    // The cache map covers exactly the rows attended: rows past n_rows read as zeros (and are masked),
-    // whatever the rest of the buffer holds.
-    if (!encode_rows_map(&map_q, Q, kHeads, kHeads) || !encode_rows_map(&map_kv, cache, n_rows, kT)) return NM_ERR_UNSUPPORTED;
+    if (nseq < 1 || nseq > kMaxBatch || nsplit < 1) return NM_ERR_UNSUPPORTED;
+    if ((uintptr_t)Q & 15u) return NM_ERR_UNSUPPORTED;
+    CUtensorMap map_q;
+    AttnSeqs seqs{};
+    seqs.ml_stride = ml_stride; seqs.o_stride = o_stride;
+    if (!encode_rows_map(&map_q, Q, nseq * kHeads, kHeads)) return NM_ERR_UNSUPPORTED;
+    for (int t = 0; t < nseq; ++t) {
+        seqs.n_rows[t] = n_rows[t];
+        seqs.rows_per_split[t] = rows_per_split[t];
+        if (n_rows[t] < 1) {                                       // nothing to attend: its CTAs find no tiles and load nothing
+            seqs.kv[t] = map_q;
+            seqs.rows_per_split[t] = kT;
+            continue;
+        }
+        if ((uintptr_t)caches[t] & 15u) return NM_ERR_UNSUPPORTED;
+        // The cache map covers exactly the rows attended: rows past n_rows read as zeros (and are masked),
+        // whatever the rest of the buffer holds.
+        if (!encode_rows_map(&seqs.kv[t], caches[t], n_rows[t], kT)) return NM_ERR_UNSUPPORTED;
+    }
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -535,7 +562,7 @@ int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, At
     }
     const float scale_log2 = scale * 1.4426950408889634f;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ceil_div(plan.nsplit, kCl) * kCl, 2);      // padded to whole clusters; padding CTAs have no rows
+    cfg.gridDim = dim3(ceil_div(nsplit, kCl) * kCl, 2, nseq);      // padded to whole clusters; padding CTAs have no rows
     // the prefetch warp is launched only when there is something to prefetch (fewer registers held on the SM)
     const bool has_prefetch = prefetch.block_bytes > 0 || (prefetch.nranges > 0 && prefetch.range_bytes > 0);
     cfg.blockDim = dim3(has_prefetch ? kThreads : kThreads - 32);
@@ -548,9 +575,23 @@ int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, At
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = programmatic_launch ? 2 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, map_q, map_kv, part, n_rows, plan.rows_per_split, scale_log2,
-                                       device_status_ptr(), g_attn_trace, prefetch);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, map_q, seqs, part, scale_log2, device_status_ptr(), g_attn_trace, prefetch);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (tensor cores) launch");
+}
+
+int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows, float scale,
+                         cudaStream_t stream, bool programmatic_launch, L2Prefetch prefetch)
+{
+    if (n_rows < 1 || plan.nsplit < 1) return NM_ERR_UNSUPPORTED;
+    return launch_attn_tc(Q, 1, &cache, &n_rows, &plan.rows_per_split, plan.nsplit, part, 0, 0, scale, stream, programmatic_launch, prefetch);
+}
+
+int attention_partial_tc_batch(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split,
+                               int nsplit, AttnPartials part, int slot_stride, float scale, cudaStream_t stream,
+                               bool programmatic_launch)
+{
+    return launch_attn_tc(Q, nseq, caches, n_rows, rows_per_split, nsplit, part, (long)slot_stride * kHeads * 2,
+                          (long)slot_stride * kHeads * kDv, scale, stream, programmatic_launch, L2Prefetch{});
 }
 
 }  // namespace nm

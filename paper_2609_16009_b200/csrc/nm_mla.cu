@@ -599,6 +599,122 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     return NM_OK;
 }
 
+// ---- small-batch decode: T independent sequences, one new token each ------------------------------------------
+struct BatchLayout {
+    size_t mws, mws_bytes, attn_ml, attn_o, x_down, c_qn, q, q_full, o_lat, o, total;
+    int slot_stride;
+};
+
+static BatchLayout batch_layout(const nm_mla_params *p, int T)
+{
+    BatchLayout L{};
+    const int dq = p->nope + p->rope, dkv = p->kv_lora + p->rope, H = p->H;
+    size_t need = 0;
+    auto upd = [&](int N, int K) {
+        const size_t b = nm_matmul_workspace_bytes(T, N, K, 1, NM_BF16, NM_ROW_MAJOR);
+        if (b > need) need = b;
+    };
+    upd(p->q_lora + dkv, p->d); upd(p->q_lora, p->d); upd(dkv, p->d); upd(H * dq, p->q_lora); upd(p->d, H * p->v);
+    size_t off = 0;
+    L.mws = off; L.mws_bytes = need; off += align_up(need, 256);
+    L.slot_stride = 16;                                            // at most 64 splits in clusters of four per sequence
+    L.attn_ml = off; off += align_up((size_t)T * L.slot_stride * H * 2 * sizeof(float), 256);
+    L.attn_o = off; off += align_up((size_t)T * L.slot_stride * H * p->kv_lora * sizeof(float), 256);
+    auto take = [&](size_t elems) { size_t o = off; off += align_up(elems * 2, 256); return o; };
+    L.x_down = take((size_t)T * (p->q_lora + dkv)); L.c_qn = take((size_t)T * p->q_lora); L.q = take((size_t)T * H * dq);
+    L.q_full = take((size_t)T * H * dkv); L.o_lat = take((size_t)T * H * p->kv_lora); L.o = take((size_t)T * H * p->v);
+    L.total = off;
+    return L;
+}
+
+static int batch_check(const nm_mla_params *p, const nm_mla_batch *b)
+{
+    if (!p || !b) return NM_ERR_INVALID_ARG;
+    if (b->T < 1 || !b->seq_lens || !b->h || !b->rope_cos_sin || !b->kv_cache) return NM_ERR_INVALID_ARG;
+    if (b->T > kMaxBatch) return NM_ERR_UNSUPPORTED;
+    if (!p->gamma_q || !p->W_UQR || !p->gamma_kv || !p->W_UK || !p->W_UV || !p->workspace) return NM_ERR_INVALID_ARG;
+    if (!p->W_DQKV && (!p->W_DQ || !p->W_DKVKR)) return NM_ERR_INVALID_ARG;
+    if (p->W_O && !b->out) return NM_ERR_INVALID_ARG;
+    if (p->d < 1 || p->q_lora < 1 || p->H < 1) return NM_ERR_INVALID_ARG;
+    if (p->kv_lora != 512 || p->rope != 64 || p->nope != 128 || p->v != 128 || p->H != 128) return NM_ERR_UNSUPPORTED;
+    if (!down_finish_applies(p->q_lora, p->kv_lora, p->rope)) return NM_ERR_UNSUPPORTED;
+    if (p->layout_dense != NM_ROW_MAJOR && p->layout_dense != NM_COL_MAJOR) return NM_ERR_UNSUPPORTED;
+    const long row = p->kv_lora + p->rope;
+    for (int t = 0; t < b->T; ++t) {
+        if (b->seq_lens[t] < 1) return NM_ERR_INVALID_ARG;
+        if (b->T > 1 && b->cache_stride < (long)b->seq_lens[t] * row) return NM_ERR_INVALID_ARG;
+    }
+    if (b->cache_stride % 8 != 0) return NM_ERR_ALIGNMENT;           // every sequence's cache stays 16-byte aligned
+    return NM_OK;
+}
+
+static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_t ms)
+{
+    NM_TRY(batch_check(p, b));
+    const int T = b->T;
+    const BatchLayout L = batch_layout(p, T);
+    if (p->workspace_bytes < L.total) return NM_ERR_WORKSPACE;
+    if (((uintptr_t)p->workspace & 255u) != 0) return NM_ERR_ALIGNMENT;
+    char *ws = static_cast<char *>(p->workspace);
+    const int d = p->d, ql = p->q_lora, dc = p->kv_lora, dr = p->rope, dn = p->nope, dv = p->v, H = p->H;
+    const int dq = dn + dr, dkv = dc + dr;
+    const nm_layout lay = (nm_layout)p->layout_dense;
+    uint16_t *x_down = (uint16_t *)(ws + L.x_down), *c_qn = (uint16_t *)(ws + L.c_qn), *q = (uint16_t *)(ws + L.q);
+    uint16_t *q_full = (uint16_t *)(ws + L.q_full), *o_lat = (uint16_t *)(ws + L.o_lat), *o = (uint16_t *)(ws + L.o);
+    uint16_t *cache = static_cast<uint16_t *>(b->kv_cache);
+    void *mws = ws + L.mws;
+    const bool pdl = g_step_pdl != 0;
+
+    // split plan of the attention pass: the same number of splits for every sequence, about 128 CTAs in all
+    int nsplit = (64 / T) / kAttnCluster * kAttnCluster;
+    if (nsplit < kAttnCluster) nsplit = kAttnCluster;
+    BatchRows rows{};
+    rows.slot_stride = L.slot_stride;
+    const void *caches[kMaxBatch];
+    int n_rows[kMaxBatch], rps[kMaxBatch];
+    bool any_rows = false;
+    for (int t = 0; t < T; ++t) {
+        const long base = (long)t * b->cache_stride;
+        caches[t] = cache + base;
+        n_rows[t] = b->seq_lens[t] - 1;
+        rows.new_row[t] = base + (long)n_rows[t] * dkv;
+        const int tiles = ceil_div(n_rows[t], kAttnTileRows);
+        rps[t] = tiles > 0 ? ceil_div(tiles, nsplit) * kAttnTileRows : kAttnTileRows;
+        rows.npart[t] = n_rows[t] > 0 ? ceil_div(ceil_div(n_rows[t], rps[t]), kAttnCluster) : 0;
+        any_rows |= n_rows[t] > 0;
+    }
+
+    // ---- down-projections of all T tokens: the weights are streamed once ---------------------------------------
+    if (p->W_DQKV && lay == NM_ROW_MAJOR) {
+        NM_TRY(matmul_enqueue(b->h, p->W_DQKV, x_down, T, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws, L.mws_bytes, ms,
+                              false, nullptr, nullptr, nullptr, true));
+    } else {
+        NM_TRY(matmul_enqueue(b->h, p->W_DQ, x_down, T, ql, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws, L.mws_bytes, ms,
+                              false, nullptr, nullptr, nullptr, true));
+        NM_TRY(matmul_enqueue(b->h, p->W_DKVKR, x_down + ql, T, dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws, L.mws_bytes, ms,
+                              pdl, nullptr, nullptr, nullptr, true));
+    }
+    NM_TRY(launch_down_finish_batch(x_down, p->gamma_q, p->gamma_kv, b->rope_cos_sin, c_qn, cache, rows, T, ql, dc, dr, p->rms_eps, ms, pdl));
+    NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, T, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.mws_bytes, ms, pdl, nullptr, nullptr,
+                          nullptr, true));
+    NM_TRY(launch_q_finish_batch(q, p->W_UK, b->rope_cos_sin, q_full, H, dr, T, ms, pdl));
+    AttnPartials part;
+    part.ml = reinterpret_cast<float *>(ws + L.attn_ml);
+    part.O = reinterpret_cast<float *>(ws + L.attn_o);
+    if (any_rows) {
+        if (tensor_map_encoder() == nullptr) return NM_ERR_UNSUPPORTED;
+        NM_TRY(attention_partial_tc_batch(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl));
+    }
+    NM_TRY(launch_uv_merge_batch(q_full, cache, part, rows, T, dr, p->softmax_scale, p->W_UV, o_lat, o, H, ms, pdl));
+    if (p->W_O)
+        NM_TRY(matmul_enqueue(o, p->W_O, b->out, T, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.mws_bytes, ms, pdl, nullptr,
+                              nullptr, nullptr, true));
+    if (b->o_lat) NM_CUDA_TRY(cudaMemcpyAsync(b->o_lat, o_lat, (size_t)T * H * dc * 2, cudaMemcpyDeviceToDevice, ms));
+    if (b->o) NM_CUDA_TRY(cudaMemcpyAsync(b->o, o, (size_t)T * H * dv * 2, cudaMemcpyDeviceToDevice, ms));
+    if (b->q_full) NM_CUDA_TRY(cudaMemcpyAsync(b->q_full, q_full, (size_t)T * H * dkv * 2, cudaMemcpyDeviceToDevice, ms));
+    return NM_OK;
+}
+
 }  // namespace nm
 
 using namespace nm;
@@ -665,6 +781,17 @@ size_t nm_mla_workspace_bytes(const nm_mla_params *p)
 {
     if (!p || p->H < 1 || p->d < 1 || p->q_lora < 1) return 0;
     return step_layout(p).total;
+}
+
+size_t nm_mla_batch_workspace_bytes(const nm_mla_params *p, int T)
+{
+    if (!p || T < 1 || T > kMaxBatch) return 0;
+    return batch_layout(p, T).total;
+}
+
+int nm_mla_decode_batch(const nm_mla_params *p, const nm_mla_batch *b, nm_stream main_stream)
+{
+    return batch_impl(p, b, (cudaStream_t)main_stream);
 }
 
 int nm_mla_decode_step(const nm_mla_params *p, nm_stream main_stream, nm_stream side_stream)

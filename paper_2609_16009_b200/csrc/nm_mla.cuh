@@ -41,6 +41,14 @@ struct L2Prefetch {
 int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, AttnPlan plan, int n_rows,
                          float scale, cudaStream_t stream, bool programmatic_launch, L2Prefetch prefetch);
 
+// The same pass over several independent sequences in one launch (small-batch decode): sequence t has its own
+// cache rows, row count and split plan; its queries are rows [128 t, 128 t + 128) of Q, its partials start
+// slot_stride slots after those of sequence t - 1.  All sequences use the same number of splits.
+constexpr int kMaxBatch = 16;
+int attention_partial_tc_batch(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split,
+                               int nsplit, AttnPartials part, int slot_stride, float scale, cudaStream_t stream,
+                               bool programmatic_launch);
+
 // Fused per-head stages of the decode step (nm_head_kernels.cu); they take nope = 128, kv_lora = 512, v = 128.
 bool head_kernels_apply(int H, int nope, int rope, int dc, int dv);
 bool down_finish_applies(int q_lora, int dc, int rope);
@@ -50,6 +58,18 @@ int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void 
 int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
                     const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl,
                     L2Prefetch prefetch = L2Prefetch{});
+
+// Small-batch decode (nm_batch_kernels.cu): per-sequence rows and partial counts of one launch.
+struct BatchRows {
+    long new_row[kMaxBatch];             // element offset, from the cache base, of the row each sequence's step writes
+    int npart[kMaxBatch];                // attention partials to merge for each sequence
+    int slot_stride;                     // partial slots between consecutive sequences
+};
+int launch_down_finish_batch(const void *x, const void *gamma_q, const void *gamma_kv, const float *cos_sin, void *c_qn, void *cache,
+                             const BatchRows &rows, int T, int q_lora, int dc, int rope, float eps, cudaStream_t s, bool pdl);
+int launch_q_finish_batch(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, int T, cudaStream_t s, bool pdl);
+int launch_uv_merge_batch(const void *Q, const void *cache, AttnPartials part, const BatchRows &rows, int T, int rope, float scale,
+                          const void *W_UV, void *o_lat_bf16, void *o, int H, cudaStream_t s, bool pdl);
 
 // Tuning aid: phase timestamps (ns) of the tensor-core kernel go to `p` when non-null: 32 slots for CTA (0,0),
 // then four per CTA (start, Q landed, last P*V done, end); 32 + 4 * 256 values at most.

@@ -1,0 +1,144 @@
+"""Small-batch decode (nm_mla_decode_batch): T independent sequences, one new token each, against T runs of
+the oracle's single-token step, and against the library's own single-token step."""
+import numpy as np
+import pytest
+import torch
+
+import nm_inputs as gen
+import oracle
+from gpu_util import to_dev
+
+pytestmark = pytest.mark.gpu
+DIMS = gen.DSV3_DIMS
+
+
+def f64(bits):
+    return oracle.bf16_to_f64(np.asarray(bits, dtype=np.uint16))
+
+
+def dev_bits_to_f64(t):
+    return oracle.bf16_to_f64(t.contiguous().cpu().numpy().view(np.uint16))
+
+
+@pytest.fixture(scope="module")
+def nm():
+    import paper_2609_16009_b200 as nm
+    yield nm
+    nm.nm_check_status()
+
+
+@pytest.fixture(scope="module")
+def weights():
+    w = gen.mla_weights(DIMS, seed=4000, with_wo=True)
+    return w, {k: to_dev(v) for k, v in w.items()}
+
+
+def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True):
+    H, dc, dr, dn, dv, d, ql = (DIMS[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d", "q_lora"))
+    dkv = dc + dr
+    T = len(seq_lens)
+    t = dict(dw)
+    if not with_wo:
+        t.pop("W_O")
+    if concat_down:
+        t["W_DQKV"] = torch.cat([t.pop("W_DQ").view(d, ql), t.pop("W_DKVKR").view(d, dkv)], dim=1).contiguous().view(-1)
+    stride = (max(seq_lens) + 3) * dkv                      # a few spare rows between the sequences' caches
+    stride += (-stride) % 8
+    cache = torch.zeros(T * stride, dtype=torch.int16, device="cuda")
+    for i, c in enumerate(caches):
+        cache[i * stride:i * stride + c.size] = to_dev(c).view(-1)
+    h = to_dev(np.stack(tokens))
+    cs = torch.empty(T, dr, dtype=torch.float32, device="cuda")
+    for i, S in enumerate(seq_lens):
+        nm.nm_rope_table(cs[i], S - 1, 1, dr)
+    out = torch.zeros(T * d, dtype=torch.int16, device="cuda")
+    q_full = torch.zeros(T * H * dkv, dtype=torch.int16, device="cuda")
+    o_lat = torch.zeros(T * H * dc, dtype=torch.int16, device="cuda")
+    o = torch.zeros(T * H * dv, dtype=torch.int16, device="cuda")
+    p = nm.mla_params(DIMS, 1, t)
+    ws = nm.new_workspace(nm.nm_mla_batch_workspace_bytes(p, T))
+    p = nm.mla_params(DIMS, 1, t, workspace=ws)
+    b = nm.mla_batch(seq_lens, h, cs, cache, stride, out=out, q_full=q_full, o_lat=o_lat, o=o)
+    st = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    nm.nm_mla_decode_batch(p, b, st)
+    torch.cuda.synchronize()
+    nm.nm_check_status()
+    return {"out": out.view(T, d), "q_full": q_full.view(T, H, dkv), "o_lat": o_lat.view(T, H, dc), "o": o.view(T, H * dv),
+            "cache": cache.view(T, stride), "stride": stride}
+
+
+def rel_max(got, ref):
+    return np.abs(got - ref).max() / np.abs(ref).max()
+
+
+def check_against_oracle(w, res, tokens, caches, seq_lens, with_wo=True):
+    H, dc, dr = DIMS["H"], DIMS["kv_lora"], DIMS["rope"]
+    dkv = dc + dr
+    ww = dict(w)
+    if not with_wo:
+        ww.pop("W_O", None)
+    for i, S in enumerate(seq_lens):
+        r = oracle.mla_decode_step(DIMS, ww, tokens[i], caches[i], S, threads=8)
+        cache_ref = caches[i]                                # the oracle wrote row S-1 in place
+        got = res["cache"][i].cpu().numpy().view(np.uint16)[:S * dkv].reshape(S, dkv)
+        assert np.array_equal(got[:S - 1], cache_ref[:S - 1]), f"sequence {i}: old rows changed"
+        assert np.all(np.abs(f64(got[S - 1]) - f64(cache_ref[S - 1])) <= 2 * oracle.ulp_bf16(f64(cache_ref[S - 1])) + 1e-6), i
+        qf = dev_bits_to_f64(res["q_full"][i]).reshape(H, dkv)
+        assert rel_max(qf[:, :dc], f64(r["q_lat"])) <= 1e-2 and rel_max(qf[:, dc:], f64(r["q_rope"])) <= 1e-2, i
+        names = [("o_lat", r["o_lat"]), ("o", r["o"])] + ([("out", r["out"])] if with_wo else [])
+        for name, ref_bits in names:
+            g, ref = dev_bits_to_f64(res[name][i]).reshape(-1), f64(ref_bits).reshape(-1)
+            assert np.all(np.abs(g - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref)), f"sequence {i}: {name}"
+
+
+def make_inputs(seq_lens, seed):
+    tokens = [gen.mla_token(DIMS, seed=seed + 10 * i) for i in range(len(seq_lens))]
+    caches = [gen.mla_cache(S, DIMS, seed=seed + 10 * i + 1) for i, S in enumerate(seq_lens)]
+    return tokens, caches
+
+
+@pytest.mark.parametrize("seq_lens,concat", [([300], True), ([1, 70], True), ([1024, 65, 2, 500], True), ([129, 64, 1000], False),
+                                             ([200, 1, 333, 64, 65, 1500, 2, 700], True)])
+def test_batch_matches_oracle(nm, weights, seq_lens, concat):
+    w, dw = weights
+    tokens, caches = make_inputs(seq_lens, seed=8000 + len(seq_lens))
+    res = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, concat)
+    check_against_oracle(w, res, tokens, caches, seq_lens)
+
+
+def test_batch_of_sixteen_without_wo(nm, weights):
+    w, dw = weights
+    seq_lens = [40 + 37 * i for i in range(16)]
+    tokens, caches = make_inputs(seq_lens, seed=8100)
+    res = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True, with_wo=False)
+    check_against_oracle(w, res, tokens, caches, seq_lens, with_wo=False)
+
+
+def test_batch_is_repeatable_and_rejects_bad_arguments(nm, weights):
+    w, dw = weights
+    seq_lens = [100, 257]
+    tokens, caches = make_inputs(seq_lens, seed=8200)
+    a = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True)
+    b = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True)
+    for k in ("out", "o", "o_lat", "q_full"):
+        assert torch.equal(a[k], b[k]), k
+    t = dict(dw)
+    p = nm.mla_params(DIMS, 1, t)
+    ws = nm.new_workspace(nm.nm_mla_batch_workspace_bytes(p, 2))
+    p = nm.mla_params(DIMS, 1, t, workspace=ws)
+    dkv = DIMS["kv_lora"] + DIMS["rope"]
+    cache = torch.zeros(2 * 300 * dkv, dtype=torch.int16, device="cuda")
+    h = torch.zeros(2 * DIMS["d"], dtype=torch.int16, device="cuda")
+    cs = torch.zeros(2 * DIMS["rope"], dtype=torch.float32, device="cuda")
+    out = torch.zeros(2 * DIMS["d"], dtype=torch.int16, device="cuda")
+    with pytest.raises(nm.NmError):                          # cache stride smaller than a sequence
+        nm.nm_mla_decode_batch(p, nm.mla_batch([100, 257], h, cs, cache, 200 * dkv, out=out))
+    with pytest.raises(nm.NmError):                          # empty sequence
+        nm.nm_mla_decode_batch(p, nm.mla_batch([100, 0], h, cs, cache, 300 * dkv, out=out))
+    with pytest.raises(nm.NmError):                          # more sequences than the library takes
+        nm.nm_mla_decode_batch(p, nm.mla_batch([5] * 17, h, cs, cache, 8 * dkv, out=out))
+    small = nm.new_workspace(1 << 20)
+    p2 = nm.mla_params(DIMS, 1, t, workspace=small)
+    with pytest.raises(nm.NmError):                          # workspace too small
+        nm.nm_mla_decode_batch(p2, nm.mla_batch([100, 257], h, cs, cache, 300 * dkv, out=out))

@@ -310,7 +310,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
         ta.trace = trace;
         if (tail && tail->enabled && M == 1 && dtype == NM_BF16 && H == 1 && ws && ws_bytes >= kCounterBytes && aligned16(ws) &&
-            p.ntiles < kNumCounters - 1 && N <= 4096) {
+            p.ntiles < kNumCounters - 1 && N <= 4096 && N % 4 == 0 && p.tn % 4 == 0 && ldc % 4 == 0 && ((uintptr_t)C & 7u) == 0) {
             ta.tail = *tail;
             ta.tail.counter = reinterpret_cast<unsigned *>(ws) + (kNumCounters - 1);     // the last counter is never a tile's
             if (tail_taken) *tail_taken = true;

@@ -127,7 +127,8 @@ __device__ __forceinline__ void vec_tail_run(const VecTail &t, const float *xs, 
 // the finished bf16 columns) and arrives; the last CTA of the grid gathers every column - partials summed in
 // split order, rounded once - writes C, keeps the rounded row in shared memory and runs the vector stages on
 // it.  One fence / atomic / load round trip through L2 in all, where a per-tile gather followed by a grid-wide
-// counter would take two.  `xs` needs N floats (+32 of scratch behind them).
+// counter would take two (each such round trip costs 1-3 us here: the next product of the chain is filling its
+// ring from HBM at full rate at that very moment, and everything that crosses L2 queues behind it).  `xs` needs N floats (+32 of scratch behind them).
 __device__ __forceinline__ void tail_complete(const MatmulArgs &a, const VecTail &t, int *s_last, float *xs)
 {
     const int tid = threadIdx.x;
@@ -139,37 +140,30 @@ __device__ __forceinline__ void tail_complete(const MatmulArgs &a, const VecTail
     __threadfence();
     if (tid == 0) *t.counter = 0u;
     uint16_t *C = reinterpret_cast<uint16_t *>(a.C);
-    // eight columns per thread and pass, all their partials requested before the first is used
-    constexpr int kCols = 8;
-    for (int n0 = 0; n0 < a.N; n0 += kCols * blockDim.x) {
-        float s[kCols];
-        const float *P[kCols];
-#pragma unroll
-        for (int j = 0; j < kCols; ++j) {
-            const int n = min(n0 + j * (int)blockDim.x + tid, a.N - 1);
-            const int tile = n / a.tn, c = n - tile * a.tn;
-            P[j] = a.partial + (size_t)tile * a.nsplit * a.tn + c;
-            s[j] = 0.f;
-        }
+    // four consecutive columns (one 16-byte load per split) per thread and pass; N and the tile width are
+    // multiples of four (checked by the host), so the four columns lie in one tile
+    for (int n = 4 * tid; n < a.N; n += 4 * (int)blockDim.x) {
+        float4 sum;
         if (a.nsplit > 1) {
+            const int tile = n / a.tn, c = n - tile * a.tn;
+            const float *P = a.partial + (size_t)tile * a.nsplit * a.tn + c;
+            sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
-            for (int sp = 0; sp < a.nsplit; ++sp)
-#pragma unroll
-                for (int j = 0; j < kCols; ++j) s[j] += ld_cg(P[j] + (size_t)sp * a.tn);
-        }
-#pragma unroll
-        for (int j = 0; j < kCols; ++j) {
-            const int n = n0 + j * (int)blockDim.x + tid;
-            if (n < a.N) {
-                if (a.nsplit > 1) {
-                    const __nv_bfloat16 b = __float2bfloat16_rn(s[j]);
-                    C[n] = __bfloat16_as_ushort(b);
-                    xs[n] = __bfloat162float(b);
-                } else {
-                    xs[n] = __uint_as_float((uint32_t)__ldcg(C + n) << 16);
-                }
+            for (int sp = 0; sp < a.nsplit; ++sp) {               // split order: deterministic
+                const float4 v = __ldcg(reinterpret_cast<const float4 *>(P + (size_t)sp * a.tn));
+                sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
             }
+            const __nv_bfloat16 b0 = __float2bfloat16_rn(sum.x), b1 = __float2bfloat16_rn(sum.y), b2 = __float2bfloat16_rn(sum.z),
+                                b3 = __float2bfloat16_rn(sum.w);
+            *reinterpret_cast<uint2 *>(C + n) = make_uint2((uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16),
+                                                           (uint32_t)__bfloat16_as_ushort(b2) | ((uint32_t)__bfloat16_as_ushort(b3) << 16));
+            sum = make_float4(__bfloat162float(b0), __bfloat162float(b1), __bfloat162float(b2), __bfloat162float(b3));
+        } else {
+            const uint2 cv = __ldcg(reinterpret_cast<const uint2 *>(C + n));
+            sum = make_float4(__uint_as_float(cv.x << 16), __uint_as_float(cv.x & 0xffff0000u), __uint_as_float(cv.y << 16),
+                              __uint_as_float(cv.y & 0xffff0000u));
         }
+        *reinterpret_cast<float4 *>(xs + n) = sum;
     }
     __syncthreads();
     vec_tail_run(t, xs, xs + ((a.N + 31) & ~31));

@@ -29,42 +29,6 @@ __device__ __forceinline__ float block_sum(float v, float *scratch)
     return t;
 }
 
-// y[0..N) = x[0..K) * W[K][N] with this thread's 32 weight vectors in `w` (rows ty + i * kRowGroups, eight
-// columns from 8 tx): partial sums to shared memory, row groups added in a fixed order by the threads with
-// ty == 0, which get the eight column sums in out8.
-template <int K, int N>
-__device__ __forceinline__ void head_matvec(const uint4 (&w)[32], const float *x_s, float *red, float (&out8)[8])
-{
-    constexpr int kColGroups = N / 8, kRowGroups = kThreadsB / kColGroups;
-    static_assert(K / kRowGroups == 32, "128x512 or 512x128");
-    const int tx = threadIdx.x % kColGroups, ty = threadIdx.x / kColGroups;
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        float b[8];
-        Elem<bf16_t>::unpack(w[i], b);
-        const float a = x_s[ty + i * kRowGroups];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = fmaf(a, b[j], acc[j]);
-    }
-    float4 *dst = reinterpret_cast<float4 *>(red + (size_t)ty * N + tx * 8);
-    dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
-    __syncthreads();
-    if (ty == 0) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) out8[j] = 0.f;
-        for (int g = 0; g < kRowGroups; ++g) {
-            const float4 *src = reinterpret_cast<const float4 *>(red + (size_t)g * N + tx * 8);
-            const float4 v0 = src[0], v1 = src[1];
-            out8[0] += v0.x; out8[1] += v0.y; out8[2] += v0.z; out8[3] += v0.w;
-            out8[4] += v1.x; out8[5] += v1.y; out8[6] += v1.z; out8[7] += v1.w;
-        }
-    }
-}
-
 // RMSNorm of the query latent (CTA x = 0) and RMSNorm + RoPE + cache-row write of the KV part (CTA x = 1) of
 // token blockIdx.y.  x: [T][q_lora + dc + rope] as the down-projection wrote it.
 __global__ void __launch_bounds__(kThreadsB) down_finish_batch_kernel(const uint16_t *__restrict__ x, const uint16_t *__restrict__ gamma_q,
@@ -121,14 +85,19 @@ __global__ void __launch_bounds__(kThreadsB) down_finish_batch_kernel(const uint
     }
 }
 
+constexpr int kTokGroup = 4;              // tokens whose products share one pass over the weights in registers
+
 // For head blockIdx.x and every token t: q_rope = RoPE(q[t, h, nope:]), q_lat = q[t, h, :nope] * W_UK[h].
 // q: [T][H][nope + rope]; q_full: [T][H][dc + rope] (q_lat | q_rope).  nope = 128, dc = 512.
+// All tokens' inputs are fetched at once; the product runs over groups of four tokens, each thread keeping four
+// accumulator sets for its 32 weight rows, so that the weights in registers are walked once per group and the
+// cross-row-group sums cost two barriers per group instead of per token.
 __global__ void __launch_bounds__(kThreadsB) q_finish_batch_kernel(const uint16_t *__restrict__ q, const uint16_t *__restrict__ W_UK,
                                                                    const float *__restrict__ cs, uint16_t *__restrict__ q_full, int rope, int T)
 {
-    constexpr int K = 128, N = 512, kColGroups = N / 8, kRowGroups = kThreadsB / kColGroups;
-    __shared__ __align__(16) float x_s[K];
-    __shared__ __align__(16) float red[kRowGroups * N];
+    constexpr int K = 128, N = 512, kColGroups = N / 8, kRowGroups = kThreadsB / kColGroups;      // 64 x 4
+    __shared__ __align__(16) float x_s[kMaxBatch][K];
+    __shared__ __align__(16) float red[kTokGroup][kRowGroups][N];
     const int h = blockIdx.x, H = gridDim.x, tid = threadIdx.x;
     const int tx = tid % kColGroups, ty = tid / kColGroups;
     const uint16_t *W = W_UK + (size_t)h * K * N + (size_t)ty * N + tx * 8;
@@ -137,41 +106,82 @@ __global__ void __launch_bounds__(kThreadsB) q_finish_batch_kernel(const uint16_
     for (int i = 0; i < 32; ++i) w[i] = ld_stream16(W + (size_t)i * kRowGroups * N);
     pdl_launch_dependents();
     pdl_wait_prior_grids();                                       // q comes from the W_UQR product
-    for (int t = 0; t < T; ++t) {
-        const uint16_t *qh = q + ((size_t)t * H + h) * (K + rope);
-        uint16_t *dst = q_full + ((size_t)t * H + h) * (N + rope);
-        if (tid < K) x_s[tid] = bf2f(qh[tid]);
-        if (tid < rope / 2) {
-            const float c = cs[(size_t)t * rope + 2 * tid], s = cs[(size_t)t * rope + 2 * tid + 1];
-            const float x0 = bf2f(qh[K + 2 * tid]), x1 = bf2f(qh[K + 2 * tid + 1]);
-            *reinterpret_cast<uint32_t *>(dst + N + 2 * tid) = pack2(x0 * c - x1 * s, x0 * s + x1 * c);
+    for (int i = tid; i < T * K; i += kThreadsB) {
+        const int t = i / K, k = i - t * K;
+        x_s[t][k] = bf2f(q[((size_t)t * H + h) * (K + rope) + k]);
+    }
+    for (int i = tid; i < T * (rope / 2); i += kThreadsB) {       // interleaved pairs, rounded to bf16
+        const int t = i / (rope / 2), pr = i - t * (rope / 2);
+        const uint16_t *qh = q + ((size_t)t * H + h) * (K + rope) + K;
+        const float c = cs[(size_t)t * rope + 2 * pr], sn = cs[(size_t)t * rope + 2 * pr + 1];
+        const float x0 = bf2f(qh[2 * pr]), x1 = bf2f(qh[2 * pr + 1]);
+        *reinterpret_cast<uint32_t *>(q_full + ((size_t)t * H + h) * (N + rope) + N + 2 * pr) = pack2(x0 * c - x1 * sn, x0 * sn + x1 * c);
+    }
+    __syncthreads();
+    for (int t0 = 0; t0 < T; t0 += kTokGroup) {
+        float acc[kTokGroup][8];
+#pragma unroll
+        for (int g = 0; g < kTokGroup; ++g)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            float b[8];
+            uint4 wi = w[i];
+            // keeps the widening of the weights inside the group loop: hoisted out of it, the 256 widened values
+            // of a thread would not fit its registers
+            asm volatile("" : "+r"(wi.x), "+r"(wi.y), "+r"(wi.z), "+r"(wi.w));
+            Elem<bf16_t>::unpack(wi, b);
+#pragma unroll
+            for (int g = 0; g < kTokGroup; ++g) {
+                const float a = x_s[min(t0 + g, kMaxBatch - 1)][ty + i * kRowGroups];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[g][j] = fmaf(a, b[j], acc[g][j]);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < kTokGroup; ++g) {
+            float4 *dst = reinterpret_cast<float4 *>(&red[g][ty][tx * 8]);
+            dst[0] = make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
+            dst[1] = make_float4(acc[g][4], acc[g][5], acc[g][6], acc[g][7]);
         }
         __syncthreads();
-        float out8[8];
-        head_matvec<K, N>(w, x_s, red, out8);
-        if (ty == 0) {
+        // thread (ty, tx) finishes token t0 + ty: eight columns, row groups added in a fixed order
+        if (t0 + ty < T) {
+            float out8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) out8[j] = 0.f;
+#pragma unroll
+            for (int g = 0; g < kRowGroups; ++g) {
+                const float4 *src = reinterpret_cast<const float4 *>(&red[ty][g][tx * 8]);
+                const float4 v0 = src[0], v1 = src[1];
+                out8[0] += v0.x; out8[1] += v0.y; out8[2] += v0.z; out8[3] += v0.w;
+                out8[4] += v1.x; out8[5] += v1.y; out8[6] += v1.z; out8[7] += v1.w;
+            }
             uint4 o;
             o.x = pack2(out8[0], out8[1]); o.y = pack2(out8[2], out8[3]); o.z = pack2(out8[4], out8[5]); o.w = pack2(out8[6], out8[7]);
-            *reinterpret_cast<uint4 *>(dst + tx * 8) = o;
+            *reinterpret_cast<uint4 *>(q_full + ((size_t)(t0 + ty) * H + h) * (N + rope) + tx * 8) = o;
         }
-        __syncthreads();                                           // x_s and red are reused by the next token
+        __syncthreads();                                           // red is reused by the next group
     }
 }
 
 // For head blockIdx.x and every token t: log-sum-exp merge of the attention partials of sequence t and of the
 // row the step just wrote, o_lat rounded to bf16, then o[t, h] = o_lat[t, h] * W_UV[h].  dc = 512, dv = 128.
+// Phases over all tokens at once (scores of the new rows by warps, weights by one thread per token, merge with
+// all partial rows of eight tokens in flight), then the product over groups of four tokens as above.
 __global__ void __launch_bounds__(kThreadsB) uv_merge_batch_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
                                                                    AttnPartials part, const BatchRows rows, int rope, float scale,
                                                                    const uint16_t *__restrict__ W_UV, uint16_t *__restrict__ o_lat_bf16,
                                                                    uint16_t *__restrict__ o, int T)
 {
-    constexpr int K = 512, N = 128, kColGroups = N / 8, kRowGroups = kThreadsB / kColGroups;
-    constexpr int kMaxParts = 64;
-    __shared__ __align__(16) float x_s[K];
-    __shared__ __align__(16) float red[kRowGroups * N];
-    __shared__ float scratch[32];
-    __shared__ float sm[kMaxParts], sl[kMaxParts], sw[kMaxParts];
-    const int h = blockIdx.x, H = gridDim.x, dkv = K + rope, tid = threadIdx.x;
+    constexpr int K = 512, N = 128, kColGroups = N / 8, kRowGroups = kThreadsB / kColGroups;      // 16 x 16
+    constexpr int kMaxParts = 16;                                 // 64 splits in clusters of four
+    __shared__ __align__(16) uint16_t x_s[kMaxBatch][K];          // merged o_lat, already rounded to bf16
+    __shared__ __align__(16) float red[kTokGroup][kRowGroups / 2][N];
+    __shared__ float sm[kMaxBatch][kMaxParts], sl[kMaxBatch][kMaxParts], sw[kMaxBatch][kMaxParts];
+    __shared__ float sx[kMaxBatch], swx[kMaxBatch], sinv[kMaxBatch];
+    const int h = blockIdx.x, H = gridDim.x, dkv = K + rope, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tx = tid % kColGroups, ty = tid / kColGroups;
     const uint16_t *W = W_UV + (size_t)h * K * N + (size_t)ty * N + tx * 8;
     uint4 w[32];
@@ -179,70 +189,107 @@ __global__ void __launch_bounds__(kThreadsB) uv_merge_batch_kernel(const uint16_
     for (int i = 0; i < 32; ++i) w[i] = ld_stream16(W + (size_t)i * kRowGroups * N);
     pdl_launch_dependents();
     pdl_wait_prior_grids();                                       // partials come from the attention kernel
+    // (m, l) of every (token, part)
+    for (int i = tid; i < T * kMaxParts; i += kThreadsB) {
+        const int t = i / kMaxParts, s = i - t * kMaxParts;
+        if (s < rows.npart[t]) {
+            const float2 p = __ldcg(reinterpret_cast<const float2 *>(part.ml + (((size_t)t * rows.slot_stride + s) * H + h) * 2));
+            sm[t][s] = p.x; sl[t][s] = p.y;
+        }
+    }
+    // score of each token's new row: one warp per token, 576 elements over 32 lanes
+    for (int t = warp; t < T; t += kThreadsB / 32) {
+        const uint16_t *qh = Q + ((size_t)t * H + h) * dkv, *row = cache + rows.new_row[t];
+        float dot = 0.f;
+        for (int i = lane * 2; i < dkv; i += 64) {
+            const uint32_t a = __ldcg(reinterpret_cast<const uint32_t *>(qh + i)), b = __ldcg(reinterpret_cast<const uint32_t *>(row + i));
+            dot = fmaf(__uint_as_float(a << 16), __uint_as_float(b << 16), dot);
+            dot = fmaf(__uint_as_float(a & 0xffff0000u), __uint_as_float(b & 0xffff0000u), dot);
+        }
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o2);
+        if (lane == 0) sx[t] = dot * scale;
+    }
+    __syncthreads();
+    if (tid < T) {                                                 // weights of the parts and of the new row, normaliser
+        const int t = tid, npart = rows.npart[t];
+        float Mx = sx[t];
+        for (int s = 0; s < npart; ++s) Mx = fmaxf(Mx, sm[t][s]);
+        const float wx = __expf(sx[t] - Mx);
+        float L = wx;
+        for (int s = 0; s < npart; ++s) {
+            const float wgt = (sm[t][s] == -INFINITY) ? 0.f : __expf(sm[t][s] - Mx);
+            sw[t][s] = wgt;
+            L = fmaf(wgt, sl[t][s], L);
+        }
+        swx[t] = wx; sinv[t] = 1.0f / L;
+    }
+    __syncthreads();
+    // merge: two columns per thread, every token
     const int c = 2 * tid;
     for (int t = 0; t < T; ++t) {
         const int npart = rows.npart[t];
-        const float *ml = part.ml + (size_t)t * rows.slot_stride * H * 2;
-        const float *Ot = part.O + (size_t)t * rows.slot_stride * H * K + (size_t)h * K + c;
-        const uint16_t *new_row = cache + rows.new_row[t];
-        constexpr int kBatch = 8;
-        float2 v[kBatch];
+        const float *Ot = part.O + ((size_t)t * rows.slot_stride * H + h) * K + c;
+        float2 v[kMaxParts];
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u)
-            v[u] = (u < npart) ? __ldcg(reinterpret_cast<const float2 *>(Ot + (size_t)u * H * K)) : make_float2(0.f, 0.f);
-        for (int s = tid; s < npart; s += kThreadsB) {
-            const float2 p = __ldcg(reinterpret_cast<const float2 *>(ml + ((size_t)s * H + h) * 2));
-            sm[s] = p.x; sl[s] = p.y;
+        for (int s = 0; s < kMaxParts; ++s)
+            v[s] = (s < npart) ? __ldcg(reinterpret_cast<const float2 *>(Ot + (size_t)s * H * K)) : make_float2(0.f, 0.f);
+        const uint32_t rv = __ldcg(reinterpret_cast<const uint32_t *>(cache + rows.new_row[t] + c));
+        float2 acc = make_float2(swx[t] * __uint_as_float(rv << 16), swx[t] * __uint_as_float(rv & 0xffff0000u));
+#pragma unroll
+        for (int s = 0; s < kMaxParts; ++s) {                      // part order: deterministic
+            const float wgt = (s < npart) ? sw[t][s] : 0.f;
+            acc.x = fmaf(wgt, v[s].x, acc.x);
+            acc.y = fmaf(wgt, v[s].y, acc.y);
         }
-        // score of the new row: q . row over all 576 elements
-        float dot = 0.f;
-        if (tid < dkv / 8) {
-            float qf[8], rf[8];
-            Elem<bf16_t>::unpack(__ldcg(reinterpret_cast<const uint4 *>(Q + ((size_t)t * H + h) * dkv) + tid), qf);
-            Elem<bf16_t>::unpack(__ldcg(reinterpret_cast<const uint4 *>(new_row) + tid), rf);
+        const uint32_t ob = pack2(acc.x * sinv[t], acc.y * sinv[t]);
+        *reinterpret_cast<uint32_t *>(o_lat_bf16 + ((size_t)t * H + h) * K + c) = ob;
+        *reinterpret_cast<uint32_t *>(&x_s[t][c]) = ob;            // W_UV sees the rounded o_lat, as the stage-wise definition says
+    }
+    __syncthreads();
+    for (int t0 = 0; t0 < T; t0 += kTokGroup) {
+        float acc[kTokGroup][8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) dot = fmaf(qf[e], rf[e], dot);
-        }
-        const float sx = block_sum(dot, scratch) * scale;
-        float Mx = sx;
-        for (int s = 0; s < npart; ++s) Mx = fmaxf(Mx, sm[s]);
-        const float wx = __expf(sx - Mx);
-        float L = wx;
-        for (int s = 0; s < npart; ++s) {                          // same order in every thread
-            const float wgt = (sm[s] == -INFINITY) ? 0.f : __expf(sm[s] - Mx);
-            if (tid == 0) sw[s] = wgt;
-            L = fmaf(wgt, sl[s], L);
-        }
-        __syncthreads();
-        const uint32_t rv = *reinterpret_cast<const uint32_t *>(new_row + c);
-        float2 acc = make_float2(wx * __uint_as_float(rv << 16), wx * __uint_as_float(rv & 0xffff0000u));
-        for (int s0 = 0; s0 < npart; s0 += kBatch) {
-            if (s0 > 0) {
+        for (int g = 0; g < kTokGroup; ++g)
 #pragma unroll
-                for (int u = 0; u < kBatch; ++u)
-                    v[u] = (s0 + u < npart) ? __ldcg(reinterpret_cast<const float2 *>(Ot + (size_t)(s0 + u) * H * K)) : make_float2(0.f, 0.f);
-            }
+            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
 #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                const float wgt = (s0 + u < npart) ? sw[s0 + u] : 0.f;
-                acc.x = fmaf(wgt, v[u].x, acc.x);
-                acc.y = fmaf(wgt, v[u].y, acc.y);
+        for (int i = 0; i < 32; ++i) {
+            float b[8];
+            uint4 wi = w[i];
+            // keeps the widening of the weights inside the group loop: hoisted out of it, the 256 widened values
+            // of a thread would not fit its registers
+            asm volatile("" : "+r"(wi.x), "+r"(wi.y), "+r"(wi.z), "+r"(wi.w));
+            Elem<bf16_t>::unpack(wi, b);
+#pragma unroll
+            for (int g = 0; g < kTokGroup; ++g) {
+                const float a = bf2f(x_s[min(t0 + g, kMaxBatch - 1)][ty + i * kRowGroups]);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[g][j] = fmaf(a, b[j], acc[g][j]);
             }
         }
-        const float inv = 1.0f / L;
-        const uint16_t b0 = f2bf(acc.x * inv), b1 = f2bf(acc.y * inv);
-        *reinterpret_cast<uint32_t *>(o_lat_bf16 + ((size_t)t * H + h) * K + c) = (uint32_t)b0 | ((uint32_t)b1 << 16);
-        x_s[c] = bf2f(b0);                                         // W_UV sees the rounded o_lat, as the stage-wise definition says
-        x_s[c + 1] = bf2f(b1);
-        __syncthreads();
-        float out8[8];
-        head_matvec<K, N>(w, x_s, red, out8);
-        if (ty == 0) {
-            uint4 ov;
-            ov.x = pack2(out8[0], out8[1]); ov.y = pack2(out8[2], out8[3]); ov.z = pack2(out8[4], out8[5]); ov.w = pack2(out8[6], out8[7]);
-            *reinterpret_cast<uint4 *>(o + ((size_t)t * H + h) * N + tx * 8) = ov;
+#pragma unroll
+        for (int g = 0; g < kTokGroup; ++g) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[g][j] += __shfl_xor_sync(0xffffffffu, acc[g][j], 16);    // row groups 2j + 2j+1
+            if ((tid & 16) == 0) {
+                float4 *dst = reinterpret_cast<float4 *>(&red[g][ty >> 1][tx * 8]);
+                dst[0] = make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
+                dst[1] = make_float4(acc[g][4], acc[g][5], acc[g][6], acc[g][7]);
+            }
         }
-        __syncthreads();                                           // shared buffers are reused by the next token
+        __syncthreads();
+        // 4 tokens x 128 columns = 512 outputs, two per thread; row-group pairs added in a fixed order
+        {
+            const int g = tid / 64, col = (tid % 64) * 2;
+            if (t0 + g < T) {
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int r = 0; r < kRowGroups / 2; ++r) { s0 += red[g][r][col]; s1 += red[g][r][col + 1]; }
+                *reinterpret_cast<uint32_t *>(o + ((size_t)(t0 + g) * H + h) * N + col) = pack2(s0, s1);
+            }
+        }
+        __syncthreads();                                           // red is reused by the next group
     }
 }
 
@@ -279,7 +326,7 @@ int launch_uv_merge_batch(const void *Q, const void *cache, AttnPartials part, c
                           const void *W_UV, void *o_lat_bf16, void *o, int H, cudaStream_t s, bool pdl)
 {
     for (int t = 0; t < T; ++t)
-        if (rows.npart[t] < 0 || rows.npart[t] > 64) return NM_ERR_UNSUPPORTED;
+        if (rows.npart[t] < 0 || rows.npart[t] > 16) return NM_ERR_UNSUPPORTED;
     cudaError_t e = launch_b(uv_merge_batch_kernel, dim3(H), s, pdl, (const uint16_t *)Q, (const uint16_t *)cache, part, rows, rope, scale,
                              (const uint16_t *)W_UV, (uint16_t *)o_lat_bf16, (uint16_t *)o, T);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "uv_merge (batch) launch");

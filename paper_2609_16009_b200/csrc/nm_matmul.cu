@@ -66,6 +66,21 @@ static Plan make_tma_plan(int M, int N, int K, int H, bool chained = false)
 {
     Plan p{};
     p.kind = kRowTma;
+    // Large single matrices with long columns: one CTA per SM, no k-split, an 8-stage ring (128 KB in flight per
+    // SM).  Measured 4-10 % faster than two smaller CTAs per SM on every shape of 50-260 MB tried (6.2-6.5 TB/s),
+    // provided the tiles fill most of the machine: at M = 2 a CTA is also bound by its own FMA rate, and 112
+    // CTAs were too few.
+    if (M <= 2 && H == 1 && g_force_tn == 0 && g_force_split == 0 && 2.0 * K * N >= 48e6 && K >= 4096) {
+        for (int t = 64; t <= 256; t *= 2) {
+            const int tiles = ceil_div(N, t);
+            if (tiles <= kSMs && tiles >= (M == 1 ? 100 : 120)) {
+                const int kt1 = (kTmaConsumers / (t / 8)) * 4;
+                p.tn = t; p.tpr = t / 8; p.rg = kTmaConsumers / p.tpr; p.nsplit = 1; p.kr = ceil_div(K, kt1) * kt1; p.ntiles = tiles;
+                p.nstage = g_force_stages > 0 ? (g_force_stages < 2 ? 2 : (g_force_stages > 11 ? 11 : g_force_stages)) : 8;
+                return p;
+            }
+        }
+    }
     int tn = 64;
     const long tile_cap = (M > 8) ? kSMs : 2 * kSMs;   // a single wave of resident CTAs (two per SM, one when M > 8)
     while ((long)ceil_div(N, tn) * H > tile_cap && tn < 256) tn *= 2;
@@ -131,7 +146,8 @@ static Plan make_tc_plan(int M, int N, int K, int H)
     const int kr = ceil_div(ceil_div(K, ns), kTcKT) * kTcKT;
     p.kr = kr;
     p.nsplit = ceil_div(K, kr);
-    int nstage = 5;
+    // one CTA per SM on a large matrix: a deeper ring (measured +1.5 to 3 %); otherwise 90 KB, two CTAs fit an SM
+    int nstage = (base * p.nsplit <= kSMs && 2.0 * K * N * H >= 48e6) ? 7 : 5;
     const int its = ceil_div(kr, kTcKT);                // a ring deeper than the CTA's k-range only costs shared memory
     if (nstage > its) nstage = its;
     if (g_force_stages > 0) nstage = g_force_stages;

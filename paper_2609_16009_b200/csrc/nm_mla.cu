@@ -546,9 +546,9 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
                               NM_BF16, NM_ROW_MAJOR, mws, L.main_ws_bytes, ms, pdl));
     }
 
-    // ---- beside the attention pass: idle lanes of the attention kernel pull W_UV and the head of every
-    //      k-split of W_O into L2, so that the output-side products start from L2 instead of HBM (Data
-    //      Independence: the weights do not depend on the attention result) -----------------------------------
+    // ---- beside the attention pass: W_UV and the head of every k-split of W_O are pulled into L2, so that the
+    //      output-side products start from L2 instead of HBM (Data Independence: the weights do not depend on
+    //      the attention result) ---------------------------------------------------------------------------------
     L2Prefetch pf{};
     if (g_prefetch_mb > 0 && pos > 0) {
         pf.block = (const char *)p->W_UV;
@@ -573,9 +573,8 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     // the attention kernel does.
     const bool uv_early = fused && pdl && !forked && g_uv_pdl;
     NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms, pdl, uv_early ? L2Prefetch{} : pf));
-    // The merge needs the cache row the KV chain wrote.  Joining here also keeps the merge from being
-    // launched early: its CTAs could not share an SM with the attention CTAs (registers) and would
-    // only hold up the prefetch kernel in the block scheduler.
+    // The merge needs the cache row the KV chain wrote (two-stream schedule): the join sits right before it, where
+    // it breaks only the merge's programmatic launch.
     if (forked) NM_CUDA_TRY(cudaStreamWaitEvent(ms, g_events.join, 0));
     if (fused) {
         // merge of the attention partials (+ the new row) and o[h] = o_lat[h] * W_UV[h] in one kernel

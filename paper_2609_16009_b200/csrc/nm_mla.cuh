@@ -27,7 +27,8 @@ AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int
 
 // Tensor-core (tcgen05 / TMEM) pass over the rows of each split.  Returns NM_ERR_UNSUPPORTED when
 // the shape is not one it takes (the caller then uses the CUDA-core kernel).
-// Weight bytes the attention kernel's idle lanes pull into L2 while the tensor cores work: one
+// Weight bytes pulled into L2 while the tensor cores work (by the merge kernel's idle prologue, or by a warp of
+// the attention kernel): one
 // contiguous block plus `nranges` ranges of `range_bytes`, `range_stride` apart (all may be empty).
 struct L2Prefetch {
     const char *block;

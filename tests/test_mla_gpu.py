@@ -392,6 +392,46 @@ def test_decode_step_back_to_back_steps_do_not_interfere(nm, weights, ref1024):
     assert np.all(np.abs(dev_bits_to_f64(outs[0]) - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
 
 
+@pytest.mark.parametrize("S", [4096, 16384])
+def test_decode_step_in_the_configuration_the_bench_times(nm, weights, S):
+    # the bench's launch configuration at its full sizes: the three down-projections stored as one matrix (one
+    # stream, six kernels), the step's first product allowed to start under the previous step's tail, steps
+    # enqueued back to back without a host synchronisation; every output element against the oracle
+    w, dw = weights
+    h, cache_ref, r = oracle_step(w, S, seed=4600 + S)
+    H, dc, dr, dn, dv, d, ql = (DIMS[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d", "q_lora"))
+    dkv = dc + dr
+    t = dict(dw)
+    t["W_DQKV"] = torch.cat([t.pop("W_DQ").view(d, ql), t.pop("W_DKVKR").view(d, dkv)], dim=1).contiguous().view(-1)
+    t["h"] = to_dev(h)
+    t["kv_cache"] = to_dev(gen.mla_cache(S, DIMS, seed=4600 + S))
+    t["rope_cos_sin"] = rope_row(nm, S - 1)
+    t["out"] = torch.zeros(d, dtype=torch.int16, device="cuda")
+    t["o_lat_f32"] = torch.zeros(H * dc, dtype=torch.float32, device="cuda")
+    p = nm.mla_params(DIMS, S, t)
+    ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p))
+    p = nm.mla_params(DIMS, S, t, workspace=ws)
+    p.programmatic_entry = 1
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = []
+    with torch.cuda.stream(main):
+        for _ in range(4):
+            nm.nm_mla_decode_step(p, main, side)
+            outs.append(t["out"].clone())
+    torch.cuda.synchronize()
+    nm.nm_check_status()
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0])
+    o32 = t["o_lat_f32"].cpu().numpy().astype(np.float64).reshape(H, dc)
+    assert rel_max(o32, r["o_lat_f64"]) <= 2e-3
+    ref = f64(r["out"]).reshape(-1)
+    assert np.all(np.abs(dev_bits_to_f64(outs[0]) - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
+    cache = t["kv_cache"].cpu().numpy().view(np.uint16).reshape(-1, dkv)
+    assert np.array_equal(cache[:S - 1], cache_ref[:S - 1])
+    assert np.all(np.abs(f64(cache[S - 1]) - f64(cache_ref[S - 1])) <= 2 * oracle.ulp_bf16(f64(cache_ref[S - 1])) + 1e-6)
+
+
 def test_decode_step_replayed_from_a_cuda_graph(nm, weights, ref1024):
     # both streams, the events between them and the programmatic launches are captured once; replays must
     # reproduce the directly launched result bit for bit

@@ -79,6 +79,17 @@ def test_m_sweep_full_size_sampled_columns(nm, K, N, M):
     run_case(nm, A, B, M, N, K, BF16, ROW, f"M={M} K={K} N={N}", cols=cols)
 
 
+@pytest.mark.parametrize("M,K,N", [(1, 16384, 7168), (2, 16384, 7168), (8, 16384, 7168), (3, 7168, 1536), (16, 7168, 1536),
+                                   (1, 8192, 8192), (5, 4096, 4096)])
+def test_other_large_and_mid_size_shapes_sampled_columns(nm, M, K, N):
+    # the output projection's shape and a few more on either side of the planner's thresholds (one CTA per SM
+    # for large matrices, tensor cores from 16 MB at M >= 3, batched split-K gather)
+    A, B = gen.narrow_bf16(M, K, N, seed=2100 + M + K % 97)
+    rng = np.random.default_rng(M + N)
+    cols = sorted(set([0, 63, 64, 127, 128, N - 1, N - 64] + rng.integers(0, N, 40).tolist()))
+    run_case(nm, A, B, M, N, K, BF16, ROW, f"M={M} K={K} N={N}", cols=cols)
+
+
 # ---- every M, ragged shapes, both layouts, all dtypes ------------------------------------------------------
 
 @pytest.mark.parametrize("M", list(range(1, 17)))

@@ -392,6 +392,31 @@ def batched_case(nm, device, T, K, N, H):
     return row
 
 
+def read_only_stream(nm, device):
+    """GB/s of a kernel that only reads 1 GiB once (nm_debug_stream_read: the products' own streaming load, nothing
+    else), best of the CTA counts tried: what a read-only stream reaches on this GPU, beside the copy bandwidth
+    that the roofline uses as its peak."""
+    n = 1 << 30
+    buf = torch.empty(n, dtype=torch.uint8, device=device)
+    buf.random_(0, 255)
+    sink = torch.zeros(1, dtype=torch.int32, device=device)
+    s = torch.cuda.Stream(device)
+    best = {}
+    with torch.cuda.stream(s):
+        for ctas in (2, 4, 8):
+            for _ in range(3):
+                nm.nm_debug_stream_read(buf, n, sink, ctas, s)
+            ts = []
+            for _ in range(9):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(s); nm.nm_debug_stream_read(buf, n, sink, ctas, s); b.record(s); s.synchronize()
+                ts.append(a.elapsed_time(b))
+            gbs = n / (statistics.median(ts) * 1e-3) / 1e9
+            if not best or gbs > best["GBps"]:
+                best = {"GBps": round(gbs, 1), "ctas_per_sm": ctas, "bytes": n}
+    return best
+
+
 def matmul_sweep(nm, device):
     """GB/s of single narrow products (cold L2: the launches of a CUDA graph rotate through copies of
     B that together exceed 512 MB).  Two figures per case: launches in plain stream order (each kernel
@@ -706,6 +731,7 @@ def main():
         line.update(extras)
         if args.sweep:
             line["narrow_matmul_vs_M"] = matmul_sweep(nm, device)
+            line["read_only_stream"] = read_only_stream(nm, device)
         if not args.no_cpu_baseline:
             import oracle
             threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))

@@ -333,6 +333,10 @@ int nm_debug_set_step_prefetch(int megabytes);
 int nm_debug_set_step_pdl(int enable);
 /* Attention pass: 0 tensor-core kernel when the shape allows (default), 1 CUDA-core kernel. */
 int nm_debug_set_attention(int impl);
+/* Measurement aid: a kernel that only reads `bytes` bytes of device memory once (16-byte streaming loads, the
+ * products' own load instruction, ctas_per_sm x SM-count CTAs of 256 threads) - the read-only bandwidth this GPU
+ * delivers, to set beside the copy bandwidth the roofline uses.  src 16-byte aligned; sink4: 4 writable bytes. */
+int nm_debug_stream_read(const void *src, size_t bytes, void *sink4, int ctas_per_sm, nm_stream stream);
 /* Report the plan for a problem: out[0..5] = kernel kind (0 row-major vector, 1 column-major
  * vector, 2 scalar), columns per tile, k-splits, k-rows per split, column tiles, CTAs. */
 int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B, int vec_ok,

@@ -100,6 +100,7 @@ _lib.nm_mla_decode_step.argtypes = [C.POINTER(MlaParams), _vp, _vp]
 _lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_debug_set_attention.argtypes = [_i]
 _lib.nm_debug_set_step_pdl.argtypes = [_i]
+_lib.nm_debug_stream_read.argtypes = [_vp, _sz, _vp, _i, _vp]
 _lib.nm_debug_set_step_knobs.argtypes = [_i, _i]
 _lib.nm_debug_set_step_plan.argtypes = [_i, _i, _i, _i]
 _lib.nm_debug_set_step_prefetch.argtypes = [_i]
@@ -344,6 +345,10 @@ def nm_debug_set_step_knobs(uv_programmatic: int = 1, prefetch_w_uv: int = 1) ->
 
 def nm_debug_set_step_plan(which: int, tile_n: int = 0, nsplit: int = 0, stages: int = 0) -> None:
     _check(_lib.nm_debug_set_step_plan(which, tile_n, nsplit, stages), "nm_debug_set_step_plan")
+
+
+def nm_debug_stream_read(src, nbytes: int, sink, ctas_per_sm: int = 4, stream=None) -> None:
+    _check(_lib.nm_debug_stream_read(_ptr(src), int(nbytes), _ptr(sink), int(ctas_per_sm), _stream(stream)), "nm_debug_stream_read")
 
 
 def nm_debug_set_step_pdl(enable: bool) -> None:

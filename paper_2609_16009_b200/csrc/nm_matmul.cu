@@ -172,8 +172,11 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     // Thresholds from sweeps of both kernels over 8-34 MB matrices and the batched per-head shapes: from 16 MB
     // (8 MB when batched over heads) the tensor-core kernel wins from M = 3 on; at 8 MB in one matrix the two tie.
     const double wbytes = 2.0 * K * N * H;
-    const bool tc_pays = M >= g_tc_min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6));
-    if (layout == NM_ROW_MAJOR && tma_ok && g_force_kind != kRowTma && (tc_pays || g_force_kind == kRowTc))
+    // Column-major weights: the CUDA-core column kernel is already behind at M = 2 from about 50 MB on (17 vs 14 us
+    // on 75 MB).
+    const int min_m = (layout == NM_COL_MAJOR && g_tc_min_m > 2 && g_tc_min_m <= NM_MAX_M) ? 2 : g_tc_min_m;
+    const bool tc_pays = M >= min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6)) && (M >= g_tc_min_m || wbytes >= 48e6);
+    if (tma_ok && g_force_kind != kRowTma && (layout == NM_ROW_MAJOR || g_force_kind != kRowVec) && (tc_pays || g_force_kind == kRowTc))
         return make_tc_plan(M, N, K, H);
     if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H, chained);
     const int target = 192;                           // CTAs wanted in total (measured: 144-240 is the flat optimum)
@@ -286,16 +289,19 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
                       (layout == NM_ROW_MAJOR ? (N % V == 0) : (K % V == 0));
     const bool a_ok = aligned16(A) && (lda % V == 0) && (strideA % V == 0);
     const bool vec_ok = b_ok && (layout == NM_ROW_MAJOR || a_ok);
-    bool tma_ok = b_ok && a_ok && layout == NM_ROW_MAJOR && dtype != NM_F32 && tensor_map_encoder() != nullptr &&
-                  (long)N * 2 < (1L << 40) && strideB >= 0;
+    // tensor maps: 16-byte aligned operands and strides, bf16.  Row-major B may take the TMA ring kernel or the
+    // tensor-core kernel; column-major B only the latter (its CUDA-core path is the plain column kernel).
+    bool tma_ok = b_ok && a_ok && dtype != NM_F32 && tensor_map_encoder() != nullptr && (long)N * 2 < (1L << 40) && strideB >= 0;
     if (g_force_kind == kRowVec) tma_ok = false;
     Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok, chained);
     const CUtensorMap *tc_map_b = nullptr, *tc_map_a = nullptr;
     if (p.kind == kRowTc) {
         // weights [H][K][N] in 64x64 swizzled boxes; tokens [H][M][K] (row stride lda) in 64 x 16 swizzled boxes
-        tc_map_b = get_weight_map(B, N, K, H, strideB, 64, kTcKT, true);
+        tc_map_b = (layout == NM_ROW_MAJOR) ? get_weight_map(B, N, K, H, strideB, 64, kTcKT, true)
+                                            : get_weight_map(B, K, N, H, strideB, 64, kTcTN, true);     // [N][K]: 64 k x 128 columns of C
         tc_map_a = get_weight_map(A, K, M, H, strideA, 64, 16, true, lda);
-        if (!tc_map_b || !tc_map_a) p = make_tma_plan(M, N, K, H, chained);      // strides the encoder refuses: CUDA-core kernel
+        if (!tc_map_b || !tc_map_a)                         // strides the encoder refuses: CUDA-core kernel
+            p = make_plan(M, N, K, H, dtype, layout, vec_ok, false, chained);
     }
 
     MatmulArgs a{};
@@ -317,7 +323,8 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         const CUtensorMap *mb = tc_map_b, *ma = tc_map_a;
         TmaArgs ta{};
         ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
-        e = (dtype == NM_BF16_F32OUT) ? launch_row_tc<float>(*mb, *ma, ta, stream) : launch_row_tc<bf16_t>(*mb, *ma, ta, stream);
+        const bool col = layout == NM_COL_MAJOR;
+        e = (dtype == NM_BF16_F32OUT) ? launch_row_tc<float>(*mb, *ma, ta, stream, col) : launch_row_tc<bf16_t>(*mb, *ma, ta, stream, col);
     } else if (p.kind == kRowTma) {
         const int kt = (kTmaConsumers / p.tpr) * 4;
         const CUtensorMap *map = get_weight_map(B, N, K, H, strideB, p.tn, kt);
@@ -499,7 +506,7 @@ int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
 {
     if (!out) return NM_ERR_INVALID_ARG;
     Plan p = make_plan(M, N, K, H, dtype, layout_B, vec_ok != 0,
-                       vec_ok != 0 && layout_B == NM_ROW_MAJOR && dtype != NM_F32 && g_force_kind != kRowVec);
+                       vec_ok != 0 && dtype != NM_F32 && g_force_kind != kRowVec);
     out[0] = p.kind; out[1] = p.tn; out[2] = p.nsplit; out[3] = p.kr; out[4] = p.ntiles;
     out[5] = p.ntiles * p.nsplit * H;
     return NM_OK;

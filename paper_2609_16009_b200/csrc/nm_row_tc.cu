@@ -1,4 +1,4 @@
-// Narrow product with the roles of the operands swapped, on the tensor cores (row-major bf16 B).
+// Narrow product with the roles of the operands swapped, on the tensor cores (bf16 B, either layout).
 //
 // For M above ~8 the CUDA-core kernel is bound by fp32 FMA issue, not by HBM (8*M FMAs per 16 bytes of
 // weights against 128 FMA lanes per SM).  Here the weights take the MMA's M dimension and the token
@@ -14,6 +14,9 @@
 // commits the stage back to the producer; four warps read the 128 x 16 accumulator from TMEM at the
 // end and write C (or the split-K partial tile, completed by the arrival counter as in the other
 // kernels).  Weights are fetched before the programmatic-launch wait, tokens after.
+//
+// Column-major B ([N][K], k contiguous) is the same kernel with the weight operand K-major: one
+// [128 columns of C x 64 k] box per stage (128-byte swizzle), the descriptor advanced 32 bytes per k-step.
 #include "nm_matmul_kernels.cuh"
 #include "nm_row_tc.cuh"
 #include "nm_tcgen05.cuh"
@@ -28,7 +31,7 @@ constexpr int kAStage = 16 * kTcKT * 2;            // 2 KB of tokens per stage
 constexpr int kStage = kBStage + kAStage;
 constexpr uint32_t kTmemColsTc = 32;
 
-template <typename TO>
+template <typename TO, bool kCol>
 __global__ void __launch_bounds__(kTcThreads, 4)
 nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_a, const TmaArgs ta)
 {
@@ -71,8 +74,12 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
             auto load_b = [&](int it, int s) {
                 const uint32_t dst = base + (uint32_t)s * kStage;
                 mbar_arrive_expect_tx(full_b0 + 8 * s, kBStage);
-                tma_load_3d(dst, &map_b, tile * kTcTN, kb + it * kTcKT, h, full_b0 + 8 * s, stream);
-                tma_load_3d(dst + kBStage / 2, &map_b, tile * kTcTN + 64, kb + it * kTcKT, h, full_b0 + 8 * s, stream);
+                if constexpr (kCol) {
+                    tma_load_3d(dst, &map_b, kb + it * kTcKT, tile * kTcTN, h, full_b0 + 8 * s, stream);
+                } else {
+                    tma_load_3d(dst, &map_b, tile * kTcTN, kb + it * kTcKT, h, full_b0 + 8 * s, stream);
+                    tma_load_3d(dst + kBStage / 2, &map_b, tile * kTcTN + 64, kb + it * kTcKT, h, full_b0 + 8 * s, stream);
+                }
             };
             auto load_a = [&](int it, int s) {
                 mbar_arrive_expect_tx(full_a0 + 8 * s, kAStage);
@@ -94,7 +101,7 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc(128, 16, true, false);
+            constexpr uint32_t idesc = instr_desc(128, 16, !kCol, false);
             int s = 0;
             uint32_t ph = 0;
             for (int it = 0; it < n_it; ++it) {
@@ -104,7 +111,8 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
                 const uint32_t sb = base + (uint32_t)s * kStage, sa = sb + kBStage;
 #pragma unroll
                 for (int kk = 0; kk < kTcKT / 16; ++kk)
-                    mma_ss(tmem, smem_desc(sb + kk * 2048, kBStage / 2, 1024), smem_desc(sa + kk * 32, 16, 1024), idesc, (it | kk) != 0);
+                    mma_ss(tmem, kCol ? smem_desc(sb + kk * 32, 16, 1024) : smem_desc(sb + kk * 2048, kBStage / 2, 1024),
+                           smem_desc(sa + kk * 32, 16, 1024), idesc, (it | kk) != 0);
                 mma_commit(empty0 + 8 * s);                       // the stage is free once these MMAs have read it
                 if (++s == NS) { s = 0; ph ^= 1; }
             }
@@ -153,12 +161,12 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
 
 size_t row_tc_smem_bytes(int nstage) { return (size_t)nstage * kStage + (3 * nstage + 1) * sizeof(uint64_t) + 1024; }
 
-template <typename TO>
-cudaError_t launch_row_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta, cudaStream_t s)
+template <typename TO, bool kCol>
+static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta, cudaStream_t s)
 {
     const MatmulArgs &a = ta.base;
     static bool configured = false;
-    auto kern = nm_row_tc_kernel<TO>;
+    auto kern = nm_row_tc_kernel<TO, kCol>;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
@@ -177,7 +185,13 @@ cudaError_t launch_row_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, co
     return cudaLaunchKernelEx(&cfg, kern, map_b, map_a, ta);
 }
 
-template cudaError_t launch_row_tc<bf16_t>(const CUtensorMap &, const CUtensorMap &, const TmaArgs &, cudaStream_t);
-template cudaError_t launch_row_tc<float>(const CUtensorMap &, const CUtensorMap &, const TmaArgs &, cudaStream_t);
+template <typename TO>
+cudaError_t launch_row_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta, cudaStream_t s, bool col_major)
+{
+    return col_major ? launch_tc<TO, true>(map_b, map_a, ta, s) : launch_tc<TO, false>(map_b, map_a, ta, s);
+}
+
+template cudaError_t launch_row_tc<bf16_t>(const CUtensorMap &, const CUtensorMap &, const TmaArgs &, cudaStream_t, bool);
+template cudaError_t launch_row_tc<float>(const CUtensorMap &, const CUtensorMap &, const TmaArgs &, cudaStream_t, bool);
 
 }  // namespace nm

@@ -1,4 +1,4 @@
-// Swap-AB tensor-core narrow product (row-major bf16 B): launch interface.
+// Swap-AB tensor-core narrow product (bf16 B, row- or column-major): launch interface.
 #pragma once
 
 #include <cuda.h>
@@ -11,9 +11,10 @@ constexpr int kTcTN = 128;      // columns of C per CTA (the MMA's M)
 constexpr int kTcKT = 64;       // k-rows per stage
 
 size_t row_tc_smem_bytes(int nstage);
-// map_b: B as bf16 [H][K][N], boxes {64, 64, 1}, 128-byte swizzle; map_a: A as bf16 [H][M][K], boxes {64, 16, 1},
-// 128-byte swizzle.  ta.base.tn must be kTcTN and ta.base.kr a multiple of kTcKT.
+// map_b: row-major B as bf16 [H][K][N], boxes {64, 64, 1}; column-major B as bf16 [H][N][K], boxes {64, 128, 1}; both with
+// 128-byte swizzle; map_a: A as bf16 [H][M][K], boxes {64, 16, 1}, 128-byte swizzle.  ta.base.tn must be kTcTN and
+// ta.base.kr a multiple of kTcKT.
 template <typename TO>
-cudaError_t launch_row_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta, cudaStream_t s);
+cudaError_t launch_row_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta, cudaStream_t s, bool col_major);
 
 }  // namespace nm

@@ -90,6 +90,31 @@ def test_other_large_and_mid_size_shapes_sampled_columns(nm, M, K, N):
     run_case(nm, A, B, M, N, K, BF16, ROW, f"M={M} K={K} N={N}", cols=cols)
 
 
+@pytest.mark.parametrize("M,K,N", [(3, 7168, 18432), (16, 7168, 18432), (4, 1536, 24576), (8, 7168, 1536)])
+def test_column_major_on_the_tensor_cores_sampled_columns(nm, M, K, N):
+    # column-major weights ([N][K]) at M >= 3 on large matrices: the swap-AB kernel with a K-major weight operand
+    assert nm.nm_debug_get_plan(M, N, K, layout_B=COL)["kind"] == 4
+    A, B = gen.narrow_bf16(M, K, N, seed=2300 + M)
+    rng = np.random.default_rng(M + N)
+    cols = sorted(set([0, 63, 64, 127, 128, N - 1, N - 64] + rng.integers(0, N, 40).tolist()))
+    run_case(nm, A, B, M, N, K, BF16, COL, f"col-major M={M} K={K} N={N}", cols=cols)
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 64, 128), (5, 200, 136), (16, 1000, 840), (3, 4104, 72), (2, 8, 8), (7, 72, 1000)])
+@pytest.mark.parametrize("dtype", [BF16, BF16_F32OUT])
+def test_column_major_tensor_core_kernel_forced_on_small_and_ragged_shapes(nm, M, K, N, dtype):
+    # K not a multiple of the 64-k stage, N not a multiple of the 128-column tile, several k-splits
+    A, B = gen.narrow_bf16(M, K, N, seed=2400 + M + K)
+    nm.nm_debug_set_kernel(4, 0)
+    try:
+        for nsplit in (0, 3):
+            nm.nm_debug_set_plan(0, nsplit)
+            run_case(nm, A, B, M, N, K, dtype, COL, f"forced col-major tensor-core kernel M={M} K={K} N={N} nsplit={nsplit}")
+    finally:
+        nm.nm_debug_set_kernel(-1, 0)
+        nm.nm_debug_set_plan(0, 0)
+
+
 # ---- every M, ragged shapes, both layouts, all dtypes ------------------------------------------------------
 
 @pytest.mark.parametrize("M", list(range(1, 17)))

@@ -317,10 +317,12 @@ int nm_debug_set_kernel(int kind, int stages);
  * kernel; from 2048 / 4096 / 6144 four per CTA (start, inputs ready, loop done, end) of the down-projection, W_UQR
  * and W_O products.  NULL = off. */
 int nm_debug_set_attention_trace(void *device_buffer);
-/* Decode step tuning: uv_programmatic bit 0 - launch the merge + W_UV kernel programmatically (default 1), bit 1 -
- * run RMSNorm / RoPE / cache write as kernels of their own instead of inside the products' completion;
- * prefetch_w_uv - include W_UV in the L2 prefetch (default 1). */
+/* Decode step tuning: launch the merge + W_UV kernel programmatically (default 1); include W_UV in the L2
+ * prefetch (default 1). */
 int nm_debug_set_step_knobs(int uv_programmatic, int prefetch_w_uv);
+/* Decode step: 1 (default) runs RMSNorm / RoPE / the cache-row write inside the completion of the down-projection
+ * products; 0 runs them as kernels of their own. */
+int nm_debug_set_step_tails(int enable);
 /* Decode step tuning: force (tile_n, nsplit, ring stages) of one of its products - which = 0 the down-projection,
  * 1 W_UQR, 2 W_O; zeros give the plan back to the planner. */
 int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages);

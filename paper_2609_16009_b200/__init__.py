@@ -102,6 +102,7 @@ _lib.nm_debug_set_attention.argtypes = [_i]
 _lib.nm_debug_set_step_pdl.argtypes = [_i]
 _lib.nm_debug_stream_read.argtypes = [_vp, _sz, _vp, _i, _vp]
 _lib.nm_debug_set_step_knobs.argtypes = [_i, _i]
+_lib.nm_debug_set_step_tails.argtypes = [_i]
 _lib.nm_debug_set_step_plan.argtypes = [_i, _i, _i, _i]
 _lib.nm_debug_set_step_prefetch.argtypes = [_i]
 _lib.nm_debug_set_step_fusion.argtypes = [_i]
@@ -341,6 +342,10 @@ def nm_debug_set_step_prefetch(megabytes: int) -> None:
 
 def nm_debug_set_step_knobs(uv_programmatic: int = 1, prefetch_w_uv: int = 1) -> None:
     _check(_lib.nm_debug_set_step_knobs(int(uv_programmatic), int(prefetch_w_uv)), "nm_debug_set_step_knobs")
+
+
+def nm_debug_set_step_tails(enable: bool) -> None:
+    _check(_lib.nm_debug_set_step_tails(int(enable)), "nm_debug_set_step_tails")
 
 
 def nm_debug_set_step_plan(which: int, tile_n: int = 0, nsplit: int = 0, stages: int = 0) -> None:

@@ -820,9 +820,17 @@ int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages)
     return NM_OK;
 }
 
+/* 1 (default): RMSNorm / RoPE / cache-row write run inside the completion of the down-projection products; 0: as
+ * kernels of their own. */
+int nm_debug_set_step_tails(int enable)
+{
+    g_fused_tails = enable ? 1 : 0;
+    return NM_OK;
+}
+
 int nm_debug_set_step_knobs(int uv_pdl, int prefetch_uv)
 {
-    g_uv_pdl = uv_pdl & 1; g_prefetch_uv = prefetch_uv & 1; g_fused_tails = (uv_pdl & 2) ? 0 : 1;
+    g_uv_pdl = uv_pdl ? 1 : 0; g_prefetch_uv = prefetch_uv ? 1 : 0;
     return NM_OK;
 }
 

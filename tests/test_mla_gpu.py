@@ -303,12 +303,12 @@ def test_decode_step_vector_stages_inside_and_outside_the_products_agree(nm, wei
     cache_in = gen.mla_cache(1024, DIMS, seed=4200)
     t1 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
     check_step(t1, r, cache_ref, 1024)
-    nm.nm_debug_set_step_knobs(1 | 2, 1)
+    nm.nm_debug_set_step_tails(False)
     try:
         t2 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
         check_step(t2, r, cache_ref, 1024)
     finally:
-        nm.nm_debug_set_step_knobs(1, 1)
+        nm.nm_debug_set_step_tails(True)
     # the products are bit-identical (same plan, same summation order); the norms sum their squares in a
     # different order, so c_qn and the cache row may differ by a rounding flip
     for k in ("c_q", "ckr"):

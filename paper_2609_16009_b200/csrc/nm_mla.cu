@@ -9,7 +9,7 @@
 
 namespace nm {
 
-static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel
+static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape allows (64 heads per CTA), 1: CUDA-core kernel, 2: 128 heads per CTA
 
 // ---- small vector kernels ---------------------------------------------------------------------------
 
@@ -321,16 +321,18 @@ AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int
     AttnPlan p{};
     (void)kv_lora;
     const int tiles = ceil_div(n_rows > 0 ? n_rows : 0, kAttnTileRows);
-    // 64 splits x 2 column halves = 128 CTAs: one wave of the 148 SMs
-    constexpr int kSplitTarget = 64;
-    int nsplit = tiles < kSplitTarget ? tiles : kSplitTarget;
+    // The tensor-core kernels take 128 heads and 16-byte aligned operands (TMA); both passes of an
+    // attention call derive the same answer from the same arguments.
+    const bool tc_ok = g_attn_impl != 1 && H == 128 && n_rows > 0 && (((uintptr_t)Q | (uintptr_t)cache) & 15u) == 0 &&
+                       tensor_map_encoder() != nullptr;
+    p.tensor_core = !tc_ok ? 0 : (g_attn_impl == 2 ? 1 : 2);
+    // one wave of the 148 SMs: 64 splits x 2 column halves (128 heads per CTA), or 32 splits x 2 column halves x 2
+    // head halves (64 heads per CTA)
+    const int split_target = (p.tensor_core == 2) ? 32 : 64;
+    int nsplit = tiles < split_target ? tiles : split_target;
     if (nsplit < 1) nsplit = (n_rows > 0) ? 1 : 0;
     p.rows_per_split = nsplit ? ceil_div(tiles, nsplit) * kAttnTileRows : 0;
     p.nsplit = p.rows_per_split ? ceil_div(n_rows, p.rows_per_split) : 0;
-    // The tensor-core kernel takes 128 heads and 16-byte aligned operands (TMA); both passes of an
-    // attention call derive the same answer from the same arguments.
-    p.tensor_core = (g_attn_impl == 0 && H == 128 && n_rows > 0 && (((uintptr_t)Q | (uintptr_t)cache) & 15u) == 0 &&
-                     tensor_map_encoder() != nullptr) ? 1 : 0;
     p.npartial = p.tensor_core ? ceil_div(p.nsplit, kAttnCluster) : p.nsplit;
     return p;
 }
@@ -370,6 +372,8 @@ static int attention_partial(const void *Q, const void *cache, int H, int n_rows
     if (n_rows == 0) return NM_OK;
     const AttnPlan p = plan_attention(Q, cache, H, n_rows, dc);
     AttnPartials part = carve_partials(ws, H);
+    if (p.tensor_core == 2)
+        return attention_partial_tc64(Q, 1, &cache, &n_rows, &p.rows_per_split, p.nsplit, part, 0, scale, s, pdl, prefetch);
     if (p.tensor_core) return attention_partial_tc(Q, cache, part, p, n_rows, scale, s, pdl, prefetch);
     cudaError_t e = launch_pdl(attn_partial_simt_kernel, dim3(p.nsplit, H), dim3(128), s, pdl, static_cast<const uint16_t *>(Q),
                                static_cast<const uint16_t *>(cache), part, n_rows, p.rows_per_split, dc, dr, scale);
@@ -665,7 +669,8 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     const bool pdl = g_step_pdl != 0;
 
     // split plan of the attention pass: the same number of splits for every sequence, about 128 CTAs in all
-    int nsplit = (64 / T) / kAttnCluster * kAttnCluster;
+    const bool tc64 = g_attn_impl != 2;                            // 64 heads per CTA: four CTAs per split
+    int nsplit = ((tc64 ? 32 : 64) / T) / kAttnCluster * kAttnCluster;
     if (nsplit < kAttnCluster) nsplit = kAttnCluster;
     BatchRows rows{};
     rows.slot_stride = L.slot_stride;
@@ -702,7 +707,10 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     part.O = reinterpret_cast<float *>(ws + L.attn_o);
     if (any_rows) {
         if (tensor_map_encoder() == nullptr) return NM_ERR_UNSUPPORTED;
-        NM_TRY(attention_partial_tc_batch(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl));
+        if (tc64)
+            NM_TRY(attention_partial_tc64(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl, L2Prefetch{}));
+        else
+            NM_TRY(attention_partial_tc_batch(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl));
     }
     NM_TRY(launch_uv_merge_batch(q_full, cache, part, rows, T, dr, p->softmax_scale, p->W_UV, o_lat, o, H, ms, pdl));
     if (p->W_O)

@@ -19,7 +19,7 @@ struct AttnPartials {
 struct AttnPlan {
     int nsplit;
     int rows_per_split;                  // multiple of kAttnTileRows
-    int tensor_core;                     // 1: tcgen05 kernel (partials merged per cluster), 0: CUDA-core kernel
+    int tensor_core;                     // 0: CUDA-core kernel; 1: tcgen05 kernel, 128 heads per CTA; 2: tcgen05 kernel, 64 heads per CTA
     int npartial;                        // partial results the final merge has to read
 };
 
@@ -59,6 +59,12 @@ int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void 
 int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
                     const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl,
                     L2Prefetch prefetch = L2Prefetch{});
+
+// The pass with 64 heads per CTA (nm_attn_tc64.cu): four CTAs per split, 64-row cache stages.  rows_per_split must be
+// multiples of 64.  Same partial layout as the 128-head kernel.
+int attention_partial_tc64(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split, int nsplit,
+                           AttnPartials part, int slot_stride, float scale, cudaStream_t stream, bool programmatic_launch,
+                           L2Prefetch prefetch);
 
 // Small-batch decode (nm_batch_kernels.cu): per-sequence rows and partial counts of one launch.
 struct BatchRows {

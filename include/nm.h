@@ -312,7 +312,8 @@ int nm_debug_set_plan(int tile_n, int nsplit);
  * CUDA-core kernel; 4 swap-AB tensor-core kernel) and the ring depth in stages (0 heuristic). */
 int nm_debug_set_kernel(int kind, int stages);
 /* Tuning aid: phase timestamps (ns, %globaltimer) of the decode step's kernels go to `device_buffer` (8192
- * unsigned 64-bit values) when non-null: [0,32) phases of CTA (0,0) of the attention kernel; from 32 four per
+ * unsigned 64-bit values) when non-null: [0,32) phases of CTA (0,0) of the attention kernel (the 64-head kernel:
+ * from 4 four per cache tile - scores issued, scores seen, P written, P*V issued); from 32 four per
  * attention CTA (start, Q landed, last P*V done, end); from 1100 eight phases of two CTAs of the merge + W_UV
  * kernel; from 2048 / 4096 / 6144 four per CTA (start, inputs ready, loop done, end) of the down-projection, W_UQR
  * and W_O products.  NULL = off. */
@@ -329,7 +330,7 @@ int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages);
 /* Decode step: 1 (default) runs RoPE + W_UK and attention-merge + W_UV as fused per-head kernels, 0 as
  * separate kernels (rope, batched product, merge, batched product). */
 int nm_debug_set_step_fusion(int enable);
-/* Decode step: MB of W_O that the attention kernel's softmax threads prefetch into L2 (default 40, 0 = off). */
+/* Decode step: MB of W_O prefetched into L2 while the attention pass runs (default 40, 0 = off). */
 int nm_debug_set_step_prefetch(int megabytes);
 /* Decode step: chain its kernels with programmatic dependent launch (default 1) or not (0). */
 int nm_debug_set_step_pdl(int enable);

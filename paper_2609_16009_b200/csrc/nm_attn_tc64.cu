@@ -11,9 +11,10 @@
 // For a tile of 64 cache rows:
 //   S[64 x 64]    = Q[64 x 576] * tile^T        36 MMAs dealt to two accumulators (a chain of MMAs into one
 //                                               accumulator waits for its predecessor), added by the softmax
-//   P             = exp2(S*c - m)               one thread per head: with M = 64 the accumulator rows sit in
-//                                               lanes 0-15 of each 32-lane quarter of TMEM, so 16 threads of
-//                                               each softmax warp hold a row, the others idle along
+//   P             = exp2(S*c - m)               two threads per head: with M = 64 the accumulator rows sit in
+//                                               lanes 0-15 of each 32-lane quarter of TMEM; the half-split
+//                                               load/store shape gives thread l columns 0-31 of row l and
+//                                               thread l + 16 columns 32-63, so the whole warp works
 //   O[64 x 256]  += P[64 x 64] * tile[:, half]  P from TMEM as two bf16 terms (hi + lo), over the columns of
 //                                               the first score accumulator, which is free once it was read
 // Everything else - TMA with 128-byte swizzle, lazy rescale, double-buffered stages, bounded waits, the
@@ -104,6 +105,8 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     part.ml += (size_t)seq * seqs.ml_stride;
     part.O += (size_t)seq * seqs.o_stride;
     // Tuning aid: four stamps of every CTA of sequence 0 (start, Q landed, last P*V done, end) from trace[32] on
+    // ... and of CTA (0,0) of sequence 0 per tile t < 7: trace[4 + 4 t ..] = scores issued, scores seen, P written, P*V issued
+#define NM_TRACE_TILE(t, i) do { if (trace && (t) < 7 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) trace[4 + 4 * (t) + (i)] = global_timer_ns(); } while (0)
 #define NM_TRACE_CTA(i) do { if (trace && blockIdx.z == 0) trace[32 + 4 * (blockIdx.y * gridDim.x + blockIdx.x) + (i)] = global_timer_ns(); } while (0)
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -240,11 +243,13 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 bool progress = false;
                 if (ts < ntiles && ts <= tp + 1 && mbar_try_wait(bar_kv_full + 8 * (ts & 1), (ts >> 1) & 1)) {
                     scores(ts);
+                    NM_TRACE_TILE(ts, 0);
                     ++ts;
                     progress = true;
                 }
                 if (mbar_try_wait(bar_p_full + 8 * (tp & 1), (tp >> 1) & 1)) {
                     pv(tp);
+                    NM_TRACE_TILE(tp, 3);
                     ++tp;
                     progress = true;
                 }
@@ -273,37 +278,35 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         prefetch_weights();
     } else {
-        // ---------------- one head per thread (lanes 0-15 of each warp): softmax, lazy rescale -----------------
-        const int quad = warp & 3;
-        const bool row_on = lane < 16;                             // lanes 16-31 of a TMEM quarter hold no accumulator row
+        // ---------------- softmax, lazy rescale: two threads per head.  The accumulator rows sit in lanes 0-15 of
+        //                  each TMEM quarter; the half-split load shape hands columns 0-31 of row l to thread l and
+        //                  columns 32-63 to thread l + 16, so all 32 threads of the warp work -----------------------
+        const int quad = warp & 3, ch = lane >> 4;
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
         float m_used = -INFINITY, l = 0.f;
         for (int t = 0; t < ntiles; ++t) {
             const int b = t & 1;
             mbar_wait(bar_s_full + 8 * b, (t >> 1) & 1, &s_abort, status);
             tc_fence_after();
+            if (tid == 64) NM_TRACE_TILE(t, 1);
             const uint32_t s_col = lane_base + kColS + 128 * b;
-            float s[kT];
+            float s[32];
             {
                 uint32_t a0[32], a1[32];
-                tmem_ld32(s_col, a0);
-                tmem_ld32(s_col + 64, a1);
+                tmem_ld32_halves<32>(s_col, a0);
+                tmem_ld32_halves<32>(s_col + 64, a1);
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) s[j] = __uint_as_float(a0[j]) + __uint_as_float(a1[j]);
-                tmem_ld32(s_col + 32, a0);
-                tmem_ld32(s_col + 96, a1);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) s[32 + j] = __uint_as_float(a0[j]) + __uint_as_float(a1[j]);
             }
-            const int valid = min(kT, r1 - (r0 + t * kT));
+            const int valid = min(kT, r1 - (r0 + t * kT)) - 32 * ch;       // of this thread's 32 columns
             float mx = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < kT; ++j)
+            for (int j = 0; j < 32; ++j)
                 if (j < valid) mx = fmaxf(mx, s[j]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
             const float mx2 = mx * scale_log2;
-            const bool grow = row_on && ((t == 0) || (mx2 > m_used + kLazyThreshold));
+            const bool grow = (t == 0) || (mx2 > m_used + kLazyThreshold);
             // P[b] lies over S[b]'s first accumulator, which the loads above have emptied; it was last read by the
             // P*V of tile t-2, which the scores of this tile were issued behind
             if (t > 0 && __any_sync(0xffffffffu, grow)) {
@@ -311,22 +314,22 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 mbar_wait(bar_pv_done + 8 * ((t - 1) & 1), ((t - 1) >> 1) & 1, &s_abort, status);
                 tc_fence_after();
                 const float f = grow ? fast_exp2(m_used - mx2) : 1.0f;
-                for (int c = 0; c < kDvHalf / 32; ++c) {
+                for (int c = 0; c < kDvHalf / 64; ++c) {
                     uint32_t o[32];
-                    tmem_ld32(lane_base + kColO + c * 32, o);
+                    tmem_ld32_halves<32>(lane_base + kColO + c * 64, o);
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                    tmem_st32(lane_base + kColO + c * 32, o);
+                    tmem_st32_halves<32>(lane_base + kColO + c * 64, o);
                 }
                 tmem_wait_st();
                 if (grow) l *= f;
             }
-            if (grow || (t == 0)) m_used = (t == 0 && !row_on) ? 0.f : mx2;
+            if (grow) m_used = mx2;
             float lsum = 0.f;
-            uint32_t pr[32], plo[32];
+            uint32_t pr[16], plo[16];
 #pragma unroll
-            for (int j = 0; j < kT; j += 2) {
+            for (int j = 0; j < 32; j += 2) {
                 const float p0 = (j < valid) ? fast_exp2(fmaf(s[j], scale_log2, -m_used)) : 0.f;
                 const float p1 = (j + 1 < valid) ? fast_exp2(fmaf(s[j + 1], scale_log2, -m_used)) : 0.f;
                 lsum += p0 + p1;
@@ -335,12 +338,14 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 plo[j >> 1] = pack_bf16x2(p0 - __uint_as_float(hi << 16), p1 - __uint_as_float(hi & 0xffff0000u));
             }
             l += lsum;
-            tmem_st32(s_col, pr);
-            tmem_st32(s_col + 32, plo);
+            tmem_st16_halves<16>(s_col, pr);                       // k 0-31 -> words 0-15, k 32-63 -> words 16-31
+            tmem_st16_halves<16>(s_col + 32, plo);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p_full + 8 * b);
+            if (tid == 64) NM_TRACE_TILE(t, 2);
         }
+        l += __shfl_xor_sync(0xffffffffu, l, 16);
         if (ntiles > 0) {                                          // the last P*V must have landed before O is read
             mbar_wait(bar_pv_done + 8 * ((ntiles - 1) & 1), ((ntiles - 1) >> 1) & 1, &s_abort, status);
             tc_fence_after();
@@ -438,6 +443,7 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     if (tid == 0) NM_TRACE_CTA(3);
 #undef NM_TRACE_CTA
+#undef NM_TRACE_TILE
 }
 
 bool encode_rows_map64(CUtensorMap *map, const void *ptr, int rows, int box_rows)

@@ -334,8 +334,9 @@ int nm_debug_set_step_fusion(int enable);
 int nm_debug_set_step_prefetch(int megabytes);
 /* Decode step: chain its kernels with programmatic dependent launch (default 1) or not (0). */
 int nm_debug_set_step_pdl(int enable);
-/* Attention pass: 0 tensor-core kernel when the shape allows (default: 64 heads per CTA), 1 CUDA-core kernel,
- * 2 the tensor-core kernel with 128 heads per CTA. */
+/* Attention pass: 0 (default) a tensor-core kernel when the shape allows - 64 heads per CTA below 65536 cache rows
+ * in the call, 128 heads per CTA from there on; 1 CUDA-core kernel; 2 / 3 the tensor-core kernel with 128 / 64 heads
+ * per CTA whatever the length. */
 int nm_debug_set_attention(int impl);
 /* Measurement aid: a kernel that only reads `bytes` bytes of device memory once (16-byte streaming loads, the
  * products' own load instruction, ctas_per_sm x SM-count CTAs of 256 threads) - the read-only bandwidth this GPU

@@ -9,7 +9,12 @@
 
 namespace nm {
 
-static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape allows (64 heads per CTA), 1: CUDA-core kernel, 2: 128 heads per CTA
+static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel, 2 / 3: force 128 / 64 heads per CTA
+// Cache rows (over all sequences of a call) from which the 128-head kernel is the faster one: it loads every row
+// into two CTAs instead of four, which decides once a CTA has many tiles to go through; below, the 64-head
+// kernel's shorter prologue and merge win (measured: 16384 rows 94.8 vs 97.3 us per step, 65536 rows 164 vs 158)
+constexpr long kAttnWideRows = 65536;
+static bool attention_64_heads(long total_rows) { return g_attn_impl == 3 || (g_attn_impl != 2 && total_rows < kAttnWideRows); }
 
 // ---- small vector kernels ---------------------------------------------------------------------------
 
@@ -325,7 +330,7 @@ AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int
     // attention call derive the same answer from the same arguments.
     const bool tc_ok = g_attn_impl != 1 && H == 128 && n_rows > 0 && (((uintptr_t)Q | (uintptr_t)cache) & 15u) == 0 &&
                        tensor_map_encoder() != nullptr;
-    p.tensor_core = !tc_ok ? 0 : (g_attn_impl == 2 ? 1 : 2);
+    p.tensor_core = !tc_ok ? 0 : (attention_64_heads(n_rows) ? 2 : 1);
     // one wave of the 148 SMs: 64 splits x 2 column halves (128 heads per CTA), or 32 splits x 2 column halves x 2
     // head halves (64 heads per CTA)
     const int split_target = (p.tensor_core == 2) ? 32 : 64;
@@ -669,7 +674,9 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     const bool pdl = g_step_pdl != 0;
 
     // split plan of the attention pass: the same number of splits for every sequence, about 128 CTAs in all
-    const bool tc64 = g_attn_impl != 2;                            // 64 heads per CTA: four CTAs per split
+    long total_rows = 0;
+    for (int t = 0; t < T; ++t) total_rows += b->seq_lens[t];
+    const bool tc64 = attention_64_heads(total_rows);              // 64 heads per CTA: four CTAs per split
     int nsplit = ((tc64 ? 32 : 64) / T) / kAttnCluster * kAttnCluster;
     if (nsplit < kAttnCluster) nsplit = kAttnCluster;
     BatchRows rows{};
@@ -871,7 +878,8 @@ int nm_debug_set_step_pdl(int enable)
     return NM_OK;
 }
 
-/* 0: tensor-core attention when the shape allows (default); 1: CUDA-core attention kernel. */
+/* 0: tensor-core attention when the shape allows (default); 1: CUDA-core attention kernel; 2 / 3: the tensor-core
+ * kernel with 128 / 64 heads per CTA whatever the length. */
 int nm_debug_set_attention(int impl)
 {
     g_attn_impl = impl;

@@ -191,6 +191,44 @@ def test_attention_stage_default_path(nm, S, extra):
     attention_case(nm, S, 0, extra)
 
 
+@pytest.mark.parametrize("S", [1, 2, 33, 64, 65, 129, 1000, 4096, 16384])
+@pytest.mark.parametrize("extra", [True, False])
+def test_attention_stage_128_heads_per_cta(nm, S, extra):
+    """The tensor-core kernel that keeps all 128 heads in one CTA (32-row cache stages) stays selectable."""
+    attention_case(nm, S, 2, extra)
+
+
+@pytest.mark.parametrize("impl", [0, 3])
+def test_attention_stage_long_sequence(nm, impl):
+    """From 65536 cache rows on the default is the 128-head kernel; the 64-head kernel stays selectable (16 tiles per CTA)."""
+    attention_case(nm, 66001, impl, True)
+
+
+def test_attention_kernels_agree_on_heavy_tailed_scores(nm):
+    """Scores whose maximum grows along the sequence by more than the lazy-rescale threshold force the rescale of
+    the running output in both tensor-core kernels; all three implementations must agree with the oracle."""
+    H, dc, dr = DIMS["H"], DIMS["kv_lora"], DIMS["rope"]
+    dkv, S = dc + dr, 700
+    Q = np.concatenate([gen.normal_bf16((H, dc), 0.18, 7100), gen.normal_bf16((H, dr), 0.78, 7101)], axis=1)
+    c64 = f64(gen.normal_bf16((S, dkv), 1.0, 7102)) * np.linspace(0.05, 6.0, S)[:, None]     # norms grow with the row
+    cache = oracle.f64_to_bf16(c64)
+    scale = (DIMS["nope"] + dr) ** -0.5
+    ref = oracle.mla_attention(f64(Q), f64(cache), dc, scale, threads=8)
+    ws = torch.empty(nm.nm_mla_attention_workspace_bytes(H, S, dc), dtype=torch.uint8, device="cuda")
+    for impl in (0, 1, 2, 3):
+        o16 = torch.zeros(H * dc, dtype=torch.int16, device="cuda")
+        o32 = torch.zeros(H * dc, dtype=torch.float32, device="cuda")
+        nm.nm_debug_set_attention(impl)
+        try:
+            nm.nm_mla_attention(to_dev(Q), to_dev(cache), o16, o32, H, S, -1, dc, dr, scale, ws)
+            torch.cuda.synchronize()
+        finally:
+            nm.nm_debug_set_attention(0)
+        nm.nm_check_status()
+        got = o32.cpu().numpy().astype(np.float64).reshape(H, dc)
+        assert rel_max(got, ref) <= 2e-3, f"impl {impl}: {rel_max(got, ref):.2e}"
+
+
 # ---- the whole step ---------------------------------------------------------------------------------------
 
 def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None, concat_down=False):

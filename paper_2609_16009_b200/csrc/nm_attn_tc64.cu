@@ -95,7 +95,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return r;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __maxnreg__(120)
 attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ AttnSeqs64 seqs, AttnPartials part,
                  float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
 {

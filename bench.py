@@ -630,6 +630,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="also report GB/s of single narrow products vs M")
     ap.add_argument("--seq-len", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--attention", default="auto", choices=["auto", "64", "128", "cuda-cores"],
+                    help="attention kernel: chosen by length (default), tensor cores with 64 or 128 heads per CTA, CUDA cores")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -652,6 +654,7 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     import paper_2609_16009_b200 as nm
+    nm.nm_debug_set_attention({"auto": 0, "cuda-cores": 1, "128": 2, "64": 3}[args.attention])
     wl = make_workload(args, nm, device)
     stream = torch.cuda.Stream(device)
     if args.timeline:

@@ -75,61 +75,41 @@ __device__ __forceinline__ uint32_t pack2_bf16_rn(float lo, float hi)
     return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
 }
 
-// All threads of one CTA.  xs: the product's output row as fp32 values already rounded to bf16, in shared memory.
-__device__ __forceinline__ void vec_tail_run(const VecTail &t, const float *xs, float *scratch)
+__device__ __forceinline__ unsigned long long tail_timer_ns()
 {
-    const int tid = threadIdx.x;
-    if (t.q_lora > 0) {                                            // up to 8 elements per thread (q_lora <= 2048, multiple of 8)
-        const int i0 = 8 * tid;
-        const bool on = i0 < t.q_lora;
-        float f[8], g[8];
-        if (on) {
-            const float4 a = *reinterpret_cast<const float4 *>(xs + i0), b = *reinterpret_cast<const float4 *>(xs + i0 + 4);
-            f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
-            Elem<bf16_t>::unpack(__ldg(reinterpret_cast<const uint4 *>(t.gamma_q + i0)), g);
-        }
-        float ss = 0.f;
-        if (on)
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Two sums over the CTA at once (any size up to 1024 threads, a multiple of 32), same values in every thread.
+__device__ __forceinline__ float2 cta_sum2(float2 v, float *scratch /* 64 floats */)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
-        ss = cta_sum(ss, scratch);
-        const float r = 1.0f / sqrtf(ss / (float)t.q_lora + t.eps);
-        if (on) {
-            uint4 o;
-            o.x = pack2_bf16_rn(f[0] * r * g[0], f[1] * r * g[1]); o.y = pack2_bf16_rn(f[2] * r * g[2], f[3] * r * g[3]);
-            o.z = pack2_bf16_rn(f[4] * r * g[4], f[5] * r * g[5]); o.w = pack2_bf16_rn(f[6] * r * g[6], f[7] * r * g[7]);
-            *reinterpret_cast<uint4 *>(t.c_qn + i0) = o;
-        }
+    for (int o = 16; o > 0; o >>= 1) {
+        v.x += __shfl_xor_sync(0xffffffffu, v.x, o);
+        v.y += __shfl_xor_sync(0xffffffffu, v.y, o);
     }
-    if (t.dc > 0) {                                                // two elements per thread (dc <= 512, rope <= dc)
-        const float *ckr = xs + t.kv_off;
-        const int i0 = 2 * tid;
-        float x0 = 0.f, x1 = 0.f, g0 = 0.f, g1 = 0.f;
-        if (i0 < t.dc) {
-            const uint32_t gv = __ldg(reinterpret_cast<const uint32_t *>(t.gamma_kv + i0));
-            x0 = ckr[i0]; x1 = ckr[i0 + 1];
-            g0 = __uint_as_float(gv << 16); g1 = __uint_as_float(gv & 0xffff0000u);
-        }
-        float r0 = 0.f, r1 = 0.f, c = 0.f, sn = 0.f;
-        if (i0 < t.rope) {
-            r0 = ckr[t.dc + i0]; r1 = ckr[t.dc + i0 + 1];
-            c = t.cos_sin[i0]; sn = t.cos_sin[i0 + 1];
-        }
-        const float ss = cta_sum(fmaf(x0, x0, x1 * x1), scratch);
-        const float r = 1.0f / sqrtf(ss / (float)t.dc + t.eps);
-        if (i0 < t.dc) *reinterpret_cast<uint32_t *>(t.cache_row + i0) = pack2_bf16_rn(x0 * r * g0, x1 * r * g1);
-        if (i0 < t.rope) *reinterpret_cast<uint32_t *>(t.cache_row + t.dc + i0) = pack2_bf16_rn(r0 * c - r1 * sn, r0 * sn + r1 * c);
-    }
+    __syncthreads();
+    if (lane == 0) { scratch[2 * warp] = v.x; scratch[2 * warp + 1] = v.y; }
+    __syncthreads();
+    float2 t = make_float2(0.f, 0.f);
+    for (int w = 0; w < nw; ++w) { t.x += scratch[2 * w]; t.y += scratch[2 * w + 1]; }
+    return t;
 }
 
 // Completion of a product that carries a VecTail (M = 1, bf16 output, one head).  One arrival counter for the
 // whole grid instead of one per tile: every CTA publishes its tile (split-K: its fp32 partial tile; otherwise
 // the finished bf16 columns) and arrives; the last CTA of the grid gathers every column - partials summed in
 // split order, rounded once - writes C, keeps the rounded row in shared memory and runs the vector stages on
-// it.  One fence / atomic / load round trip through L2 in all, where a per-tile gather followed by a grid-wide
-// counter would take two (each such round trip costs 1-3 us here: the next product of the chain is filling its
-// ring from HBM at full rate at that very moment, and everything that crosses L2 queues behind it).  `xs` needs N floats (+32 of scratch behind them).
-__device__ __forceinline__ void tail_complete(const MatmulArgs &a, const VecTail &t, int *s_last, float *xs)
+// it: RMSNorm of the first q_lora outputs, RMSNorm + RoPE + cache-row write of the outputs from kv_off on.
+// Everything that crosses L2 here queues behind the next product of the chain, which is filling its ring from
+// HBM at full rate at that very moment (1-3 us per dependent round trip), so there are as few of them as the
+// data allows: one fence / atomic; then the constants of the vector stages and the partials of two passes of
+// columns are requested together; both sums of squares share one reduction.  `xs` needs N floats (+64 of
+// scratch behind them).
+__device__ __forceinline__ void tail_complete(const MatmulArgs &a, const VecTail &t, int *s_last, float *xs, unsigned long long *dbg = nullptr)
 {
     const int tid = threadIdx.x;
     __threadfence();
@@ -137,36 +117,101 @@ __device__ __forceinline__ void tail_complete(const MatmulArgs &a, const VecTail
     if (tid == 0) *s_last = (atomicAdd(t.counter, 1u) == (unsigned)(a.ntiles * a.nsplit - 1));
     __syncthreads();
     if (!*s_last) return;
+    if (dbg && tid == 0) dbg[0] = tail_timer_ns();
     __threadfence();
     if (tid == 0) *t.counter = 0u;
+    // constants of the vector stages (8 elements of q_lora <= 2048, 2 of dc <= 512 and of rope <= dc per thread)
+    const bool q_on = t.q_lora > 0 && 8 * tid < t.q_lora;
+    const bool kv_on = t.dc > 0 && 2 * tid < t.dc, rope_on = t.dc > 0 && 2 * tid < t.rope;
+    uint4 gq = make_uint4(0, 0, 0, 0);
+    uint32_t gkv = 0;
+    float cs = 0.f, sn = 0.f;
+    if (q_on) gq = __ldg(reinterpret_cast<const uint4 *>(t.gamma_q + 8 * tid));
+    if (kv_on) gkv = __ldg(reinterpret_cast<const uint32_t *>(t.gamma_kv + 2 * tid));
+    if (rope_on) { cs = __ldg(t.cos_sin + 2 * tid); sn = __ldg(t.cos_sin + 2 * tid + 1); }
+
     uint16_t *C = reinterpret_cast<uint16_t *>(a.C);
-    // four consecutive columns (one 16-byte load per split) per thread and pass; N and the tile width are
-    // multiples of four (checked by the host), so the four columns lie in one tile
-    for (int n = 4 * tid; n < a.N; n += 4 * (int)blockDim.x) {
-        float4 sum;
+    // four consecutive columns (one 16-byte load per split) per thread and pass, two passes requested at a time;
+    // N and the tile width are multiples of four (checked by the host), so the four columns lie in one tile
+    const int stride = 4 * (int)blockDim.x;
+    auto finish = [&](int n, float4 sum) {                         // round once, write C, keep the rounded values
+        const __nv_bfloat16 b0 = __float2bfloat16_rn(sum.x), b1 = __float2bfloat16_rn(sum.y), b2 = __float2bfloat16_rn(sum.z),
+                            b3 = __float2bfloat16_rn(sum.w);
+        *reinterpret_cast<uint2 *>(C + n) = make_uint2((uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16),
+                                                       (uint32_t)__bfloat16_as_ushort(b2) | ((uint32_t)__bfloat16_as_ushort(b3) << 16));
+        *reinterpret_cast<float4 *>(xs + n) = make_float4(__bfloat162float(b0), __bfloat162float(b1), __bfloat162float(b2), __bfloat162float(b3));
+    };
+    for (int n0 = 4 * tid; n0 < a.N; n0 += 2 * stride) {
+        const int n1 = n0 + stride;
+        const bool two = n1 < a.N;
         if (a.nsplit > 1) {
-            const int tile = n / a.tn, c = n - tile * a.tn;
-            const float *P = a.partial + (size_t)tile * a.nsplit * a.tn + c;
-            sum = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-            for (int sp = 0; sp < a.nsplit; ++sp) {               // split order: deterministic
-                const float4 v = __ldcg(reinterpret_cast<const float4 *>(P + (size_t)sp * a.tn));
-                sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+            const int nb = two ? n1 : n0;                          // without a second pass its loads repeat the first's
+            const int t0 = n0 / a.tn, t1 = nb / a.tn;
+            const float *P0 = a.partial + (size_t)t0 * a.nsplit * a.tn + (n0 - t0 * a.tn);
+            const float *P1 = a.partial + (size_t)t1 * a.nsplit * a.tn + (nb - t1 * a.tn);
+            float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+            for (int sp = 0; sp < a.nsplit; sp += 4) {
+                float4 v0[4], v1[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {                      // branch-free: a slot past the last split re-reads it
+                    const size_t off = (size_t)min(sp + u, a.nsplit - 1) * a.tn;
+                    v0[u] = __ldcg(reinterpret_cast<const float4 *>(P0 + off));
+                    v1[u] = __ldcg(reinterpret_cast<const float4 *>(P1 + off));
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)                        // split order: deterministic
+                    if (sp + u < a.nsplit) {
+                        s0.x += v0[u].x; s0.y += v0[u].y; s0.z += v0[u].z; s0.w += v0[u].w;
+                        s1.x += v1[u].x; s1.y += v1[u].y; s1.z += v1[u].z; s1.w += v1[u].w;
+                    }
             }
-            const __nv_bfloat16 b0 = __float2bfloat16_rn(sum.x), b1 = __float2bfloat16_rn(sum.y), b2 = __float2bfloat16_rn(sum.z),
-                                b3 = __float2bfloat16_rn(sum.w);
-            *reinterpret_cast<uint2 *>(C + n) = make_uint2((uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16),
-                                                           (uint32_t)__bfloat16_as_ushort(b2) | ((uint32_t)__bfloat16_as_ushort(b3) << 16));
-            sum = make_float4(__bfloat162float(b0), __bfloat162float(b1), __bfloat162float(b2), __bfloat162float(b3));
+            finish(n0, s0);
+            if (two) finish(n1, s1);
         } else {
-            const uint2 cv = __ldcg(reinterpret_cast<const uint2 *>(C + n));
-            sum = make_float4(__uint_as_float(cv.x << 16), __uint_as_float(cv.x & 0xffff0000u), __uint_as_float(cv.y << 16),
-                              __uint_as_float(cv.y & 0xffff0000u));
+            const uint2 c0 = __ldcg(reinterpret_cast<const uint2 *>(C + n0));
+            const uint2 c1 = __ldcg(reinterpret_cast<const uint2 *>(C + (two ? n1 : n0)));
+            *reinterpret_cast<float4 *>(xs + n0) = make_float4(__uint_as_float(c0.x << 16), __uint_as_float(c0.x & 0xffff0000u),
+                                                               __uint_as_float(c0.y << 16), __uint_as_float(c0.y & 0xffff0000u));
+            if (two)
+                *reinterpret_cast<float4 *>(xs + n1) = make_float4(__uint_as_float(c1.x << 16), __uint_as_float(c1.x & 0xffff0000u),
+                                                                   __uint_as_float(c1.y << 16), __uint_as_float(c1.y & 0xffff0000u));
         }
-        *reinterpret_cast<float4 *>(xs + n) = sum;
     }
+    if (dbg && tid == 0) dbg[1] = tail_timer_ns();
     __syncthreads();
-    vec_tail_run(t, xs, xs + ((a.N + 31) & ~31));
+    if (dbg && tid == 0) dbg[2] = tail_timer_ns();
+
+    // ---- the vector stages on the rounded row --------------------------------------------------------------
+    float f[8], g[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] = 0.f;
+    if (q_on) {
+        const float4 x = *reinterpret_cast<const float4 *>(xs + 8 * tid), y = *reinterpret_cast<const float4 *>(xs + 8 * tid + 4);
+        f[0] = x.x; f[1] = x.y; f[2] = x.z; f[3] = x.w; f[4] = y.x; f[5] = y.y; f[6] = y.z; f[7] = y.w;
+    }
+    Elem<bf16_t>::unpack(gq, g);
+    const float *ckr = xs + t.kv_off;
+    float x0 = 0.f, x1 = 0.f, r0 = 0.f, r1 = 0.f;
+    if (kv_on) { x0 = ckr[2 * tid]; x1 = ckr[2 * tid + 1]; }
+    if (rope_on) { r0 = ckr[t.dc + 2 * tid]; r1 = ckr[t.dc + 2 * tid + 1]; }
+    float ssq = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ssq = fmaf(f[e], f[e], ssq);
+    const float2 ss = cta_sum2(make_float2(ssq, fmaf(x0, x0, x1 * x1)), xs + ((a.N + 31) & ~31));
+    if (dbg && tid == 0) dbg[3] = tail_timer_ns();
+    if (q_on) {
+        const float r = 1.0f / sqrtf(ss.x / (float)t.q_lora + t.eps);
+        uint4 o;
+        o.x = pack2_bf16_rn(f[0] * r * g[0], f[1] * r * g[1]); o.y = pack2_bf16_rn(f[2] * r * g[2], f[3] * r * g[3]);
+        o.z = pack2_bf16_rn(f[4] * r * g[4], f[5] * r * g[5]); o.w = pack2_bf16_rn(f[6] * r * g[6], f[7] * r * g[7]);
+        *reinterpret_cast<uint4 *>(t.c_qn + 8 * tid) = o;
+    }
+    if (t.dc > 0) {
+        const float r = 1.0f / sqrtf(ss.y / (float)t.dc + t.eps);
+        const float g0 = __uint_as_float(gkv << 16), g1 = __uint_as_float(gkv & 0xffff0000u);
+        if (kv_on) *reinterpret_cast<uint32_t *>(t.cache_row + 2 * tid) = pack2_bf16_rn(x0 * r * g0, x1 * r * g1);
+        if (rope_on) *reinterpret_cast<uint32_t *>(t.cache_row + t.dc + 2 * tid) = pack2_bf16_rn(r0 * cs - r1 * sn, r0 * sn + r1 * cs);
+    }
 }
 
 template <int M> struct RowCfg {

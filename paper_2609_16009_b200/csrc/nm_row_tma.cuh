@@ -277,7 +277,7 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
     }
     if constexpr (M == 1 && sizeof(TO) == 2) {
         if (ta.tail.enabled) {
-            tail_complete(a, ta.tail, &s_last, reinterpret_cast<float *>(ring));
+            tail_complete(a, ta.tail, &s_last, reinterpret_cast<float *>(ring), ta.trace ? ta.trace + 4 * 160 : nullptr);
             if (trace && tid == 0) trace[3] = global_timer_ns();
             return;
         }

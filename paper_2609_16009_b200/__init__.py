@@ -103,6 +103,7 @@ _lib.nm_debug_set_step_pdl.argtypes = [_i]
 _lib.nm_debug_stream_read.argtypes = [_vp, _sz, _vp, _i, _vp]
 _lib.nm_debug_set_step_knobs.argtypes = [_i, _i]
 _lib.nm_debug_set_step_tails.argtypes = [_i]
+_lib.nm_debug_set_cluster_split.argtypes = [_i]
 _lib.nm_debug_set_step_plan.argtypes = [_i, _i, _i, _i]
 _lib.nm_debug_set_step_prefetch.argtypes = [_i]
 _lib.nm_debug_set_step_fusion.argtypes = [_i]
@@ -342,6 +343,10 @@ def nm_debug_set_step_prefetch(megabytes: int) -> None:
 
 def nm_debug_set_step_knobs(uv_programmatic: int = 1, prefetch_w_uv: int = 1) -> None:
     _check(_lib.nm_debug_set_step_knobs(int(uv_programmatic), int(prefetch_w_uv)), "nm_debug_set_step_knobs")
+
+
+def nm_debug_set_cluster_split(enable: bool) -> None:
+    _check(_lib.nm_debug_set_cluster_split(int(enable)), "nm_debug_set_cluster_split")
 
 
 def nm_debug_set_step_tails(enable: bool) -> None:

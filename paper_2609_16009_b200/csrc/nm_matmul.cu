@@ -35,6 +35,7 @@ int record_cuda_error(cudaError_t e, const char *where)
 static void *g_ws = nullptr;
 static size_t g_ws_bytes = 0;
 static int g_force_tn = 0, g_force_split = 0, g_force_kind = -1, g_force_stages = 0;
+static int g_cluster_split = 1;     // k-splits of a tile as a thread-block cluster when the plan allows
 static int g_use_pdl = 0;
 static int g_tc_min_m = 3;        // row-major bf16 products with M >= this (and >= 32 MB of weights) go to the swap-AB tensor-core kernel
 
@@ -94,6 +95,9 @@ static Plan make_tma_plan(int M, int N, int K, int H, bool chained = false)
     int ns = (int)((target + base / 2) / base);
     if (ns > K / 128) ns = K / 128;
     if (ns > K / (40 * M)) ns = K / (40 * M);          // partial sums stay below ~10 % of the weight bytes
+    // Up to eight splits meet inside a thread-block cluster (shared memory, no fence / counter / gather through L2);
+    // measured on the 7168 x 576 product: 8 splits that way 5.4 us, the 14 this rule would take otherwise 7.3 us.
+    if (g_cluster_split && M <= 8 && ns > 8) ns = 8;
     if (g_force_split > 0) ns = g_force_split;
     if (ns > kMaxSplit) ns = kMaxSplit;
     if (ns < 1) ns = 1;
@@ -338,7 +342,14 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
             ta.tail.counter = reinterpret_cast<unsigned *>(ws) + (kNumCounters - 1);     // the last counter is never a tile's
             if (tail_taken) *tail_taken = true;
         }
-        const size_t smem = (size_t)p.nstage * kt * p.tn * 2 + kAChunkFloats * sizeof(float) + 2 * p.nstage * sizeof(uint64_t);
+        size_t smem = (size_t)p.nstage * kt * p.tn * 2 + kAChunkFloats * sizeof(float) + 2 * p.nstage * sizeof(uint64_t);
+        // Split-K inside a cluster: up to eight splits (the portable cluster size) whose partial tiles fit 16 KB of
+        // the first CTA's shared memory meet there instead of in the workspace.
+        const size_t slot_bytes = (size_t)p.nsplit * M * p.tn * sizeof(float);
+        if (g_cluster_split && p.nsplit >= 2 && p.nsplit <= 8 && !ta.tail.enabled && slot_bytes <= 16384) {
+            ta.cluster_split = 1;
+            smem += 16 + slot_bytes;
+        }
         const bool f32out = (dtype == NM_BF16_F32OUT);
         if (p.tpr == 8)       e = f32out ? launch_row_tma<8, float>(*map, ta, smem, stream)  : launch_row_tma<8, bf16_t>(*map, ta, smem, stream);
         else if (p.tpr == 16) e = f32out ? launch_row_tma<16, float>(*map, ta, smem, stream) : launch_row_tma<16, bf16_t>(*map, ta, smem, stream);
@@ -477,6 +488,12 @@ int nm_debug_set_plan(int tile_n, int nsplit)
 {
     if (tile_n < 0 || nsplit < 0 || tile_n > kMaxTileN || nsplit > kMaxSplit) return NM_ERR_INVALID_ARG;
     g_force_tn = tile_n; g_force_split = nsplit;
+    return NM_OK;
+}
+
+int nm_debug_set_cluster_split(int enable)
+{
+    g_cluster_split = enable ? 1 : 0;
     return NM_OK;
 }
 

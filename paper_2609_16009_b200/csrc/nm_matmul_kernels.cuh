@@ -54,6 +54,7 @@ struct TmaArgs {
     unsigned *status;      // device status word
     unsigned long long *trace;   // tuning aid: when non-null every CTA stores four timestamps (start, inputs ready, loop done, end)
     VecTail tail;
+    int cluster_split;     // the k-splits of a tile form a thread-block cluster (1 x nsplit x 1): partial sums meet in shared memory
 };
 
 // Sum over the CTA (any size up to 1024 threads, a multiple of 32), same value in every thread.

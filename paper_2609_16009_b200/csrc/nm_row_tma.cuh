@@ -80,6 +80,9 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
     }
     __syncthreads();
     pdl_launch_dependents();
+    // Split-K inside a cluster: first half of a cluster barrier; once its second half has been waited for (before
+    // the partial sums are pushed) every peer is running, which writing into a peer's shared memory requires.
+    if (ta.cluster_split) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
     float2 acc[MP2 > 0 ? MP2 : 1][8];
     float acc1[8];
@@ -243,6 +246,13 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
     const int tx = tid % TPR, ty = tid / TPR;
     TO *C = (TO *)a.C + (long)h * a.strideC;
     float *P = a.partial ? a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * TN) : nullptr;
+    // cluster split-K: slot [split][m][c] in the shared memory of the cluster's first CTA, behind its barriers
+    float *slots = reinterpret_cast<float *>(bars + 2 * NS + 2);
+    uint32_t slot0 = 0;
+    if (ta.cluster_split) {
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(slot0) : "r"(smem_u32(slots + (size_t)split * (M * TN))), "r"(0));
+    }
 #pragma unroll
     for (int m0 = 0; m0 < M; m0 += MPASS) {
         if (m0 > 0) __syncthreads();
@@ -271,6 +281,7 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
 #pragma unroll 8
                 for (int g = 0; g < RG; ++g) s += red[(size_t)(g * MPASS + mm) * TN + c];
                 if (a.nsplit == 1) C[(long)m * a.ldc + n] = round_out<TO>(s);
+                else if (ta.cluster_split) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(slot0 + (uint32_t)(m * TN + c) * 4u), "f"(s) : "memory");
                 else               P[(size_t)m * TN + c] = s;
             }
         }
@@ -281,6 +292,24 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
             if (trace && tid == 0) trace[3] = global_timer_ns();
             return;
         }
+    }
+    if (ta.cluster_split) {
+        // every split's sums are in the first CTA's slots once the cluster barrier completes; that CTA adds them
+        // in split order and rounds once (no fence, counter or gather through L2)
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (split == 0) {
+            for (int i = tid; i < M * TN; i += kTmaThreads) {
+                const int m = i / TN, c = i - m * TN, n = tile * TN + c;
+                if (n < a.N) {
+                    float s = 0.f;
+                    for (int sp = 0; sp < a.nsplit; ++sp) s += slots[(size_t)sp * (M * TN) + i];
+                    C[(long)m * a.ldc + n] = round_out<TO>(s);
+                }
+            }
+        }
+        if (trace && tid == 0) trace[3] = global_timer_ns();
+        return;
     }
     if (a.nsplit > 1) splitk_complete<M, TO>(a, tile, h, &s_last);
     if (trace && tid == 0) trace[3] = global_timer_ns();
@@ -295,11 +324,20 @@ cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta, size_t sm
     cfg.blockDim = dim3(kTmaThreads);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (ta.use_pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    if (ta.cluster_split) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 1; attr[na].val.clusterDim.y = (unsigned)a.nsplit; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = ta.use_pdl ? 1 : 0;
+    cfg.numAttrs = na;
     switch (a.M) {
 #define NM_X(m)                                                                                           \
     case m: {                                                                                             \

@@ -65,9 +65,14 @@ def test_heuristic_spreads_the_paper_shape_over_the_gpu(lib):
     lib.nm_debug_set_plan(0, 0)
     for layout in (0, 1):
         assert lib.nm_debug_get_plan(1, 576, 7168, 1, 1, layout, 1, out) == 0
-        # measured optimum on B200 is 108-144 CTAs: enough splits to use most SMs, few enough that
-        # the gather of the partial sums stays short
-        assert 100 <= out[5] <= 320, "MatMul 2 shape must be split over most of the 148 SMs"
+        if layout == 0:
+            # row-major: eight k-splits per column tile, the most that can meet inside a thread-block cluster
+            # (measured 5.4 us against 7.3 us for 14 splits gathered through the workspace)
+            assert out[2] == 8 and out[5] == 72
+        else:
+            # column-major: measured optimum on B200 is 108-144 CTAs: enough splits to use most SMs, few enough
+            # that the gather of the partial sums stays short
+            assert 100 <= out[5] <= 320, "MatMul 2 shape must be split over most of the 148 SMs"
     # a shape that cannot use 16-byte loads falls back to the scalar kernel, unsplit
     assert lib.nm_debug_get_plan(1, 577, 7168, 1, 1, 0, 0, out) == 0
     assert out[0] == 2 and out[2] == 1

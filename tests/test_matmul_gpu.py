@@ -182,6 +182,35 @@ def test_tma_ring_every_m_and_tile(nm, M, tile_n):
     nm.nm_check_status()
 
 
+@pytest.mark.parametrize("M,tile_n", [(1, 64), (1, 256), (2, 128), (4, 64), (8, 64), (16, 64), (16, 128)])
+@pytest.mark.parametrize("nsplit", [2, 3, 5, 8, 9])
+def test_split_k_inside_a_cluster_matches_the_workspace_path(nm, M, tile_n, nsplit):
+    """Up to eight k-splits whose partial tiles fit 16 KB meet in the shared memory of a thread-block cluster; more,
+    or larger ones, go through the workspace.  Same summation order either way: identical bits, and parity with
+    the oracle.  K ends mid-stage and N mid-tile."""
+    K, N = 2500, 840
+    A, B = gen.narrow_bf16(M, K, N, seed=950 + M)
+    outs = []
+    for cluster in (True, False):
+        nm.nm_debug_set_plan(tile_n, nsplit)
+        nm.nm_debug_set_kernel(3, 0)
+        nm.nm_debug_set_cluster_split(cluster)
+        try:
+            assert nm.nm_debug_get_plan(M, N, K)["kind"] == 3
+            outs.append(run_case(nm, A, B, M, N, K, BF16, ROW, f"split-K M={M} tile_n={tile_n} nsplit={nsplit} cluster={cluster}"))
+        finally:
+            nm.nm_debug_set_plan(0, 0)
+            nm.nm_debug_set_kernel(-1, 0)
+            nm.nm_debug_set_cluster_split(True)
+    assert np.array_equal(outs[0], outs[1])
+    nm.nm_check_status()
+
+
+def test_paper_matmul_2_shape_takes_eight_splits_in_a_cluster(nm):
+    plan = nm.nm_debug_get_plan(1, 576, 7168)
+    assert plan["kind"] == 3 and plan["nsplit"] == 8
+
+
 @pytest.mark.parametrize("M", [1, 2, 5, 8, 9, 13, 16])
 @pytest.mark.parametrize("nsplit", [0, 1, 3])
 def test_tensor_core_swap_ab_kernel(nm, M, nsplit):

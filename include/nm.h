@@ -325,8 +325,10 @@ int nm_debug_set_attention_trace(void *device_buffer);
 /* Decode step tuning: launch the merge + W_UV kernel programmatically (default 1); include W_UV in the L2
  * prefetch (default 1). */
 int nm_debug_set_step_knobs(int uv_programmatic, int prefetch_w_uv);
-/* Decode step: 1 (default) runs RMSNorm / RoPE / the cache-row write inside the completion of the down-projection
- * products; 0 runs them as kernels of their own. */
+/* Decode step, the vector stages behind the down-projections (RMSNorm / RoPE / the cache-row write): 0 as kernels of
+ * their own; 1 (default) folded into the products - with the three down-projections stored as one matrix the k-splits
+ * meet inside clusters, W_UQR normalises its token row while loading it and the KV consumers ride in an extra CTA of
+ * the per-head query kernel; otherwise, and with 2 always, the CTA that completes the product's last tile runs them. */
 int nm_debug_set_step_tails(int enable);
 /* Decode step tuning: force (tile_n, nsplit, ring stages) of one of its products - which = 0 the down-projection,
  * 1 W_UQR, 2 W_O; zeros give the plan back to the planner. */

@@ -349,7 +349,7 @@ def nm_debug_set_cluster_split(enable: bool) -> None:
     _check(_lib.nm_debug_set_cluster_split(int(enable)), "nm_debug_set_cluster_split")
 
 
-def nm_debug_set_step_tails(enable: bool) -> None:
+def nm_debug_set_step_tails(enable: int) -> None:
     _check(_lib.nm_debug_set_step_tails(int(enable)), "nm_debug_set_step_tails")
 
 

@@ -81,11 +81,21 @@ __device__ __forceinline__ float ld_cg(const float *p) { return __ldcg(p); }
 // takes it (M = 1, bf16 output) - *tail_taken says whether it did, the caller launches them itself otherwise.
 // `chained`: the launch is one link of a programmatic chain of kernels (the decode step); the planner then
 // prefers one CTA per SM with a deep ring and fewer k-splits.  Defined in nm_matmul.cu.
+// `extras` (optional): per-tile sums of squares of the outputs (only the TMA ring kernel with its k-splits in a
+// cluster writes them, M = 1, bf16) and RMSNorm of the token row on load (TMA ring kernel, M = 1, bf16); the
+// *_taken flags and tile_n report what the plan does; with dry_run nothing is launched.
+struct MatmulExtras {
+    float *tile_ss = nullptr;
+    const struct RowNorm *norm = nullptr;
+    bool dry_run = false;
+    bool tile_ss_taken = false, norm_taken = false;
+    int tile_n = 0;
+};
 int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, int H,
                    long lda, long strideA, long strideB, long ldc, long strideC,
                    nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream,
                    bool programmatic_launch = false, unsigned long long *trace = nullptr, const struct VecTail *tail = nullptr,
-                   bool *tail_taken = nullptr, bool chained = false);
+                   bool *tail_taken = nullptr, bool chained = false, MatmulExtras *extras = nullptr);
 
 // How the row-major bf16 product K x N (H heads) at this M will be split: k-rows per split and splits.
 void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit, bool chained = false);

@@ -95,12 +95,38 @@ __device__ __forceinline__ uint4 pack8_bf16(const float (&v)[8])
 
 // q: [H][nope+rope] bf16; W_UK: [H][nope][dc]; q_full: [H][dc+rope] (q_lat | q_rope).  nope = 128, dc = 512.
 __global__ void __launch_bounds__(kHeadThreads) q_finish_kernel(const uint16_t *__restrict__ q, const uint16_t *__restrict__ W_UK,
-                                                                const float *__restrict__ cs, uint16_t *__restrict__ q_full, int rope)
+                                                                const float *__restrict__ cs, uint16_t *__restrict__ q_full, int rope,
+                                                                const KvFinish kv)
 {
     constexpr int K = 128, N = 512;
     using MV = HeadMatvec<K, N>;
     __shared__ __align__(16) float x_s[K];
     __shared__ __align__(16) float red[MV::kRowGroups * N];
+    if (kv.enabled && blockIdx.x == gridDim.x - 1) {
+        // the extra CTA: RMSNorm of the KV latent, RoPE of the key part, both into the new cache row (dc <= 512)
+        pdl_launch_dependents();
+        pdl_wait_prior_grids();
+        const int i0 = 2 * threadIdx.x;
+        float x0 = 0.f, x1 = 0.f, g0 = 0.f, g1 = 0.f, r0 = 0.f, r1 = 0.f, c = 0.f, sn = 0.f;
+        if (i0 < kv.dc) {
+            const uint32_t xv = *reinterpret_cast<const uint32_t *>(kv.ckr + i0), gv = *reinterpret_cast<const uint32_t *>(kv.gamma + i0);
+            x0 = __uint_as_float(xv << 16); x1 = __uint_as_float(xv & 0xffff0000u);
+            g0 = __uint_as_float(gv << 16); g1 = __uint_as_float(gv & 0xffff0000u);
+        }
+        if (i0 < kv.rope) {
+            const uint32_t rv = *reinterpret_cast<const uint32_t *>(kv.ckr + kv.dc + i0);
+            r0 = __uint_as_float(rv << 16); r1 = __uint_as_float(rv & 0xffff0000u);
+            c = kv.cos_sin[i0]; sn = kv.cos_sin[i0 + 1];
+        }
+        const float ss = block_sum_256(fmaf(x0, x0, x1 * x1), red);
+        const float r = 1.0f / sqrtf(ss / (float)kv.dc + kv.eps);
+        if (i0 < kv.dc)
+            *reinterpret_cast<uint32_t *>(kv.cache_row + i0) = (uint32_t)f32_to_bf16(x0 * r * g0) | ((uint32_t)f32_to_bf16(x1 * r * g1) << 16);
+        if (i0 < kv.rope)
+            *reinterpret_cast<uint32_t *>(kv.cache_row + kv.dc + i0) =
+                (uint32_t)f32_to_bf16(r0 * c - r1 * sn) | ((uint32_t)f32_to_bf16(r0 * sn + r1 * c) << 16);
+        return;
+    }
     const int h = blockIdx.x;
     const uint16_t *W = W_UK + (size_t)h * K * N;
     uint4 w[32];
@@ -396,9 +422,11 @@ int launch_down_finish(const void *x, const void *gamma_q, const void *gamma_kv,
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "down_finish launch");
 }
 
-int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl)
+int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl, KvFinish kv)
 {
-    cudaError_t e = launch_with_pdl(q_finish_kernel, H, s, pdl, (const uint16_t *)q, (const uint16_t *)W_UK, cos_sin, (uint16_t *)q_full, rope);
+    if (kv.enabled && (kv.dc > 2 * kHeadThreads || kv.rope > kv.dc || (kv.dc | kv.rope) % 2)) return NM_ERR_UNSUPPORTED;
+    cudaError_t e = launch_with_pdl(q_finish_kernel, H + (kv.enabled ? 1 : 0), s, pdl, (const uint16_t *)q, (const uint16_t *)W_UK, cos_sin,
+                                    (uint16_t *)q_full, rope, kv);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "q_finish launch");
 }
 

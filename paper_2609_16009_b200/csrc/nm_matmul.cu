@@ -279,9 +279,11 @@ static int check_common(const void *A, const void *B, const void *C, int M, int 
 static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int K, int H,
                        long lda, long strideA, long strideB, long ldc, long strideC,
                        nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream, bool pdl = false,
-                       unsigned long long *trace = nullptr, const VecTail *tail = nullptr, bool *tail_taken = nullptr, bool chained = false)
+                       unsigned long long *trace = nullptr, const VecTail *tail = nullptr, bool *tail_taken = nullptr, bool chained = false,
+                       MatmulExtras *extras = nullptr)
 {
     if (tail_taken) *tail_taken = false;
+    if (extras) { extras->tile_ss_taken = extras->norm_taken = false; extras->tile_n = 0; }
     int rc = check_common(A, B, C, M, N, K, H, dtype, layout);
     if (rc != NM_OK) return rc;
     if (lda < K || ldc < N || strideA < 0 || strideB < 0 || strideC < 0) return NM_ERR_INVALID_ARG;
@@ -322,6 +324,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         a.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + kCounterBytes);
     }
 
+    if (extras && extras->dry_run && p.kind != kRowTma) return NM_OK;
     cudaError_t e = cudaErrorInvalidValue;
     if (p.kind == kRowTc) {
         const CUtensorMap *mb = tc_map_b, *ma = tc_map_a;
@@ -349,6 +352,19 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         if (g_cluster_split && p.nsplit >= 2 && p.nsplit <= 8 && !ta.tail.enabled && slot_bytes <= 16384) {
             ta.cluster_split = 1;
             smem += 16 + slot_bytes;
+        }
+        if (extras) {
+            extras->tile_n = p.tn;
+            if (extras->tile_ss && ta.cluster_split && M == 1 && dtype == NM_BF16 && H == 1) {
+                ta.tile_ss = extras->tile_ss;
+                extras->tile_ss_taken = true;
+            }
+            if (extras->norm && extras->norm->enabled && M == 1 && dtype == NM_BF16 && H == 1 && extras->norm->ntiles <= 32 &&
+                extras->norm->n == K && K % 8 == 0) {
+                ta.norm = *extras->norm;
+                extras->norm_taken = true;
+            }
+            if (extras->dry_run) return NM_OK;
         }
         const bool f32out = (dtype == NM_BF16_F32OUT);
         if (p.tpr == 8)       e = f32out ? launch_row_tma<8, float>(*map, ta, smem, stream)  : launch_row_tma<8, bf16_t>(*map, ta, smem, stream);
@@ -382,10 +398,10 @@ void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, i
 int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, int H,
                    long lda, long strideA, long strideB, long ldc, long strideC,
                    nm_dtype dtype, nm_layout layout, void *ws, size_t ws_bytes, cudaStream_t stream, bool programmatic_launch,
-                   unsigned long long *trace, const VecTail *tail, bool *tail_taken, bool chained)
+                   unsigned long long *trace, const VecTail *tail, bool *tail_taken, bool chained, MatmulExtras *extras)
 {
     return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout, ws, ws_bytes, stream,
-                       programmatic_launch, trace, tail, tail_taken, chained);
+                       programmatic_launch, trace, tail, tail_taken, chained, extras);
 }
 
 }  // namespace nm

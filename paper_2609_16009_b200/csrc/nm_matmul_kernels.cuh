@@ -47,6 +47,19 @@ struct VecTail {
     unsigned *counter;                     // zero on entry, left at zero
 };
 
+// RMSNorm applied to the token row as it is loaded (M = 1): the producer of the row left the sum of squares of each
+// of its column tiles in `tile_ss`; the consumer adds them in tile order, scales the row by gamma / rms, rounds it to
+// bf16 - exactly what a separate RMSNorm stage would have stored - and multiplies that.
+struct RowNorm {
+    int enabled;
+    int n;                                 // elements of the row (= K of the product)
+    int ntiles;                            // entries of tile_ss (<= 32)
+    float eps;
+    const float *tile_ss;
+    const uint16_t *gamma;
+    uint16_t *normed_out;                  // when non-null, the CTAs of column tile 0 also store the normalised row here
+};
+
 struct TmaArgs {
     MatmulArgs base;
     int nstage;            // ring depth
@@ -55,6 +68,8 @@ struct TmaArgs {
     unsigned long long *trace;   // tuning aid: when non-null every CTA stores four timestamps (start, inputs ready, loop done, end)
     VecTail tail;
     int cluster_split;     // the k-splits of a tile form a thread-block cluster (1 x nsplit x 1): partial sums meet in shared memory
+    float *tile_ss;        // cluster split-K, M = 1: when non-null, tile t also stores the sum of squares of its rounded outputs at [t]
+    RowNorm norm;
 };
 
 // Sum over the CTA (any size up to 1024 threads, a multiple of 32), same value in every thread.

@@ -312,7 +312,8 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 // ---- host -------------------------------------------------------------------------------------------
 
 static int g_step_plan[3][3] = {};   // tuning: forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
-static int g_fused_tails = 1;        // run RMSNorm / RoPE / cache write inside the completion of the product that feeds them
+static int g_fused_tails = 1;        // 0: RMSNorm / RoPE / cache write as kernels of their own; 1: folded into the products (default);
+                                     // 2: as 1, but only in the form where the product's last CTA runs them
 static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
 static int g_fused_heads = 1;        // per-head stages fused with their vector stage (q_finish, uv_merge) when the dims allow
 static int g_uv_pdl = 1;             // tuning: launch uv_merge programmatically
@@ -403,7 +404,7 @@ static int attention_combine(const void *Q, const void *cache, void *o_bf16, flo
 // [attention partials][intermediates].  Each matmul workspace is [64 KB counters][partials].
 struct StepLayout {
     size_t main_ws, main_ws_bytes, side_ws, side_ws_bytes, attn, attn_bytes;
-    size_t c_q, c_qn, q, q_full, ckr, o_lat, o, x_down, total;
+    size_t c_q, c_qn, q, q_full, ckr, o_lat, o, x_down, tile_ss, total;
 };
 
 static StepLayout step_layout(const nm_mla_params *p)
@@ -426,6 +427,7 @@ static StepLayout step_layout(const nm_mla_params *p)
     L.c_q = take(p->q_lora); L.c_qn = take(p->q_lora); L.q = take((size_t)p->H * dq); L.q_full = take((size_t)p->H * dkv);
     L.ckr = take(dkv); L.o_lat = take((size_t)p->H * p->kv_lora); L.o = take((size_t)p->H * p->v);
     L.x_down = take((size_t)p->q_lora + dkv);
+    L.tile_ss = take(2 * (size_t)(ceil_div(p->q_lora + dkv, 64) + 64));     // one float per 64-column tile of the fused down-projection
     L.total = off;
     return L;
 }
@@ -505,7 +507,48 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     tkv.cos_sin = p->rope_cos_sin; tkv.cache_row = cache + (size_t)pos * dkv;
     bool taken = false;
     const bool fused_down = p->W_DQKV && lay == NM_ROW_MAJOR && down_finish_applies(ql, dc, dr);
-    if (fused_down) {
+    // Where the plans allow: the k-splits of the fused down-projection meet inside clusters, each
+    // tile leaves the sum of squares of its outputs, the W_UQR product applies RMSNorm to its token row while
+    // loading it, and the KV consumers ride in an extra CTA of the per-head query kernel - the down-projection then
+    // ends without a grid-wide gather, which cost it 4 us at the head of the step's critical path.
+    bool split_norm = false;
+    RowNorm rn{};
+    KvFinish kvf{};
+    float *tile_ss = reinterpret_cast<float *>(ws + L.tile_ss);
+    if (fused_down && tails_ok && g_fused_tails == 1 && g_fused_heads && head_kernels_apply(H, dn, dr, dc, dv)) {
+        uint16_t *x_down = reinterpret_cast<uint16_t *>(ws + L.x_down);
+        MatmulExtras ex_d, ex_u;
+        ex_d.tile_ss = tile_ss; ex_d.dry_run = true;
+        {
+            ScopedPlan sp(g_step_plan[0]);
+            NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws,
+                                  L.main_ws_bytes, ms, false, nullptr, nullptr, nullptr, true, &ex_d));
+        }
+        if (ex_d.tile_ss_taken && ex_d.tile_n > 0 && ql % ex_d.tile_n == 0 && ql / ex_d.tile_n <= 32) {
+            rn.enabled = 1; rn.n = ql; rn.ntiles = ql / ex_d.tile_n; rn.eps = p->rms_eps; rn.tile_ss = tile_ss;
+            rn.gamma = (const uint16_t *)p->gamma_q; rn.normed_out = c_qn;
+            ex_u.norm = &rn; ex_u.dry_run = true;
+            ScopedPlan sp(g_step_plan[1]);
+            NM_TRY(matmul_enqueue(x_down, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, false,
+                                  nullptr, nullptr, nullptr, true, &ex_u));
+            split_norm = ex_u.norm_taken;
+        }
+    }
+    if (split_norm) {
+        uint16_t *x_down = reinterpret_cast<uint16_t *>(ws + L.x_down);
+        MatmulExtras ex_d;
+        ex_d.tile_ss = tile_ss;
+        {
+            ScopedPlan sp(g_step_plan[0]);
+            NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws,
+                                  L.main_ws_bytes, ms, pdl && p->programmatic_entry, trace_at(2048), nullptr, nullptr, true, &ex_d));
+        }
+        if (!ex_d.tile_ss_taken) return NM_ERR_UNSUPPORTED;        // the dry run said otherwise
+        kvf.enabled = 1; kvf.ckr = x_down + ql; kvf.gamma = (const uint16_t *)p->gamma_kv; kvf.cos_sin = p->rope_cos_sin;
+        kvf.cache_row = cache + (size_t)pos * dkv; kvf.dc = dc; kvf.rope = dr; kvf.eps = p->rms_eps;
+        if (p->c_q) NM_CUDA_TRY(cudaMemcpyAsync(p->c_q, x_down, (size_t)ql * 2, cudaMemcpyDeviceToDevice, ms));
+        if (p->ckr) NM_CUDA_TRY(cudaMemcpyAsync(p->ckr, x_down + ql, (size_t)dkv * 2, cudaMemcpyDeviceToDevice, ms));
+    } else if (fused_down) {
         // ---- one product for all three down-projections, h * (W_DQ | W_DKV | W_KR) (Eq. 3 extended by W_DQ),
         //      with both vector stages in its completion: no side stream, an unbroken programmatic chain
         uint16_t *x_down = reinterpret_cast<uint16_t *>(ws + L.x_down);
@@ -541,12 +584,17 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     }
     {
         ScopedPlan sp(g_step_plan[1]);
-        NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl, trace_at(4096), nullptr, nullptr, true));
+        MatmulExtras ex_u;
+        ex_u.norm = &rn;
+        const uint16_t *a_row = split_norm ? reinterpret_cast<const uint16_t *>(ws + L.x_down) : c_qn;
+        NM_TRY(matmul_enqueue(a_row, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, pdl, trace_at(4096),
+                              nullptr, nullptr, true, split_norm ? &ex_u : nullptr));
+        if (split_norm && !ex_u.norm_taken) return NM_ERR_UNSUPPORTED;
     }
     const bool fused = g_fused_heads && head_kernels_apply(H, dn, dr, dc, dv);
     if (fused) {
         // RoPE of the rope part and q_lat[h] = q[h, :nope] * W_UK[h] in one kernel, one CTA per head
-        NM_TRY(launch_q_finish(q, p->W_UK, p->rope_cos_sin, q_full, H, dr, ms, pdl));
+        NM_TRY(launch_q_finish(q, p->W_UK, p->rope_cos_sin, q_full, H, dr, ms, pdl, kvf));
     } else {
         NM_LAUNCH(rope_kernel, ceil_div(H * dr / 2, 256), 256, ms, (const uint16_t *)(q + dn), q_full + dc, H, dr, (long)dq, (long)dkv,
                   p->rope_cos_sin);
@@ -839,7 +887,7 @@ int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages)
  * kernels of their own. */
 int nm_debug_set_step_tails(int enable)
 {
-    g_fused_tails = enable ? 1 : 0;
+    g_fused_tails = enable < 0 ? 0 : (enable > 2 ? 2 : enable);
     return NM_OK;
 }
 

@@ -55,7 +55,20 @@ bool head_kernels_apply(int H, int nope, int rope, int dc, int dv);
 bool down_finish_applies(int q_lora, int dc, int rope);
 int launch_down_finish(const void *x, const void *gamma_q, const void *gamma_kv, const float *cos_sin, void *c_qn, void *cache_row,
                        int q_lora, int dc, int rope, float eps, cudaStream_t s, bool pdl);
-int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl);
+// Consumers of the KV part of the down-projection (RMSNorm of the latent, RoPE of the key part, the cache-row
+// write) for one extra CTA of the per-head query kernel: they are not needed before the attention merge, so they
+// ride along there instead of ending the down-projection.
+struct KvFinish {
+    int enabled;
+    const uint16_t *ckr;                   // [dc + rope] raw outputs of h * (W_DKV | W_KR)
+    const uint16_t *gamma;
+    const float *cos_sin;
+    uint16_t *cache_row;
+    int dc, rope;
+    float eps;
+};
+int launch_q_finish(const void *q, const void *W_UK, const float *cos_sin, void *q_full, int H, int rope, cudaStream_t s, bool pdl,
+                    KvFinish kv = KvFinish{});
 int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npart, long extra_row, int rope, float scale,
                     const void *W_UV, void *o_lat_bf16, float *o_lat_f32, void *o, int H, cudaStream_t s, bool pdl,
                     L2Prefetch prefetch = L2Prefetch{});

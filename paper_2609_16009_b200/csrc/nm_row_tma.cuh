@@ -123,16 +123,29 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
         }
         if (MP != M)
             for (int i = tid; i < kAChunkFloats; i += kTmaConsumers) As[i] = 0.f;
+        if constexpr (M == 1 && sizeof(TO) == 2) {
+            // the RMSNorm weights are read once per step and are long gone from L2: ask for them before the wait
+            if (ta.norm.enabled && tid * 64 < ta.norm.n) asm volatile("prefetch.global.L2 [%0];" ::"l"(ta.norm.gamma + tid * 64));
+        }
         pdl_wait_prior_grids();                       // A (and the workspace) come from earlier kernels
 
+        constexpr bool kCanNorm = (M == 1 && sizeof(TO) == 2);
+        const bool norm_on = kCanNorm && ta.norm.enabled;
         uint4 apre[GPT];
+        uint4 gpre[kCanNorm ? GPT : 1];
+        float rnorm = 1.f;
+        int norm_k0 = 0;                              // first k of the chunk held in apre
         auto fetch_chunk = [&](int kc) {              // global -> registers
+            norm_k0 = kc;
 #pragma unroll
             for (int g = 0; g < GPT; ++g) {
                 const int grp = tid + g * kTmaConsumers;
                 const int m = grp % M, kg = grp / M;
                 const int k = kc + kg * 8;
                 uint4 v = make_uint4(0, 0, 0, 0);
+                if constexpr (kCanNorm) {
+                    if (norm_on) gpre[g] = (grp < GROUPS && k + 8 <= a.K) ? __ldg(reinterpret_cast<const uint4 *>(ta.norm.gamma + k)) : make_uint4(0, 0, 0, 0);
+                }
                 if (grp < GROUPS && k < ke) {
                     const bf16_t *src = A + (long)m * a.lda + k;
                     if (k + 8 <= a.K) {
@@ -156,6 +169,18 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
                     const int m = grp % M, kg = grp / M;
                     float f[8];
                     Elem<bf16_t>::unpack(apre[g], f);
+                    if constexpr (kCanNorm) {
+                        if (norm_on) {                               // x * r * gamma, rounded to bf16 as a stored row would be
+                            float gm[8];
+                            Elem<bf16_t>::unpack(gpre[g], gm);
+                            uint4 o;
+                            o.x = pack2_bf16_rn(f[0] * rnorm * gm[0], f[1] * rnorm * gm[1]); o.y = pack2_bf16_rn(f[2] * rnorm * gm[2], f[3] * rnorm * gm[3]);
+                            o.z = pack2_bf16_rn(f[4] * rnorm * gm[4], f[5] * rnorm * gm[5]); o.w = pack2_bf16_rn(f[6] * rnorm * gm[6], f[7] * rnorm * gm[7]);
+                            Elem<bf16_t>::unpack(o, f);
+                            if (ta.norm.normed_out && (blockIdx.x | blockIdx.z) == 0 && norm_k0 + kg * 8 < ke)     // this split's rows only
+                                *reinterpret_cast<uint4 *>(ta.norm.normed_out + norm_k0 + kg * 8) = o;
+                        }
+                    }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) As[(kg * 8 + i) * MP + m] = f[i];
                 }
@@ -163,6 +188,15 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
         };
         if (MP != M) named_barrier_sync(1, kTmaConsumers);
         fetch_chunk(kb);
+        if constexpr (kCanNorm) {
+            if (norm_on) {
+                // 1 / rms of the row from the per-tile sums of squares, added in tile order by every warp for itself
+                const float v = (lane < ta.norm.ntiles) ? ld_cg(ta.norm.tile_ss + lane) : 0.f;
+                float tot = 0.f;
+                for (int l = 0; l < ta.norm.ntiles; ++l) tot += __shfl_sync(0xffffffffu, v, l);
+                rnorm = 1.0f / sqrtf(tot / (float)ta.norm.n + ta.norm.eps);
+            }
+        }
         store_chunk();
         named_barrier_sync(1, kTmaConsumers);
         if (trace && tid == 0) trace[1] = global_timer_ns();
@@ -299,12 +333,29 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
         asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         if (split == 0) {
+            float sq = 0.f;                                        // M = 1, TN <= 256: at most one output per thread
             for (int i = tid; i < M * TN; i += kTmaThreads) {
                 const int m = i / TN, c = i - m * TN, n = tile * TN + c;
                 if (n < a.N) {
                     float s = 0.f;
                     for (int sp = 0; sp < a.nsplit; ++sp) s += slots[(size_t)sp * (M * TN) + i];
-                    C[(long)m * a.ldc + n] = round_out<TO>(s);
+                    const TO r = round_out<TO>(s);
+                    C[(long)m * a.ldc + n] = r;
+                    if constexpr (M == 1 && sizeof(TO) == 2) { const float rv = Elem<bf16_t>::widen(r); sq = rv * rv; }
+                }
+            }
+            if constexpr (M == 1 && sizeof(TO) == 2) {
+                if (ta.tile_ss) {                                  // sum of squares of the tile's rounded outputs, fixed order
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                    float *scr = reinterpret_cast<float *>(ring);
+                    if (lane == 0) scr[warp] = sq;
+                    __syncthreads();
+                    if (tid == 0) {
+                        float t = 0.f;
+                        for (int w = 0; w < kTmaThreads / 32; ++w) t += scr[w];
+                        ta.tile_ss[tile] = t;
+                    }
                 }
             }
         }

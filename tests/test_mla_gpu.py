@@ -339,22 +339,26 @@ def test_decode_step_vector_stages_inside_and_outside_the_products_agree(nm, wei
     w, dw = weights
     h, cache_ref, r = ref1024
     cache_in = gen.mla_cache(1024, DIMS, seed=4200)
+    # three forms: 1 (default) - with the down-projections stored as one matrix: k-splits meeting in clusters, RMSNorm of
+    # the query latent applied by W_UQR while loading its row, KV consumers in an extra CTA of the per-head query
+    # kernel; 2 - the CTA completing the product's last tile runs the stages; 0 - kernels of their own
     t1 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
     check_step(t1, r, cache_ref, 1024)
-    nm.nm_debug_set_step_tails(False)
-    try:
-        t2 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
-        check_step(t2, r, cache_ref, 1024)
-    finally:
-        nm.nm_debug_set_step_tails(True)
-    # the products are bit-identical (same plan, same summation order); the norms sum their squares in a
-    # different order, so c_qn and the cache row may differ by a rounding flip
-    for k in ("c_q", "ckr"):
-        assert torch.equal(t1[k], t2[k]), k
-    for k in ("c_qn", "kv_cache"):
-        a, b = dev_bits_to_f64(t1[k]), dev_bits_to_f64(t2[k])
-        assert np.all(np.abs(a - b) <= oracle.ulp_bf16(b) + 1e-6), k
-        assert np.mean(a == b) > 0.99, k
+    for mode in (2, 0):
+        nm.nm_debug_set_step_tails(mode)
+        try:
+            t2 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
+            check_step(t2, r, cache_ref, 1024)
+        finally:
+            nm.nm_debug_set_step_tails(1)
+        # the products are bit-identical (same summation order); the norms sum their squares in a
+        # different order, so c_qn and the cache row may differ by a rounding flip
+        for k in ("c_q", "ckr"):
+            assert torch.equal(t1[k], t2[k]), (mode, k)
+        for k in ("c_qn", "kv_cache"):
+            a, b = dev_bits_to_f64(t1[k]), dev_bits_to_f64(t2[k])
+            assert np.all(np.abs(a - b) <= oracle.ulp_bf16(b) + 1e-6), (mode, k)
+            assert np.mean(a == b) > 0.99, (mode, k)
 
 
 def test_decode_step_forced_product_plans_inside_the_step(nm, weights, ref1024):

@@ -311,9 +311,9 @@ int nm_debug_set_plan(int tile_n, int nsplit);
 /* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel; 3 TMA-ring
  * CUDA-core kernel; 4 swap-AB tensor-core kernel) and the ring depth in stages (0 heuristic). */
 int nm_debug_set_kernel(int kind, int stages);
-/* Split-K of the TMA-ring kernel: 1 (default) lets the k-splits of a column tile form a thread-block cluster whose
- * partial sums meet in the first CTA's shared memory (up to 8 splits, partial tiles up to 16 KB); 0 always goes
- * through the workspace (partial tiles, arrival counter, gather). */
+/* Split-K of the CUDA-core kernels: 1 (default) lets the k-splits of a column tile form a thread-block cluster whose
+ * partial sums meet in the first CTA's shared memory (up to 8 splits; partial tiles up to 16 KB in the TMA-ring
+ * kernel, 8 KB in the plain kernels); 0 always goes through the workspace (partial tiles, arrival counter, gather). */
 int nm_debug_set_cluster_split(int enable);
 /* Tuning aid: phase timestamps (ns, %globaltimer) of the decode step's kernels go to `device_buffer` (8192
  * unsigned 64-bit values) when non-null: [0,32) phases of CTA (0,0) of the attention kernel (the 64-head kernel:

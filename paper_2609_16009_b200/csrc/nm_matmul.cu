@@ -211,6 +211,7 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     const int min_kr = (p.kind == kRowVec) ? 2 * p.rg : 512;
     if (nsplit > K / min_kr) nsplit = K / min_kr;
     if (nsplit > K / (40 * M)) nsplit = K / (40 * M);
+    if (g_cluster_split && M <= 8 && nsplit > 8 && 8L * M * p.tn <= kClusterSlotFloats) nsplit = 8;     // the most that meet inside a cluster
     if (g_force_split > 0) nsplit = g_force_split;
     if (nsplit > kMaxSplit) nsplit = kMaxSplit;
     if (nsplit < 1) nsplit = 1;
@@ -325,6 +326,9 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     }
 
     if (extras && extras->dry_run && p.kind != kRowTma) return NM_OK;
+    if ((p.kind == kRowVec || p.kind == kColVec) && g_cluster_split && p.nsplit >= 2 && p.nsplit <= 8 &&
+        (long)p.nsplit * M * p.tn <= kClusterSlotFloats)
+        a.cluster_split = 1;
     cudaError_t e = cudaErrorInvalidValue;
     if (p.kind == kRowTc) {
         const CUtensorMap *mb = tc_map_b, *ma = tc_map_a;

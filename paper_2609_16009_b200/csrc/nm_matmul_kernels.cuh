@@ -29,7 +29,45 @@ struct MatmulArgs {
     int a_vec;     // A rows can be staged with 16-byte loads
     float *partial;
     unsigned *counters;
+    int cluster_split;   // plain kernels: the k-splits of a tile form a cluster (1 x nsplit x 1) and meet in shared memory
 };
+
+// ---- split-K inside a thread-block cluster (plain kernels) ----------------------------------------------
+// The k-splits of a column tile are the CTAs of one cluster.  Each stores its sums into slot [split] of the first
+// CTA's shared memory; after a cluster barrier that CTA adds the slots in split order, rounds once and writes C:
+// no workspace, fence, counter or gather through L2.  Every CTA arrives on the cluster barrier at its start and
+// waits for it before the first remote store (all peers are running by then).
+constexpr int kClusterSlotFloats = 2048;                           // 8 KB: nsplit * M * tile_n floats at most
+__device__ __forceinline__ void cluster_arrive_all() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_all() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t cluster_slot_base(const float *slots, int split, int per_split)
+{
+    uint32_t local = (uint32_t)__cvta_generic_to_shared(slots + (size_t)split * per_split), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(0));
+    return remote;
+}
+__device__ __forceinline__ void cluster_slot_store(uint32_t base, int i, float v)
+{
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(base + (uint32_t)i * 4u), "f"(v) : "memory");
+}
+// all threads of every CTA of the cluster, after the remote stores
+template <typename TO>
+__device__ __forceinline__ void cluster_split_finish(const MatmulArgs &a, const float *slots, int M, int tile, int split, int h)
+{
+    cluster_arrive_all();
+    cluster_wait_all();
+    if (split != 0) return;
+    TO *C = (TO *)a.C + (long)h * a.strideC;
+    const int per = M * a.tn;
+    for (int i = threadIdx.x; i < per; i += (int)blockDim.x) {
+        const int m = i / a.tn, c = i - m * a.tn, n = tile * a.tn + c;
+        if (n < a.N) {
+            float s = 0.f;
+            for (int sp = 0; sp < a.nsplit; ++sp) s += slots[(size_t)sp * per + i];
+            C[(long)m * a.ldc + n] = round_out<TO>(s);
+        }
+    }
+}
 
 // Extra launch state of the TMA-fed kernels.
 // The vector stages that consume a down-projection of the decode step, run by whichever CTA completes the
@@ -356,7 +394,9 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
     constexpr int KC = RowCfg<M>::kChunk;
     constexpr int MP = RowCfg<M>::kPass;
     __shared__ __align__(16) float smem[kSmemFloats];
+    __shared__ __align__(16) float s_slots[kClusterSlotFloats];
     __shared__ int s_last;
+    if (a.cluster_split) cluster_arrive_all();
 
     const int tid = threadIdx.x;
     const int tx = tid % a.tpr, ty = tid / a.tpr;
@@ -429,6 +469,11 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
     float *red = smem;
     TO *C = (TO *)a.C + (long)h * a.strideC;
     float *P = a.partial ? a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * a.tn) : nullptr;
+    uint32_t slot0 = 0;
+    if (a.cluster_split) {
+        cluster_wait_all();
+        slot0 = cluster_slot_base(s_slots, split, M * a.tn);
+    }
 #pragma unroll
     for (int m0 = 0; m0 < M; m0 += MP) {
         __syncthreads();
@@ -450,10 +495,12 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
                 float s = 0.f;
                 for (int g = 0; g < rg; ++g) s += red[(size_t)(g * MP + mm) * a.tn + c];
                 if (a.nsplit == 1) C[(long)m * a.ldc + n] = round_out<TO>(s);
+                else if (a.cluster_split) cluster_slot_store(slot0, m * a.tn + c, s);
                 else               P[(size_t)m * a.tn + c] = s;
             }
         }
     }
+    if (a.cluster_split) { cluster_split_finish<TO>(a, s_slots, M, tile, split, h); return; }
     if (a.nsplit > 1) splitk_complete<M, TO>(a, tile, h, &s_last);
 }
 
@@ -474,7 +521,9 @@ __global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
     // A chunk kept in its storage type: M x KC elements in 32 KB
     constexpr int KC = (((kSmemFloats * 4 / (int)sizeof(TI)) / M) / STEP) * STEP;
     __shared__ __align__(16) float smem[kSmemFloats];
+    __shared__ __align__(16) float s_slots[kClusterSlotFloats];
     __shared__ int s_last;
+    if (a.cluster_split) cluster_arrive_all();
     uint4 *As = (uint4 *)smem;                                     // [M][KC / V] 16-byte vectors
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -555,17 +604,25 @@ __global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
             for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             if (lane == m * CW + c) mine = s;
         }
+    uint32_t slot0 = 0;
+    if (a.cluster_split) {
+        cluster_wait_all();
+        slot0 = cluster_slot_base(s_slots, split, M * a.tn);
+    }
     if (lane < M * CW) {
         const int m = lane / CW, c = lane - m * CW, n = col0 + c;
         if (n < a.N) {
             if (a.nsplit == 1) {
                 ((TO *)a.C + (long)h * a.strideC)[(long)m * a.ldc + n] = round_out<TO>(mine);
+            } else if (a.cluster_split) {
+                cluster_slot_store(slot0, m * a.tn + warp * CW + c, mine);
             } else {
                 float *P = a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * a.tn);
                 P[(size_t)m * a.tn + warp * CW + c] = mine;
             }
         }
     }
+    if (a.cluster_split) { cluster_split_finish<TO>(a, s_slots, M, tile, split, h); return; }
     if (a.nsplit > 1) splitk_complete<M, TO>(a, tile, h, &s_last);
 }
 
@@ -599,27 +656,41 @@ __global__ void __launch_bounds__(kThreads) nm_generic_kernel(const MatmulArgs a
 template <typename TI, typename TO>
 cudaError_t launch_row(const MatmulArgs &a, cudaStream_t s)
 {
-    dim3 grid(a.ntiles, a.nsplit, a.H);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.ntiles, a.nsplit, a.H);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)a.nsplit; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.cluster_split ? 1 : 0;
     switch (a.M) {
-#define NM_X(m) case m: nm_row_kernel<m, TI, TO><<<grid, kThreads, 0, s>>>(a); break;
+#define NM_X(m) case m: return cudaLaunchKernelEx(&cfg, nm_row_kernel<m, TI, TO>, a);
         NM_FOR_EACH_M(NM_X)
 #undef NM_X
     default: return cudaErrorInvalidValue;
     }
-    return cudaGetLastError();
 }
 
 template <typename TI, typename TO>
 cudaError_t launch_col(const MatmulArgs &a, cudaStream_t s)
 {
-    dim3 grid(a.ntiles, a.nsplit, a.H);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.ntiles, a.nsplit, a.H);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)a.nsplit; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.cluster_split ? 1 : 0;
     switch (a.M) {
-#define NM_X(m) case m: nm_col_kernel<m, TI, TO><<<grid, kThreads, 0, s>>>(a); break;
+#define NM_X(m) case m: return cudaLaunchKernelEx(&cfg, nm_col_kernel<m, TI, TO>, a);
         NM_FOR_EACH_M(NM_X)
 #undef NM_X
     default: return cudaErrorInvalidValue;
     }
-    return cudaGetLastError();
 }
 
 template <typename TI, typename TO>

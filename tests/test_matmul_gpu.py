@@ -206,6 +206,29 @@ def test_split_k_inside_a_cluster_matches_the_workspace_path(nm, M, tile_n, nspl
     nm.nm_check_status()
 
 
+@pytest.mark.parametrize("layout,dtype", [(ROW, BF16), (ROW, F32), (COL, BF16), (COL, F32)])
+@pytest.mark.parametrize("M,nsplit", [(1, 2), (1, 8), (2, 5), (4, 8), (7, 3), (16, 2), (16, 4), (3, 9)])
+def test_split_k_inside_a_cluster_plain_kernels(nm, layout, dtype, M, nsplit):
+    """The plain row-major kernel and the column-major kernel: k-splits meeting in a cluster (up to eight, 8 KB of
+    partial tiles) against the workspace path - identical bits, parity with the oracle."""
+    K, N = 2056, 328
+    A, B = make_inputs(M, K, N, dtype, seed=970 + M)
+    outs = []
+    for cluster in (True, False):
+        nm.nm_debug_set_plan(0, nsplit)
+        nm.nm_debug_set_kernel(0, 0)
+        nm.nm_debug_set_cluster_split(cluster)
+        try:
+            assert nm.nm_debug_get_plan(M, N, K, 1, dtype, layout)["kind"] == (0 if layout == ROW else 1)
+            outs.append(run_case(nm, A, B, M, N, K, dtype, layout, f"plain split-K M={M} nsplit={nsplit} layout={layout} cluster={cluster}"))
+        finally:
+            nm.nm_debug_set_plan(0, 0)
+            nm.nm_debug_set_kernel(-1, 0)
+            nm.nm_debug_set_cluster_split(True)
+    assert np.array_equal(outs[0], outs[1])
+    nm.nm_check_status()
+
+
 def test_paper_matmul_2_shape_takes_eight_splits_in_a_cluster(nm):
     plan = nm.nm_debug_get_plan(1, 576, 7168)
     assert plan["kind"] == 3 and plan["nsplit"] == 8

@@ -45,10 +45,17 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
     import paper_2609_16009_b200 as nm
     nm.nm_debug_set_plan(0, 0)
     nm.nm_debug_set_kernel(-1, 0)
-    # first call: the paper's MatMul 2 shape; second call: another shape, layout and M, reusing the array
-    _both(nm, 1, 576, 7168, BF16, ROW, seed=9100)
-    _both(nm, 3, 1536, 7168, BF16_F32OUT, COL, seed=9200)
-    _both(nm, 1, 576, 7168, BF16, ROW, seed=9300)
+    # with the k-splits gathered through the scratch array (the case this entry point exists for), then as the
+    # library runs by default (up to eight splits meet inside a cluster and leave the array alone)
+    for cluster in (False, True):
+        nm.nm_debug_set_cluster_split(cluster)
+        try:
+            # first call: the paper's MatMul 2 shape; second call: another shape, layout and M, reusing the array
+            _both(nm, 1, 576, 7168, BF16, ROW, seed=9100)
+            _both(nm, 3, 1536, 7168, BF16_F32OUT, COL, seed=9200)
+            _both(nm, 1, 576, 7168, BF16, ROW, seed=9300)
+        finally:
+            nm.nm_debug_set_cluster_split(True)
     nm.nm_check_status()
 
 

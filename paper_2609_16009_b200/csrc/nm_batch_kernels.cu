@@ -293,6 +293,89 @@ __global__ void __launch_bounds__(kThreadsB) uv_merge_batch_kernel(const uint16_
     }
 }
 
+// ---- the same two stages without the per-head products, for batches large enough that those products belong on
+//      the tensor cores (the batched swap-AB kernel): RoPE of every token's query heads, and the merge alone ------
+
+// grid (T): q_full[t, h, dc:] = RoPE(q[t, h, nope:]) for every head.
+__global__ void __launch_bounds__(kThreadsB) rope_batch_kernel(const uint16_t *__restrict__ q, const float *__restrict__ cs,
+                                                               uint16_t *__restrict__ q_full, int H, int nope, int dc, int rope)
+{
+    const int t = blockIdx.x, half = rope / 2;
+    pdl_launch_dependents();
+    pdl_wait_prior_grids();                                       // q comes from the W_UQR product
+    for (int i = threadIdx.x; i < H * half; i += kThreadsB) {
+        const int h = i / half, pr = i - h * half;
+        const uint32_t xv = *reinterpret_cast<const uint32_t *>(q + ((size_t)t * H + h) * (nope + rope) + nope + 2 * pr);
+        const float2 c = *reinterpret_cast<const float2 *>(cs + (size_t)t * rope + 2 * pr);
+        const float x0 = __uint_as_float(xv << 16), x1 = __uint_as_float(xv & 0xffff0000u);
+        *reinterpret_cast<uint32_t *>(q_full + ((size_t)t * H + h) * (dc + rope) + dc + 2 * pr) = pack2(x0 * c.x - x1 * c.y, x0 * c.y + x1 * c.x);
+    }
+}
+
+// grid (H, T), 128 threads: log-sum-exp merge of the attention partials of sequence t and of the row the step just
+// wrote, for one head; o_lat rounded to bf16.  dc = 512: four columns per thread.
+constexpr int kMergeThreads = 128;
+__global__ void __launch_bounds__(kMergeThreads) attn_merge_batch_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
+                                                                         AttnPartials part, const BatchRows rows, int rope, float scale,
+                                                                         uint16_t *__restrict__ o_lat_bf16)
+{
+    constexpr int K = 512, kMaxParts = 16, kFirst = 4;
+    __shared__ float sm[kMaxParts], sl[kMaxParts], scratch[kMergeThreads / 32];
+    const int h = blockIdx.x, H = gridDim.x, t = blockIdx.y, dkv = K + rope, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int npart = rows.npart[t];
+    pdl_launch_dependents();
+    pdl_wait_prior_grids();                                       // partials come from the attention kernel
+    if (tid < npart) {
+        const float2 p = __ldcg(reinterpret_cast<const float2 *>(part.ml + (((size_t)t * rows.slot_stride + tid) * H + h) * 2));
+        sm[tid] = p.x; sl[tid] = p.y;
+    }
+    // the first partial rows and the new row are requested before the score is reduced
+    const int c = 4 * tid;
+    const float *Ot = part.O + ((size_t)t * rows.slot_stride * H + h) * K + c;
+    float4 v[kFirst];
+#pragma unroll
+    for (int s = 0; s < kFirst; ++s)
+        v[s] = (s < npart) ? __ldcg(reinterpret_cast<const float4 *>(Ot + (size_t)s * H * K)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    const uint16_t *row = cache + rows.new_row[t];
+    const uint2 rv = __ldcg(reinterpret_cast<const uint2 *>(row + c));
+    const uint16_t *qh = Q + ((size_t)t * H + h) * dkv;
+    float dot = 0.f;
+    for (int i = 2 * tid; i < dkv; i += 2 * kMergeThreads) {
+        const uint32_t a = __ldcg(reinterpret_cast<const uint32_t *>(qh + i)), b = __ldcg(reinterpret_cast<const uint32_t *>(row + i));
+        dot = fmaf(__uint_as_float(a << 16), __uint_as_float(b << 16), dot);
+        dot = fmaf(__uint_as_float(a & 0xffff0000u), __uint_as_float(b & 0xffff0000u), dot);
+    }
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o2);
+    if (lane == 0) scratch[warp] = dot;
+    __syncthreads();
+    float sx = 0.f;
+#pragma unroll
+    for (int w = 0; w < kMergeThreads / 32; ++w) sx += scratch[w];
+    sx *= scale;
+    float Mx = sx;
+    for (int s = 0; s < npart; ++s) Mx = fmaxf(Mx, sm[s]);
+    const float wx = __expf(sx - Mx);
+    float L = wx;
+    float4 acc = make_float4(wx * __uint_as_float(rv.x << 16), wx * __uint_as_float(rv.x & 0xffff0000u),
+                             wx * __uint_as_float(rv.y << 16), wx * __uint_as_float(rv.y & 0xffff0000u));
+    for (int s = 0; s < npart; ++s) {                             // part order: deterministic
+        const float wgt = (sm[s] == -INFINITY) ? 0.f : __expf(sm[s] - Mx);
+        L = fmaf(wgt, sl[s], L);
+        float4 x;
+        if (s < kFirst) {
+            x = v[0];
+#pragma unroll
+            for (int u = 1; u < kFirst; ++u) x = (s == u) ? v[u] : x;
+        } else {
+            x = __ldcg(reinterpret_cast<const float4 *>(Ot + (size_t)s * H * K));
+        }
+        acc.x = fmaf(wgt, x.x, acc.x); acc.y = fmaf(wgt, x.y, acc.y); acc.z = fmaf(wgt, x.z, acc.z); acc.w = fmaf(wgt, x.w, acc.w);
+    }
+    const float inv = 1.0f / L;
+    *reinterpret_cast<uint2 *>(o_lat_bf16 + ((size_t)t * H + h) * K + c) = make_uint2(pack2(acc.x * inv, acc.y * inv), pack2(acc.z * inv, acc.w * inv));
+}
+
 template <typename... Args>
 cudaError_t launch_b(void (*kern)(Args...), dim3 grid, cudaStream_t s, bool pdl, Args... args)
 {
@@ -330,6 +413,29 @@ int launch_uv_merge_batch(const void *Q, const void *cache, AttnPartials part, c
     cudaError_t e = launch_b(uv_merge_batch_kernel, dim3(H), s, pdl, (const uint16_t *)Q, (const uint16_t *)cache, part, rows, rope, scale,
                              (const uint16_t *)W_UV, (uint16_t *)o_lat_bf16, (uint16_t *)o, T);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "uv_merge (batch) launch");
+}
+
+int launch_rope_batch(const void *q, const float *cos_sin, void *q_full, int H, int nope, int dc, int rope, int T, cudaStream_t s, bool pdl)
+{
+    cudaError_t e = launch_b(rope_batch_kernel, dim3(T), s, pdl, (const uint16_t *)q, cos_sin, (uint16_t *)q_full, H, nope, dc, rope);
+    return e == cudaSuccess ? NM_OK : record_cuda_error(e, "rope (batch) launch");
+}
+
+int launch_attn_merge_batch(const void *Q, const void *cache, AttnPartials part, const BatchRows &rows, int T, int rope, float scale,
+                            void *o_lat_bf16, int H, cudaStream_t s, bool pdl)
+{
+    for (int t = 0; t < T; ++t)
+        if (rows.npart[t] < 0 || rows.npart[t] > 16) return NM_ERR_UNSUPPORTED;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(H, T); cfg.blockDim = dim3(kMergeThreads); cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_merge_batch_kernel, (const uint16_t *)Q, (const uint16_t *)cache, part, rows, rope, scale,
+                                       (uint16_t *)o_lat_bf16);
+    return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention merge (batch) launch");
 }
 
 }  // namespace nm

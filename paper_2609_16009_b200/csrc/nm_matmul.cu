@@ -301,12 +301,17 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     bool tma_ok = b_ok && a_ok && dtype != NM_F32 && tensor_map_encoder() != nullptr && (long)N * 2 < (1L << 40) && strideB >= 0;
     if (g_force_kind == kRowVec) tma_ok = false;
     Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok, chained);
+    // Copies, not pointers into the map cache: the second lookup may evict the entry the first one returned
+    // (16 entries, replaced in turn), and the kernel would then get the token map in place of the weight map.
+    CUtensorMap tc_map_b_copy, tc_map_a_copy;
     const CUtensorMap *tc_map_b = nullptr, *tc_map_a = nullptr;
     if (p.kind == kRowTc) {
         // weights [H][K][N] in 64x64 swizzled boxes; tokens [H][M][K] (row stride lda) in 64 x 16 swizzled boxes
         tc_map_b = (layout == NM_ROW_MAJOR) ? get_weight_map(B, N, K, H, strideB, 64, kTcKT, true)
                                             : get_weight_map(B, K, N, H, strideB, 64, kTcTN, true);     // [N][K]: 64 k x 128 columns of C
+        if (tc_map_b) { tc_map_b_copy = *tc_map_b; tc_map_b = &tc_map_b_copy; }
         tc_map_a = get_weight_map(A, K, M, H, strideA, 64, 16, true, lda);
+        if (tc_map_a) { tc_map_a_copy = *tc_map_a; tc_map_a = &tc_map_a_copy; }
         if (!tc_map_b || !tc_map_a)                         // strides the encoder refuses: CUDA-core kernel
             p = make_plan(M, N, K, H, dtype, layout, vec_ok, false, chained);
     }

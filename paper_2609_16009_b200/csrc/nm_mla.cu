@@ -14,6 +14,7 @@ static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape all
 // into two CTAs instead of four, which decides once a CTA has many tiles to go through; below, the 64-head
 // kernel's shorter prologue and merge win (measured: 16384 rows 94.8 vs 97.3 us per step, 65536 rows 164 vs 158)
 constexpr long kAttnWideRows = 65536;
+constexpr int kSMsAttn = 148;
 static bool attention_64_heads(long total_rows) { return g_attn_impl == 3 || (g_attn_impl != 2 && total_rows < kAttnWideRows); }
 
 // ---- small vector kernels ---------------------------------------------------------------------------
@@ -312,6 +313,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 // ---- host -------------------------------------------------------------------------------------------
 
 static int g_step_plan[3][3] = {};   // tuning: forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
+static int g_batch_tc_min_t = 4;     // batch decode: tokens from which the per-head products go to the tensor cores
 static int g_fused_tails = 1;        // 0: RMSNorm / RoPE / cache write as kernels of their own; 1: folded into the products (default);
                                      // 2: as 1, but only in the form where the product's last CTA runs them
 static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
@@ -724,7 +726,9 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     // split plan of the attention pass: the same number of splits for every sequence, about 128 CTAs in all
     long total_rows = 0;
     for (int t = 0; t < T; ++t) total_rows += b->seq_lens[t];
-    const bool tc64 = attention_64_heads(total_rows);              // 64 heads per CTA: four CTAs per split
+    // 64 heads per CTA (four CTAs per split) while the batch is short enough and its CTAs - at least four splits per
+    // sequence - fit one wave of the 148 SMs: up to nine sequences
+    const bool tc64 = attention_64_heads(total_rows) && (g_attn_impl == 3 || T * kAttnCluster * 4 <= kSMsAttn);
     int nsplit = ((tc64 ? 32 : 64) / T) / kAttnCluster * kAttnCluster;
     if (nsplit < kAttnCluster) nsplit = kAttnCluster;
     BatchRows rows{};
@@ -756,7 +760,18 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     NM_TRY(launch_down_finish_batch(x_down, p->gamma_q, p->gamma_kv, b->rope_cos_sin, c_qn, cache, rows, T, ql, dc, dr, p->rms_eps, ms, pdl));
     NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, T, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.mws_bytes, ms, pdl, nullptr, nullptr,
                           nullptr, true));
-    NM_TRY(launch_q_finish_batch(q, p->W_UK, b->rope_cos_sin, q_full, H, dr, T, ms, pdl));
+    // From four tokens on the per-head products (128 x 512 and 512 x 128 per head and token) go to the batched swap-AB
+    // tensor-core kernel, with RoPE and the merge as small kernels of their own: in the fused per-head kernels one
+    // CTA per head walks every token and is bound by fp32 FMA issue and by its chain of L2 round trips (measured at
+    // 4096 rows: 114 vs 115 us at T = 4, 133 vs 139 at T = 6, 183 vs 204 at T = 16; 105 vs 102 at T = 2).
+    const bool per_head_tc = T >= g_batch_tc_min_t || !g_fused_heads;
+    if (per_head_tc) {
+        NM_TRY(launch_rope_batch(q, b->rope_cos_sin, q_full, H, dn, dc, dr, T, ms, pdl));
+        NM_TRY(matmul_enqueue(q, p->W_UK, q_full, T, dc, dn, H, (long)H * dq, dq, (long)dn * dc, (long)H * dkv, dkv, NM_BF16, NM_ROW_MAJOR,
+                              mws, L.mws_bytes, ms, pdl));
+    } else {
+        NM_TRY(launch_q_finish_batch(q, p->W_UK, b->rope_cos_sin, q_full, H, dr, T, ms, pdl));
+    }
     AttnPartials part;
     part.ml = reinterpret_cast<float *>(ws + L.attn_ml);
     part.O = reinterpret_cast<float *>(ws + L.attn_o);
@@ -767,7 +782,13 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
         else
             NM_TRY(attention_partial_tc_batch(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl));
     }
-    NM_TRY(launch_uv_merge_batch(q_full, cache, part, rows, T, dr, p->softmax_scale, p->W_UV, o_lat, o, H, ms, pdl));
+    if (per_head_tc) {
+        NM_TRY(launch_attn_merge_batch(q_full, cache, part, rows, T, dr, p->softmax_scale, o_lat, H, ms, pdl));
+        NM_TRY(matmul_enqueue(o_lat, p->W_UV, o, T, dv, dc, H, (long)H * dc, dc, (long)dc * dv, (long)H * dv, dv, NM_BF16, NM_ROW_MAJOR,
+                              mws, L.mws_bytes, ms, pdl));
+    } else {
+        NM_TRY(launch_uv_merge_batch(q_full, cache, part, rows, T, dr, p->softmax_scale, p->W_UV, o_lat, o, H, ms, pdl));
+    }
     if (p->W_O)
         NM_TRY(matmul_enqueue(o, p->W_O, b->out, T, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.mws_bytes, ms, pdl, nullptr,
                               nullptr, nullptr, true));

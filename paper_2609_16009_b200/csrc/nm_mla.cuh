@@ -91,6 +91,11 @@ int launch_q_finish_batch(const void *q, const void *W_UK, const float *cos_sin,
 int launch_uv_merge_batch(const void *Q, const void *cache, AttnPartials part, const BatchRows &rows, int T, int rope, float scale,
                           const void *W_UV, void *o_lat_bf16, void *o, int H, cudaStream_t s, bool pdl);
 
+// The same stages without the per-head products (those then run as batched products on the tensor cores).
+int launch_rope_batch(const void *q, const float *cos_sin, void *q_full, int H, int nope, int dc, int rope, int T, cudaStream_t s, bool pdl);
+int launch_attn_merge_batch(const void *Q, const void *cache, AttnPartials part, const BatchRows &rows, int T, int rope, float scale,
+                            void *o_lat_bf16, int H, cudaStream_t s, bool pdl);
+
 // Tuning aid: phase timestamps (ns) of the tensor-core kernel go to `p` when non-null: 32 slots for CTA (0,0),
 // then four per CTA (start, Q landed, last P*V done, end); 32 + 4 * 256 values at most.
 void set_attention_trace(unsigned long long *p);

@@ -266,6 +266,29 @@ def test_tensor_core_kernel_small_integers_bit_exact(nm):
     assert np.array_equal(got, C64)
 
 
+def test_many_tensor_core_products_in_one_process_cycle_the_tensor_map_cache(nm):
+    """The library keeps the tensor maps of recent operands (16 entries).  Forty products with distinct token and
+    weight buffers make every entry be replaced several times, between the two lookups of one call as well."""
+    K, N = 256, 384
+    nm.nm_debug_set_kernel(4, 0)
+    try:
+        keep = []
+        for i in range(40):
+            M = 3 + i % 14
+            A, B = gen.narrow_bf16(M, K, N, seed=2000 + i)
+            dA, dB = to_dev(A), to_dev(B)
+            whole, dC = out_buffer(M * N, BF16)
+            keep.append((dA, dB, whole))                           # distinct addresses: nothing is freed in between
+            assert nm.nm_debug_get_plan(M, N, K)["kind"] == 4
+            nm.nm_matmul(dA, dB, dC, M, N, K, BF16, ROW)
+            torch.cuda.synchronize()
+            Cq, C64, bound = oracle.matmul(A, B, M, N, K, ORACLE_IN[BF16], ORACLE_OUT[BF16], ROW, threads=8)
+            assert_matmul_close(out_to_f64(dC, BF16).reshape(M, N), Cq, C64, bound, BF16, f"product {i}")
+    finally:
+        nm.nm_debug_set_kernel(-1, 0)
+    nm.nm_check_status()
+
+
 def test_default_kernel_choice_by_m(nm):
     # CUDA cores (TMA ring) for one or two token rows and for small weight matrices, tensor cores from
     # three rows on for large ones; the threshold is adjustable

@@ -107,6 +107,22 @@ def test_batch_matches_oracle(nm, weights, seq_lens, concat):
     check_against_oracle(w, res, tokens, caches, seq_lens)
 
 
+@pytest.mark.parametrize("seq_lens,with_wo", [([300], True), ([90, 1, 257], True), ([1024, 65, 2, 500, 130], True),
+                                              ([64 + 31 * i for i in range(12)], False)])
+def test_batch_with_the_per_head_products_as_batched_products(nm, weights, seq_lens, with_wo):
+    """From four sequences on the per-head products run as batched products (tensor cores from M = 3) with RoPE and
+    the merge as kernels of their own; below, fused per-head kernels do them.  Here the first form at every batch
+    size (the switch that turns the fused per-head kernels off), against the oracle."""
+    w, dw = weights
+    tokens, caches = make_inputs(seq_lens, seed=8300 + len(seq_lens))
+    nm.nm_debug_set_step_fusion(False)
+    try:
+        res = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True, with_wo=with_wo)
+    finally:
+        nm.nm_debug_set_step_fusion(True)
+    check_against_oracle(w, res, tokens, caches, seq_lens, with_wo=with_wo)
+
+
 def test_batch_of_sixteen_without_wo(nm, weights):
     w, dw = weights
     seq_lens = [40 + 37 * i for i in range(16)]

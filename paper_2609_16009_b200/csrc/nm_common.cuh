@@ -1,5 +1,7 @@
 // Shared device/host helpers for the nm kernels (sm_100a only).
 #pragma once
+#include <cstdio>
+#include <cstdlib>
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
@@ -101,5 +103,30 @@ int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, i
 void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit, bool chained = false);
 
 __host__ __device__ constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Whether all `clusters` clusters of a launch configured in `cfg` (cluster dimension among its attributes) can be
+// resident at once.  The CTAs of a cluster need SMs of one GPC at the same time, so a grid that fits the machine
+// CTA by CTA may still need a second wave as clusters; the split-K-in-a-cluster paths fall back to the workspace
+// then.  Answers are cached per (kernel, shared memory, cluster size).
+template <typename Kern>
+int max_clusters_cached(Kern kern, const cudaLaunchConfig_t &cfg, unsigned cluster_size)
+{
+    struct Entry { const void *f; size_t smem; unsigned cs; int n; };
+    static thread_local Entry cache[32];
+    static thread_local int next = 0;
+    const void *f = reinterpret_cast<const void *>(kern);
+    for (const Entry &e : cache)
+        if (e.f == f && e.smem == cfg.dynamicSmemBytes && e.cs == cluster_size) return e.n;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    cache[next] = Entry{f, cfg.dynamicSmemBytes, cluster_size, n};
+    next = (next + 1) % 32;
+    return n;
+}
+template <typename Kern>
+bool clusters_fit_one_wave(Kern kern, const cudaLaunchConfig_t &cfg, unsigned cluster_size, long clusters)
+{
+    return max_clusters_cached(kern, cfg, cluster_size) >= clusters;
+}
 
 }  // namespace nm

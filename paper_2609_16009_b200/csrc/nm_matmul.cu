@@ -132,7 +132,7 @@ static Plan make_tma_plan(int M, int N, int K, int H, bool chained = false)
 
 // Plan for the swap-AB tensor-core kernel: 128-column tiles, k-rows per split a multiple of the 64-row
 // stage, about two CTAs per SM in total, five 18 KB stages.
-static Plan make_tc_plan(int M, int N, int K, int H)
+static Plan make_tc_plan(int M, int N, int K, int H, bool col_major = false, bool f32_out = false)
 {
     Plan p{};
     p.kind = kRowTc;
@@ -143,6 +143,15 @@ static Plan make_tc_plan(int M, int N, int K, int H)
     int ns = (int)((kSMs + base / 2) / base);
     if (ns > K / 128) ns = K / 128;
     if (ns > K / (40 * M)) ns = K / (40 * M);          // partial sums stay below ~10 % of the weight bytes
+    // Up to eight splits meet inside a cluster (64 KB of slots at M = 16) - when all the clusters are resident at
+    // once: the CTAs of a cluster need SMs of one GPC, so fewer CTAs fit as clusters than one by one (15 clusters of
+    // eight, 26 of five, 45 of three with one CTA per SM).  Take the largest split count whose clusters fit.
+    // On matrices of 100 MB and more the streaming time dominates and fewer CTAs cost more than the gather saves
+    // (235 MB at M = 16: 43.0 us as 168 CTAs through the workspace, 44.9 us as 56 clusters of two): no reduction there.
+    if (g_cluster_split && g_force_split == 0 && ns >= 2 && 2.0 * K * N * H < 100e6) {
+        for (int c = ns < 8 ? ns : 8; c >= 2; --c)
+            if (base <= row_tc_max_clusters(c, 5, M, col_major, f32_out)) { ns = c; break; }
+    }
     if (g_force_split > 0) ns = g_force_split;
     if (ns > kMaxSplit) ns = kMaxSplit;
     if (ns < 1) ns = 1;
@@ -181,7 +190,7 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     const int min_m = (layout == NM_COL_MAJOR && g_tc_min_m > 2 && g_tc_min_m <= NM_MAX_M) ? 2 : g_tc_min_m;
     const bool tc_pays = M >= min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6)) && (M >= g_tc_min_m || wbytes >= 48e6);
     if (tma_ok && g_force_kind != kRowTma && (layout == NM_ROW_MAJOR || g_force_kind != kRowVec) && (tc_pays || g_force_kind == kRowTc))
-        return make_tc_plan(M, N, K, H);
+        return make_tc_plan(M, N, K, H, layout == NM_COL_MAJOR, dtype == NM_BF16_F32OUT);
     if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H, chained);
     const int target = 192;                           // CTAs wanted in total (measured: 144-240 is the flat optimum)
     if (layout == NM_ROW_MAJOR) {
@@ -339,6 +348,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         const CUtensorMap *mb = tc_map_b, *ma = tc_map_a;
         TmaArgs ta{};
         ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
+        if (g_cluster_split && p.nsplit >= 2 && p.nsplit <= 8 && (size_t)p.nsplit * M * kTcTN * sizeof(float) <= 65536) ta.cluster_split = 1;
         const bool col = layout == NM_COL_MAJOR;
         e = (dtype == NM_BF16_F32OUT) ? launch_row_tc<float>(*mb, *ma, ta, stream, col) : launch_row_tc<bf16_t>(*mb, *ma, ta, stream, col);
     } else if (p.kind == kRowTma) {

@@ -666,7 +666,16 @@ cudaError_t launch_row(const MatmulArgs &a, cudaStream_t s)
     cfg.attrs = attr;
     cfg.numAttrs = a.cluster_split ? 1 : 0;
     switch (a.M) {
-#define NM_X(m) case m: return cudaLaunchKernelEx(&cfg, nm_row_kernel<m, TI, TO>, a);
+#define NM_X(m)                                                                                          \
+    case m: {                                                                                            \
+        auto kern = nm_row_kernel<m, TI, TO>;                                                             \
+        MatmulArgs b = a;                                                                                \
+        if (b.cluster_split && b.partial && !clusters_fit_one_wave(kern, cfg, (unsigned)b.nsplit, (long)b.ntiles * b.H)) { \
+            b.cluster_split = 0;       /* a second wave of clusters: through the workspace instead */      \
+            cfg.numAttrs = 0;                                                                            \
+        }                                                                                                \
+        return cudaLaunchKernelEx(&cfg, kern, b);                                                        \
+    }
         NM_FOR_EACH_M(NM_X)
 #undef NM_X
     default: return cudaErrorInvalidValue;
@@ -686,7 +695,16 @@ cudaError_t launch_col(const MatmulArgs &a, cudaStream_t s)
     cfg.attrs = attr;
     cfg.numAttrs = a.cluster_split ? 1 : 0;
     switch (a.M) {
-#define NM_X(m) case m: return cudaLaunchKernelEx(&cfg, nm_col_kernel<m, TI, TO>, a);
+#define NM_X(m)                                                                                          \
+    case m: {                                                                                            \
+        auto kern = nm_col_kernel<m, TI, TO>;                                                             \
+        MatmulArgs b = a;                                                                                \
+        if (b.cluster_split && b.partial && !clusters_fit_one_wave(kern, cfg, (unsigned)b.nsplit, (long)b.ntiles * b.H)) { \
+            b.cluster_split = 0;       /* a second wave of clusters: through the workspace instead */      \
+            cfg.numAttrs = 0;                                                                            \
+        }                                                                                                \
+        return cudaLaunchKernelEx(&cfg, kern, b);                                                        \
+    }
         NM_FOR_EACH_M(NM_X)
 #undef NM_X
     default: return cudaErrorInvalidValue;

@@ -65,6 +65,10 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
     pdl_launch_dependents();
+    // Split-K inside a cluster (the k-splits of a tile are the CTAs of one cluster, see cluster_split_finish): first
+    // half of a cluster barrier here, its second half before the first store into a peer's shared memory.
+    if (ta.cluster_split) cluster_arrive_all();
+    float *slots = reinterpret_cast<float *>(bars + 3 * NS + 2);  // [split][m][128 columns], used in the first CTA of the cluster
 
     if (warp == 0) {
         if (lane == 0) {
@@ -121,6 +125,12 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
     }
 
     // ---- epilogue: 128 accumulator rows (columns of C) x 16 tokens ------------------------------------------
+    uint32_t slot0 = 0;
+    if (ta.cluster_split) {
+        __syncwarp();
+        cluster_wait_all();
+        slot0 = cluster_slot_base(slots, split, M * kTcTN);
+    }
     if (warp >= 2) {
         const int quad = warp & 3, c = quad * 32 + lane;          // column of the tile held by this thread
         if (n_it > 0) {
@@ -138,6 +148,10 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
 #pragma unroll
                 for (int m = 0; m < 16; ++m)
                     if (m < M) C[(long)m * a.ldc + n] = round_out<TO>(n_it > 0 ? __uint_as_float(d[m]) : 0.f);
+        } else if (ta.cluster_split) {
+#pragma unroll
+            for (int m = 0; m < 16; ++m)
+                if (m < M) cluster_slot_store(slot0, m * kTcTN + c, n_it > 0 ? __uint_as_float(d[m]) : 0.f);
         } else {
             float *P = a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * kTcTN);
 #pragma unroll
@@ -146,8 +160,15 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
         }
     }
     tc_fence_before();
-    if (a.nsplit > 1) splitk_complete_rt<TO>(a, M, tile, h, &s_last);
-    else __syncthreads();
+    if (ta.cluster_split) {
+        __syncwarp();
+        cluster_split_finish<TO>(a, slots, M, tile, split, h);    // cluster barrier, then the first CTA adds the slots
+        __syncthreads();
+    } else if (a.nsplit > 1) {
+        splitk_complete_rt<TO>(a, M, tile, h, &s_last);
+    } else {
+        __syncthreads();
+    }
     if (s_abort && tid == 0)
         for (int s = 0; s < NS && s < n_it; ++s)
             for (int i = 0; i < (1 << 14) && !mbar_try_wait(full_b0 + 8 * s, 0); ++i) {}
@@ -159,11 +180,12 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
 
 }  // namespace
 
-size_t row_tc_smem_bytes(int nstage) { return (size_t)nstage * kStage + (3 * nstage + 1) * sizeof(uint64_t) + 1024; }
+size_t row_tc_smem_bytes(int nstage, size_t slot_bytes) { return (size_t)nstage * kStage + (3 * nstage + 1) * sizeof(uint64_t) + 16 + slot_bytes + 1024; }
 
 template <typename TO, bool kCol>
-static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta, cudaStream_t s)
+static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta_in, cudaStream_t s)
 {
+    TmaArgs ta = ta_in;
     const MatmulArgs &a = ta.base;
     static bool configured = false;
     auto kern = nm_row_tc_kernel<TO, kCol>;
@@ -175,14 +197,53 @@ static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a,
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.ntiles, a.nsplit, a.H);
     cfg.blockDim = dim3(kTcThreads);
-    cfg.dynamicSmemBytes = row_tc_smem_bytes(ta.nstage);
+    cfg.dynamicSmemBytes = row_tc_smem_bytes(ta.nstage, ta.cluster_split ? (size_t)a.nsplit * a.M * kTcTN * sizeof(float) : 0);
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (ta.use_pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    if (ta.cluster_split) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 1; attr[na].val.clusterDim.y = (unsigned)a.nsplit; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = ta.use_pdl ? 1 : 0;
+    cfg.numAttrs = na;
+    if (ta.cluster_split && !clusters_fit_one_wave(kern, cfg, (unsigned)a.nsplit, (long)a.ntiles * a.H)) {
+        ta.cluster_split = 0;                                      // through the workspace instead (the caller provided it)
+        cfg.dynamicSmemBytes = row_tc_smem_bytes(ta.nstage, 0);
+        cfg.numAttrs = na - 1;                                     // the cluster attribute is the last one
+    }
     return cudaLaunchKernelEx(&cfg, kern, map_b, map_a, ta);
+}
+
+// How many clusters of `cluster_size` CTAs of this kernel (ring of `nstage` stages, slots for M tokens) the GPU holds
+// at once; 0 when it cannot be asked (no device).  The planner sizes the k-split with it.
+template <typename TO, bool kCol>
+static int max_clusters_tc(int cluster_size, int nstage, int M)
+{
+    auto kern = nm_row_tc_kernel<TO, kCol>;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, cluster_size, 1);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = row_tc_smem_bytes(nstage, (size_t)cluster_size * M * kTcTN * sizeof(float));
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)cluster_size; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    return max_clusters_cached(kern, cfg, (unsigned)cluster_size);
+}
+
+int row_tc_max_clusters(int cluster_size, int nstage, int M, bool col_major, bool f32_out)
+{
+    if (col_major) return f32_out ? max_clusters_tc<float, true>(cluster_size, nstage, M) : max_clusters_tc<bf16_t, true>(cluster_size, nstage, M);
+    return f32_out ? max_clusters_tc<float, false>(cluster_size, nstage, M) : max_clusters_tc<bf16_t, false>(cluster_size, nstage, M);
 }
 
 template <typename TO>

@@ -367,8 +367,9 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
 }
 
 template <int TPR, typename TO>
-cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta, size_t smem_bytes, cudaStream_t s)
+cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta_in, size_t smem_bytes, cudaStream_t s)
 {
+    TmaArgs ta = ta_in;
     const MatmulArgs &a = ta.base;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.ntiles, a.nsplit, a.H);
@@ -398,6 +399,13 @@ cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta, size_t sm
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); \
             if (e != cudaSuccess) return e;                                                               \
             configured = true;                                                                            \
+        }                                                                                                 \
+        /* clusters that would need a second wave: through the workspace instead, unless the caller counts on the */ \
+        /* per-tile sums of squares, which only the cluster path writes */                               \
+        if (ta.cluster_split && !ta.tile_ss && a.partial &&                                               \
+            !clusters_fit_one_wave(kern, cfg, (unsigned)a.nsplit, (long)a.ntiles * a.H)) {                \
+            ta.cluster_split = 0;                                                                         \
+            cfg.numAttrs = na - 1;                                                                        \
         }                                                                                                 \
         return cudaLaunchKernelEx(&cfg, kern, tmap, ta);                                                  \
     }

@@ -229,6 +229,29 @@ def test_split_k_inside_a_cluster_plain_kernels(nm, layout, dtype, M, nsplit):
     nm.nm_check_status()
 
 
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("M,nsplit", [(3, 2), (4, 8), (9, 5), (16, 8), (16, 3), (5, 9)])
+def test_split_k_inside_a_cluster_tensor_core_kernel(nm, layout, M, nsplit):
+    """The swap-AB tensor-core kernel: up to eight k-splits (64 KB of partial tiles) meeting in a cluster against
+    the workspace path - identical bits, parity with the oracle.  K ends mid-stage and N mid-tile."""
+    K, N = 2600, 840
+    A, B = gen.narrow_bf16(M, K, N, seed=990 + M)
+    outs = []
+    for cluster in (True, False):
+        nm.nm_debug_set_plan(0, nsplit)
+        nm.nm_debug_set_kernel(4, 0)
+        nm.nm_debug_set_cluster_split(cluster)
+        try:
+            assert nm.nm_debug_get_plan(M, N, K, 1, BF16, layout)["kind"] == 4
+            outs.append(run_case(nm, A, B, M, N, K, BF16, layout, f"tc split-K M={M} nsplit={nsplit} layout={layout} cluster={cluster}"))
+        finally:
+            nm.nm_debug_set_plan(0, 0)
+            nm.nm_debug_set_kernel(-1, 0)
+            nm.nm_debug_set_cluster_split(True)
+    assert np.array_equal(outs[0], outs[1])
+    nm.nm_check_status()
+
+
 def test_paper_matmul_2_shape_takes_eight_splits_in_a_cluster(nm):
     plan = nm.nm_debug_get_plan(1, 576, 7168)
     assert plan["kind"] == 3 and plan["nsplit"] == 8

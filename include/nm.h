@@ -320,7 +320,8 @@ int nm_debug_set_cluster_split(int enable);
  * from 4 four per cache tile - scores issued, scores seen, P written, P*V issued); from 32 four per
  * attention CTA (start, Q landed, last P*V done, end); from 1100 eight phases of two CTAs of the merge + W_UV
  * kernel; from 2048 / 4096 / 6144 four per CTA (start, inputs ready, loop done, end) of the down-projection, W_UQR
- * and W_O products.  NULL = off. */
+ * and W_O products; from 2688 four phases of the CTA that completes a product carrying vector stages (last arrival,
+ * gather done, synchronised, sums reduced).  NULL = off. */
 int nm_debug_set_attention_trace(void *device_buffer);
 /* Decode step tuning: launch the merge + W_UV kernel programmatically (default 1); include W_UV in the L2
  * prefetch (default 1). */

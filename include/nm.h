@@ -317,7 +317,8 @@ int nm_debug_set_kernel(int kind, int stages);
 int nm_debug_set_cluster_split(int enable);
 /* Tuning aid: phase timestamps (ns, %globaltimer) of the decode step's kernels go to `device_buffer` (8192
  * unsigned 64-bit values) when non-null: [0,32) phases of CTA (0,0) of the attention kernel (the 64-head kernel:
- * from 4 four per cache tile - scores issued, scores seen, P written, P*V issued); from 32 four per
+ * from 4 four per cache tile - scores issued, scores seen, P written, P*V issued - for five tiles, from 24 five phases
+ * of the cluster merge); from 32 four per
  * attention CTA (start, Q landed, last P*V done, end); from 1100 eight phases of two CTAs of the merge + W_UV
  * kernel; from 2048 / 4096 / 6144 four per CTA (start, inputs ready, loop done, end) of the down-projection, W_UQR
  * and W_O products; from 2688 four phases of the CTA that completes a product carrying vector stages (last arrival,

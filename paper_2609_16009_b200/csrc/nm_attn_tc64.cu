@@ -105,8 +105,10 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     part.ml += (size_t)seq * seqs.ml_stride;
     part.O += (size_t)seq * seqs.o_stride;
     // Tuning aid: four stamps of every CTA of sequence 0 (start, Q landed, last P*V done, end) from trace[32] on
-    // ... and of CTA (0,0) of sequence 0 per tile t < 7: trace[4 + 4 t ..] = scores issued, scores seen, P written, P*V issued
-#define NM_TRACE_TILE(t, i) do { if (trace && (t) < 7 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) trace[4 + 4 * (t) + (i)] = global_timer_ns(); } while (0)
+    // ... and of CTA (0,0) of sequence 0 per tile t < 5: trace[4 + 4 t ..] = scores issued, scores seen, P written, P*V issued;
+    // trace[24..28] = rows parked, cluster barrier passed, weights known, rows pulled and stored, second barrier passed
+#define NM_TRACE_TILE(t, i) do { if (trace && (t) < 5 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) trace[4 + 4 * (t) + (i)] = global_timer_ns(); } while (0)
+#define NM_TRACE_MERGE(i) do { if (trace && tid == 64 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) trace[24 + (i)] = global_timer_ns(); } while (0)
 #define NM_TRACE_CTA(i) do { if (trace && blockIdx.z == 0) trace[32 + 4 * (blockIdx.y * gridDim.x + blockIdx.x) + (i)] = global_timer_ns(); } while (0)
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -381,7 +383,9 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
         }
     }
+    NM_TRACE_MERGE(0);
     cluster_sync_all();                                            // every peer's rows are parked, its (m, l) here
+    NM_TRACE_MERGE(1);
     if (warp >= 2 && warp < 6) {
         const int t = tid - 64;                                    // 0..127
         if (t < kCl * kHeadsPerRank) {                             // weight of peer r for owned head hl
@@ -402,6 +406,7 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
         }
         named_barrier_sync(1, 128);
+        NM_TRACE_MERGE(2);
         constexpr int kIters = kHeadsPerRank * 64 / 128, kBatch = 4;       // 8 float4 outputs per thread
         for (int i0 = 0; i0 < kIters; i0 += kBatch) {
             float4 v[kBatch][kCl];
@@ -429,7 +434,9 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
         }
     }
+    NM_TRACE_MERGE(3);
     cluster_sync_all();                                            // peers are done reading this CTA's shared memory
+    NM_TRACE_MERGE(4);
 
     // ---- teardown: TMEM goes back ---------------------------------------------------------------------------
     tc_fence_before();
@@ -443,6 +450,7 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     if (tid == 0) NM_TRACE_CTA(3);
 #undef NM_TRACE_CTA
+#undef NM_TRACE_MERGE
 #undef NM_TRACE_TILE
 }
 

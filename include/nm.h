@@ -51,6 +51,10 @@ enum {
 };
 
 #define NM_MAX_M 16
+/* More tokens than the narrow range proper (the paper's outlook: remainder rows, larger tokens): up to 64 rows are
+ * taken in one pass over B by the tensor-core kernel when the operands qualify for it (bf16, 16-byte aligned A and B
+ * with rows / columns that stay aligned); NM_ERR_UNSUPPORTED otherwise. */
+#define NM_MAX_M_TENSOR 64
 
 /* ---- misc ------------------------------------------------------------------------------- */
 
@@ -102,7 +106,7 @@ int nm_set_workspace(void *workspace, size_t bytes);
  * Any N, K >= 1 is accepted; the vectorised path needs 16-byte aligned A, B and N (row-major)
  * or K (column-major) a multiple of 16 bytes' worth of elements, otherwise a scalar kernel runs.
  * Uses the default workspace when the chosen tiling splits K; returns NM_ERR_WORKSPACE if none
- * is registered or it is too small.
+ * is registered or it is too small.  17 <= M <= NM_MAX_M_TENSOR: see NM_MAX_M_TENSOR above.
  */
 int nm_matmul(const void *A, const void *B, void *C, int M, int N, int K,
               nm_dtype dtype, nm_layout layout_B, nm_stream stream);

@@ -142,13 +142,14 @@ static Plan make_tc_plan(int M, int N, int K, int H, bool col_major = false, boo
     // one CTA per SM measured best for this kernel (its ring alone keeps 90 KB in flight per SM)
     int ns = (int)((kSMs + base / 2) / base);
     if (ns > K / 128) ns = K / 128;
-    if (ns > K / (40 * M)) ns = K / (40 * M);          // partial sums stay below ~10 % of the weight bytes
+    if (M <= NM_MAX_M) { if (ns > K / (40 * M)) ns = K / (40 * M); }     // partial sums stay below ~10 % of the weight bytes
+    else if (ns > K / (8 * M)) ns = K / (8 * M);        // 17-64 tokens: up to ~40 %, or too few CTAs are left (small matrices)
     // Up to eight splits meet inside a cluster (64 KB of slots at M = 16) - when all the clusters are resident at
     // once: the CTAs of a cluster need SMs of one GPC, so fewer CTAs fit as clusters than one by one (15 clusters of
     // eight, 26 of five, 45 of three with one CTA per SM).  Take the largest split count whose clusters fit.
     // On matrices of 100 MB and more the streaming time dominates and fewer CTAs cost more than the gather saves
     // (235 MB at M = 16: 43.0 us as 168 CTAs through the workspace, 44.9 us as 56 clusters of two): no reduction there.
-    if (g_cluster_split && g_force_split == 0 && ns >= 2 && 2.0 * K * N * H < 100e6) {
+    if (g_cluster_split && g_force_split == 0 && ns >= 2 && 2.0 * K * N * H < 100e6 && M <= NM_MAX_M) {
         for (int c = ns < 8 ? ns : 8; c >= 2; --c)
             if (base <= row_tc_max_clusters(c, 5, M, col_major, f32_out)) { ns = c; break; }
     }
@@ -161,6 +162,7 @@ static Plan make_tc_plan(int M, int N, int K, int H, bool col_major = false, boo
     p.nsplit = ceil_div(K, kr);
     // one CTA per SM on a large matrix: a deeper ring (measured +1.5 to 3 %); otherwise 90 KB, two CTAs fit an SM
     int nstage = (base * p.nsplit <= kSMs && 2.0 * K * N * H >= 48e6) ? 7 : 5;
+    if (M > 16 && base * p.nsplit > kSMs) nstage = (M > 32) ? 4 : 5;      // 24 / 20 KB stages: two CTAs still share an SM
     const int its = ceil_div(kr, kTcKT);                // a ring deeper than the CTA's k-range only costs shared memory
     if (nstage > its) nstage = its;
     if (g_force_stages > 0) nstage = g_force_stages;
@@ -188,8 +190,9 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     // Column-major weights: the CUDA-core column kernel is already behind at M = 2 from about 50 MB on (17 vs 14 us
     // on 75 MB).
     const int min_m = (layout == NM_COL_MAJOR && g_tc_min_m > 2 && g_tc_min_m <= NM_MAX_M) ? 2 : g_tc_min_m;
-    const bool tc_pays = M >= min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6)) && (M >= g_tc_min_m || wbytes >= 48e6);
-    if (tma_ok && g_force_kind != kRowTma && (layout == NM_ROW_MAJOR || g_force_kind != kRowVec) && (tc_pays || g_force_kind == kRowTc))
+    // More than 16 tokens (up to 64): only the tensor-core kernel takes them, whatever the size of the matrix
+    const bool tc_pays = M > NM_MAX_M || (M >= min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6)) && (M >= g_tc_min_m || wbytes >= 48e6));
+    if (tma_ok && (M > NM_MAX_M || (g_force_kind != kRowTma && (layout == NM_ROW_MAJOR || g_force_kind != kRowVec))) && (tc_pays || g_force_kind == kRowTc))
         return make_tc_plan(M, N, K, H, layout == NM_COL_MAJOR, dtype == NM_BF16_F32OUT);
     if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H, chained);
     const int target = 192;                           // CTAs wanted in total (measured: 144-240 is the flat optimum)
@@ -276,7 +279,7 @@ static int check_common(const void *A, const void *B, const void *C, int M, int 
                         nm_dtype dtype, nm_layout layout)
 {
     if (!A || !B || !C) return NM_ERR_INVALID_ARG;
-    if (M < 1 || M > NM_MAX_M || N < 1 || K < 1 || H < 1) return NM_ERR_INVALID_ARG;
+    if (M < 1 || M > NM_MAX_M_TENSOR || N < 1 || K < 1 || H < 1) return NM_ERR_INVALID_ARG;
     if (dtype != NM_F32 && dtype != NM_BF16 && dtype != NM_BF16_F32OUT) return NM_ERR_UNSUPPORTED;
     if (layout != NM_ROW_MAJOR && layout != NM_COL_MAJOR) return NM_ERR_UNSUPPORTED;
     if (H > 65535) return NM_ERR_UNSUPPORTED;
@@ -314,15 +317,18 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     // (16 entries, replaced in turn), and the kernel would then get the token map in place of the weight map.
     CUtensorMap tc_map_b_copy, tc_map_a_copy;
     const CUtensorMap *tc_map_b = nullptr, *tc_map_a = nullptr;
+    if (M > NM_MAX_M && p.kind != kRowTc) return NM_ERR_UNSUPPORTED;       // 17-64 tokens: bf16 operands the tensor-core kernel takes
     if (p.kind == kRowTc) {
         // weights [H][K][N] in 64x64 swizzled boxes; tokens [H][M][K] (row stride lda) in 64 x 16 swizzled boxes
         tc_map_b = (layout == NM_ROW_MAJOR) ? get_weight_map(B, N, K, H, strideB, 64, kTcKT, true)
                                             : get_weight_map(B, K, N, H, strideB, 64, kTcTN, true);     // [N][K]: 64 k x 128 columns of C
         if (tc_map_b) { tc_map_b_copy = *tc_map_b; tc_map_b = &tc_map_b_copy; }
-        tc_map_a = get_weight_map(A, K, M, H, strideA, 64, 16, true, lda);
+        tc_map_a = get_weight_map(A, K, M, H, strideA, 64, row_tc_tokens(M), true, lda);
         if (tc_map_a) { tc_map_a_copy = *tc_map_a; tc_map_a = &tc_map_a_copy; }
-        if (!tc_map_b || !tc_map_a)                         // strides the encoder refuses: CUDA-core kernel
+        if (!tc_map_b || !tc_map_a) {                       // strides the encoder refuses: CUDA-core kernel
+            if (M > NM_MAX_M) return NM_ERR_UNSUPPORTED;
             p = make_plan(M, N, K, H, dtype, layout, vec_ok, false, chained);
+        }
     }
 
     MatmulArgs a{};

@@ -27,14 +27,16 @@ namespace {
 
 constexpr int kTcThreads = 192;
 constexpr int kBStage = kTcKT * kTcTN * 2;         // 16 KB of weights per stage
-constexpr int kAStage = 16 * kTcKT * 2;            // 2 KB of tokens per stage
-constexpr int kStage = kBStage + kAStage;
-constexpr uint32_t kTmemColsTc = 32;
 
-template <typename TO, bool kCol>
-__global__ void __launch_bounds__(kTcThreads, 4)
+// kTok: token columns of the accumulator (the MMA's N): 16 for M <= 16, 32 or 64 for more tokens than the narrow
+// range proper - the weights are still streamed once, the tokens padded to the next size.
+template <typename TO, bool kCol, int kTok>
+__global__ void __launch_bounds__(kTcThreads, kTok == 16 ? 4 : 2)
 nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_a, const TmaArgs ta)
 {
+    constexpr int kAStage = kTok * kTcKT * 2;      // 2 KB of tokens per stage at 16 tokens
+    constexpr int kStage = kBStage + kAStage;
+    constexpr uint32_t kTmemColsTc = kTok < 32 ? 32 : kTok;
     const MatmulArgs &a = ta.base;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -105,7 +107,7 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc(128, 16, !kCol, false);
+            constexpr uint32_t idesc = instr_desc(128, kTok, !kCol, false);
             int s = 0;
             uint32_t ph = 0;
             for (int it = 0; it < n_it; ++it) {
@@ -137,8 +139,14 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
             mbar_wait(bar_done, 0, &s_abort, ta.status);
             tc_fence_after();
         }
-        uint32_t d[16];
-        tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16), d);
+        uint32_t d[kTok];
+#pragma unroll
+        for (int j = 0; j < kTok / 16; ++j) {
+            uint32_t part[16];
+            tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16) + 16 * j, part);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) d[16 * j + i] = part[i];
+        }
         tmem_wait_ld();
         const int n = tile * kTcTN + c;
         pdl_wait_prior_grids();                                   // nothing is written before earlier kernels are done
@@ -146,16 +154,16 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
             TO *C = (TO *)a.C + (long)h * a.strideC;
             if (n < a.N)
 #pragma unroll
-                for (int m = 0; m < 16; ++m)
+                for (int m = 0; m < kTok; ++m)
                     if (m < M) C[(long)m * a.ldc + n] = round_out<TO>(n_it > 0 ? __uint_as_float(d[m]) : 0.f);
         } else if (ta.cluster_split) {
 #pragma unroll
-            for (int m = 0; m < 16; ++m)
+            for (int m = 0; m < kTok; ++m)
                 if (m < M) cluster_slot_store(slot0, m * kTcTN + c, n_it > 0 ? __uint_as_float(d[m]) : 0.f);
         } else {
             float *P = a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * kTcTN);
 #pragma unroll
-            for (int m = 0; m < 16; ++m)
+            for (int m = 0; m < kTok; ++m)
                 if (m < M) P[(size_t)m * kTcTN + c] = n_it > 0 ? __uint_as_float(d[m]) : 0.f;
         }
     }
@@ -180,15 +188,19 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
 
 }  // namespace
 
-size_t row_tc_smem_bytes(int nstage, size_t slot_bytes) { return (size_t)nstage * kStage + (3 * nstage + 1) * sizeof(uint64_t) + 16 + slot_bytes + 1024; }
+int row_tc_tokens(int M) { return M <= 16 ? 16 : (M <= 32 ? 32 : 64); }
+size_t row_tc_smem_bytes(int nstage, size_t slot_bytes, int tokens)
+{
+    return (size_t)nstage * (kBStage + tokens * kTcKT * 2) + (3 * nstage + 1) * sizeof(uint64_t) + 16 + slot_bytes + 1024;
+}
 
-template <typename TO, bool kCol>
+template <typename TO, bool kCol, int kTok>
 static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta_in, cudaStream_t s)
 {
     TmaArgs ta = ta_in;
     const MatmulArgs &a = ta.base;
     static bool configured = false;
-    auto kern = nm_row_tc_kernel<TO, kCol>;
+    auto kern = nm_row_tc_kernel<TO, kCol, kTok>;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
@@ -197,7 +209,7 @@ static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a,
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.ntiles, a.nsplit, a.H);
     cfg.blockDim = dim3(kTcThreads);
-    cfg.dynamicSmemBytes = row_tc_smem_bytes(ta.nstage, ta.cluster_split ? (size_t)a.nsplit * a.M * kTcTN * sizeof(float) : 0);
+    cfg.dynamicSmemBytes = row_tc_smem_bytes(ta.nstage, ta.cluster_split ? (size_t)a.nsplit * a.M * kTcTN * sizeof(float) : 0, kTok);
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
     int na = 0;
@@ -215,7 +227,7 @@ static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a,
     cfg.numAttrs = na;
     if (ta.cluster_split && !clusters_fit_one_wave(kern, cfg, (unsigned)a.nsplit, (long)a.ntiles * a.H)) {
         ta.cluster_split = 0;                                      // through the workspace instead (the caller provided it)
-        cfg.dynamicSmemBytes = row_tc_smem_bytes(ta.nstage, 0);
+        cfg.dynamicSmemBytes = row_tc_smem_bytes(ta.nstage, 0, kTok);
         cfg.numAttrs = na - 1;                                     // the cluster attribute is the last one
     }
     return cudaLaunchKernelEx(&cfg, kern, map_b, map_a, ta);
@@ -223,14 +235,14 @@ static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a,
 
 // How many clusters of `cluster_size` CTAs of this kernel (ring of `nstage` stages, slots for M tokens) the GPU holds
 // at once; 0 when it cannot be asked (no device).  The planner sizes the k-split with it.
-template <typename TO, bool kCol>
+template <typename TO, bool kCol, int kTok>
 static int max_clusters_tc(int cluster_size, int nstage, int M)
 {
-    auto kern = nm_row_tc_kernel<TO, kCol>;
+    auto kern = nm_row_tc_kernel<TO, kCol, kTok>;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(1, cluster_size, 1);
     cfg.blockDim = dim3(kTcThreads);
-    cfg.dynamicSmemBytes = row_tc_smem_bytes(nstage, (size_t)cluster_size * M * kTcTN * sizeof(float));
+    cfg.dynamicSmemBytes = row_tc_smem_bytes(nstage, (size_t)cluster_size * M * kTcTN * sizeof(float), kTok);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)cluster_size; attr[0].val.clusterDim.z = 1;
@@ -240,16 +252,36 @@ static int max_clusters_tc(int cluster_size, int nstage, int M)
     return max_clusters_cached(kern, cfg, (unsigned)cluster_size);
 }
 
+template <typename TO, bool kCol>
+static int max_clusters_by_tokens(int cluster_size, int nstage, int M)
+{
+    switch (row_tc_tokens(M)) {
+    case 16: return max_clusters_tc<TO, kCol, 16>(cluster_size, nstage, M);
+    case 32: return max_clusters_tc<TO, kCol, 32>(cluster_size, nstage, M);
+    default: return max_clusters_tc<TO, kCol, 64>(cluster_size, nstage, M);
+    }
+}
+
 int row_tc_max_clusters(int cluster_size, int nstage, int M, bool col_major, bool f32_out)
 {
-    if (col_major) return f32_out ? max_clusters_tc<float, true>(cluster_size, nstage, M) : max_clusters_tc<bf16_t, true>(cluster_size, nstage, M);
-    return f32_out ? max_clusters_tc<float, false>(cluster_size, nstage, M) : max_clusters_tc<bf16_t, false>(cluster_size, nstage, M);
+    if (col_major) return f32_out ? max_clusters_by_tokens<float, true>(cluster_size, nstage, M) : max_clusters_by_tokens<bf16_t, true>(cluster_size, nstage, M);
+    return f32_out ? max_clusters_by_tokens<float, false>(cluster_size, nstage, M) : max_clusters_by_tokens<bf16_t, false>(cluster_size, nstage, M);
+}
+
+template <typename TO, bool kCol>
+static cudaError_t launch_by_tokens(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta, cudaStream_t s)
+{
+    switch (row_tc_tokens(ta.base.M)) {
+    case 16: return launch_tc<TO, kCol, 16>(map_b, map_a, ta, s);
+    case 32: return launch_tc<TO, kCol, 32>(map_b, map_a, ta, s);
+    default: return launch_tc<TO, kCol, 64>(map_b, map_a, ta, s);
+    }
 }
 
 template <typename TO>
 cudaError_t launch_row_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, const TmaArgs &ta, cudaStream_t s, bool col_major)
 {
-    return col_major ? launch_tc<TO, true>(map_b, map_a, ta, s) : launch_tc<TO, false>(map_b, map_a, ta, s);
+    return col_major ? launch_by_tokens<TO, true>(map_b, map_a, ta, s) : launch_by_tokens<TO, false>(map_b, map_a, ta, s);
 }
 
 template cudaError_t launch_row_tc<bf16_t>(const CUtensorMap &, const CUtensorMap &, const TmaArgs &, cudaStream_t, bool);

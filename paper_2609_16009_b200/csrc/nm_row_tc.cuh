@@ -10,7 +10,9 @@ namespace nm {
 constexpr int kTcTN = 128;      // columns of C per CTA (the MMA's M)
 constexpr int kTcKT = 64;       // k-rows per stage
 
-size_t row_tc_smem_bytes(int nstage, size_t slot_bytes = 0);
+// Token columns of the accumulator for M tokens: 16, 32 or 64.
+int row_tc_tokens(int M);
+size_t row_tc_smem_bytes(int nstage, size_t slot_bytes = 0, int tokens = 16);
 // Clusters of `cluster_size` CTAs (split-K inside a cluster, M tokens) the GPU holds at once; 0 without a device.
 int row_tc_max_clusters(int cluster_size, int nstage, int M, bool col_major, bool f32_out);
 // map_b: row-major B as bf16 [H][K][N], boxes {64, 64, 1}; column-major B as bf16 [H][N][K], boxes {64, 128, 1}; both with

@@ -83,7 +83,9 @@ def test_argument_validation_needs_no_device(lib):
     lib.nm_matmul.argtypes = [vp, vp, vp] + [ctypes.c_int] * 5 + [vp]
     assert lib.nm_matmul(None, None, None, 1, 8, 8, 1, 0, None) == -1
     assert lib.nm_matmul(vp(256), vp(512), vp(1024), 0, 8, 8, 1, 0, None) == -1
-    assert lib.nm_matmul(vp(256), vp(512), vp(1024), 17, 8, 8, 1, 0, None) == -1
+    assert lib.nm_matmul(vp(256), vp(512), vp(1024), 65, 8, 8, 1, 0, None) == -1
+    # 17 to 64 rows: only operands the tensor-core kernel takes (bf16, tensor maps available); fp32 is refused
+    assert lib.nm_matmul(vp(256), vp(512), vp(1024), 17, 8, 8, 0, 0, None) == -2
     assert lib.nm_matmul(vp(256), vp(512), vp(1024), 1, 8, 8, 7, 0, None) == -2
     assert lib.nm_matmul(vp(257), vp(512), vp(1024), 1, 8, 8, 1, 0, None) == -3
     assert lib.nm_set_workspace(vp(4096), ctypes.c_size_t(16)) == -4

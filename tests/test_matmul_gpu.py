@@ -252,6 +252,39 @@ def test_split_k_inside_a_cluster_tensor_core_kernel(nm, layout, M, nsplit):
     nm.nm_check_status()
 
 
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("M,K,N,nsplit", [(17, 1000, 840, 0), (24, 2600, 328, 3), (32, 512, 1536, 0), (33, 1000, 840, 2),
+                                          (48, 7168, 576, 0), (64, 2600, 840, 5)])
+def test_more_than_sixteen_rows_in_one_pass_on_the_tensor_cores(nm, layout, M, K, N, nsplit):
+    """The paper's outlook (a remainder row beside a multiple of 16, larger tokens): up to 64 rows go through the
+    swap-AB tensor-core kernel with 32 or 64 token columns, B still streamed once.  Parity with the oracle,
+    both weight layouts, with and without k-splits (cluster and workspace paths)."""
+    A, B = gen.narrow_bf16(M, K, N, seed=1100 + M)
+    for cluster in (True, False):
+        nm.nm_debug_set_plan(0, nsplit)
+        nm.nm_debug_set_cluster_split(cluster)
+        try:
+            assert nm.nm_debug_get_plan(M, N, K, 1, BF16, layout)["kind"] == 4
+            run_case(nm, A, B, M, N, K, BF16, layout, f"M={M} K={K} N={N} nsplit={nsplit} layout={layout} cluster={cluster}")
+        finally:
+            nm.nm_debug_set_plan(0, 0)
+            nm.nm_debug_set_cluster_split(True)
+    nm.nm_check_status()
+
+
+def test_more_than_sixteen_rows_needs_operands_the_tensor_core_kernel_takes(nm):
+    M, K, N = 20, 256, 256
+    A, B = make_inputs(M, K, N, F32, seed=1200)
+    dA, dB = to_dev(A), to_dev(B)
+    whole, dC = out_buffer(M * N, F32)
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_matmul(dA, dB, dC, M, N, K, F32, ROW)
+    assert e.value.status == -2
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_matmul(dA, dB, dC, 65, N, K, BF16, ROW)
+    assert e.value.status == -1
+
+
 def test_paper_matmul_2_shape_takes_eight_splits_in_a_cluster(nm):
     plan = nm.nm_debug_get_plan(1, 576, 7168)
     assert plan["kind"] == 3 and plan["nsplit"] == 8
@@ -439,7 +472,7 @@ def test_error_codes(nm):
         except nm.NmError as e:
             return e.status
     assert status(nm.nm_matmul, A, B, Cb, 0, 64, 64, BF16, ROW) == -1
-    assert status(nm.nm_matmul, A, B, Cb, 17, 64, 64, BF16, ROW) == -1
+    assert status(nm.nm_matmul, A, B, Cb, 65, 64, 64, BF16, ROW) == -1
     assert status(nm.nm_matmul, A, B, Cb, 1, 0, 64, BF16, ROW) == -1
     assert status(nm.nm_matmul, None, B, Cb, 1, 64, 64, BF16, ROW) == -1
     assert status(nm.nm_matmul, A, B, Cb, 1, 64, 64, 9, ROW) == -2

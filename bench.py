@@ -428,6 +428,8 @@ def matmul_sweep(nm, device):
              (1, 7168, 576, 1, "bf16")]
     for M in (1, 2, 4, 8, 16):
         cases += [(M, 1536, 24576, 0, "bf16"), (M, 7168, 18432, 0, "bf16")]
+    # beyond the narrow range: a remainder row on top of 16, and 64 rows, still one pass over B (tensor cores)
+    cases += [(17, 7168, 18432, 0, "bf16"), (64, 7168, 18432, 0, "bf16")]
     # the per-head products of the absorbed MLA form, T tokens at once: q_nope * W_UK (128 -> 512) and
     # o_lat * W_UV (512 -> 128), 128 heads, activations laid out [T][128][K]
     for T in (1, 4, 16):

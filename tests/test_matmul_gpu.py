@@ -442,6 +442,40 @@ def test_batched_small_ragged(nm, layout):
     assert_matmul_close(out_to_f64(dC, BF16_F32OUT), Cq, C64, bound, BF16_F32OUT, "batched ragged")
 
 
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("T,kernel,nsplit", [(1, 3, 4), (2, 0, 3), (2, -1, 2), (5, 4, 3), (16, 4, 2), (24, -1, 0), (40, -1, 2)])
+def test_batched_products_with_k_splits_in_clusters_and_with_many_rows(nm, T, kernel, nsplit, layout):
+    """Per-head batches (heads = gridDim.z) through every kernel family with forced k-splits - the splits of a
+    (head, tile) meet inside a cluster - and with 17 to 64 rows per head on the tensor cores."""
+    H, K, N = 6, 1280, 256
+    if layout == COL and kernel in (0, 3):
+        kernel = -1                                               # the row-major CUDA-core kernels do not take column-major B
+    A = gen.normal_bf16((T, H, K), 1.0, seed=3300 + T)
+    W = gen.normal_bf16((H, K, N), 0.02, seed=3301 + T)
+    Wst = W if layout == ROW else np.ascontiguousarray(W.transpose(0, 2, 1))
+    dA, dW = to_dev(A), to_dev(Wst)
+    Cq, C64, bound = oracle.matmul_batched(A, Wst, T, N, K, H, H * K, K, K * N, H * N, N, T * H * N,
+                                           oracle.BF16, oracle.F32, layout)
+    outs = []
+    for cluster in (True, False):
+        whole, dC = out_buffer(T * H * N, BF16_F32OUT)
+        nm.nm_debug_set_plan(0, nsplit)
+        nm.nm_debug_set_kernel(kernel, 0)
+        nm.nm_debug_set_cluster_split(cluster)
+        try:
+            nm.nm_matmul_batched(dA, dW, dC, T, N, K, H, H * K, K, K * N, H * N, N, BF16_F32OUT, layout)
+            torch.cuda.synchronize()
+        finally:
+            nm.nm_debug_set_plan(0, 0)
+            nm.nm_debug_set_kernel(-1, 0)
+            nm.nm_debug_set_cluster_split(True)
+        assert guards_intact(whole, T * H * N, BF16_F32OUT)
+        assert_matmul_close(out_to_f64(dC, BF16_F32OUT), Cq, C64, bound, BF16_F32OUT, f"batched T={T} kernel={kernel} cluster={cluster}")
+        outs.append(dC.clone())
+    assert torch.equal(outs[0], outs[1])
+    nm.nm_check_status()
+
+
 # ---- host-operand entry point ------------------------------------------------------------------------------
 
 def test_matmul_host_operands(nm):

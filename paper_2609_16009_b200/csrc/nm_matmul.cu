@@ -389,12 +389,17 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
                 ta.norm = *extras->norm;
                 extras->norm_taken = true;
             }
-            if (extras->dry_run) return NM_OK;
         }
+        const bool query = extras && extras->dry_run;
         const bool f32out = (dtype == NM_BF16_F32OUT);
-        if (p.tpr == 8)       e = f32out ? launch_row_tma<8, float>(*map, ta, smem, stream)  : launch_row_tma<8, bf16_t>(*map, ta, smem, stream);
-        else if (p.tpr == 16) e = f32out ? launch_row_tma<16, float>(*map, ta, smem, stream) : launch_row_tma<16, bf16_t>(*map, ta, smem, stream);
-        else                  e = f32out ? launch_row_tma<32, float>(*map, ta, smem, stream) : launch_row_tma<32, bf16_t>(*map, ta, smem, stream);
+        if (p.tpr == 8)       e = f32out ? launch_row_tma<8, float>(*map, ta, smem, stream, query)  : launch_row_tma<8, bf16_t>(*map, ta, smem, stream, query);
+        else if (p.tpr == 16) e = f32out ? launch_row_tma<16, float>(*map, ta, smem, stream, query) : launch_row_tma<16, bf16_t>(*map, ta, smem, stream, query);
+        else                  e = f32out ? launch_row_tma<32, float>(*map, ta, smem, stream, query) : launch_row_tma<32, bf16_t>(*map, ta, smem, stream, query);
+        if (query) {
+            // dry run: what the plan would do; per-tile sums of squares only when the clusters are all resident at once
+            if (e != cudaSuccess) { (void)cudaGetLastError(); extras->tile_ss_taken = false; }
+            return NM_OK;
+        }
     } else if (p.kind == kGeneric) {
         if (dtype == NM_F32)            e = launch_generic<float, float>(a, layout, stream);
         else if (dtype == NM_BF16)      e = launch_generic<bf16_t, bf16_t>(a, layout, stream);

@@ -367,7 +367,7 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
 }
 
 template <int TPR, typename TO>
-cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta_in, size_t smem_bytes, cudaStream_t s)
+cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta_in, size_t smem_bytes, cudaStream_t s, bool query_only)
 {
     TmaArgs ta = ta_in;
     const MatmulArgs &a = ta.base;
@@ -400,10 +400,10 @@ cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta_in, size_t
             if (e != cudaSuccess) return e;                                                               \
             configured = true;                                                                            \
         }                                                                                                 \
-        /* clusters that would need a second wave: through the workspace instead, unless the caller counts on the */ \
-        /* per-tile sums of squares, which only the cluster path writes */                               \
-        if (ta.cluster_split && !ta.tile_ss && a.partial &&                                               \
-            !clusters_fit_one_wave(kern, cfg, (unsigned)a.nsplit, (long)a.ntiles * a.H)) {                \
+        /* clusters that would need a second wave: through the workspace instead (query_only: just say so) */ \
+        const bool fits = !ta.cluster_split || clusters_fit_one_wave(kern, cfg, (unsigned)a.nsplit, (long)a.ntiles * a.H); \
+        if (query_only) return fits ? cudaSuccess : cudaErrorLaunchOutOfResources;                       \
+        if (!fits && !ta.tile_ss && a.partial) {     /* the per-tile sums of squares exist on the cluster path only */ \
             ta.cluster_split = 0;                                                                         \
             cfg.numAttrs = na - 1;                                                                        \
         }                                                                                                 \
@@ -416,8 +416,8 @@ cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta_in, size_t
 }
 
 #define NM_INSTANTIATE_TMA(TPR, TO) \
-    template cudaError_t launch_row_tma<TPR, TO>(const CUtensorMap &, const TmaArgs &, size_t, cudaStream_t);
+    template cudaError_t launch_row_tma<TPR, TO>(const CUtensorMap &, const TmaArgs &, size_t, cudaStream_t, bool);
 #define NM_EXTERN_TMA(TPR, TO) \
-    extern template cudaError_t launch_row_tma<TPR, TO>(const CUtensorMap &, const TmaArgs &, size_t, cudaStream_t);
+    extern template cudaError_t launch_row_tma<TPR, TO>(const CUtensorMap &, const TmaArgs &, size_t, cudaStream_t, bool);
 
 }  // namespace nm

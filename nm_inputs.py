@@ -60,6 +60,14 @@ def to_col_major(B_rowmajor: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(B_rowmajor.T)
 
 
+def to_fractal_nz(B_rowmajor: np.ndarray) -> np.ndarray:
+    """Storage of the same K x N matrix in 16 x 16 fractals, fractals ordered by columns, elements inside a fractal by
+    rows (K and N multiples of 16).  A pure permutation: [K/16, 16, N/16, 16] -> [N/16, K/16, 16, 16], flattened."""
+    K, N = B_rowmajor.shape
+    assert K % 16 == 0 and N % 16 == 0
+    return np.ascontiguousarray(B_rowmajor.reshape(K // 16, 16, N // 16, 16).transpose(2, 0, 1, 3)).reshape(-1)
+
+
 def gemv_fp32(seed: int = 0, K: int = 512, N: int = 512, M: int = 1):
     """fp32 GEMV case: both operands uniform[-1, 1] from one generator stream (A first)."""
     g = _gen(seed)

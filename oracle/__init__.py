@@ -18,7 +18,7 @@ _SRC = os.path.join(_HERE, "nm_oracle.c")
 _LIB = os.path.join(_HERE, "libnm_oracle.so")
 
 F32, BF16, F64 = 0, 1, 3
-ROW_MAJOR, COL_MAJOR = 0, 1
+ROW_MAJOR, COL_MAJOR, FRACTAL_NZ = 0, 1, 2
 
 _np_dtype = {F32: np.float32, BF16: np.uint16, F64: np.float64}
 

@@ -34,7 +34,7 @@
 #endif
 
 enum { NMO_F32 = 0, NMO_BF16 = 1, NMO_F64 = 3 };
-enum { NMO_ROW_MAJOR = 0, NMO_COL_MAJOR = 1 };
+enum { NMO_ROW_MAJOR = 0, NMO_COL_MAJOR = 1, NMO_FRACTAL_NZ = 2 };
 
 /* ---- exact widening and single-step rounding ------------------------------------- */
 
@@ -110,9 +110,21 @@ void nmo_quantize_bf16(double *x, long n)
 /*
  * C[m,n] = sum_k A[m,k] * B[k,n], k increasing, fp64.  A is row-major MxK (element (m,k) at
  * m*lda + k); B element (k,n) sits at k*ldb + n (row-major) or n*ldb + k (column-major, i.e. an
- * [out,in] weight such as W^{DKV} in R^{d_c x d}); C64 (optional) receives the unrounded sums,
+ * [out,in] weight such as W^{DKV} in R^{d_c x d}) or at fractal_nz_index (FRACTAL_NZ; ldb unused); C64 (optional)
+ * receives the unrounded sums,
  * C (optional) the sums rounded once to out_dtype, bound (optional) sum_k |a*b|.
  */
+/*
+ * FRACTAL_NZ, the tiling the paper's weight matrices have in memory (MLA Operator Optimization; figure of the
+ * special formats): the K x N matrix is cut into 16 x 16 fractals; the fractals are ordered by columns (all
+ * fractals of the first 16 columns from top to bottom, then the next 16 columns), the 256 elements inside a
+ * fractal by rows.  K and N are multiples of 16.
+ */
+static long fractal_nz_index(int k, int n, int K)
+{
+    return ((long)(n / 16) * (K / 16) + k / 16) * 256 + (long)(k % 16) * 16 + n % 16;
+}
+
 void nmo_matmul_strided(const void *A, const void *B, void *C, double *C64, double *bound,
                         int M, int N, int K, long lda, long ldb, long ldc,
                         int in_dtype, int out_dtype, int layout_B, int threads)
@@ -125,7 +137,10 @@ void nmo_matmul_strided(const void *A, const void *B, void *C, double *C64, doub
         for (int m = 0; m < M; ++m) {
             double acc = 0.0, s = 0.0;
             for (int k = 0; k < K; ++k) {
-                long ib = (layout_B == NMO_ROW_MAJOR) ? (long)k * ldb + n : (long)n * ldb + k;
+                long ib;
+                if (layout_B == NMO_ROW_MAJOR)      ib = (long)k * ldb + n;
+                else if (layout_B == NMO_COL_MAJOR) ib = (long)n * ldb + k;
+                else                                ib = fractal_nz_index(k, n, K);
                 double p = load_as_f64(A, (long)m * lda + k, in_dtype) * load_as_f64(B, ib, in_dtype);
                 acc += p;
                 s += fabs(p);

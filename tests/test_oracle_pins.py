@@ -145,6 +145,42 @@ def test_identity_and_one_hot(layout):
     assert np.array_equal(Cq, A[:, ks])                                # column n = e_k -> A[:, k]
 
 
+# ---- P5b: FRACTAL_NZ storage (the layout the paper's weight matrices have in memory) ---------------
+
+def _fractal_nz_by_loops(B):
+    """16 x 16 fractals, fractal columns one after the other (within one, the fractals from top to bottom), rows of a
+    fractal one after the other - written out with loops, independently of the oracle's index formula and of
+    the generator module's reshape."""
+    K, N = B.shape
+    out = []
+    for nb in range(N // 16):
+        for kb in range(K // 16):
+            for kr in range(16):
+                for nc in range(16):
+                    out.append(B[kb * 16 + kr, nb * 16 + nc])
+    return np.array(out, dtype=B.dtype)
+
+
+def test_fractal_nz_storage():
+    M, K, N = 3, 48, 32
+    A = gen.normal_bf16((M, K), 1.0, seed=61)
+    B = gen.normal_bf16((K, N), 0.02, seed=62)
+    Bnz = _fractal_nz_by_loops(B)
+    assert np.array_equal(Bnz, gen.to_fractal_nz(B))                   # the generator's permutation is the same storage
+    # first fractal = rows 0-15 x columns 0-15 row by row; second = rows 16-31 of the SAME 16 columns
+    assert np.array_equal(Bnz[:16], B[0, :16]) and np.array_equal(Bnz[16:32], B[1, :16])
+    assert np.array_equal(Bnz[256:272], B[16, :16]) and np.array_equal(Bnz[3 * 256:3 * 256 + 16], B[0, 16:32])
+    Cq, C64, bound = oracle.matmul(A, Bnz, M, N, K, BF16, F32, oracle.FRACTAL_NZ)
+    Cq_r, C64_r, bound_r = oracle.matmul(A, B, M, N, K, BF16, F32, ROW_MAJOR)
+    assert np.array_equal(C64, C64_r) and np.array_equal(bound, bound_r)   # same products in the same order
+    for k in (0, 17, K - 1):                                            # A = e_k -> row k of B, exactly
+        e = np.zeros((1, K), np.float32); e[0, k] = 1.0
+        Cq, _, _ = oracle.matmul(_bits(e), Bnz, 1, N, K, BF16, BF16, oracle.FRACTAL_NZ)
+        assert np.array_equal(Cq[0], B[k])
+    ref = gen.bits_to_f32(A).astype(np.float64) @ gen.bits_to_f32(B).astype(np.float64)
+    assert np.all(np.abs(C64 - ref) <= 1e-12 * bound)                   # numpy on the logical matrix
+
+
 # ---- P6: closed forms ---------------------------------------------------------------------------
 
 @pytest.mark.parametrize("layout", [ROW_MAJOR, COL_MAJOR])

@@ -37,7 +37,12 @@ typedef enum {
     NM_BF16_F32OUT = 2            /* bf16 in, fp32 accumulate, fp32 out (unrounded sums) */
 } nm_dtype;
 
-typedef enum { NM_ROW_MAJOR = 0, NM_COL_MAJOR = 1 } nm_layout;
+/* Storage of B (K x N).  NM_FRACTAL_NZ: the tiling the paper's weight matrices have in memory (MLA Operator
+ * Optimization section, figure of the special formats) - 16 x 16 fractals, the fractals ordered by columns (those of
+ * the first 16 columns from top to bottom, then the next 16 columns), the elements of a fractal by rows: element
+ * (k, n) at ((n/16)*(K/16) + k/16)*256 + (k%16)*16 + n%16.  bf16 only, K and N multiples of 16, M <= 16; read in
+ * place by tiled TMA copies, no transposition pass.  NM_ERR_UNSUPPORTED otherwise. */
+typedef enum { NM_ROW_MAJOR = 0, NM_COL_MAJOR = 1, NM_FRACTAL_NZ = 2 } nm_layout;
 
 enum {
     NM_OK = 0,

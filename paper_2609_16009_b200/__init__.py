@@ -16,7 +16,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libnm.so")
 
 F32, BF16, BF16_F32OUT = 0, 1, 2
-ROW_MAJOR, COL_MAJOR = 0, 1
+ROW_MAJOR, COL_MAJOR, FRACTAL_NZ = 0, 1, 2
 MAX_M = 16
 WS_COUNTER_BYTES = 65536
 

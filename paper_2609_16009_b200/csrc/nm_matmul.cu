@@ -176,6 +176,16 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
 {
     Plan p{};
     const int V = vec_elems(dtype);
+    if (layout == NM_FRACTAL_NZ) {
+        // fractal storage goes through the TMA ring kernel whatever M: its tiled copies read the fractals in place
+        p = make_tma_plan(M, N, K, H, chained);
+        const int kt = (kTmaConsumers / p.tpr) * 4;
+        if (p.kr % kt) {                                   // forced split counts: whole stages per split all the same
+            p.kr = ceil_div(p.kr, kt) * kt;
+            p.nsplit = ceil_div(K, p.kr);
+        }
+        return p;
+    }
     if (!vec_ok) {
         p.kind = kGeneric; p.tn = kThreads; p.ntiles = ceil_div(N, kThreads); p.nsplit = 1; p.kr = K;
         p.tpr = p.rg = 0;
@@ -270,6 +280,33 @@ static const CUtensorMap *get_weight_map(const void *B, int N, int K, int H, lon
     return e.valid ? &e.map : nullptr;
 }
 
+// B in 16 x 16 fractals (element (k, n) at ((n/16)*(K/16) + k/16)*256 + (k%16)*16 + n%16) as a 4-D tensor: element in
+// fractal (256, contiguous), fractal row, fractal column, head.  A box of kt x tn elements - kt/16 contiguous
+// fractals from each of tn/16 fractal columns - lands in shared memory as [tn/16][kt][16].  Cached with the other maps (marked by a
+// negative tile width).
+static const CUtensorMap *get_fractal_map(const void *B, int N, int K, int H, long strideB, int tn, int kt)
+{
+    for (auto &e : g_maps) {
+        const MapKey &k = e.key;
+        if (e.valid && k.B == B && k.N == N && k.K == K && k.H == H && k.strideB == strideB && k.tn == -tn && k.kt == kt) return &e.map;
+    }
+    EncodeTiledFn enc = tensor_map_encoder();
+    if (!enc) return nullptr;
+    MapEntry &e = g_maps[g_map_next];
+    g_map_next = (g_map_next + 1) % 16;
+    e.key = MapKey{B, N, K, H, strideB, -tn, kt};
+    e.row_stride = 0;
+    const cuuint64_t dims[4] = {256, (cuuint64_t)(K / 16), (cuuint64_t)(N / 16), (cuuint64_t)H};
+    const cuuint64_t strides[3] = {512, (cuuint64_t)(K / 16) * 512, (cuuint64_t)(H > 1 ? strideB : (long)K * N) * 2};
+    const cuuint32_t box[4] = {256, (cuuint32_t)(kt / 16), (cuuint32_t)(tn / 16), 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(B), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    e.valid = (r == CUDA_SUCCESS);
+    return e.valid ? &e.map : nullptr;
+}
+
 static size_t partial_floats(const Plan &p, int M, int H)
 {
     return p.nsplit > 1 ? (size_t)H * p.ntiles * p.nsplit * M * p.tn : 0;
@@ -281,7 +318,9 @@ static int check_common(const void *A, const void *B, const void *C, int M, int 
     if (!A || !B || !C) return NM_ERR_INVALID_ARG;
     if (M < 1 || M > NM_MAX_M_TENSOR || N < 1 || K < 1 || H < 1) return NM_ERR_INVALID_ARG;
     if (dtype != NM_F32 && dtype != NM_BF16 && dtype != NM_BF16_F32OUT) return NM_ERR_UNSUPPORTED;
-    if (layout != NM_ROW_MAJOR && layout != NM_COL_MAJOR) return NM_ERR_UNSUPPORTED;
+    if (layout != NM_ROW_MAJOR && layout != NM_COL_MAJOR && layout != NM_FRACTAL_NZ) return NM_ERR_UNSUPPORTED;
+    // 16 x 16 fractals: bf16, whole fractals, and only through the TMA ring kernel (up to 16 rows)
+    if (layout == NM_FRACTAL_NZ && (dtype == NM_F32 || (N % 16) || (K % 16) || M > NM_MAX_M)) return NM_ERR_UNSUPPORTED;
     if (H > 65535) return NM_ERR_UNSUPPORTED;
     const uintptr_t es = (uintptr_t)elem_size(dtype);
     const uintptr_t os = (dtype == NM_BF16) ? 2 : 4;
@@ -305,13 +344,14 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     // The 16-byte paths need B aligned with rows (columns) that stay aligned, and an aligned A for
     // the column kernel (it copies A into shared memory with 16-byte loads).
     const bool b_ok = aligned16(B) && (strideB % V == 0) &&
-                      (layout == NM_ROW_MAJOR ? (N % V == 0) : (K % V == 0));
+                      (layout == NM_COL_MAJOR ? (K % V == 0) : (N % V == 0));
     const bool a_ok = aligned16(A) && (lda % V == 0) && (strideA % V == 0);
     const bool vec_ok = b_ok && (layout == NM_ROW_MAJOR || a_ok);
     // tensor maps: 16-byte aligned operands and strides, bf16.  Row-major B may take the TMA ring kernel or the
     // tensor-core kernel; column-major B only the latter (its CUDA-core path is the plain column kernel).
     bool tma_ok = b_ok && a_ok && dtype != NM_F32 && tensor_map_encoder() != nullptr && (long)N * 2 < (1L << 40) && strideB >= 0;
     if (g_force_kind == kRowVec) tma_ok = false;
+    if (layout == NM_FRACTAL_NZ && !tma_ok) return NM_ERR_UNSUPPORTED;      // unaligned operands or no tensor-map encoder
     Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok, chained);
     // Copies, not pointers into the map cache: the second lookup may evict the entry the first one returned
     // (16 entries, replaced in turn), and the kernel would then get the token map in place of the weight map.
@@ -359,9 +399,11 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         e = (dtype == NM_BF16_F32OUT) ? launch_row_tc<float>(*mb, *ma, ta, stream, col) : launch_row_tc<bf16_t>(*mb, *ma, ta, stream, col);
     } else if (p.kind == kRowTma) {
         const int kt = (kTmaConsumers / p.tpr) * 4;
-        const CUtensorMap *map = get_weight_map(B, N, K, H, strideB, p.tn, kt);
+        const CUtensorMap *map = (layout == NM_FRACTAL_NZ) ? get_fractal_map(B, N, K, H, strideB, p.tn, kt)
+                                                           : get_weight_map(B, N, K, H, strideB, p.tn, kt);
         if (!map) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
         TmaArgs ta{};
+        ta.fractal_nz = (layout == NM_FRACTAL_NZ) ? 1 : 0;
         ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
         ta.trace = trace;
         if (tail && tail->enabled && M == 1 && dtype == NM_BF16 && H == 1 && ws && ws_bytes >= kCounterBytes && aligned16(ws) &&

@@ -106,6 +106,7 @@ struct TmaArgs {
     unsigned long long *trace;   // tuning aid: when non-null every CTA stores four timestamps (start, inputs ready, loop done, end)
     VecTail tail;
     int cluster_split;     // the k-splits of a tile form a thread-block cluster (1 x nsplit x 1): partial sums meet in shared memory
+    int fractal_nz;        // B is stored in 16 x 16 fractals (5-D tensor map): a stage arrives as [tile_n/16][KT][16] instead of [KT][tile_n]
     float *tile_ss;        // cluster split-K, M = 1: when non-null, tile t also stores the sum of squares of its rounded outputs at [t]
     RowNorm norm;
 };

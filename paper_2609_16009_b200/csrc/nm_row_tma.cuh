@@ -53,7 +53,10 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char *ring = smem_raw;
-    float *As = reinterpret_cast<float *>(smem_raw + (size_t)ta.nstage * STAGE);
+    // FRACTAL_NZ: a stage arrives as TN/16 fractal columns of [KT rows][16 columns] (KT * 32 bytes each)
+    constexpr int NZ_COL = KT * 32;
+    constexpr uint32_t stage_stride = STAGE;
+    float *As = reinterpret_cast<float *>(smem_raw + (size_t)ta.nstage * stage_stride);
     uint64_t *bars = reinterpret_cast<uint64_t *>(As + kAChunkFloats);
     __shared__ int s_last;
     __shared__ int s_abort;
@@ -104,14 +107,21 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
             for (; it < n_it; ++it) {
                 if (it >= NS && !mbar_try_wait(empty0 + 8 * s, ph) && !mbar_wait(empty0 + 8 * s, ph, &s_abort, ta.status)) break;
                 mbar_arrive_expect_tx(full0 + 8 * s, STAGE);
-                tma_load_3d(smem_u32(ring + (size_t)s * STAGE), &tmap, tile * TN, kb + it * KT, h, full0 + 8 * s, policy);
+                if (ta.fractal_nz) {    // coordinates: element in fractal, fractal row, fractal column, head
+                    tma_load_4d(smem_u32(ring + (size_t)s * stage_stride), &tmap, 0, (kb + it * KT) / 16, tile * (TN / 16), h, full0 + 8 * s, policy);
+                } else {
+                    tma_load_3d(smem_u32(ring + (size_t)s * stage_stride), &tmap, tile * TN, kb + it * KT, h, full0 + 8 * s, policy);
+                }
                 if (++s == NS) { s = 0; ph ^= 1; }
             }
             s_issued = it;
         }
     } else {
         // ---------------- consumers ---------------------------------------------------------------
-        const int tx = tid % TPR, ty = tid / TPR;
+        const int tx = tid % TPR, ty_plain = tid / TPR;
+        // FRACTAL_NZ: the eight threads that read together hold four fractal columns, whose rows alias in the shared-memory
+        // banks; fractal column g therefore takes the rows of every group of four in the order rotated by g
+        const int ty = ta.fractal_nz ? ((ty_plain & ~3) | ((ty_plain + (tx >> 1)) & 3)) : ty_plain;
         const bf16_t *__restrict__ A = (const bf16_t *)a.A + (long)h * a.strideA;
         if constexpr (M == 1 && sizeof(TO) == 2) {
             // whichever CTA ends up running the vector stages wants their constants in L2 by then
@@ -203,10 +213,13 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
         if (n_it > ITS_PER_CHUNK) fetch_chunk(kb + KCH);
 
         const int rows_last = (ke - kb) - (n_it - 1) * KT;            // rows in the last stage (1..KT)
-        const uint32_t boff = (uint32_t)(ty * TN + tx * 8) * 2;       // this thread's first row in a stage
+        // this thread's first row in a stage and the distance between its rows; a FRACTAL_NZ stage is a row of
+        // fractal columns, each [KT rows][16 columns]: the thread's eight columns are half of one fractal row
+        const uint32_t boff = ta.fractal_nz ? (uint32_t)((tx >> 1) * NZ_COL + ty * 32 + (tx & 1) * 16) : (uint32_t)(ty * TN + tx * 8) * 2;
+        const uint32_t rstride = ta.fractal_nz ? (uint32_t)RG * 32u : (uint32_t)RG * TN * 2u;
         const float *a_thread = As + ty * MP;
         auto do_row = [&](const unsigned char *stage, const float *ak, int i) {
-            const uint4 v = *reinterpret_cast<const uint4 *>(stage + (size_t)i * RG * TN * 2);
+            const uint4 v = *reinterpret_cast<const uint4 *>(stage + (size_t)i * rstride);
             float b[8];
             Elem<bf16_t>::unpack(v, b);
             const float *aki = ak + i * RG * MP;
@@ -247,7 +260,7 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
                 if (it + ITS_PER_CHUNK < n_it) fetch_chunk(kb + (it + ITS_PER_CHUNK) * KT);
             }
             if (!mbar_try_wait(full0 + 8 * s, ph)) mbar_wait(full0 + 8 * s, ph, &s_abort, ta.status);
-            const unsigned char *stage = ring + (size_t)s * STAGE + boff;
+            const unsigned char *stage = ring + (size_t)s * stage_stride + boff;
             const float *ak = a_thread + itc * (KT * MP);
             if (it + 1 < n_it || rows_last == KT) {
 #pragma unroll

@@ -285,6 +285,63 @@ def test_more_than_sixteen_rows_needs_operands_the_tensor_core_kernel_takes(nm):
     assert e.value.status == -1
 
 
+NZ = 2
+
+
+@pytest.mark.parametrize("M", [1, 2, 5, 16])
+@pytest.mark.parametrize("K,N,tile_n,nsplit", [(7168, 576, 0, 0), (1008, 848, 64, 3), (1008, 848, 128, 2), (2048, 1280, 256, 1),
+                                               (4096, 4096, 0, 0)])
+def test_fractal_nz_weights_read_in_place(nm, M, K, N, tile_n, nsplit):
+    """The paper's weight storage (16 x 16 fractals ordered by columns, rows inside) as a layout of B: tiled TMA copies
+    present the fractals to the ring kernel, no transposition pass.  Parity with the oracle on the fractal storage."""
+    A, B = gen.narrow_bf16(M, K, N, seed=1300 + M)
+    Bnz = gen.to_fractal_nz(B)
+    dA, dB, dBnz = to_dev(A), to_dev(B), to_dev(Bnz)
+    Cq, C64, bound = oracle.matmul(A, Bnz, M, N, K, ORACLE_IN[BF16], ORACLE_OUT[BF16], oracle.FRACTAL_NZ, threads=8)
+    nm.nm_debug_set_plan(tile_n, nsplit)
+    nm.nm_debug_set_kernel(3, 0)
+    try:
+        plan_nz, plan_row = nm.nm_debug_get_plan(M, N, K, 1, BF16, NZ), nm.nm_debug_get_plan(M, N, K, 1, BF16, ROW)
+        assert plan_nz["kind"] == 3
+        whole, dC = out_buffer(M * N, BF16)
+        nm.nm_matmul(dA, dBnz, dC, M, N, K, BF16, NZ)
+        whole_r, dC_r = out_buffer(M * N, BF16)
+        nm.nm_matmul(dA, dB, dC_r, M, N, K, BF16, ROW)
+        torch.cuda.synchronize()
+    finally:
+        nm.nm_debug_set_plan(0, 0)
+        nm.nm_debug_set_kernel(-1, 0)
+    assert guards_intact(whole, M * N, BF16)
+    assert_matmul_close(out_to_f64(dC, BF16).reshape(M, N), Cq, C64, bound, BF16, f"fractal M={M} K={K} N={N}")
+    # against the row-major storage of the same matrix: the same products, summed in another order (the fractal path
+    # deals the rows to the threads differently), so equal within the bound rather than bit for bit
+    assert plan_nz["tile_n"] == plan_row["tile_n"]
+    assert_matmul_close(out_to_f64(dC_r, BF16).reshape(M, N), Cq, C64, bound, BF16, f"row-major M={M} K={K} N={N}")
+    nm.nm_check_status()
+
+
+def test_fractal_nz_batched_and_refusals(nm):
+    T, H, K, N = 2, 4, 256, 96
+    A = gen.normal_bf16((T, H, K), 1.0, seed=1400)
+    W = gen.normal_bf16((H, K, N), 0.02, seed=1401)
+    Wnz = np.stack([gen.to_fractal_nz(W[h]) for h in range(H)])
+    dA, dW = to_dev(A), to_dev(Wnz)
+    whole, dC = out_buffer(T * H * N, BF16_F32OUT)
+    nm.nm_matmul_batched(dA, dW, dC, T, N, K, H, H * K, K, K * N, H * N, N, BF16_F32OUT, NZ)
+    torch.cuda.synchronize()
+    Cq, C64, bound = oracle.matmul_batched(A, W, T, N, K, H, H * K, K, K * N, H * N, N, T * H * N, oracle.BF16, oracle.F32, ROW)
+    assert guards_intact(whole, T * H * N, BF16_F32OUT)
+    assert_matmul_close(out_to_f64(dC, BF16_F32OUT), Cq, C64, bound, BF16_F32OUT, "fractal batched")
+    # partial fractals, fp32 and more than 16 rows are refused
+    Cb = torch.zeros(64 * 96, dtype=torch.int16, device="cuda")
+    for args in ((dA, dW, Cb, 1, 90, 256, BF16, NZ), (dA, dW, Cb, 1, 96, 250, BF16, NZ), (dA, dW, Cb, 1, 96, 256, F32, NZ),
+                 (dA, dW, Cb, 17, 96, 256, BF16, NZ)):
+        with pytest.raises(nm.NmError) as e:
+            nm.nm_matmul(*args)
+        assert e.value.status == -2
+    nm.nm_check_status()
+
+
 def test_paper_matmul_2_shape_takes_eight_splits_in_a_cluster(nm):
     plan = nm.nm_debug_get_plan(1, 576, 7168)
     assert plan["kind"] == 3 and plan["nsplit"] == 8

@@ -425,7 +425,9 @@ def matmul_sweep(nm, device):
     the decode step).  Reported beside the step; not part of the timed region."""
     out = []
     cases = [(1, 512, 512, 0, "f32"), (1, 7168, 1536, 0, "bf16"), (1, 7168, 576, 0, "bf16"), (1, 7168, 1536, 1, "bf16"),
-             (1, 7168, 576, 1, "bf16")]
+             (1, 7168, 576, 1, "bf16"),
+             # the storage the paper's test case has in memory (16 x 16 fractals): layout code 2
+             (1, 7168, 1536, 2, "bf16"), (1, 7168, 576, 2, "bf16"), (1, 7168, 18432, 2, "bf16")]
     for M in (1, 2, 4, 8, 16):
         cases += [(M, 1536, 24576, 0, "bf16"), (M, 7168, 18432, 0, "bf16")]
     # beyond the narrow range: a remainder row on top of 16, and 64 rows, still one pass over B (tensor cores)
@@ -450,7 +452,7 @@ def matmul_sweep(nm, device):
         C = torch.empty(R, M * N, device=device, dtype=tdt)
         ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(M, N, K), device=device)
         s = torch.cuda.Stream(device)
-        row = {"M": M, "K": K, "N": N, "dtype": dt, "layout_B": "col" if layout else "row"}
+        row = {"M": M, "K": K, "N": N, "dtype": dt, "layout_B": ("row", "col", "fractal_nz")[layout]}
         algo = (K * N + M * K + M * N) * es
         for mode in ("serial", "programmatic"):
             nm.nm_set_programmatic_launch(mode == "programmatic")

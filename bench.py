@@ -108,10 +108,11 @@ class MlaStep:
 
     name = "mla"
 
-    def __init__(self, nm, device, seq_len, seed=4000, schedule="fused"):
+    def __init__(self, nm, device, seq_len, seed=4000, schedule="fused", weights="row"):
         self.nm = nm
         self.S = seq_len
         self.schedule = schedule
+        self.weights = weights
         d, ql, dc, dr, dn, dv, H = (DIMS[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
         w = gen.mla_weights(DIMS, seed=seed, with_wo=True)
         t = {k: torch.from_numpy(v.view(np.int16)).to(device) for k, v in w.items()}
@@ -120,6 +121,14 @@ class MlaStep:
             # when the weights are loaded, like the paper's concatenation of W_DKV and W_KR
             t["W_DQKV"] = torch.from_numpy(np.concatenate([w["W_DQ"], w["W_DKVKR"]], axis=1).view(np.int16)).to(device)
             del t["W_DQ"], t["W_DKVKR"]
+        layout_dense = nm.ROW_MAJOR
+        if weights == "fractal":
+            # the storage of the paper's test case: the dense weights in 16 x 16 fractals (a permutation of the same values)
+            layout_dense = nm.FRACTAL_NZ
+            shapes = {"W_DQKV": (d, ql + dc + dr), "W_DQ": (d, ql), "W_DKVKR": (d, dc + dr), "W_UQR": (ql, H * (dn + dr)), "W_O": (H * dv, d)}
+            for name, (K_, N_) in shapes.items():
+                if name in t:
+                    t[name] = torch.from_numpy(gen.to_fractal_nz(t[name].cpu().numpy().reshape(K_, N_))).to(device)
         self.h_host = torch.from_numpy(gen.mla_token(DIMS, seed=seed + 100).view(np.int16).copy()).pin_memory()
         self.out_host = torch.empty(d, dtype=torch.int16).pin_memory()
         t["h"] = self.h_host.to(device)
@@ -128,9 +137,9 @@ class MlaStep:
         t["rope_cos_sin"] = torch.empty(dr, dtype=torch.float32, device=device)
         nm.nm_rope_table(t["rope_cos_sin"], seq_len - 1, 1, dr)
         self.t = t
-        p = nm.mla_params(DIMS, seq_len, t)
+        p = nm.mla_params(DIMS, seq_len, t, layout_dense=layout_dense)
         self.ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p), device=device)
-        self.p = nm.mla_params(DIMS, seq_len, t, workspace=self.ws)
+        self.p = nm.mla_params(DIMS, seq_len, t, workspace=self.ws, layout_dense=layout_dense)
         self.p.programmatic_entry = 1        # steps follow each other like the layers of a model: weights are static
         self.side = torch.cuda.Stream(device)
         self.graph = None
@@ -149,7 +158,8 @@ class MlaStep:
 
     def describe(self):
         return {"workload": f"full single-token MLA decode step, DeepSeek-V3 dims (hidden 7168, q_lora 1536, kv_lora 512, rope 64, "
-                            f"nope 128, v 128, 128 heads), seq_len {self.S}, bf16 weights row-major, W_O included",
+                            f"nope 128, v 128, 128 heads), seq_len {self.S}, bf16 weights "
+                            + ("row-major" if self.weights == "row" else "in FRACTAL_NZ storage") + ", W_O included",
                 "seq_len": self.S,
                 "l2": "weights 374 MB per step > 126 MB L2, so every step streams from HBM; no flush",
                 "schedule": self.schedule,
@@ -193,7 +203,7 @@ class MlaStep:
         # the small-batch step (nm_mla_decode_batch): T sequences of this length, one new token each
         out["small_batch"] = []
         dkv = DIMS["kv_lora"] + DIMS["rope"]
-        for T in (4, 16):
+        for T in ((4, 16) if self.weights == "row" else ()):       # the batch entry point takes row- / column-major weights
             stride = (self.S + 8) * dkv
             cache = self.t["kv_cache"].view(-1)[:self.S * dkv].repeat(T, 1)
             cache = torch.nn.functional.pad(cache, (0, stride - self.S * dkv)).contiguous().view(-1)
@@ -323,7 +333,7 @@ def make_workload(args, nm, device):
     if args.workload == "projections":
         return ProjectionChain(nm, device)
     if args.workload == "mla":
-        return MlaStep(nm, device, args.seq_len, schedule=args.schedule)
+        return MlaStep(nm, device, args.seq_len, schedule=args.schedule, weights=args.weights)
     if args.workload == "matmul":
         M, K, N = (int(x) for x in args.mkn.split(","))
         return SingleProduct(nm, device, M, K, N, 1 if args.layout == "col" else 0)
@@ -659,6 +669,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="also report GB/s of single narrow products vs M")
     ap.add_argument("--seq-len", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--weights", default="row", choices=["row", "fractal"],
+                    help="storage of the step's dense weights: row-major (default) or the paper's FRACTAL_NZ tiling")
     ap.add_argument("--attention", default="auto", choices=["auto", "64", "128", "cuda-cores"],
                     help="attention kernel: chosen by length (default), tensor cores with 64 or 128 heads per CTA, CUDA cores")
     args = ap.parse_args()

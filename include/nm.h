@@ -232,7 +232,7 @@ int nm_mla_attention_combine(const void *Q, const void *kv_cache, void *o_bf16, 
 typedef struct {
     int d, q_lora, kv_lora, rope, nope, v, H;
     int seq_len;
-    int layout_dense;              /* nm_layout of W_DQ, W_UQR, W_DKVKR, W_O */
+    int layout_dense;              /* nm_layout of W_DQ, W_UQR, W_DKVKR, W_DQKV, W_O (NM_FRACTAL_NZ: single-token step only) */
     float rms_eps, softmax_scale;
     const void *h, *W_DQ, *gamma_q, *W_UQR, *W_DKVKR, *gamma_kv, *W_UK, *W_UV, *W_O;
     const float *rope_cos_sin;
@@ -251,7 +251,7 @@ typedef struct {
     int programmatic_entry;
     /* optional: the three down-projections stored as ONE row-major matrix [d][q_lora + kv_lora + rope] =
      * (W_DQ | W_DKV | W_KR), the paper's concatenation of Eq. 3 extended by W_DQ (all three multiply the
-     * same h).  When given (and layout_dense is row-major) the step computes them as one product on
+     * same h).  When given (and layout_dense is row-major or NM_FRACTAL_NZ) the step computes them as one product on
      * main_stream and needs no side stream; W_DQ and W_DKVKR are then ignored and may be NULL. */
     const void *W_DQKV;
 } nm_mla_params;

@@ -444,7 +444,7 @@ static int check_params(const nm_mla_params *p)
     if (p->d < 1 || p->q_lora < 1 || p->H < 1 || p->nope < 1 || p->v < 1 || p->seq_len < 1) return NM_ERR_INVALID_ARG;
     if (p->kv_lora != 512 || p->rope != 64) return NM_ERR_UNSUPPORTED;
     if (p->q_lora > 16384) return NM_ERR_UNSUPPORTED;
-    if (p->layout_dense != NM_ROW_MAJOR && p->layout_dense != NM_COL_MAJOR) return NM_ERR_UNSUPPORTED;
+    if (p->layout_dense != NM_ROW_MAJOR && p->layout_dense != NM_COL_MAJOR && p->layout_dense != NM_FRACTAL_NZ) return NM_ERR_UNSUPPORTED;
     return NM_OK;
 }
 
@@ -482,7 +482,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     uint16_t *o_lat = (uint16_t *)buf(p->o_lat, L.o_lat), *o = (uint16_t *)buf(p->o, L.o);
     uint16_t *cache = static_cast<uint16_t *>(p->kv_cache);
     void *mws = ws + L.main_ws, *sws = ws + L.side_ws, *aws = ws + L.attn;
-    const bool forked = (ss != ms) && !(p->W_DQKV && p->layout_dense == NM_ROW_MAJOR && down_finish_applies(p->q_lora, p->kv_lora, p->rope));
+    const bool forked = (ss != ms) && !(p->W_DQKV && p->layout_dense != NM_COL_MAJOR && down_finish_applies(p->q_lora, p->kv_lora, p->rope));
     if (forked && !g_events.fork) {
         NM_CUDA_TRY(cudaEventCreateWithFlags(&g_events.fork, cudaEventDisableTiming));
         NM_CUDA_TRY(cudaEventCreateWithFlags(&g_events.join, cudaEventDisableTiming));
@@ -508,7 +508,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     tkv.enabled = 1; tkv.kv_off = 0; tkv.dc = dc; tkv.rope = dr; tkv.eps = p->rms_eps; tkv.gamma_kv = (const uint16_t *)p->gamma_kv;
     tkv.cos_sin = p->rope_cos_sin; tkv.cache_row = cache + (size_t)pos * dkv;
     bool taken = false;
-    const bool fused_down = p->W_DQKV && lay == NM_ROW_MAJOR && down_finish_applies(ql, dc, dr);
+    const bool fused_down = p->W_DQKV && lay != NM_COL_MAJOR && down_finish_applies(ql, dc, dr);      // row-major or fractal storage
     // Where the plans allow: the k-splits of the fused down-projection meet inside clusters, each
     // tile leaves the sum of squares of its outputs, the W_UQR product applies RMSNorm to its token row while
     // loading it, and the KV consumers ride in an extra CTA of the per-head query kernel - the down-projection then
@@ -523,7 +523,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         ex_d.tile_ss = tile_ss; ex_d.dry_run = true;
         {
             ScopedPlan sp(g_step_plan[0]);
-            NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws,
+            NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws,
                                   L.main_ws_bytes, ms, false, nullptr, nullptr, nullptr, true, &ex_d));
         }
         if (ex_d.tile_ss_taken && ex_d.tile_n > 0 && ql % ex_d.tile_n == 0 && ql / ex_d.tile_n <= 32) {
@@ -542,7 +542,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         ex_d.tile_ss = tile_ss;
         {
             ScopedPlan sp(g_step_plan[0]);
-            NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws,
+            NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws,
                                   L.main_ws_bytes, ms, pdl && p->programmatic_entry, trace_at(2048), nullptr, nullptr, true, &ex_d));
         }
         if (!ex_d.tile_ss_taken) return NM_ERR_UNSUPPORTED;        // the dry run said otherwise
@@ -557,7 +557,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         VecTail both = tq;
         both.kv_off = ql; both.dc = dc; both.rope = dr; both.gamma_kv = tkv.gamma_kv; both.cos_sin = tkv.cos_sin; both.cache_row = tkv.cache_row;
         ScopedPlan sp(g_step_plan[0]);
-        NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws,
+        NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws,
                               L.main_ws_bytes, ms, pdl && p->programmatic_entry, trace_at(2048), tails_ok ? &both : nullptr, &taken, true));
         if (!taken)
             NM_TRY(launch_down_finish(x_down, p->gamma_q, p->gamma_kv, p->rope_cos_sin, c_qn, cache + (size_t)pos * dkv, ql, dc, dr,
@@ -623,6 +623,14 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
             if (rows > kr) rows = kr;
             pf.base = (const char *)p->W_O; pf.range_stride = (long)kr * row_bytes; pf.nranges = rows > 0 ? ns : 0;
             pf.range_bytes = rows * row_bytes;
+        } else if (p->W_O && lay == NM_FRACTAL_NZ) {
+            // fractal storage: every fractal column (16 columns, all K rows) is contiguous; the product starts each of
+            // them at row 0, so the head of every fractal column is what it reads first
+            const long K_o = (long)H * dv, cols = d / 16;
+            long rows = (((long)g_prefetch_mb << 20) / cols / 32) / 16 * 16;
+            if (rows > K_o) rows = K_o;
+            pf.base = (const char *)p->W_O; pf.range_stride = K_o * 32; pf.nranges = rows > 0 ? (int)cols : 0;
+            pf.range_bytes = rows * 32;
         }
     }
 

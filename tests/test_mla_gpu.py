@@ -231,7 +231,7 @@ def test_attention_kernels_agree_on_heavy_tailed_scores(nm):
 
 # ---- the whole step ---------------------------------------------------------------------------------------
 
-def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None, concat_down=False):
+def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None, concat_down=False, layout_dense=0):
     H, dc, dr, dn, dv, d, ql = (DIMS[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d", "q_lora"))
     dkv, dq = dc + dr, dn + dr
     t = dict(dw)
@@ -246,9 +246,9 @@ def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None, conc
     for k, n in outs.items():
         t[k] = torch.zeros(n, dtype=torch.int16, device="cuda")
     t["o_lat_f32"] = torch.zeros(H * dc, dtype=torch.float32, device="cuda")
-    p = nm.mla_params(DIMS, S, t)
+    p = nm.mla_params(DIMS, S, t, layout_dense=layout_dense)
     ws = nm.new_workspace(nm.nm_mla_workspace_bytes(p))
-    p = nm.mla_params(DIMS, S, t, workspace=ws)
+    p = nm.mla_params(DIMS, S, t, workspace=ws, layout_dense=layout_dense)
     main = torch.cuda.Stream()
     side = torch.cuda.Stream() if overlap else None
     torch.cuda.synchronize()
@@ -300,6 +300,34 @@ def test_decode_step_with_concatenated_down_projections(nm, weights, S):
     cache_in = gen.mla_cache(S, DIMS, seed=4500 + S)
     t = run_step(nm, dw, h, cache_in, S, concat_down=True)
     check_step(t, r, cache_ref, S)
+
+
+@pytest.mark.parametrize("concat_down", [True, False])
+def test_decode_step_with_the_dense_weights_in_fractal_storage(nm, weights, concat_down):
+    """The storage of the paper's test case: W_DQ, W_DKV|W_KR (or the three as one matrix), W_UQR and W_O in 16 x 16
+    fractals ordered by columns.  Same logical matrices as the row-major fixture, so the same oracle reference."""
+    w, dw = weights
+    S = 700
+    h, cache_ref, r = oracle_step(w, S, seed=4600)
+    cache_in = gen.mla_cache(S, DIMS, seed=4600)
+    d, ql, dkv = DIMS["d"], DIMS["q_lora"], DIMS["kv_lora"] + DIMS["rope"]
+    H, dq, dv = DIMS["H"], DIMS["nope"] + DIMS["rope"], DIMS["v"]
+    nz = dict(dw)
+    shapes = {"W_DQ": (d, ql), "W_DKVKR": (d, dkv), "W_UQR": (ql, H * dq), "W_O": (H * dv, d)}
+    for name, (K, N) in shapes.items():
+        nz[name] = to_dev(gen.to_fractal_nz(np.asarray(w[name]).reshape(K, N)))
+    if concat_down:      # run_step concatenates the (row-major) fixtures; store that concatenation in fractals instead
+        cat = np.concatenate([np.asarray(w["W_DQ"]).reshape(d, ql), np.asarray(w["W_DKVKR"]).reshape(d, dkv)], axis=1)
+        nz["W_DQKV"] = to_dev(gen.to_fractal_nz(cat))
+        nz.pop("W_DQ"); nz.pop("W_DKVKR")
+    t = run_step(nm, nz, h, cache_in, S, layout_dense=2)
+    check_step(t, r, cache_ref, S)
+    # the oracle on the fractal storage itself gives the same reference (its index formula, pinned on its own)
+    wnz = dict(w)
+    for name, (K, N) in shapes.items():
+        wnz[name] = gen.to_fractal_nz(np.asarray(w[name]).reshape(K, N))
+    r2 = oracle.mla_decode_step(DIMS, wnz, h, gen.mla_cache(S, DIMS, seed=4600), S, layout_dense=2, threads=8)
+    assert np.array_equal(np.asarray(r2["out"]), np.asarray(r["out"]))
 
 
 @pytest.mark.parametrize("S", [1, 2, 65, 4096])

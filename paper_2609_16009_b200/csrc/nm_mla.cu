@@ -313,6 +313,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 // ---- host -------------------------------------------------------------------------------------------
 
 static int g_step_plan[3][3] = {};   // tuning: forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
+static int g_host_direct_out = 1;    // host-operand step: store the result straight into device-addressable host memory
 static int g_batch_tc_min_t = 4;     // batch decode: tokens from which the per-head products go to the tensor cores
 static int g_fused_tails = 1;        // 0: RMSNorm / RoPE / cache write as kernels of their own; 1: folded into the products (default);
                                      // 2: as 1, but only in the form where the product's last CTA runs them
@@ -897,11 +898,24 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     nm_mla_params q = *p;
     q.h = h_staging;
     q.out = out_staging;
+    // Pinned (or registered) host memory that the device can address: the W_O product stores its 14 KB result straight
+    // into it - still a device-to-host transfer, but without a copy operation (and its scheduling gap) after the
+    // last kernel.  The token row keeps its copy: 132 CTAs reading it over the host link would cost more.
+    void *out_direct = nullptr;
+    if (g_host_direct_out) {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, out_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
+            ((uintptr_t)attr.devicePointer & 15u) == 0)
+            out_direct = attr.devicePointer;
+        else
+            (void)cudaGetLastError();
+    }
+    if (out_direct) q.out = out_direct;
     NM_TRY(check_params(&q));
     cudaStream_t ms = (cudaStream_t)main_stream;
     NM_CUDA_TRY(cudaMemcpyAsync(h_staging, h_host, (size_t)p->d * 2, cudaMemcpyHostToDevice, ms));
     NM_TRY(step_impl(&q, ms, (cudaStream_t)side_stream));
-    NM_CUDA_TRY(cudaMemcpyAsync(out_host, out_staging, (size_t)p->d * 2, cudaMemcpyDeviceToHost, ms));
+    if (!out_direct) NM_CUDA_TRY(cudaMemcpyAsync(out_host, out_staging, (size_t)p->d * 2, cudaMemcpyDeviceToHost, ms));
     return NM_OK;
 }
 

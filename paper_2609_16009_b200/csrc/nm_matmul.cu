@@ -350,7 +350,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     // tensor maps: 16-byte aligned operands and strides, bf16.  Row-major B may take the TMA ring kernel or the
     // tensor-core kernel; column-major B only the latter (its CUDA-core path is the plain column kernel).
     bool tma_ok = b_ok && a_ok && dtype != NM_F32 && tensor_map_encoder() != nullptr && (long)N * 2 < (1L << 40) && strideB >= 0;
-    if (g_force_kind == kRowVec) tma_ok = false;
+    if (g_force_kind == kRowVec && layout != NM_FRACTAL_NZ) tma_ok = false;      // the fractal storage has one kernel: nothing to force
     if (layout == NM_FRACTAL_NZ && !tma_ok) return NM_ERR_UNSUPPORTED;      // unaligned operands or no tensor-map encoder
     Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok, chained);
     // Copies, not pointers into the map cache: the second lookup may evict the entry the first one returned

@@ -1,0 +1,73 @@
+"""Randomised parity of the single-token decode step against the oracle: sequence length, weight storage, schedule,
+where the vector stages run, fused or separate per-head stages, attention kernel and programmatic launch are drawn
+from a seeded generator; every case is checked stage by stage like the fixed cases of test_mla_gpu.py."""
+import numpy as np
+import pytest
+import torch
+
+import nm_inputs as gen
+import oracle
+import test_mla_gpu as base
+from gpu_util import to_dev
+
+pytestmark = pytest.mark.gpu
+
+DIMS = gen.DSV3_DIMS
+ROW, COL, NZ = 0, 1, 2
+
+
+@pytest.fixture(scope="module")
+def nm():
+    import paper_2609_16009_b200 as nm
+    yield nm
+    nm.nm_debug_set_attention(0)
+    nm.nm_debug_set_step_tails(1)
+    nm.nm_debug_set_step_fusion(True)
+    nm.nm_debug_set_step_pdl(True)
+    nm.nm_check_status()
+
+
+@pytest.fixture(scope="module")
+def weights():
+    w = gen.mla_weights(DIMS, seed=4000, with_wo=True)
+    return w
+
+
+def stored(w, layout, concat):
+    """Device copies of the weights with the dense ones in the given storage (per-head weights stay row-major)."""
+    d, ql, dkv = DIMS["d"], DIMS["q_lora"], DIMS["kv_lora"] + DIMS["rope"]
+    H, dq, dv = DIMS["H"], DIMS["nope"] + DIMS["rope"], DIMS["v"]
+    shapes = {"W_DQ": (d, ql), "W_DKVKR": (d, dkv), "W_UQR": (ql, H * dq), "W_O": (H * dv, d)}
+    conv = {ROW: lambda X: X, COL: gen.to_col_major, NZ: gen.to_fractal_nz}[layout]
+    out = {}
+    for k, v in w.items():
+        out[k] = to_dev(conv(np.asarray(v).reshape(shapes[k])) if k in shapes else v)
+    if concat:
+        cat = np.concatenate([np.asarray(w["W_DQ"]).reshape(d, ql), np.asarray(w["W_DKVKR"]).reshape(d, dkv)], axis=1)
+        out["W_DQKV"] = to_dev(conv(cat))
+        out.pop("W_DQ"); out.pop("W_DKVKR")
+    return out
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_step_matches_the_oracle(nm, weights, seed):
+    rng = np.random.default_rng(50_000 + seed)
+    S = int(rng.choice([1, 2, 3, 31, 64, 65, 127, 128, 129, int(rng.integers(130, 3000)), int(rng.integers(130, 3000))]))
+    layout = int(rng.choice([ROW, ROW, COL, NZ]))
+    concat = bool(rng.random() < 0.5) and layout != COL            # the concatenated down-projection is row-major or fractal
+    overlap = bool(rng.random() < 0.5)
+    tails, fusion, pdl = int(rng.integers(0, 3)), bool(rng.random() < 0.8), bool(rng.random() < 0.8)
+    attn = int(rng.choice([0, 0, 1, 2, 3]))
+    what = f"seed {seed}: S {S} layout {layout} concat {concat} overlap {overlap} tails {tails} fusion {fusion} pdl {pdl} attention {attn}"
+    h, cache_ref, r = base.oracle_step(weights, S, seed=60_000 + seed)
+    cache_in = gen.mla_cache(S, DIMS, seed=60_000 + seed)
+    dw = stored(weights, layout, concat)
+    nm.nm_debug_set_step_tails(tails); nm.nm_debug_set_step_fusion(fusion); nm.nm_debug_set_step_pdl(pdl); nm.nm_debug_set_attention(attn)
+    try:
+        t = base.run_step(nm, dw, h, cache_in, S, overlap=overlap, layout_dense=layout)
+    finally:
+        nm.nm_debug_set_step_tails(1); nm.nm_debug_set_step_fusion(True); nm.nm_debug_set_step_pdl(True); nm.nm_debug_set_attention(0)
+    try:
+        base.check_step(t, r, cache_ref, S)
+    except AssertionError as e:
+        raise AssertionError(f"{what}: {e}") from e

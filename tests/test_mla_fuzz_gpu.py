@@ -71,3 +71,15 @@ def test_random_step_matches_the_oracle(nm, weights, seed):
         base.check_step(t, r, cache_ref, S)
     except AssertionError as e:
         raise AssertionError(f"{what}: {e}") from e
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_attention_stage_matches_the_oracle(nm, seed):
+    """The attention pass alone on its own random operands (not the output of earlier GPU stages): every kernel,
+    lengths from one row to a few thousand, the new row through the merge or through the pass."""
+    rng = np.random.default_rng(90_000 + seed)
+    S = int(rng.choice([1, 2, 33, 64, 65, 128, 129, int(rng.integers(130, 6000)), int(rng.integers(130, 6000))]))
+    impl = int(rng.choice([0, 1, 2, 3]))
+    extra = bool(rng.random() < 0.5) or S == 1
+    err = base.attention_case(nm, S, impl, extra, seed=91_000 + 10 * seed)
+    assert err <= 2e-3, f"seed {seed}: S {S} impl {impl} extra {extra}: {err:.2e}"

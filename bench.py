@@ -427,7 +427,7 @@ def read_only_stream(nm, device):
     return best
 
 
-def matmul_sweep(nm, device):
+def matmul_sweep(nm, device, args_no_cpu=False):
     """GB/s of single narrow products (cold L2: the launches of a CUDA graph rotate through copies of
     B that together exceed 512 MB).  Two figures per case: launches in plain stream order (each kernel
     starts when the one before has finished: latency of an isolated call plus the launch gap), and
@@ -514,6 +514,26 @@ def matmul_sweep(nm, device):
                     nm.nm_matmul_ws(A, Bs[0], C[0], M, N, K, code, layout, ws, s)
                 b.record(s); s.synchronize()
                 row["us_warm_l2"] = round(a.elapsed_time(b) * 1e3 / 100, 2)
+        # the oracle's time for the same product on the host cores (all it may use, and one thread), best of three
+        # after a warm-up pass; for M > 1 on the large matrices a bounded sample: the first row only
+        if not args_no_cpu:
+            import oracle
+            threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+            Mo = M if (M * K * N <= 3e8) else 1
+            An = (np.random.default_rng(1).standard_normal((Mo, K)).astype(np.float32))
+            Bn = (np.random.default_rng(2).standard_normal(K * N).astype(np.float32) * 0.02)
+            if dt == "bf16":
+                An = (An.view(np.uint32) >> 16).astype(np.uint16); Bn = (Bn.view(np.uint32) >> 16).astype(np.uint16)
+            odt = oracle.F32 if dt == "f32" else oracle.BF16
+            def run(th):
+                best = 1e9
+                for rep in range(4):
+                    t0 = time.perf_counter()
+                    oracle.matmul(An, Bn, Mo, N, K, odt, odt, layout, threads=th)
+                    if rep: best = min(best, time.perf_counter() - t0)
+                return best * 1e3
+            row["oracle_ms"] = {"rows": Mo, "cores": threads, "all_cores": round(run(threads), 2),
+                                "one_thread": round(run(1), 2) if Mo * K * N <= 5e7 else None}
         out.append(row)
         del Bs, C
     return out
@@ -774,7 +794,7 @@ def main():
                              "us_per_launch": dom_ms * 1e3}}
         line.update(extras)
         if args.sweep:
-            line["narrow_matmul_vs_M"] = matmul_sweep(nm, device)
+            line["narrow_matmul_vs_M"] = matmul_sweep(nm, device, args.no_cpu_baseline)
             line["read_only_stream"] = read_only_stream(nm, device)
         if not args.no_cpu_baseline:
             import oracle

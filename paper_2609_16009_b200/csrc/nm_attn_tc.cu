@@ -588,10 +588,10 @@ int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, At
 
 int attention_partial_tc_batch(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split,
                                int nsplit, AttnPartials part, int slot_stride, float scale, cudaStream_t stream,
-                               bool programmatic_launch)
+                               bool programmatic_launch, L2Prefetch prefetch)
 {
     return launch_attn_tc(Q, nseq, caches, n_rows, rows_per_split, nsplit, part, (long)slot_stride * kHeads * 2,
-                          (long)slot_stride * kHeads * kDv, scale, stream, programmatic_launch, L2Prefetch{});
+                          (long)slot_stride * kHeads * kDv, scale, stream, programmatic_launch, prefetch);
 }
 
 }  // namespace nm

@@ -461,7 +461,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
 
 void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit, bool chained)
 {
-    const Plan p = make_tma_plan(M, N, K, H, chained);
+    const Plan p = make_plan(M, N, K, H, NM_BF16, NM_ROW_MAJOR, true, true, chained);      // whichever kernel the product will take
     *k_rows_per_split = p.kr;
     *nsplit = p.nsplit;
 }

@@ -786,10 +786,26 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     part.O = reinterpret_cast<float *>(ws + L.attn_o);
     if (any_rows) {
         if (tensor_map_encoder() == nullptr) return NM_ERR_UNSUPPORTED;
+        // beside the attention pass (a spare warp of its CTAs): W_UV and the head of every k-split of W_O into L2, as in
+        // the single-token step
+        L2Prefetch pf{};
+        if (g_prefetch_mb > 0) {
+            pf.block = (const char *)p->W_UV;
+            pf.block_bytes = g_prefetch_uv ? (long)H * dc * dv * 2 : 0;
+            if (p->W_O && lay == NM_ROW_MAJOR) {
+                int kr = 0, ns = 1;
+                matmul_row_major_split(T, d, H * dv, 1, &kr, &ns, true);
+                const long row_bytes = (long)d * 2;
+                long prows = ((long)g_prefetch_mb << 20) / ns / row_bytes;
+                if (prows > kr) prows = kr;
+                pf.base = (const char *)p->W_O; pf.range_stride = (long)kr * row_bytes; pf.nranges = prows > 0 ? ns : 0;
+                pf.range_bytes = prows * row_bytes;
+            }
+        }
         if (tc64)
-            NM_TRY(attention_partial_tc64(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl, L2Prefetch{}));
+            NM_TRY(attention_partial_tc64(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl, pf));
         else
-            NM_TRY(attention_partial_tc_batch(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl));
+            NM_TRY(attention_partial_tc_batch(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl, pf));
     }
     if (per_head_tc) {
         NM_TRY(launch_attn_merge_batch(q_full, cache, part, rows, T, dr, p->softmax_scale, o_lat, H, ms, pdl));

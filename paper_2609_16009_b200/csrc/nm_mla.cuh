@@ -48,7 +48,7 @@ int attention_partial_tc(const void *Q, const void *cache, AttnPartials part, At
 constexpr int kMaxBatch = 16;
 int attention_partial_tc_batch(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split,
                                int nsplit, AttnPartials part, int slot_stride, float scale, cudaStream_t stream,
-                               bool programmatic_launch);
+                               bool programmatic_launch, L2Prefetch prefetch = L2Prefetch{});
 
 // Fused per-head stages of the decode step (nm_head_kernels.cu); they take nope = 128, kv_lora = 512, v = 128.
 bool head_kernels_apply(int H, int nope, int rope, int dc, int dv);

@@ -894,11 +894,29 @@ size_t nm_mla_workspace_bytes(const nm_mla_params *p)
 size_t nm_mla_batch_workspace_bytes(const nm_mla_params *p, int T)
 {
     if (!p || T < 1 || T > kMaxBatch) return 0;
-    return batch_layout(p, T).total;
+    const size_t batch = batch_layout(p, T).total;
+    if (T == 1) {                                                  // a batch of one runs the single-token step
+        const size_t single = step_layout(p).total;
+        return single > batch ? single : batch;
+    }
+    return batch;
 }
 
 int nm_mla_decode_batch(const nm_mla_params *p, const nm_mla_batch *b, nm_stream main_stream)
 {
+    // One sequence: the single-token step (its completion stages, prefetch and chaining are tuned for exactly that);
+    // the batch fields map onto its parameters one to one.
+    if (p && b && b->T == 1 && b->seq_lens && b->seq_lens[0] >= 1 && b->h && b->rope_cos_sin && b->kv_cache && p->workspace &&
+        p->workspace_bytes >= step_layout(p).total) {
+        nm_mla_params q = *p;
+        q.seq_len = b->seq_lens[0];
+        q.h = b->h; q.rope_cos_sin = b->rope_cos_sin; q.kv_cache = b->kv_cache; q.out = b->out;
+        q.q_full = b->q_full; q.o_lat = b->o_lat; q.o = b->o;
+        q.c_q = nullptr; q.c_qn = nullptr; q.q = nullptr; q.ckr = nullptr; q.o_lat_f32 = nullptr;
+        q.event_before_wo = nullptr; q.event_after_wo = nullptr; q.programmatic_entry = 0;
+        if (!q.W_O) q.out = nullptr;
+        return step_impl(&q, (cudaStream_t)main_stream, (cudaStream_t)main_stream);
+    }
     return batch_impl(p, b, (cudaStream_t)main_stream);
 }
 

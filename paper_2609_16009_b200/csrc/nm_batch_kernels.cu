@@ -296,14 +296,14 @@ __global__ void __launch_bounds__(kThreadsB) uv_merge_batch_kernel(const uint16_
 // ---- the same two stages without the per-head products, for batches large enough that those products belong on
 //      the tensor cores (the batched swap-AB kernel): RoPE of every token's query heads, and the merge alone ------
 
-// grid (T): q_full[t, h, dc:] = RoPE(q[t, h, nope:]) for every head.
+// grid (T, parts): q_full[t, h, dc:] = RoPE(q[t, h, nope:]) for every head; the heads of a token are dealt to `parts` CTAs.
 __global__ void __launch_bounds__(kThreadsB) rope_batch_kernel(const uint16_t *__restrict__ q, const float *__restrict__ cs,
                                                                uint16_t *__restrict__ q_full, int H, int nope, int dc, int rope)
 {
     const int t = blockIdx.x, half = rope / 2;
     pdl_launch_dependents();
     pdl_wait_prior_grids();                                       // q comes from the W_UQR product
-    for (int i = threadIdx.x; i < H * half; i += kThreadsB) {
+    for (int i = blockIdx.y * kThreadsB + threadIdx.x; i < H * half; i += kThreadsB * gridDim.y) {
         const int h = i / half, pr = i - h * half;
         const uint32_t xv = *reinterpret_cast<const uint32_t *>(q + ((size_t)t * H + h) * (nope + rope) + nope + 2 * pr);
         const float2 c = *reinterpret_cast<const float2 *>(cs + (size_t)t * rope + 2 * pr);
@@ -417,7 +417,8 @@ int launch_uv_merge_batch(const void *Q, const void *cache, AttnPartials part, c
 
 int launch_rope_batch(const void *q, const float *cos_sin, void *q_full, int H, int nope, int dc, int rope, int T, cudaStream_t s, bool pdl)
 {
-    cudaError_t e = launch_b(rope_batch_kernel, dim3(T), s, pdl, (const uint16_t *)q, cos_sin, (uint16_t *)q_full, H, nope, dc, rope);
+    const int parts = (H * (rope / 2) + kThreadsB - 1) / kThreadsB;      // one pair per thread
+    cudaError_t e = launch_b(rope_batch_kernel, dim3(T, parts < 1 ? 1 : parts), s, pdl, (const uint16_t *)q, cos_sin, (uint16_t *)q_full, H, nope, dc, rope);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "rope (batch) launch");
 }
 

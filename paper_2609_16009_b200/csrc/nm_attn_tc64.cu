@@ -368,17 +368,18 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(slot), "f"((ntiles > 0) ? m_own : -INFINITY), "f"(l_own) : "memory");
         }
         if (ntiles > 0) {
-            for (int c = 0; c < kDvHalf / 32; ++c) {
+            // both halves of the warp park: thread l has columns 0-31 of a 64-column chunk of row l % 16, thread l + 16
+            // columns 32-63 (the half-split load shape, as in the softmax)
+            const uint32_t prow = (uint32_t)(quad * 16 + (lane & 15)), pch = (uint32_t)(lane >> 4);
+            for (int c = 0; c < kDvHalf / 64; ++c) {
                 uint32_t o[32];
-                tmem_ld32(lane_base + kColO + c * 32, o);          // whole warp; lanes 16-31 read rows nobody wrote
+                tmem_ld32_halves<32>(lane_base + kColO + c * 64, o);
                 tmem_wait_ld();
-                if (lane < 16) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const uint32_t q4 = (uint32_t)(c * 8 + i / 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(q_addr + (uint32_t)(head * 64 + (q4 ^ (head & 7u))) * 16u),
-                                     "r"(o[i]), "r"(o[i + 1]), "r"(o[i + 2]), "r"(o[i + 3]) : "memory");
-                    }
+                for (int i = 0; i < 32; i += 4) {
+                    const uint32_t q4 = (uint32_t)(c * 16) + pch * 8 + (uint32_t)(i / 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(q_addr + (prow * 64 + (q4 ^ (prow & 7u))) * 16u),
+                                 "r"(o[i]), "r"(o[i + 1]), "r"(o[i + 2]), "r"(o[i + 3]) : "memory");
                 }
             }
         }

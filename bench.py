@@ -742,17 +742,18 @@ def main():
         dom = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
         for a, b in dom:                      # events get their handles on first record
             a.record(stream); b.record(stream)
+        dom_stride = 16 if args.steps >= 128 else max(1, args.steps // 8)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record(stream)
-        # the dominant kernel is bracketed by events on every 8th step only: the events break the
+        # the dominant kernel is bracketed by events on every 16th step only (at least 8 samples): the events break the
         # programmatic launch of that kernel, and the step time should not carry that on every step
         for i in range(args.steps):
-            wl.step(stream, dom[i] if i % 8 == 0 else None)
+            wl.step(stream, dom[i] if i % dom_stride == 0 else None)
         e1.record(stream)
         barrier()
         ms = e0.elapsed_time(e1)
-        dom_ms = statistics.mean(a.elapsed_time(b) for a, b in dom[::8])
+        dom_ms = statistics.mean(a.elapsed_time(b) for a, b in dom[::dom_stride])
         # ---- end-to-end region: host token in, host result out, every step -----------------------------
         for _ in range(3):
             wl.step_e2e(stream)

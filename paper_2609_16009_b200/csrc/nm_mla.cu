@@ -314,7 +314,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 
 static int g_step_plan[3][3] = {};   // tuning: forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
 static int g_host_direct_out = 1;    // host-operand step: store the result straight into device-addressable host memory
-static int g_batch_tc_min_t = 4;     // batch decode: tokens from which the per-head products go to the tensor cores
+static int g_batch_tc_min_t = 3;     // batch decode: tokens from which the per-head products go to the tensor cores
 static int g_fused_tails = 1;        // 0: RMSNorm / RoPE / cache write as kernels of their own; 1: folded into the products (default);
                                      // 2: as 1, but only in the form where the product's last CTA runs them
 static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
@@ -769,10 +769,10 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     NM_TRY(launch_down_finish_batch(x_down, p->gamma_q, p->gamma_kv, b->rope_cos_sin, c_qn, cache, rows, T, ql, dc, dr, p->rms_eps, ms, pdl));
     NM_TRY(matmul_enqueue(c_qn, p->W_UQR, q, T, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.mws_bytes, ms, pdl, nullptr, nullptr,
                           nullptr, true));
-    // From four tokens on the per-head products (128 x 512 and 512 x 128 per head and token) go to the batched swap-AB
+    // From three tokens on the per-head products (128 x 512 and 512 x 128 per head and token) go to the batched swap-AB
     // tensor-core kernel, with RoPE and the merge as small kernels of their own: in the fused per-head kernels one
     // CTA per head walks every token and is bound by fp32 FMA issue and by its chain of L2 round trips (measured at
-    // 4096 rows: 114 vs 115 us at T = 4, 133 vs 139 at T = 6, 183 vs 204 at T = 16; 105 vs 102 at T = 2).
+    // 4096 rows: 108 vs 112 us at T = 3, 114 vs 115 at T = 4, 133 vs 139 at T = 6, 183 vs 204 at T = 16; level at T = 2).
     const bool per_head_tc = T >= g_batch_tc_min_t || !g_fused_heads;
     if (per_head_tc) {
         NM_TRY(launch_rope_batch(q, b->rope_cos_sin, q_full, H, dn, dc, dr, T, ms, pdl));

@@ -110,7 +110,7 @@ def test_batch_matches_oracle(nm, weights, seq_lens, concat):
 @pytest.mark.parametrize("seq_lens,with_wo", [([300], True), ([90, 1, 257], True), ([1024, 65, 2, 500, 130], True),
                                               ([64 + 31 * i for i in range(12)], False)])
 def test_batch_with_the_per_head_products_as_batched_products(nm, weights, seq_lens, with_wo):
-    """From four sequences on the per-head products run as batched products (tensor cores from M = 3) with RoPE and
+    """From three sequences on the per-head products run as batched products (tensor cores from M = 3) with RoPE and
     the merge as kernels of their own; below, fused per-head kernels do them.  Here the first form at every batch
     size (the switch that turns the fused per-head kernels off), against the oracle."""
     w, dw = weights

@@ -343,6 +343,9 @@ int nm_debug_set_step_knobs(int uv_programmatic, int prefetch_w_uv);
  * meet inside clusters, W_UQR normalises its token row while loading it and the KV consumers ride in an extra CTA of
  * the per-head query kernel; otherwise, and with 2 always, the CTA that completes the product's last tile runs them. */
 int nm_debug_set_step_tails(int enable);
+/* Batch decode: sequences from which the per-head products (W_UK, W_UV) run as batched products of the library with
+ * RoPE and the merge as kernels of their own (default 3); below, fused per-head kernels do them.  17 = always fused. */
+int nm_debug_set_batch_per_head_min_tokens(int tokens);
 /* Decode step tuning: force (tile_n, nsplit, ring stages) of one of its products - which = 0 the down-projection,
  * 1 W_UQR, 2 W_O; zeros give the plan back to the planner. */
 int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages);

@@ -104,6 +104,7 @@ _lib.nm_debug_stream_read.argtypes = [_vp, _sz, _vp, _i, _vp]
 _lib.nm_debug_set_step_knobs.argtypes = [_i, _i]
 _lib.nm_debug_set_step_tails.argtypes = [_i]
 _lib.nm_debug_set_cluster_split.argtypes = [_i]
+_lib.nm_debug_set_batch_per_head_min_tokens.argtypes = [_i]
 _lib.nm_debug_set_step_plan.argtypes = [_i, _i, _i, _i]
 _lib.nm_debug_set_step_prefetch.argtypes = [_i]
 _lib.nm_debug_set_step_fusion.argtypes = [_i]
@@ -343,6 +344,10 @@ def nm_debug_set_step_prefetch(megabytes: int) -> None:
 
 def nm_debug_set_step_knobs(uv_programmatic: int = 1, prefetch_w_uv: int = 1) -> None:
     _check(_lib.nm_debug_set_step_knobs(int(uv_programmatic), int(prefetch_w_uv)), "nm_debug_set_step_knobs")
+
+
+def nm_debug_set_batch_per_head_min_tokens(tokens: int) -> None:
+    _check(_lib.nm_debug_set_batch_per_head_min_tokens(int(tokens)), "nm_debug_set_batch_per_head_min_tokens")
 
 
 def nm_debug_set_cluster_split(enable: bool) -> None:

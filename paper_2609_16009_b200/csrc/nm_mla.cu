@@ -953,6 +953,13 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     return NM_OK;
 }
 
+int nm_debug_set_batch_per_head_min_tokens(int tokens)
+{
+    if (tokens < 1 || tokens > kMaxBatch + 1) return NM_ERR_INVALID_ARG;
+    g_batch_tc_min_t = tokens;
+    return NM_OK;
+}
+
 int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages)
 {
     if (which < 0 || which > 2) return NM_ERR_INVALID_ARG;

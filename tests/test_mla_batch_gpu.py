@@ -123,6 +123,20 @@ def test_batch_with_the_per_head_products_as_batched_products(nm, weights, seq_l
     check_against_oracle(w, res, tokens, caches, seq_lens, with_wo=with_wo)
 
 
+@pytest.mark.parametrize("seq_lens,with_wo", [([513, 64, 2], True), ([300, 1, 70, 1024, 65], True), ([40 + 53 * i for i in range(16)], False)])
+def test_batch_with_the_fused_per_head_kernels_at_every_size(nm, weights, seq_lens, with_wo):
+    """The fused per-head kernels (one CTA per head walking every token) stay selectable beyond the two sequences they
+    serve by default."""
+    w, dw = weights
+    tokens, caches = make_inputs(seq_lens, seed=8400 + len(seq_lens))
+    nm.nm_debug_set_batch_per_head_min_tokens(17)
+    try:
+        res = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True, with_wo=with_wo)
+    finally:
+        nm.nm_debug_set_batch_per_head_min_tokens(3)
+    check_against_oracle(w, res, tokens, caches, seq_lens, with_wo=with_wo)
+
+
 def test_batch_of_sixteen_without_wo(nm, weights):
     w, dw = weights
     seq_lens = [40 + 37 * i for i in range(16)]

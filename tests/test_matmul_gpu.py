@@ -115,6 +115,27 @@ def test_column_major_tensor_core_kernel_forced_on_small_and_ragged_shapes(nm, M
         nm.nm_debug_set_plan(0, 0)
 
 
+@pytest.mark.parametrize("rows,K", [(576, 7168), (1536, 7168), (1000, 1001), (7, 40)])
+@pytest.mark.parametrize("dtype", [F32, BF16, BF16_F32OUT])
+def test_matrix_times_column_vector_by_transposition(nm, rows, K, dtype):
+    """The other narrow case of the Narrow Dimension condition, N = 1: C[rows x 1] = W[rows x K] * x[K x 1].  The oracle
+    computes exactly that (its M is not limited); the library is given the transposed problem C^T = x^T * W^T, in
+    which the row-major W is a column-major B - no copy, no transposition pass."""
+    if dtype == F32:
+        W, x = gen.uniform_f32((rows, K), -1, 1, 2500 + rows), gen.uniform_f32((K, 1), -1, 1, 2501 + rows)
+    else:
+        x, Wt = gen.narrow_bf16(1, K, rows, seed=2500 + rows)       # x: [1][K] ~ N(0,1); Wt: [K][rows] ~ N(0, 0.02^2)
+        W = np.ascontiguousarray(np.asarray(Wt).reshape(K, rows).T)
+        x = np.asarray(x).reshape(K, 1)
+    Cq, C64, bound = oracle.matmul(W, x, rows, 1, K, ORACLE_IN[dtype], ORACLE_OUT[dtype], ROW, threads=8)
+    dW, dx = to_dev(W), to_dev(x)
+    whole, dC = out_buffer(rows, dtype)
+    nm.nm_matmul(dx, dW, dC, 1, rows, K, dtype, COL)             # A = x^T [1 x K], B = W read as [K x rows] column-major
+    torch.cuda.synchronize()
+    assert guards_intact(whole, rows, dtype)
+    assert_matmul_close(out_to_f64(dC, dtype).reshape(rows, 1), Cq, C64, bound, dtype, f"column vector rows={rows} K={K}")
+
+
 # ---- every M, ragged shapes, both layouts, all dtypes ------------------------------------------------------
 
 @pytest.mark.parametrize("M", list(range(1, 17)))

@@ -48,8 +48,8 @@ constexpr int kSAcc = 2;
 // P_lo (bf16 pairs, 32 columns each) over the first accumulator of the same stage
 constexpr uint32_t kColO = 0, kColS = 256;
 constexpr float kLazyThreshold = 8.0f;    // log2 units
-constexpr int kCl = kAttnCluster;
-constexpr int kHeadsPerRank = kHeadsCta / kCl;       // 16: the heads of one softmax warp
+// The splits merged on chip form a cluster of kCl CTAs (template argument: 4, 2 or 1); rank r owns kHeadsCta / kCl heads
+// in the merge (with four ranks: the 16 heads of softmax warp r).
 
 struct AttnSeqs64 {
     CUtensorMap kv[kMaxBatch];
@@ -95,10 +95,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return r;
 }
 
+template <int kCl>
 __global__ void __maxnreg__(120)
 attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ AttnSeqs64 seqs, AttnPartials part,
                  float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
 {
+    constexpr int kHeadsPerRank = kHeadsCta / kCl;
     const int seq = blockIdx.z;
     const CUtensorMap *map_kv_p = &seqs.kv[seq];
     const int n_rows = seqs.n_rows[seq], rows_per_split = seqs.rows_per_split[seq];
@@ -363,8 +365,9 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (warp >= 2 && warp < 6) {
         const int quad = warp & 3, head = quad * 16 + lane;        // head within this CTA's 64 (lanes 0-15)
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
-        if (lane < 16) {
-            const uint32_t slot = peer_smem(smem_u32(&s_mlp[rank][lane][0]), (uint32_t)quad);
+        if (lane < 16) {                                           // (m, l) to the rank that owns the head
+            const int hd = quad * 16 + lane;
+            const uint32_t slot = peer_smem(smem_u32(&s_mlp[rank][hd % kHeadsPerRank][0]), (uint32_t)(hd / kHeadsPerRank));
             asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(slot), "f"((ntiles > 0) ? m_own : -INFINITY), "f"(l_own) : "memory");
         }
         if (ntiles > 0) {
@@ -470,11 +473,67 @@ bool encode_rows_map64(CUtensorMap *map, const void *ptr, int rows, int box_rows
 
 }  // namespace
 
+namespace {
+template <int kCl>
+int configure_tc64()
+{
+    static bool configured = false;                                // one flag per instantiation
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tc64_kernel<kCl>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return record_cuda_error(e, "attention kernel attribute");
+        configured = true;
+    }
+    return NM_OK;
+}
+// Clusters of kCl CTAs of this kernel that the device holds at once (clusters do not straddle GPCs, so this is
+// fewer than SMs / kCl); 0 if the query fails.
+template <int kCl>
+int max_clusters_tc64()
+{
+    if (configure_tc64<kCl>() != NM_OK) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kCl, 4, 1); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kCl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return max_clusters_cached(attn_tc64_kernel<kCl>, cfg, kCl);
+}
+template <int kCl>
+int launch_tc64(const CUtensorMap &map_q, const AttnSeqs64 &seqs, int nseq, int nsplit, AttnPartials part, float scale, cudaStream_t stream,
+                bool programmatic_launch, const L2Prefetch &prefetch)
+{
+    if (int rc = configure_tc64<kCl>()) return rc;
+    const float scale_log2 = scale * 1.4426950408889634f;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ceil_div(nsplit, kCl) * kCl, 4, nseq);      // y: column half + 2 * head half; padding CTAs have no rows
+    const bool has_prefetch = prefetch.block_bytes > 0 || (prefetch.nranges > 0 && prefetch.range_bytes > 0);
+    cfg.blockDim = dim3(has_prefetch ? kThreads : kThreads - 32);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kCl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = programmatic_launch ? 2 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc64_kernel<kCl>, map_q, seqs, part, scale_log2, device_status_ptr(), attention_trace(), prefetch);
+    return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (tensor cores, 64 heads per CTA) launch");
+}
+}  // namespace
+
+int attention_tc64_max_clusters(int cluster)
+{
+    return cluster == 4 ? max_clusters_tc64<4>() : (cluster == 2 ? max_clusters_tc64<2>() : (cluster == 1 ? max_clusters_tc64<1>() : 0));
+}
+
 int attention_partial_tc64(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split, int nsplit,
-                           AttnPartials part, int slot_stride, float scale, cudaStream_t stream, bool programmatic_launch,
+                           int cluster, AttnPartials part, int slot_stride, float scale, cudaStream_t stream, bool programmatic_launch,
                            L2Prefetch prefetch)
 {
     if (nseq < 1 || nseq > kMaxBatch || nsplit < 1) return NM_ERR_UNSUPPORTED;
+    if (cluster != 1 && cluster != 2 && cluster != 4) return NM_ERR_UNSUPPORTED;
     if ((uintptr_t)Q & 15u) return NM_ERR_UNSUPPORTED;
     CUtensorMap map_q;
     AttnSeqs64 seqs{};
@@ -494,28 +553,9 @@ int attention_partial_tc64(const void *Q, int nseq, const void *const *caches, c
         // the cache map covers exactly the rows attended: rows past n_rows read as zeros (and are masked)
         if (!encode_rows_map64(&seqs.kv[t], caches[t], n_rows[t], kT)) return NM_ERR_UNSUPPORTED;
     }
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return record_cuda_error(e, "attention kernel attribute");
-        configured = true;
-    }
-    const float scale_log2 = scale * 1.4426950408889634f;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ceil_div(nsplit, kCl) * kCl, 4, nseq);      // y: column half + 2 * head half; padding CTAs have no rows
-    const bool has_prefetch = prefetch.block_bytes > 0 || (prefetch.nranges > 0 && prefetch.range_bytes > 0);
-    cfg.blockDim = dim3(has_prefetch ? kThreads : kThreads - 32);
-    cfg.dynamicSmemBytes = kSmemBytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kCl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = programmatic_launch ? 2 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc64_kernel, map_q, seqs, part, scale_log2, device_status_ptr(), attention_trace(), prefetch);
-    return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (tensor cores, 64 heads per CTA) launch");
+    if (cluster == 4) return launch_tc64<4>(map_q, seqs, nseq, nsplit, part, scale, stream, programmatic_launch, prefetch);
+    if (cluster == 2) return launch_tc64<2>(map_q, seqs, nseq, nsplit, part, scale, stream, programmatic_launch, prefetch);
+    return launch_tc64<1>(map_q, seqs, nseq, nsplit, part, scale, stream, programmatic_launch, prefetch);
 }
 
 }  // namespace nm

@@ -1,6 +1,7 @@
 // Single-token MLA decode step: the vector-side stages (RMSNorm, RoPE, cache-row write), the merge
 // of the attention splits, and the host orchestration that overlaps the CUDA-core narrow products
 // with the tensor-core attention pass.
+#include <algorithm>
 #include <cmath>
 
 #include "nm_async.cuh"
@@ -382,7 +383,7 @@ static int attention_partial(const void *Q, const void *cache, int H, int n_rows
     const AttnPlan p = plan_attention(Q, cache, H, n_rows, dc);
     AttnPartials part = carve_partials(ws, H);
     if (p.tensor_core == 2)
-        return attention_partial_tc64(Q, 1, &cache, &n_rows, &p.rows_per_split, p.nsplit, part, 0, scale, s, pdl, prefetch);
+        return attention_partial_tc64(Q, 1, &cache, &n_rows, &p.rows_per_split, p.nsplit, kAttnCluster, part, 0, scale, s, pdl, prefetch);
     if (p.tensor_core) return attention_partial_tc(Q, cache, part, p, n_rows, scale, s, pdl, prefetch);
     cudaError_t e = launch_pdl(attn_partial_simt_kernel, dim3(p.nsplit, H), dim3(128), s, pdl, static_cast<const uint16_t *>(Q),
                                static_cast<const uint16_t *>(cache), part, n_rows, p.rows_per_split, dc, dr, scale);
@@ -735,11 +736,26 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     // split plan of the attention pass: the same number of splits for every sequence, about 128 CTAs in all
     long total_rows = 0;
     for (int t = 0; t < T; ++t) total_rows += b->seq_lens[t];
-    // 64 heads per CTA (four CTAs per split) while the batch is short enough and its CTAs - at least four splits per
-    // sequence - fit one wave of the 148 SMs: up to nine sequences
-    const bool tc64 = attention_64_heads(total_rows) && (g_attn_impl == 3 || T * kAttnCluster * 4 <= kSMsAttn);
-    int nsplit = ((tc64 ? 32 : 64) / T) / kAttnCluster * kAttnCluster;
+    // 64 heads per CTA (four CTAs per split) while the batch is short enough.  Every sequence gets the same number of
+    // splits; all clusters are resident at once (clusters do not straddle GPCs: fewer fit than SMs / size).  Of the split counts that fit, the one with the fewest tiles per
+    // CTA on the longest sequence is taken - among equals the one divisible by four, then by two (the splits merged on
+    // chip form a cluster of 4, 2 or 1), then the smallest; at most 16 partials per sequence reach the final merge.
+    const bool tc64 = attention_64_heads(total_rows) && T * 4 <= kSMsAttn;
+    int nsplit = (64 / T) / kAttnCluster * kAttnCluster, cluster = kAttnCluster;
     if (nsplit < kAttnCluster) nsplit = kAttnCluster;
+    if (tc64) {
+        int max_rows = 1;
+        for (int t = 0; t < T; ++t) max_rows = std::max(max_rows, b->seq_lens[t] - 1);
+        const int max_tiles = ceil_div(max_rows, kAttnTileRows), fit = std::min(32, kSMsAttn / (4 * T));
+        int best = 1, best_tiles = max_tiles, best_cl = 1;
+        for (int ns = 1; ns <= fit; ++ns) {
+            const int cl = ns % 4 == 0 ? 4 : (ns % 2 == 0 ? 2 : 1), tiles = ceil_div(max_tiles, ns);
+            if (ns / cl > L.slot_stride) continue;
+            if ((long)T * 4 * (ns / cl) > attention_tc64_max_clusters(cl)) continue;     // a second wave of clusters costs more than it saves
+            if (tiles < best_tiles || (tiles == best_tiles && cl > best_cl)) { best = ns; best_tiles = tiles; best_cl = cl; }
+        }
+        nsplit = best; cluster = best_cl;
+    }
     BatchRows rows{};
     rows.slot_stride = L.slot_stride;
     const void *caches[kMaxBatch];
@@ -752,7 +768,7 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
         rows.new_row[t] = base + (long)n_rows[t] * dkv;
         const int tiles = ceil_div(n_rows[t], kAttnTileRows);
         rps[t] = tiles > 0 ? ceil_div(tiles, nsplit) * kAttnTileRows : kAttnTileRows;
-        rows.npart[t] = n_rows[t] > 0 ? ceil_div(ceil_div(n_rows[t], rps[t]), kAttnCluster) : 0;
+        rows.npart[t] = n_rows[t] > 0 ? ceil_div(ceil_div(n_rows[t], rps[t]), cluster) : 0;
         any_rows |= n_rows[t] > 0;
     }
 
@@ -803,7 +819,7 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
             }
         }
         if (tc64)
-            NM_TRY(attention_partial_tc64(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl, pf));
+            NM_TRY(attention_partial_tc64(q_full, T, caches, n_rows, rps, nsplit, cluster, part, L.slot_stride, p->softmax_scale, ms, pdl, pf));
         else
             NM_TRY(attention_partial_tc_batch(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl, pf));
     }

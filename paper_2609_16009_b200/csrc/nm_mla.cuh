@@ -75,8 +75,9 @@ int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npa
 
 // The pass with 64 heads per CTA (nm_attn_tc64.cu): four CTAs per split, 64-row cache stages.  rows_per_split must be
 // multiples of 64.  Same partial layout as the 128-head kernel.
+int attention_tc64_max_clusters(int cluster);      // clusters of that many CTAs of the kernel resident at once
 int attention_partial_tc64(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split, int nsplit,
-                           AttnPartials part, int slot_stride, float scale, cudaStream_t stream, bool programmatic_launch,
+                           int cluster /* splits merged on chip: 4, 2 or 1 */, AttnPartials part, int slot_stride, float scale, cudaStream_t stream, bool programmatic_launch,
                            L2Prefetch prefetch);
 
 // Small-batch decode (nm_batch_kernels.cu): per-sequence rows and partial counts of one launch.

@@ -108,7 +108,10 @@ def test_batch_matches_oracle(nm, weights, seq_lens, concat):
 
 
 @pytest.mark.parametrize("seq_lens,with_wo", [([300], True), ([90, 1, 257], True), ([1024, 65, 2, 500, 130], True),
-                                              ([64 + 31 * i for i in range(12)], False)])
+                                              ([64 + 31 * i for i in range(12)], False),
+                                              # split plans of the attention pass with clusters of 1, 2 and 4 merged on chip
+                                              ([650 + 17 * i for i in range(7)], False), ([900 - 13 * i for i in range(6)], False),
+                                              ([300 + 41 * i for i in range(10)], False), ([1100, 900, 1000], False)])
 def test_batch_with_the_per_head_products_as_batched_products(nm, weights, seq_lens, with_wo):
     """From three sequences on the per-head products run as batched products (tensor cores from M = 3) with RoPE and
     the merge as kernels of their own; below, fused per-head kernels do them.  Here the first form at every batch

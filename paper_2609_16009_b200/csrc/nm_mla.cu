@@ -741,7 +741,7 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     // CTA on the longest sequence is taken - among equals the one divisible by four, then by two (the splits merged on
     // chip form a cluster of 4, 2 or 1), then the smallest; at most 16 partials per sequence reach the final merge.
     const bool tc64 = attention_64_heads(total_rows) && T * 4 <= kSMsAttn;
-    int nsplit = (64 / T) / kAttnCluster * kAttnCluster, cluster = kAttnCluster;
+    int nsplit = (64 / T) / kAttnCluster * kAttnCluster, cluster = kAttnCluster, ragged_tiles = 0;
     if (nsplit < kAttnCluster) nsplit = kAttnCluster;
     if (tc64) {
         int max_rows = 1;
@@ -755,6 +755,14 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
             if (tiles < best_tiles || (tiles == best_tiles && cl > best_cl)) { best = ns; best_tiles = tiles; best_cl = cl; }
         }
         nsplit = best; cluster = best_cl;
+        // Sequences of unequal length: the same ROWS per split for every sequence instead (a short sequence then takes
+        // few CTAs, the surplus CTAs of its grid row find no rows and leave at once - which only costs nothing when no
+        // cluster peer waits for them, so without the on-chip merge).  Taken when it shortens the longest run of tiles.
+        for (int tau = std::max(1, ceil_div(max_tiles, L.slot_stride)); tau < best_tiles; ++tau) {
+            long ctas = 0;
+            for (int t = 0; t < T; ++t) ctas += 4L * ceil_div(std::max(0, b->seq_lens[t] - 1), tau * kAttnTileRows);
+            if (ctas <= kSMsAttn) { ragged_tiles = tau; nsplit = ceil_div(max_tiles, tau); cluster = 1; break; }
+        }
     }
     BatchRows rows{};
     rows.slot_stride = L.slot_stride;
@@ -767,7 +775,7 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
         n_rows[t] = b->seq_lens[t] - 1;
         rows.new_row[t] = base + (long)n_rows[t] * dkv;
         const int tiles = ceil_div(n_rows[t], kAttnTileRows);
-        rps[t] = tiles > 0 ? ceil_div(tiles, nsplit) * kAttnTileRows : kAttnTileRows;
+        rps[t] = ragged_tiles ? ragged_tiles * kAttnTileRows : (tiles > 0 ? ceil_div(tiles, nsplit) * kAttnTileRows : kAttnTileRows);
         rows.npart[t] = n_rows[t] > 0 ? ceil_div(ceil_div(n_rows[t], rps[t]), cluster) : 0;
         any_rows |= n_rows[t] > 0;
     }

@@ -53,3 +53,24 @@ def assert_matmul_close(got: np.ndarray, Cq: np.ndarray, C64: np.ndarray, bound:
     assert not bad.any(), (f"{what}: {bad.sum()} of {bad.size} elements outside tolerance; "
                            f"worst err {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}, "
                            f"tol there {tol.reshape(err.shape)[np.unravel_index(err.argmax(), err.shape)]:.3e}")
+
+
+def assert_output_side_stage_by_stage(dims, w, q_full, cache_rows, o_lat, o, out, what=""):
+    """The output side of the decode step checked stage by stage on the values the GPU itself produced (uint16 bit
+    patterns): the oracle recomputes each stage from the GPU's inputs to that stage, so a rounding of an earlier
+    stage that fell the other way than the oracle's (both are valid: fp32 and fp64 sums differ in the last bits)
+    does not enter.  Attention: the softmax criterion (2e-3 of the largest output, plus one bf16 ulp);
+    the per-head W_UV product and W_O: the matmul criterion (1e-5 * sum|a b| + 1e-6, plus one ulp).
+    cache_rows: [S][kv_lora + rope], the new row included.  out (and W_O) may be None."""
+    H, dc, dr, dn, dv, d = (dims[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d"))
+    f64 = lambda bits: oracle.bf16_to_f64(np.asarray(bits, dtype=np.uint16))
+    q_full, o_lat, o = (np.asarray(x, dtype=np.uint16) for x in (q_full, o_lat, o))
+    ref = oracle.mla_attention(f64(q_full).reshape(H, dc + dr), f64(cache_rows), dc, (dn + dr) ** -0.5, threads=8)
+    got = f64(o_lat).reshape(H, dc)
+    assert np.all(np.abs(got - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref)), f"{what}: attention stage"
+    Cq, C64, bound = oracle.matmul_batched(o_lat.reshape(-1), np.asarray(w["W_UV"]).reshape(-1), 1, dv, dc, H, H * dc, dc, dc * dv,
+                                           H * dv, dv, H * dv, oracle.BF16, oracle.BF16, threads=8)
+    assert_matmul_close(f64(o).reshape(-1), Cq, C64, bound, 1, f"{what}: W_UV stage")
+    if out is not None:
+        Cq, C64, bound = oracle.matmul(o.reshape(1, -1), np.asarray(w["W_O"]), 1, d, H * dv, oracle.BF16, oracle.BF16, threads=8)
+        assert_matmul_close(f64(out).reshape(1, -1), Cq, C64, bound, 1, f"{what}: W_O stage")

@@ -6,7 +6,7 @@ import torch
 
 import nm_inputs as gen
 import oracle
-from gpu_util import to_dev
+from gpu_util import assert_output_side_stage_by_stage, to_dev
 
 pytestmark = pytest.mark.gpu
 DIMS = gen.DSV3_DIMS
@@ -83,13 +83,31 @@ def check_against_oracle(w, res, tokens, caches, seq_lens, with_wo=True):
         cache_ref = caches[i]                                # the oracle wrote row S-1 in place
         got = res["cache"][i].cpu().numpy().view(np.uint16)[:S * dkv].reshape(S, dkv)
         assert np.array_equal(got[:S - 1], cache_ref[:S - 1]), f"sequence {i}: old rows changed"
-        assert np.all(np.abs(f64(got[S - 1]) - f64(cache_ref[S - 1])) <= 2 * oracle.ulp_bf16(f64(cache_ref[S - 1])) + 1e-6), i
+        new_row, ref_row = f64(got[S - 1]), f64(cache_ref[S - 1])
+        # normalised part: one ulp of the product's own rounding flip is up to two ulps of an output at the top of its binade,
+        # plus the output's own rounding
+        assert np.all(np.abs(new_row[:dc] - ref_row[:dc]) <= 3 * oracle.ulp_bf16(ref_row[:dc]) + 1e-6), i
+        # the rotated part: a rounding flip of an input moves a pair's outputs on the scale of the pair, not of the
+        # (possibly cancelled) output element
+        assert np.all(np.abs(new_row[dc:] - ref_row[dc:]) <= 2 * oracle.ulp_bf16(np.abs(ref_row[dc:]).max()) + 1e-6), i
         qf = dev_bits_to_f64(res["q_full"][i]).reshape(H, dkv)
         assert rel_max(qf[:, :dc], f64(r["q_lat"])) <= 1e-2 and rel_max(qf[:, dc:], f64(r["q_rope"])) <= 1e-2, i
-        names = [("o_lat", r["o_lat"]), ("o", r["o"])] + ([("out", r["out"])] if with_wo else [])
-        for name, ref_bits in names:
+        # End to end against the oracle's own chain.  The attention output: the softmax criterion.  What follows it inherits
+        # the bf16 roundings of o_lat (and of o) that fell the other way than the oracle's - a valid result, since fp32 and
+        # fp64 sums differ in their last bits, and more frequent after a flip early in the chain (one flipped element of
+        # the normalised query latent moves 1-2 % of q) - each such stage adds up to the same 2e-3 of the largest output
+        # again; so o and out are held to twice the softmax criterion end to end, and to the matmul criterion stage by
+        # stage on the GPU's own stage inputs, where no earlier rounding enters.
+        # Where an early rounding fell the other way (q_full then differs from the oracle's on more than 0.5 % of its elements)
+        # the scores themselves differ, and every end-to-end bound is taken twice.
+        k = 1 if np.mean(qf == np.concatenate([f64(r["q_lat"]), f64(r["q_rope"])], axis=1)) >= 0.995 else 2
+        names = [("o_lat", r["o_lat"], k * 2e-3), ("o", r["o"], k * 4e-3)] + ([("out", r["out"], k * 4e-3)] if with_wo else [])
+        for name, ref_bits, tol in names:
             g, ref = dev_bits_to_f64(res[name][i]).reshape(-1), f64(ref_bits).reshape(-1)
-            assert np.all(np.abs(g - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref)), f"sequence {i}: {name}"
+            assert np.all(np.abs(g - ref) <= tol * np.abs(ref).max() + oracle.ulp_bf16(ref)), f"sequence {i}: {name}"
+        bits = lambda t: t.contiguous().cpu().numpy().view(np.uint16)
+        assert_output_side_stage_by_stage(DIMS, ww, bits(res["q_full"][i]), got, bits(res["o_lat"][i]), bits(res["o"][i]),
+                                          bits(res["out"][i]) if with_wo else None, f"sequence {i}")
 
 
 def make_inputs(seq_lens, seed):

@@ -74,6 +74,32 @@ def test_random_step_matches_the_oracle(nm, weights, seed):
 
 
 @pytest.mark.parametrize("seed", range(16))
+def test_random_tokens_match_the_oracle(nm, weights, seed):
+    """A different token per case (the cases above share one token and vary everything else).  The bf16 rounding after
+    every stage makes the chain sensitive to the last bits of a sum: where the GPU's fp32 sum and the oracle's fp64 sum
+    round one element of the query latent to different neighbours (both valid; about one token in ten), 1-2 % of q
+    and up to a quarter of q_lat follow, and o and out, which inherit the roundings of o_lat, move by up to the softmax
+    criterion again.  So: o_lat end to end within the softmax criterion, o and out within twice that, and the output
+    side stage by stage on the GPU's own stage inputs within the stage criteria."""
+    rng = np.random.default_rng(51_000 + seed)
+    S = int(rng.choice([1, 2, 64, 65, 129, int(rng.integers(130, 3000)), int(rng.integers(130, 3000))]))
+    concat = bool(rng.random() < 0.7)
+    attn = int(rng.choice([0, 0, 1, 2, 3]))
+    h, cache_ref, r = base.oracle_step(weights, S, seed=62_000 + seed, token_seed=63_000 + seed)
+    cache_in = gen.mla_cache(S, DIMS, seed=62_000 + seed)
+    dw = stored(weights, ROW, concat)
+    nm.nm_debug_set_attention(attn)
+    try:
+        t = base.run_step(nm, dw, h, cache_in, S)
+    finally:
+        nm.nm_debug_set_attention(0)
+    try:
+        base.check_step(t, r, cache_ref, S, w=weights, downstream_tol=4e-3)
+    except AssertionError as e:
+        raise AssertionError(f"seed {seed}: S {S} concat {concat} attention {attn}: {e}") from e
+
+
+@pytest.mark.parametrize("seed", range(16))
 def test_random_attention_stage_matches_the_oracle(nm, seed):
     """The attention pass alone on its own random operands (not the output of earlier GPU stages): every kernel,
     lengths from one row to a few thousand, the new row through the merge or through the pass."""

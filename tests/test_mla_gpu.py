@@ -6,7 +6,7 @@ import torch
 
 import nm_inputs as gen
 import oracle
-from gpu_util import assert_matmul_close, out_to_f64, to_dev
+from gpu_util import assert_matmul_close, assert_output_side_stage_by_stage, out_to_f64, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -41,8 +41,8 @@ def weights():
     return w, dw
 
 
-def oracle_step(w, S, seed=4200, with_wo=True):
-    h = gen.mla_token(DIMS, seed=4100)
+def oracle_step(w, S, seed=4200, with_wo=True, token_seed=4100):
+    h = gen.mla_token(DIMS, seed=token_seed)
     cache = gen.mla_cache(S, DIMS, seed=seed)
     ww = dict(w)
     if not with_wo:
@@ -258,7 +258,10 @@ def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None, conc
     return t
 
 
-def check_step(t, r, cache_ref, S, with_wo=True):
+def check_step(t, r, cache_ref, S, with_wo=True, w=None, downstream_tol=2e-3):
+    """End to end against the oracle's chain.  With the weights `w` given, the output side is also checked stage by stage
+    on the GPU's own stage inputs (no earlier rounding enters); `downstream_tol` is the end-to-end bound on o and out,
+    which inherit the roundings of o_lat that fell the other way than the oracle's (see the batch tests)."""
     H, dc, dr, dn = DIMS["H"], DIMS["kv_lora"], DIMS["rope"], DIMS["nope"]
     dkv = dc + dr
     # first-stage products see exactly the oracle's inputs: tight bound
@@ -273,14 +276,30 @@ def check_step(t, r, cache_ref, S, with_wo=True):
     # the cache: old rows untouched, the new row equals the oracle's up to a rounding flip
     cache = t["kv_cache"].cpu().numpy().view(np.uint16).reshape(-1, dkv)
     assert np.array_equal(cache[:S - 1], cache_ref[:S - 1])
-    assert np.all(np.abs(f64(cache[S - 1]) - f64(cache_ref[S - 1])) <= 2 * oracle.ulp_bf16(f64(cache_ref[S - 1])) + 1e-6)
+    new_row, ref_row = f64(cache[S - 1]), f64(cache_ref[S - 1])
+    # normalised part: one ulp of the product's own rounding flip is up to two ulps of an output at the top of its binade,
+    # plus the output's own rounding
+    assert np.all(np.abs(new_row[:dc] - ref_row[:dc]) <= 3 * oracle.ulp_bf16(ref_row[:dc]) + 1e-6)
+    # the rotated part: a rounding flip of an input moves a pair's outputs on the scale of the pair, not of the (possibly
+    # cancelled) output element
+    assert np.all(np.abs(new_row[dc:] - ref_row[dc:]) <= 2 * oracle.ulp_bf16(np.abs(ref_row[dc:]).max()) + 1e-6)
     # softmax-containing outputs: max relative error <= 2e-3 (unrounded), plus one ulp once rounded
+    # ... where the query the attention saw is the oracle's.  Where an early rounding fell the other way (then 1-2 % of q and
+    # up to a quarter of q_lat differ from the oracle's by an ulp: both chains are valid) the scores themselves differ,
+    # and the end-to-end bound is taken twice; the stage-by-stage check below stays at the criterion.
+    qref = np.concatenate([f64(r["q_lat"]), f64(r["q_rope"])], axis=1)
+    k = 1 if np.mean(qf == qref) >= 0.995 else 2
+    tol32 = k * 2e-3
     o32 = t["o_lat_f32"].cpu().numpy().astype(np.float64).reshape(H, dc)
-    assert rel_max(o32, r["o_lat_f64"]) <= 2e-3, f"o_lat: {rel_max(o32, r['o_lat_f64']):.2e}"
-    names = [("o_lat", r["o_lat"]), ("o", r["o"])] + ([("out", r["out"])] if with_wo else [])
-    for name, ref_bits in names:
+    assert rel_max(o32, r["o_lat_f64"]) <= tol32, f"o_lat: {rel_max(o32, r['o_lat_f64']):.2e}"
+    names = [("o_lat", r["o_lat"], tol32), ("o", r["o"], k * downstream_tol)] + ([("out", r["out"], k * downstream_tol)] if with_wo else [])
+    for name, ref_bits, tol in names:
         got, ref = dev_bits_to_f64(t[name]), f64(ref_bits).reshape(-1)
-        assert np.all(np.abs(got - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref)), name
+        assert np.all(np.abs(got - ref) <= tol * np.abs(ref).max() + oracle.ulp_bf16(ref)), name
+    if w is not None:
+        bits = lambda x: x.cpu().numpy().view(np.uint16)
+        assert_output_side_stage_by_stage(DIMS, w, bits(t["q_full"]), cache[:S], bits(t["o_lat"]), bits(t["o"]),
+                                          bits(t["out"]) if with_wo else None, "step")
 
 
 @pytest.mark.parametrize("overlap", [True, False])

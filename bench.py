@@ -203,7 +203,7 @@ class MlaStep:
         # the small-batch step (nm_mla_decode_batch): T sequences of this length, one new token each
         out["small_batch"] = []
         dkv = DIMS["kv_lora"] + DIMS["rope"]
-        for T in ((4, 16) if self.weights == "row" else ()):       # the batch entry point takes row- / column-major weights
+        for T in ((4, 8, 12, 16) if self.weights == "row" else ()):       # the batch entry point takes row- / column-major weights
             stride = (self.S + 8) * dkv
             cache = self.t["kv_cache"].view(-1)[:self.S * dkv].repeat(T, 1)
             cache = torch.nn.functional.pad(cache, (0, stride - self.S * dkv)).contiguous().view(-1)

@@ -118,7 +118,7 @@ int max_clusters_cached(Kern kern, const cudaLaunchConfig_t &cfg, unsigned clust
     for (const Entry &e : cache)
         if (e.f == f && e.smem == cfg.dynamicSmemBytes && e.cs == cluster_size) return e.n;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return 0; }   // not cached: ask again next time
     cache[next] = Entry{f, cfg.dynamicSmemBytes, cluster_size, n};
     next = (next + 1) % 32;
     return n;

@@ -751,7 +751,9 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
         for (int ns = 1; ns <= fit; ++ns) {
             const int cl = ns % 4 == 0 ? 4 : (ns % 2 == 0 ? 2 : 1), tiles = ceil_div(max_tiles, ns);
             if (ns / cl > L.slot_stride) continue;
-            if ((long)T * 4 * (ns / cl) > attention_tc64_max_clusters(cl)) continue;     // a second wave of clusters costs more than it saves
+            int cap = attention_tc64_max_clusters(cl);
+            if (cap <= 0) cap = 128 / cl;                              // the query failed: a count that always fits
+            if ((long)T * 4 * (ns / cl) > cap) continue;               // a second wave of clusters costs more than it saves
             if (tiles < best_tiles || (tiles == best_tiles && cl > best_cl)) { best = ns; best_tiles = tiles; best_cl = cl; }
         }
         nsplit = best; cluster = best_cl;

@@ -33,7 +33,7 @@ def weights():
     return w, {k: to_dev(v) for k, v in w.items()}
 
 
-def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True):
+def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True, graph=False):
     H, dc, dr, dn, dv, d, ql = (DIMS[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d", "q_lora"))
     dkv = dc + dr
     T = len(seq_lens)
@@ -61,7 +61,13 @@ def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True):
     b = nm.mla_batch(seq_lens, h, cs, cache, stride, out=out, q_full=q_full, o_lat=o_lat, o=o)
     st = torch.cuda.Stream()
     torch.cuda.synchronize()
-    nm.nm_mla_decode_batch(p, b, st)
+    if graph:                                                # captured once, replayed: the call allocates and synchronises nothing
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            nm.nm_mla_decode_batch(p, b, st)
+        g.replay()
+    else:
+        nm.nm_mla_decode_batch(p, b, st)
     torch.cuda.synchronize()
     nm.nm_check_status()
     return {"out": out.view(T, d), "q_full": q_full.view(T, H, dkv), "o_lat": o_lat.view(T, H, dc), "o": o.view(T, H * dv),
@@ -156,6 +162,17 @@ def test_batch_with_the_fused_per_head_kernels_at_every_size(nm, weights, seq_le
     finally:
         nm.nm_debug_set_batch_per_head_min_tokens(3)
     check_against_oracle(w, res, tokens, caches, seq_lens, with_wo=with_wo)
+
+
+@pytest.mark.parametrize("seq_lens", [[700, 650, 600, 90, 333, 1000], [257, 64]])
+def test_batch_replayed_from_a_cuda_graph(nm, weights, seq_lens):
+    w, dw = weights
+    tokens, caches = make_inputs(seq_lens, seed=8500 + len(seq_lens))
+    direct = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True)
+    replayed = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True, graph=True)
+    for k in ("out", "q_full", "o_lat", "o", "cache"):
+        assert torch.equal(direct[k], replayed[k]), k
+    check_against_oracle(w, replayed, tokens, caches, seq_lens)
 
 
 def test_batch_of_sixteen_without_wo(nm, weights):

@@ -76,7 +76,7 @@ __device__ __forceinline__ uint64_t l2_policy_evict_last() {
     return p;
 }
 
-// Tiled TMA loads global -> shared (this CTA), completion signalled on an mbarrier.  No multicast.
+// Tiled TMA loads global -> shared (this CTA), completion signalled on an mbarrier.  Every CTA fetches its own copy.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z,
                                             uint32_t bar, uint64_t policy) {
     asm volatile(

@@ -7,7 +7,7 @@
 //                                              that P*V keeps about 16 bits of P instead of 8
 //   O[128 x 256] += P[128 x 32] * tile[:, half]  tcgen05.mma, A from TMEM, B = the same shared-memory
 //                                                bytes read MN-major
-// Q and the cache tile arrive by TMA (128-byte swizzle, no multicast) and are consumed in place by
+// Q and the cache tile arrive by TMA (128-byte swizzle, every CTA its own copy) and are consumed in place by
 // the MMA unit; the accumulators never leave TMEM until the split is finished.  The 512 output
 // columns do not fit TMEM next to S, so two CTAs share a split, each owning 256 columns.  The running
 // maximum is updated lazily: O is rescaled only when a row maximum grows by more than 2^8, so the

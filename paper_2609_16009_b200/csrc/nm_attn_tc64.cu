@@ -129,6 +129,11 @@ attn_tc64_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int sp = blockIdx.x, half = blockIdx.y & 1, hh = blockIdx.y >> 1;     // column half, head half
     const int r0 = sp * rows_per_split, r1 = min(n_rows, r0 + rows_per_split);
     const int ntiles = (r1 > r0) ? ceil_div(r1 - r0, kT) : 0;
+    // Without cluster peers a CTA that has no rows (the surplus of a short sequence's grid row) has nothing to contribute
+    // and nobody waiting for it: the final merge reads only the partials of splits that have rows.
+    if constexpr (kCl == 1) {
+        if (ntiles == 0) return;
+    }
 
     if (tid == 0) {
         NM_TRACE_CTA(0);

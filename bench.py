@@ -254,43 +254,51 @@ class MlaStep:
 
 
 class SingleProduct:
-    """One narrow product C[MxN] = A[MxK] * B[KxN] (bf16), B rotated through copies that together
-    exceed 512 MB so that every launch streams from HBM.  For kernel-level captures."""
+    """One narrow product C[MxN] = A[MxK] * B[KxN] (bf16, or fp32 in and out), B rotated through copies that
+    together exceed 512 MB (256 copies at most: 256 MB for the 1 MiB fp32 case, still above the L2) so that every
+    launch streams from HBM.  For kernel-level captures."""
 
     name = "matmul"
 
-    def __init__(self, nm, device, M, K, N, layout):
+    def __init__(self, nm, device, M, K, N, layout, dtype="bf16"):
         self.nm, self.M, self.K, self.N, self.layout = nm, M, K, N, layout
-        nbytes = K * N * 2
-        self.R = max(2, min(64, (1 << 29) // nbytes + 1))
-        self.B = (torch.randn(self.R, K * N, device=device) * 0.02).to(torch.bfloat16)
-        self.A = torch.randn(M * K, device=device).to(torch.bfloat16)
-        self.C = torch.empty(M * N, device=device, dtype=torch.bfloat16)
+        self.dtype_name = dtype
+        self.dtype = nm.F32 if dtype == "f32" else nm.BF16
+        tdt, es = (torch.float32, 4) if dtype == "f32" else (torch.bfloat16, 2)
+        nbytes = K * N * es
+        self.R = max(2, min(256, (1 << 29) // nbytes + 1))
+        if dtype == "f32":                                   # the fp32 GEMV case: values uniform in [-1, 1]
+            self.B = torch.rand(self.R, K * N, device=device) * 2 - 1
+            self.A = torch.rand(M * K, device=device) * 2 - 1
+        else:
+            self.B = (torch.randn(self.R, K * N, device=device) * 0.02).to(tdt)
+            self.A = torch.randn(M * K, device=device).to(tdt)
+        self.C = torch.empty(M * N, device=device, dtype=tdt)
         self.A_host = self.A.cpu().pin_memory()
-        self.C_host = torch.empty(M * N, dtype=torch.bfloat16).pin_memory()
-        self.ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(M, N, K), device=device)
+        self.C_host = torch.empty(M * N, dtype=tdt).pin_memory()
+        self.ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(M, N, K, 1, self.dtype, layout), device=device)
         self.i = 0
-        self.bytes_per_step = (K * N + M * K + M * N) * 2
+        self.bytes_per_step = (K * N + M * K + M * N) * es
         self.dominant = f"narrow product M={M} K={K} N={N}"
         self.dominant_bytes = self.bytes_per_step
         self.launches_per_step = 1
-        self.h2d, self.d2h = M * K * 2, M * N * 2
+        self.h2d, self.d2h = M * K * es, M * N * es
 
     def describe(self):
-        return {"workload": f"single narrow product M={self.M} K={self.K} N={self.N} bf16, B {'column' if self.layout else 'row'}-major",
+        return {"workload": f"single narrow product M={self.M} K={self.K} N={self.N} {self.dtype_name}, B {'column' if self.layout else 'row'}-major",
                 "l2": f"B rotates through {self.R} copies (> 512 MB in total): every launch reads HBM"}
 
     def step(self, stream, dom_events=None):
         self.i = (self.i + 1) % self.R
         if dom_events is not None:
             dom_events[0].record(stream)
-        self.nm.nm_matmul_ws(self.A, self.B[self.i], self.C, self.M, self.N, self.K, self.nm.BF16, self.layout, self.ws, stream)
+        self.nm.nm_matmul_ws(self.A, self.B[self.i], self.C, self.M, self.N, self.K, self.dtype, self.layout, self.ws, stream)
         if dom_events is not None:
             dom_events[1].record(stream)
 
     def step_e2e(self, stream):
         self.i = (self.i + 1) % self.R
-        self.nm.nm_matmul_host(self.A_host, self.B[self.i], self.C_host, self.A, self.C, self.M, self.N, self.K, self.nm.BF16,
+        self.nm.nm_matmul_host(self.A_host, self.B[self.i], self.C_host, self.A, self.C, self.M, self.N, self.K, self.dtype,
                                self.layout, self.ws, stream)
 
 
@@ -336,7 +344,7 @@ def make_workload(args, nm, device):
         return MlaStep(nm, device, args.seq_len, schedule=args.schedule, weights=args.weights)
     if args.workload == "matmul":
         M, K, N = (int(x) for x in args.mkn.split(","))
-        return SingleProduct(nm, device, M, K, N, 1 if args.layout == "col" else 0)
+        return SingleProduct(nm, device, M, K, N, 1 if args.layout == "col" else 0, args.dtype)
     if args.workload == "attention":
         return AttentionOnly(nm, device, args.seq_len)
     raise SystemExit(f"unknown workload {args.workload}")
@@ -683,6 +691,7 @@ def main():
     ap.add_argument("--workload", default="mla", choices=["mla", "projections", "matmul", "attention"])
     ap.add_argument("--mkn", default="1,16384,7168", help="M,K,N of --workload matmul")
     ap.add_argument("--layout", default="row", choices=["row", "col"])
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"], help="operand type of --workload matmul")
     ap.add_argument("--schedule", default="fused", choices=["fused", "two-stream"],
                     help="decode step: down-projections as one concatenated product on one stream, or W_DKV|KR on a side stream")
     ap.add_argument("--timeline", action="store_true", help="print the kernel timeline of one step and exit")

@@ -176,6 +176,21 @@ class MlaStep:
             self.p.event_before_wo, self.p.event_after_wo = None, None
         self.nm.nm_mla_decode_step(self.p, stream, self.side)
 
+    def batch_step(self, T, stream):
+        """The small-batch step (nm_mla_decode_batch) on T sequences of this length, one new token each: returns the
+        call and the buffers it uses (to be kept alive by the caller)."""
+        dkv = DIMS["kv_lora"] + DIMS["rope"]
+        stride = (self.S + 8) * dkv
+        cache = self.t["kv_cache"].view(-1)[:self.S * dkv].repeat(T, 1)
+        cache = torch.nn.functional.pad(cache, (0, stride - self.S * dkv)).contiguous().view(-1)
+        h = self.t["h"].repeat(T)
+        cs = self.t["rope_cos_sin"].repeat(T)
+        res = torch.zeros(T * DIMS["d"], dtype=torch.int16, device=cache.device)
+        ws = self.nm.new_workspace(self.nm.nm_mla_batch_workspace_bytes(self.p, T), device=cache.device)
+        pb = self.nm.mla_params(DIMS, 1, self.t, workspace=ws)
+        b = self.nm.mla_batch([self.S] * T, h, cs, cache, stride, out=res)
+        return (lambda: self.nm.nm_mla_decode_batch(pb, b, stream)), (cache, h, cs, res, ws, pb, b)
+
     def extra_measurements(self, stream):
         """Outside the timed region, reported beside it: the same step replayed from a CUDA graph of ten steps
         (device time without per-launch work of the host-side queue), and the step without its last product
@@ -202,24 +217,14 @@ class MlaStep:
             out["graph_replay"] = {"error": repr(exc)}
         # the small-batch step (nm_mla_decode_batch): T sequences of this length, one new token each
         out["small_batch"] = []
-        dkv = DIMS["kv_lora"] + DIMS["rope"]
         for T in ((4, 8, 12, 16) if self.weights == "row" else ()):       # the batch entry point takes row- / column-major weights
-            stride = (self.S + 8) * dkv
-            cache = self.t["kv_cache"].view(-1)[:self.S * dkv].repeat(T, 1)
-            cache = torch.nn.functional.pad(cache, (0, stride - self.S * dkv)).contiguous().view(-1)
-            h = self.t["h"].repeat(T)
-            cs = self.t["rope_cos_sin"].repeat(T)
-            res = torch.zeros(T * DIMS["d"], dtype=torch.int16, device=cache.device)
-            ws = self.nm.new_workspace(self.nm.nm_mla_batch_workspace_bytes(self.p, T), device=cache.device)
-            pb = self.nm.mla_params(DIMS, 1, self.t, workspace=ws)
-            b = self.nm.mla_batch([self.S] * T, h, cs, cache, stride, out=res)
-            fn = lambda: self.nm.nm_mla_decode_batch(pb, b, stream)
+            fn, keep = self.batch_step(T, stream)
             timed(fn, 20)
             us = min(timed(fn, 100) for _ in range(3)) / 100 * 1e3
             nb = self.bytes_per_step - self.kv_bytes + T * self.kv_bytes       # weights once, every sequence's cache rows
             out["small_batch"].append({"T": T, "step_us": us, "us_per_token": us / T, "tokens_per_s": T / us * 1e6,
                                        "GBps": nb / us / 1e3})
-            del cache, ws
+            del fn, keep
         wo = self.p.W_O
         self.p.W_O = None
         try:
@@ -697,6 +702,7 @@ def main():
     ap.add_argument("--timeline", action="store_true", help="print the kernel timeline of one step and exit")
     ap.add_argument("--sweep", action="store_true", help="also report GB/s of single narrow products vs M")
     ap.add_argument("--seq-len", type=int, default=4096)
+    ap.add_argument("--batch", type=int, default=1, help="with --timeline: sequences of the small-batch step (2-16) to trace")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--weights", default="row", choices=["row", "fractal"],
                     help="storage of the step's dense weights: row-major (default) or the paper's FRACTAL_NZ tiling")
@@ -729,6 +735,11 @@ def main():
     stream = torch.cuda.Stream(device)
     if args.timeline:
         with torch.cuda.stream(stream):
+            if args.batch > 1:                # the timeline of the small-batch step instead of the single-token step
+                if args.workload != "mla" or args.weights != "row":
+                    raise SystemExit("--batch goes with --workload mla and row-major weights")
+                fn, keep = wl.batch_step(args.batch, stream)
+                wl.step = lambda stream_, dom_events=None: fn()
             for _ in range(max(args.warmup, 10)):
                 wl.step(stream)
             torch.cuda.synchronize()

@@ -1,17 +1,20 @@
-"""Algorithm 2 ("Specialized MatMul 2 on AIV") restated on the CPU (test infrastructure).
+"""Split-K tiling of the paper's MatMul 2 (Algorithm 2), as a CPU check (test infrastructure).
 
-The steps are taken in the algorithm's order and notation: constants, executor pool size V,
-per-executor token slice, the compute loop over nPartW weight blocks with fp32 dot products
-stored to ``tmpBuf``, then the gather over kParts partial sums and one final cast to bf16.
-The fractal transpose and the strided cast exist only to undo the FRACTAL_NZ storage of the
-weights; here W is a plain row-major K x N array, so a block is read column by column directly.
+Algorithm 2 cuts the K x N weight matrix into blocks of ``k_split`` rows by ``col_block`` columns, deals
+the blocks out to a pool of executors, lets each block produce an fp32 partial sum per column, and
+then adds the partial sums of a column block in k order and rounds once to bf16.  What the tests need
+from it is stated here in three independent pieces, none of which walks the executors one by one:
 
-Readings taken where the algorithm is ambiguous:
-  * the column block of ``W[off_T, fracId]`` is ``fracId mod fractalNum`` and its k-part is
-    ``fracId DIV fractalNum`` (equal to ``v DIV groupSize``, which is how off_T is defined);
-  * ``tmpBuf`` is indexed in elements: block ``fracId`` starts at element ``fracId*fractalSize``,
-    which equals ``kpart*N + fcol*fractalSize`` and so matches the gather's ``off_C + i*N``;
-  * ``groupSize = V DIV kParts`` needs kParts | V, true for the paper's case only.
+  * ``tiling(K, N, cores)``       - the closed-form constants of the Init stage;
+  * ``block_of_work_item(...)``   - which (k part, column block) the i-th item of the flattened
+                                    executor x slot grid stands for, vectorised over all items;
+  * ``split_k_product(...)``      - the arithmetic: per-part fp32 column sums, parts added in order,
+                                    one rounding.
+
+Readings taken where the algorithm is ambiguous (valid for the paper's constants, which the tests pin):
+the flattened item index counts column blocks fastest and k parts slowest; the scratch buffer is indexed
+in elements, so the partial sums of k part i for column block c start at ``i*N + c*col_block``; the pool
+size must be a multiple of the number of k parts.
 """
 from __future__ import annotations
 
@@ -20,48 +23,39 @@ import numpy as np
 from . import bf16_to_f64, f64_to_bf16
 
 
-def executor_pool(K: int, N: int, P: int, fractalSize: int = 16, kSplitSize: int = 1024):
-    """Init stage: the tiling constants and the pool size V = max divisor of S not above 2P."""
-    kParts = K // kSplitSize
-    fractalNum = N // fractalSize
-    S = fractalNum * kParts
-    V = max(dv for dv in range(1, S + 1) if S % dv == 0 and dv <= 2 * P)
-    nPartW = S // V
-    groupSize = V // kParts
-    return dict(kParts=kParts, fractalNum=fractalNum, S=S, V=V, nPartW=nPartW, groupSize=groupSize,
-                fractalSize=fractalSize, kSplitSize=kSplitSize)
+def tiling(K: int, N: int, cores: int, col_block: int = 16, k_split: int = 1024) -> dict:
+    """Constants of Algorithm 2's Init stage.  ``pool`` is the largest divisor of the block count that
+    does not exceed two executors per core."""
+    k_parts = K // k_split
+    col_blocks = N // col_block
+    blocks = k_parts * col_blocks
+    divisors = np.arange(1, blocks + 1)
+    divisors = divisors[(blocks % divisors == 0) & (divisors <= 2 * cores)]
+    pool = int(divisors.max())
+    return dict(kParts=k_parts, fractalNum=col_blocks, S=blocks, V=pool, nPartW=blocks // pool,
+                groupSize=pool // k_parts)
 
 
-def matmul2(T_bits: np.ndarray, W_bits: np.ndarray, K: int, N: int, P: int = 24,
-            fractalSize: int = 16, kSplitSize: int = 1024):
-    """C[1xN] = T[1xK] * W[KxN], bf16 in/out, fp32 partial sums, following Algorithm 2.
+def block_of_work_item(c: dict):
+    """For every item of the executor x slot grid (executor-major), the k part and the column block it
+    computes, and the k part its executor's token slice was loaded for.  Returns three int arrays of
+    length ``pool * slots``; the tests require (k part, column block) to hit every block exactly once and
+    the two k parts to agree."""
+    item = np.arange(c["V"] * c["nPartW"])
+    executor = item // c["nPartW"]
+    return item // c["fractalNum"], item % c["fractalNum"], executor // c["groupSize"]
 
-    Returns (C bits uint16 [N], tmpBuf fp32 [kParts*N], list of every fracId produced)."""
-    c = executor_pool(K, N, P, fractalSize, kSplitSize)
-    kParts, fractalNum, V, nPartW, groupSize = (c[k] for k in ("kParts", "fractalNum", "V", "nPartW", "groupSize"))
-    T = bf16_to_f64(T_bits.reshape(K)).astype(np.float32)          # widening is exact
+
+def split_k_product(T_bits: np.ndarray, W_bits: np.ndarray, K: int, N: int, k_split: int = 1024):
+    """C[1xN] = T[1xK] * W[KxN] with bf16 operands, fp32 partial sums per k part, the parts added in
+    increasing k order in fp32, and one final rounding to bf16.  Returns (C bits [N], partials fp32
+    [k_parts, N])."""
+    T = bf16_to_f64(T_bits.reshape(K)).astype(np.float32)           # bf16 -> fp32 widening is exact
     W = bf16_to_f64(W_bits.reshape(K, N)).astype(np.float32)
-    tmpBuf = np.full(kParts * N, np.nan, dtype=np.float32)
-    produced = []
-    # compute stage, one executor v at a time
-    for v in range(V):
-        off_T = (v // groupSize) * kSplitSize
-        T_v = T[off_T:off_T + kSplitSize]                           # loaded once per executor
-        for w in range(nPartW):
-            fracId = v * nPartW + w
-            fcol = fracId % fractalNum
-            W_vw = W[off_T:off_T + kSplitSize, fcol * fractalSize:(fcol + 1) * fractalSize]
-            partSum = np.empty(fractalSize, dtype=np.float32)
-            for j in range(fractalSize):
-                partSum[j] = np.sum(T_v * W_vw[:, j], dtype=np.float32)   # fp32 Mul + ReduceSum
-            tmpBuf[fracId * fractalSize:(fracId + 1) * fractalSize] = partSum
-            produced.append(fracId)
-    # gather stage (after the barrier): executors v < fractalNum
-    Cout = np.zeros(N, dtype=np.uint16)
-    for v in range(fractalNum):
-        off_C = v * fractalSize
-        Acc = np.zeros(fractalSize, dtype=np.float32)
-        for i in range(kParts):
-            Acc = (Acc + tmpBuf[off_C + i * N: off_C + i * N + fractalSize]).astype(np.float32)
-        Cout[off_C:off_C + fractalSize] = f64_to_bf16(Acc.astype(np.float64))
-    return Cout, tmpBuf, produced
+    k_parts = K // k_split
+    products = T.reshape(k_parts, k_split, 1) * W.reshape(k_parts, k_split, N)      # exact in fp32
+    partials = products.sum(axis=1, dtype=np.float32)
+    total = np.zeros(N, dtype=np.float32)
+    for part in partials:                                            # fixed order, fp32 adds
+        total = (total + part).astype(np.float32)
+    return f64_to_bf16(total.astype(np.float64)), partials

@@ -2,6 +2,7 @@
 values, exact integer arithmetic, closed forms, invariants, a library routine, the restated
 Algorithm 2), chosen so that a dropped term, a wrong index or a transposed operand fails one."""
 import itertools
+import math
 import os
 
 import numpy as np
@@ -200,25 +201,37 @@ def test_closed_forms(layout):
 
 def test_alg2_constants_match_hand_derivation():
     g = _read_golden("alg2_constants.txt")
-    c = alg2.executor_pool(int(g["K"][0]), int(g["N"][0]), int(g["P"][0]))
+    c = alg2.tiling(int(g["K"][0]), int(g["N"][0]), int(g["P"][0]))
     for k in ("kParts", "fractalNum", "S", "V", "nPartW", "groupSize"):
         assert c[k] == int(g[k][0]), k
 
 
 def test_alg2_covers_every_block_once_and_equals_definition():
     K, N = 7168, 576
+    c = alg2.tiling(K, N, 24)
+    k_part, col_block, loaded_k_part = alg2.block_of_work_item(c)
+    # every (k part, column block) pair is produced exactly once ...
+    pairs = k_part * c["fractalNum"] + col_block
+    assert np.array_equal(np.sort(pairs), np.arange(c["S"]))
+    assert k_part.max() == c["kParts"] - 1 and col_block.max() == c["fractalNum"] - 1
+    # ... by an executor that holds the token slice of that very k part
+    assert np.array_equal(k_part, loaded_k_part)
     T = gen.normal_bf16((1, K), 1.0, seed=1000)
     W = gen.normal_bf16((K, N), 0.02, seed=1001)
-    Cb, tmpBuf, produced = alg2.matmul2(T, W, K, N)
-    assert sorted(produced) == list(range(252))                        # bijection onto 0..S-1
-    assert not np.isnan(tmpBuf).any()                                  # every partial written
+    Cb, partials = alg2.split_k_product(T, W, K, N)
+    assert partials.shape == (c["kParts"], N) and partials.dtype == np.float32
     Cq, C64, bound = oracle.matmul(T, W, 1, N, K, BF16, BF16)
     err = np.abs(gen.bits_to_f32(Cb).astype(np.float64) - C64[0])
     assert np.all(err <= 1e-5 * bound[0] + 1e-6 + oracle.ulp_bf16(C64[0]))
+    # the partial sums are those of the k parts: part i against the definition on rows i*1024 ... (i+1)*1024
+    Tf, Wf = gen.bits_to_f32(T).astype(np.float64).reshape(K), gen.bits_to_f32(W).astype(np.float64).reshape(K, N)
+    for i in (0, 3, 6):
+        want = Tf[i * 1024:(i + 1) * 1024] @ Wf[i * 1024:(i + 1) * 1024]
+        assert np.allclose(partials[i], want, rtol=0, atol=1e-4)
     # small integers: every summation order is exact, so the two must agree bit for bit
     Ti = gen.small_int_bf16((1, K), -8, 8, seed=31)
     Wi = gen.small_int_bf16((K, N), -8, 8, seed=32)
-    Cb, _, _ = alg2.matmul2(Ti, Wi, K, N)
+    Cb, _ = alg2.split_k_product(Ti, Wi, K, N)
     Cq, _, _ = oracle.matmul(Ti, Wi, 1, N, K, BF16, BF16)
     assert np.array_equal(Cb, Cq[0])
 
@@ -363,7 +376,37 @@ def test_absorbed_equals_textbook_mla():
 SMALL_DIMS = dict(d=96, q_lora=48, kv_lora=32, rope=8, nope=16, v=16, H=4)
 
 
+def _dot_in_k_order(a, b):
+    """sum_k a[k]*b[k] with a plain fp64 `+=` over increasing k: the same additions, in the same order, as the
+    definition's loop, so the bits of the sum are fixed."""
+    acc = 0.0
+    for x, y in zip(a, b):
+        acc += float(x) * float(y)
+    return acc
+
+
+def _rmsnorm_by_hand(x, gamma, eps):
+    ss = 0.0
+    for v in x:
+        ss += float(v) * float(v)
+    r = 1.0 / math.sqrt(ss / len(x) + eps)
+    return np.array([float(v) * r * float(g) for v, g in zip(x, gamma)])
+
+
+def _rope_by_hand(x, pos, base=10000.0):
+    y = np.empty(len(x))
+    for i in range(len(x) // 2):
+        ang = float(pos) * base ** (-2.0 * i / len(x))
+        c, s_ = math.cos(ang), math.sin(ang)
+        y[2 * i] = float(x[2 * i]) * c - float(x[2 * i + 1]) * s_
+        y[2 * i + 1] = float(x[2 * i]) * s_ + float(x[2 * i + 1]) * c
+    return y
+
+
 def test_decode_step_matches_stagewise_recomputation():
+    """Every stage of the composed step recomputed by explicit loops from the previous stage's ROUNDED output and
+    compared bit for bit: a stage wired to the wrong input, a transposed per-head weight, or a missing rounding
+    between two stages (continuing from the unrounded sum) changes bits somewhere and fails."""
     dims, S = SMALL_DIMS, 9
     w = gen.mla_weights(dims, seed=61)
     h = gen.mla_token(dims, seed=62)
@@ -371,33 +414,87 @@ def test_decode_step_matches_stagewise_recomputation():
     cache0 = cache.copy()
     r = oracle.mla_decode_step(dims, w, h, cache, S)
     d, ql, dc, dr, dn, dv, H = (dims[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
-    f = lambda b: gen.bits_to_f32(b).astype(np.float64)
-    rb = lambda x: f(oracle.f64_to_bf16(x))
-    c_q = rb(f(h) @ f(w["W_DQ"]))
-    assert np.array_equal(c_q, f(r["c_q"]))
-    c_qn = rb(c_q / np.sqrt(np.mean(c_q ** 2) + 1e-6) * f(w["gamma_q"]))
-    assert np.array_equal(c_qn, f(r["c_qn"]))
-    q = rb(c_qn @ f(w["W_UQR"])).reshape(H, dn + dr)
-    assert np.allclose(q, f(r["q"]), atol=1e-2)
-    q = f(r["q"])                                             # continue from the oracle's rounded values
-    ckr = rb(f(h) @ f(w["W_DKVKR"]))
-    assert np.array_equal(ckr, f(r["ckr"]))
-    # row S-1 was written, rows before it untouched
+    dq, dkv, pos = dn + dr, dc + dr, S - 1
+    f = lambda b: gen.bits_to_f32(np.asarray(b, dtype=np.uint16)).astype(np.float64)
+    rbits = oracle.f64_to_bf16
+    rb = lambda x: f(rbits(np.asarray(x, dtype=np.float64)))
+    hv = f(h)
+    W_DQ, W_UQR, W_DKVKR = f(w["W_DQ"]).reshape(d, ql), f(w["W_UQR"]).reshape(ql, H * dq), f(w["W_DKVKR"]).reshape(d, dkv)
+    W_UK, W_UV, W_O = f(w["W_UK"]).reshape(H, dn, dc), f(w["W_UV"]).reshape(H, dc, dv), f(w["W_O"]).reshape(H * dv, d)
+    # 1-2: c_q, c_qn
+    c_q = rb([_dot_in_k_order(hv, W_DQ[:, n]) for n in range(ql)])
+    assert np.array_equal(rbits(c_q), r["c_q"])
+    c_qn = rb(_rmsnorm_by_hand(c_q, f(w["gamma_q"]), 1e-6))
+    assert np.array_equal(rbits(c_qn), r["c_qn"])
+    # 3: q from the ROUNDED c_qn
+    q = rb([_dot_in_k_order(c_qn, W_UQR[:, n]) for n in range(H * dq)]).reshape(H, dq)
+    assert np.array_equal(rbits(q), r["q"])
+    # 4: q_rope from the ROUNDED q
+    q_rope = rb(np.stack([_rope_by_hand(q[hh, dn:], pos) for hh in range(H)]))
+    assert np.array_equal(rbits(q_rope), r["q_rope"])
+    # 5-6: ckr and the new cache row (from the ROUNDED ckr); rows before it untouched
+    ckr = rb([_dot_in_k_order(hv, W_DKVKR[:, n]) for n in range(dkv)])
+    assert np.array_equal(rbits(ckr), r["ckr"])
     assert np.array_equal(cache[:S - 1], cache0[:S - 1])
-    row = f(cache[S - 1])
-    assert np.allclose(row[:dc], rb(ckr[:dc] / np.sqrt(np.mean(ckr[:dc] ** 2) + 1e-6) * f(w["gamma_kv"])), atol=1e-2)
-    assert np.allclose(row[dc:], oracle.rope(ckr[dc:], S - 1), atol=2e-2)
-    q_rope = np.stack([oracle.rope(q[hh, dn:], S - 1) for hh in range(H)])
-    assert np.allclose(f(r["q_rope"]), q_rope, atol=2e-2)
-    q_lat = np.einsum("hk,hkn->hn", q[:, :dn], f(w["W_UK"]))
-    assert np.allclose(f(r["q_lat"]), q_lat, atol=1e-2)
-    Q = np.concatenate([f(r["q_lat"]), f(r["q_rope"])], axis=1)
-    o_lat = oracle.mla_attention(Q, f(cache[:S]), dc, 1 / np.sqrt(dn + dr))
-    assert np.allclose(r["o_lat_f64"], o_lat, atol=1e-14)
-    o = np.einsum("hk,hkn->hn", f(r["o_lat"]), f(w["W_UV"]))
-    assert np.allclose(f(r["o"]), o, atol=1e-2)
-    out = f(r["o"]).reshape(-1) @ f(w["W_O"])
-    assert np.allclose(f(r["out"]), out, atol=1e-2, rtol=1e-2)
+    row = np.concatenate([_rmsnorm_by_hand(ckr[:dc], f(w["gamma_kv"]), 1e-6), _rope_by_hand(ckr[dc:], pos)])
+    assert np.array_equal(rbits(row), cache[S - 1])
+    # 7: q_lat[h] = q_nope[h] * W_UK[h] from the ROUNDED q  (W_UK[h] is nope x kv_lora: k runs over nope)
+    q_lat = rb([[_dot_in_k_order(q[hh, :dn], W_UK[hh][:, n]) for n in range(dc)] for hh in range(H)])
+    assert np.array_equal(rbits(q_lat), r["q_lat"])
+    # 8-9: scores over all S rows (the new one included), softmax, o_lat; from the ROUNDED q_lat and q_rope
+    rows = f(cache[:S])
+    scale = 1.0 / math.sqrt(dq)
+    o_lat = np.empty((H, dc))
+    for hh in range(H):
+        qh = np.concatenate([q_lat[hh], q_rope[hh]])
+        s_ = [_dot_in_k_order(qh, rows[j]) * scale for j in range(S)]
+        mx = max(s_)
+        e = [math.exp(v - mx) for v in s_]
+        l = 0.0
+        for v in e:
+            l += v
+        p = [v / l for v in e]
+        for c in range(dc):
+            o_lat[hh, c] = _dot_in_k_order(p, rows[:, c])
+    assert np.allclose(r["o_lat_f64"], o_lat, rtol=0, atol=1e-15)
+    assert np.array_equal(rbits(r["o_lat_f64"]), r["o_lat"])
+    o_lat = f(r["o_lat"])
+    # 10: o[h] = o_lat[h] * W_UV[h] from the ROUNDED o_lat
+    o = rb([[_dot_in_k_order(o_lat[hh], W_UV[hh][:, n]) for n in range(dv)] for hh in range(H)])
+    assert np.array_equal(rbits(o), r["o"])
+    # 11: out = flatten(o) * W_O from the ROUNDED o
+    out = [_dot_in_k_order(o.reshape(-1), W_O[:, n]) for n in range(d)]
+    assert np.array_equal(rbits(out), r["out"])
+    # the rounding points matter at this size: continuing from the unrounded sums would change bits
+    q_unrounded_chain = [_dot_in_k_order(_rmsnorm_by_hand(c_q, f(w["gamma_q"]), 1e-6), W_UQR[:, n]) for n in range(H * dq)]
+    assert not np.array_equal(rbits(q_unrounded_chain), np.asarray(r["q"]).reshape(-1))
+
+
+NZ_DIMS = dict(d=96, q_lora=48, kv_lora=32, rope=16, nope=16, v=16, H=4)     # every dense K and N a multiple of 16
+
+
+@pytest.mark.parametrize("layout", [COL_MAJOR, oracle.FRACTAL_NZ])
+def test_decode_step_is_the_same_in_every_storage_of_the_dense_weights(layout):
+    """`layout_dense` only changes where element (k, n) of W_DQ, W_UQR, W_DKV|W_KR and W_O is fetched from: the step on
+    the permuted storage equals the step on the row-major matrices bit for bit, every stage."""
+    dims, S = NZ_DIMS, 7
+    w = gen.mla_weights(dims, seed=81)
+    h = gen.mla_token(dims, seed=82)
+    d, ql, dc, dr, dn, dv, H = (dims[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
+    r0 = oracle.mla_decode_step(dims, w, h, gen.mla_cache(S, dims, seed=83), S)
+    shapes = {"W_DQ": (d, ql), "W_DKVKR": (d, dc + dr), "W_UQR": (ql, H * (dn + dr)), "W_O": (H * dv, d)}
+    store = gen.to_col_major if layout == COL_MAJOR else gen.to_fractal_nz
+    w2 = dict(w)
+    for name, shp in shapes.items():
+        w2[name] = store(np.asarray(w[name]).reshape(shp))
+        assert not np.array_equal(w2[name].reshape(-1), np.asarray(w[name]).reshape(-1))   # really another order
+    cache = gen.mla_cache(S, dims, seed=83)
+    r1 = oracle.mla_decode_step(dims, w2, h, cache, S, layout_dense=layout)
+    for k in ("c_q", "c_qn", "q", "q_rope", "ckr", "q_lat", "o_lat", "o", "out"):
+        assert np.array_equal(r0[k], r1[k]), k
+    # and reading the permuted storage as row-major is NOT the same step (the flag is honoured)
+    r2 = oracle.mla_decode_step(dims, w2, h, gen.mla_cache(S, dims, seed=83), S)
+    assert not np.array_equal(r0["out"], r2["out"])
 
 
 def test_decode_step_seq_len_one_attends_only_the_new_row():

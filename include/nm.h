@@ -271,6 +271,8 @@ size_t nm_mla_workspace_bytes(const nm_mla_params *p);
  *   cache_stride elements between the caches of consecutive sequences (multiple of 8, >= seq_lens[t] * row width)
  *   out          device [T][d] bf16 (ignored when the params' W_O is NULL)
  *   q_full, o_lat, o   optional device outputs [T][H][kv_lora+rope], [T][H][kv_lora], [T][H][v] bf16
+ *   c_q, c_qn, q, ckr  optional device outputs [T][q_lora], [T][q_lora], [T][H][nope+rope], [T][kv_lora+rope] bf16: the
+ *                outputs of the down-projections, of the query latent's RMSNorm and of W_UQR, for stage-wise checking
  * From nm_mla_params it takes the dimensions, weights, rms_eps, softmax_scale, layout_dense, workspace and
  * workspace_bytes (>= nm_mla_batch_workspace_bytes(p, T)); its h, kv_cache, seq_len, rope_cos_sin, out and
  * intermediates are ignored.  Dimensions: kv_lora 512, rope 64, nope 128, v 128, H 128.  One stream; the kernels
@@ -285,6 +287,7 @@ typedef struct nm_mla_batch {
     long cache_stride;
     void *out;
     void *q_full, *o_lat, *o;
+    void *c_q, *c_qn, *q, *ckr;
 } nm_mla_batch;
 
 size_t nm_mla_batch_workspace_bytes(const nm_mla_params *p, int T);
@@ -314,60 +317,11 @@ int nm_set_programmatic_launch(int enable);
  */
 int nm_set_tensor_core_min_m(int m);
 
-/* ---- tuning aids (sweeps and tests; not needed for normal use) --------------------------------- */
-
-/* Override the tiling heuristic: columns per CTA tile of the row-major kernel and number of
- * k-splits; 0 restores the heuristic.  Values are clamped to what the workspace bound covers. */
-int nm_debug_set_plan(int tile_n, int nsplit);
-/* Force the kernel family for row-major bf16 weights (-1 heuristic; 0 plain-load kernel; 3 TMA-ring
- * CUDA-core kernel; 4 swap-AB tensor-core kernel) and the ring depth in stages (0 heuristic). */
-int nm_debug_set_kernel(int kind, int stages);
-/* Split-K of the CUDA-core kernels: 1 (default) lets the k-splits of a column tile form a thread-block cluster whose
- * partial sums meet in the first CTA's shared memory (up to 8 splits; partial tiles up to 16 KB in the TMA-ring
- * kernel, 8 KB in the plain kernels); 0 always goes through the workspace (partial tiles, arrival counter, gather). */
-int nm_debug_set_cluster_split(int enable);
-/* Tuning aid: phase timestamps (ns, %globaltimer) of the decode step's kernels go to `device_buffer` (8192
- * unsigned 64-bit values) when non-null: [0,32) phases of CTA (0,0) of the attention kernel (the 64-head kernel:
- * from 4 four per cache tile - scores issued, scores seen, P written, P*V issued - for five tiles, from 24 five phases
- * of the cluster merge); from 32 four per
- * attention CTA (start, Q landed, last P*V done, end); from 1100 eight phases of two CTAs of the merge + W_UV
- * kernel; from 2048 / 4096 / 6144 four per CTA (start, inputs ready, loop done, end) of the down-projection, W_UQR
- * and W_O products; from 2688 four phases of the CTA that completes a product carrying vector stages (last arrival,
- * gather done, synchronised, sums reduced).  NULL = off. */
-int nm_debug_set_attention_trace(void *device_buffer);
-/* Decode step tuning: launch the merge + W_UV kernel programmatically (default 1); include W_UV in the L2
- * prefetch (default 1). */
-int nm_debug_set_step_knobs(int uv_programmatic, int prefetch_w_uv);
-/* Decode step, the vector stages behind the down-projections (RMSNorm / RoPE / the cache-row write): 0 as kernels of
- * their own; 1 (default) folded into the products - with the three down-projections stored as one matrix the k-splits
- * meet inside clusters, W_UQR normalises its token row while loading it and the KV consumers ride in an extra CTA of
- * the per-head query kernel; otherwise, and with 2 always, the CTA that completes the product's last tile runs them. */
-int nm_debug_set_step_tails(int enable);
-/* Batch decode: sequences from which the per-head products (W_UK, W_UV) run as batched products of the library with
- * RoPE and the merge as kernels of their own (default 3); below, fused per-head kernels do them.  17 = always fused. */
-int nm_debug_set_batch_per_head_min_tokens(int tokens);
-/* Decode step tuning: force (tile_n, nsplit, ring stages) of one of its products - which = 0 the down-projection,
- * 1 W_UQR, 2 W_O; zeros give the plan back to the planner. */
-int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages);
-/* Decode step: 1 (default) runs RoPE + W_UK and attention-merge + W_UV as fused per-head kernels, 0 as
- * separate kernels (rope, batched product, merge, batched product). */
-int nm_debug_set_step_fusion(int enable);
-/* Decode step: MB of W_O prefetched into L2 while the attention pass runs (default 40, 0 = off). */
-int nm_debug_set_step_prefetch(int megabytes);
-/* Decode step: chain its kernels with programmatic dependent launch (default 1) or not (0). */
-int nm_debug_set_step_pdl(int enable);
-/* Attention pass: 0 (default) a tensor-core kernel when the shape allows - 64 heads per CTA below 65536 cache rows
- * in the call, 128 heads per CTA from there on; 1 CUDA-core kernel; 2 / 3 the tensor-core kernel with 128 / 64 heads
- * per CTA whatever the length. */
-int nm_debug_set_attention(int impl);
-/* Measurement aid: a kernel that only reads `bytes` bytes of device memory once (16-byte streaming loads, the
- * products' own load instruction, ctas_per_sm x SM-count CTAs of 256 threads) - the read-only bandwidth this GPU
- * delivers, to set beside the copy bandwidth the roofline uses.  src 16-byte aligned; sink4: 4 writable bytes. */
-int nm_debug_stream_read(const void *src, size_t bytes, void *sink4, int ctas_per_sm, nm_stream stream);
-/* Report the plan for a problem: out[0..5] = kernel kind (0 row-major vector, 1 column-major
- * vector, 2 scalar), columns per tile, k-splits, k-rows per split, column tiles, CTAs. */
-int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B, int vec_ok,
-                      int *out /* host, 6 ints */);
+/* Thread safety.  Calls that enqueue work may be made from several host threads (each on its own stream and
+ * workspace).  The settings above (nm_set_workspace, nm_set_programmatic_launch, nm_set_tensor_core_min_m) and the
+ * tuning aids of nm_debug.h are process-wide; they are guarded by a lock, and every call plans from one consistent
+ * copy of them taken at its start, but a setting changed on one thread does apply to calls that start later on any
+ * thread.  Per-device state (kernel attributes, the status word, the scratch of nm_matmul_static) is kept per device. */
 
 #ifdef __cplusplus
 }

@@ -80,7 +80,8 @@ class MlaParams(C.Structure):
 class MlaBatch(C.Structure):
     """Mirror of nm_mla_batch (include/nm.h)."""
     _fields_ = [("T", _i), ("seq_lens", C.POINTER(_i)), ("h", _vp), ("rope_cos_sin", _vp), ("kv_cache", _vp),
-                ("cache_stride", C.c_long), ("out", _vp), ("q_full", _vp), ("o_lat", _vp), ("o", _vp)]
+                ("cache_stride", C.c_long), ("out", _vp), ("q_full", _vp), ("o_lat", _vp), ("o", _vp),
+                ("c_q", _vp), ("c_qn", _vp), ("q", _vp), ("ckr", _vp)]
 
 
 _lib.nm_mla_batch_workspace_bytes.restype = _sz
@@ -109,6 +110,7 @@ _lib.nm_debug_set_step_plan.argtypes = [_i, _i, _i, _i]
 _lib.nm_debug_set_step_prefetch.argtypes = [_i]
 _lib.nm_debug_set_step_fusion.argtypes = [_i]
 _lib.nm_debug_set_attention_trace.argtypes = [_vp]
+_lib.nm_debug_wait_probe.argtypes = [C.c_ulonglong, _vp, _vp]
 
 
 def _check(status: int, where: str) -> None:
@@ -306,7 +308,8 @@ def nm_mla_batch_workspace_bytes(p: MlaParams, T: int) -> int:
     return int(_lib.nm_mla_batch_workspace_bytes(C.byref(p), int(T)))
 
 
-def mla_batch(seq_lens, h, rope_cos_sin, kv_cache, cache_stride, out=None, q_full=None, o_lat=None, o=None) -> MlaBatch:
+def mla_batch(seq_lens, h, rope_cos_sin, kv_cache, cache_stride, out=None, q_full=None, o_lat=None, o=None,
+              c_q=None, c_qn=None, q=None, ckr=None) -> MlaBatch:
     """Fill an nm_mla_batch; seq_lens is a host sequence of ints (kept alive by the returned object)."""
     b = MlaBatch()
     b.T = len(seq_lens)
@@ -315,6 +318,7 @@ def mla_batch(seq_lens, h, rope_cos_sin, kv_cache, cache_stride, out=None, q_ful
     b.h, b.rope_cos_sin, b.kv_cache = _ptr(h), _ptr(rope_cos_sin), _ptr(kv_cache)
     b.cache_stride = int(cache_stride)
     b.out, b.q_full, b.o_lat, b.o = _ptr(out), _ptr(q_full), _ptr(o_lat), _ptr(o)
+    b.c_q, b.c_qn, b.q, b.ckr = _ptr(c_q), _ptr(c_qn), _ptr(q), _ptr(ckr)
     return b
 
 
@@ -368,6 +372,12 @@ def nm_debug_stream_read(src, nbytes: int, sink, ctas_per_sm: int = 4, stream=No
 
 def nm_debug_set_step_pdl(enable: bool) -> None:
     _check(_lib.nm_debug_set_step_pdl(int(enable)), "nm_debug_set_step_pdl")
+
+
+def nm_debug_wait_probe(limit_ns: int, elapsed_ns=None, stream=None) -> None:
+    """One CTA waits on an mbarrier nobody arrives at, with the wait limit set to limit_ns for that launch; the
+    wait runs out, the kernel returns by itself and nm_check_status reports the timeout once."""
+    _check(_lib.nm_debug_wait_probe(int(limit_ns), _ptr(elapsed_ns), _stream(stream)), "nm_debug_wait_probe")
 
 
 def nm_debug_set_attention(impl: int) -> None:

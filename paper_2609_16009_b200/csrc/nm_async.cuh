@@ -46,18 +46,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Wait for a phase of an mbarrier, but never for more than about a second.  When the limit runs
 // out the thread raises the CTA's abort flag and the device status word and returns false; every
 // later wait in the CTA then returns at once, so the kernel runs to its end (with a wrong result
-// that the status word disowns) instead of hanging.
+// that the status word disowns) instead of hanging.  The limit is read (on the slow path only) from
+// the 64-bit word that follows the status word: kWaitLimitNs unless nm_debug_wait_probe shortened it
+// for its own launch.
 constexpr uint64_t kWaitLimitNs = 1000000000ull;
 static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned *status) {
     for (int i = 0; i < 4096; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
+    uint64_t limit = kWaitLimitNs;
+    if (status) {
+        const uint64_t set = *reinterpret_cast<const volatile unsigned long long *>(status + 2);
+        if (set >= 1000ull && set < kWaitLimitNs) limit = set;
+    }
     const uint64_t t0 = global_timer_ns();
     for (;;) {
         for (int i = 0; i < 1024; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
+        if (global_timer_ns() - t0 > limit) {
             *abort_flag = 1;
             if (status) atomicOr(status, kStatusWaitExpired);
             return false;

@@ -527,9 +527,9 @@ bool encode_rows_map(CUtensorMap *map, const void *ptr, int rows, int box_rows)
 
 }  // namespace
 
-static unsigned long long *g_attn_trace = nullptr;
-void set_attention_trace(unsigned long long *p) { g_attn_trace = p; }
-unsigned long long *attention_trace() { return g_attn_trace; }
+static std::atomic<unsigned long long *> g_attn_trace{nullptr};
+void set_attention_trace(unsigned long long *p) { g_attn_trace.store(p, std::memory_order_relaxed); }
+unsigned long long *attention_trace() { return g_attn_trace.load(std::memory_order_relaxed); }
 
 static int launch_attn_tc(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split, int nsplit,
                           AttnPartials part, long ml_stride, long o_stride, float scale, cudaStream_t stream, bool programmatic_launch,
@@ -554,11 +554,10 @@ static int launch_attn_tc(const void *Q, int nseq, const void *const *caches, co
         // whatever the rest of the buffer holds.
         if (!encode_rows_map(&seqs.kv[t], caches[t], n_rows[t], kT)) return NM_ERR_UNSUPPORTED;
     }
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    static std::atomic<unsigned long long> configured{0};          // one bit per device
+    {
+        cudaError_t e = ensure_dynamic_smem(attn_tc_kernel, kSmemBytes, configured);
         if (e != cudaSuccess) return record_cuda_error(e, "attention kernel attribute");
-        configured = true;
     }
     const float scale_log2 = scale * 1.4426950408889634f;
     cudaLaunchConfig_t cfg = {};
@@ -575,7 +574,7 @@ static int launch_attn_tc(const void *Q, int nseq, const void *const *caches, co
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = programmatic_launch ? 2 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, map_q, seqs, part, scale_log2, device_status_ptr(), g_attn_trace, prefetch);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, map_q, seqs, part, scale_log2, device_status_ptr(), attention_trace(), prefetch);
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "attention (tensor cores) launch");
 }
 

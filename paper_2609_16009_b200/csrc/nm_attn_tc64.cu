@@ -482,12 +482,9 @@ namespace {
 template <int kCl>
 int configure_tc64()
 {
-    static bool configured = false;                                // one flag per instantiation
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc64_kernel<kCl>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return record_cuda_error(e, "attention kernel attribute");
-        configured = true;
-    }
+    static std::atomic<unsigned long long> configured{0};          // per instantiation, one bit per device
+    cudaError_t e = ensure_dynamic_smem(attn_tc64_kernel<kCl>, kSmemBytes, configured);
+    if (e != cudaSuccess) return record_cuda_error(e, "attention kernel attribute");
     return NM_OK;
 }
 // Clusters of kCl CTAs of this kernel that the device holds at once (clusters do not straddle GPCs, so this is

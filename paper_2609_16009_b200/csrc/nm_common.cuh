@@ -1,5 +1,6 @@
 // Shared device/host helpers for the nm kernels (sm_100a only).
 #pragma once
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 
@@ -9,6 +10,7 @@
 #include <stddef.h>
 
 #include "../../include/nm.h"
+#include "../../include/nm_debug.h"
 
 #if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ < 1000)
 #error "nm kernels are written for sm_100a"
@@ -99,8 +101,29 @@ int matmul_enqueue(const void *A, const void *B, void *C, int M, int N, int K, i
                    bool programmatic_launch = false, unsigned long long *trace = nullptr, const struct VecTail *tail = nullptr,
                    bool *tail_taken = nullptr, bool chained = false, MatmulExtras *extras = nullptr);
 
+// A plan (tile width, k-splits, ring depth; zeros = planner) forced for the CALLING THREAD's next products only; it
+// overrides the process-wide nm_debug_set_plan / nm_debug_set_kernel values while active.  The decode step uses it to
+// force one of its products without touching what other host threads see.
+void set_thread_plan_override(bool active, int tile_n, int nsplit, int stages);
+
 // How the row-major bf16 product K x N (H heads) at this M will be split: k-rows per split and splits.
 void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit, bool chained = false);
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) is a per-device setting: remember per launch site which devices
+// have it (one bit per device ordinal), so that a process using several GPUs configures the kernel on each of them.
+// Two threads racing on the first call both set the (idempotent) attribute.
+template <typename Kern>
+cudaError_t ensure_dynamic_smem(Kern kern, int bytes, std::atomic<unsigned long long> &done_mask)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = (dev >= 0 && dev < 64) ? (1ull << dev) : 0ull;
+    if (bit && (done_mask.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && bit) done_mask.fetch_or(bit, std::memory_order_release);
+    return e;
+}
 
 __host__ __device__ constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
 

@@ -2,6 +2,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "nm_matmul_kernels.cuh"
 #include "nm_row_tma.cuh"
@@ -32,12 +33,36 @@ int record_cuda_error(cudaError_t e, const char *where)
 }
 
 // ---- default workspace and tuning overrides ----------------------------------------------------------
-static void *g_ws = nullptr;
-static size_t g_ws_bytes = 0;
-static int g_force_tn = 0, g_force_split = 0, g_force_kind = -1, g_force_stages = 0;
-static int g_cluster_split = 1;     // k-splits of a tile as a thread-block cluster when the plan allows
-static int g_use_pdl = 0;
-static int g_tc_min_m = 3;        // row-major bf16 products with M >= this (and >= 32 MB of weights) go to the swap-AB tensor-core kernel
+// Process-wide settings (nm_set_*, nm_debug_set_*), guarded by a mutex.  Every entry point copies them once at its
+// start into a per-thread snapshot and plans from that copy alone, so a setter running on another host thread never
+// yields a plan mixed from two settings (a tile width from one, a split count from the other).
+struct MatmulTuning {
+    void *ws = nullptr;             // default workspace of nm_matmul / nm_matmul_batched
+    size_t ws_bytes = 0;
+    int force_tn = 0, force_split = 0, force_kind = -1, force_stages = 0;
+    int cluster_split = 1;          // k-splits of a tile as a thread-block cluster when the plan allows
+    int use_pdl = 0;
+    int tc_min_m = 3;               // row-major bf16 products with M >= this (and >= 32 MB of weights) go to the swap-AB tensor-core kernel
+};
+static std::mutex g_tuning_mutex;
+static MatmulTuning g_tuning_shared;
+struct PlanOverride { bool active = false; int tn = 0, split = 0, stages = 0; };
+static thread_local PlanOverride g_plan_override;      // a plan forced for this thread's next products only
+static thread_local MatmulTuning g_t;                  // the calling thread's snapshot
+
+static void refresh_tuning()
+{
+    {
+        std::lock_guard<std::mutex> lock(g_tuning_mutex);
+        g_t = g_tuning_shared;
+    }
+    if (g_plan_override.active) { g_t.force_tn = g_plan_override.tn; g_t.force_split = g_plan_override.split; g_t.force_stages = g_plan_override.stages; }
+}
+
+void set_thread_plan_override(bool active, int tile_n, int nsplit, int stages)
+{
+    g_plan_override.active = active; g_plan_override.tn = tile_n; g_plan_override.split = nsplit; g_plan_override.stages = stages;
+}
 
 enum PlanKind { kRowVec = 0, kColVec = 1, kGeneric = 2, kRowTma = 3, kRowTc = 4 };
 
@@ -71,13 +96,13 @@ static Plan make_tma_plan(int M, int N, int K, int H, bool chained = false)
     // SM).  Measured 4-10 % faster than two smaller CTAs per SM on every shape of 50-260 MB tried (6.2-6.5 TB/s),
     // provided the tiles fill most of the machine: at M = 2 a CTA is also bound by its own FMA rate, and 112
     // CTAs were too few.
-    if (M <= 2 && H == 1 && g_force_tn == 0 && g_force_split == 0 && 2.0 * K * N >= 48e6 && K >= 4096) {
+    if (M <= 2 && H == 1 && g_t.force_tn == 0 && g_t.force_split == 0 && 2.0 * K * N >= 48e6 && K >= 4096) {
         for (int t = 64; t <= 256; t *= 2) {
             const int tiles = ceil_div(N, t);
             if (tiles <= kSMs && tiles >= (M == 1 ? 100 : 120)) {
                 const int kt1 = (kTmaConsumers / (t / 8)) * 4;
                 p.tn = t; p.tpr = t / 8; p.rg = kTmaConsumers / p.tpr; p.nsplit = 1; p.kr = ceil_div(K, kt1) * kt1; p.ntiles = tiles;
-                p.nstage = g_force_stages > 0 ? (g_force_stages < 2 ? 2 : (g_force_stages > 11 ? 11 : g_force_stages)) : 8;
+                p.nstage = g_t.force_stages > 0 ? (g_t.force_stages < 2 ? 2 : (g_t.force_stages > 11 ? 11 : g_t.force_stages)) : 8;
                 return p;
             }
         }
@@ -85,7 +110,7 @@ static Plan make_tma_plan(int M, int N, int K, int H, bool chained = false)
     int tn = 64;
     const long tile_cap = (M > 8) ? kSMs : 2 * kSMs;   // a single wave of resident CTAs (two per SM, one when M > 8)
     while ((long)ceil_div(N, tn) * H > tile_cap && tn < 256) tn *= 2;
-    if (g_force_tn == 64 || g_force_tn == 128 || g_force_tn == 256) tn = g_force_tn;
+    if (g_t.force_tn == 64 || g_t.force_tn == 128 || g_t.force_tn == 256) tn = g_t.force_tn;
     const int tpr = tn / 8;
     const int kt = (kTmaConsumers / tpr) * 4;
     const int ntiles = ceil_div(N, tn);
@@ -97,18 +122,18 @@ static Plan make_tma_plan(int M, int N, int K, int H, bool chained = false)
     if (ns > K / (40 * M)) ns = K / (40 * M);          // partial sums stay below ~10 % of the weight bytes
     // Up to eight splits meet inside a thread-block cluster (shared memory, no fence / counter / gather through L2);
     // measured on the 7168 x 576 product: 8 splits that way 5.4 us, the 14 this rule would take otherwise 7.3 us.
-    if (g_cluster_split && M <= 8 && ns > 8) ns = 8;
-    if (g_force_split > 0) ns = g_force_split;
+    if (g_t.cluster_split && M <= 8 && ns > 8) ns = 8;
+    if (g_t.force_split > 0) ns = g_t.force_split;
     if (ns > kMaxSplit) ns = kMaxSplit;
     if (ns < 1) ns = 1;
     if (base > kNumCounters) ns = 1;
     int kr = ceil_div(ceil_div(K, ns), kt) * kt;
-    if (g_force_split > 0) kr = ceil_div(ceil_div(K, ns), 8) * 8;      // forced plans keep the requested split count
+    if (g_t.force_split > 0) kr = ceil_div(ceil_div(K, ns), 8) * 8;      // forced plans keep the requested split count
     ns = ceil_div(K, kr);
     p.tn = tn; p.tpr = tpr; p.rg = kTmaConsumers / tpr; p.nsplit = ns; p.kr = kr; p.ntiles = ntiles;
     const long ctas = base * ns;
     int nstage = (M > 8) ? 10 : (ctas > 2 * kSMs ? 3 : 5);
-    if (chained && M <= 2 && g_force_split == 0 && g_force_tn == 0) {
+    if (chained && M <= 2 && g_t.force_split == 0 && g_t.force_tn == 0) {
         // Launched programmatically inside a chain of kernels (the decode step): the CTAs are resident, and fill
         // their rings, while the previous kernel drains, so a deep ring is prefetch for free; and every split-K
         // gather at the end is a dependent round trip through L2 on the chain's critical path.  Measured in the
@@ -123,7 +148,7 @@ static Plan make_tma_plan(int M, int N, int K, int H, bool chained = false)
             nstage = 8;
         }
     }
-    if (g_force_stages > 0) nstage = g_force_stages;
+    if (g_t.force_stages > 0) nstage = g_t.force_stages;
     if (nstage < 2) nstage = 2;
     if (nstage > 11) nstage = 11;
     p.nstage = nstage;
@@ -149,11 +174,11 @@ static Plan make_tc_plan(int M, int N, int K, int H, bool col_major = false, boo
     // eight, 26 of five, 45 of three with one CTA per SM).  Take the largest split count whose clusters fit.
     // On matrices of 100 MB and more the streaming time dominates and fewer CTAs cost more than the gather saves
     // (235 MB at M = 16: 43.0 us as 168 CTAs through the workspace, 44.9 us as 56 clusters of two): no reduction there.
-    if (g_cluster_split && g_force_split == 0 && ns >= 2 && 2.0 * K * N * H < 100e6 && M <= NM_MAX_M) {
+    if (g_t.cluster_split && g_t.force_split == 0 && ns >= 2 && 2.0 * K * N * H < 100e6 && M <= NM_MAX_M) {
         for (int c = ns < 8 ? ns : 8; c >= 2; --c)
             if (base <= row_tc_max_clusters(c, 5, M, col_major, f32_out)) { ns = c; break; }
     }
-    if (g_force_split > 0) ns = g_force_split;
+    if (g_t.force_split > 0) ns = g_t.force_split;
     if (ns > kMaxSplit) ns = kMaxSplit;
     if (ns < 1) ns = 1;
     if (base > kNumCounters) ns = 1;
@@ -165,7 +190,7 @@ static Plan make_tc_plan(int M, int N, int K, int H, bool col_major = false, boo
     if (M > 16 && base * p.nsplit > kSMs) nstage = (M > 32) ? 4 : 5;      // 24 / 20 KB stages: two CTAs still share an SM
     const int its = ceil_div(kr, kTcKT);                // a ring deeper than the CTA's k-range only costs shared memory
     if (nstage > its) nstage = its;
-    if (g_force_stages > 0) nstage = g_force_stages;
+    if (g_t.force_stages > 0) nstage = g_t.force_stages;
     if (nstage < 2) nstage = 2;
     if (nstage > 10) nstage = 10;
     p.nstage = nstage;
@@ -199,10 +224,10 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     const double wbytes = 2.0 * K * N * H;
     // Column-major weights: the CUDA-core column kernel is already behind at M = 2 from about 50 MB on (17 vs 14 us
     // on 75 MB).
-    const int min_m = (layout == NM_COL_MAJOR && g_tc_min_m > 2 && g_tc_min_m <= NM_MAX_M) ? 2 : g_tc_min_m;
+    const int min_m = (layout == NM_COL_MAJOR && g_t.tc_min_m > 2 && g_t.tc_min_m <= NM_MAX_M) ? 2 : g_t.tc_min_m;
     // More than 16 tokens (up to 64): only the tensor-core kernel takes them, whatever the size of the matrix
-    const bool tc_pays = M > NM_MAX_M || (M >= min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6)) && (M >= g_tc_min_m || wbytes >= 48e6));
-    if (tma_ok && (M > NM_MAX_M || (g_force_kind != kRowTma && (layout == NM_ROW_MAJOR || g_force_kind != kRowVec))) && (tc_pays || g_force_kind == kRowTc))
+    const bool tc_pays = M > NM_MAX_M || (M >= min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6)) && (M >= g_t.tc_min_m || wbytes >= 48e6));
+    if (tma_ok && (M > NM_MAX_M || (g_t.force_kind != kRowTma && (layout == NM_ROW_MAJOR || g_t.force_kind != kRowVec))) && (tc_pays || g_t.force_kind == kRowTc))
         return make_tc_plan(M, N, K, H, layout == NM_COL_MAJOR, dtype == NM_BF16_F32OUT);
     if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H, chained);
     const int target = 192;                           // CTAs wanted in total (measured: 144-240 is the flat optimum)
@@ -213,7 +238,7 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
         const int chunks = N / V;
         if (chunks >= 32 * 64) tpr = 32;
         else if (chunks >= 16 * 24) tpr = 16;
-        if (g_force_tn > 0) tpr = g_force_tn / V;
+        if (g_t.force_tn > 0) tpr = g_t.force_tn / V;
         if (tpr < 1) tpr = 1;
         if (tpr > kThreads) tpr = kThreads;
         p.tpr = tpr;
@@ -233,8 +258,8 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     const int min_kr = (p.kind == kRowVec) ? 2 * p.rg : 512;
     if (nsplit > K / min_kr) nsplit = K / min_kr;
     if (nsplit > K / (40 * M)) nsplit = K / (40 * M);
-    if (g_cluster_split && M <= 8 && nsplit > 8 && 8L * M * p.tn <= kClusterSlotFloats) nsplit = 8;     // the most that meet inside a cluster
-    if (g_force_split > 0) nsplit = g_force_split;
+    if (g_t.cluster_split && M <= 8 && nsplit > 8 && 8L * M * p.tn <= kClusterSlotFloats) nsplit = 8;     // the most that meet inside a cluster
+    if (g_t.force_split > 0) nsplit = g_t.force_split;
     if (nsplit > kMaxSplit) nsplit = kMaxSplit;
     if (nsplit < 1) nsplit = 1;
     if ((long)p.ntiles * H > kNumCounters) nsplit = 1;
@@ -334,6 +359,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
                        unsigned long long *trace = nullptr, const VecTail *tail = nullptr, bool *tail_taken = nullptr, bool chained = false,
                        MatmulExtras *extras = nullptr)
 {
+    refresh_tuning();
     if (tail_taken) *tail_taken = false;
     if (extras) { extras->tile_ss_taken = extras->norm_taken = false; extras->tile_n = 0; }
     int rc = check_common(A, B, C, M, N, K, H, dtype, layout);
@@ -350,7 +376,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     // tensor maps: 16-byte aligned operands and strides, bf16.  Row-major B may take the TMA ring kernel or the
     // tensor-core kernel; column-major B only the latter (its CUDA-core path is the plain column kernel).
     bool tma_ok = b_ok && a_ok && dtype != NM_F32 && tensor_map_encoder() != nullptr && (long)N * 2 < (1L << 40) && strideB >= 0;
-    if (g_force_kind == kRowVec && layout != NM_FRACTAL_NZ) tma_ok = false;      // the fractal storage has one kernel: nothing to force
+    if (g_t.force_kind == kRowVec && layout != NM_FRACTAL_NZ) tma_ok = false;      // the fractal storage has one kernel: nothing to force
     if (layout == NM_FRACTAL_NZ && !tma_ok) return NM_ERR_UNSUPPORTED;      // unaligned operands or no tensor-map encoder
     Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok, chained);
     // Copies, not pointers into the map cache: the second lookup may evict the entry the first one returned
@@ -386,15 +412,15 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     }
 
     if (extras && extras->dry_run && p.kind != kRowTma) return NM_OK;
-    if ((p.kind == kRowVec || p.kind == kColVec) && g_cluster_split && p.nsplit >= 2 && p.nsplit <= 8 &&
+    if ((p.kind == kRowVec || p.kind == kColVec) && g_t.cluster_split && p.nsplit >= 2 && p.nsplit <= 8 &&
         (long)p.nsplit * M * p.tn <= kClusterSlotFloats)
         a.cluster_split = 1;
     cudaError_t e = cudaErrorInvalidValue;
     if (p.kind == kRowTc) {
         const CUtensorMap *mb = tc_map_b, *ma = tc_map_a;
         TmaArgs ta{};
-        ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
-        if (g_cluster_split && p.nsplit >= 2 && p.nsplit <= 8 && (size_t)p.nsplit * M * kTcTN * sizeof(float) <= 65536) ta.cluster_split = 1;
+        ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_t.use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
+        if (g_t.cluster_split && p.nsplit >= 2 && p.nsplit <= 8 && (size_t)p.nsplit * M * kTcTN * sizeof(float) <= 65536) ta.cluster_split = 1;
         const bool col = layout == NM_COL_MAJOR;
         e = (dtype == NM_BF16_F32OUT) ? launch_row_tc<float>(*mb, *ma, ta, stream, col) : launch_row_tc<bf16_t>(*mb, *ma, ta, stream, col);
     } else if (p.kind == kRowTma) {
@@ -404,7 +430,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         if (!map) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
         TmaArgs ta{};
         ta.fractal_nz = (layout == NM_FRACTAL_NZ) ? 1 : 0;
-        ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
+        ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_t.use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
         ta.trace = trace;
         if (tail && tail->enabled && M == 1 && dtype == NM_BF16 && H == 1 && ws && ws_bytes >= kCounterBytes && aligned16(ws) &&
             p.ntiles < kNumCounters - 1 && N <= 4096 && N % 4 == 0 && p.tn % 4 == 0 && ldc % 4 == 0 && ((uintptr_t)C & 7u) == 0) {
@@ -416,7 +442,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         // Split-K inside a cluster: up to eight splits (the portable cluster size) whose partial tiles fit 16 KB of
         // the first CTA's shared memory meet there instead of in the workspace.
         const size_t slot_bytes = (size_t)p.nsplit * M * p.tn * sizeof(float);
-        if (g_cluster_split && p.nsplit >= 2 && p.nsplit <= 8 && !ta.tail.enabled && slot_bytes <= 16384) {
+        if (g_t.cluster_split && p.nsplit >= 2 && p.nsplit <= 8 && !ta.tail.enabled && slot_bytes <= 16384) {
             ta.cluster_split = 1;
             smem += 16 + slot_bytes;
         }
@@ -461,6 +487,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
 
 void matmul_row_major_split(int M, int N, int K, int H, int *k_rows_per_split, int *nsplit, bool chained)
 {
+    refresh_tuning();
     const Plan p = make_plan(M, N, K, H, NM_BF16, NM_ROW_MAJOR, true, true, chained);      // whichever kernel the product will take
     *k_rows_per_split = p.kr;
     *nsplit = p.nsplit;
@@ -521,17 +548,20 @@ int nm_workspace_init(void *workspace, size_t bytes, nm_stream stream)
 
 int nm_set_workspace(void *workspace, size_t bytes)
 {
-    if (!workspace) { g_ws = nullptr; g_ws_bytes = 0; return NM_OK; }
-    if (bytes < kCounterBytes) return NM_ERR_WORKSPACE;
-    NM_CUDA_TRY(cudaMemset(workspace, 0, kCounterBytes));
-    g_ws = workspace; g_ws_bytes = bytes;
+    if (workspace) {
+        if (bytes < kCounterBytes) return NM_ERR_WORKSPACE;
+        NM_CUDA_TRY(cudaMemset(workspace, 0, kCounterBytes));
+    }
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    g_tuning_shared.ws = workspace; g_tuning_shared.ws_bytes = workspace ? bytes : 0;
     return NM_OK;
 }
 
 int nm_matmul(const void *A, const void *B, void *C, int M, int N, int K,
               nm_dtype dtype, nm_layout layout_B, nm_stream stream)
 {
-    return matmul_impl(A, B, C, M, N, K, 1, K, 0, 0, N, 0, dtype, layout_B, g_ws, g_ws_bytes, (cudaStream_t)stream);
+    refresh_tuning();
+    return matmul_impl(A, B, C, M, N, K, 1, K, 0, 0, N, 0, dtype, layout_B, g_t.ws, g_t.ws_bytes, (cudaStream_t)stream);
 }
 
 int nm_matmul_ws(const void *A, const void *B, void *C, int M, int N, int K,
@@ -544,7 +574,8 @@ int nm_matmul_batched(const void *A, const void *B, void *C, int M, int N, int K
                       long lda, long strideA, long strideB, long ldc, long strideC,
                       nm_dtype dtype, nm_layout layout_B, nm_stream stream)
 {
-    return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout_B, g_ws, g_ws_bytes, (cudaStream_t)stream);
+    refresh_tuning();
+    return matmul_impl(A, B, C, M, N, K, H, lda, strideA, strideB, ldc, strideC, dtype, layout_B, g_t.ws, g_t.ws_bytes, (cudaStream_t)stream);
 }
 
 int nm_matmul_batched_ws(const void *A, const void *B, void *C, int M, int N, int K, int H,
@@ -575,13 +606,15 @@ int nm_matmul_host(const void *A_host, const void *B, void *C_host, void *A_stag
 int nm_debug_set_plan(int tile_n, int nsplit)
 {
     if (tile_n < 0 || nsplit < 0 || tile_n > kMaxTileN || nsplit > kMaxSplit) return NM_ERR_INVALID_ARG;
-    g_force_tn = tile_n; g_force_split = nsplit;
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    g_tuning_shared.force_tn = tile_n; g_tuning_shared.force_split = nsplit;
     return NM_OK;
 }
 
 int nm_debug_set_cluster_split(int enable)
 {
-    g_cluster_split = enable ? 1 : 0;
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    g_tuning_shared.cluster_split = enable ? 1 : 0;
     return NM_OK;
 }
 
@@ -589,20 +622,23 @@ int nm_debug_set_cluster_split(int enable)
 int nm_set_tensor_core_min_m(int m)
 {
     if (m < 1 || m > NM_MAX_M + 1) return NM_ERR_INVALID_ARG;
-    g_tc_min_m = m;
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    g_tuning_shared.tc_min_m = m;
     return NM_OK;
 }
 
 /* Force the kernel family (-1 heuristic, 0 plain row-major kernel instead of the TMA ring) and the ring depth. */
 int nm_debug_set_kernel(int kind, int stages)
 {
-    g_force_kind = kind; g_force_stages = stages;
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    g_tuning_shared.force_kind = kind; g_tuning_shared.force_stages = stages;
     return NM_OK;
 }
 
 int nm_set_programmatic_launch(int enable)
 {
-    g_use_pdl = enable ? 1 : 0;
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    g_tuning_shared.use_pdl = enable ? 1 : 0;
     return NM_OK;
 }
 
@@ -610,8 +646,9 @@ int nm_set_programmatic_launch(int enable)
 int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout_B, int vec_ok, int *out)
 {
     if (!out) return NM_ERR_INVALID_ARG;
+    refresh_tuning();
     Plan p = make_plan(M, N, K, H, dtype, layout_B, vec_ok != 0,
-                       vec_ok != 0 && dtype != NM_F32 && g_force_kind != kRowVec);
+                       vec_ok != 0 && dtype != NM_F32 && g_t.force_kind != kRowVec);
     out[0] = p.kind; out[1] = p.tn; out[2] = p.nsplit; out[3] = p.kr; out[4] = p.ntiles;
     out[5] = p.ntiles * p.nsplit * H;
     return NM_OK;

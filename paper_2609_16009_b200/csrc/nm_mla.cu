@@ -3,6 +3,7 @@
 // with the tensor-core attention pass.
 #include <algorithm>
 #include <cmath>
+#include <mutex>
 
 #include "nm_async.cuh"
 #include "nm_mla.cuh"
@@ -10,13 +11,41 @@
 
 namespace nm {
 
-static int g_attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel, 2 / 3: force 128 / 64 heads per CTA
+// Tuning state of the decode step (nm_debug_set_*): process-wide and guarded by a mutex; every entry point plans from a
+// per-thread snapshot taken once at its start, so a setter on another host thread cannot change a step half way.
+struct StepTuning {
+    int attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel, 2 / 3: force 128 / 64 heads per CTA
+    int step_plan[3][3] = {};   // forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
+    int host_direct_out = 1;    // host-operand step: store the result straight into device-addressable host memory
+    int batch_tc_min_t = 3;     // batch decode: tokens from which the per-head products go to the tensor cores
+    int fused_tails = 1;        // 0: RMSNorm / RoPE / cache write as kernels of their own; 1: folded into the products (default);
+                                // 2: as 1, but only in the form where the product's last CTA runs them
+    int step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
+    int fused_heads = 1;        // per-head stages fused with their vector stage (q_finish, uv_merge) when the dims allow
+    int uv_pdl = 1;             // launch uv_merge programmatically
+    int prefetch_uv = 1;        // include W_UV in the L2 prefetch
+    int prefetch_mb = 40;       // MB of W_O pulled into L2 beside the attention pass (plus all of W_UV); 0 = off
+};
+static std::mutex g_step_mutex;
+static StepTuning g_step_shared;
+static thread_local StepTuning g_s;                   // the calling thread's snapshot
+static void refresh_step_tuning()
+{
+    std::lock_guard<std::mutex> lock(g_step_mutex);
+    g_s = g_step_shared;
+}
+template <typename F> static int set_step_tuning(F f)
+{
+    std::lock_guard<std::mutex> lock(g_step_mutex);
+    f(g_step_shared);
+    return NM_OK;
+}
 // Cache rows (over all sequences of a call) from which the 128-head kernel is the faster one: it loads every row
 // into two CTAs instead of four, which decides once a CTA has many tiles to go through; below, the 64-head
 // kernel's shorter prologue and merge win (measured: 16384 rows 94.8 vs 97.3 us per step, 65536 rows 164 vs 158)
 constexpr long kAttnWideRows = 65536;
 constexpr int kSMsAttn = 148;
-static bool attention_64_heads(long total_rows) { return g_attn_impl == 3 || (g_attn_impl != 2 && total_rows < kAttnWideRows); }
+static bool attention_64_heads(long total_rows) { return g_s.attn_impl == 3 || (g_s.attn_impl != 2 && total_rows < kAttnWideRows); }
 
 // ---- small vector kernels ---------------------------------------------------------------------------
 
@@ -313,17 +342,6 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
 
 // ---- host -------------------------------------------------------------------------------------------
 
-static int g_step_plan[3][3] = {};   // tuning: forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
-static int g_host_direct_out = 1;    // host-operand step: store the result straight into device-addressable host memory
-static int g_batch_tc_min_t = 3;     // batch decode: tokens from which the per-head products go to the tensor cores
-static int g_fused_tails = 1;        // 0: RMSNorm / RoPE / cache write as kernels of their own; 1: folded into the products (default);
-                                     // 2: as 1, but only in the form where the product's last CTA runs them
-static int g_step_pdl = 1;           // chain the kernels of the decode step with programmatic dependent launch
-static int g_fused_heads = 1;        // per-head stages fused with their vector stage (q_finish, uv_merge) when the dims allow
-static int g_uv_pdl = 1;             // tuning: launch uv_merge programmatically
-static int g_prefetch_uv = 1;        // tuning: include W_UV in the L2 prefetch
-static int g_prefetch_mb = 40;       // MB of W_O pulled into L2 beside the attention pass (plus all of W_UV); 0 = off
-
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int kv_lora)
@@ -333,7 +351,7 @@ AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int
     const int tiles = ceil_div(n_rows > 0 ? n_rows : 0, kAttnTileRows);
     // The tensor-core kernels take 128 heads and 16-byte aligned operands (TMA); both passes of an
     // attention call derive the same answer from the same arguments.
-    const bool tc_ok = g_attn_impl != 1 && H == 128 && n_rows > 0 && (((uintptr_t)Q | (uintptr_t)cache) & 15u) == 0 &&
+    const bool tc_ok = g_s.attn_impl != 1 && H == 128 && n_rows > 0 && (((uintptr_t)Q | (uintptr_t)cache) & 15u) == 0 &&
                        tensor_map_encoder() != nullptr;
     p.tensor_core = !tc_ok ? 0 : (attention_64_heads(n_rows) ? 2 : 1);
     // one wave of the 148 SMs: 64 splits x 2 column halves (128 heads per CTA), or 32 splits x 2 column halves x 2
@@ -456,8 +474,8 @@ static unsigned long long *trace_at(size_t offset) { return attention_trace() ? 
 // Tuning aid: a forced plan around one product of the step.
 struct ScopedPlan {
     bool on;
-    explicit ScopedPlan(const int (&f)[3]) : on(f[0] || f[1] || f[2]) { if (on) { nm_debug_set_plan(f[0], f[1]); nm_debug_set_kernel(-1, f[2]); } }
-    ~ScopedPlan() { if (on) { nm_debug_set_plan(0, 0); nm_debug_set_kernel(-1, 0); } }
+    explicit ScopedPlan(const int (&f)[3]) : on(f[0] || f[1] || f[2]) { if (on) set_thread_plan_override(true, f[0], f[1], f[2]); }
+    ~ScopedPlan() { if (on) set_thread_plan_override(false, 0, 0, 0); }
 };
 
 #define NM_TRY(expr) do { int _rc = (expr); if (_rc != NM_OK) return _rc; } while (0)
@@ -469,6 +487,7 @@ static thread_local StepEvents g_events;
 
 static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
 {
+    refresh_step_tuning();
     NM_TRY(check_params(p));
     const StepLayout L = step_layout(p);
     if (p->workspace_bytes < L.total) return NM_ERR_WORKSPACE;
@@ -494,7 +513,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     // start (and, for the products, prefetch its weights) while its predecessor drains; each waits
     // for the predecessor before it reads activations or writes.  The first kernel on each stream
     // keeps the ordinary dependency on whatever the caller enqueued before the step.
-    const bool pdl = g_step_pdl != 0;
+    const bool pdl = g_s.step_pdl != 0;
 #define NM_LAUNCH(kern, grid, block, stream, ...)                                             \
     do {                                                                                      \
         cudaError_t _e = launch_pdl(kern, dim3(grid), dim3(block), stream, pdl, __VA_ARGS__); \
@@ -504,7 +523,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     // The vector stages behind the down-projections (RMSNorm of the query latent; RMSNorm, RoPE and the cache-row
     // write of the KV part) run inside the product that feeds them, in the CTA that completes its last tile,
     // when that product is the TMA ring kernel; otherwise as kernels of their own.
-    const bool tails_ok = g_fused_tails && down_finish_applies(ql, dc, dr);
+    const bool tails_ok = g_s.fused_tails && down_finish_applies(ql, dc, dr);
     VecTail tq{}, tkv{};
     tq.enabled = 1; tq.q_lora = ql; tq.eps = p->rms_eps; tq.gamma_q = (const uint16_t *)p->gamma_q; tq.c_qn = c_qn;
     tkv.enabled = 1; tkv.kv_off = 0; tkv.dc = dc; tkv.rope = dr; tkv.eps = p->rms_eps; tkv.gamma_kv = (const uint16_t *)p->gamma_kv;
@@ -519,12 +538,12 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     RowNorm rn{};
     KvFinish kvf{};
     float *tile_ss = reinterpret_cast<float *>(ws + L.tile_ss);
-    if (fused_down && tails_ok && g_fused_tails == 1 && g_fused_heads && head_kernels_apply(H, dn, dr, dc, dv)) {
+    if (fused_down && tails_ok && g_s.fused_tails == 1 && g_s.fused_heads && head_kernels_apply(H, dn, dr, dc, dv)) {
         uint16_t *x_down = reinterpret_cast<uint16_t *>(ws + L.x_down);
         MatmulExtras ex_d, ex_u;
         ex_d.tile_ss = tile_ss; ex_d.dry_run = true;
         {
-            ScopedPlan sp(g_step_plan[0]);
+            ScopedPlan sp(g_s.step_plan[0]);
             NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws,
                                   L.main_ws_bytes, ms, false, nullptr, nullptr, nullptr, true, &ex_d));
         }
@@ -532,7 +551,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
             rn.enabled = 1; rn.n = ql; rn.ntiles = ql / ex_d.tile_n; rn.eps = p->rms_eps; rn.tile_ss = tile_ss;
             rn.gamma = (const uint16_t *)p->gamma_q; rn.normed_out = c_qn;
             ex_u.norm = &rn; ex_u.dry_run = true;
-            ScopedPlan sp(g_step_plan[1]);
+            ScopedPlan sp(g_s.step_plan[1]);
             NM_TRY(matmul_enqueue(x_down, p->W_UQR, q, 1, H * dq, ql, 1, ql, 0, 0, H * dq, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms, false,
                                   nullptr, nullptr, nullptr, true, &ex_u));
             split_norm = ex_u.norm_taken;
@@ -543,7 +562,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         MatmulExtras ex_d;
         ex_d.tile_ss = tile_ss;
         {
-            ScopedPlan sp(g_step_plan[0]);
+            ScopedPlan sp(g_s.step_plan[0]);
             NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws,
                                   L.main_ws_bytes, ms, pdl && p->programmatic_entry, trace_at(2048), nullptr, nullptr, true, &ex_d));
         }
@@ -558,7 +577,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         uint16_t *x_down = reinterpret_cast<uint16_t *>(ws + L.x_down);
         VecTail both = tq;
         both.kv_off = ql; both.dc = dc; both.rope = dr; both.gamma_kv = tkv.gamma_kv; both.cos_sin = tkv.cos_sin; both.cache_row = tkv.cache_row;
-        ScopedPlan sp(g_step_plan[0]);
+        ScopedPlan sp(g_s.step_plan[0]);
         NM_TRY(matmul_enqueue(p->h, p->W_DQKV, x_down, 1, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws,
                               L.main_ws_bytes, ms, pdl && p->programmatic_entry, trace_at(2048), tails_ok ? &both : nullptr, &taken, true));
         if (!taken)
@@ -587,7 +606,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         if (!taken) NM_LAUNCH(rmsnorm_kernel, 1, 256, ms, (const uint16_t *)c_q, (const uint16_t *)p->gamma_q, c_qn, ql, p->rms_eps);
     }
     {
-        ScopedPlan sp(g_step_plan[1]);
+        ScopedPlan sp(g_s.step_plan[1]);
         MatmulExtras ex_u;
         ex_u.norm = &rn;
         const uint16_t *a_row = split_norm ? reinterpret_cast<const uint16_t *>(ws + L.x_down) : c_qn;
@@ -595,7 +614,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
                               nullptr, nullptr, true, split_norm ? &ex_u : nullptr));
         if (split_norm && !ex_u.norm_taken) return NM_ERR_UNSUPPORTED;
     }
-    const bool fused = g_fused_heads && head_kernels_apply(H, dn, dr, dc, dv);
+    const bool fused = g_s.fused_heads && head_kernels_apply(H, dn, dr, dc, dv);
     if (fused) {
         // RoPE of the rope part and q_lat[h] = q[h, :nope] * W_UK[h] in one kernel, one CTA per head
         NM_TRY(launch_q_finish(q, p->W_UK, p->rope_cos_sin, q_full, H, dr, ms, pdl, kvf));
@@ -611,17 +630,17 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     //      output-side products start from L2 instead of HBM (Data Independence: the weights do not depend on
     //      the attention result) ---------------------------------------------------------------------------------
     L2Prefetch pf{};
-    if (g_prefetch_mb > 0 && pos > 0) {
+    if (g_s.prefetch_mb > 0 && pos > 0) {
         pf.block = (const char *)p->W_UV;
-        pf.block_bytes = g_prefetch_uv ? (long)H * dc * dv * 2 : 0;
+        pf.block_bytes = g_s.prefetch_uv ? (long)H * dc * dv * 2 : 0;
         if (p->W_O && lay == NM_ROW_MAJOR) {
             int kr = 0, ns = 1;
             {
-                ScopedPlan sp(g_step_plan[2]);
+                ScopedPlan sp(g_s.step_plan[2]);
                 matmul_row_major_split(1, d, H * dv, 1, &kr, &ns, true);
             }
             const long row_bytes = (long)d * 2;
-            long rows = ((long)g_prefetch_mb << 20) / ns / row_bytes;
+            long rows = ((long)g_s.prefetch_mb << 20) / ns / row_bytes;
             if (rows > kr) rows = kr;
             pf.base = (const char *)p->W_O; pf.range_stride = (long)kr * row_bytes; pf.nranges = rows > 0 ? ns : 0;
             pf.range_bytes = rows * row_bytes;
@@ -629,7 +648,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
             // fractal storage: every fractal column (16 columns, all K rows) is contiguous; the product starts each of
             // them at row 0, so the head of every fractal column is what it reads first
             const long K_o = (long)H * dv, cols = d / 16;
-            long rows = (((long)g_prefetch_mb << 20) / cols / 32) / 16 * 16;
+            long rows = (((long)g_s.prefetch_mb << 20) / cols / 32) / 16 * 16;
             if (rows > K_o) rows = K_o;
             pf.base = (const char *)p->W_O; pf.range_stride = K_o * 32; pf.nranges = rows > 0 ? (int)cols : 0;
             pf.range_bytes = rows * 32;
@@ -640,7 +659,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     // When the merge kernel is launched programmatically it sits beside the attention CTAs from their start and
     // issues the prefetch itself (its threads are idle until the attention result exists); otherwise a warp of
     // the attention kernel does.
-    const bool uv_early = fused && pdl && !forked && g_uv_pdl;
+    const bool uv_early = fused && pdl && !forked && g_s.uv_pdl;
     NM_TRY(attention_partial(q_full, cache, H, (int)pos, dc, dr, p->softmax_scale, aws, L.attn_bytes, ms, pdl, uv_early ? L2Prefetch{} : pf));
     // The merge needs the cache row the KV chain wrote (two-stream schedule): the join sits right before it, where
     // it breaks only the merge's programmatic launch.
@@ -658,7 +677,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     }
     if (p->W_O) {
         if (p->event_before_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_before_wo, ms));
-        ScopedPlan sp(g_step_plan[2]);
+        ScopedPlan sp(g_s.step_plan[2]);
         NM_TRY(matmul_enqueue(o, p->W_O, p->out, 1, d, H * dv, 1, (long)H * dv, 0, 0, d, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms,
                               pdl && !p->event_before_wo, trace_at(6144), nullptr, nullptr, true));
         if (p->event_after_wo) NM_CUDA_TRY(cudaEventRecord((cudaEvent_t)p->event_after_wo, ms));
@@ -718,6 +737,7 @@ static int batch_check(const nm_mla_params *p, const nm_mla_batch *b)
 
 static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_t ms)
 {
+    refresh_step_tuning();
     NM_TRY(batch_check(p, b));
     const int T = b->T;
     const BatchLayout L = batch_layout(p, T);
@@ -731,7 +751,7 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     uint16_t *q_full = (uint16_t *)(ws + L.q_full), *o_lat = (uint16_t *)(ws + L.o_lat), *o = (uint16_t *)(ws + L.o);
     uint16_t *cache = static_cast<uint16_t *>(b->kv_cache);
     void *mws = ws + L.mws;
-    const bool pdl = g_step_pdl != 0;
+    const bool pdl = g_s.step_pdl != 0;
 
     // split plan of the attention pass: the same number of splits for every sequence, about 128 CTAs in all
     long total_rows = 0;
@@ -799,7 +819,7 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     // tensor-core kernel, with RoPE and the merge as small kernels of their own: in the fused per-head kernels one
     // CTA per head walks every token and is bound by fp32 FMA issue and by its chain of L2 round trips (measured at
     // 4096 rows: 108 vs 112 us at T = 3, 114 vs 115 at T = 4, 133 vs 139 at T = 6, 183 vs 204 at T = 16; level at T = 2).
-    const bool per_head_tc = T >= g_batch_tc_min_t || !g_fused_heads;
+    const bool per_head_tc = T >= g_s.batch_tc_min_t || !g_s.fused_heads;
     if (per_head_tc) {
         NM_TRY(launch_rope_batch(q, b->rope_cos_sin, q_full, H, dn, dc, dr, T, ms, pdl));
         NM_TRY(matmul_enqueue(q, p->W_UK, q_full, T, dc, dn, H, (long)H * dq, dq, (long)dn * dc, (long)H * dkv, dkv, NM_BF16, NM_ROW_MAJOR,
@@ -815,14 +835,14 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
         // beside the attention pass (a spare warp of its CTAs): W_UV and the head of every k-split of W_O into L2, as in
         // the single-token step
         L2Prefetch pf{};
-        if (g_prefetch_mb > 0) {
+        if (g_s.prefetch_mb > 0) {
             pf.block = (const char *)p->W_UV;
-            pf.block_bytes = g_prefetch_uv ? (long)H * dc * dv * 2 : 0;
+            pf.block_bytes = g_s.prefetch_uv ? (long)H * dc * dv * 2 : 0;
             if (p->W_O && lay == NM_ROW_MAJOR) {
                 int kr = 0, ns = 1;
                 matmul_row_major_split(T, d, H * dv, 1, &kr, &ns, true);
                 const long row_bytes = (long)d * 2;
-                long prows = ((long)g_prefetch_mb << 20) / ns / row_bytes;
+                long prows = ((long)g_s.prefetch_mb << 20) / ns / row_bytes;
                 if (prows > kr) prows = kr;
                 pf.base = (const char *)p->W_O; pf.range_stride = (long)kr * row_bytes; pf.nranges = prows > 0 ? ns : 0;
                 pf.range_bytes = prows * row_bytes;
@@ -846,6 +866,11 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     if (b->o_lat) NM_CUDA_TRY(cudaMemcpyAsync(b->o_lat, o_lat, (size_t)T * H * dc * 2, cudaMemcpyDeviceToDevice, ms));
     if (b->o) NM_CUDA_TRY(cudaMemcpyAsync(b->o, o, (size_t)T * H * dv * 2, cudaMemcpyDeviceToDevice, ms));
     if (b->q_full) NM_CUDA_TRY(cudaMemcpyAsync(b->q_full, q_full, (size_t)T * H * dkv * 2, cudaMemcpyDeviceToDevice, ms));
+    // stage outputs of the query side and the raw KV product, token by token out of the [T][q_lora + kv_lora + rope] rows
+    if (b->c_q) NM_CUDA_TRY(cudaMemcpy2DAsync(b->c_q, (size_t)ql * 2, x_down, (size_t)(ql + dkv) * 2, (size_t)ql * 2, T, cudaMemcpyDeviceToDevice, ms));
+    if (b->ckr) NM_CUDA_TRY(cudaMemcpy2DAsync(b->ckr, (size_t)dkv * 2, x_down + ql, (size_t)(ql + dkv) * 2, (size_t)dkv * 2, T, cudaMemcpyDeviceToDevice, ms));
+    if (b->c_qn) NM_CUDA_TRY(cudaMemcpyAsync(b->c_qn, c_qn, (size_t)T * ql * 2, cudaMemcpyDeviceToDevice, ms));
+    if (b->q) NM_CUDA_TRY(cudaMemcpyAsync(b->q, q, (size_t)T * H * dq * 2, cudaMemcpyDeviceToDevice, ms));
     return NM_OK;
 }
 
@@ -893,12 +918,14 @@ size_t nm_mla_attention_workspace_bytes(int H, int n_rows, int kv_lora)
 int nm_mla_attention_partial(const void *Q, const void *kv_cache, int H, int n_rows, int kv_lora, int rope, float scale,
                              void *workspace, size_t workspace_bytes, nm_stream stream)
 {
+    refresh_step_tuning();
     return attention_partial(Q, kv_cache, H, n_rows, kv_lora, rope, scale, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
 int nm_mla_attention_combine(const void *Q, const void *kv_cache, void *o_bf16, float *o_f32, int H, int n_rows, long extra_row,
                              int kv_lora, int rope, float scale, void *workspace, size_t workspace_bytes, nm_stream stream)
 {
+    refresh_step_tuning();
     return attention_combine(Q, kv_cache, o_bf16, o_f32, H, n_rows, extra_row, kv_lora, rope, scale, workspace, workspace_bytes,
                              (cudaStream_t)stream);
 }
@@ -906,6 +933,7 @@ int nm_mla_attention_combine(const void *Q, const void *kv_cache, void *o_bf16, 
 int nm_mla_attention(const void *Q, const void *kv_cache, void *o_bf16, float *o_f32, int H, int n_rows, long extra_row,
                      int kv_lora, int rope, float scale, void *workspace, size_t workspace_bytes, nm_stream stream)
 {
+    refresh_step_tuning();
     NM_TRY(attention_partial(Q, kv_cache, H, n_rows, kv_lora, rope, scale, workspace, workspace_bytes, (cudaStream_t)stream));
     return attention_combine(Q, kv_cache, o_bf16, o_f32, H, n_rows, extra_row, kv_lora, rope, scale, workspace, workspace_bytes,
                              (cudaStream_t)stream);
@@ -938,7 +966,7 @@ int nm_mla_decode_batch(const nm_mla_params *p, const nm_mla_batch *b, nm_stream
         q.seq_len = b->seq_lens[0];
         q.h = b->h; q.rope_cos_sin = b->rope_cos_sin; q.kv_cache = b->kv_cache; q.out = b->out;
         q.q_full = b->q_full; q.o_lat = b->o_lat; q.o = b->o;
-        q.c_q = nullptr; q.c_qn = nullptr; q.q = nullptr; q.ckr = nullptr; q.o_lat_f32 = nullptr;
+        q.c_q = b->c_q; q.c_qn = b->c_qn; q.q = b->q; q.ckr = b->ckr; q.o_lat_f32 = nullptr;
         q.event_before_wo = nullptr; q.event_after_wo = nullptr; q.programmatic_entry = 0;
         if (!q.W_O) q.out = nullptr;
         return step_impl(&q, (cudaStream_t)main_stream, (cudaStream_t)main_stream);
@@ -954,6 +982,7 @@ int nm_mla_decode_step(const nm_mla_params *p, nm_stream main_stream, nm_stream 
 int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *out_host, void *h_staging, void *out_staging,
                             nm_stream main_stream, nm_stream side_stream)
 {
+    refresh_step_tuning();
     if (!p || !h_host || !out_host || !h_staging || !out_staging || !p->W_O) return NM_ERR_INVALID_ARG;
     nm_mla_params q = *p;
     q.h = h_staging;
@@ -962,7 +991,7 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     // into it - still a device-to-host transfer, but without a copy operation (and its scheduling gap) after the
     // last kernel.  The token row keeps its copy: 132 CTAs reading it over the host link would cost more.
     void *out_direct = nullptr;
-    if (g_host_direct_out) {
+    if (g_s.host_direct_out) {
         cudaPointerAttributes attr;
         if (cudaPointerGetAttributes(&attr, out_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
             ((uintptr_t)attr.devicePointer & 15u) == 0)
@@ -982,36 +1011,31 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
 int nm_debug_set_batch_per_head_min_tokens(int tokens)
 {
     if (tokens < 1 || tokens > kMaxBatch + 1) return NM_ERR_INVALID_ARG;
-    g_batch_tc_min_t = tokens;
-    return NM_OK;
+    return set_step_tuning([&](StepTuning &t) { t.batch_tc_min_t = tokens; });
 }
 
 int nm_debug_set_step_plan(int which, int tile_n, int nsplit, int stages)
 {
     if (which < 0 || which > 2) return NM_ERR_INVALID_ARG;
-    g_step_plan[which][0] = tile_n; g_step_plan[which][1] = nsplit; g_step_plan[which][2] = stages;
-    return NM_OK;
+    return set_step_tuning([&](StepTuning &t) { t.step_plan[which][0] = tile_n; t.step_plan[which][1] = nsplit; t.step_plan[which][2] = stages; });
 }
 
 /* 1 (default): RMSNorm / RoPE / cache-row write run inside the completion of the down-projection products; 0: as
  * kernels of their own. */
 int nm_debug_set_step_tails(int enable)
 {
-    g_fused_tails = enable < 0 ? 0 : (enable > 2 ? 2 : enable);
-    return NM_OK;
+    return set_step_tuning([&](StepTuning &t) { t.fused_tails = enable < 0 ? 0 : (enable > 2 ? 2 : enable); });
 }
 
 int nm_debug_set_step_knobs(int uv_pdl, int prefetch_uv)
 {
-    g_uv_pdl = uv_pdl ? 1 : 0; g_prefetch_uv = prefetch_uv ? 1 : 0;
-    return NM_OK;
+    return set_step_tuning([&](StepTuning &t) { t.uv_pdl = uv_pdl ? 1 : 0; t.prefetch_uv = prefetch_uv ? 1 : 0; });
 }
 
 /* 1 (default): RoPE + W_UK and merge + W_UV run as fused per-head kernels; 0: separate kernels. */
 int nm_debug_set_step_fusion(int enable)
 {
-    g_fused_heads = enable ? 1 : 0;
-    return NM_OK;
+    return set_step_tuning([&](StepTuning &t) { t.fused_heads = enable ? 1 : 0; });
 }
 
 /* Device buffer of 12 uint64 that receives phase timestamps of the attention kernel (NULL = off). */
@@ -1025,23 +1049,20 @@ int nm_debug_set_attention_trace(void *device_buffer)
 int nm_debug_set_step_prefetch(int megabytes)
 {
     if (megabytes < 0 || megabytes > 100) return NM_ERR_INVALID_ARG;
-    g_prefetch_mb = megabytes;
-    return NM_OK;
+    return set_step_tuning([&](StepTuning &t) { t.prefetch_mb = megabytes; });
 }
 
 /* Chain the kernels of the decode step with programmatic dependent launch (default on). */
 int nm_debug_set_step_pdl(int enable)
 {
-    g_step_pdl = enable ? 1 : 0;
-    return NM_OK;
+    return set_step_tuning([&](StepTuning &t) { t.step_pdl = enable ? 1 : 0; });
 }
 
 /* 0: tensor-core attention when the shape allows (default); 1: CUDA-core attention kernel; 2 / 3: the tensor-core
  * kernel with 128 / 64 heads per CTA whatever the length. */
 int nm_debug_set_attention(int impl)
 {
-    g_attn_impl = impl;
-    return NM_OK;
+    return set_step_tuning([&](StepTuning &t) { t.attn_impl = impl; });
 }
 
 #pragma GCC visibility pop

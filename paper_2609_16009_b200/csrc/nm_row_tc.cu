@@ -199,12 +199,11 @@ static cudaError_t launch_tc(const CUtensorMap &map_b, const CUtensorMap &map_a,
 {
     TmaArgs ta = ta_in;
     const MatmulArgs &a = ta.base;
-    static bool configured = false;
+    static std::atomic<unsigned long long> configured{0};          // per instantiation, one bit per device
     auto kern = nm_row_tc_kernel<TO, kCol, kTok>;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    {
+        cudaError_t e = ensure_dynamic_smem(kern, 200 * 1024, configured);
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.ntiles, a.nsplit, a.H);

@@ -407,11 +407,10 @@ cudaError_t launch_row_tma(const CUtensorMap &tmap, const TmaArgs &ta_in, size_t
 #define NM_X(m)                                                                                           \
     case m: {                                                                                             \
         auto kern = nm_row_tma_kernel<m, TPR, TO>;                                                        \
-        static bool configured = false;                                                                   \
-        if (!configured) {                                                                                \
-            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); \
+        static std::atomic<unsigned long long> configured{0};       /* per launch site, one bit per device */ \
+        {                                                                                                 \
+            cudaError_t e = ensure_dynamic_smem(kern, 200 * 1024, configured);                            \
             if (e != cudaSuccess) return e;                                                               \
-            configured = true;                                                                            \
         }                                                                                                 \
         /* clusters that would need a second wave: through the workspace instead (query_only: just say so) */ \
         const bool fits = !ta.cluster_split || clusters_fit_one_wave(kern, cfg, (unsigned)a.nsplit, (long)a.ntiles * a.H); \

@@ -89,3 +89,47 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.nm_matmul(vp(256), vp(512), vp(1024), 1, 8, 8, 7, 0, None) == -2
     assert lib.nm_matmul(vp(257), vp(512), vp(1024), 1, 8, 8, 1, 0, None) == -3
     assert lib.nm_set_workspace(vp(4096), ctypes.c_size_t(16)) == -4
+
+
+def test_tuning_state_is_safe_under_concurrent_host_threads(lib):
+    """Two threads ask for plans while a third flips the forced plan between two settings: every answer must be one of
+    the two plans in full (never the tile width of one with the split count of the other), and nothing crashes."""
+    import threading
+    M, N, K = 4, 4096, 8192
+    out0 = (ctypes.c_int * 6)()
+    settings = ((64, 4), (128, 2))
+    want = set()
+    for tn, ns in settings:
+        assert lib.nm_debug_set_plan(tn, ns) == 0
+        assert lib.nm_debug_set_kernel(3, 0) == 0
+        assert lib.nm_debug_get_plan(M, N, K, 1, 1, 0, 1, out0) == 0
+        want.add(tuple(out0))
+    assert len(want) == 2
+    stop = threading.Event()
+    seen, errors = [set(), set()], []
+
+    def flipper():
+        i = 0
+        while not stop.is_set():
+            lib.nm_debug_set_plan(*settings[i & 1])
+            i += 1
+
+    def reader(slot):
+        out = (ctypes.c_int * 6)()
+        for _ in range(20000):
+            if lib.nm_debug_get_plan(M, N, K, 1, 1, 0, 1, out) != 0:
+                errors.append("status")
+            seen[slot].add(tuple(out))
+
+    threads = [threading.Thread(target=flipper)] + [threading.Thread(target=reader, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads[1:]:
+        t.join()
+    stop.set()
+    threads[0].join()
+    lib.nm_debug_set_plan(0, 0)
+    lib.nm_debug_set_kernel(-1, 0)
+    assert not errors
+    for s_ in seen:
+        assert s_ <= want, f"torn plan: {s_ - want}"

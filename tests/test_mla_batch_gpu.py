@@ -6,7 +6,7 @@ import torch
 
 import nm_inputs as gen
 import oracle
-from gpu_util import assert_output_side_stage_by_stage, to_dev
+from gpu_util import END_TO_END_BOUND, assert_step_stage_by_stage, end_to_end_distance, to_dev
 
 pytestmark = pytest.mark.gpu
 DIMS = gen.DSV3_DIMS
@@ -55,10 +55,14 @@ def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True, graph
     q_full = torch.zeros(T * H * dkv, dtype=torch.int16, device="cuda")
     o_lat = torch.zeros(T * H * dc, dtype=torch.int16, device="cuda")
     o = torch.zeros(T * H * dv, dtype=torch.int16, device="cuda")
+    dq = dn + dr
+    c_q, c_qn = (torch.zeros(T * ql, dtype=torch.int16, device="cuda") for _ in range(2))
+    q = torch.zeros(T * H * dq, dtype=torch.int16, device="cuda")
+    ckr = torch.zeros(T * dkv, dtype=torch.int16, device="cuda")
     p = nm.mla_params(DIMS, 1, t)
     ws = nm.new_workspace(nm.nm_mla_batch_workspace_bytes(p, T))
     p = nm.mla_params(DIMS, 1, t, workspace=ws)
-    b = nm.mla_batch(seq_lens, h, cs, cache, stride, out=out, q_full=q_full, o_lat=o_lat, o=o)
+    b = nm.mla_batch(seq_lens, h, cs, cache, stride, out=out, q_full=q_full, o_lat=o_lat, o=o, c_q=c_q, c_qn=c_qn, q=q, ckr=ckr)
     st = torch.cuda.Stream()
     torch.cuda.synchronize()
     if graph:                                                # captured once, replayed: the call allocates and synchronises nothing
@@ -71,6 +75,7 @@ def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True, graph
     torch.cuda.synchronize()
     nm.nm_check_status()
     return {"out": out.view(T, d), "q_full": q_full.view(T, H, dkv), "o_lat": o_lat.view(T, H, dc), "o": o.view(T, H * dv),
+            "c_q": c_q.view(T, ql), "c_qn": c_qn.view(T, ql), "q": q.view(T, H * dq), "ckr": ckr.view(T, dkv),
             "cache": cache.view(T, stride), "stride": stride}
 
 
@@ -79,41 +84,35 @@ def rel_max(got, ref):
 
 
 def check_against_oracle(w, res, tokens, caches, seq_lens, with_wo=True):
+    """Each sequence of the batch as a single-token step: every stage against the oracle on the GPU's own input to that
+    stage at the stated criteria (gpu_util.assert_step_stage_by_stage) - this covers the batch-only kernels of the query
+    side (RMSNorm and the cache-row write after the down-projections, RoPE, the per-head products in both forms) as well as
+    the attention pass and the output side; old cache rows bit for bit; and the end-to-end distance to the oracle's own
+    chain, printed and held to one fixed bound."""
     H, dc, dr = DIMS["H"], DIMS["kv_lora"], DIMS["rope"]
     dkv = dc + dr
     ww = dict(w)
     if not with_wo:
         ww.pop("W_O", None)
+    worst = {}
     for i, S in enumerate(seq_lens):
         r = oracle.mla_decode_step(DIMS, ww, tokens[i], caches[i], S, threads=8)
         cache_ref = caches[i]                                # the oracle wrote row S-1 in place
         got = res["cache"][i].cpu().numpy().view(np.uint16)[:S * dkv].reshape(S, dkv)
         assert np.array_equal(got[:S - 1], cache_ref[:S - 1]), f"sequence {i}: old rows changed"
-        new_row, ref_row = f64(got[S - 1]), f64(cache_ref[S - 1])
-        # normalised part: one ulp of the product's own rounding flip is up to two ulps of an output at the top of its binade,
-        # plus the output's own rounding
-        assert np.all(np.abs(new_row[:dc] - ref_row[:dc]) <= 3 * oracle.ulp_bf16(ref_row[:dc]) + 1e-6), i
-        # the rotated part: a rounding flip of an input moves a pair's outputs on the scale of the pair, not of the
-        # (possibly cancelled) output element
-        assert np.all(np.abs(new_row[dc:] - ref_row[dc:]) <= 2 * oracle.ulp_bf16(np.abs(ref_row[dc:]).max()) + 1e-6), i
-        qf = dev_bits_to_f64(res["q_full"][i]).reshape(H, dkv)
-        assert rel_max(qf[:, :dc], f64(r["q_lat"])) <= 1e-2 and rel_max(qf[:, dc:], f64(r["q_rope"])) <= 1e-2, i
-        # End to end against the oracle's own chain.  The attention output: the softmax criterion.  What follows it inherits
-        # the bf16 roundings of o_lat (and of o) that fell the other way than the oracle's - a valid result, since fp32 and
-        # fp64 sums differ in their last bits, and more frequent after a flip early in the chain (one flipped element of
-        # the normalised query latent moves 1-2 % of q) - each such stage adds up to the same 2e-3 of the largest output
-        # again; so o and out are held to twice the softmax criterion end to end, and to the matmul criterion stage by
-        # stage on the GPU's own stage inputs, where no earlier rounding enters.
-        # Where an early rounding fell the other way (q_full then differs from the oracle's on more than 0.5 % of its elements)
-        # the scores themselves differ, and every end-to-end bound is taken twice.
-        k = 1 if np.mean(qf == np.concatenate([f64(r["q_lat"]), f64(r["q_rope"])], axis=1)) >= 0.995 else 2
-        names = [("o_lat", r["o_lat"], k * 2e-3), ("o", r["o"], k * 4e-3)] + ([("out", r["out"], k * 4e-3)] if with_wo else [])
-        for name, ref_bits, tol in names:
-            g, ref = dev_bits_to_f64(res[name][i]).reshape(-1), f64(ref_bits).reshape(-1)
-            assert np.all(np.abs(g - ref) <= tol * np.abs(ref).max() + oracle.ulp_bf16(ref)), f"sequence {i}: {name}"
-        bits = lambda t: t.contiguous().cpu().numpy().view(np.uint16)
-        assert_output_side_stage_by_stage(DIMS, ww, bits(res["q_full"][i]), got, bits(res["o_lat"][i]), bits(res["o"][i]),
-                                          bits(res["out"][i]) if with_wo else None, f"sequence {i}")
+        g = {k: res[k][i] for k in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o")}
+        g["cache"] = got
+        g["out"] = res["out"][i] if with_wo else None
+        assert_step_stage_by_stage(DIMS, ww, tokens[i], S - 1, g, f"sequence {i} (S {S})")
+        refs = {"q_full": np.concatenate([np.asarray(r["q_lat"]), np.asarray(r["q_rope"])], axis=1), "o_lat": r["o_lat"], "o": r["o"]}
+        if with_wo:
+            refs["out"] = r["out"]
+        for k, v in refs.items():
+            worst[k] = max(worst.get(k, 0.0), end_to_end_distance(res[k][i], v))
+        worst["cache row"] = max(worst.get("cache row", 0.0), end_to_end_distance(got[S - 1], cache_ref[S - 1]))
+    print(f"batch of {len(seq_lens)}: end-to-end distance to the oracle's chain: " + ", ".join(f"{k} {v:.1e}" for k, v in worst.items()))
+    k = max(worst, key=worst.get)
+    assert worst[k] <= END_TO_END_BOUND, f"{k} is {worst[k]:.2e} from the oracle's chain"
 
 
 def make_inputs(seq_lens, seed):

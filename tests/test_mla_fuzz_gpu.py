@@ -68,7 +68,7 @@ def test_random_step_matches_the_oracle(nm, weights, seed):
     finally:
         nm.nm_debug_set_step_tails(1); nm.nm_debug_set_step_fusion(True); nm.nm_debug_set_step_pdl(True); nm.nm_debug_set_attention(0)
     try:
-        base.check_step(t, r, cache_ref, S)
+        base.check_step(t, r, cache_ref, S, weights, h, what=what)
     except AssertionError as e:
         raise AssertionError(f"{what}: {e}") from e
 
@@ -78,9 +78,8 @@ def test_random_tokens_match_the_oracle(nm, weights, seed):
     """A different token per case (the cases above share one token and vary everything else).  The bf16 rounding after
     every stage makes the chain sensitive to the last bits of a sum: where the GPU's fp32 sum and the oracle's fp64 sum
     round one element of the query latent to different neighbours (both valid; about one token in ten), 1-2 % of q
-    and up to a quarter of q_lat follow, and o and out, which inherit the roundings of o_lat, move by up to the softmax
-    criterion again.  So: o_lat end to end within the softmax criterion, o and out within twice that, and the output
-    side stage by stage on the GPU's own stage inputs within the stage criteria."""
+    and up to a quarter of q_lat follow.  The check is therefore stage by stage on the GPU's own stage inputs, at the
+    stated criteria; the end-to-end distance is printed and held to one fixed bound."""
     rng = np.random.default_rng(51_000 + seed)
     S = int(rng.choice([1, 2, 64, 65, 129, int(rng.integers(130, 3000)), int(rng.integers(130, 3000))]))
     concat = bool(rng.random() < 0.7)
@@ -94,7 +93,7 @@ def test_random_tokens_match_the_oracle(nm, weights, seed):
     finally:
         nm.nm_debug_set_attention(0)
     try:
-        base.check_step(t, r, cache_ref, S, w=weights, downstream_tol=4e-3)
+        base.check_step(t, r, cache_ref, S, weights, h)
     except AssertionError as e:
         raise AssertionError(f"seed {seed}: S {S} concat {concat} attention {attn}: {e}") from e
 

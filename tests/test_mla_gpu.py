@@ -6,7 +6,7 @@ import torch
 
 import nm_inputs as gen
 import oracle
-from gpu_util import assert_matmul_close, assert_output_side_stage_by_stage, out_to_f64, to_dev
+from gpu_util import END_TO_END_BOUND, assert_matmul_close, assert_step_stage_by_stage, end_to_end_distance, out_to_f64, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -121,30 +121,32 @@ def test_matmul_stages_of_the_step(nm, ref1024, weights):
     dq, dkv = dn + dr, dc + dr
     ws = nm.new_workspace(max(nm.nm_matmul_workspace_bytes(1, H * dq, ql), nm.nm_matmul_workspace_bytes(1, dc, dn, H)))
 
-    def run(A, Wd, M, N, K, ref_bits, bound, what):
+    def run(A, Wd, W_bits, M, N, K, ref_bits, what):
         C = torch.zeros(M * N, dtype=torch.int16, device="cuda")
         nm.nm_matmul_ws(to_dev(A), Wd, C, M, N, K, BF16, ROW, ws)
         torch.cuda.synchronize()
-        ref = f64(ref_bits).reshape(M, N)
-        tol = 1e-5 * bound.reshape(M, N) + 1e-6 + 2 * oracle.ulp_bf16(ref)   # oracle value already rounded: one ulp each side
-        err = np.abs(dev_bits_to_f64(C).reshape(M, N) - ref)
-        assert np.all(err <= tol), f"{what}: {np.sum(err > tol)} outside tolerance, worst {err.max()}"
+        Cq, C64, bound = oracle.matmul(np.asarray(A).reshape(M, K), W_bits, M, N, K, oracle.BF16, oracle.BF16, threads=8)
+        assert np.array_equal(Cq.reshape(-1), np.asarray(ref_bits).reshape(-1)), what      # the step's stage IS this product
+        assert_matmul_close(dev_bits_to_f64(C).reshape(M, N), Cq, C64, bound, 1, what)
 
-    run(h, dw["W_DQ"], 1, ql, d, r["c_q"], r["bound_c_q"], "c_q = h*W_DQ")
-    run(r["c_qn"], dw["W_UQR"], 1, H * dq, ql, r["q"], r["bound_q"], "q = c_qn*W_UQR")
-    run(h, dw["W_DKVKR"], 1, dkv, d, r["ckr"], r["bound_ckr"], "ckr = h*(W_DKV|W_KR)")
-    run(r["o"].reshape(-1), dw["W_O"], 1, d, H * dv, r["out"], r["bound_out"], "out = o*W_O")
+    run(h, dw["W_DQ"], w["W_DQ"], 1, ql, d, r["c_q"], "c_q = h*W_DQ")
+    run(r["c_qn"], dw["W_UQR"], w["W_UQR"], 1, H * dq, ql, r["q"], "q = c_qn*W_UQR")
+    run(h, dw["W_DKVKR"], w["W_DKVKR"], 1, dkv, d, r["ckr"], "ckr = h*(W_DKV|W_KR)")
+    run(r["o"].reshape(-1), dw["W_O"], w["W_O"], 1, d, H * dv, r["out"], "out = o*W_O")
     # per-head: q_lat written with the attention operand's stride, o from o_lat
     qfull = torch.zeros(H * dkv, dtype=torch.int16, device="cuda")
     nm.nm_matmul_batched_ws(to_dev(r["q"]), dw["W_UK"], qfull, 1, dc, dn, H, H * dq, dq, dn * dc, H * dkv, dkv, BF16, ROW, ws)
     o = torch.zeros(H * dv, dtype=torch.int16, device="cuda")
     nm.nm_matmul_batched_ws(to_dev(r["o_lat"]), dw["W_UV"], o, 1, dv, dc, H, H * dc, dc, dc * dv, H * dv, dv, BF16, ROW, ws)
     torch.cuda.synchronize()
-    got = dev_bits_to_f64(qfull).reshape(H, dkv)[:, :dc]
-    ref = f64(r["q_lat"])
-    assert np.all(np.abs(got - ref) <= 1e-5 * r["bound_q_lat"] + 1e-6 + 2 * oracle.ulp_bf16(ref))
-    got, ref = dev_bits_to_f64(o).reshape(H, dv), f64(r["o"])
-    assert np.all(np.abs(got - ref) <= 1e-5 * r["bound_o"] + 1e-6 + 2 * oracle.ulp_bf16(ref))
+    Cq, C64, bound = oracle.matmul_batched(np.asarray(r["q"]).reshape(-1), np.asarray(w["W_UK"]).reshape(-1), 1, dc, dn, H, H * dq, dq,
+                                           dn * dc, H * dc, dc, H * dc, oracle.BF16, oracle.BF16, threads=8)
+    assert np.array_equal(Cq.reshape(H, dc), np.asarray(r["q_lat"]))
+    assert_matmul_close(dev_bits_to_f64(qfull).reshape(H, dkv)[:, :dc].reshape(-1), Cq, C64, bound, 1, "q_lat = q_nope*W_UK")
+    Cq, C64, bound = oracle.matmul_batched(np.asarray(r["o_lat"]).reshape(-1), np.asarray(w["W_UV"]).reshape(-1), 1, dv, dc, H, H * dc, dc,
+                                           dc * dv, H * dv, dv, H * dv, oracle.BF16, oracle.BF16, threads=8)
+    assert np.array_equal(Cq.reshape(H, dv), np.asarray(r["o"]))
+    assert_matmul_close(dev_bits_to_f64(o).reshape(-1), Cq, C64, bound, 1, "o = o_lat*W_UV")
 
 
 # ---- attention stage -----------------------------------------------------------------------------------
@@ -258,48 +260,38 @@ def run_step(nm, dw, h, cache_in, S, with_wo=True, overlap=True, rows=None, conc
     return t
 
 
-def check_step(t, r, cache_ref, S, with_wo=True, w=None, downstream_tol=2e-3):
-    """End to end against the oracle's chain.  With the weights `w` given, the output side is also checked stage by stage
-    on the GPU's own stage inputs (no earlier rounding enters); `downstream_tol` is the end-to-end bound on o and out,
-    which inherit the roundings of o_lat that fell the other way than the oracle's (see the batch tests)."""
+def check_step(t, r, cache_ref, S, w, h, with_wo=True, what="step"):
+    """The parity check of a whole step.
+    (a) Stage by stage, every stage, at the stated criteria: the oracle recomputes each stage from the GPU's own input
+        to that stage (gpu_util.assert_step_stage_by_stage).  This is what the parity claim rests on.
+    (b) The cache rows before the new one are untouched, bit for bit.
+    (c) End to end against the oracle's own chain from h: the first-stage products (whose inputs ARE the oracle's) at
+        the matmul criterion; for everything downstream the distance max|g - o| / max|o| is printed and held to one
+        fixed bound (gpu_util.END_TO_END_BOUND) that does not depend on the data: two valid chains of eleven bf16
+        roundings may part by a rounding flip early on, so the stated criteria are applied per stage in (a), not here."""
     H, dc, dr, dn = DIMS["H"], DIMS["kv_lora"], DIMS["rope"], DIMS["nope"]
     dkv = dc + dr
-    # first-stage products see exactly the oracle's inputs: tight bound
+    cache = t["kv_cache"].cpu().numpy().view(np.uint16).reshape(-1, dkv)
+    g = {k: t[k] for k in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o", "o_lat_f32")}
+    g["cache"] = cache[:S]
+    g["out"] = t["out"] if with_wo else None
+    ww = dict(w)
+    if not with_wo:
+        ww.pop("W_O", None)
+    assert_step_stage_by_stage(DIMS, ww, h, S - 1, g, what)
+    assert np.array_equal(cache[:S - 1], cache_ref[:S - 1]), f"{what}: old cache rows changed"
     for name, bound in (("c_q", "bound_c_q"), ("ckr", "bound_ckr")):
         got, ref = dev_bits_to_f64(t[name]), f64(r[name])
-        assert np.all(np.abs(got - ref) <= 1e-5 * r[bound] + 1e-6 + 2 * oracle.ulp_bf16(ref)), name
-    # later stages inherit at most a rounding flip from their inputs: compare against the scale of the tensor
-    for name, ref in (("c_qn", f64(r["c_qn"])), ("q", f64(r["q"]).reshape(-1))):
-        assert rel_max(dev_bits_to_f64(t[name]), ref) <= 1e-2, name
-    qf = dev_bits_to_f64(t["q_full"]).reshape(H, dkv)
-    assert rel_max(qf[:, :dc], f64(r["q_lat"])) <= 1e-2 and rel_max(qf[:, dc:], f64(r["q_rope"])) <= 1e-2
-    # the cache: old rows untouched, the new row equals the oracle's up to a rounding flip
-    cache = t["kv_cache"].cpu().numpy().view(np.uint16).reshape(-1, dkv)
-    assert np.array_equal(cache[:S - 1], cache_ref[:S - 1])
-    new_row, ref_row = f64(cache[S - 1]), f64(cache_ref[S - 1])
-    # normalised part: one ulp of the product's own rounding flip is up to two ulps of an output at the top of its binade,
-    # plus the output's own rounding
-    assert np.all(np.abs(new_row[:dc] - ref_row[:dc]) <= 3 * oracle.ulp_bf16(ref_row[:dc]) + 1e-6)
-    # the rotated part: a rounding flip of an input moves a pair's outputs on the scale of the pair, not of the (possibly
-    # cancelled) output element
-    assert np.all(np.abs(new_row[dc:] - ref_row[dc:]) <= 2 * oracle.ulp_bf16(np.abs(ref_row[dc:]).max()) + 1e-6)
-    # softmax-containing outputs: max relative error <= 2e-3 (unrounded), plus one ulp once rounded
-    # ... where the query the attention saw is the oracle's.  Where an early rounding fell the other way (then 1-2 % of q and
-    # up to a quarter of q_lat differ from the oracle's by an ulp: both chains are valid) the scores themselves differ,
-    # and the end-to-end bound is taken twice; the stage-by-stage check below stays at the criterion.
-    qref = np.concatenate([f64(r["q_lat"]), f64(r["q_rope"])], axis=1)
-    k = 1 if np.mean(qf == qref) >= 0.995 else 2
-    tol32 = k * 2e-3
-    o32 = t["o_lat_f32"].cpu().numpy().astype(np.float64).reshape(H, dc)
-    assert rel_max(o32, r["o_lat_f64"]) <= tol32, f"o_lat: {rel_max(o32, r['o_lat_f64']):.2e}"
-    names = [("o_lat", r["o_lat"], tol32), ("o", r["o"], k * downstream_tol)] + ([("out", r["out"], k * downstream_tol)] if with_wo else [])
-    for name, ref_bits, tol in names:
-        got, ref = dev_bits_to_f64(t[name]), f64(ref_bits).reshape(-1)
-        assert np.all(np.abs(got - ref) <= tol * np.abs(ref).max() + oracle.ulp_bf16(ref)), name
-    if w is not None:
-        bits = lambda x: x.cpu().numpy().view(np.uint16)
-        assert_output_side_stage_by_stage(DIMS, w, bits(t["q_full"]), cache[:S], bits(t["o_lat"]), bits(t["o"]),
-                                          bits(t["out"]) if with_wo else None, "step")
+        assert np.all(np.abs(got - ref) <= 1e-5 * r[bound] + 1e-6 + oracle.ulp_bf16(ref)), f"{what}: {name} end to end"
+    refs = {"c_qn": r["c_qn"], "q": r["q"], "q_full": np.concatenate([np.asarray(r["q_lat"]), np.asarray(r["q_rope"])], axis=1),
+            "kv_cache row": cache_ref[S - 1], "o_lat": r["o_lat"], "o": r["o"]}
+    if with_wo:
+        refs["out"] = r["out"]
+    dist = {k: end_to_end_distance(cache[S - 1] if k == "kv_cache row" else t[k], v) for k, v in refs.items()}
+    dist["o_lat_f32"] = rel_max(t["o_lat_f32"].cpu().numpy().astype(np.float64).reshape(H, dc), r["o_lat_f64"])
+    print(f"{what}: S {S}: end-to-end distance to the oracle's chain: " + ", ".join(f"{k} {v:.1e}" for k, v in dist.items()))
+    worst = max(dist, key=dist.get)
+    assert dist[worst] <= END_TO_END_BOUND, f"{what}: {worst} is {dist[worst]:.2e} from the oracle's chain"
 
 
 @pytest.mark.parametrize("overlap", [True, False])
@@ -308,7 +300,7 @@ def test_decode_step_s1024(nm, weights, ref1024, overlap):
     h, cache_ref, r = ref1024
     cache_in = gen.mla_cache(1024, DIMS, seed=4200)
     t = run_step(nm, dw, h, cache_in, 1024, overlap=overlap)
-    check_step(t, r, cache_ref, 1024)
+    check_step(t, r, cache_ref, 1024, w, h)
 
 
 @pytest.mark.parametrize("S", [1, 70, 1024])
@@ -318,7 +310,7 @@ def test_decode_step_with_concatenated_down_projections(nm, weights, S):
     h, cache_ref, r = oracle_step(w, S, seed=4500 + S)
     cache_in = gen.mla_cache(S, DIMS, seed=4500 + S)
     t = run_step(nm, dw, h, cache_in, S, concat_down=True)
-    check_step(t, r, cache_ref, S)
+    check_step(t, r, cache_ref, S, w, h)
 
 
 @pytest.mark.parametrize("concat_down", [True, False])
@@ -340,7 +332,7 @@ def test_decode_step_with_the_dense_weights_in_fractal_storage(nm, weights, conc
         nz["W_DQKV"] = to_dev(gen.to_fractal_nz(cat))
         nz.pop("W_DQ"); nz.pop("W_DKVKR")
     t = run_step(nm, nz, h, cache_in, S, layout_dense=2)
-    check_step(t, r, cache_ref, S)
+    check_step(t, r, cache_ref, S, w, h)
     # the oracle on the fractal storage itself gives the same reference (its index formula, pinned on its own)
     wnz = dict(w)
     for name, (K, N) in shapes.items():
@@ -355,7 +347,7 @@ def test_decode_step_other_lengths(nm, weights, S):
     h, cache_ref, r = oracle_step(w, S, seed=4300 + S)
     cache_in = gen.mla_cache(S, DIMS, seed=4300 + S)
     t = run_step(nm, dw, h, cache_in, S)
-    check_step(t, r, cache_ref, S)
+    check_step(t, r, cache_ref, S, w, h)
 
 
 def test_decode_step_fused_and_unfused_per_head_stages_agree(nm, weights, ref1024):
@@ -366,7 +358,7 @@ def test_decode_step_fused_and_unfused_per_head_stages_agree(nm, weights, ref102
     nm.nm_debug_set_step_fusion(False)
     try:
         t2 = run_step(nm, dw, h, cache_in, 1024)
-        check_step(t2, r, cache_ref, 1024)
+        check_step(t2, r, cache_ref, 1024, w, h)
     finally:
         nm.nm_debug_set_step_fusion(True)
     # the two routes sum in different orders: q_full is the same bf16 value up to a rounding flip on a few
@@ -390,12 +382,12 @@ def test_decode_step_vector_stages_inside_and_outside_the_products_agree(nm, wei
     # the query latent applied by W_UQR while loading its row, KV consumers in an extra CTA of the per-head query
     # kernel; 2 - the CTA completing the product's last tile runs the stages; 0 - kernels of their own
     t1 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
-    check_step(t1, r, cache_ref, 1024)
+    check_step(t1, r, cache_ref, 1024, w, h)
     for mode in (2, 0):
         nm.nm_debug_set_step_tails(mode)
         try:
             t2 = run_step(nm, dw, h, cache_in, 1024, concat_down=concat_down)
-            check_step(t2, r, cache_ref, 1024)
+            check_step(t2, r, cache_ref, 1024, w, h)
         finally:
             nm.nm_debug_set_step_tails(1)
         # the products are bit-identical (same summation order); the norms sum their squares in a
@@ -418,7 +410,7 @@ def test_decode_step_forced_product_plans_inside_the_step(nm, weights, ref1024):
         for which, plan in ((0, (64, 7, 3)), (1, (256, 2, 4)), (2, (128, 3, 5)), (2, (64, 2, 5))):
             nm.nm_debug_set_step_plan(which, *plan)
             t = run_step(nm, dw, h, cache_in, 1024, concat_down=True)
-            check_step(t, r, cache_ref, 1024)
+            check_step(t, r, cache_ref, 1024, w, h)
             nm.nm_debug_set_step_plan(which, 0, 0, 0)
     finally:
         for which in range(3):
@@ -431,7 +423,7 @@ def test_decode_step_without_wo_and_repeatable(nm, weights):
     h, cache_ref, r = oracle_step(w, S, seed=4400, with_wo=False)
     cache_in = gen.mla_cache(S, DIMS, seed=4400)
     t1 = run_step(nm, dw, h, cache_in, S, with_wo=False)
-    check_step(t1, r, cache_ref, S, with_wo=False)
+    check_step(t1, r, cache_ref, S, w, h, with_wo=False)
     t2 = run_step(nm, dw, h, cache_in, S, with_wo=False)
     for k in ("c_q", "q_full", "o_lat", "o"):
         assert torch.equal(t1[k], t2[k]), f"{k}: two runs differ"
@@ -449,7 +441,7 @@ def test_decode_step_same_bits_with_and_without_programmatic_launch(nm, weights,
         nm.nm_debug_set_step_pdl(True)
     for k in ("c_q", "c_qn", "q", "q_full", "ckr", "o_lat", "o", "out", "kv_cache"):
         assert torch.equal(t1[k], t2[k]), k
-    check_step(t2, r, cache_ref, 1024)
+    check_step(t2, r, cache_ref, 1024, w, h)
 
 
 def test_decode_step_back_to_back_steps_do_not_interfere(nm, weights, ref1024):
@@ -512,13 +504,24 @@ def test_decode_step_in_the_configuration_the_bench_times(nm, weights, S):
     nm.nm_check_status()
     for o in outs[1:]:
         assert torch.equal(o, outs[0])
+    # on these fixed inputs the two chains agree closely enough that the stated criteria also hold end to end
     o32 = t["o_lat_f32"].cpu().numpy().astype(np.float64).reshape(H, dc)
     assert rel_max(o32, r["o_lat_f64"]) <= 2e-3
     ref = f64(r["out"]).reshape(-1)
     assert np.all(np.abs(dev_bits_to_f64(outs[0]) - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
-    cache = t["kv_cache"].cpu().numpy().view(np.uint16).reshape(-1, dkv)
-    assert np.array_equal(cache[:S - 1], cache_ref[:S - 1])
-    assert np.all(np.abs(f64(cache[S - 1]) - f64(cache_ref[S - 1])) <= 2 * oracle.ulp_bf16(f64(cache_ref[S - 1])) + 1e-6)
+    # once more with every stage output requested (the copies that deliver them sit between the kernels, so this is
+    # not the timed configuration any more): same result bit for bit, and every stage at its criterion
+    dq = dn + dr
+    for k, n in {"c_q": ql, "c_qn": ql, "q": H * dq, "q_full": H * dkv, "ckr": dkv, "o_lat": H * dc, "o": H * dv}.items():
+        t[k] = torch.zeros(n, dtype=torch.int16, device="cuda")
+    p2 = nm.mla_params(DIMS, S, t, workspace=ws)
+    p2.programmatic_entry = 1
+    with torch.cuda.stream(main):
+        nm.nm_mla_decode_step(p2, main, side)
+    torch.cuda.synchronize()
+    nm.nm_check_status()
+    assert torch.equal(t["out"], outs[0])
+    check_step(t, r, cache_ref, S, w, h, what="bench configuration")
 
 
 def test_decode_step_replayed_from_a_cuda_graph(nm, weights, ref1024):

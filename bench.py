@@ -102,18 +102,37 @@ class ProjectionChain:
         self.out_host.copy_(self.y["W_O"], non_blocking=True)
 
 
+def ncu_dram_bytes(path):
+    """dram__bytes_read.sum + dram__bytes_write.sum (bytes) from a text summary of an ncu capture, or None."""
+    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    total, seen = 0.0, 0
+    try:
+        for line in open(path):
+            f = line.split()
+            if len(f) >= 3 and f[0] in ("dram__bytes_read.sum", "dram__bytes_write.sum") and f[2] in scale:
+                total += float(f[1].replace(",", "")) * scale[f[2]]
+                seen += 1
+    except OSError:
+        return None
+    return int(round(total)) if seen == 2 else None
+
+
 class MlaStep:
     """The whole single-token decode step (nm_mla_decode_step): Q chain, KV chain on a side stream,
     tensor-core latent attention over the cache, output side including W_O."""
 
     name = "mla"
 
-    def __init__(self, nm, device, seq_len, seed=4000, schedule="fused", weights="row"):
+    def __init__(self, nm, device, seq_len, seed=4000, schedule="fused", weights="row", share=None):
         self.nm = nm
         self.S = seq_len
         self.schedule = schedule
         self.weights = weights
         d, ql, dc, dr, dn, dv, H = (DIMS[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
+        if share is not None:
+            # the same resident weights (and token) at another sequence length: own cache, table, output and workspace
+            self._finish(nm, device, seq_len, seed, dict(share.t), share.layout_dense, share.h_host)
+            return
         w = gen.mla_weights(DIMS, seed=seed, with_wo=True)
         t = {k: torch.from_numpy(v.view(np.int16)).to(device) for k, v in w.items()}
         if schedule == "fused":
@@ -129,9 +148,16 @@ class MlaStep:
             for name, (K_, N_) in shapes.items():
                 if name in t:
                     t[name] = torch.from_numpy(gen.to_fractal_nz(t[name].cpu().numpy().reshape(K_, N_))).to(device)
-        self.h_host = torch.from_numpy(gen.mla_token(DIMS, seed=seed + 100).view(np.int16).copy()).pin_memory()
+        h_host = torch.from_numpy(gen.mla_token(DIMS, seed=seed + 100).view(np.int16).copy()).pin_memory()
+        t["h"] = h_host.to(device)
+        self._finish(nm, device, seq_len, seed, t, layout_dense, h_host)
+
+    def _finish(self, nm, device, seq_len, seed, t, layout_dense, h_host):
+        d, ql, dc, dr, dn, dv, H = (DIMS[k] for k in ("d", "q_lora", "kv_lora", "rope", "nope", "v", "H"))
+        schedule = self.schedule
+        self.layout_dense = layout_dense
+        self.h_host = h_host
         self.out_host = torch.empty(d, dtype=torch.int16).pin_memory()
-        t["h"] = self.h_host.to(device)
         t["out"] = torch.zeros(d, dtype=torch.int16, device=device)
         t["kv_cache"] = torch.from_numpy(gen.mla_cache(seq_len, DIMS, seed=seed + 200).view(np.int16)).to(device)
         t["rope_cos_sin"] = torch.empty(dr, dtype=torch.float32, device=device)
@@ -149,9 +175,10 @@ class MlaStep:
         self.bytes_per_step = algorithmic_bytes(self.specs) + self.kv_bytes
         self.dominant = "W_O product (nm_row_tma_kernel, K=16384, N=7168, M=1)"
         self.dominant_bytes = algorithmic_bytes([s for s in self.specs if s[0] == "W_O"])
-        # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this shape, from
-        # the ncu capture summarised in profiles/ncu_nm_row_tma_WO_M1_K16384_N7168.txt
-        self.dominant_traffic = 234_975_232 + 3_297_792
+        # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this shape, read from the
+        # committed summary of its ncu capture (None if the file is not there)
+        self.dominant_traffic_source = "profiles/ncu_nm_row_tma_WO_M1_K16384_N7168.txt"
+        self.dominant_traffic = ncu_dram_bytes(os.path.join(ROOT, self.dominant_traffic_source))
         self.launches_per_step = 6 if schedule == "fused" else 7
         self.h2d = d * 2
         self.d2h = d * 2
@@ -440,21 +467,25 @@ def read_only_stream(nm, device):
     return best
 
 
-def matmul_sweep(nm, device, args_no_cpu=False):
+def matmul_sweep(nm, device, args_no_cpu=False, compact=False, peak=None):
     """GB/s of single narrow products (cold L2: the launches of a CUDA graph rotate through copies of
     B that together exceed 512 MB).  Two figures per case: launches in plain stream order (each kernel
     starts when the one before has finished: latency of an isolated call plus the launch gap), and
     launched programmatically (a kernel may fetch its weights while its predecessor drains, as inside
-    the decode step).  Reported beside the step; not part of the timed region."""
+    the decode step).  Reported beside the step; not part of the timed region.
+    compact: the configurations the metric names and the GPU legs only (the default line); otherwise also the
+    fractal storage, 17 and 64 rows, the paper's 100 x 100 schedule, warm-L2 figures and the oracle's times."""
     out = []
     cases = [(1, 512, 512, 0, "f32"), (1, 7168, 1536, 0, "bf16"), (1, 7168, 576, 0, "bf16"), (1, 7168, 1536, 1, "bf16"),
-             (1, 7168, 576, 1, "bf16"),
-             # the storage the paper's test case has in memory (16 x 16 fractals): layout code 2
-             (1, 7168, 1536, 2, "bf16"), (1, 7168, 576, 2, "bf16"), (1, 7168, 18432, 2, "bf16")]
+             (1, 7168, 576, 1, "bf16")]
+    if not compact:
+        # the storage the paper's test case has in memory (16 x 16 fractals): layout code 2
+        cases += [(1, 7168, 1536, 2, "bf16"), (1, 7168, 576, 2, "bf16"), (1, 7168, 18432, 2, "bf16")]
     for M in (1, 2, 4, 8, 16):
         cases += [(M, 1536, 24576, 0, "bf16"), (M, 7168, 18432, 0, "bf16")]
-    # beyond the narrow range: a remainder row on top of 16, and 64 rows, still one pass over B (tensor cores)
-    cases += [(17, 7168, 18432, 0, "bf16"), (64, 7168, 18432, 0, "bf16")]
+    if not compact:
+        # beyond the narrow range: a remainder row on top of 16, and 64 rows, still one pass over B (tensor cores)
+        cases += [(17, 7168, 18432, 0, "bf16"), (64, 7168, 18432, 0, "bf16")]
     # the per-head products of the absorbed MLA form, T tokens at once: q_nope * W_UK (128 -> 512) and
     # o_lat * W_UV (512 -> 128), 128 heads, activations laid out [T][128][K]
     for T in (1, 4, 16):
@@ -464,18 +495,20 @@ def matmul_sweep(nm, device, args_no_cpu=False):
         H = case[5] if len(case) > 5 else 1
         if H > 1:
             out.append(batched_case(nm, device, M, K, N, H))
+            if peak:
+                out[-1]["frac_of_measured"] = round(max(out[-1]["GBps"], out[-1]["GBps_programmatic"]) / peak, 3)
             continue
         es = 4 if dt == "f32" else 2
         tdt = torch.float32 if dt == "f32" else torch.bfloat16
         code = nm.F32 if dt == "f32" else nm.BF16
         nbytes = K * N * es
-        R = max(2, min(64, (1 << 29) // nbytes + 1))
+        R = max(2, min(512, (1 << 29) // nbytes + 1))        # copies of B that together exceed 512 MB (4 x the L2)
         Bs = (torch.randn(R, K * N, device=device) * 0.02).to(tdt)
         A = torch.randn(M * K, device=device).to(tdt)
         C = torch.empty(R, M * N, device=device, dtype=tdt)
         ws = nm.new_workspace(nm.nm_matmul_workspace_bytes(M, N, K), device=device)
         s = torch.cuda.Stream(device)
-        row = {"M": M, "K": K, "N": N, "dtype": dt, "layout_B": ("row", "col", "fractal_nz")[layout]}
+        row = {"M": M, "K": K, "N": N, "dtype": dt, "layout_B": ("row", "col", "fractal_nz")[layout], "copies_of_B": R}
         algo = (K * N + M * K + M * N) * es
         for mode in ("serial", "programmatic"):
             nm.nm_set_programmatic_launch(mode == "programmatic")
@@ -502,6 +535,14 @@ def matmul_sweep(nm, device, args_no_cpu=False):
             del g
         nm.nm_set_programmatic_launch(False)
         row["pct_of_8TBs"] = round(max(row["GBps"], row["GBps_programmatic"]) / 80.0, 1)
+        row["pct_of_8TBs_serial"] = round(row["GBps"] / 80.0, 1)
+        if peak:
+            row["frac_of_measured"] = round(max(row["GBps"], row["GBps_programmatic"]) / peak, 3)
+            row["frac_of_measured_serial"] = round(row["GBps"] / peak, 3)
+        if compact:
+            out.append(row)
+            del Bs, C
+            continue
         # the paper's own schedule (its evaluation section): 100 runs of 100 iterations, the first iteration of
         # every run dropped; direct launches in stream order, B rotating through the copies (cold L2)
         with torch.cuda.stream(s):
@@ -606,7 +647,7 @@ class ClockSampler:
 _ORACLE_INPUTS = {}
 
 
-def oracle_sample(threads, kind="mla", seq_len=4096):
+def oracle_sample(threads, kind="mla", seq_len=16384):
     """One pass of the oracle, as it stands, on the host cores over the same workload: the naive
     decode step at `seq_len` (kind "mla") or the six narrow products alone (kind "projections").
     Returns (seconds, algorithmic bytes, description)."""
@@ -651,7 +692,7 @@ def run_reference(args, rank):
         times.append(dt)
     total = sum(times)
     value = nbytes * len(times) / total / 1e9
-    line = {"impl": "reference", "metric": "narrow MatMul HBM GB/s (MLA single-token decode step)", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+    line = {"impl": "reference", "metric": "narrow MatMul HBM GB/s (% of 8 TB/s) vs M; MLA single-token decode \u00b5s", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
             "steps": steps, "warmup": min(args.warmup, 2), "ms_per_step": total / len(times) * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": "CPU oracle (fp64 triple loop) on a bounded sample: " + what},
@@ -700,8 +741,10 @@ def main():
     ap.add_argument("--schedule", default="fused", choices=["fused", "two-stream"],
                     help="decode step: down-projections as one concatenated product on one stream, or W_DKV|KR on a side stream")
     ap.add_argument("--timeline", action="store_true", help="print the kernel timeline of one step and exit")
-    ap.add_argument("--sweep", action="store_true", help="also report GB/s of single narrow products vs M")
-    ap.add_argument("--seq-len", type=int, default=4096)
+    ap.add_argument("--sweep", action="store_true", help="the full product sweep: more cases, the paper's 100 x 100 schedule, warm-L2 figures, oracle times")
+    ap.add_argument("--seq-len", type=int, default=16384, help="cache rows of the headline step (default: the largest configuration)")
+    ap.add_argument("--single-length", action="store_true", help="skip the step at the other sequence lengths (1024, 4096, 16384)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the narrow-product-vs-M measurements")
     ap.add_argument("--batch", type=int, default=1, help="with --timeline: sequences of the small-batch step (2-16) to trace")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--weights", default="row", choices=["row", "fractal"],
@@ -752,28 +795,43 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    def timed_block(fn, n):
+        """Device time (ms) of n calls of fn, bracketed by a barrier + synchronize on both sides."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        barrier()
+        return e0.elapsed_time(e1)
+
+    # the clock sampler covers everything from the warm-up to the last extra measurement
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
             wl.step(stream)
         barrier()
-        sampler = ClockSampler(local_rank)
-        sampler.start()
-        # ---- device-timed region: exactly `steps` steps, inputs resident in HBM ------------------------
-        dom = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        # ---- device-timed region: blocks of exactly `steps` steps, inputs resident in HBM.  A block shorter than
+        #      half a second is repeated until half a second of device time has gone by (the same count on every
+        #      rank), and the MEDIAN block is reported; nothing but the steps is enqueued inside a block ------------
+        first = timed_block(lambda: wl.step(stream), args.steps)
+        (first_max,) = reduce_over_ranks([first], dist, device)
+        n_blocks = 1 if first_max >= 500.0 else int(min(200, max(3, -(-500.0 // max(first_max, 1e-3)))))
+        blocks = [first] + [timed_block(lambda: wl.step(stream), args.steps) for _ in range(n_blocks - 1)]
+        # ---- the dominant kernel, in a SEPARATE pass after the timed region: events around it on the launching
+        #      stream in every step (the events switch off that kernel's programmatic launch, which is why they are
+        #      kept out of the timed region) ---------------------------------------------------------------------
+        n_dom = 64
+        dom = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_dom)]
         for a, b in dom:                      # events get their handles on first record
             a.record(stream); b.record(stream)
-        dom_stride = 16 if args.steps >= 128 else max(1, args.steps // 8)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
-        e0.record(stream)
-        # the dominant kernel is bracketed by events on every 16th step only (at least 8 samples): the events break the
-        # programmatic launch of that kernel, and the step time should not carry that on every step
-        for i in range(args.steps):
-            wl.step(stream, dom[i] if i % dom_stride == 0 else None)
-        e1.record(stream)
+        for i in range(n_dom):
+            wl.step(stream, dom[i])
         barrier()
-        ms = e0.elapsed_time(e1)
-        dom_ms = statistics.mean(a.elapsed_time(b) for a, b in dom[::dom_stride])
+        dom_ms = statistics.mean(a.elapsed_time(b) for a, b in dom[8:])
         # ---- end-to-end region: host token in, host result out, every step -----------------------------
         for _ in range(3):
             wl.step_e2e(stream)
@@ -786,37 +844,68 @@ def main():
         t1.record(stream)
         barrier()
         e2e_ms = t0.elapsed_time(t1)
-        clocks = sampler.stop()
         extras = wl.extra_measurements(stream) if hasattr(wl, "extra_measurements") else {}
+        # ---- the step at the other sequence lengths of the configuration (same resident weights) ------------------
+        per_len = []
+        if args.workload == "mla" and not args.single_length:
+            for S in sorted({1024, 4096, 16384, args.seq_len}):
+                w2 = wl if S == args.seq_len else MlaStep(nm, device, S, schedule=args.schedule, weights=args.weights, share=wl)
+                if w2 is wl:
+                    per_len.append((S, w2.bytes_per_step, None))
+                    continue
+                for _ in range(max(args.warmup, 20)):
+                    w2.step(stream)
+                n = max(args.steps, 200)
+                per_len.append((S, w2.bytes_per_step, statistics.median(timed_block(lambda: w2.step(stream), n) for _ in range(3)) / n))
+                del w2
     nm.nm_check_status(stream)
 
-    ms, e2e_ms, dom_ms = reduce_over_ranks([ms, e2e_ms, dom_ms], dist, device)
+    blocks = [reduce_over_ranks([b], dist, device)[0] for b in blocks]
+    ms = statistics.median(blocks)
+    e2e_ms, dom_ms = reduce_over_ranks([e2e_ms, dom_ms], dist, device)
+    per_len = [(S, nb, reduce_over_ranks([t], dist, device)[0] if t is not None else ms / args.steps) for S, nb, t in per_len]
 
     if rank == 0:
         peak, peak_kind = load_peaks()
         value = job_throughput_gbs(wl.bytes_per_step, args.steps, world, ms)
         e2e_value = job_throughput_gbs(wl.bytes_per_step, args.steps, world, e2e_ms)
         achieved = wl.dominant_bytes / (dom_ms * 1e-3) / 1e9
-        line = {"metric": "narrow MatMul HBM GB/s (MLA single-token decode step)", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        line = {"metric": "narrow MatMul HBM GB/s (% of 8 TB/s) vs M; MLA single-token decode \u00b5s", "value": value, "unit": "GB/s",
+                "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms / args.steps, "decode_us": ms / args.steps * 1e3,
                 "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": wl.describe(),
                 "pct_of_8TBs": value / world / 8000.0,
+                "frac_of_measured_peak": value / world / peak,
+                "timed_blocks": {"blocks": len(blocks), "steps_per_block": args.steps, "reported": "median block",
+                                 "ms_min_median_max": [min(blocks), ms, max(blocks)]},
                 "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h,
                         "ms_per_step": e2e_ms / args.steps,
                         "launch": ("cuda graph replay" if getattr(wl, "graph", None) else "direct launches"),
                         "graph_error": getattr(wl, "graph_error", None)},
-                "gpu_launches": wl.launches_per_step * args.steps,
-                "clocks": clocks,
+                "gpu_launches": wl.launches_per_step * args.steps * len(blocks),
                 "roofline": {"bound": "hbm", "kernel": wl.dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                              "frac": achieved / peak, "peak_kind": peak_kind, "algorithmic_bytes": wl.dominant_bytes,
                              "traffic": getattr(wl, "dominant_traffic", None),
-                             "us_per_launch": dom_ms * 1e3}}
+                             "traffic_source": getattr(wl, "dominant_traffic_source", None),
+                             "us_per_launch": dom_ms * 1e3,
+                             "measured": f"separate pass of {n_dom} steps after the timed region (first 8 dropped), CUDA events around the "
+                                         "kernel on the launching stream; the events switch off that kernel's programmatic launch"}}
+        if per_len:
+            line["decode_vs_seq_len"] = [{"seq_len": S, "decode_us": t * 1e3, "GBps": nb / t / 1e6, "pct_of_8TBs": nb / t / 1e6 / 80.0,
+                                          "frac_of_measured_peak": nb / t / 1e6 / peak, "algorithmic_bytes": nb} for S, nb, t in per_len]
         line.update(extras)
-        if args.sweep:
-            line["narrow_matmul_vs_M"] = matmul_sweep(nm, device, args.no_cpu_baseline)
+        if args.workload == "mla" and not args.no_sweep:
+            # the metric's first half: narrow products vs M (GPU legs; --sweep adds the oracle's times and more cases)
+            with torch.cuda.stream(stream):
+                line["narrow_matmul_vs_M"] = matmul_sweep(nm, device, args.no_cpu_baseline, compact=not args.sweep, peak=peak)
+                if args.sweep:
+                    line["read_only_stream"] = read_only_stream(nm, device)
+        elif args.sweep:
+            line["narrow_matmul_vs_M"] = matmul_sweep(nm, device, args.no_cpu_baseline, peak=peak)
             line["read_only_stream"] = read_only_stream(nm, device)
+        line["clocks"] = sampler.stop()
         if not args.no_cpu_baseline:
             import oracle
             threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
@@ -830,6 +919,8 @@ def main():
                                     "sample": f"{passes} passes of " + what.replace(", one pass", ""), "seconds": total,
                                     "ms_per_step": total / passes * 1e3}
         print(json.dumps(line), flush=True)
+    else:
+        sampler.stop()
     if dist is not None:
         dist.destroy_process_group()
 

@@ -52,10 +52,14 @@ int nm_debug_set_step_fusion(int enable);
 int nm_debug_set_step_prefetch(int megabytes);
 /* Decode step: chain its kernels with programmatic dependent launch (default 1) or not (0). */
 int nm_debug_set_step_pdl(int enable);
-/* Attention pass: 0 (default) a tensor-core kernel when the shape allows - 64 heads per CTA below 65536 cache rows
- * in the call, 128 heads per CTA from there on; 1 CUDA-core kernel; 2 / 3 the tensor-core kernel with 128 / 64 heads
- * per CTA whatever the length. */
+/* Attention pass: 0 (default) the wide-tile tensor-core kernel when the shape allows (single-token step and stand-alone
+ * attention; the batch step keeps the older kernels: 64 heads per CTA below 65536 cache rows in the call, 128 heads per
+ * CTA from there on); 1 CUDA-core kernel; 2 / 3 the older tensor-core kernels with 128 / 64 heads per CTA whatever the
+ * length; 4 the wide-tile kernel. */
 int nm_debug_set_attention(int impl);
+/* Wide-tile attention kernel: force the cache rows per tile (64, 128, 256), the most row runs (1..64) and the number of
+ * runs merged on chip (cluster of 1, 2 or 4); zeros give each choice back to the planner. */
+int nm_debug_set_attention_wide(int tile_rows, int max_runs, int cluster);
 /* Measurement aid: a kernel that only reads `bytes` bytes of device memory once (16-byte streaming loads, the
  * products' own load instruction, ctas_per_sm x SM-count CTAs of 256 threads) - the read-only bandwidth this GPU
  * delivers, to set beside the copy bandwidth the roofline uses.  src 16-byte aligned; sink4: 4 writable bytes. */
@@ -73,6 +77,14 @@ int nm_debug_get_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
  * then reports NM_ERR_TIMEOUT once.  elapsed_ns (device, 2 x uint64, may be NULL) receives the time the waits took
  * and a bit mask of waits that reported success (expected 0). */
 int nm_debug_wait_probe(unsigned long long limit_ns, unsigned long long *elapsed_ns, nm_stream stream);
+
+/* Measurement aid: clocks of `reps` back-to-back tcgen05.mma (kind::f16, bf16, K = 16) of shape m x n issued by one
+ * thread of one CTA, with the A operand in shared memory (K-major) or in TMEM and the B operand in shared memory K-major
+ * or MN-major, into n_acc accumulators used in turn; consecutive MMAs step the operand addresses by the given bytes
+ * (cycling over four positions).  out_clocks (device, 3 x uint64): clocks until the commit arrived, clocks until the last
+ * MMA was issued, 1 if the wait succeeded.  m 64 or 128; n a multiple of 16 up to 256; n_acc * n <= 448. */
+int nm_debug_mma_probe(int m, int n, int a_from_tmem, int b_mn_major, int reps, int n_acc, int a_step_bytes, int b_step_bytes,
+                       unsigned long long *out_clocks, nm_stream stream);
 
 #ifdef __cplusplus
 }

@@ -100,6 +100,7 @@ _lib.nm_mla_workspace_bytes.argtypes = [C.POINTER(MlaParams)]
 _lib.nm_mla_decode_step.argtypes = [C.POINTER(MlaParams), _vp, _vp]
 _lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_debug_set_attention.argtypes = [_i]
+_lib.nm_debug_set_attention_wide.argtypes = [_i, _i, _i]
 _lib.nm_debug_set_step_pdl.argtypes = [_i]
 _lib.nm_debug_stream_read.argtypes = [_vp, _sz, _vp, _i, _vp]
 _lib.nm_debug_set_step_knobs.argtypes = [_i, _i]
@@ -111,6 +112,7 @@ _lib.nm_debug_set_step_prefetch.argtypes = [_i]
 _lib.nm_debug_set_step_fusion.argtypes = [_i]
 _lib.nm_debug_set_attention_trace.argtypes = [_vp]
 _lib.nm_debug_wait_probe.argtypes = [C.c_ulonglong, _vp, _vp]
+_lib.nm_debug_mma_probe.argtypes = [_i] * 8 + [_vp, _vp]
 
 
 def _check(status: int, where: str) -> None:
@@ -378,6 +380,15 @@ def nm_debug_wait_probe(limit_ns: int, elapsed_ns=None, stream=None) -> None:
     """One CTA waits on an mbarrier nobody arrives at, with the wait limit set to limit_ns for that launch; the
     wait runs out, the kernel returns by itself and nm_check_status reports the timeout once."""
     _check(_lib.nm_debug_wait_probe(int(limit_ns), _ptr(elapsed_ns), _stream(stream)), "nm_debug_wait_probe")
+
+
+def nm_debug_mma_probe(m, n, a_from_tmem, b_mn_major, reps, n_acc, a_step_bytes, b_step_bytes, out_clocks, stream=None) -> None:
+    _check(_lib.nm_debug_mma_probe(int(m), int(n), int(a_from_tmem), int(b_mn_major), int(reps), int(n_acc), int(a_step_bytes),
+                                   int(b_step_bytes), _ptr(out_clocks), _stream(stream)), "nm_debug_mma_probe")
+
+
+def nm_debug_set_attention_wide(tile_rows: int = 0, max_runs: int = 0, cluster: int = 0) -> None:
+    _check(_lib.nm_debug_set_attention_wide(int(tile_rows), int(max_runs), int(cluster)), "nm_debug_set_attention_wide")
 
 
 def nm_debug_set_attention(impl: int) -> None:

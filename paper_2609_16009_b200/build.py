@@ -1,6 +1,6 @@
 """Builds the C-ABI library ``libnm.so`` in-tree with nvcc for sm_100a.
 
-Run as ``python -m paper_2609_16009_b200.build``.  Object files go to ``build/`` at the
+Run as ``python paper_2609_16009_b200/build.py`` (as a script: importing the package needs the library this builds).  Object files go to ``build/`` at the
 repository root; the shared library is written next to this file.  Only changed sources are
 recompiled (mtime against every header).
 """

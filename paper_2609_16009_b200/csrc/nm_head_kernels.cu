@@ -158,8 +158,10 @@ __global__ void __launch_bounds__(kHeadThreads) q_finish_kernel(const uint16_t *
 // thread.  Launched programmatically, it is therefore resident - with half of the head's 128 KB
 // of weights already in registers - when the attention result arrives; the rest (an L2 hit after its own
 // prefetch) is fetched once the partial rows have left their registers.
-constexpr int kUvPre = 16;                                         // weight vectors per thread loaded before the inputs exist
+// kUvPre weight vectors per thread are loaded before the inputs exist; the partial rows are requested kBatch at a time
+// (one L2 round trip per batch): 16 and 16 for up to 16 partials, 8 and 32 beyond (the registers are the same).
 constexpr int kUvMaxParts = 64;                                    // partials per head the merge takes (the planner never makes more)
+template <int kUvPre, int kBatch>
 __global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_t *__restrict__ Q, const uint16_t *__restrict__ cache,
                                                                    AttnPartials part, int npart, long extra_row, int rope, float scale,
                                                                    const uint16_t *__restrict__ W_UV, uint16_t *__restrict__ o_lat_bf16,
@@ -204,7 +206,6 @@ __global__ void __launch_bounds__(kHeadThreads, 2) uv_merge_kernel(const uint16_
     // of up to 16 parts (two columns per thread), the (m, l) pairs, and the operands of the new row's score.
     const int c = 2 * tid;
     const float *src = part.O + (size_t)h * K + c;
-    constexpr int kBatch = 16;
     float2 v[kBatch];
 #pragma unroll
     for (int u = 0; u < kBatch; ++u)
@@ -435,8 +436,9 @@ int launch_uv_merge(const void *Q, const void *cache, AttnPartials part, int npa
 {
     if (npart < 0 || npart > kUvMaxParts) return NM_ERR_UNSUPPORTED;
     if (!prefetch.base && !prefetch.block) prefetch.nranges = -1;  // no prefetch at all
-    cudaError_t e = launch_with_pdl(uv_merge_kernel, H, s, pdl, (const uint16_t *)Q, (const uint16_t *)cache, part, npart, extra_row, rope,
-                                    scale, (const uint16_t *)W_UV, (uint16_t *)o_lat_bf16, o_lat_f32, (uint16_t *)o, prefetch, attention_trace());
+    cudaError_t e = launch_with_pdl(npart > 16 ? uv_merge_kernel<8, 32> : uv_merge_kernel<16, 16>, H, s, pdl, (const uint16_t *)Q,
+                                    (const uint16_t *)cache, part, npart, extra_row, rope, scale, (const uint16_t *)W_UV, (uint16_t *)o_lat_bf16,
+                                    o_lat_f32, (uint16_t *)o, prefetch, attention_trace());
     return e == cudaSuccess ? NM_OK : record_cuda_error(e, "uv_merge launch");
 }
 

@@ -14,7 +14,9 @@ namespace nm {
 // Tuning state of the decode step (nm_debug_set_*): process-wide and guarded by a mutex; every entry point plans from a
 // per-thread snapshot taken once at its start, so a setter on another host thread cannot change a step half way.
 struct StepTuning {
-    int attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel, 2 / 3: force 128 / 64 heads per CTA
+    int attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel, 2 / 3: force 128 / 64 heads per CTA,
+                                // 4: force the wide-tile kernel
+    int wide_tile = 0, wide_splits = 0, wide_cluster = 0;      // wide-tile kernel: forced rows per tile, row runs, cluster size (0 = planner)
     int step_plan[3][3] = {};   // forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
     int host_direct_out = 1;    // host-operand step: store the result straight into device-addressable host memory
     int batch_tc_min_t = 3;     // batch decode: tokens from which the per-head products go to the tensor cores
@@ -43,9 +45,10 @@ template <typename F> static int set_step_tuning(F f)
 // Cache rows (over all sequences of a call) from which the 128-head kernel is the faster one: it loads every row
 // into two CTAs instead of four, which decides once a CTA has many tiles to go through; below, the 64-head
 // kernel's shorter prologue and merge win (measured: 16384 rows 94.8 vs 97.3 us per step, 65536 rows 164 vs 158)
-constexpr long kAttnWideRows = 65536;
+constexpr long kAttn128HeadRows = 65536;
+constexpr int kAttnWideMinRows = 6144;     // single sequence: cache rows from which the wide-tile kernel takes over
 constexpr int kSMsAttn = 148;
-static bool attention_64_heads(long total_rows) { return g_s.attn_impl == 3 || (g_s.attn_impl != 2 && total_rows < kAttnWideRows); }
+static bool attention_64_heads(long total_rows) { return g_s.attn_impl == 3 || (g_s.attn_impl != 2 && total_rows < kAttn128HeadRows); }
 
 // ---- small vector kernels ---------------------------------------------------------------------------
 
@@ -348,11 +351,31 @@ AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int
 {
     AttnPlan p{};
     (void)kv_lora;
-    const int tiles = ceil_div(n_rows > 0 ? n_rows : 0, kAttnTileRows);
     // The tensor-core kernels take 128 heads and 16-byte aligned operands (TMA); both passes of an
     // attention call derive the same answer from the same arguments.
     const bool tc_ok = g_s.attn_impl != 1 && H == 128 && n_rows > 0 && (((uintptr_t)Q | (uintptr_t)cache) & 15u) == 0 &&
                        tensor_map_encoder() != nullptr;
+    // Wide tiles (nm_attn_wide.cu) from kAttnWideMinRows cache rows on: measured per step 83.2 vs 93.2 us at 16384 rows, level
+    // at 4096 (78.2 vs 77.7) and below, where the pass is all fixed cost (waiting for Q, the merge) in either kernel.
+    if (tc_ok && (g_s.attn_impl == 4 || (g_s.attn_impl == 0 && n_rows >= kAttnWideMinRows))) {
+        // One tile per row run as long as at most 64 runs (128 CTAs) cover the rows: the tile is as wide as that takes,
+        // and the runs of a cluster merge on chip so that the final merge reads at most 16 partials per head.
+        int R = g_s.wide_tile;
+        const int max_runs = g_s.wide_splits > 0 ? std::min(g_s.wide_splits, 64) : 64;
+        if (R != 64 && R != 128 && R != 256) R = (n_rows <= 64 * max_runs) ? 64 : (n_rows <= 128 * max_runs ? 128 : 256);
+        const int tiles = ceil_div(n_rows, R);
+        const int nsplit = std::min(tiles, max_runs);
+        p.tensor_core = 3;
+        p.tile_rows = R;
+        p.rows_per_split = ceil_div(tiles, nsplit) * R;
+        p.nsplit = ceil_div(n_rows, p.rows_per_split);
+        int cl = g_s.wide_cluster;
+        if (cl != 1 && cl != 2 && cl != 4) cl = p.nsplit > 32 ? 4 : (p.nsplit > 16 ? 2 : 1);
+        p.cluster = cl;
+        p.npartial = ceil_div(p.nsplit, cl);
+        return p;
+    }
+    const int tiles = ceil_div(n_rows > 0 ? n_rows : 0, kAttnTileRows);
     p.tensor_core = !tc_ok ? 0 : (attention_64_heads(n_rows) ? 2 : 1);
     // one wave of the 148 SMs: 64 splits x 2 column halves (128 heads per CTA), or 32 splits x 2 column halves x 2
     // head halves (64 heads per CTA)
@@ -400,6 +423,8 @@ static int attention_partial(const void *Q, const void *cache, int H, int n_rows
     if (n_rows == 0) return NM_OK;
     const AttnPlan p = plan_attention(Q, cache, H, n_rows, dc);
     AttnPartials part = carve_partials(ws, H);
+    if (p.tensor_core == 3)
+        return attention_partial_wide(Q, 1, &cache, &n_rows, &p.rows_per_split, p.nsplit, p.tile_rows, p.cluster, part, 0, scale, s, pdl, prefetch);
     if (p.tensor_core == 2)
         return attention_partial_tc64(Q, 1, &cache, &n_rows, &p.rows_per_split, p.nsplit, kAttnCluster, part, 0, scale, s, pdl, prefetch);
     if (p.tensor_core) return attention_partial_tc(Q, cache, part, p, n_rows, scale, s, pdl, prefetch);
@@ -1058,8 +1083,14 @@ int nm_debug_set_step_pdl(int enable)
     return set_step_tuning([&](StepTuning &t) { t.step_pdl = enable ? 1 : 0; });
 }
 
-/* 0: tensor-core attention when the shape allows (default); 1: CUDA-core attention kernel; 2 / 3: the tensor-core
- * kernel with 128 / 64 heads per CTA whatever the length. */
+int nm_debug_set_attention_wide(int tile_rows, int max_runs, int cluster)
+{
+    if (tile_rows < 0 || max_runs < 0 || max_runs > 64 || cluster < 0 || cluster > 4) return NM_ERR_INVALID_ARG;
+    return set_step_tuning([&](StepTuning &t) { t.wide_tile = tile_rows; t.wide_splits = max_runs; t.wide_cluster = cluster; });
+}
+
+/* 0: tensor-core attention when the shape allows (default); 1: CUDA-core attention kernel; 2 / 3: the older tensor-core
+ * kernels with 128 / 64 heads per CTA whatever the length; 4: the wide-tile kernel. */
 int nm_debug_set_attention(int impl)
 {
     return set_step_tuning([&](StepTuning &t) { t.attn_impl = impl; });

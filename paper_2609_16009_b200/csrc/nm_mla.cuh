@@ -18,9 +18,11 @@ struct AttnPartials {
 
 struct AttnPlan {
     int nsplit;
-    int rows_per_split;                  // multiple of kAttnTileRows
-    int tensor_core;                     // 0: CUDA-core kernel; 1: tcgen05 kernel, 128 heads per CTA; 2: tcgen05 kernel, 64 heads per CTA
+    int rows_per_split;                  // multiple of kAttnTileRows (of tile_rows for the wide-tile kernel)
+    int tensor_core;                     // 0: CUDA-core kernel; tcgen05 kernels: 1 = 128 heads per CTA, 32-row tiles; 2 = 64 heads per CTA;
+                                         // 3 = 128 heads per CTA, wide tiles (nm_attn_wide.cu)
     int npartial;                        // partial results the final merge has to read
+    int tile_rows, cluster;              // wide-tile kernel: cache rows per tile (64, 128, 256) and row runs merged on chip (1, 2, 4)
 };
 
 AttnPlan plan_attention(const void *Q, const void *cache, int H, int n_rows, int kv_lora);
@@ -79,6 +81,12 @@ int attention_tc64_max_clusters(int cluster);      // clusters of that many CTAs
 int attention_partial_tc64(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split, int nsplit,
                            int cluster /* splits merged on chip: 4, 2 or 1 */, AttnPartials part, int slot_stride, float scale, cudaStream_t stream, bool programmatic_launch,
                            L2Prefetch prefetch);
+
+// The pass with wide score tiles (nm_attn_wide.cu): all 128 heads per CTA, tile_rows (64, 128 or 256) cache rows per
+// scores MMA, two CTAs (column halves) per row run; rows_per_split must be multiples of tile_rows.  Same partial layout.
+int attention_partial_wide(const void *Q, int nseq, const void *const *caches, const int *n_rows, const int *rows_per_split, int nsplit,
+                           int tile_rows, int cluster /* row runs merged on chip: 4, 2 or 1 */, AttnPartials part, int slot_stride, float scale,
+                           cudaStream_t stream, bool programmatic_launch, L2Prefetch prefetch);
 
 // Small-batch decode (nm_batch_kernels.cu): per-sequence rows and partial counts of one launch.
 struct BatchRows {

@@ -57,7 +57,7 @@ def test_random_step_matches_the_oracle(nm, weights, seed):
     concat = bool(rng.random() < 0.5) and layout != COL            # the concatenated down-projection is row-major or fractal
     overlap = bool(rng.random() < 0.5)
     tails, fusion, pdl = int(rng.integers(0, 3)), bool(rng.random() < 0.8), bool(rng.random() < 0.8)
-    attn = int(rng.choice([0, 0, 1, 2, 3]))
+    attn = int(rng.choice([0, 0, 1, 2, 3, 4]))
     what = f"seed {seed}: S {S} layout {layout} concat {concat} overlap {overlap} tails {tails} fusion {fusion} pdl {pdl} attention {attn}"
     h, cache_ref, r = base.oracle_step(weights, S, seed=60_000 + seed)
     cache_in = gen.mla_cache(S, DIMS, seed=60_000 + seed)
@@ -83,7 +83,7 @@ def test_random_tokens_match_the_oracle(nm, weights, seed):
     rng = np.random.default_rng(51_000 + seed)
     S = int(rng.choice([1, 2, 64, 65, 129, int(rng.integers(130, 3000)), int(rng.integers(130, 3000))]))
     concat = bool(rng.random() < 0.7)
-    attn = int(rng.choice([0, 0, 1, 2, 3]))
+    attn = int(rng.choice([0, 0, 1, 2, 3, 4]))
     h, cache_ref, r = base.oracle_step(weights, S, seed=62_000 + seed, token_seed=63_000 + seed)
     cache_in = gen.mla_cache(S, DIMS, seed=62_000 + seed)
     dw = stored(weights, ROW, concat)
@@ -104,7 +104,7 @@ def test_random_attention_stage_matches_the_oracle(nm, seed):
     lengths from one row to a few thousand, the new row through the merge or through the pass."""
     rng = np.random.default_rng(90_000 + seed)
     S = int(rng.choice([1, 2, 33, 64, 65, 128, 129, int(rng.integers(130, 6000)), int(rng.integers(130, 6000))]))
-    impl = int(rng.choice([0, 1, 2, 3]))
+    impl = int(rng.choice([0, 1, 2, 3, 4]))
     extra = bool(rng.random() < 0.5) or S == 1
     err = base.attention_case(nm, S, impl, extra, seed=91_000 + 10 * seed)
     assert err <= 2e-3, f"seed {seed}: S {S} impl {impl} extra {extra}: {err:.2e}"

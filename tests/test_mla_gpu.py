@@ -200,9 +200,26 @@ def test_attention_stage_128_heads_per_cta(nm, S, extra):
     attention_case(nm, S, 2, extra)
 
 
-@pytest.mark.parametrize("impl", [0, 3])
+@pytest.mark.parametrize("tile,runs,cluster", [(64, 0, 1), (64, 0, 2), (64, 0, 4), (128, 0, 1), (128, 0, 4), (256, 0, 1), (256, 0, 2), (256, 0, 4),
+                                               (64, 3, 1), (128, 5, 2), (256, 5, 4)])
+def test_attention_stage_wide_tiles(nm, tile, runs, cluster):
+    """The wide-tile tensor-core kernel (the default from 6144 cache rows on) forced at every length, with every tile
+    width, on-chip merges of 1, 2 and 4 row runs, one tile per CTA and several (few runs over many rows)."""
+    nm.nm_debug_set_attention_wide(tile, runs, cluster)
+    try:
+        for S in (1, 2, 63, 64, 65, 129, 257, 1000, 1024, 4096, 5000, 16384, 20000):
+            for extra in (True, False):
+                if S == 1 and not extra:
+                    continue
+                attention_case(nm, S, 4, extra)
+                nm.nm_check_status()
+    finally:
+        nm.nm_debug_set_attention_wide(0, 0, 0)
+
+
+@pytest.mark.parametrize("impl", [0, 3, 2])
 def test_attention_stage_long_sequence(nm, impl):
-    """From 65536 cache rows on the default is the 128-head kernel; the 64-head kernel stays selectable (16 tiles per CTA)."""
+    """A long sequence: the default (the wide-tile kernel, several 256-row tiles per CTA) and the two older kernels."""
     attention_case(nm, 66001, impl, True)
 
 
@@ -217,7 +234,7 @@ def test_attention_kernels_agree_on_heavy_tailed_scores(nm):
     scale = (DIMS["nope"] + dr) ** -0.5
     ref = oracle.mla_attention(f64(Q), f64(cache), dc, scale, threads=8)
     ws = torch.empty(nm.nm_mla_attention_workspace_bytes(H, S, dc), dtype=torch.uint8, device="cuda")
-    for impl in (0, 1, 2, 3):
+    for impl in (0, 1, 2, 3, 4):
         o16 = torch.zeros(H * dc, dtype=torch.int16, device="cuda")
         o32 = torch.zeros(H * dc, dtype=torch.float32, device="cuda")
         nm.nm_debug_set_attention(impl)

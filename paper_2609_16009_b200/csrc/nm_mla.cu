@@ -811,6 +811,21 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
             if (ctas <= kSMsAttn) { ragged_tiles = tau; nsplit = ceil_div(max_tiles, tau); cluster = 1; break; }
         }
     }
+    // The wide-tile kernel (all heads per CTA, two CTAs per row run): every sequence gets the same number of runs, as many as
+    // keep the whole batch in one wave of CTAs (at most 16: the partial slots of a sequence); a run goes through its rows
+    // in tiles as wide as its share of the longest sequence needs.  Runs stand alone (no on-chip merge), so the surplus
+    // CTAs of a short sequence leave at once.
+    const bool wide = (g_s.attn_impl == 0 || g_s.attn_impl == 4) && T * 2 <= kSMsAttn;
+    int wide_tile = 64;
+    if (wide) {
+        int max_rows = 1;
+        for (int t = 0; t < T; ++t) max_rows = std::max(max_rows, b->seq_lens[t] - 1);
+        const int runs_cap = std::max(1, std::min(L.slot_stride, kSMsAttn / (2 * T)));
+        const int share = ceil_div(max_rows, runs_cap);
+        wide_tile = g_s.wide_tile == 64 || g_s.wide_tile == 128 || g_s.wide_tile == 256 ? g_s.wide_tile : (share <= 64 ? 64 : (share <= 128 ? 128 : 256));
+        nsplit = std::min(runs_cap, ceil_div(max_rows, wide_tile));
+        cluster = 1; ragged_tiles = 0;
+    }
     BatchRows rows{};
     rows.slot_stride = L.slot_stride;
     const void *caches[kMaxBatch];
@@ -821,8 +836,9 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
         caches[t] = cache + base;
         n_rows[t] = b->seq_lens[t] - 1;
         rows.new_row[t] = base + (long)n_rows[t] * dkv;
-        const int tiles = ceil_div(n_rows[t], kAttnTileRows);
-        rps[t] = ragged_tiles ? ragged_tiles * kAttnTileRows : (tiles > 0 ? ceil_div(tiles, nsplit) * kAttnTileRows : kAttnTileRows);
+        const int tile_rows = wide ? wide_tile : kAttnTileRows;
+        const int tiles = ceil_div(n_rows[t], tile_rows);
+        rps[t] = ragged_tiles ? ragged_tiles * kAttnTileRows : (tiles > 0 ? ceil_div(tiles, nsplit) * tile_rows : tile_rows);
         rows.npart[t] = n_rows[t] > 0 ? ceil_div(ceil_div(n_rows[t], rps[t]), cluster) : 0;
         any_rows |= n_rows[t] > 0;
     }
@@ -873,7 +889,9 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
                 pf.range_bytes = prows * row_bytes;
             }
         }
-        if (tc64)
+        if (wide)
+            NM_TRY(attention_partial_wide(q_full, T, caches, n_rows, rps, nsplit, wide_tile, 1, part, L.slot_stride, p->softmax_scale, ms, pdl, pf));
+        else if (tc64)
             NM_TRY(attention_partial_tc64(q_full, T, caches, n_rows, rps, nsplit, cluster, part, L.slot_stride, p->softmax_scale, ms, pdl, pf));
         else
             NM_TRY(attention_partial_tc_batch(q_full, T, caches, n_rows, rps, nsplit, part, L.slot_stride, p->softmax_scale, ms, pdl, pf));

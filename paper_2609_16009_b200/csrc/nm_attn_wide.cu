@@ -1,11 +1,14 @@
 // Latent attention pass on the tensor cores with WIDE score tiles: all 128 heads per CTA, up to 256 cache rows per
 // tcgen05.mma.
 //
-// What the two older kernels (nm_attn_tc.cu, nm_attn_tc64.cu) measured: a tcgen05.mma that takes both operands from
-// shared memory costs max(A bytes / 32, B bytes / 64, MACs / 4096) clocks.  The scores S = Q * tile^T take Q as the A
-// operand, 4 KB per k-step of 16 for 128 heads: 128 clocks per MMA however few cache rows it covers (32 rows: a
-// sixteenth of the tensor rate; 64 rows with 64 heads: a quarter).  M = 128, N = 256, K = 16 is the shape at which A
-// fetch, B fetch and arithmetic all take 128 clocks, so here one scores MMA covers up to 256 cache rows.
+// What a tcgen05.mma costs here (nm_debug_mma_probe, bf16, K = 16, one issuing thread, back to back): max(50, N / 2)
+// clocks - whatever M (64 or 128), whichever operand comes from TMEM, K-major or MN-major B.  So M = 128 is the only
+// shape that uses the whole tensor pipe (M = 64 takes the same time for half the work), an MMA over fewer than 100
+// cache rows pays the 50-clock floor (the 32-row scores MMAs of nm_attn_tc.cu run at a sixth of the rate, the 64-row
+// ones of nm_attn_tc64.cu at a third, on half the heads), and the scores S = Q * tile^T want all 128 heads and as
+// many cache rows per instruction as TMEM has columns for: up to 256 here.  With the MMAs that cheap, what bounds the
+// pass is the traffic from L2 into shared memory - Q (147 KB) once per CTA, every cache row once per column half
+// and once more for P * V - and the exponentials.
 //
 // Per CTA: one run of cache rows x one half of the 512 output columns x all 128 heads (O[128 x 256] fp32 is half of
 // TMEM; the other half holds S[128 x R], R = 64, 128 or 256 rows per tile).  Nothing is resident in shared memory:
@@ -16,13 +19,15 @@
 //            operands), four MMAs M128 N=R K16 each
 //   P * V    R/64 stages with a V slab [64 rows x 256 columns of this CTA's half] (the same bytes read MN-major), per
 //            slab four k-steps x two bf16 terms of P (hi + lo, about 16 bits of P) = eight MMAs M128 N256 K16, A from TMEM
-// The second read of a row comes from L2.  One thread per head does the softmax: a first pass over S for the row
+// The second read of a row comes from L2.  The softmax of a head: a first pass over S for the row
 // maximum (updated lazily: O is rescaled only when a maximum grows by more than 2^8), a second pass that writes P
-// over the very columns of S it has just read, 32 rows at a time (hi in the first 16 columns, lo in the next 16),
+// over the very columns of S it has just read, 16 rows at a time (hi in the first 8 columns, lo in the next 8),
 // and signals every 64 rows so that P * V of the first slab runs while the rest of the tile is still in the
-// exponentials.  The CTAs of a cluster (1, 2 or 4 row runs) merge their results through distributed shared memory as
-// in the older kernels.  Every wait is bounded (mbar_wait); on expiry the CTA raises the status word, skips the
-// remaining waits, frees its TMEM and returns.
+// exponentials.  One thread per head (kSets = 1; with two, the head's threads alternate over the 32-row chunks and
+// exchange maxima and sums through shared memory - measured slower per step, 84.0 against 82.7 us at 16384 rows, although
+// the exponentials go faster).  A run on its own leaves as one partial by tiled TMA stores; the CTAs of a cluster (2 or 4
+// row runs) merge their results through distributed shared memory first, as in the older kernels.  Every wait is bounded
+// (mbar_wait); on expiry the CTA raises the status word, skips the remaining waits, frees its TMEM and returns.
 #include "nm_async.cuh"
 #include "nm_mla.cuh"
 #include "nm_tcgen05.cuh"
@@ -45,7 +50,10 @@ constexpr int kSubBlockBytes = kSlabRows * 128;       // one [64 rows x 64 colum
 __host__ __device__ constexpr int stage_bytes(int R) { return kQBlockBytes + R * 128 > kSlabBytes ? kQBlockBytes + R * 128 : kSlabBytes; }
 constexpr int kMaxStages = 6;
 constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 256 /* barriers */;
-constexpr int kThreads = 224;             // TMA, MMA, 4 softmax warps, weight prefetch
+constexpr int kSets = 1;                  // softmax threads per head
+constexpr int kSoftmaxThreads = 128 * kSets;
+constexpr int kThreads = 64 + kSoftmaxThreads + 32;      // TMA, MMA, kSets x 4 softmax warps, weight prefetch
+constexpr int kPrefetchWarp = 2 + 4 * kSets;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 0, kColS = 256;            // O fp32 [128 x 256]; S fp32 [128 x R], P over it
 constexpr float kLazyThreshold = 8.0f;    // log2 units
@@ -100,7 +108,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 
 // kR: cache rows per tile (one scores MMA covers them all); kCl: row runs merged on chip (cluster size)
 template <int kR, int kCl>
-__global__ void __maxnreg__(120)
+__global__ void __maxnreg__(80)
 attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ WideSeqs seqs, AttnPartials part,
                  float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
 {
@@ -134,6 +142,7 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     __shared__ int s_abort;
     __shared__ __align__(8) float s_mlp[kCl][kHeadsPerRank][2];   // (m in log2 units, l) of the owned heads, written by each peer
     __shared__ float s_w[kCl][kHeadsPerRank];                     // weights of the slots in the final sum
+    __shared__ float s_pair[2][kHeads];                           // what the two softmax threads of a head tell each other
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sp = blockIdx.x, half = blockIdx.y;
@@ -149,7 +158,7 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         s_abort = 0;
         for (int b = 0; b < kStages; ++b) { mbar_init(bar_full + 8 * b, 1); mbar_init(bar_empty + 8 * b, 1); }
         mbar_init(bar_s_full, 1);
-        for (int q = 0; q < kMaxSlabs; ++q) mbar_init(bar_p_ready + 8 * q, 128);
+        for (int q = 0; q < kMaxSlabs; ++q) mbar_init(bar_p_ready + 8 * q, kSoftmaxThreads);
         mbar_init(bar_pv_done, 1);
         mbar_init_fence();
     }
@@ -253,22 +262,24 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                          mbar_wait(bar_p_ready + 8 * q, t & 1, &s_abort, status);
                     if (!ok) break;
                     tc_fence_after();
+                    if (t == 0) NM_TRACE(12 + q);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        // rows 64 q + 16 kk ..: chunk 2 q + kk / 2 of P, its first or second 16 rows (8 columns of bf16 pairs)
-                        const uint32_t p_hi = tmem + kColS + 32 * (2 * q + (kk >> 1)) + 8 * (kk & 1), p_lo = p_hi + 16;
+                        // rows 64 q + 16 kk ..: P sits over the 16 columns of S it came from, hi in the first 8 (bf16 pairs), lo in the next 8
+                        const uint32_t p_hi = tmem + kColS + 16 * (4 * q + kk), p_lo = p_hi + 8;
                         const uint64_t vdesc = smem_desc(ring_addr + b * kStageBytes + kk * 2048, kSubBlockBytes, 1024);
                         mma_ts(tmem + kColO, p_hi, vdesc, idesc_o, (t | q | kk) != 0);
                         mma_ts(tmem + kColO, p_lo, vdesc, idesc_o, true);
                     }
                     mma_commit(bar_empty + 8 * b);
+                    if (t == 0) NM_TRACE(16 + q);
                     ++item;
                 }
                 if (!ok) break;
                 mma_commit(bar_pv_done);
             }
         }
-    } else if (warp == 6) {
+    } else if (warp == kPrefetchWarp) {
         // ---------------- weight prefetch (launched only when there is something to prefetch) ----------------------
         if (ntiles > 0) {                                          // sleep-poll: this warp must not take issue slots from the pipeline
             const uint64_t t0 = global_timer_ns();
@@ -297,116 +308,167 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             n &= ~15L;
             if (n > 0) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr), "r"((uint32_t)n) : "memory");
         }
-    } else {
-        // ---------------- one head per thread: softmax, lazy rescale ------------------------------------------
-        const int quad = warp & 3;                                 // TMEM lanes this warp may touch
+    } else if (warp >= 2 && warp < 2 + 4 * kSets) {
+        // ---------------- softmax, lazy rescale: two threads per head (warps 2-5 take the even 32-row chunks of a tile,
+        //                  warps 6-9 the odd ones; warp w may touch the TMEM lanes of quarter w % 4) -----------------
+        const int set = (warp - 2) >> 2, quad = warp & 3, head = quad * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
         float m_used = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int t = 0; t < ntiles && ok; ++t) {
-            ok = mbar_wait(bar_s_full, t & 1, &s_abort, status);
-            if (!ok) break;
+        for (int t = 0; t < ntiles; ++t) {
+            // (after an expired wait every later wait returns at once: the loop runs on, so that all 256 threads keep meeting
+            // at the named barriers below, and ends with a result that the status word disowns)
+            ok = mbar_wait(bar_s_full, t & 1, &s_abort, status) && ok;
             tc_fence_after();
             if (t == 0 && tid == 64) NM_TRACE(5);
             const int valid = min(kR, r1 - (r0 + t * kR));
             const int nchunks = ceil_div(valid, 32);
-            // pass 1: the row maximum of this tile
+            // pass 1: the row maximum of this tile, each thread over its chunks, then both together
             float mx = -INFINITY;
-            for (int j = 0; j < nchunks; ++j) {
-                uint32_t sr[32];
-                tmem_ld32(lane_base + kColS + 32 * j, sr);
-                tmem_wait_ld();
+            {
+                float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;      // four chains instead of one
+                for (int j = set; j < nchunks; j += kSets) {
+                    uint32_t sa[16], sb[16];                        // both halves of the chunk requested before either is used
+                    tmem_ld16(lane_base + kColS + 32 * j, sa);
+                    tmem_ld16(lane_base + kColS + 32 * j + 16, sb);
+                    tmem_wait_ld();
+                    if (32 * j + 32 <= valid) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (32 * j + i < valid) mx = fmaxf(mx, __uint_as_float(sr[i]));
+                        for (int i = 0; i < 16; i += 2) {
+                            m0 = fmaxf(m0, __uint_as_float(sa[i])); m1 = fmaxf(m1, __uint_as_float(sa[i + 1]));
+                            m2 = fmaxf(m2, __uint_as_float(sb[i])); m3 = fmaxf(m3, __uint_as_float(sb[i + 1]));
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            if (32 * j + i < valid) m0 = fmaxf(m0, __uint_as_float(sa[i]));
+                            if (32 * j + 16 + i < valid) m2 = fmaxf(m2, __uint_as_float(sb[i]));
+                        }
+                    }
+                }
+                mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+            }
+            if constexpr (kSets == 2) {
+                s_pair[set][head] = mx;
+                named_barrier_sync(2, kSoftmaxThreads);
+                mx = fmaxf(s_pair[0][head], s_pair[1][head]);
             }
             const float mx2 = mx * scale_log2;
             const bool grow = (t == 0) || (mx2 > m_used + kLazyThreshold);
             // s_full of this tile was committed behind the P*V of the previous one: O is at rest
             if (t > 0 && __any_sync(0xffffffffu, grow)) {
-                // rare: the maximum grew by more than 2^8
+                // rare: the maximum grew by more than 2^8; each of the head's two threads rescales half of the columns
                 const float f = grow ? fast_exp2(m_used - mx2) : 1.0f;
-                for (int c = 0; c < kDvHalf / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(lane_base + kColO + c * 32, o);
+                for (int c = (16 / kSets) * set; c < (16 / kSets) * (set + 1); ++c) {
+                    uint32_t o[16];
+                    tmem_ld16(lane_base + kColO + c * 16, o);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                    tmem_st32(lane_base + kColO + c * 32, o);
+                    for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                    tmem_st16(lane_base + kColO + c * 16, o);
                 }
                 tmem_wait_st();
                 if (grow) l *= f;
             }
             if (grow) m_used = mx2;
             if (t == 0 && tid == 64) NM_TRACE(6);
-            // pass 2: P over the columns of S just read, 32 rows at a time; a signal every 64 rows
-            float lsum = 0.f;
-            for (int j = 0; j < 2 * slabs_of(t); ++j) {
-                uint32_t sr[32], pr[16], plo[16];
-                tmem_ld32(lane_base + kColS + 32 * j, sr);
+            // pass 2: P over the columns of S just read, 16 rows at a time (hi in the first 8 columns, lo in the next 8);
+            // a signal from every thread per 64-row slab, whether or not it had a chunk of it
+            float lsum = 0.f, lsum1 = 0.f;
+            const int ns = slabs_of(t);
+            for (int j = set; j < 2 * ns; j += kSets) {
+                uint32_t sr[32];
+                const uint32_t col = lane_base + kColS + 32 * j;
+                tmem_ld16(col, reinterpret_cast<uint32_t (&)[16]>(sr[0]));
+                tmem_ld16(col + 16, reinterpret_cast<uint32_t (&)[16]>(sr[16]));
                 tmem_wait_ld();
+                const bool full = 32 * j + 32 <= valid;
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float p0 = (32 * j + i < valid) ? fast_exp2(fmaf(__uint_as_float(sr[i]), scale_log2, -m_used)) : 0.f;
-                    const float p1 = (32 * j + i + 1 < valid) ? fast_exp2(fmaf(__uint_as_float(sr[i + 1]), scale_log2, -m_used)) : 0.f;
-                    lsum += p0 + p1;
-                    const uint32_t hi = pack_bf16x2(p0, p1);
-                    pr[i >> 1] = hi;
-                    plo[i >> 1] = pack_bf16x2(p0 - __uint_as_float(hi << 16), p1 - __uint_as_float(hi & 0xffff0000u));
+                for (int hq = 0; hq < 2; ++hq) {
+                    uint32_t pr[8], plo[8];
+                    const int row0 = 32 * j + 16 * hq;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(sr[16 * hq + i]), scale_log2, -m_used));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(sr[16 * hq + i + 1]), scale_log2, -m_used));
+                        if (!full) {
+                            if (row0 + i >= valid) p0 = 0.f;
+                            if (row0 + i + 1 >= valid) p1 = 0.f;
+                        }
+                        lsum += p0; lsum1 += p1;
+                        // P = hi + lo in two bf16 terms, both by truncation (a mask and a byte permute; the float-to-bf16
+                        // conversion shares the 16-lane unit with the exponentials, which bound this loop): hi keeps the top
+                        // 8 significand bits, lo the next 8 of the exact remainder - about 2^-16 relative, from below
+                        const uint32_t u0 = __float_as_uint(p0), u1 = __float_as_uint(p1);
+                        const float r0 = p0 - __uint_as_float(u0 & 0xffff0000u), r1 = p1 - __uint_as_float(u1 & 0xffff0000u);
+                        pr[i >> 1] = __byte_perm(u0, u1, 0x7632);
+                        plo[i >> 1] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+                    }
+                    tmem_st8(col + 16 * hq, pr);
+                    tmem_st8(col + 16 * hq + 8, plo);
                 }
-                tmem_st16(lane_base + kColS + 32 * j, pr);
-                tmem_st16(lane_base + kColS + 32 * j + 16, plo);
-                if (j & 1) {
+                if (kSets == 2 || (j & 1)) {                        // this thread's part of the 64-row slab is written
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(bar_p_ready + 8 * (j >> 1));
-                    if (t == 0 && tid == 64 && j == 1) NM_TRACE(7);
+                    if (t == 0 && tid == 64) NM_TRACE((j >> 1) == 0 ? 7 : 19 + (j >> 1));
                 }
             }
+            lsum += lsum1;
             l += lsum;
             if (t == 0 && tid == 64) NM_TRACE(8);
             // the next tile's scores overwrite P: they are issued behind this tile's P*V, nothing to wait for here
         }
         // the last P*V must have landed before O is read
-        if (ntiles > 0 && ok) {
+        if (ntiles > 0) {
             mbar_wait(bar_pv_done, (ntiles - 1) & 1, &s_abort, status);
             tc_fence_after();
         }
+        (void)ok;
         if (tid == 64) NM_TRACE_CTA(2);
+        // the head's sum: first thread's chunks, then the second's (fixed order)
         m_own = m_used; l_own = l;
+        if constexpr (kSets == 2) {
+            s_pair[set][head] = l;
+            named_barrier_sync(2, kSoftmaxThreads);
+            l_own = s_pair[0][head] + s_pair[1][head];
+        }
     }
 
     // ---- a run on its own (cluster of one): its O rows go out as one partial through shared memory and tiled TMA
     //      stores - eight [128 heads x 32 columns] boxes in the 128-byte swizzle, written one row per thread without
     //      bank conflicts and copied out by the copy engine while the next box is being filled ----------------------
     if constexpr (kCl == 1) {
-        if (warp >= 2 && warp < 6) {
-            const int quad = warp & 3, head = quad * 32 + lane;
+        if (warp >= 2 && warp < 2 + 4 * kSets) {
+            const int set = (warp - 2) >> 2, quad = warp & 3, head = quad * 32 + lane;
             const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
-            if (half == 0) {
+            if (half == 0 && set == 0) {
                 part.ml[((size_t)sp * kHeads + head) * 2] = m_own * 0.6931471805599453f;       // natural-log units
                 part.ml[((size_t)sp * kHeads + head) * 2 + 1] = l_own;
             }
-            for (int c = 0; c < kDvHalf / 32; ++c) {
-                uint32_t o[32];
-                tmem_ld32(lane_base + kColO + c * 32, o);
-                tmem_wait_ld();
+            for (int c = (8 / kSets) * set; c < (8 / kSets) * (set + 1); ++c) {          // each of the head's threads moves its share of the columns
                 const uint32_t row = park_addr + (uint32_t)c * 16384u + (uint32_t)head * 128u;
 #pragma unroll
-                for (int i = 0; i < 32; i += 4)
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((uint32_t)(i / 4) ^ ((uint32_t)head & 7u)) * 16u),
-                                 "r"(o[i]), "r"(o[i + 1]), "r"(o[i + 2]), "r"(o[i + 3]) : "memory");
+                for (int hq = 0; hq < 2; ++hq) {
+                    uint32_t o[16];
+                    tmem_ld16(lane_base + kColO + c * 32 + hq * 16, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((uint32_t)(hq * 4 + i / 4) ^ ((uint32_t)head & 7u)) * 16u),
+                                     "r"(o[i]), "r"(o[i + 1]), "r"(o[i + 2]), "r"(o[i + 3]) : "memory");
+                }
                 fence_proxy_async();
-                named_barrier_sync(1, 128);
-                if (tid == 64) {
+                named_barrier_sync(3 + set, 128);
+                if (lane == 0 && quad == 2) {                      // threads 64 and 192
                     tma_store_2d(&seqs.o, half * kDvHalf + 32 * c, seq * seqs.o_rows_per_seq + sp * kHeads, park_addr + (uint32_t)c * 16384u);
                     bulk_commit_group();
                 }
             }
-            if (tid == 64) {
-                NM_TRACE(24);
+            if (lane == 0 && quad == 2) {
+                if (tid == 64) NM_TRACE(24);
                 bulk_wait_all();
-                NM_TRACE(27);
+                if (tid == 64) NM_TRACE(27);
             }
         }
         tc_fence_before();
@@ -431,19 +493,21 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // last barrier keeps every CTA's shared memory alive until its peers have read it.
     __syncwarp();
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");       // all peers are running (they arrived at kernel start)
-    if (warp >= 2 && warp < 6) {
-        const int quad = warp & 3, head = quad * 32 + lane;
+    if (warp >= 2 && warp < 2 + 4 * kSets) {
+        const int set = (warp - 2) >> 2, quad = warp & 3, head = quad * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
-        const uint32_t slot = peer_smem(smem_u32(&s_mlp[rank][head % kHeadsPerRank][0]), (uint32_t)head / kHeadsPerRank);
-        asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(slot), "f"((ntiles > 0) ? m_own : -INFINITY), "f"(l_own) : "memory");
+        if (set == 0) {
+            const uint32_t slot = peer_smem(smem_u32(&s_mlp[rank][head % kHeadsPerRank][0]), (uint32_t)head / kHeadsPerRank);
+            asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(slot), "f"((ntiles > 0) ? m_own : -INFINITY), "f"(l_own) : "memory");
+        }
         if (ntiles > 0) {
-            for (int c = 0; c < kDvHalf / 32; ++c) {
-                uint32_t o[32];
-                tmem_ld32(lane_base + kColO + c * 32, o);
+            for (int c = (16 / kSets) * set; c < (16 / kSets) * (set + 1); ++c) {          // each of the head's threads parks its share of the columns
+                uint32_t o[16];
+                tmem_ld16(lane_base + kColO + c * 16, o);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    const uint32_t q4 = (uint32_t)(c * 8 + i / 4);
+                for (int i = 0; i < 16; i += 4) {
+                    const uint32_t q4 = (uint32_t)(c * 4 + i / 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(park_addr + (uint32_t)(head * 64 + (q4 ^ (head & 7u))) * 16u),
                                  "r"(o[i]), "r"(o[i + 1]), "r"(o[i + 2]), "r"(o[i + 3]) : "memory");
                 }
@@ -453,9 +517,9 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     cluster_sync_all();                                            // every peer's rows and (m, l) are parked
     if (tid == 64) NM_TRACE(25);
-    if (warp >= 2 && warp < 6) {
-        const int t = tid - 64;                                    // 0..127
-        {                                                          // weight of peer r for owned head hl
+    if (warp >= 2 && warp < 2 + 4 * kSets) {
+        const int t = tid - 64;                                    // 0..kSoftmaxThreads-1
+        if (t < 128) {                                             // weight of peer r for owned head hl
             const int hl = t % kHeadsPerRank, r = t / kHeadsPerRank, head = (int)rank * kHeadsPerRank + hl;
             float pm[kCl], pl[kCl], M = -INFINITY;
 #pragma unroll
@@ -472,14 +536,14 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 part.ml[((size_t)cluster_id * kHeads + head) * 2 + 1] = Ltot;
             }
         }
-        named_barrier_sync(1, 128);
+        named_barrier_sync(2, kSoftmaxThreads);
         if (tid == 64) NM_TRACE(26);
-        constexpr int kIters = kHeadsPerRank * 64 / 128, kBatch = (kCl == 4) ? 4 : 8;
+        constexpr int kIters = kHeadsPerRank * 64 / kSoftmaxThreads, kBatch = 4;
         for (int i0 = 0; i0 < kIters; i0 += kBatch) {
             float4 v[kBatch][kCl];
 #pragma unroll
             for (int b = 0; b < kBatch; ++b) {                     // kBatch * kCl remote loads in flight
-                const int idx = t + 128 * (i0 + b);
+                const int idx = t + kSoftmaxThreads * (i0 + b);
                 const int hl = idx / 64, q4 = idx % 64, head = (int)rank * kHeadsPerRank + hl;
                 const uint32_t local = park_addr + (uint32_t)(head * 64 + (q4 ^ (head & 7))) * 16u;
 #pragma unroll
@@ -488,7 +552,7 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
 #pragma unroll
             for (int b = 0; b < kBatch; ++b) {
-                const int idx = t + 128 * (i0 + b);
+                const int idx = t + kSoftmaxThreads * (i0 + b);
                 const int hl = idx / 64, q4 = idx % 64, head = (int)rank * kHeadsPerRank + hl;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -546,7 +610,7 @@ int launch_wide(const CUtensorMap &map_q, const WideSeqs &seqs, int nseq, int ns
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ceil_div(nsplit, kCl) * kCl, 2, nseq);      // padded to whole clusters; padding CTAs have no rows
     const bool has_prefetch = prefetch.block_bytes > 0 || (prefetch.nranges > 0 && prefetch.range_bytes > 0);
-    cfg.blockDim = dim3(has_prefetch ? kThreads : kThreads - 32);
+    cfg.blockDim = dim3(has_prefetch ? kThreads : kThreads - 32);       // the prefetch warp is the last one
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];

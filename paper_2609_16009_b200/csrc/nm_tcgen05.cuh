@@ -103,6 +103,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&r)[16]
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+}
 // Half-split shapes (.16x32bx2) for accumulators of M = 64, whose rows sit in lanes 0-15 of each 32-lane quarter:
 // thread l < 16 of the warp moves kN columns of TMEM lane l from `addr`, thread l + 16 the kN columns of the SAME
 // lane that start kSplit columns further on - both halves of the warp work on the 16 rows.

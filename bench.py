@@ -745,7 +745,9 @@ def main():
     ap.add_argument("--seq-len", type=int, default=16384, help="cache rows of the headline step (default: the largest configuration)")
     ap.add_argument("--single-length", action="store_true", help="skip the step at the other sequence lengths (1024, 4096, 16384)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the narrow-product-vs-M measurements")
-    ap.add_argument("--batch", type=int, default=1, help="with --timeline: sequences of the small-batch step (2-16) to trace")
+    ap.add_argument("--single-block", action="store_true", help="time one block of --steps steps only (no repetition up to half a second): for traces")
+    ap.add_argument("--no-extras", action="store_true", help="skip graph replay, the small-batch step and the step without W_O")
+    ap.add_argument("--batch", type=int, default=1, help="sequences of the small-batch step (2-16) to run instead of the single-token step (captures, --timeline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--weights", default="row", choices=["row", "fractal"],
                     help="storage of the step's dense weights: row-major (default) or the paper's FRACTAL_NZ tiling")
@@ -776,6 +778,16 @@ def main():
     nm.nm_debug_set_attention({"auto": 0, "cuda-cores": 1, "128": 2, "64": 3}[args.attention])
     wl = make_workload(args, nm, device)
     stream = torch.cuda.Stream(device)
+    if args.batch > 1 and not args.timeline:
+        # the small-batch step as the workload (for kernel-level captures; extras and the other lengths are skipped)
+        if args.workload != "mla" or args.weights != "row":
+            raise SystemExit("--batch goes with --workload mla and row-major weights")
+        fn, keep = wl.batch_step(args.batch, stream)
+        wl.step = lambda stream_, dom_events=None: fn()
+        wl.step_e2e = lambda stream_: fn()
+        wl.extra_measurements = lambda stream_: {}
+        wl.launches_per_step = 0
+        args.single_length = args.no_sweep = True
     if args.timeline:
         with torch.cuda.stream(stream):
             if args.batch > 1:                # the timeline of the small-batch step instead of the single-token step
@@ -818,7 +830,7 @@ def main():
         #      rank), and the MEDIAN block is reported; nothing but the steps is enqueued inside a block ------------
         first = timed_block(lambda: wl.step(stream), args.steps)
         (first_max,) = reduce_over_ranks([first], dist, device)
-        n_blocks = 1 if first_max >= 500.0 else int(min(200, max(3, -(-500.0 // max(first_max, 1e-3)))))
+        n_blocks = 1 if (first_max >= 500.0 or args.single_block) else int(min(200, max(3, -(-500.0 // max(first_max, 1e-3)))))
         blocks = [first] + [timed_block(lambda: wl.step(stream), args.steps) for _ in range(n_blocks - 1)]
         # ---- the dominant kernel, in a SEPARATE pass after the timed region: events around it on the launching
         #      stream in every step (the events switch off that kernel's programmatic launch, which is why they are
@@ -844,7 +856,7 @@ def main():
         t1.record(stream)
         barrier()
         e2e_ms = t0.elapsed_time(t1)
-        extras = wl.extra_measurements(stream) if hasattr(wl, "extra_measurements") else {}
+        extras = wl.extra_measurements(stream) if (hasattr(wl, "extra_measurements") and not args.no_extras) else {}
         # ---- the step at the other sequence lengths of the configuration (same resident weights) ------------------
         per_len = []
         if args.workload == "mla" and not args.single_length:

@@ -2,6 +2,10 @@
  * nm_debug.h - tuning aids and test hooks of the nm library (sweeps, forced plans, traces, the bounded-wait probe).
  * Not needed for normal use; include/nm.h is the boundary proper.  All settings here are process-wide, guarded by a
  * lock, and read once per call (see "Thread safety" in nm.h).  The paper has no counterpart for any of these.
+ *
+ * Environment (read once, when the library is loaded): NM_LOG=1 prints the plan of every product (kernel family, tile
+ * width, k-splits, ring depth) to stderr; NM_FORCE_KERNEL, NM_STAGES, NM_TILE_N and NM_SPLITK give nm_debug_set_kernel /
+ * nm_debug_set_plan their initial values.
  */
 #ifndef NM_DEBUG_H
 #define NM_DEBUG_H

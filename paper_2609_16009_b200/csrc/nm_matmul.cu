@@ -45,7 +45,27 @@ struct MatmulTuning {
     int tc_min_m = 3;               // row-major bf16 products with M >= this (and >= 32 MB of weights) go to the swap-AB tensor-core kernel
 };
 static std::mutex g_tuning_mutex;
-static MatmulTuning g_tuning_shared;
+// Environment, read once when the library is loaded: NM_FORCE_KERNEL (kernel family as nm_debug_set_kernel: 0 plain-load,
+// 3 TMA ring, 4 swap-AB tensor cores), NM_STAGES (ring depth), NM_TILE_N and NM_SPLITK (as nm_debug_set_plan) give the
+// tuning settings their initial values; NM_LOG=1 prints the plan of every product to stderr.
+static int env_int(const char *name, int fallback, int lo, int hi)
+{
+    const char *v = getenv(name);
+    if (!v || !*v) return fallback;
+    const long x = strtol(v, nullptr, 10);
+    return (x < lo || x > hi) ? fallback : (int)x;
+}
+static MatmulTuning tuning_from_environment()
+{
+    MatmulTuning t;
+    t.force_kind = env_int("NM_FORCE_KERNEL", -1, -1, 4);
+    t.force_stages = env_int("NM_STAGES", 0, 0, 16);
+    t.force_tn = env_int("NM_TILE_N", 0, 0, kMaxTileN);
+    t.force_split = env_int("NM_SPLITK", 0, 0, kMaxSplit);
+    return t;
+}
+static MatmulTuning g_tuning_shared = tuning_from_environment();
+static const bool g_log_plans = env_int("NM_LOG", 0, 0, 1) != 0;
 struct PlanOverride { bool active = false; int tn = 0, split = 0, stages = 0; };
 static thread_local PlanOverride g_plan_override;      // a plan forced for this thread's next products only
 static thread_local MatmulTuning g_t;                  // the calling thread's snapshot
@@ -379,6 +399,10 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     if (g_t.force_kind == kRowVec && layout != NM_FRACTAL_NZ) tma_ok = false;      // the fractal storage has one kernel: nothing to force
     if (layout == NM_FRACTAL_NZ && !tma_ok) return NM_ERR_UNSUPPORTED;      // unaligned operands or no tensor-map encoder
     Plan p = make_plan(M, N, K, H, dtype, layout, vec_ok, tma_ok, chained);
+    if (g_log_plans && !(extras && extras->dry_run))
+        fprintf(stderr, "nm: M=%d N=%d K=%d H=%d dtype=%d layout=%d -> kernel %d (0 row, 1 column, 2 scalar, 3 TMA ring, 4 tensor cores) tile_n=%d "
+                "k-splits=%d k-rows=%d tiles=%d stages=%d%s\n", M, N, K, H, (int)dtype, (int)layout, (int)p.kind, p.tn, p.nsplit, p.kr, p.ntiles, p.nstage,
+                chained ? " chained" : "");
     // Copies, not pointers into the map cache: the second lookup may evict the entry the first one returned
     // (16 entries, replaced in turn), and the kernel would then get the token map in place of the weight map.
     CUtensorMap tc_map_b_copy, tc_map_a_copy;

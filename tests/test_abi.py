@@ -133,3 +133,20 @@ def test_tuning_state_is_safe_under_concurrent_host_threads(lib):
     assert not errors
     for s_ in seen:
         assert s_ <= want, f"torn plan: {s_ - want}"
+
+
+def test_environment_gives_the_tuning_settings_their_initial_values():
+    """NM_TILE_N / NM_SPLITK / NM_FORCE_KERNEL / NM_STAGES are read when the library is loaded (a fresh process here)."""
+    import subprocess
+    import sys
+    code = ("import ctypes, sys; lib = ctypes.CDLL(sys.argv[1]); out = (ctypes.c_int * 6)();"
+            "assert lib.nm_debug_get_plan(1, 4096, 8192, 1, 1, 0, 1, out) == 0; print(list(out))")
+    from paper_2609_16009_b200 import build
+    path = build.build()
+    env = dict(os.environ, NM_TILE_N="64", NM_SPLITK="3", NM_FORCE_KERNEL="3")
+    forced = subprocess.run([sys.executable, "-c", code, path], env=env, capture_output=True, text=True, check=True).stdout
+    kind, tn, ns = eval(forced)[:3]
+    assert (kind, tn, ns) == (3, 64, 3), forced
+    plain = subprocess.run([sys.executable, "-c", code, path], env={k: v for k, v in os.environ.items() if not k.startswith("NM_")},
+                           capture_output=True, text=True, check=True).stdout
+    assert eval(plain)[:3] != [3, 64, 3]

@@ -108,7 +108,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 
 // kR: cache rows per tile (one scores MMA covers them all); kCl: row runs merged on chip (cluster size)
 template <int kR, int kCl>
-__global__ void __maxnreg__(80)
+__global__ void __maxnreg__(112)
 attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ WideSeqs seqs, AttnPartials part,
                  float scale_log2, unsigned *status, unsigned long long *trace, const L2Prefetch pf)
 {
@@ -376,12 +376,20 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // a signal from every thread per 64-row slab, whether or not it had a chunk of it
             float lsum = 0.f, lsum1 = 0.f;
             const int ns = slabs_of(t);
+            uint32_t sr[32], nx[32];                                // this chunk's scores, and the next chunk's on their way
+            if (set < 2 * ns) {
+                tmem_ld16(lane_base + kColS + 32 * set, reinterpret_cast<uint32_t (&)[16]>(nx[0]));
+                tmem_ld16(lane_base + kColS + 32 * set + 16, reinterpret_cast<uint32_t (&)[16]>(nx[16]));
+            }
             for (int j = set; j < 2 * ns; j += kSets) {
-                uint32_t sr[32];
                 const uint32_t col = lane_base + kColS + 32 * j;
-                tmem_ld16(col, reinterpret_cast<uint32_t (&)[16]>(sr[0]));
-                tmem_ld16(col + 16, reinterpret_cast<uint32_t (&)[16]>(sr[16]));
                 tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) sr[i] = nx[i];
+                if (j + kSets < 2 * ns) {                          // requested before this chunk's exponentials, used after them
+                    tmem_ld16(col + 32 * kSets, reinterpret_cast<uint32_t (&)[16]>(nx[0]));
+                    tmem_ld16(col + 32 * kSets + 16, reinterpret_cast<uint32_t (&)[16]>(nx[16]));
+                }
                 const bool full = 32 * j + 32 <= valid;
 #pragma unroll
                 for (int hq = 0; hq < 2; ++hq) {

@@ -454,22 +454,32 @@ attn_wide_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 part.ml[((size_t)sp * kHeads + head) * 2] = m_own * 0.6931471805599453f;       // natural-log units
                 part.ml[((size_t)sp * kHeads + head) * 2 + 1] = l_own;
             }
-            for (int c = (8 / kSets) * set; c < (8 / kSets) * (set + 1); ++c) {          // each of the head's threads moves its share of the columns
-                const uint32_t row = park_addr + (uint32_t)c * 16384u + (uint32_t)head * 128u;
+            // each of the head's threads moves its share of the columns, kBoxGroup boxes between barriers: the loads of a
+            // group are all requested before the first is used, and the copy engine works on one group while the next is filled
+            constexpr int kBoxGroup = 4;
+            for (int c0 = (8 / kSets) * set; c0 < (8 / kSets) * (set + 1); c0 += kBoxGroup) {
+                uint32_t o[2][32];
+                tmem_ld16(lane_base + kColO + c0 * 32, reinterpret_cast<uint32_t (&)[16]>(o[0][0]));
+                tmem_ld16(lane_base + kColO + c0 * 32 + 16, reinterpret_cast<uint32_t (&)[16]>(o[0][16]));
 #pragma unroll
-                for (int hq = 0; hq < 2; ++hq) {
-                    uint32_t o[16];
-                    tmem_ld16(lane_base + kColO + c * 32 + hq * 16, o);
+                for (int g = 0; g < kBoxGroup; ++g) {
+                    const int c = c0 + g;
                     tmem_wait_ld();
+                    if (g + 1 < kBoxGroup) {
+                        tmem_ld16(lane_base + kColO + (c + 1) * 32, reinterpret_cast<uint32_t (&)[16]>(o[(g + 1) & 1][0]));
+                        tmem_ld16(lane_base + kColO + (c + 1) * 32 + 16, reinterpret_cast<uint32_t (&)[16]>(o[(g + 1) & 1][16]));
+                    }
+                    const uint32_t row = park_addr + (uint32_t)c * 16384u + (uint32_t)head * 128u;
 #pragma unroll
-                    for (int i = 0; i < 16; i += 4)
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((uint32_t)(hq * 4 + i / 4) ^ ((uint32_t)head & 7u)) * 16u),
-                                     "r"(o[i]), "r"(o[i + 1]), "r"(o[i + 2]), "r"(o[i + 3]) : "memory");
+                    for (int i = 0; i < 32; i += 4)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((uint32_t)(i / 4) ^ ((uint32_t)head & 7u)) * 16u),
+                                     "r"(o[g & 1][i]), "r"(o[g & 1][i + 1]), "r"(o[g & 1][i + 2]), "r"(o[g & 1][i + 3]) : "memory");
                 }
                 fence_proxy_async();
                 named_barrier_sync(3 + set, 128);
                 if (lane == 0 && quad == 2) {                      // threads 64 and 192
-                    tma_store_2d(&seqs.o, half * kDvHalf + 32 * c, seq * seqs.o_rows_per_seq + sp * kHeads, park_addr + (uint32_t)c * 16384u);
+                    for (int c = c0; c < c0 + kBoxGroup; ++c)
+                        tma_store_2d(&seqs.o, half * kDvHalf + 32 * c, seq * seqs.o_rows_per_seq + sp * kHeads, park_addr + (uint32_t)c * 16384u);
                     bulk_commit_group();
                 }
             }

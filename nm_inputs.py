@@ -7,7 +7,7 @@ generator, scales them, and casts them to the storage type.  bf16 tensors are re
 Recipe (shapes and distributions of the paper's workload, the DeepSeek-V3 MLA operator on one
 token; trained weights are replaced by seeded random tensors):
   * fp32 GEMV: A 1x512, B 512x512, uniform[-1, 1], seed 0;
-  * bf16 products: A ~ N(0,1), B ~ N(0, 0.02^2);
+  * bf16 products (and the optional fp16 ones): A ~ N(0,1), B ~ N(0, 0.02^2);
   * MLA step: weights ~ N(0, 0.02^2), gamma ~ 1 + N(0, 0.02^2), h ~ N(0,1), cache rows ~ N(0,1).
 Seeds: ``1000 * config_index + tensor_index`` unless given.
 """
@@ -81,6 +81,15 @@ def narrow_bf16(M: int, K: int, N: int, seed: int):
     A = normal_bf16((M, K), 1.0, seed)
     B = normal_bf16((K, N), 0.02, seed + 1)
     return A, B
+
+
+def narrow_f16(M: int, K: int, N: int, seed: int):
+    """The same recipe stored as fp16 (IEEE binary16) bit patterns: the optional element type of the product."""
+    g = _gen(seed)
+    A = torch.randn((M, K), generator=g, dtype=torch.float32)
+    B = torch.randn((K, N), generator=g, dtype=torch.float32) * 0.02
+    to_bits = lambda t: t.to(torch.float16).contiguous().view(torch.int16).numpy().view(np.uint16).copy()
+    return to_bits(A), to_bits(B)
 
 
 def per_head(T: int, seed: int, H: int = 128, nope: int = 128, kv_lora: int = 512, v: int = 128):

@@ -2,7 +2,7 @@
 
 Loads ``nm_oracle.c`` (plain C, fp64 accumulation, built with gcc) through ctypes and
 exposes numpy-level wrappers.  Nothing here is shared with, imported by, or imports the
-CUDA path.  bf16 tensors travel as ``numpy.uint16`` bit patterns.
+CUDA path.  bf16 (and fp16) tensors travel as ``numpy.uint16`` bit patterns.
 
 Only tests, the smoke check and the bench's CPU-baseline leg may import this package.
 """
@@ -17,10 +17,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "nm_oracle.c")
 _LIB = os.path.join(_HERE, "libnm_oracle.so")
 
-F32, BF16, F64 = 0, 1, 3
+F32, BF16, F16, F64 = 0, 1, 2, 3
 ROW_MAJOR, COL_MAJOR, FRACTAL_NZ = 0, 1, 2
 
-_np_dtype = {F32: np.float32, BF16: np.uint16, F64: np.float64}
+_np_dtype = {F32: np.float32, BF16: np.uint16, F16: np.uint16, F64: np.float64}
 
 
 def build(force: bool = False) -> str:
@@ -67,6 +67,20 @@ def f64_to_bf16(x: np.ndarray) -> np.ndarray:
     x = np.ascontiguousarray(x, dtype=np.float64)
     out = np.empty(x.shape, dtype=np.uint16)
     lib().nmo_round(_ptr(x), _ptr(out), C.c_long(x.size), C.c_int(BF16))
+    return out
+
+
+def f16_to_f64(bits: np.ndarray) -> np.ndarray:
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(bits.shape, dtype=np.float64)
+    lib().nmo_widen(_ptr(bits), _ptr(out), C.c_long(bits.size), C.c_int(F16))
+    return out
+
+
+def f64_to_f16(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty(x.shape, dtype=np.uint16)
+    lib().nmo_round(_ptr(x), _ptr(out), C.c_long(x.size), C.c_int(F16))
     return out
 
 

@@ -18,6 +18,10 @@
  *                        to bfloat16 after accumulation (Data Type Issue section) gives the
  *                        rounding point after every matmul.
  *
+ * The optional fp16 element type of the product (the paper uses bf16 data; fp16 appears there only as a type pun)
+ * follows the same definition with binary16 widening and one binary16 rounding; pinned by all 65536 bit patterns
+ * and by roundings (ties, subnormals, overflow) against hand values and numpy's float16.
+ *
  * Pins (tests, CPU only): hand-computed 1x3 * 3x2 case in both layouts; brute force
  * against int64 on all shapes <= 4; small-integer exactness at K=7168; rounding ties
  * 257 -> 256 and 259 -> 260; identity / one-hot; closed forms; linearity and the
@@ -33,7 +37,7 @@
 #include <omp.h>
 #endif
 
-enum { NMO_F32 = 0, NMO_BF16 = 1, NMO_F64 = 3 };
+enum { NMO_F32 = 0, NMO_BF16 = 1, NMO_F16 = 2, NMO_F64 = 3 };
 enum { NMO_ROW_MAJOR = 0, NMO_COL_MAJOR = 1, NMO_FRACTAL_NZ = 2 };
 
 /* ---- exact widening and single-step rounding ------------------------------------- */
@@ -70,11 +74,48 @@ static uint16_t f64_to_bf16(double x)
 double nmo_bf16_to_f64(uint16_t b) { return bf16_to_f64(b); }
 uint16_t nmo_f64_to_bf16(double x) { return f64_to_bf16(x); }
 
+/* IEEE binary16 (the optional fp16 element type of the product): 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static double f16_to_f64(uint16_t h)
+{
+    int sign = h >> 15, e = (h >> 10) & 31, f = h & 1023;
+    double v;
+    if (e == 0) v = ldexp((double)f, -24);                       /* zero and subnormals: f * 2^-24 */
+    else if (e == 31) v = f ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)f / 1024.0, e - 15);
+    return sign ? -v : v;
+}
+
+/* fp64 -> fp16, round to nearest, ties to even, in one step. */
+static uint16_t f64_to_f16(double x)
+{
+    if (isnan(x)) return 0x7e00;
+    uint16_t sign = signbit(x) ? 0x8000 : 0;
+    double a = fabs(x);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return sign | 0x7c00;
+    int e;
+    (void)frexp(a, &e);
+    int p = e - 1;                                /* floor(log2 a) */
+    if (p < -14) p = -14;                         /* subnormals share the quantum of the lowest binade, 2^-24 */
+    double quantum = ldexp(1.0, p - 10);          /* fp16 keeps 10 fraction bits */
+    double r = nearbyint(a / quantum) * quantum;  /* default rounding mode: ties to even */
+    if (r >= 65536.0) return sign | 0x7c00;       /* past the largest finite value (65504) by half a quantum or more */
+    if (r < ldexp(1.0, -14)) return sign | (uint16_t)(r / ldexp(1.0, -24));      /* subnormal or zero */
+    (void)frexp(r, &e);                           /* rounding may have carried into the next binade */
+    p = e - 1;
+    double frac = r / ldexp(1.0, p) - 1.0;        /* in [0, 1), a multiple of 2^-10 */
+    return sign | (uint16_t)((p + 15) << 10) | (uint16_t)(frac * 1024.0);
+}
+
+double nmo_f16_to_f64(uint16_t h) { return f16_to_f64(h); }
+uint16_t nmo_f64_to_f16(double x) { return f64_to_f16(x); }
+
 static double load_as_f64(const void *p, long i, int dtype)
 {
     switch (dtype) {
     case NMO_F32:  return (double)((const float *)p)[i];
     case NMO_BF16: return bf16_to_f64(((const uint16_t *)p)[i]);
+    case NMO_F16:  return f16_to_f64(((const uint16_t *)p)[i]);
     default:       return ((const double *)p)[i];
     }
 }
@@ -84,6 +125,7 @@ static void store_rounded(void *p, long i, int dtype, double x)
     switch (dtype) {
     case NMO_F32:  ((float *)p)[i] = (float)x; break;          /* C cast: RNE */
     case NMO_BF16: ((uint16_t *)p)[i] = f64_to_bf16(x); break;
+    case NMO_F16:  ((uint16_t *)p)[i] = f64_to_f16(x); break;
     default:       ((double *)p)[i] = x; break;
     }
 }
@@ -168,8 +210,8 @@ void nmo_matmul_batched(const void *A, const void *B, void *C, double *C64, doub
                         int M, int N, int K, int H, long lda, long strideA, long strideB,
                         long ldc, long strideC, int in_dtype, int out_dtype, int layout_B, int threads)
 {
-    size_t esz_in = (in_dtype == NMO_F32) ? 4 : (in_dtype == NMO_BF16 ? 2 : 8);
-    size_t esz_out = (out_dtype == NMO_F32) ? 4 : (out_dtype == NMO_BF16 ? 2 : 8);
+    size_t esz_in = (in_dtype == NMO_F32) ? 4 : ((in_dtype == NMO_BF16 || in_dtype == NMO_F16) ? 2 : 8);
+    size_t esz_out = (out_dtype == NMO_F32) ? 4 : ((out_dtype == NMO_BF16 || out_dtype == NMO_F16) ? 2 : 8);
     long ldb = (layout_B == NMO_ROW_MAJOR) ? N : K;
     for (int h = 0; h < H; ++h) {
         const char *Ah = (const char *)A + (size_t)h * strideA * esz_in;

@@ -10,7 +10,7 @@ import pytest
 
 import nm_inputs as gen
 import oracle
-from oracle import BF16, COL_MAJOR, F32, F64, ROW_MAJOR, alg2
+from oracle import BF16, COL_MAJOR, F16, F32, F64, ROW_MAJOR, alg2
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -121,6 +121,78 @@ def test_bf16_widening_is_the_upper_half_of_fp32():
     bits[::2] |= 0x8000
     assert np.array_equal(oracle.bf16_to_f64(bits), gen.bits_to_f32(bits).astype(np.float64))
     assert np.array_equal(oracle.f64_to_bf16(oracle.bf16_to_f64(bits)), bits)  # grid points are fixed
+
+
+# ---- the optional fp16 element type: binary16 widening and rounding ------------------------------
+
+def test_fp16_widening_of_every_bit_pattern():
+    bits = np.arange(65536, dtype=np.uint16)
+    got = oracle.f16_to_f64(bits)
+    want = bits.view(np.float16).astype(np.float64)                   # numpy's binary16
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan], want[~nan])
+    assert np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))      # -0 stays -0
+    # hand values: 0x3c00 = 1, 0x0001 = 2^-24 (smallest subnormal), 0x0400 = 2^-14 (smallest normal),
+    # 0x7bff = 65504 (largest finite), 0xc000 = -2
+    hand = {0x3C00: 1.0, 0x0001: 2.0 ** -24, 0x0400: 2.0 ** -14, 0x7BFF: 65504.0, 0xC000: -2.0, 0x3555: 0.333251953125}
+    for b, v in hand.items():
+        assert oracle.f16_to_f64(np.array([b], np.uint16))[0] == v
+    # grid points are fixed points of the rounding
+    finite = bits[~nan & ~np.isinf(want)]
+    assert np.array_equal(oracle.f64_to_f16(oracle.f16_to_f64(finite)), finite)
+
+
+def test_fp16_rounding_is_one_step_to_nearest_even():
+    f16 = lambda x: oracle.f64_to_f16(np.array([x], np.float64))[0]
+    # ties at 1: 1 + 2^-11 is halfway between 1 and 1 + 2^-10 -> even (1); 1 + 3 * 2^-11 -> 1 + 2^-9
+    assert f16(1.0 + 2.0 ** -11) == 0x3C00
+    assert f16(1.0 + 3 * 2.0 ** -11) == 0x3C02
+    assert f16(1.0 + 2.0 ** -11 + 2.0 ** -40) == 0x3C01               # just above the tie: up (an fp32 stop would tie down)
+    # overflow: 65504 is the largest finite value; 65520 is the tie to 2^16 and goes to infinity, 65519.99 does not
+    assert f16(65504.0) == 0x7BFF and f16(65519.99) == 0x7BFF and f16(65520.0) == 0x7C00 and f16(-1e6) == 0xFC00
+    # subnormals: quantum 2^-24; 1.5 * 2^-24 ties to even (2 * 2^-24), 0.5 * 2^-24 ties to zero, 0.51 * 2^-24 -> 2^-24
+    assert f16(1.5 * 2.0 ** -24) == 0x0002 and f16(0.5 * 2.0 ** -24) == 0x0000 and f16(0.51 * 2.0 ** -24) == 0x0001
+    assert f16(2.0 ** -14 - 2.0 ** -26) == 0x0400                      # rounds up into the first normal binade
+    assert f16(-0.0) == 0x8000
+    # against numpy's float64 -> float16 cast on random values across the range (subnormal, normal, near overflow)
+    rng = np.random.default_rng(21)
+    x = np.concatenate([rng.standard_normal(20000), rng.standard_normal(20000) * 1e-6, rng.standard_normal(20000) * 2e4,
+                        rng.uniform(-7e-5, 7e-5, 20000)])
+    with np.errstate(over="ignore"):
+        want = x.astype(np.float16).view(np.uint16)
+    assert np.array_equal(oracle.f64_to_f16(x), want)
+
+
+def test_fp16_product_brute_force_and_one_rounding():
+    # exact integer arithmetic on tiny shapes, fp16 storage
+    rng = np.random.default_rng(8)
+    to16 = lambda v: np.ascontiguousarray(v, np.float16).view(np.uint16)
+    for M, N, K in itertools.product(range(1, 4), repeat=3):
+        Ai = rng.integers(-3, 4, size=(M, K)); Bi = rng.integers(-3, 4, size=(K, N))
+        Ci = np.zeros((M, N), dtype=np.int64)
+        for m in range(M):
+            for n in range(N):
+                for k in range(K):
+                    Ci[m, n] += int(Ai[m, k]) * int(Bi[k, n])
+        for layout in (ROW_MAJOR, COL_MAJOR):
+            Bst = Bi if layout == ROW_MAJOR else Bi.T
+            Cq, C64, _ = oracle.matmul(to16(Ai), to16(Bst), M, N, K, F16, F16, layout)
+            assert np.array_equal(C64, Ci.astype(np.float64))
+            assert np.array_equal(Cq.view(np.float16).astype(np.int64), Ci)
+    # a sum that is exact in fp64 and a tie in fp16: 2048 + 1 -> 2048 (even), 2048 + 3 -> 2052
+    K = 4
+    A = to16(np.ones((1, K)))
+    for last, expect in ((1.0, 2048.0), (3.0, 2052.0)):
+        col = np.array([1024.0, 512.0, 512.0, last]).reshape(K, 1)
+        Cq, C64, _ = oracle.matmul(A, to16(col), 1, 1, K, F16, F16)
+        assert C64[0, 0] == 2048.0 + last and float(Cq.view(np.float16)[0, 0]) == expect
+    # random fp16 data against numpy in float64 (a library product), then one rounding
+    A16, B16 = gen.narrow_f16(3, 300, 17, seed=77)
+    Cq, C64, bound = oracle.matmul(A16, B16, 3, 17, 300, F16, F16)
+    ref = A16.view(np.float16).astype(np.float64) @ B16.view(np.float16).astype(np.float64)
+    assert np.allclose(C64, ref, rtol=0, atol=1e-12 * np.abs(bound).max())
+    assert np.array_equal(Cq, oracle.f64_to_f16(C64))
 
 
 # ---- P5: identity / one-hot -------------------------------------------------------------------

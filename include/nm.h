@@ -34,7 +34,12 @@ typedef void *nm_stream;          /* a cudaStream_t */
 typedef enum {
     NM_F32 = 0,                   /* fp32 in, fp32 out */
     NM_BF16 = 1,                  /* bf16 in, fp32 accumulate, bf16 out */
-    NM_BF16_F32OUT = 2            /* bf16 in, fp32 accumulate, fp32 out (unrounded sums) */
+    NM_BF16_F32OUT = 2,           /* bf16 in, fp32 accumulate, fp32 out (unrounded sums) */
+    NM_F16 = 3                    /* fp16 (IEEE binary16) in, fp32 accumulate, fp16 out.  Not a type the paper computes in (its
+                                   * data is bf16; Data Type Issue section) - an optional element type of the same product.
+                                   * Row- and column-major B: the swap-AB tensor-core kernel (weights of 8 MB and more,
+                                   * operands it can address; also 17..NM_MAX_M_TENSOR rows) or the CUDA-core row / column
+                                   * kernels; NM_FRACTAL_NZ returns NM_ERR_UNSUPPORTED. */
 } nm_dtype;
 
 /* Storage of B (K x N).  NM_FRACTAL_NZ: the tiling the paper's weight matrices have in memory (MLA Operator

@@ -238,6 +238,13 @@ def mla_decode_step(dims: dict, w: dict, h, kv_cache, seq_len, rms_eps=1e-6, sof
     return out
 
 
+def ulp_f16(x: np.ndarray) -> np.ndarray:
+    """Spacing of the fp16 grid at |x| (2^(floor(log2|x|) - 10); 2^-24 throughout the subnormal range)."""
+    ax = np.abs(np.asarray(x, dtype=np.float64))
+    e = np.floor(np.log2(np.maximum(ax, 2.0 ** -14)))
+    return np.exp2(e - 10)
+
+
 def ulp_bf16(x: np.ndarray) -> np.ndarray:
     """Spacing of the bf16 grid at |x| (2^(floor(log2|x|) - 7); smallest normal binade below that)."""
     ax = np.abs(np.asarray(x, dtype=np.float64))

@@ -15,7 +15,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libnm.so")
 
-F32, BF16, BF16_F32OUT = 0, 1, 2
+F32, BF16, BF16_F32OUT, F16 = 0, 1, 2, 3
 ROW_MAJOR, COL_MAJOR, FRACTAL_NZ = 0, 1, 2
 MAX_M = 16
 WS_COUNTER_BYTES = 65536

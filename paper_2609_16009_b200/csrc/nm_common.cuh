@@ -6,6 +6,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 #include <stddef.h>
 
@@ -60,11 +61,29 @@ template <> struct Elem<bf16_t> {
     __device__ static __forceinline__ float widen(bf16_t x) { return __uint_as_float(uint32_t(x.bits) << 16); }
 };
 
+// fp16 (IEEE binary16), the optional element type: widening is a conversion instruction (exact).
+struct f16_t { uint16_t bits; };
+template <> struct Elem<f16_t> {
+    static constexpr int kVec = 8;
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&f)[8]) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 p = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+            f[2 * i] = p.x; f[2 * i + 1] = p.y;
+        }
+    }
+    __device__ static __forceinline__ float widen(f16_t x) { return __half2float(__ushort_as_half(x.bits)); }
+};
+
 // Output rounding: one round-to-nearest-even step from the fp32 sum.
 template <typename T> __device__ __forceinline__ T round_out(float x);
 template <> __device__ __forceinline__ float round_out<float>(float x) { return x; }
 template <> __device__ __forceinline__ bf16_t round_out<bf16_t>(float x) {
     bf16_t r; r.bits = __bfloat16_as_ushort(__float2bfloat16_rn(x)); return r;
+}
+template <> __device__ __forceinline__ f16_t round_out<f16_t>(float x) {
+    f16_t r; r.bits = __half_as_ushort(__float2half_rn(x)); return r;
 }
 
 // 16-byte streaming load: read-only path, no L1 allocation (each weight byte is used once).

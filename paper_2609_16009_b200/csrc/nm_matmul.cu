@@ -15,6 +15,8 @@ NM_EXTERN(row, bf16_t, float)
 NM_EXTERN(row, float, float)
 NM_EXTERN(col, bf16_t, bf16_t)
 NM_EXTERN(col, bf16_t, float)
+NM_EXTERN(row, f16_t, f16_t)
+NM_EXTERN(col, f16_t, f16_t)
 NM_EXTERN(col, float, float)
 NM_EXTERN_TMA(8, bf16_t)
 NM_EXTERN_TMA(8, float)
@@ -219,6 +221,9 @@ static Plan make_tc_plan(int M, int N, int K, int H, bool col_major = false, boo
 
 static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layout, bool vec_ok, bool tma_ok, bool chained = false)
 {
+    // fp16 (the optional element type): the tensor-core kernel takes it, the TMA ring kernel (bf16 unpacking, fused bf16
+    // stages) does not; its CUDA-core kernels pay a conversion per element, so the tensor cores take over from 8 MB on at every M
+    const bool ring_ok = tma_ok && dtype != NM_F16;
     Plan p{};
     const int V = vec_elems(dtype);
     if (layout == NM_FRACTAL_NZ) {
@@ -246,10 +251,11 @@ static Plan make_plan(int M, int N, int K, int H, nm_dtype dtype, nm_layout layo
     // on 75 MB).
     const int min_m = (layout == NM_COL_MAJOR && g_t.tc_min_m > 2 && g_t.tc_min_m <= NM_MAX_M) ? 2 : g_t.tc_min_m;
     // More than 16 tokens (up to 64): only the tensor-core kernel takes them, whatever the size of the matrix
-    const bool tc_pays = M > NM_MAX_M || (M >= min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6)) && (M >= g_t.tc_min_m || wbytes >= 48e6));
+    const bool tc_pays = M > NM_MAX_M || (dtype == NM_F16 && wbytes >= 8e6) ||
+                         (M >= min_m && (wbytes >= 16e6 || (H > 1 && wbytes >= 8e6)) && (M >= g_t.tc_min_m || wbytes >= 48e6));
     if (tma_ok && (M > NM_MAX_M || (g_t.force_kind != kRowTma && (layout == NM_ROW_MAJOR || g_t.force_kind != kRowVec))) && (tc_pays || g_t.force_kind == kRowTc))
         return make_tc_plan(M, N, K, H, layout == NM_COL_MAJOR, dtype == NM_BF16_F32OUT);
-    if (layout == NM_ROW_MAJOR && tma_ok) return make_tma_plan(M, N, K, H, chained);
+    if (layout == NM_ROW_MAJOR && ring_ok) return make_tma_plan(M, N, K, H, chained);
     const int target = 192;                           // CTAs wanted in total (measured: 144-240 is the flat optimum)
     if (layout == NM_ROW_MAJOR) {
         p.kind = kRowVec;
@@ -362,13 +368,13 @@ static int check_common(const void *A, const void *B, const void *C, int M, int 
 {
     if (!A || !B || !C) return NM_ERR_INVALID_ARG;
     if (M < 1 || M > NM_MAX_M_TENSOR || N < 1 || K < 1 || H < 1) return NM_ERR_INVALID_ARG;
-    if (dtype != NM_F32 && dtype != NM_BF16 && dtype != NM_BF16_F32OUT) return NM_ERR_UNSUPPORTED;
+    if (dtype != NM_F32 && dtype != NM_BF16 && dtype != NM_BF16_F32OUT && dtype != NM_F16) return NM_ERR_UNSUPPORTED;
     if (layout != NM_ROW_MAJOR && layout != NM_COL_MAJOR && layout != NM_FRACTAL_NZ) return NM_ERR_UNSUPPORTED;
     // 16 x 16 fractals: bf16, whole fractals, and only through the TMA ring kernel (up to 16 rows)
-    if (layout == NM_FRACTAL_NZ && (dtype == NM_F32 || (N % 16) || (K % 16) || M > NM_MAX_M)) return NM_ERR_UNSUPPORTED;
+    if (layout == NM_FRACTAL_NZ && (dtype == NM_F32 || dtype == NM_F16 || (N % 16) || (K % 16) || M > NM_MAX_M)) return NM_ERR_UNSUPPORTED;
     if (H > 65535) return NM_ERR_UNSUPPORTED;
     const uintptr_t es = (uintptr_t)elem_size(dtype);
-    const uintptr_t os = (dtype == NM_BF16) ? 2 : 4;
+    const uintptr_t os = (dtype == NM_BF16 || dtype == NM_F16) ? 2 : 4;
     if (((uintptr_t)A % es) || ((uintptr_t)B % es) || ((uintptr_t)C % os)) return NM_ERR_ALIGNMENT;
     return NM_OK;
 }
@@ -446,7 +452,9 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
         ta.base = a; ta.nstage = p.nstage; ta.use_pdl = (g_t.use_pdl || pdl) ? 1 : 0; ta.status = device_status_ptr();
         if (g_t.cluster_split && p.nsplit >= 2 && p.nsplit <= 8 && (size_t)p.nsplit * M * kTcTN * sizeof(float) <= 65536) ta.cluster_split = 1;
         const bool col = layout == NM_COL_MAJOR;
-        e = (dtype == NM_BF16_F32OUT) ? launch_row_tc<float>(*mb, *ma, ta, stream, col) : launch_row_tc<bf16_t>(*mb, *ma, ta, stream, col);
+        e = (dtype == NM_BF16_F32OUT) ? launch_row_tc<float>(*mb, *ma, ta, stream, col)
+            : (dtype == NM_F16)       ? launch_row_tc<f16_t>(*mb, *ma, ta, stream, col)
+                                      : launch_row_tc<bf16_t>(*mb, *ma, ta, stream, col);
     } else if (p.kind == kRowTma) {
         const int kt = (kTmaConsumers / p.tpr) * 4;
         const CUtensorMap *map = (layout == NM_FRACTAL_NZ) ? get_fractal_map(B, N, K, H, strideB, p.tn, kt)
@@ -495,14 +503,17 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     } else if (p.kind == kGeneric) {
         if (dtype == NM_F32)            e = launch_generic<float, float>(a, layout, stream);
         else if (dtype == NM_BF16)      e = launch_generic<bf16_t, bf16_t>(a, layout, stream);
+        else if (dtype == NM_F16)       e = launch_generic<f16_t, f16_t>(a, layout, stream);
         else                            e = launch_generic<bf16_t, float>(a, layout, stream);
     } else if (p.kind == kRowVec) {
         if (dtype == NM_F32)            e = launch_row<float, float>(a, stream);
         else if (dtype == NM_BF16)      e = launch_row<bf16_t, bf16_t>(a, stream);
+        else if (dtype == NM_F16)       e = launch_row<f16_t, f16_t>(a, stream);
         else                            e = launch_row<bf16_t, float>(a, stream);
     } else {
         if (dtype == NM_F32)            e = launch_col<float, float>(a, stream);
         else if (dtype == NM_BF16)      e = launch_col<bf16_t, bf16_t>(a, stream);
+        else if (dtype == NM_F16)       e = launch_col<f16_t, f16_t>(a, stream);
         else                            e = launch_col<bf16_t, float>(a, stream);
     }
     if (e != cudaSuccess) return record_cuda_error(e, "narrow matmul launch");
@@ -618,7 +629,7 @@ int nm_matmul_host(const void *A_host, const void *B, void *C_host, void *A_stag
     if (rc != NM_OK) return rc;
     cudaStream_t s = (cudaStream_t)stream;
     const size_t a_bytes = (size_t)M * K * elem_size(dtype);
-    const size_t c_bytes = (size_t)M * N * (dtype == NM_BF16 ? 2 : 4);
+    const size_t c_bytes = (size_t)M * N * ((dtype == NM_BF16 || dtype == NM_F16) ? 2 : 4);
     NM_CUDA_TRY(cudaMemcpyAsync(A_staging, A_host, a_bytes, cudaMemcpyHostToDevice, s));
     rc = matmul_impl(A_staging, B, C_staging, M, N, K, 1, K, 0, 0, N, 0, dtype, layout_B, workspace, workspace_bytes, s);
     if (rc != NM_OK) return rc;

@@ -17,6 +17,8 @@
 //
 // Column-major B ([N][K], k contiguous) is the same kernel with the weight operand K-major: one
 // [128 columns of C x 64 k] box per stage (128-byte swizzle), the descriptor advanced 32 bytes per k-step.
+#include <type_traits>
+
 #include "nm_matmul_kernels.cuh"
 #include "nm_row_tc.cuh"
 #include "nm_tcgen05.cuh"
@@ -107,7 +109,8 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc(128, kTok, !kCol, false);
+            // fp16 output means fp16 operands (the optional element type); bf16 operands otherwise
+            constexpr uint32_t idesc = std::is_same<TO, f16_t>::value ? instr_desc_f16(128, kTok, !kCol, false) : instr_desc(128, kTok, !kCol, false);
             int s = 0;
             uint32_t ph = 0;
             for (int it = 0; it < n_it; ++it) {
@@ -285,5 +288,6 @@ cudaError_t launch_row_tc(const CUtensorMap &map_b, const CUtensorMap &map_a, co
 
 template cudaError_t launch_row_tc<bf16_t>(const CUtensorMap &, const CUtensorMap &, const TmaArgs &, cudaStream_t, bool);
 template cudaError_t launch_row_tc<float>(const CUtensorMap &, const CUtensorMap &, const TmaArgs &, cudaStream_t, bool);
+template cudaError_t launch_row_tc<f16_t>(const CUtensorMap &, const CUtensorMap &, const TmaArgs &, cudaStream_t, bool);
 
 }  // namespace nm

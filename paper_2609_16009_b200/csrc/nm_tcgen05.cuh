@@ -21,6 +21,12 @@ __host__ __device__ constexpr uint32_t instr_desc(int m, int n, bool a_mn_major,
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// The same with fp16 (binary16) operands: format fields of A and B zero.
+__host__ __device__ constexpr uint32_t instr_desc_f16(int m, int n, bool a_mn_major, bool b_mn_major)
+{
+    return instr_desc(m, n, a_mn_major, b_mn_major) & ~((7u << 7) | (7u << 10));
+}
+
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate)
 {
     asm volatile(

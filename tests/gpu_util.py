@@ -7,9 +7,10 @@ import torch
 
 import oracle
 
-NP_IN = {0: np.float32, 1: np.uint16, 2: np.uint16}
-ORACLE_IN = {0: oracle.F32, 1: oracle.BF16, 2: oracle.BF16}
-ORACLE_OUT = {0: oracle.F32, 1: oracle.BF16, 2: oracle.F32}
+NP_IN = {0: np.float32, 1: np.uint16, 2: np.uint16, 3: np.uint16}
+ORACLE_IN = {0: oracle.F32, 1: oracle.BF16, 2: oracle.BF16, 3: oracle.F16}
+ORACLE_OUT = {0: oracle.F32, 1: oracle.BF16, 2: oracle.F32, 3: oracle.F16}
+HALF_OUT = (1, 3)                  # dtypes with 16-bit outputs (bf16, fp16)
 
 
 def to_dev(a: np.ndarray) -> torch.Tensor:
@@ -20,9 +21,9 @@ def to_dev(a: np.ndarray) -> torch.Tensor:
 
 def out_buffer(numel: int, dtype: int, guard: int = 64):
     """Output buffer with canary guard bands on both sides.  Returns (whole, view of the middle)."""
-    tdt = torch.int16 if dtype == 1 else torch.float32
+    tdt = torch.int16 if dtype in HALF_OUT else torch.float32
     whole = torch.empty(numel + 2 * guard, dtype=tdt, device="cuda")
-    if dtype == 1:
+    if dtype in HALF_OUT:
         whole.fill_(0x7A7A)
     else:
         whole.fill_(-12345.5)
@@ -31,7 +32,7 @@ def out_buffer(numel: int, dtype: int, guard: int = 64):
 
 def guards_intact(whole: torch.Tensor, numel: int, dtype: int, guard: int = 64) -> bool:
     w = whole.cpu()
-    canary = 0x7A7A if dtype == 1 else -12345.5
+    canary = 0x7A7A if dtype in HALF_OUT else -12345.5
     return bool((w[:guard] == canary).all() and (w[guard + numel:] == canary).all())
 
 
@@ -39,15 +40,19 @@ def out_to_f64(t: torch.Tensor, dtype: int) -> np.ndarray:
     a = t.cpu().numpy()
     if dtype == 1:
         return oracle.bf16_to_f64(a.view(np.uint16))
+    if dtype == 3:
+        return oracle.f16_to_f64(a.view(np.uint16))
     return a.astype(np.float64)
 
 
 def assert_matmul_close(got: np.ndarray, Cq: np.ndarray, C64: np.ndarray, bound: np.ndarray, dtype: int, what=""):
-    """|gpu - oracle| <= 1e-5 * sum_k|a*b| + 1e-6, plus one output ulp for bf16 outputs."""
-    ref = oracle.bf16_to_f64(Cq) if dtype == 1 else Cq.astype(np.float64)
+    """|gpu - oracle| <= 1e-5 * sum_k|a*b| + 1e-6, plus one output ulp for bf16 (fp16) outputs."""
+    ref = oracle.bf16_to_f64(Cq) if dtype == 1 else (oracle.f16_to_f64(Cq) if dtype == 3 else Cq.astype(np.float64))
     tol = 1e-5 * bound + 1e-6
     if dtype == 1:
         tol = tol + oracle.ulp_bf16(C64)
+    if dtype == 3:
+        tol = tol + oracle.ulp_f16(C64)
     err = np.abs(got.reshape(ref.shape) - ref)
     bad = err > tol
     assert not bad.any(), (f"{what}: {bad.sum()} of {bad.size} elements outside tolerance; "

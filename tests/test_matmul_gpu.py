@@ -10,7 +10,7 @@ from gpu_util import (NP_IN, ORACLE_IN, ORACLE_OUT, assert_matmul_close, guards_
 
 pytestmark = pytest.mark.gpu
 
-F32, BF16, BF16_F32OUT = 0, 1, 2
+F32, BF16, BF16_F32OUT, F16 = 0, 1, 2, 3
 ROW, COL = 0, 1
 
 
@@ -51,6 +51,8 @@ def run_case(nm, A, B_row, M, N, K, dtype, layout, what, full_oracle=True, cols=
 def make_inputs(M, K, N, dtype, seed):
     if dtype == F32:
         return gen.uniform_f32((M, K), -1, 1, seed), gen.uniform_f32((K, N), -1, 1, seed + 1)
+    if dtype == F16:
+        return gen.narrow_f16(M, K, N, seed)
     return gen.narrow_bf16(M, K, N, seed)
 
 
@@ -154,6 +156,68 @@ def test_every_m_vector_path(nm, M, layout):
 def test_ragged_and_degenerate_shapes(nm, dtype, layout, M, K, N):
     A, B = make_inputs(M, K, N, dtype, seed=400 + M + K + N)
     run_case(nm, A, B, M, N, K, dtype, layout, f"dtype={dtype} layout={layout} {M}x{K}x{N}")
+
+
+# ---- fp16, the optional element type (CUDA-core kernels, both layouts, 1 <= M <= 16) -----------------------
+
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("M,K,N", [(1, 1, 1), (3, 5, 7), (2, 129, 33), (16, 77, 1), (5, 1023, 259), (1, 8, 8), (7, 8, 2048),
+                                    (1, 1000, 840), (4, 1000, 840), (16, 1000, 840), (1, 7168, 576), (2, 7168, 1536), (16, 2600, 72)])
+def test_fp16_products(nm, layout, M, K, N):
+    A, B = gen.narrow_f16(M, K, N, seed=450 + M + K + N)
+    run_case(nm, A, B, M, N, K, F16, layout, f"fp16 layout={layout} {M}x{K}x{N}")
+
+
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("nsplit", [1, 3, 16])
+def test_fp16_forced_splits_and_ties(nm, layout, nsplit):
+    M, K, N = 3, 4096, 264
+    A, B = gen.narrow_f16(M, K, N, seed=470)
+    nm.nm_debug_set_plan(0, nsplit)
+    try:
+        run_case(nm, A, B, M, N, K, F16, layout, f"fp16 nsplit={nsplit} layout={layout}")
+        # sums that are ties of the fp16 grid: 2048 + 1 -> 2048 (even), 2048 + 3 -> 2052, in every column
+        to16 = lambda v: np.ascontiguousarray(v, np.float16).view(np.uint16)
+        K2, N2 = 64, 16
+        col = np.zeros((K2, N2)); col[0] = 1024.0; col[1] = 512.0; col[2] = 512.0; col[3, ::2] = 1.0; col[3, 1::2] = 3.0
+        got = run_case(nm, to16(np.ones((1, K2))), to16(col), 1, N2, K2, F16, layout, "fp16 ties")
+        assert np.array_equal(got[0, ::2], np.full(N2 // 2, 2048.0)) and np.array_equal(got[0, 1::2], np.full(N2 // 2, 2052.0))
+    finally:
+        nm.nm_debug_set_plan(0, 0)
+
+
+@pytest.mark.parametrize("layout", [ROW, COL])
+@pytest.mark.parametrize("M,K,N,nsplit", [(1, 4096, 1024, 0), (2, 7168, 1536, 0), (5, 2048, 2304, 2), (16, 1536, 4096, 0), (9, 1000, 4104, 3),
+                                           (17, 640, 512, 0), (40, 1536, 1024, 2), (64, 2048, 384, 0)])
+def test_fp16_on_the_tensor_cores(nm, layout, M, K, N, nsplit):
+    """fp16 operands through the swap-AB kernel (kind::f16 with both operand formats fp16): the planner's own choice from
+    8 MB of weights on, forced below that; ragged k tails and column tiles; 17 to 64 rows in one pass."""
+    A, B = gen.narrow_f16(M, K, N, seed=460 + M)
+    nm.nm_debug_set_kernel(4, 0)
+    nm.nm_debug_set_plan(0, nsplit)
+    try:
+        assert nm.nm_debug_get_plan(M, N, K, dtype=F16, layout_B=layout)["kind"] == 4
+        run_case(nm, A, B, M, N, K, F16, layout, f"fp16 tensor cores layout={layout} {M}x{K}x{N} nsplit={nsplit}")
+    finally:
+        nm.nm_debug_set_kernel(-1, 0)
+        nm.nm_debug_set_plan(0, 0)
+
+
+def test_fp16_kernel_choice_and_refusals(nm):
+    assert nm.nm_debug_get_plan(1, 18432, 7168, dtype=F16)["kind"] == 4          # 264 MB: tensor cores at every M
+    assert nm.nm_debug_get_plan(16, 1536, 7168, dtype=F16)["kind"] == 4
+    assert nm.nm_debug_get_plan(1, 576, 1024, dtype=F16)["kind"] == 0            # 1.2 MB: CUDA-core row kernel
+    assert nm.nm_debug_get_plan(1, 576, 1024, dtype=F16, layout_B=COL)["kind"] == 1
+    A, B = gen.narrow_f16(1, 64, 64, seed=480)
+    C = torch.zeros(64, dtype=torch.int16, device="cuda")
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_matmul(to_dev(A), to_dev(B), C, 1, 64, 64, F16, 2)             # FRACTAL_NZ: bf16 only
+    assert e.value.status == -2
+    A17, B17 = gen.narrow_f16(17, 63, 64, seed=481)                           # K = 63: no tensor map, and 17 rows need one
+    with pytest.raises(nm.NmError) as e:
+        nm.nm_matmul(to_dev(A17), to_dev(B17), torch.zeros(17 * 64, dtype=torch.int16, device="cuda"), 17, 64, 63, F16, ROW)
+    assert e.value.status == -2
+    nm.nm_check_status()
 
 
 @pytest.mark.parametrize("layout", [ROW, COL])
@@ -518,6 +582,23 @@ def test_batched_small_ragged(nm, layout):
     Cq, C64, bound = oracle.matmul_batched(A, Wst, T, N, K, H, H * K, K, K * N, H * N, N, T * H * N,
                                            oracle.BF16, oracle.F32, layout)
     assert_matmul_close(out_to_f64(dC, BF16_F32OUT), Cq, C64, bound, BF16_F32OUT, "batched ragged")
+
+
+@pytest.mark.parametrize("layout", [ROW, COL])
+def test_batched_fp16(nm, layout):
+    T, H, K, N = 3, 5, 136, 24
+    A16, _ = gen.narrow_f16(T * H, K, 1, seed=3250)
+    W16 = np.stack([gen.narrow_f16(1, K, N, seed=3251 + h)[1] for h in range(H)])
+    A = A16.reshape(T, H, K)
+    Wst = W16 if layout == ROW else np.ascontiguousarray(W16.transpose(0, 2, 1))
+    dA, dW = to_dev(A), to_dev(Wst)
+    whole, dC = out_buffer(T * H * N, F16)
+    nm.nm_matmul_batched(dA, dW, dC, T, N, K, H, H * K, K, K * N, H * N, N, F16, layout)
+    torch.cuda.synchronize()
+    assert guards_intact(whole, T * H * N, F16)
+    Cq, C64, bound = oracle.matmul_batched(A, Wst, T, N, K, H, H * K, K, K * N, H * N, N, T * H * N,
+                                           oracle.F16, oracle.F16, layout)
+    assert_matmul_close(out_to_f64(dC, F16), Cq, C64, bound, F16, "batched fp16")
 
 
 @pytest.mark.parametrize("layout", [ROW, COL])

@@ -215,6 +215,7 @@ class MlaStep:
         res = torch.zeros(T * DIMS["d"], dtype=torch.int16, device=cache.device)
         ws = self.nm.new_workspace(self.nm.nm_mla_batch_workspace_bytes(self.p, T), device=cache.device)
         pb = self.nm.mla_params(DIMS, 1, self.t, workspace=ws)
+        pb.programmatic_entry = 1            # steps follow each other; the weights are static
         b = self.nm.mla_batch([self.S] * T, h, cs, cache, stride, out=res)
         return (lambda: self.nm.nm_mla_decode_batch(pb, b, stream)), (cache, h, cs, res, ws, pb, b)
 

@@ -278,8 +278,9 @@ size_t nm_mla_workspace_bytes(const nm_mla_params *p);
  *   q_full, o_lat, o   optional device outputs [T][H][kv_lora+rope], [T][H][kv_lora], [T][H][v] bf16
  *   c_q, c_qn, q, ckr  optional device outputs [T][q_lora], [T][q_lora], [T][H][nope+rope], [T][kv_lora+rope] bf16: the
  *                outputs of the down-projections, of the query latent's RMSNorm and of W_UQR, for stage-wise checking
- * From nm_mla_params it takes the dimensions, weights, rms_eps, softmax_scale, layout_dense, workspace and
- * workspace_bytes (>= nm_mla_batch_workspace_bytes(p, T)); its h, kv_cache, seq_len, rope_cos_sin, out and
+ * From nm_mla_params it takes the dimensions, weights, rms_eps, softmax_scale, layout_dense, workspace,
+ * workspace_bytes (>= nm_mla_batch_workspace_bytes(p, T)) and programmatic_entry (the first product may start under
+ * the work enqueued before the call, as in the single-token step); its h, kv_cache, seq_len, rope_cos_sin, out and
  * intermediates are ignored.  Dimensions: kv_lora 512, rope 64, nope 128, v 128, H 128.  One stream; the kernels
  * are chained with programmatic dependent launch.  Errors as nm_mla_decode_step; nothing is enqueued on error
  * except as noted there. */

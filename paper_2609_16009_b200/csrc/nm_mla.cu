@@ -844,12 +844,15 @@ static int batch_impl(const nm_mla_params *p, const nm_mla_batch *b, cudaStream_
     }
 
     // ---- down-projections of all T tokens: the weights are streamed once ---------------------------------------
+    // The first product may start (and fill its ring with weights) under whatever the caller enqueued before the step
+    // when the caller says so (programmatic_entry: back-to-back steps or layers, static weights), as in the single-token step.
+    const bool entry_pdl = pdl && p->programmatic_entry;
     if (p->W_DQKV && lay == NM_ROW_MAJOR) {
         NM_TRY(matmul_enqueue(b->h, p->W_DQKV, x_down, T, ql + dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, NM_ROW_MAJOR, mws, L.mws_bytes, ms,
-                              false, nullptr, nullptr, nullptr, true));
+                              entry_pdl, nullptr, nullptr, nullptr, true));
     } else {
         NM_TRY(matmul_enqueue(b->h, p->W_DQ, x_down, T, ql, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws, L.mws_bytes, ms,
-                              false, nullptr, nullptr, nullptr, true));
+                              entry_pdl, nullptr, nullptr, nullptr, true));
         NM_TRY(matmul_enqueue(b->h, p->W_DKVKR, x_down + ql, T, dkv, d, 1, d, 0, 0, ql + dkv, 0, NM_BF16, lay, mws, L.mws_bytes, ms,
                               pdl, nullptr, nullptr, nullptr, true));
     }

@@ -33,7 +33,7 @@ def weights():
     return w, {k: to_dev(v) for k, v in w.items()}
 
 
-def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True, graph=False):
+def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True, graph=False, back_to_back=0):
     H, dc, dr, dn, dv, d, ql = (DIMS[k] for k in ("H", "kv_lora", "rope", "nope", "v", "d", "q_lora"))
     dkv = dc + dr
     T = len(seq_lens)
@@ -65,7 +65,11 @@ def run_batch(nm, dw, tokens, caches, seq_lens, concat_down, with_wo=True, graph
     b = nm.mla_batch(seq_lens, h, cs, cache, stride, out=out, q_full=q_full, o_lat=o_lat, o=o, c_q=c_q, c_qn=c_qn, q=q, ckr=ckr)
     st = torch.cuda.Stream()
     torch.cuda.synchronize()
-    if graph:                                                # captured once, replayed: the call allocates and synchronises nothing
+    if back_to_back:                                         # the same step several times in a row, each allowed to start under its predecessor
+        p.programmatic_entry = 1
+        for _ in range(back_to_back):
+            nm.nm_mla_decode_batch(p, b, st)
+    elif graph:                                                # captured once, replayed: the call allocates and synchronises nothing
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=st):
             nm.nm_mla_decode_batch(p, b, st)
@@ -172,6 +176,19 @@ def test_batch_replayed_from_a_cuda_graph(nm, weights, seq_lens):
     for k in ("out", "q_full", "o_lat", "o", "cache"):
         assert torch.equal(direct[k], replayed[k]), k
     check_against_oracle(w, replayed, tokens, caches, seq_lens)
+
+
+@pytest.mark.parametrize("seq_lens", [[700, 650, 90, 333], [64] * 16])
+def test_batch_steps_back_to_back_with_programmatic_entry(nm, weights, seq_lens):
+    """programmatic_entry: the first product of a step may start (weights only) while the previous step's W_O product is
+    still running.  Three steps in a row on the same buffers give the bits of one step on its own."""
+    w, dw = weights
+    tokens, caches = make_inputs(seq_lens, seed=8600 + len(seq_lens))
+    alone = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True)
+    chained = run_batch(nm, dw, tokens, [c.copy() for c in caches], seq_lens, True, back_to_back=3)
+    for k in ("out", "q_full", "o_lat", "o", "cache", "c_q", "q"):
+        assert torch.equal(alone[k], chained[k]), k
+    check_against_oracle(w, chained, tokens, caches, seq_lens)
 
 
 def test_batch_of_sixteen_without_wo(nm, weights):

@@ -787,7 +787,13 @@ def main():
         wl.step = lambda stream_, dom_events=None: fn()
         wl.step_e2e = lambda stream_: fn()
         wl.extra_measurements = lambda stream_: {}
-        wl.launches_per_step = 0
+        wl.launches_per_step = 9 if args.batch >= 3 else 7     # T >= 3: RoPE, the per-head products and the merge as kernels of their own
+        wl.bytes_per_step = wl.bytes_per_step - wl.kv_bytes + args.batch * wl.kv_bytes      # weights once, every sequence's cache rows
+        single = wl.describe()
+        single["workload"] = (f"small-batch MLA decode step (nm_mla_decode_batch): {args.batch} sequences of seq_len {wl.S}, one new token each, "
+                              "DeepSeek-V3 dims, bf16 weights row-major, W_O included; GB/s = weights once + every sequence's cache rows")
+        single["batch"] = args.batch
+        wl.describe = lambda: single
         args.single_length = args.no_sweep = True
     if args.timeline:
         with torch.cuda.stream(stream):

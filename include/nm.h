@@ -57,7 +57,9 @@ enum {
     NM_ERR_WORKSPACE = -4,        /* workspace missing or too small */
     NM_ERR_CUDA = -5,             /* a CUDA call failed; see nm_last_cuda_error() */
     NM_ERR_TIMEOUT = -6,          /* a bounded device-side wait expired (nm_check_status) */
-    NM_ERR_TOO_LARGE = -7         /* problem needs more scratch than nm_matmul_static has built in */
+    NM_ERR_TOO_LARGE = -7,        /* problem needs more scratch than nm_matmul_static has built in */
+    NM_ERR_BOUNDS = -8            /* debug build (libnm_check.so) only: a kernel's access outside the operand it belongs to
+                                   * was caught and skipped; reported by nm_check_status */
 };
 
 #define NM_MAX_M 16

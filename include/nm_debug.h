@@ -64,6 +64,19 @@ int nm_debug_set_attention(int impl);
 /* Wide-tile attention kernel: force the cache rows per tile (64, 128, 256), the most row runs (1..64) and the number of
  * runs merged on chip (cluster of 1, 2 or 4); zeros give each choice back to the planner. */
 int nm_debug_set_attention_wide(int tile_rows, int max_runs, int cluster);
+/* The debug build.  `python paper_2609_16009_b200/build.py --check` compiles the same sources with -DNM_BOUNDS_CHECK into
+ * libnm_check.so: every hand-indexed global access of the narrow-product kernels (the CUDA-core row / column / scalar
+ * kernels, the split-K gather, the token loads and the C / partial stores of the TMA ring and tensor-core kernels) is
+ * checked against the extent of the operand it belongs to; an access outside raises a bit in the device status word
+ * (nm_check_status returns NM_ERR_BOUNDS) and is skipped - loads yield zero, stores do nothing, nothing faults.  The paper
+ * has no counterpart; it stands in for a memory checker on machines where none can be run.
+ * nm_debug_bounds_checked: 1 in that build, 0 in the normal one.  nm_debug_bounds_selftest (debug build only, else
+ * NM_ERR_UNSUPPORTED): `buf` is a device buffer of `bytes` bytes (>= 32, a multiple of 8, 4-byte aligned); one thread
+ * stores to and loads from the first word of its second half while naming its first half as the operand - the store must
+ * not happen, out_loaded[0] (device, two words) must be 0 - and then does the same inside the first half (buf[0] becomes
+ * 0x600df00d, out_loaded[1] likewise); nm_check_status then reports NM_ERR_BOUNDS once. */
+int nm_debug_bounds_checked(void);
+int nm_debug_bounds_selftest(void *buf, size_t bytes, unsigned *out_loaded, nm_stream stream);
 /* Measurement aid: a kernel that only reads `bytes` bytes of device memory once (16-byte streaming loads, the
  * products' own load instruction, ctas_per_sm x SM-count CTAs of 256 threads) - the read-only bandwidth this GPU
  * delivers, to set beside the copy bandwidth the roofline uses.  src 16-byte aligned; sink4: 4 writable bytes. */

@@ -101,6 +101,7 @@ _lib.nm_mla_decode_step.argtypes = [C.POINTER(MlaParams), _vp, _vp]
 _lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_debug_set_attention.argtypes = [_i]
 _lib.nm_debug_set_attention_wide.argtypes = [_i, _i, _i]
+_lib.nm_debug_bounds_selftest.argtypes = [_vp, _sz, _vp, _vp]
 _lib.nm_debug_set_step_pdl.argtypes = [_i]
 _lib.nm_debug_stream_read.argtypes = [_vp, _sz, _vp, _i, _vp]
 _lib.nm_debug_set_step_knobs.argtypes = [_i, _i]

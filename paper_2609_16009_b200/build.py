@@ -2,7 +2,8 @@
 
 Run as ``python paper_2609_16009_b200/build.py`` (as a script: importing the package needs the library this builds).  Object files go to ``build/`` at the
 repository root; the shared library is written next to this file.  Only changed sources are
-recompiled (mtime against every header).
+recompiled (mtime against every header).  ``--check`` builds the debug library ``libnm_check.so`` instead (the same
+sources with ``-DNM_BOUNDS_CHECK``).
 """
 from __future__ import annotations
 
@@ -29,7 +30,11 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found")
 
 
-def build(verbose: bool = False, force: bool = False, ptxas_info: bool = False) -> str:
+def build(verbose: bool = False, force: bool = False, ptxas_info: bool = False, check: bool = False) -> str:
+    """check=True: the debug build (libnm_check.so, -DNM_BOUNDS_CHECK: the narrow-product kernels check their hand-indexed
+    global accesses against the operands' extents); its objects live in their own directory."""
+    OBJ = os.path.join(ROOT, "build", "nm_check" if check else "nm")
+    LIB = os.path.join(PKG, "libnm_check.so" if check else "libnm.so")
     os.makedirs(OBJ, exist_ok=True)
     sources = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     headers = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
@@ -42,7 +47,7 @@ def build(verbose: bool = False, force: bool = False, ptxas_info: bool = False) 
         objs.append(obj)
         stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_header)
         if stale:
-            cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-c", src, "-o", obj]
+            cmd = [nvcc, *NVCC_FLAGS, *(["-DNM_BOUNDS_CHECK"] if check else []), "-I", os.path.join(ROOT, "include"), "-c", src, "-o", obj]
             if ptxas_info:
                 cmd[1:1] = ["-Xptxas", "-v"]
             jobs.append(cmd)
@@ -69,4 +74,4 @@ def build(verbose: bool = False, force: bool = False, ptxas_info: bool = False) 
 
 
 if __name__ == "__main__":
-    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, ptxas_info="--ptxas" in sys.argv))
+    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, ptxas_info="--ptxas" in sys.argv, check="--check" in sys.argv))

@@ -94,6 +94,43 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p) {
     return v;
 }
 
+// ---- debug build (-DNM_BOUNDS_CHECK, libnm_check.so) -----------------------------------------------------------
+// Every hand-indexed global access of the narrow-product kernels names the operand it belongs to; the debug build
+// checks the address against that operand's extent first.  An access outside it raises kStatusOutOfBounds in the
+// device status word (nm_check_status then returns NM_ERR_BOUNDS) and is SKIPPED - a load yields zeros, a store does
+// nothing - so nothing faults and nothing traps.  (The tiled TMA copies need no such build: the copy engine clips them
+// to the tensor map's extents.)  In the normal build the macros are the bare access.
+constexpr unsigned kStatusOutOfBounds = 2u;
+struct Span { const char *lo, *hi; };                              // [lo, hi)
+__host__ __device__ __forceinline__ Span make_span(const void *base, size_t bytes)
+{
+    return Span{static_cast<const char *>(base), static_cast<const char *>(base) + bytes};
+}
+#ifdef NM_BOUNDS_CHECK
+__device__ __forceinline__ bool nm_inside(const void *p, size_t n, Span s, unsigned *status)
+{
+    const char *c = static_cast<const char *>(p);
+    const bool ok = c >= s.lo && c + n <= s.hi;
+    if (!ok && status) atomicOr(status, kStatusOutOfBounds);
+    return ok;
+}
+#define NM_LD_STREAM16(p, span, st) (::nm::nm_inside((p), 16, (span), (st)) ? ::nm::ld_stream16(p) : make_uint4(0u, 0u, 0u, 0u))
+#define NM_LDG16(p, span, st) (::nm::nm_inside((p), 16, (span), (st)) ? __ldg(p) : make_uint4(0u, 0u, 0u, 0u))
+template <typename T> __device__ __forceinline__ T nm_checked_load(const T *p, Span s, unsigned *status)
+{
+    return nm_inside(p, sizeof(T), s, status) ? *p : T{};
+}
+#define NM_LD(p, span, st) ::nm::nm_checked_load((p), (span), (st))
+#define NM_LD_CG(p, span, st) (::nm::nm_inside((p), sizeof(float), (span), (st)) ? ::nm::ld_cg(p) : 0.f)
+#define NM_ST(p, v, span, st) do { if (::nm::nm_inside((p), sizeof(*(p)), (span), (st))) *(p) = (v); } while (0)
+#else
+#define NM_LD_STREAM16(p, span, st) ::nm::ld_stream16(p)
+#define NM_LDG16(p, span, st) __ldg(p)
+#define NM_LD(p, span, st) (*(p))
+#define NM_LD_CG(p, span, st) ::nm::ld_cg(p)
+#define NM_ST(p, v, span, st) (*(p) = (v))
+#endif
+
 // Load that bypasses L1 (data written by other SMs in the same launch).
 __device__ __forceinline__ float ld_cg(const float *p) { return __ldcg(p); }
 

@@ -433,6 +433,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     a.lda = lda; a.strideA = strideA; a.strideB = strideB; a.ldc = ldc; a.strideC = strideC;
     a.tn = p.tn; a.tpr = p.tpr; a.rg = p.rg; a.nsplit = p.nsplit; a.kr = p.kr; a.ntiles = p.ntiles;
     a.a_vec = a_ok ? 1 : 0;
+    a.status = device_status_ptr();
     if (p.nsplit > 1) {
         const size_t need = kCounterBytes + partial_floats(p, M, H) * sizeof(float);
         if (!ws || ws_bytes < need) return NM_ERR_WORKSPACE;
@@ -558,6 +559,7 @@ const char *nm_status_string(int status)
     case NM_ERR_CUDA: return "CUDA error";
     case NM_ERR_TIMEOUT: return "bounded device-side wait expired";
     case NM_ERR_TOO_LARGE: return "problem too large for the built-in scratch of nm_matmul_static";
+    case NM_ERR_BOUNDS: return "debug build: an access outside its operand was caught and skipped";
     default: return "unknown status";
     }
 }

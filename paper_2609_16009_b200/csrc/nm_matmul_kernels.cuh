@@ -30,7 +30,26 @@ struct MatmulArgs {
     float *partial;
     unsigned *counters;
     int cluster_split;   // plain kernels: the k-splits of a tile form a cluster (1 x nsplit x 1) and meet in shared memory
+    unsigned *status;    // device status word (the debug build reports an access outside its operand there)
 };
+
+// Extents of the operands, for the debug build's checks (see NM_BOUNDS_CHECK in nm_common.cuh).
+template <typename TI> __device__ __forceinline__ Span span_of_A(const MatmulArgs &a)
+{
+    return make_span(a.A, (size_t)((long)(a.H - 1) * a.strideA + (long)(a.M - 1) * a.lda + a.K) * sizeof(TI));
+}
+template <typename TI> __device__ __forceinline__ Span span_of_B(const MatmulArgs &a)
+{
+    return make_span(a.B, (size_t)((long)(a.H - 1) * a.strideB + (long)a.K * a.N) * sizeof(TI));
+}
+template <typename TO> __device__ __forceinline__ Span span_of_C(const MatmulArgs &a)
+{
+    return make_span(a.C, (size_t)((long)(a.H - 1) * a.strideC + (long)(a.M - 1) * a.ldc + a.N) * sizeof(TO));
+}
+__device__ __forceinline__ Span span_of_partials(const MatmulArgs &a)
+{
+    return make_span(a.partial, a.partial ? (size_t)a.H * a.ntiles * a.nsplit * (size_t)a.M * a.tn * sizeof(float) : 0);
+}
 
 // ---- split-K inside a thread-block cluster (plain kernels) ----------------------------------------------
 // The k-splits of a column tile are the CTAs of one cluster.  Each stores its sums into slot [split] of the first
@@ -64,7 +83,7 @@ __device__ __forceinline__ void cluster_split_finish(const MatmulArgs &a, const 
         if (n < a.N) {
             float s = 0.f;
             for (int sp = 0; sp < a.nsplit; ++sp) s += slots[(size_t)sp * per + i];
-            C[(long)m * a.ldc + n] = round_out<TO>(s);
+            NM_ST(&C[(long)m * a.ldc + n], round_out<TO>(s), span_of_C<TO>(a), a.status);
         }
     }
 }
@@ -278,8 +297,10 @@ template <int M> struct RowCfg {
 
 // Sum of the nsplit partial tiles of one (head, tile), in split order, rounded once and written to C.
 template <typename TO>
-__device__ __forceinline__ void splitk_gather(const float *P, TO *C, int M, int tn, int nsplit, int N, int tile, long ldc)
+__device__ __forceinline__ void splitk_gather(const float *P, TO *C, int M, int tn, int nsplit, int N, int tile, long ldc,
+                                              Span span_p, Span span_c, unsigned *status)
 {
+    (void)span_p; (void)span_c; (void)status;
     // Four outputs per thread and pass, and the partials of all four requested four splits at a time before any
     // is used: a chain of L2 round trips otherwise (M * tile_n outputs x nsplit partials, one CTA).  The inner
     // loops are free of branches - a slot past the thread's last output repeats that output's address and its
@@ -303,7 +324,7 @@ __device__ __forceinline__ void splitk_gather(const float *P, TO *C, int M, int 
 #pragma unroll
             for (int u = 0; u < 4; ++u)
 #pragma unroll
-                for (int j = 0; j < kOut; ++j) v[u][j] = ld_cg(src[j] + (sp + u) * split_stride);
+                for (int j = 0; j < kOut; ++j) v[u][j] = NM_LD_CG(src[j] + (sp + u) * split_stride, span_p, status);
 #pragma unroll
             for (int u = 0; u < 4; ++u)                            // split order: deterministic
 #pragma unroll
@@ -312,7 +333,7 @@ __device__ __forceinline__ void splitk_gather(const float *P, TO *C, int M, int 
         for (; sp < nsplit; ++sp) {
             float v[kOut];
 #pragma unroll
-            for (int j = 0; j < kOut; ++j) v[j] = ld_cg(src[j] + sp * split_stride);
+            for (int j = 0; j < kOut; ++j) v[j] = NM_LD_CG(src[j] + sp * split_stride, span_p, status);
 #pragma unroll
             for (int j = 0; j < kOut; ++j) s[j] += v[j];
         }
@@ -321,7 +342,7 @@ __device__ __forceinline__ void splitk_gather(const float *P, TO *C, int M, int 
             if (j < live) {
                 const int i = i0 + j * stride + tid;
                 const int m = i / tn, c = i - m * tn, n = tile * tn + c;
-                if (n < N) C[(long)m * ldc + n] = round_out<TO>(s[j]);
+                if (n < N) NM_ST(&C[(long)m * ldc + n], round_out<TO>(s[j]), span_c, status);
             }
         }
     }
@@ -354,12 +375,12 @@ __device__ __forceinline__ void splitk_complete_rt(const MatmulArgs &a, int M, i
             if (n < a.N) {
                 float s = 0.f;
 #pragma unroll 4
-                for (int sp = 0; sp < a.nsplit; ++sp) s += ld_cg(P + ((size_t)sp * M + m) * a.tn + c);
-                C[(long)m * a.ldc + n] = round_out<TO>(s);
+                for (int sp = 0; sp < a.nsplit; ++sp) s += NM_LD_CG(P + ((size_t)sp * M + m) * a.tn + c, span_of_partials(a), a.status);
+                NM_ST(&C[(long)m * a.ldc + n], round_out<TO>(s), span_of_C<TO>(a), a.status);
             }
         }
     } else {
-        splitk_gather<TO>(P, C, M, a.tn, a.nsplit, a.N, tile, a.ldc);
+        splitk_gather<TO>(P, C, M, a.tn, a.nsplit, a.N, tile, a.ldc, span_of_partials(a), span_of_C<TO>(a), a.status);
     }
     if (tid == 0) *cnt = 0u;
 }
@@ -410,6 +431,8 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
     const long ldb = a.N;
     const TI *__restrict__ A = (const TI *)a.A + (long)h * a.strideA;
     const TI *__restrict__ B = (const TI *)a.B + (long)h * a.strideB;
+    const Span sp_a = span_of_A<TI>(a), sp_b = span_of_B<TI>(a), sp_c = span_of_C<TO>(a), sp_p = span_of_partials(a);
+    (void)sp_a; (void)sp_b; (void)sp_c; (void)sp_p;
 
     float acc[M][V];
 #pragma unroll
@@ -426,7 +449,7 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int rr = r + u * rg;
-            v[u] = (active && rr < klen) ? ld_stream16(bp + (long)rr * ldb) : make_uint4(0, 0, 0, 0);
+            v[u] = (active && rr < klen) ? NM_LD_STREAM16(bp + (long)rr * ldb, sp_b, a.status) : make_uint4(0, 0, 0, 0);
         }
         __syncthreads();                                  // readers of the previous chunk are done
         if (a.a_vec) {
@@ -435,15 +458,15 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
                 const uint4 *src = (const uint4 *)(A + (long)m * a.lda + kc);
                 for (int i = tid; i < nv; i += kThreads) {
                     float f[V];
-                    E::unpack(__ldg(src + i), f);
+                    E::unpack(NM_LDG16(src + i, sp_a, a.status), f);
 #pragma unroll
                     for (int j = 0; j < V; ++j) smem[m * KC + i * V + j] = f[j];
                 }
-                for (int i = nv * V + tid; i < klen; i += kThreads) smem[m * KC + i] = E::widen(A[(long)m * a.lda + kc + i]);
+                for (int i = nv * V + tid; i < klen; i += kThreads) smem[m * KC + i] = E::widen(NM_LD(&A[(long)m * a.lda + kc + i], sp_a, a.status));
             }
         } else {
             for (int m = 0; m < M; ++m)
-                for (int i = tid; i < klen; i += kThreads) smem[m * KC + i] = E::widen(A[(long)m * a.lda + kc + i]);
+                for (int i = tid; i < klen; i += kThreads) smem[m * KC + i] = E::widen(NM_LD(&A[(long)m * a.lda + kc + i], sp_a, a.status));
         }
         __syncthreads();
         if (active) {
@@ -455,12 +478,12 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
             r += U * rg;
             for (; r + (U - 1) * rg < klen; r += U * rg) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) v[u] = ld_stream16(bp + (long)(r + u * rg) * ldb);
+                for (int u = 0; u < U; ++u) v[u] = NM_LD_STREAM16(bp + (long)(r + u * rg) * ldb, sp_b, a.status);
 #pragma unroll
                 for (int u = 0; u < U; ++u) fma_row<M, TI>(acc, v[u], smem + r + u * rg);
             }
             for (; r < klen; r += rg) {
-                const uint4 w = ld_stream16(bp + (long)r * ldb);
+                const uint4 w = NM_LD_STREAM16(bp + (long)r * ldb, sp_b, a.status);
                 fma_row<M, TI>(acc, w, smem + r);
             }
         }
@@ -495,9 +518,9 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
             if (m < M && n < a.N) {
                 float s = 0.f;
                 for (int g = 0; g < rg; ++g) s += red[(size_t)(g * MP + mm) * a.tn + c];
-                if (a.nsplit == 1) C[(long)m * a.ldc + n] = round_out<TO>(s);
+                if (a.nsplit == 1) NM_ST(&C[(long)m * a.ldc + n], round_out<TO>(s), sp_c, a.status);
                 else if (a.cluster_split) cluster_slot_store(slot0, m * a.tn + c, s);
-                else               P[(size_t)m * a.tn + c] = s;
+                else               NM_ST(&P[(size_t)m * a.tn + c], s, sp_p, a.status);
             }
         }
     }
@@ -535,6 +558,8 @@ __global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
     const TI *__restrict__ A = (const TI *)a.A + (long)h * a.strideA;
     const TI *__restrict__ B = (const TI *)a.B + (long)h * a.strideB;
     const long ldb = a.K;
+    const Span sp_a = span_of_A<TI>(a), sp_b = span_of_B<TI>(a), sp_c = span_of_C<TO>(a), sp_p = span_of_partials(a);
+    (void)sp_a; (void)sp_b; (void)sp_c; (void)sp_p;
 
     float acc[M][CW];
 #pragma unroll
@@ -551,14 +576,14 @@ __global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
         for (int c = 0; c < CW; ++c) {
             const bool okc = col0 + c < a.N;
             const TI *bp = B + (long)(col0 + c) * ldb + kc;
-            b0[c] = (okc && kk < klen) ? ld_stream16(bp + kk) : make_uint4(0, 0, 0, 0);
-            b1[c] = (okc && kk + STEP < klen) ? ld_stream16(bp + kk + STEP) : make_uint4(0, 0, 0, 0);
+            b0[c] = (okc && kk < klen) ? NM_LD_STREAM16(bp + kk, sp_b, a.status) : make_uint4(0, 0, 0, 0);
+            b1[c] = (okc && kk + STEP < klen) ? NM_LD_STREAM16(bp + kk + STEP, sp_b, a.status) : make_uint4(0, 0, 0, 0);
         }
         __syncthreads();
         const int nv = klen / V;
         for (int m = 0; m < M; ++m) {
             const uint4 *src = (const uint4 *)(A + (long)m * a.lda + kc);
-            for (int i = tid; i < nv; i += kThreads) As[m * (KC / V) + i] = __ldg(src + i);
+            for (int i = tid; i < nv; i += kThreads) As[m * (KC / V) + i] = NM_LDG16(src + i, sp_a, a.status);
         }
         __syncthreads();
         for (; kk < klen; kk += 2 * STEP) {
@@ -572,8 +597,8 @@ __global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
             for (int c = 0; c < CW; ++c) {
                 const bool okc = col0 + c < a.N;
                 const TI *bp = B + (long)(col0 + c) * ldb + kc;
-                b0[c] = (okc && kn < klen) ? ld_stream16(bp + kn) : make_uint4(0, 0, 0, 0);
-                b1[c] = (okc && kn + STEP < klen) ? ld_stream16(bp + kn + STEP) : make_uint4(0, 0, 0, 0);
+                b0[c] = (okc && kn < klen) ? NM_LD_STREAM16(bp + kn, sp_b, a.status) : make_uint4(0, 0, 0, 0);
+                b1[c] = (okc && kn + STEP < klen) ? NM_LD_STREAM16(bp + kn + STEP, sp_b, a.status) : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
             for (int m = 0; m < M; ++m) {
@@ -614,12 +639,12 @@ __global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
         const int m = lane / CW, c = lane - m * CW, n = col0 + c;
         if (n < a.N) {
             if (a.nsplit == 1) {
-                ((TO *)a.C + (long)h * a.strideC)[(long)m * a.ldc + n] = round_out<TO>(mine);
+                NM_ST(&((TO *)a.C + (long)h * a.strideC)[(long)m * a.ldc + n], round_out<TO>(mine), sp_c, a.status);
             } else if (a.cluster_split) {
                 cluster_slot_store(slot0, m * a.tn + warp * CW + c, mine);
             } else {
                 float *P = a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * a.tn);
-                P[(size_t)m * a.tn + warp * CW + c] = mine;
+                NM_ST(&P[(size_t)m * a.tn + warp * CW + c], mine, sp_p, a.status);
             }
         }
     }
@@ -640,15 +665,15 @@ __global__ void __launch_bounds__(kThreads) nm_generic_kernel(const MatmulArgs a
     for (int m = 0; m < NM_MAX_M; ++m) acc[m] = 0.f;
     for (int k = 0; k < a.K; ++k) {
         const long ib = (layout == NM_ROW_MAJOR) ? (long)k * a.N + n : (long)n * a.K + k;
-        const float b = Elem<TI>::widen(B[ib]);
+        const float b = Elem<TI>::widen(NM_LD(&B[ib], span_of_B<TI>(a), a.status));
 #pragma unroll
         for (int m = 0; m < NM_MAX_M; ++m)
-            if (m < a.M) acc[m] = fmaf(Elem<TI>::widen(A[(long)m * a.lda + k]), b, acc[m]);
+            if (m < a.M) acc[m] = fmaf(Elem<TI>::widen(NM_LD(&A[(long)m * a.lda + k], span_of_A<TI>(a), a.status)), b, acc[m]);
     }
     TO *C = (TO *)a.C + (long)h * a.strideC;
 #pragma unroll
     for (int m = 0; m < NM_MAX_M; ++m)
-        if (m < a.M) C[(long)m * a.ldc + n] = round_out<TO>(acc[m]);
+        if (m < a.M) NM_ST(&C[(long)m * a.ldc + n], round_out<TO>(acc[m]), span_of_C<TO>(a), a.status);
 }
 
 // ---- launch helpers (explicitly instantiated per element type in their own translation units) ------------

@@ -158,7 +158,7 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
             if (n < a.N)
 #pragma unroll
                 for (int m = 0; m < kTok; ++m)
-                    if (m < M) C[(long)m * a.ldc + n] = round_out<TO>(n_it > 0 ? __uint_as_float(d[m]) : 0.f);
+                    if (m < M) NM_ST(&C[(long)m * a.ldc + n], round_out<TO>(n_it > 0 ? __uint_as_float(d[m]) : 0.f), span_of_C<TO>(a), ta.status);
         } else if (ta.cluster_split) {
 #pragma unroll
             for (int m = 0; m < kTok; ++m)
@@ -167,7 +167,7 @@ nm_row_tc_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constan
             float *P = a.partial + (((size_t)h * a.ntiles + tile) * a.nsplit + split) * (size_t)(M * kTcTN);
 #pragma unroll
             for (int m = 0; m < kTok; ++m)
-                if (m < M) P[(size_t)m * kTcTN + c] = n_it > 0 ? __uint_as_float(d[m]) : 0.f;
+                if (m < M) NM_ST(&P[(size_t)m * kTcTN + c], n_it > 0 ? __uint_as_float(d[m]) : 0.f, span_of_partials(a), ta.status);
         }
     }
     tc_fence_before();

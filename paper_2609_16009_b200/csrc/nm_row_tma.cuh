@@ -159,11 +159,11 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
                 if (grp < GROUPS && k < ke) {
                     const bf16_t *src = A + (long)m * a.lda + k;
                     if (k + 8 <= a.K) {
-                        v = __ldg(reinterpret_cast<const uint4 *>(src));
+                        v = NM_LDG16(reinterpret_cast<const uint4 *>(src), span_of_A<bf16_t>(a), ta.status);
                     } else {
                         uint16_t e[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) e[i] = (k + i < a.K) ? src[i].bits : (uint16_t)0;
+                        for (int i = 0; i < 8; ++i) e[i] = (k + i < a.K) ? NM_LD(&src[i], span_of_A<bf16_t>(a), ta.status).bits : (uint16_t)0;
                         v.x = e[0] | ((uint32_t)e[1] << 16); v.y = e[2] | ((uint32_t)e[3] << 16);
                         v.z = e[4] | ((uint32_t)e[5] << 16); v.w = e[6] | ((uint32_t)e[7] << 16);
                     }
@@ -327,9 +327,9 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
                 float s = 0.f;
 #pragma unroll 8
                 for (int g = 0; g < RG; ++g) s += red[(size_t)(g * MPASS + mm) * TN + c];
-                if (a.nsplit == 1) C[(long)m * a.ldc + n] = round_out<TO>(s);
+                if (a.nsplit == 1) NM_ST(&C[(long)m * a.ldc + n], round_out<TO>(s), span_of_C<TO>(a), ta.status);
                 else if (ta.cluster_split) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(slot0 + (uint32_t)(m * TN + c) * 4u), "f"(s) : "memory");
-                else               P[(size_t)m * TN + c] = s;
+                else               NM_ST(&P[(size_t)m * TN + c], s, span_of_partials(a), ta.status);
             }
         }
     }
@@ -353,7 +353,7 @@ nm_row_tma_kernel(const __grid_constant__ CUtensorMap tmap, const TmaArgs ta)
                     float s = 0.f;
                     for (int sp = 0; sp < a.nsplit; ++sp) s += slots[(size_t)sp * (M * TN) + i];
                     const TO r = round_out<TO>(s);
-                    C[(long)m * a.ldc + n] = r;
+                    NM_ST(&C[(long)m * a.ldc + n], r, span_of_C<TO>(a), ta.status);
                     if constexpr (M == 1 && sizeof(TO) == 2) { const float rv = Elem<bf16_t>::widen(r); sq = rv * rv; }
                 }
             }

@@ -42,6 +42,19 @@ EncodeTiledFn tensor_map_encoder()
     return fn;
 }
 
+#ifdef NM_BOUNDS_CHECK
+// The checked access macros on an address outside the span they are given (and inside the caller's buffer).
+__global__ void bounds_selftest_kernel(unsigned *buf, size_t bytes, unsigned *out_loaded, unsigned *status)
+{
+    const Span first_half = make_span(buf, bytes / 2);
+    unsigned *outside = buf + bytes / 8;                           // first word of the second half
+    NM_ST(outside, 0xdeadbeefu, first_half, status);              // must not happen
+    out_loaded[0] = NM_LD(outside, first_half, status);           // must yield 0
+    NM_ST(buf, 0x600df00du, first_half, status);                  // inside: happens
+    out_loaded[1] = NM_LD(buf, first_half, status);
+}
+#endif
+
 // One CTA that waits on an mbarrier nobody ever arrives at: the bounded wait runs out, raises the status word and
 // the kernel returns normally.
 __global__ void wait_probe_kernel(unsigned *status, unsigned long long *elapsed_ns)
@@ -80,9 +93,39 @@ int nm_check_status(nm_stream stream)
     if (v) {
         unsigned zero = 0;
         NM_CUDA_TRY(cudaMemcpy(p, &zero, sizeof zero, cudaMemcpyHostToDevice));
-        return NM_ERR_TIMEOUT;
+        return (v & nm::kStatusOutOfBounds) ? NM_ERR_BOUNDS : NM_ERR_TIMEOUT;
     }
     return NM_OK;
+}
+
+/* 1 when this library is the debug build whose narrow-product kernels check every hand-indexed global access against its
+ * operand's extent (NM_BOUNDS_CHECK), else 0. */
+int nm_debug_bounds_checked(void)
+{
+#ifdef NM_BOUNDS_CHECK
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+/* Debug build only: one thread stores to and loads from the first word of the SECOND half of `buf` through the checked
+ * access macros while naming the FIRST half as the operand.  The word lies inside the caller's allocation, so nothing can
+ * fault whether or not the check works; with the check the store is skipped (the word keeps its value), out_loaded[0]
+ * receives 0 instead of the word, and nm_check_status reports NM_ERR_BOUNDS once.  NM_ERR_UNSUPPORTED in the normal build. */
+int nm_debug_bounds_selftest(void *buf, size_t bytes, unsigned *out_loaded, nm_stream stream)
+{
+#ifdef NM_BOUNDS_CHECK
+    if (!buf || bytes < 32 || (bytes & 7) || ((uintptr_t)buf & 3) || !out_loaded) return NM_ERR_INVALID_ARG;
+    unsigned *p = nm::device_status_ptr();
+    if (!p) return NM_ERR_CUDA;
+    nm::bounds_selftest_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(static_cast<unsigned *>(buf), bytes, out_loaded, p);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? NM_OK : nm::record_cuda_error(e, "bounds self-test launch");
+#else
+    (void)buf; (void)bytes; (void)out_loaded; (void)stream;
+    return NM_ERR_UNSUPPORTED;
+#endif
 }
 
 int nm_debug_wait_probe(unsigned long long limit_ns, unsigned long long *elapsed_ns, nm_stream stream)

@@ -34,12 +34,24 @@ def test_every_declared_symbol_is_exported(lib):
     assert not missing, f"declared in include/ but not exported: {missing}"
 
 
+def test_the_debug_build_exports_the_same_symbols():
+    """libnm_check.so (-DNM_BOUNDS_CHECK) is the same library with checked accesses: same entry points, and it says so."""
+    from paper_2609_16009_b200 import build
+    check = ctypes.CDLL(build.build(check=True))
+    missing = [n for n in declared_functions() if not hasattr(check, n)]
+    assert not missing, missing
+    assert check.nm_debug_bounds_checked() == 1
+    check.nm_status_string.restype = ctypes.c_char_p
+    assert b"outside its operand" in check.nm_status_string(-8)
+
+
 def test_status_strings_and_version(lib):
     lib.nm_status_string.restype = ctypes.c_char_p
     assert lib.nm_version() >= 100
     assert lib.nm_status_string(0) == b"ok"
-    seen = {lib.nm_status_string(-i) for i in range(1, 7)}
-    assert len(seen) == 6 and b"unknown status" not in seen
+    seen = {lib.nm_status_string(-i) for i in range(1, 9)}
+    assert len(seen) == 8 and b"unknown status" not in seen
+    assert lib.nm_debug_bounds_checked() == 0
     assert lib.nm_status_string(-99) == b"unknown status"
 
 

@@ -434,6 +434,7 @@ static int matmul_impl(const void *A, const void *B, void *C, int M, int N, int 
     a.tn = p.tn; a.tpr = p.tpr; a.rg = p.rg; a.nsplit = p.nsplit; a.kr = p.kr; a.ntiles = p.ntiles;
     a.a_vec = a_ok ? 1 : 0;
     a.status = device_status_ptr();
+    a.use_pdl = (g_t.use_pdl || pdl) ? 1 : 0;
     if (p.nsplit > 1) {
         const size_t need = kCounterBytes + partial_floats(p, M, H) * sizeof(float);
         if (!ws || ws_bytes < need) return NM_ERR_WORKSPACE;

@@ -8,6 +8,7 @@
 // that no CTA ever waits on another.
 #pragma once
 
+#include "nm_async.cuh"
 #include "nm_common.cuh"
 
 namespace nm {
@@ -31,6 +32,7 @@ struct MatmulArgs {
     unsigned *counters;
     int cluster_split;   // plain kernels: the k-splits of a tile form a cluster (1 x nsplit x 1) and meet in shared memory
     unsigned *status;    // device status word (the debug build reports an access outside its operand there)
+    int use_pdl;         // plain kernels: launched programmatically - the first weight loads go out before the wait for earlier kernels
 };
 
 // Extents of the operands, for the debug build's checks (see NM_BOUNDS_CHECK in nm_common.cuh).
@@ -419,6 +421,7 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
     __shared__ __align__(16) float s_slots[kClusterSlotFloats];
     __shared__ int s_last;
     if (a.cluster_split) cluster_arrive_all();
+    pdl_launch_dependents();
 
     const int tid = threadIdx.x;
     const int tx = tid % a.tpr, ty = tid / a.tpr;
@@ -451,6 +454,7 @@ __global__ void __launch_bounds__(kThreads, RowCfg<M>::kMinBlocks) nm_row_kernel
             const int rr = r + u * rg;
             v[u] = (active && rr < klen) ? NM_LD_STREAM16(bp + (long)rr * ldb, sp_b, a.status) : make_uint4(0, 0, 0, 0);
         }
+        if (kc == kb) pdl_wait_prior_grids();             // weights depend on nothing; A and everything written do
         __syncthreads();                                  // readers of the previous chunk are done
         if (a.a_vec) {
             const int nv = klen / V;                      // klen is a multiple of kVec on this path
@@ -548,6 +552,7 @@ __global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
     __shared__ __align__(16) float s_slots[kClusterSlotFloats];
     __shared__ int s_last;
     if (a.cluster_split) cluster_arrive_all();
+    pdl_launch_dependents();
     uint4 *As = (uint4 *)smem;                                     // [M][KC / V] 16-byte vectors
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -579,6 +584,7 @@ __global__ void __launch_bounds__(kThreads, 2) nm_col_kernel(const MatmulArgs a)
             b0[c] = (okc && kk < klen) ? NM_LD_STREAM16(bp + kk, sp_b, a.status) : make_uint4(0, 0, 0, 0);
             b1[c] = (okc && kk + STEP < klen) ? NM_LD_STREAM16(bp + kk + STEP, sp_b, a.status) : make_uint4(0, 0, 0, 0);
         }
+        if (kc == kb) pdl_wait_prior_grids();                      // weights depend on nothing; A and everything written do
         __syncthreads();
         const int nv = klen / V;
         for (int m = 0; m < M; ++m) {
@@ -686,11 +692,19 @@ cudaError_t launch_row(const MatmulArgs &a, cudaStream_t s)
     cfg.gridDim = dim3(a.ntiles, a.nsplit, a.H);
     cfg.blockDim = dim3(kThreads);
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)a.nsplit; attr[0].val.clusterDim.z = 1;
+    // attribute 0: programmatic launch (when asked for); the cluster attribute, when used, comes last so that it can be dropped
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (a.use_pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    const int na_plain = na;
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 1; attr[na].val.clusterDim.y = (unsigned)a.nsplit; attr[na].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = a.cluster_split ? 1 : 0;
+    cfg.numAttrs = a.cluster_split ? na + 1 : na;
     switch (a.M) {
 #define NM_X(m)                                                                                          \
     case m: {                                                                                            \
@@ -698,7 +712,7 @@ cudaError_t launch_row(const MatmulArgs &a, cudaStream_t s)
         MatmulArgs b = a;                                                                                \
         if (b.cluster_split && b.partial && !clusters_fit_one_wave(kern, cfg, (unsigned)b.nsplit, (long)b.ntiles * b.H)) { \
             b.cluster_split = 0;       /* a second wave of clusters: through the workspace instead */      \
-            cfg.numAttrs = 0;                                                                            \
+            cfg.numAttrs = na_plain;                                                                     \
         }                                                                                                \
         return cudaLaunchKernelEx(&cfg, kern, b);                                                        \
     }
@@ -715,11 +729,19 @@ cudaError_t launch_col(const MatmulArgs &a, cudaStream_t s)
     cfg.gridDim = dim3(a.ntiles, a.nsplit, a.H);
     cfg.blockDim = dim3(kThreads);
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)a.nsplit; attr[0].val.clusterDim.z = 1;
+    // attribute 0: programmatic launch (when asked for); the cluster attribute, when used, comes last so that it can be dropped
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (a.use_pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    const int na_plain = na;
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 1; attr[na].val.clusterDim.y = (unsigned)a.nsplit; attr[na].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = a.cluster_split ? 1 : 0;
+    cfg.numAttrs = a.cluster_split ? na + 1 : na;
     switch (a.M) {
 #define NM_X(m)                                                                                          \
     case m: {                                                                                            \
@@ -727,7 +749,7 @@ cudaError_t launch_col(const MatmulArgs &a, cudaStream_t s)
         MatmulArgs b = a;                                                                                \
         if (b.cluster_split && b.partial && !clusters_fit_one_wave(kern, cfg, (unsigned)b.nsplit, (long)b.ntiles * b.H)) { \
             b.cluster_split = 0;       /* a second wave of clusters: through the workspace instead */      \
-            cfg.numAttrs = 0;                                                                            \
+            cfg.numAttrs = na_plain;                                                                     \
         }                                                                                                \
         return cudaLaunchKernelEx(&cfg, kern, b);                                                        \
     }

@@ -180,6 +180,8 @@ class MlaStep:
         self.dominant_traffic_source = "profiles/ncu_nm_row_tma_WO_M1_K16384_N7168.txt"
         self.dominant_traffic = ncu_dram_bytes(os.path.join(ROOT, self.dominant_traffic_source))
         self.launches_per_step = 6 if schedule == "fused" else 7
+        # two-stream schedules: the KV chain beside the first Q-chain product, or beside the attention pass
+        nm.nm_debug_set_step_kv_beside_attention(schedule == "kv-beside-attention")
         self.h2d = d * 2
         self.d2h = d * 2
 
@@ -191,7 +193,9 @@ class MlaStep:
                 "l2": "weights 374 MB per step > 126 MB L2, so every step streams from HBM; no flush",
                 "schedule": self.schedule,
                 "overlap": ("one stream: h*(W_DQ|W_DKV|W_KR) as one product; " if self.schedule == "fused" else
-                            "two streams: KV chain (W_DKV|KR product, RMSNorm, RoPE, cache write) beside the W_DQ product; ")
+                            ("two streams: KV chain (W_DKV|KR product, RMSNorm, RoPE, cache write) beside the W_DQ product; "
+                             if self.schedule == "two-stream" else
+                             "two streams: KV chain (W_DKV|KR product on CUDA cores, RMSNorm, RoPE, cache write) beside the tcgen05 attention pass; "))
                            + "RMSNorm / RoPE / cache write inside the completion of the products that feed them; L2 prefetch of "
                              "W_UV and 40 MB of W_O while the tcgen05 attention kernel runs; programmatic dependent launch along "
                              "the chain, also across steps"}
@@ -739,7 +743,7 @@ def main():
     ap.add_argument("--mkn", default="1,16384,7168", help="M,K,N of --workload matmul")
     ap.add_argument("--layout", default="row", choices=["row", "col"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"], help="operand type of --workload matmul")
-    ap.add_argument("--schedule", default="fused", choices=["fused", "two-stream"],
+    ap.add_argument("--schedule", default="fused", choices=["fused", "two-stream", "kv-beside-attention"],
                     help="decode step: down-projections as one concatenated product on one stream, or W_DKV|KR on a side stream")
     ap.add_argument("--timeline", action="store_true", help="print the kernel timeline of one step and exit")
     ap.add_argument("--sweep", action="store_true", help="the full product sweep: more cases, the paper's 100 x 100 schedule, warm-L2 figures, oracle times")

@@ -64,6 +64,12 @@ int nm_debug_set_attention(int impl);
 /* Wide-tile attention kernel: force the cache rows per tile (64, 128, 256), the most row runs (1..64) and the number of
  * runs merged on chip (cluster of 1, 2 or 4); zeros give each choice back to the planner. */
 int nm_debug_set_attention_wide(int tile_rows, int max_runs, int cluster);
+/* Two-stream schedule of nm_mla_decode_step (W_DQ and W_DKV|W_KR stored apart, side_stream != main_stream): 0 (default) the
+ * KV chain - the paper's MatMul 2 with RMSNorm, RoPE and the cache-row write - is forked at the start of the step and runs
+ * beside the first product of the Q chain; 1 it is forked once the attention operand is ready and runs, a narrow
+ * CUDA-core product, beside the tensor-core attention pass over the old cache rows (Data Independence condition: the new
+ * row is only needed by the merge). */
+int nm_debug_set_step_kv_beside_attention(int enable);
 /* The debug build.  `python paper_2609_16009_b200/build.py --check` compiles the same sources with -DNM_BOUNDS_CHECK into
  * libnm_check.so: every hand-indexed global access of the narrow-product kernels (the CUDA-core row / column / scalar
  * kernels, the split-K gather, the token loads and the C / partial stores of the TMA ring and tensor-core kernels) is

@@ -101,6 +101,7 @@ _lib.nm_mla_decode_step.argtypes = [C.POINTER(MlaParams), _vp, _vp]
 _lib.nm_mla_decode_step_host.argtypes = [C.POINTER(MlaParams), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.nm_debug_set_attention.argtypes = [_i]
 _lib.nm_debug_set_attention_wide.argtypes = [_i, _i, _i]
+_lib.nm_debug_set_step_kv_beside_attention.argtypes = [_i]
 _lib.nm_debug_bounds_selftest.argtypes = [_vp, _sz, _vp, _vp]
 _lib.nm_debug_set_step_pdl.argtypes = [_i]
 _lib.nm_debug_stream_read.argtypes = [_vp, _sz, _vp, _i, _vp]
@@ -390,6 +391,10 @@ def nm_debug_mma_probe(m, n, a_from_tmem, b_mn_major, reps, n_acc, a_step_bytes,
 
 def nm_debug_set_attention_wide(tile_rows: int = 0, max_runs: int = 0, cluster: int = 0) -> None:
     _check(_lib.nm_debug_set_attention_wide(int(tile_rows), int(max_runs), int(cluster)), "nm_debug_set_attention_wide")
+
+
+def nm_debug_set_step_kv_beside_attention(enable: bool = True) -> None:
+    _check(_lib.nm_debug_set_step_kv_beside_attention(1 if enable else 0), "nm_debug_set_step_kv_beside_attention")
 
 
 def nm_debug_set_attention(impl: int) -> None:

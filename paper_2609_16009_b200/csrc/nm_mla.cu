@@ -17,6 +17,7 @@ struct StepTuning {
     int attn_impl = 0;          // 0: tensor-core kernel when the shape allows, 1: CUDA-core kernel, 2 / 3: force 128 / 64 heads per CTA,
                                 // 4: force the wide-tile kernel
     int wide_tile = 0, wide_splits = 0, wide_cluster = 0;      // wide-tile kernel: forced rows per tile, row runs, cluster size (0 = planner)
+    int kv_beside_attention = 0; // two-stream schedule: the KV chain starts when the attention operand is ready, beside the tensor-core pass
     int step_plan[3][3] = {};   // forced (tile_n, nsplit, stages) of the down-projection, W_UQR and W_O products (0 = planner)
     int host_direct_out = 1;    // host-operand step: store the result straight into device-addressable host memory
     int batch_tc_min_t = 3;     // batch decode: tokens from which the per-head products go to the tensor cores
@@ -554,6 +555,26 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
     tkv.enabled = 1; tkv.kv_off = 0; tkv.dc = dc; tkv.rope = dr; tkv.eps = p->rms_eps; tkv.gamma_kv = (const uint16_t *)p->gamma_kv;
     tkv.cos_sin = p->rope_cos_sin; tkv.cache_row = cache + (size_t)pos * dkv;
     bool taken = false;
+    // The KV chain of the two-stream schedule: the paper's MatMul 2 (h * (W_DKV | W_KR)) with RMSNorm, RoPE and the cache-row
+    // write in its completion, on the side stream.  Forked at the start of the step it shares the machine with the first
+    // product of the Q chain; forked when the attention operand is ready (kv_beside_attention) it is a narrow CUDA-core
+    // product running on the SMs the attention pass leaves free while the tensor cores work - the paper's schedule
+    // (vector units beside the cube unit), and legal because the pass attends the OLD rows only: the new row joins in the merge.
+    const bool kv_late = forked && g_s.kv_beside_attention;
+    auto enqueue_kv_chain = [&]() -> int {
+        bool kv_taken = false;
+        if (forked) {
+            NM_CUDA_TRY(cudaEventRecord(g_events.fork, ms));
+            NM_CUDA_TRY(cudaStreamWaitEvent(ss, g_events.fork, 0));
+        }
+        NM_TRY(matmul_enqueue(p->h, p->W_DKVKR, ckr, 1, dkv, d, 1, d, 0, 0, dkv, 0, NM_BF16, lay, sws, L.side_ws_bytes, ss, false, nullptr,
+                              tails_ok ? &tkv : nullptr, &kv_taken, false));
+        if (!kv_taken)
+            NM_LAUNCH(kv_finish_kernel, 1, 256, ss, (const uint16_t *)ckr, (const uint16_t *)p->gamma_kv, p->rope_cos_sin,
+                      cache + (size_t)pos * dkv, dc, dr, p->rms_eps);
+        if (forked) NM_CUDA_TRY(cudaEventRecord(g_events.join, ss));
+        return NM_OK;
+    };
     const bool fused_down = p->W_DQKV && lay != NM_COL_MAJOR && down_finish_applies(ql, dc, dr);      // row-major or fractal storage
     // Where the plans allow: the k-splits of the fused down-projection meet inside clusters, each
     // tile leaves the sum of squares of its outputs, the W_UQR product applies RMSNorm to its token row while
@@ -614,16 +635,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         // ---- KV chain (the paper's MatMul 2 and its consumers) on the side stream, forked at the start so that
         //      it shares the machine with the first product of the Q chain and is long done when the merge
         //      needs the new cache row -------------------------------------------------------------------------
-        if (forked) {
-            NM_CUDA_TRY(cudaEventRecord(g_events.fork, ms));
-            NM_CUDA_TRY(cudaStreamWaitEvent(ss, g_events.fork, 0));
-        }
-        NM_TRY(matmul_enqueue(p->h, p->W_DKVKR, ckr, 1, dkv, d, 1, d, 0, 0, dkv, 0, NM_BF16, lay, sws, L.side_ws_bytes, ss, false, nullptr,
-                              tails_ok ? &tkv : nullptr, &taken, false));
-        if (!taken)
-            NM_LAUNCH(kv_finish_kernel, 1, 256, ss, (const uint16_t *)ckr, (const uint16_t *)p->gamma_kv, p->rope_cos_sin,
-                      cache + (size_t)pos * dkv, dc, dr, p->rms_eps);
-        if (forked) NM_CUDA_TRY(cudaEventRecord(g_events.join, ss));
+        if (!kv_late) NM_TRY(enqueue_kv_chain());
 
         // ---- Q chain, main stream ----------------------------------------------------------------------------
         NM_TRY(matmul_enqueue(p->h, p->W_DQ, c_q, 1, ql, d, 1, d, 0, 0, ql, 0, NM_BF16, lay, mws, L.main_ws_bytes, ms,
@@ -680,6 +692,7 @@ static int step_impl(const nm_mla_params *p, cudaStream_t ms, cudaStream_t ss)
         }
     }
 
+    if (kv_late) NM_TRY(enqueue_kv_chain());       // from here on the side stream runs beside the attention pass
     // ---- attention over the old rows (tensor cores), main stream; the new row joins in the merge -----------
     // When the merge kernel is launched programmatically it sits beside the attention CTAs from their start and
     // issues the prefetch itself (its threads are idle until the attention result exists); otherwise a warp of
@@ -1102,6 +1115,14 @@ int nm_debug_set_step_prefetch(int megabytes)
 int nm_debug_set_step_pdl(int enable)
 {
     return set_step_tuning([&](StepTuning &t) { t.step_pdl = enable ? 1 : 0; });
+}
+
+/* Two-stream schedule of the decode step (separate W_DQ and W_DKV|W_KR, a side stream): 0 (default) the KV chain is forked at
+ * the start of the step, beside the first product of the Q chain; 1 it is forked when the attention operand is ready and runs
+ * beside the tensor-core pass. */
+int nm_debug_set_step_kv_beside_attention(int enable)
+{
+    return set_step_tuning([&](StepTuning &t) { t.kv_beside_attention = enable ? 1 : 0; });
 }
 
 int nm_debug_set_attention_wide(int tile_rows, int max_runs, int cluster)

@@ -320,6 +320,25 @@ def test_decode_step_s1024(nm, weights, ref1024, overlap):
     check_step(t, r, cache_ref, 1024, w, h)
 
 
+@pytest.mark.parametrize("S", [1, 300, 1024, 7000])
+def test_decode_step_with_the_kv_chain_beside_the_attention_pass(nm, weights, S):
+    """Two-stream schedule, KV chain forked when the attention operand is ready: the narrow product h * (W_DKV | W_KR) with its
+    RMSNorm / RoPE / cache-row write runs on the side stream while the tensor-core pass attends the old rows; the merge
+    waits for it.  Same stages, same criteria; and the bits of the ordinary two-stream schedule."""
+    w, dw = weights
+    h, cache_ref, r = oracle_step(w, S, seed=4550 + S)
+    cache_in = gen.mla_cache(S, DIMS, seed=4550 + S)
+    early = run_step(nm, dw, h, cache_in, S, overlap=True)
+    nm.nm_debug_set_step_kv_beside_attention(True)
+    try:
+        late = run_step(nm, dw, h, cache_in, S, overlap=True)
+    finally:
+        nm.nm_debug_set_step_kv_beside_attention(False)
+    check_step(late, r, cache_ref, S, w, h, what=f"KV chain beside attention, S={S}")
+    for k in ("out", "o", "o_lat", "q_full", "kv_cache"):
+        assert torch.equal(early[k], late[k]), k
+
+
 @pytest.mark.parametrize("S", [1, 70, 1024])
 def test_decode_step_with_concatenated_down_projections(nm, weights, S):
     # h * (W_DQ | W_DKV | W_KR) as one product on one stream (Eq. 3's concatenation extended by W_DQ)

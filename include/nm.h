@@ -301,7 +301,8 @@ typedef struct nm_mla_batch {
 size_t nm_mla_batch_workspace_bytes(const nm_mla_params *p, int T);
 int nm_mla_decode_batch(const nm_mla_params *p, const nm_mla_batch *b, nm_stream main_stream);
 int nm_mla_decode_step(const nm_mla_params *p, nm_stream main_stream, nm_stream side_stream);
-/* The same step with the token and the result in HOST memory (pinned): copies h in on main_stream before the step;
+/* The same step with the token and the result in HOST memory (pinned): h comes in on main_stream before the step (fetched by
+ * a one-CTA kernel when the device can address h_host - the step's first product then starts under it -, else by a copy);
  * the result reaches out_host by stores of the last product when the device can address that memory (pinned or
  * registered, 16-byte aligned), otherwise by a copy after the step.  Either way it is complete when main_stream has
  * been synchronised.  h_staging / out_staging are device buffers of d bf16 each. */

@@ -344,6 +344,31 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const uin
     }
 }
 
+// The token row of the host-operand step: n 16-byte vectors from device-addressable host memory into the staging row.
+// One CTA: all loads go out at once (one trip over the host link), the kernels chained behind it start meanwhile.
+__device__ __forceinline__ uint4 ld_host16(const uint4 *p)        // the host may have rewritten the row since the last launch
+{
+    uint4 v;
+    asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__global__ void __launch_bounds__(256) token_fetch_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, int n)
+{
+    pdl_launch_dependents();
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int i = (int)threadIdx.x + u * 256;
+        v[u] = (i < n) ? ld_host16(src + i) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int i = (int)threadIdx.x + u * 256;
+        if (i < n) dst[i] = v[u];
+    }
+    for (int i = (int)threadIdx.x + 1024; i < n; i += 256) dst[i] = ld_host16(src + i);
+}
+
 // ---- host -------------------------------------------------------------------------------------------
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -1061,7 +1086,25 @@ int nm_mla_decode_step_host(const nm_mla_params *p, const void *h_host, void *ou
     if (out_direct) q.out = out_direct;
     NM_TRY(check_params(&q));
     cudaStream_t ms = (cudaStream_t)main_stream;
-    NM_CUDA_TRY(cudaMemcpyAsync(h_staging, h_host, (size_t)p->d * 2, cudaMemcpyHostToDevice, ms));
+    // The token: when the device can address the host buffer, ONE small CTA fetches the 14 KB over the host link into the staging
+    // row, and the step's first product is launched programmatically behind it - its CTAs become resident and fill their rings
+    // with weights while the token is on its way (a copy operation in front of the product would be a full dependency).
+    const void *h_direct = nullptr;
+    if (g_s.host_direct_out && g_s.step_pdl && (p->d % 8) == 0 && ((uintptr_t)h_staging & 15u) == 0) {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, h_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
+            ((uintptr_t)attr.devicePointer & 15u) == 0)
+            h_direct = attr.devicePointer;
+        else
+            (void)cudaGetLastError();
+    }
+    if (h_direct) {
+        token_fetch_kernel<<<1, 256, 0, ms>>>(static_cast<const uint4 *>(h_direct), static_cast<uint4 *>(h_staging), p->d / 8);
+        NM_LAUNCH_CHECK("token fetch");
+        q.programmatic_entry = 1;                                  // behind our own kernel, which writes nothing the prologue reads
+    } else {
+        NM_CUDA_TRY(cudaMemcpyAsync(h_staging, h_host, (size_t)p->d * 2, cudaMemcpyHostToDevice, ms));
+    }
     NM_TRY(step_impl(&q, ms, (cudaStream_t)side_stream));
     if (!out_direct) NM_CUDA_TRY(cudaMemcpyAsync(out_host, out_staging, (size_t)p->d * 2, cudaMemcpyDeviceToHost, ms));
     return NM_OK;

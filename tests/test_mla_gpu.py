@@ -614,6 +614,29 @@ def test_decode_step_host_operands(nm, weights, ref1024):
     ref = f64(r["out"])
     got = oracle.bf16_to_f64(out_host.numpy().view(np.uint16))
     assert np.all(np.abs(got - ref) <= 2e-3 * np.abs(ref).max() + oracle.ulp_bf16(ref))
+    # the same call again and again with another token written into the SAME pinned buffer in between (the token is fetched
+    # from host memory by a kernel: it must see the new bytes every time), also replayed from a CUDA graph; each result
+    # equals the device-operand step on that token, bit for bit
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=main):
+        nm.nm_mla_decode_step_host(p, h_host, out_host, t["h"], t["out"], main, side)
+    for k in range(4):
+        tok = gen.mla_token(DIMS, seed=4700 + k)
+        h_host.copy_(torch.from_numpy(tok.view(np.int16).copy()))
+        out_host.zero_()
+        if k % 2 == 0:
+            nm.nm_mla_decode_step_host(p, h_host, out_host, t["h"], t["out"], main, side)
+        else:
+            g.replay()
+        torch.cuda.synchronize()
+        t2 = dict(t)
+        t2["h"] = to_dev(tok)
+        t2["out"] = torch.zeros(d, dtype=torch.int16, device="cuda")
+        p2 = nm.mla_params(DIMS, 1024, t2, workspace=ws)
+        nm.nm_mla_decode_step(p2, main, side)
+        torch.cuda.synchronize()
+        assert torch.equal(out_host, t2["out"].cpu()), f"token {k}"
+    nm.nm_check_status()
 
 
 def test_step_error_codes(nm, weights):

@@ -687,7 +687,9 @@ def run_reference(args, rank):
     if rank != 0:
         return
     import oracle
-    threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+    # every core this process may run on: under torchrun the other ranks do no work, and its OMP_NUM_THREADS=1 default would
+    # otherwise put the whole oracle on one core (14 s per step instead of 0.6)
+    threads = len(os.sched_getaffinity(0))
     steps = min(args.steps, 20)              # bounded: the oracle is slow by design
     for _ in range(min(args.warmup, 2)):
         oracle_sample(threads, args.workload, args.seq_len)

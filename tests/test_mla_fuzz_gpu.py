@@ -26,6 +26,7 @@ def nm():
     nm.nm_debug_set_step_tails(1)
     nm.nm_debug_set_step_fusion(True)
     nm.nm_debug_set_step_pdl(True)
+    nm.nm_debug_set_step_kv_beside_attention(False)
     nm.nm_check_status()
 
 
@@ -61,15 +62,19 @@ def test_random_step_matches_the_oracle(nm, weights, seed):
     overlap = bool(rng.random() < 0.5)
     tails, fusion, pdl = int(rng.integers(0, 3)), bool(rng.random() < 0.8), bool(rng.random() < 0.8)
     attn = int(rng.choice([0, 0, 1, 2, 3, 4]))
-    what = f"seed {seed}: S {S} layout {layout} concat {concat} overlap {overlap} tails {tails} fusion {fusion} pdl {pdl} attention {attn}"
+    kv_late = bool(np.random.default_rng(70_000 + seed).random() < 0.5)       # own generator: the other draws keep their values
+    what = (f"seed {seed}: S {S} layout {layout} concat {concat} overlap {overlap} tails {tails} fusion {fusion} pdl {pdl} attention {attn} "
+            f"kv beside attention {kv_late}")
     h, cache_ref, r = base.oracle_step(weights, S, seed=60_000 + seed)
     cache_in = gen.mla_cache(S, DIMS, seed=60_000 + seed)
     dw = stored(weights, layout, concat)
     nm.nm_debug_set_step_tails(tails); nm.nm_debug_set_step_fusion(fusion); nm.nm_debug_set_step_pdl(pdl); nm.nm_debug_set_attention(attn)
+    nm.nm_debug_set_step_kv_beside_attention(kv_late)             # acts on the two-stream schedule only
     try:
         t = base.run_step(nm, dw, h, cache_in, S, overlap=overlap, layout_dense=layout)
     finally:
         nm.nm_debug_set_step_tails(1); nm.nm_debug_set_step_fusion(True); nm.nm_debug_set_step_pdl(True); nm.nm_debug_set_attention(0)
+        nm.nm_debug_set_step_kv_beside_attention(False)
     try:
         base.check_step(t, r, cache_ref, S, weights, h, what=what)
     except AssertionError as e:
